@@ -1,0 +1,224 @@
+/*
+ * catekv.h - C ABI of the CateKV hot path on one NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel part of CateKV (hybrid-head KV-cache
+ * attention for long-context decoding):
+ *
+ *   catekv_head_cv         Section 3.2, Eq. 1-4: per-head coefficient-of-variation score
+ *   catekv_classify_heads  Section 3.2, Eq. 5 + "Reference-Based Static Identification"
+ *   catekv_select_compact  Algorithm 1, pre-filling stage: window scores, pooling,
+ *                          per-KV-head top-k, Cache()
+ *   catekv_append          growth of every head's list by the decoded token
+ *                          (the paper is silent; implied by autoregressive decoding)
+ *   catekv_decode_attn     Algorithm 1, decoding stage: Attention(q, k, v) over the
+ *                          per-head lists ("all" retrieval on adaptive heads)
+ *
+ * Conventions
+ *   - Every function returns 0 (CATEKV_OK) or a negative error code.  Arguments
+ *     are checked on the host before anything is launched; a failed check
+ *     launches nothing and changes no buffer.
+ *   - "device" pointers are CUDA device memory owned by the caller; "host"
+ *     pointers are ordinary host memory owned by the caller.  The library
+ *     allocates no device memory and keeps no state between calls except the
+ *     last CUDA error code (thread-local).
+ *   - Kernels are enqueued on the caller's stream (a cudaStream_t passed as
+ *     void*); calls do not synchronise unless stated.
+ *   - bf16 values are raw 16-bit patterns.  The head dimension d is the
+ *     contiguous inner dimension and must be 128.  Hq / Hkv = G <= 8.
+ *   - A "segment" is the cached list of one (sequence b, KV head h), index
+ *     b * Hkv + h.  All segments of a layer live in two pools, k_pool and
+ *     v_pool, each [total_rows, d] bf16; segment s owns rows
+ *     [seg_off[s], seg_off[s] + seg_cap[s]) of which the first seg_len[s] are
+ *     valid, in ascending token order.
+ */
+#ifndef CATEKV_H_
+#define CATEKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CATEKV_OK 0
+#define CATEKV_ERR_INVALID_ARG (-1) /* null pointer, negative size, inconsistent shapes */
+#define CATEKV_ERR_UNSUPPORTED (-2) /* d != 128, G > 8, unknown mode */
+#define CATEKV_ERR_CAPACITY (-3)    /* a segment would outgrow its capacity */
+#define CATEKV_ERR_WORKSPACE (-4)   /* workspace or plan buffer too small */
+#define CATEKV_ERR_CUDA (-5)        /* a CUDA call failed: see catekv_last_cuda_error() */
+
+#define CATEKV_POOL_NONE 0    /* top-k on the raw criticality C */
+#define CATEKV_POOL_CHUNK 1   /* BlockMax(C, cs) of Algorithm 1; whole chunks are selected */
+#define CATEKV_POOL_SLIDING 2 /* stride-1 max pool of odd width w, -inf padding */
+
+#define CATEKV_OUT_BF16 0
+#define CATEKV_OUT_FP32 1
+
+#define CATEKV_HEAD_DIM 128
+#define CATEKV_MAX_GROUP 8
+#define CATEKV_SEG_ALIGN 128 /* rows; segment offsets and capacities are multiples of it */
+
+typedef void* catekv_stream; /* cudaStream_t */
+
+/* Hybrid per-head KV cache of one layer (Section 1; Section 3.2 last paragraph). */
+typedef struct catekv_cache {
+  int32_t B;              /* sequences */
+  int32_t Hkv;            /* KV heads */
+  int32_t d;              /* head dim, 128 */
+  int32_t reserved;
+  int64_t total_rows;     /* rows of each pool */
+  void* k_pool;           /* device, bf16 [total_rows, d] */
+  void* v_pool;           /* device, bf16 [total_rows, d] */
+  const int32_t* seg_off_dev; /* device [B*Hkv], first row of each segment */
+  int32_t* seg_len_dev;       /* device [B*Hkv], valid rows; written by select_compact and append */
+  const int32_t* seg_off;     /* host   [B*Hkv] */
+  const int32_t* seg_cap;     /* host   [B*Hkv] */
+  int32_t* seg_len;           /* host   [B*Hkv], mirror of seg_len_dev kept by the library's calls */
+} catekv_cache;
+
+/* Version of this ABI (major * 1000 + minor). */
+int catekv_version(void);
+/* Static text for an error code. */
+const char* catekv_error_string(int code);
+/* cudaError_t value of the last CUDA failure seen by this thread (0 if none). */
+int catekv_last_cuda_error(void);
+
+/*
+ * Canonical pool layout.  Host only.
+ * len0 [B*Hkv]: rows each segment starts with; max_new: rows it may still grow by.
+ * Writes seg_cap[s] = round_up(len0[s] + max_new, 128), seg_off = exclusive prefix
+ * sum of seg_cap, *total_rows = sum of seg_cap.  All arrays are host arrays.
+ */
+int catekv_cache_layout(int32_t B, int32_t Hkv, const int32_t* len0, int32_t max_new,
+                        int32_t* seg_off, int32_t* seg_cap, int64_t* total_rows);
+
+/* ---------------------------------------------------------------- head identification */
+
+/*
+ * CV score of every (sequence, KV head): Section 3.2, Eq. 1-4.
+ *
+ * For each group: A = mean over the group's G query heads of
+ * softmax(Q[-L_obs:] K[L_init : n - L_rec]^T / sqrt(d)) (Eq. 1, row softmax over
+ * the sliced keys; with `causal` != 0 window row i, at position n - L_obs + i,
+ * does not see later keys and those entries of A are 0);
+ * Phi = alpha * (the floor(k (N-1))-th ascending element of the whole matrix A),
+ * N = L_obs * m, m = n - L_init - L_rec (Eq. 2); C_j = #{i : A_ij >= Phi}
+ * (Eq. 3); cv = population std(C) / mean(C), 0 when the mean is 0 (Eq. 4).
+ *
+ *   q_win   device bf16 [B, Hq, L_obs, d], contiguous
+ *   k       device bf16, element strides (k_stride_b, k_stride_h, k_stride_t), d contiguous
+ *   seq_len host [B], n of each sequence (n - L_init - L_rec >= 1, n >= L_obs)
+ *   cv_out  device float [B*Hkv]
+ *   ws      device scratch of at least catekv_head_cv_workspace_bytes(...)
+ */
+size_t catekv_head_cv_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t n_max, int32_t L_obs,
+                                      int32_t L_init, int32_t L_rec);
+int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride_b, int64_t k_stride_h,
+                   int64_t k_stride_t, const int32_t* seq_len, int32_t B, int32_t Hq, int32_t Hkv,
+                   int32_t d, int32_t L_obs, int32_t L_init, int32_t L_rec, float quantile_k, float alpha,
+                   int32_t causal, float* cv_out, void* ws, size_t ws_bytes, catekv_stream stream);
+
+/*
+ * Eq. 5 per sample and the static vote over a reference set.  Host only.
+ * cv [n_samples, n_heads] host (n_heads = all KV heads of the model, flattened);
+ * r = share of adaptive heads.  Per sample, Gamma = the floor(r (H-1))-th ascending
+ * score and a head is consistent iff its score > Gamma.  mask_out[h] = 1 for the
+ * H - (floor(r (H-1)) + 1) heads ranked first by (times classified consistent
+ * descending, mean score descending, index ascending), else 0.
+ */
+int catekv_classify_heads(const float* cv, int32_t n_samples, int32_t n_heads, float r, uint8_t* mask_out);
+
+/* ---------------------------------------------------------------- prefill-end selection */
+
+typedef struct catekv_select_params {
+  int32_t B, Hq, Hkv, d;
+  int32_t L_obs;             /* observation window: the last L_obs queries */
+  int32_t sink;              /* S: first tokens always kept */
+  int32_t local;             /* Lc: last tokens always kept; must be >= L_obs */
+  int32_t budget_consistent; /* token budget T of a consistent head (sink and local included) */
+  float eta_adaptive;        /* adaptive head keeps T = floor(eta * n) tokens; >= 1 keeps all */
+  int32_t pool_mode;         /* CATEKV_POOL_* */
+  int32_t pool_param;        /* chunk size cs, or odd window w */
+  int32_t reserved;
+  const void* q_win;         /* device bf16 [B, Hq, L_obs, d], contiguous */
+  const void* k;             /* device bf16 prefill keys   */
+  const void* v;             /* device bf16 prefill values */
+  int64_t kv_stride_b, kv_stride_h, kv_stride_t; /* element strides of k and v; d contiguous */
+  const int32_t* seq_len;    /* host [B]: n of each sequence */
+  const uint8_t* head_mask;  /* host [B*Hkv]: 1 = consistent, 0 = adaptive */
+} catekv_select_params;
+
+/*
+ * Algorithm 1, pre-filling stage, for every (sequence, KV head):
+ *   C_j = mean over the group's heads of sum_i softmax(Q_win K[:n-L_obs]^T / sqrt(d))_ij;
+ *   pooled scores over the candidates [S, n - Lc);
+ *   the k_rest = max(0, T - S - Lc) best candidates (ties: lowest index; CHUNK mode:
+ *   floor(k_rest / cs) whole chunks, chunk origin at S, last chunk may be short);
+ *   kept = [0, S) + selected + [n - Lc, n), ascending; K and V rows gathered in that
+ *   order into the segment; seg_len set (device and host).  T >= n or S + Lc >= n
+ *   keeps every token.
+ *
+ *   idx_out  device int32 [B*Hkv, idx_stride] or NULL: the kept indices of each segment
+ *   The host mirror cache->seg_len is exact on return.  It is computed on the host,
+ *   except in CHUNK mode when (n - Lc - S) is not a multiple of cs: then the length
+ *   depends on the data and the call synchronises the stream to read it back.
+ *   Errors: CATEKV_ERR_CAPACITY if a kept list can exceed its segment capacity.
+ */
+size_t catekv_select_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t n_max, int32_t L_obs);
+int catekv_select_compact(const catekv_select_params* p, catekv_cache* cache, int32_t* idx_out,
+                          int64_t idx_stride, void* ws, size_t ws_bytes, catekv_stream stream);
+
+/* ---------------------------------------------------------------- decoding */
+
+/*
+ * Append the decoded token's key and value to every segment.
+ * k_new, v_new: device bf16 [B, Hkv, d] contiguous.  Row seg_off + seg_len of each
+ * segment is written and seg_len grows by one on the device and in the host
+ * mirror.  CATEKV_ERR_CAPACITY (nothing launched) if any segment is full.
+ */
+int catekv_append(catekv_cache* cache, const void* k_new, const void* v_new, catekv_stream stream);
+
+/*
+ * Work-balanced split-KV schedule for catekv_decode_attn.
+ *
+ * The rows of all segments, laid end to end, are cut into num_ctas near-equal
+ * ranges; a range that crosses segment boundaries yields one work item per
+ * segment it touches, so short (consistent) and long (adaptive) segments load
+ * every CTA evenly.  The plan is built on the host from cache->seg_len, stored
+ * in plan_host and copied to plan_dev (cudaMemcpyAsync on `stream`; plan_host
+ * must stay untouched until that copy has run - use pinned memory to make it
+ * asynchronous).  A plan stays valid while segments only grow (append): the
+ * last item of a segment reads the current length on the device; rebuild it
+ * now and then to restore balance.
+ *
+ * catekv_decode_num_ctas: SM count * resident CTAs per SM of the decode kernel
+ * on the current device (a CUDA query); < 0 on error.
+ */
+int catekv_decode_num_ctas(void);
+size_t catekv_decode_plan_bytes(int32_t B, int32_t Hkv, int32_t num_ctas);
+size_t catekv_decode_workspace_bytes(int32_t B, int32_t Hkv, int32_t num_ctas);
+int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, void* plan_host, void* plan_dev,
+                       size_t plan_bytes, catekv_stream stream);
+
+/*
+ * Attention(q, k, v) of Algorithm 1 for one decode step: for every query head hq
+ * of every sequence, softmax(sm_scale * q . K^T) V over the current list of KV
+ * head hq / G.  bf16 inputs, fp32 accumulation; the logit scale is applied in
+ * fp32 after the dot product.
+ *
+ *   q        device bf16 [B, Hq, d] contiguous
+ *   sm_scale 0 means 1/sqrt(d)
+ *   out      device [B, Hq, d], bf16 or float per out_dtype; an empty list gives 0
+ *   lse_out  device float [B, Hq] or NULL: natural-log sum of exp(logits); -inf if empty
+ *   plan_host / plan_dev  the plan built by catekv_decode_plan for this cache
+ *   ws       device scratch of at least catekv_decode_workspace_bytes(...)
+ */
+int catekv_decode_attn(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
+                       int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
+                       size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CATEKV_H_ */

@@ -1,0 +1,246 @@
+"""ctypes binding of libcatekv.so: argument marshalling only.
+
+Every step of the hot path runs in the library's CUDA kernels; PyTorch is used
+here for device memory and the current stream.  The entry points carry the
+names of the C ABI (include/catekv.h).  There is no CPU fallback: importing
+this module without the built library raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcatekv.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA = 0, -1, -2, -3, -4, -5
+POOL_NONE, POOL_CHUNK, POOL_SLIDING = 0, 1, 2
+OUT_BF16, OUT_FP32 = 0, 1
+SEG_ALIGN = 128
+
+
+class CatekvError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = _lib.catekv_error_string(code).decode()
+        if code == ERR_CUDA:
+            msg += f" (cudaError {_lib.catekv_last_cuda_error()})"
+        super().__init__(f"{where}: {msg} [{code}]")
+
+
+class CacheStruct(C.Structure):
+    _fields_ = [("B", C.c_int32), ("Hkv", C.c_int32), ("d", C.c_int32), ("reserved", C.c_int32),
+                ("total_rows", C.c_int64), ("k_pool", C.c_void_p), ("v_pool", C.c_void_p),
+                ("seg_off_dev", C.c_void_p), ("seg_len_dev", C.c_void_p),
+                ("seg_off", C.c_void_p), ("seg_cap", C.c_void_p), ("seg_len", C.c_void_p)]
+
+
+class SelectParams(C.Structure):
+    _fields_ = [("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("d", C.c_int32),
+                ("L_obs", C.c_int32), ("sink", C.c_int32), ("local", C.c_int32), ("budget_consistent", C.c_int32),
+                ("eta_adaptive", C.c_float), ("pool_mode", C.c_int32), ("pool_param", C.c_int32),
+                ("reserved", C.c_int32),
+                ("q_win", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p),
+                ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64), ("kv_stride_t", C.c_int64),
+                ("seq_len", C.c_void_p), ("head_mask", C.c_void_p)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2608_30295_b200.build` "
+                          "(there is no fallback path)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
+    sig = {
+        "catekv_version": (C.c_int, []),
+        "catekv_error_string": (C.c_char_p, [C.c_int]),
+        "catekv_last_cuda_error": (C.c_int, []),
+        "catekv_cache_layout": (C.c_int, [i32, i32, vp, i32, vp, vp, C.POINTER(i64)]),
+        "catekv_head_cv_workspace_bytes": (sz, [i32, i32, i32, i32, i32, i32, i32]),
+        "catekv_head_cv": (C.c_int, [vp, vp, i64, i64, i64, vp, i32, i32, i32, i32, i32, i32, i32, f32, f32, i32,
+                                     vp, vp, sz, vp]),
+        "catekv_classify_heads": (C.c_int, [vp, i32, i32, f32, vp]),
+        "catekv_select_workspace_bytes": (sz, [i32, i32, i32, i32, i32]),
+        "catekv_select_compact": (C.c_int, [C.POINTER(SelectParams), C.POINTER(CacheStruct), vp, i64, vp, sz, vp]),
+        "catekv_append": (C.c_int, [C.POINTER(CacheStruct), vp, vp, vp]),
+        "catekv_decode_num_ctas": (C.c_int, []),
+        "catekv_decode_plan_bytes": (sz, [i32, i32, i32]),
+        "catekv_decode_workspace_bytes": (sz, [i32, i32, i32]),
+        "catekv_decode_plan": (C.c_int, [C.POINTER(CacheStruct), i32, vp, vp, sz, vp]),
+        "catekv_decode_attn": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    return lib, tuple(sig)
+
+
+_lib, EXPORTS = _load()
+
+
+def _check(rc: int, where: str):
+    if rc != OK:
+        raise CatekvError(rc, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _np_ptr(a: np.ndarray) -> int:
+    return a.ctypes.data
+
+
+def _dev_ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def catekv_version() -> int:
+    return _lib.catekv_version()
+
+
+def catekv_cache_layout(B: int, Hkv: int, len0, max_new: int):
+    """-> (seg_off int32[B*Hkv], seg_cap int32[B*Hkv], total_rows)."""
+    len0 = np.ascontiguousarray(len0, dtype=np.int32).reshape(-1)
+    off = np.zeros(B * Hkv, dtype=np.int32)
+    cap = np.zeros(B * Hkv, dtype=np.int32)
+    total = C.c_int64(0)
+    _check(_lib.catekv_cache_layout(B, Hkv, _np_ptr(len0), max_new, _np_ptr(off), _np_ptr(cap), C.byref(total)),
+           "catekv_cache_layout")
+    return off, cap, int(total.value)
+
+
+class Cache:
+    """Device pools and segment tables of one layer's hybrid cache (memory only)."""
+
+    def __init__(self, B: int, Hkv: int, len0, max_new: int, device="cuda", d: int = 128):
+        self.B, self.Hkv, self.d = B, Hkv, d
+        self.seg_off, self.seg_cap, self.total_rows = catekv_cache_layout(B, Hkv, len0, max_new)
+        self.seg_len = np.zeros(B * Hkv, dtype=np.int32)
+        self.device = torch.device(device)
+        rows = max(self.total_rows, 1)
+        self.k_pool = torch.empty((rows, d), dtype=torch.bfloat16, device=device)
+        self.v_pool = torch.empty((rows, d), dtype=torch.bfloat16, device=device)
+        self.seg_off_dev = torch.from_numpy(self.seg_off).to(device)
+        self.seg_len_dev = torch.zeros(B * Hkv, dtype=torch.int32, device=device)
+        self.struct = CacheStruct(B, Hkv, d, 0, self.total_rows, self.k_pool.data_ptr(), self.v_pool.data_ptr(),
+                                  self.seg_off_dev.data_ptr(), self.seg_len_dev.data_ptr(),
+                                  _np_ptr(self.seg_off), _np_ptr(self.seg_cap), _np_ptr(self.seg_len))
+
+    def set_lengths(self, lens):
+        """Set host mirror and device lengths (used when rows are written by the caller)."""
+        self.seg_len[:] = np.asarray(lens, dtype=np.int32).reshape(-1)
+        self.seg_len_dev.copy_(torch.from_numpy(self.seg_len))
+
+    def kept_rows(self) -> int:
+        return int(self.seg_len.sum())
+
+
+def catekv_append(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor):
+    assert k_new.is_contiguous() and v_new.is_contiguous()
+    _check(_lib.catekv_append(C.byref(cache.struct), k_new.data_ptr(), v_new.data_ptr(), _stream()), "catekv_append")
+
+
+def catekv_decode_num_ctas() -> int:
+    n = _lib.catekv_decode_num_ctas()
+    if n < 0:
+        raise CatekvError(n, "catekv_decode_num_ctas")
+    return n
+
+
+class DecodePlan:
+    """Plan and workspace buffers of catekv_decode_attn for one cache (memory only)."""
+
+    def __init__(self, cache: Cache, num_ctas: int):
+        self.num_ctas = num_ctas
+        self.bytes = _lib.catekv_decode_plan_bytes(cache.B, cache.Hkv, num_ctas)
+        self.host = torch.empty(self.bytes, dtype=torch.uint8).pin_memory()
+        self.dev = torch.empty(self.bytes, dtype=torch.uint8, device=cache.device)
+        self.ws_bytes = _lib.catekv_decode_workspace_bytes(cache.B, cache.Hkv, num_ctas)
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=cache.device)
+
+
+def catekv_decode_plan(cache: Cache, plan: DecodePlan):
+    _check(_lib.catekv_decode_plan(C.byref(cache.struct), plan.num_ctas, plan.host.data_ptr(), plan.dev.data_ptr(),
+                                   plan.bytes, _stream()), "catekv_decode_plan")
+
+
+def plan_header(plan: DecodePlan) -> dict:
+    h = plan.host[:32].numpy().view(np.int32)
+    return {"num_ctas": int(h[1]), "n_segs": int(h[2]), "n_items": int(h[3]), "n_slots": int(h[4]),
+            "tile": int(h[5]), "total_rows": int(plan.host[24:32].numpy().view(np.int64)[0])}
+
+
+def catekv_decode_attn(cache: Cache, q: torch.Tensor, plan: DecodePlan, out: torch.Tensor,
+                       lse_out: Optional[torch.Tensor] = None, sm_scale: float = 0.0):
+    assert q.is_contiguous() and out.is_contiguous() and q.dtype == torch.bfloat16
+    Hq = q.shape[1]
+    if out.dtype == torch.bfloat16:
+        od = OUT_BF16
+    elif out.dtype == torch.float32:
+        od = OUT_FP32
+    else:
+        raise TypeError("out must be bf16 or fp32")
+    _check(_lib.catekv_decode_attn(C.byref(cache.struct), q.data_ptr(), Hq, sm_scale, out.data_ptr(), od,
+                                   _dev_ptr(lse_out), plan.host.data_ptr(), plan.dev.data_ptr(), plan.bytes,
+                                   plan.ws.data_ptr(), plan.ws_bytes, _stream()), "catekv_decode_attn")
+
+
+def catekv_select_workspace_bytes(B, Hq, Hkv, n_max, L_obs) -> int:
+    return _lib.catekv_select_workspace_bytes(B, Hq, Hkv, n_max, L_obs)
+
+
+def catekv_select_compact(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_len, head_mask, cache: Cache,
+                          budget_consistent: int, eta_adaptive: float, sink: int, local: int, pool_mode: int,
+                          pool_param: int, ws: Optional[torch.Tensor] = None,
+                          idx_out: Optional[torch.Tensor] = None):
+    """q_win [B,Hq,L_obs,d] bf16 contiguous; k, v [B,Hkv,n_max,d] bf16 (any strides, d contiguous)."""
+    B, Hq, L_obs, d = q_win.shape
+    Hkv, n_max = k.shape[1], k.shape[2]
+    assert q_win.is_contiguous() and k.stride(3) == 1 and v.stride() == k.stride()
+    seq_len = np.ascontiguousarray(seq_len, dtype=np.int32).reshape(-1)
+    head_mask = np.ascontiguousarray(head_mask, dtype=np.uint8).reshape(-1)
+    if ws is None:
+        ws = torch.empty(catekv_select_workspace_bytes(B, Hq, Hkv, n_max, L_obs), dtype=torch.uint8, device=k.device)
+    p = SelectParams(B, Hq, Hkv, d, L_obs, sink, local, budget_consistent, eta_adaptive, pool_mode, pool_param, 0,
+                     q_win.data_ptr(), k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1), k.stride(2),
+                     _np_ptr(seq_len), _np_ptr(head_mask))
+    stride = 0 if idx_out is None else idx_out.stride(0)
+    _check(_lib.catekv_select_compact(C.byref(p), C.byref(cache.struct), _dev_ptr(idx_out), stride, ws.data_ptr(),
+                                      ws.numel(), _stream()), "catekv_select_compact")
+    return ws
+
+
+def catekv_head_cv_workspace_bytes(B, Hq, Hkv, n_max, L_obs, L_init, L_rec) -> int:
+    return _lib.catekv_head_cv_workspace_bytes(B, Hq, Hkv, n_max, L_obs, L_init, L_rec)
+
+
+def catekv_head_cv(q_win: torch.Tensor, k: torch.Tensor, seq_len, L_init: int, L_rec: int, quantile_k: float,
+                   alpha: float, causal: bool, ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """-> cv float32 [B, Hkv] on the device."""
+    B, Hq, L_obs, d = q_win.shape
+    Hkv, n_max = k.shape[1], k.shape[2]
+    assert q_win.is_contiguous() and k.stride(3) == 1
+    seq_len = np.ascontiguousarray(seq_len, dtype=np.int32).reshape(-1)
+    if ws is None:
+        ws = torch.empty(catekv_head_cv_workspace_bytes(B, Hq, Hkv, n_max, L_obs, L_init, L_rec), dtype=torch.uint8,
+                         device=k.device)
+    cv = torch.empty((B, Hkv), dtype=torch.float32, device=k.device)
+    _check(_lib.catekv_head_cv(q_win.data_ptr(), k.data_ptr(), k.stride(0), k.stride(1), k.stride(2),
+                               _np_ptr(seq_len), B, Hq, Hkv, d, L_obs, L_init, L_rec, quantile_k, alpha,
+                               1 if causal else 0, cv.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "catekv_head_cv")
+    return cv
+
+
+def catekv_classify_heads(cv, r: float) -> np.ndarray:
+    cv = np.ascontiguousarray(cv, dtype=np.float32)
+    n_samples, n_heads = cv.shape
+    mask = np.zeros(n_heads, dtype=np.uint8)
+    _check(_lib.catekv_classify_heads(_np_ptr(cv), n_samples, n_heads, r, _np_ptr(mask)), "catekv_classify_heads")
+    return mask

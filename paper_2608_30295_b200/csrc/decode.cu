@@ -1,0 +1,594 @@
+// Decoding stage of Algorithm 1: append, work-balanced split-KV schedule, attention partials
+// and the combine pass, for per-(sequence, KV head) variable-length caches.
+//
+// The attention kernel is a memory-bound stream over the K and V rows of the cache.  Each CTA
+// owns a contiguous range of the rows of all segments laid end to end (so short consistent
+// heads and long adaptive heads load the SMs evenly), stages 64-row K/V tiles through a
+// multi-stage cp.async pipeline into XOR-swizzled shared memory, and uses the tensor cores
+// only to keep the ALU work off the critical path: the G <= 8 query heads of the group are
+// packed into the N = 8 dimension of mma.m16n8k16 (tokens are M), softmax runs online per
+// warp in fp32, and P enters the P.V product as a bf16 hi + lo pair so that no precision of
+// the fp32 probabilities is lost.
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace catekv {
+
+// ------------------------------------------------------------------------------------------
+// Plan (host)
+// ------------------------------------------------------------------------------------------
+constexpr uint32_t kPlanMagic = 0x43544B56u;  // "CTKV"
+constexpr int kTile = 64;                     // rows per pipeline stage
+constexpr int kDecodeWarps = kTile / 16;
+constexpr int kDecodeThreads = kDecodeWarps * 32;
+constexpr int kStages = 3;
+constexpr int kSplitAlign = 16;               // CTA ranges are cut at multiples of this many rows
+
+struct PlanHeader {
+  uint32_t magic;
+  int32_t num_ctas;
+  int32_t n_segs;
+  int32_t n_items;
+  int32_t n_slots;
+  int32_t tile;
+  int64_t total_rows;
+};
+static_assert(sizeof(PlanHeader) == 32, "plan header layout");
+
+struct WorkItem {
+  int32_t seg;
+  int32_t t0;    // first row of the piece, relative to the segment
+  int32_t t1;    // one past the last row; -1 = up to the segment's current length (last piece)
+  int32_t slot;  // partial slot, or -1 when the piece is the whole segment (final output written directly)
+};
+struct SegInfo {
+  int32_t slot_begin;
+  int32_t n_pieces;
+};
+
+struct PlanLayout {
+  size_t off_cta, off_items, off_seg, bytes;
+  int n_items_cap;
+};
+static PlanLayout plan_layout(int n_segs, int num_ctas) {
+  PlanLayout L;
+  L.n_items_cap = num_ctas + n_segs;
+  L.off_cta = sizeof(PlanHeader);
+  L.off_items = align_up(L.off_cta + sizeof(int32_t) * (size_t)(num_ctas + 1), 16);
+  L.off_seg = L.off_items + sizeof(WorkItem) * (size_t)L.n_items_cap;
+  L.bytes = align_up(L.off_seg + sizeof(SegInfo) * (size_t)n_segs, 16);
+  return L;
+}
+
+constexpr size_t kPartOBytes = (size_t)kMaxG * kD * sizeof(float);  // one partial: 8 heads x 128 floats
+static size_t ws_layout(int n_segs, int num_ctas, size_t* off_lse) {
+  size_t slots = (size_t)num_ctas + n_segs;
+  size_t o = slots * kPartOBytes;
+  if (off_lse) *off_lse = o;
+  return o + slots * kMaxG * sizeof(float);
+}
+
+// ------------------------------------------------------------------------------------------
+// Attention partials
+// ------------------------------------------------------------------------------------------
+struct DecodeArgs {
+  const uint8_t* k_pool;
+  const uint8_t* v_pool;
+  const int32_t* seg_off;
+  const int32_t* seg_len;
+  const uint16_t* q;  // [B, Hq, d]
+  int32_t Hq, Hkv, G;
+  float scale_log2;  // sm_scale * log2(e)
+  const int32_t* cta_item_begin;
+  const WorkItem* items;
+  float* part_o;    // [slots, 8, 128]
+  float* part_lse;  // [slots, 8], log2 domain
+  void* out;
+  int32_t out_fp32;
+  float* lse_out;
+};
+
+constexpr int kStageBytes = 2 * kTile * kRowBytes;     // K tile + V tile
+constexpr int kQSlotBytes = kMaxG * kRowBytes;         // 8 query rows
+constexpr int kMergeRegs = 36;                         // 32 accumulators + m0, m1, l0, l1
+constexpr int kMergeSlotBytes = kMergeRegs * 32 * 4;
+constexpr int kDecodeSmem = kStages * (kStageBytes + kQSlotBytes) + 2 * kMergeSlotBytes;
+
+struct ItemCursor {
+  int seg, t0, t1, ntiles, slot;
+  int64_t row_base;  // first pool row of the piece
+};
+
+__device__ __forceinline__ ItemCursor read_item(const DecodeArgs& a, int it) {
+  const int4 w = __ldg(reinterpret_cast<const int4*>(a.items) + it);
+  ItemCursor c;
+  c.seg = w.x;
+  c.t0 = w.y;
+  c.t1 = (w.z < 0) ? __ldg(a.seg_len + w.x) : w.z;
+  c.slot = w.w;
+  const int rows = c.t1 - c.t0;
+  c.ntiles = rows > 0 ? (rows + kTile - 1) / kTile : 1;
+  c.row_base = (int64_t)__ldg(a.seg_off + w.x) + c.t0;
+  return c;
+}
+
+__global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const DecodeArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int item_begin = a.cta_item_begin[blockIdx.x];
+  const int item_end = a.cta_item_begin[blockIdx.x + 1];
+  if (item_begin >= item_end) return;
+
+  const uint32_t s_stage = smem_u32(smem);
+  const uint32_t s_q = s_stage + kStages * kStageBytes;
+  float* merge = reinterpret_cast<float*>(smem + kStages * (kStageBytes + kQSlotBytes));
+
+  // ---- producer: issues one tile (and the item's queries with its first tile) per call
+  int p_item = item_begin, p_tile = 0, p_seq = 0;
+  ItemCursor pc = read_item(a, p_item);
+  auto issue = [&]() {
+    if (p_item < item_end) {
+      const uint32_t sb = s_stage + (p_seq % kStages) * kStageBytes;
+      const int rows_left = pc.t1 - pc.t0 - p_tile * kTile;
+      const int64_t row0 = pc.row_base + (int64_t)p_tile * kTile;
+#pragma unroll
+      for (int i = 0; i < (kTile * 16) / kDecodeThreads; ++i) {
+        const int id = tid + i * kDecodeThreads;
+        const int r = id >> 4, c = id & 15;
+        const int ok = r < rows_left ? 16 : 0;
+        const int64_t goff = (ok ? row0 + r : 0) * kRowBytes + c * 16;  // padding rows read nothing
+        const uint32_t so = tile_off(r, c);
+        cp_async16(sb + so, a.k_pool + goff, ok);
+        cp_async16(sb + kTile * kRowBytes + so, a.v_pool + goff, ok);
+      }
+      if (p_tile == 0) {
+        // the group's G query rows; heads >= G are zero-filled
+        const uint32_t qb = s_q + ((p_item - item_begin) % kStages) * kQSlotBytes;
+        const int b = pc.seg / a.Hkv, h = pc.seg % a.Hkv;
+        const int r = tid >> 4, c = tid & 15;  // 128 threads = 8 rows x 16 chunks
+        const int ok = r < a.G ? 16 : 0;
+        const uint16_t* src = a.q + ((int64_t)b * a.Hq + h * a.G + (ok ? r : 0)) * kD + c * 8;
+        cp_async16(qb + r * kRowBytes + c * 16, src, ok);
+      }
+      ++p_seq;
+      if (++p_tile == pc.ntiles) {
+        p_tile = 0;
+        if (++p_item < item_end) pc = read_item(a, p_item);
+      }
+    }
+    cp_async_commit();
+  };
+
+#pragma unroll
+  for (int s = 0; s < kStages - 1; ++s) issue();
+
+  int seq = 0;
+  for (int c_item = item_begin; c_item < item_end; ++c_item) {
+    const ItemCursor cc = read_item(a, c_item);
+    uint32_t qf[8][2];
+    float o[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+    for (int tile = 0; tile < cc.ntiles; ++tile, ++seq) {
+      cp_async_wait<kStages - 2>();
+      __syncthreads();
+      issue();
+      if (tile == 0) {
+        const uint8_t* qs = smem + kStages * kStageBytes + ((c_item - item_begin) % kStages) * kQSlotBytes;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          qf[ks][0] = *reinterpret_cast<const uint32_t*>(qs + g * kRowBytes + (ks * 16 + 2 * t) * 2);
+          qf[ks][1] = *reinterpret_cast<const uint32_t*>(qs + g * kRowBytes + (ks * 16 + 8 + 2 * t) * 2);
+        }
+      }
+      const int nvalid = cc.t1 - cc.t0 - tile * kTile;  // valid rows of this tile (may exceed kTile)
+      const int row0 = warp * 16;
+      if (row0 >= nvalid) continue;  // warp-uniform: this warp's 16 rows are all padding
+      const uint32_t kb = s_stage + (seq % kStages) * kStageBytes;
+      const uint32_t vb = kb + kTile * kRowBytes;
+
+      // ---- S[16 tokens x 8 heads] = K_tile . Q^T
+      float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb2[4] = {0.f, 0.f, 0.f, 0.f};
+      {
+        const int r = row0 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int cadd = lane >> 4;
+#pragma unroll
+        for (int ks = 0; ks < 8; ks += 2) {
+          uint32_t af[4];
+          ldmatrix_x4(af, kb + tile_off(r, ks * 2 + cadd));
+          mma_bf16_16816(sa, af, qf[ks][0], qf[ks][1]);
+          ldmatrix_x4(af, kb + tile_off(r, ks * 2 + 2 + cadd));
+          mma_bf16_16816(sb2, af, qf[ks + 1][0], qf[ks + 1][1]);
+        }
+      }
+      // x0: (token g, head 2t)  x1: (token g, head 2t+1)  x2: (token g+8, head 2t)  x3: (token g+8, head 2t+1)
+      const bool v_lo = row0 + g < nvalid, v_hi = row0 + g + 8 < nvalid;
+      const float x0 = v_lo ? (sa[0] + sb2[0]) * a.scale_log2 : -INFINITY;
+      const float x1 = v_lo ? (sa[1] + sb2[1]) * a.scale_log2 : -INFINITY;
+      const float x2 = v_hi ? (sa[2] + sb2[2]) * a.scale_log2 : -INFINITY;
+      const float x3 = v_hi ? (sa[3] + sb2[3]) * a.scale_log2 : -INFINITY;
+      float mx0 = fmaxf(x0, x2), mx1 = fmaxf(x1, x3);
+#pragma unroll
+      for (int sh = 4; sh <= 16; sh <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
+      }
+      // row 0 of the warp's block is valid here, so the new maxima are finite
+      const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+      const float al0 = fast_exp2(m0 - mn0), al1 = fast_exp2(m1 - mn1);  // exp2(-inf) = 0 on the first block
+      m0 = mn0;
+      m1 = mn1;
+      const float p0 = fast_exp2(x0 - mn0), p1 = fast_exp2(x1 - mn1);
+      const float p2 = fast_exp2(x2 - mn0), p3 = fast_exp2(x3 - mn1);
+      l0 = l0 * al0 + p0 + p2;
+      l1 = l1 * al1 + p1 + p3;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        o[i][0] *= al0;
+        o[i][1] *= al1;
+        o[i][2] *= al0;
+        o[i][3] *= al1;
+      }
+      // P as bf16 hi + lo, transposed into the B-operand layout (k = token, n = head)
+      const float h0 = bf16_round(p0), h1 = bf16_round(p1), h2 = bf16_round(p2), h3 = bf16_round(p3);
+      const uint32_t bh0 = movmatrix_trans(pack_bf16(h0, h1));
+      const uint32_t bh1 = movmatrix_trans(pack_bf16(h2, h3));
+      const uint32_t bl0 = movmatrix_trans(pack_bf16(p0 - h0, p1 - h1));
+      const uint32_t bl1 = movmatrix_trans(pack_bf16(p2 - h2, p3 - h3));
+      // ---- O^T[128 d x 8 heads] += V_tile^T . P
+      {
+        const int r = row0 + (lane & 7) + ((lane >> 4) & 1) * 8;
+        const int cadd = (lane >> 3) & 1;
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          uint32_t af[4];
+          ldmatrix_x4_trans(af, vb + tile_off(r, mt * 2 + cadd));
+          mma_bf16_16816(o[mt], af, bh0, bh1);
+          mma_bf16_16816(o[mt], af, bl0, bl1);
+        }
+      }
+    }
+
+    // ---- end of the piece: finish the row sums, merge the four warps, write the result
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+      l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
+      l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
+    }
+#pragma unroll
+    for (int round = 0; round < 2; ++round) {
+      const int stride = 1 << round;                       // 1, then 2
+      const bool writer = (warp & (2 * stride - 1)) == stride;  // round 0: warps 1,3; round 1: warp 2
+      const bool reader = (warp & (2 * stride - 1)) == 0;       // round 0: warps 0,2; round 1: warp 0
+      float* mb = merge + (warp >> (round + 1)) * (kMergeRegs * 32);
+      if (writer) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mb[(i * 4 + j) * 32 + lane] = o[i][j];
+        mb[32 * 32 + lane] = m0;
+        mb[33 * 32 + lane] = m1;
+        mb[34 * 32 + lane] = l0;
+        mb[35 * 32 + lane] = l1;
+      }
+      __syncthreads();
+      if (reader) {
+        const float om0 = mb[32 * 32 + lane], om1 = mb[33 * 32 + lane];
+        const float ol0 = mb[34 * 32 + lane], ol1 = mb[35 * 32 + lane];
+        const float mn0 = fmaxf(m0, om0), mn1 = fmaxf(m1, om1);
+        const float a0 = (m0 == -INFINITY) ? 0.f : fast_exp2(m0 - mn0);
+        const float b0 = (om0 == -INFINITY) ? 0.f : fast_exp2(om0 - mn0);
+        const float a1 = (m1 == -INFINITY) ? 0.f : fast_exp2(m1 - mn1);
+        const float b1 = (om1 == -INFINITY) ? 0.f : fast_exp2(om1 - mn1);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          o[i][0] = o[i][0] * a0 + mb[(i * 4 + 0) * 32 + lane] * b0;
+          o[i][1] = o[i][1] * a1 + mb[(i * 4 + 1) * 32 + lane] * b1;
+          o[i][2] = o[i][2] * a0 + mb[(i * 4 + 2) * 32 + lane] * b0;
+          o[i][3] = o[i][3] * a1 + mb[(i * 4 + 3) * 32 + lane] * b1;
+        }
+        l0 = l0 * a0 + ol0 * b0;
+        l1 = l1 * a1 + ol1 * b1;
+        m0 = mn0;
+        m1 = mn1;
+      }
+      if (round == 0) __syncthreads();  // slot 0 is rewritten by warp 2 in the next round
+    }
+    if (warp == 0) {
+      // stage the normalised [8 heads x 128] block in shared memory, then write whole rows
+      float* st = merge;  // slot 0: free again (its reader is this warp)
+      const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        st[(2 * t) * kD + i * 16 + g] = o[i][0] * i0;
+        st[(2 * t + 1) * kD + i * 16 + g] = o[i][1] * i1;
+        st[(2 * t) * kD + i * 16 + g + 8] = o[i][2] * i0;
+        st[(2 * t + 1) * kD + i * 16 + g + 8] = o[i][3] * i1;
+      }
+      __syncwarp();
+      const float lse0 = l0 > 0.f ? m0 + log2f(l0) : -INFINITY;
+      const float lse1 = l1 > 0.f ? m1 + log2f(l1) : -INFINITY;
+      const int b = cc.seg / a.Hkv, h = cc.seg % a.Hkv;
+      if (cc.slot >= 0) {
+        float* po = a.part_o + (size_t)cc.slot * (kMaxG * kD);
+        for (int hd = 0; hd < a.G; ++hd)
+          reinterpret_cast<float4*>(po + hd * kD)[lane] = reinterpret_cast<const float4*>(st + hd * kD)[lane];
+        if (g == 0) {
+          if (2 * t < a.G) a.part_lse[(size_t)cc.slot * kMaxG + 2 * t] = lse0;
+          if (2 * t + 1 < a.G) a.part_lse[(size_t)cc.slot * kMaxG + 2 * t + 1] = lse1;
+        }
+      } else {
+        const size_t obase = ((size_t)b * a.Hq + (size_t)h * a.G) * kD;
+        for (int hd = 0; hd < a.G; ++hd) {
+          const float4 v = reinterpret_cast<const float4*>(st + hd * kD)[lane];
+          if (a.out_fp32) {
+            reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + obase + hd * kD)[lane] = v;
+          } else {
+            uint2 pk;
+            pk.x = pack_bf16(v.x, v.y);
+            pk.y = pack_bf16(v.z, v.w);
+            reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(a.out) + obase + hd * kD)[lane] = pk;
+          }
+        }
+        if (a.lse_out && g == 0) {
+          const float ln2 = 0.6931471805599453f;
+          if (2 * t < a.G) a.lse_out[(size_t)b * a.Hq + h * a.G + 2 * t] = lse0 * ln2;
+          if (2 * t + 1 < a.G) a.lse_out[(size_t)b * a.Hq + h * a.G + 2 * t + 1] = lse1 * ln2;
+        }
+      }
+    }
+  }
+  cp_async_wait<0>();
+}
+
+// ------------------------------------------------------------------------------------------
+// Combine: merge the partials of every segment that was cut into several pieces
+// ------------------------------------------------------------------------------------------
+struct CombineArgs {
+  const SegInfo* seg_info;
+  const float* part_o;
+  const float* part_lse;
+  void* out;
+  float* lse_out;
+  int32_t Hq, Hkv, G, out_fp32;
+};
+
+__global__ void __launch_bounds__(kD) decode_combine_kernel(const CombineArgs a) {
+  const int seg = blockIdx.x, hd = blockIdx.y, dI = threadIdx.x;
+  const SegInfo si = a.seg_info[seg];
+  if (si.n_pieces == 1) return;  // written directly by the attention kernel
+  const int b = seg / a.Hkv, h = seg % a.Hkv;
+  const size_t oidx = ((size_t)b * a.Hq + (size_t)h * a.G + hd) * kD + dI;
+  float acc = 0.f, wsum = 0.f, M = -INFINITY;
+  for (int p = 0; p < si.n_pieces; ++p) M = fmaxf(M, a.part_lse[(size_t)(si.slot_begin + p) * kMaxG + hd]);
+  if (M > -INFINITY) {
+    for (int p = 0; p < si.n_pieces; ++p) {
+      const size_t s = (size_t)(si.slot_begin + p);
+      const float w = exp2f(a.part_lse[s * kMaxG + hd] - M);
+      acc += w * a.part_o[s * (kMaxG * kD) + hd * kD + dI];
+      wsum += w;
+    }
+    acc /= wsum;
+  }
+  if (a.out_fp32)
+    reinterpret_cast<float*>(a.out)[oidx] = acc;
+  else
+    reinterpret_cast<__nv_bfloat16*>(a.out)[oidx] = __float2bfloat16_rn(acc);
+  if (a.lse_out && dI == 0)
+    a.lse_out[(size_t)b * a.Hq + h * a.G + hd] = (M > -INFINITY) ? (M + log2f(wsum)) * 0.6931471805599453f : -INFINITY;
+}
+
+// ------------------------------------------------------------------------------------------
+// Append
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) append_kernel(uint8_t* k_pool, uint8_t* v_pool, const int32_t* seg_off,
+                                                     int32_t* seg_len, const uint8_t* k_new, const uint8_t* v_new,
+                                                     int n_segs) {
+  const int seg = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (seg >= n_segs) return;
+  const int len = seg_len[seg];
+  const int64_t row = (int64_t)seg_off[seg] + len;
+  const int c = lane & 15;
+  const uint8_t* src = (lane < 16 ? k_new : v_new) + (size_t)seg * kRowBytes + c * 16;
+  uint8_t* dst = (lane < 16 ? k_pool : v_pool) + row * kRowBytes + c * 16;
+  *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+  __syncwarp();
+  if (lane == 0) seg_len[seg] = len + 1;
+}
+
+static int check_cache(const catekv_cache* c) {
+  if (!c) return CATEKV_ERR_INVALID_ARG;
+  if (c->B <= 0 || c->Hkv <= 0 || c->total_rows < 0) return CATEKV_ERR_INVALID_ARG;
+  if (c->d != kD) return CATEKV_ERR_UNSUPPORTED;
+  if (!c->k_pool || !c->v_pool || !c->seg_off_dev || !c->seg_len_dev || !c->seg_off || !c->seg_cap || !c->seg_len)
+    return CATEKV_ERR_INVALID_ARG;
+  return CATEKV_OK;
+}
+
+}  // namespace catekv
+
+using namespace catekv;
+
+extern "C" int catekv_append(catekv_cache* cache, const void* k_new, const void* v_new, catekv_stream stream) {
+  int rc = check_cache(cache);
+  if (rc) return rc;
+  if (!k_new || !v_new) return CATEKV_ERR_INVALID_ARG;
+  const int n = cache->B * cache->Hkv;
+  for (int s = 0; s < n; ++s) {
+    if (cache->seg_len[s] < 0) return CATEKV_ERR_INVALID_ARG;
+    if (cache->seg_len[s] + 1 > cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+  }
+  append_kernel<<<(n + 3) / 4, 128, 0, (cudaStream_t)stream>>>(
+      (uint8_t*)cache->k_pool, (uint8_t*)cache->v_pool, cache->seg_off_dev, cache->seg_len_dev,
+      (const uint8_t*)k_new, (const uint8_t*)v_new, n);
+  CATEKV_CUDA_TRY(cudaGetLastError());
+  for (int s = 0; s < n; ++s) cache->seg_len[s] += 1;
+  return CATEKV_OK;
+}
+
+extern "C" int catekv_decode_num_ctas(void) {
+  int dev = 0, sms = 0, per_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return CATEKV_ERR_CUDA;
+  cudaError_t e = cudaFuncSetAttribute(decode_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
+  if (e != cudaSuccess) { set_cuda_error(e); return CATEKV_ERR_CUDA; }
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) { set_cuda_error(e); return CATEKV_ERR_CUDA; }
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_partial_kernel, kDecodeThreads, kDecodeSmem);
+  if (e != cudaSuccess) { set_cuda_error(e); return CATEKV_ERR_CUDA; }
+  if (per_sm < 1) per_sm = 1;
+  return sms * per_sm;
+}
+
+extern "C" size_t catekv_decode_plan_bytes(int32_t B, int32_t Hkv, int32_t num_ctas) {
+  if (B <= 0 || Hkv <= 0 || num_ctas <= 0) return 0;
+  return plan_layout(B * Hkv, num_ctas).bytes;
+}
+
+extern "C" size_t catekv_decode_workspace_bytes(int32_t B, int32_t Hkv, int32_t num_ctas) {
+  if (B <= 0 || Hkv <= 0 || num_ctas <= 0) return 0;
+  return ws_layout(B * Hkv, num_ctas, nullptr);
+}
+
+extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, void* plan_host, void* plan_dev,
+                                  size_t plan_bytes, catekv_stream stream) {
+  int rc = check_cache(cache);
+  if (rc) return rc;
+  if (num_ctas <= 0 || !plan_host) return CATEKV_ERR_INVALID_ARG;
+  const int n_segs = cache->B * cache->Hkv;
+  const PlanLayout L = plan_layout(n_segs, num_ctas);
+  if (plan_bytes < L.bytes) return CATEKV_ERR_WORKSPACE;
+  int64_t total = 0;
+  for (int s = 0; s < n_segs; ++s) {
+    if (cache->seg_len[s] < 0 || cache->seg_len[s] > cache->seg_cap[s]) return CATEKV_ERR_INVALID_ARG;
+    total += cache->seg_len[s];
+  }
+  uint8_t* base = (uint8_t*)plan_host;
+  PlanHeader* hdr = (PlanHeader*)base;
+  int32_t* cta_begin = (int32_t*)(base + L.off_cta);
+  WorkItem* items = (WorkItem*)(base + L.off_items);
+  SegInfo* segs = (SegInfo*)(base + L.off_seg);
+
+  // rows per CTA: an equal share of all rows, rounded up to the split alignment
+  int64_t quota = (total + num_ctas - 1) / num_ctas;
+  quota = (quota + kSplitAlign - 1) / kSplitAlign * kSplitAlign;
+  if (quota < kSplitAlign) quota = kSplitAlign;
+
+  int n_items = 0, n_slots = 0;
+  int seg = 0;
+  int32_t pos = 0;  // next unassigned row of `seg`
+  while (seg < n_segs && cache->seg_len[seg] == 0) { segs[seg] = SegInfo{0, 0}; ++seg; }
+  int seg_first_item = n_items;
+  for (int c = 0; c < num_ctas; ++c) {
+    cta_begin[c] = n_items;
+    int64_t room = quota;
+    while (room > 0 && seg < n_segs) {
+      const int32_t len = cache->seg_len[seg];
+      const int32_t take = (int32_t)((int64_t)(len - pos) < room ? (len - pos) : room);
+      items[n_items++] = WorkItem{seg, pos, pos + take, 0};
+      pos += take;
+      room -= take;
+      if (pos == len) {
+        // segment finished: fix up its pieces
+        const int pieces = n_items - seg_first_item;
+        items[n_items - 1].t1 = -1;  // the last piece follows the segment's current length
+        if (pieces == 1) {
+          items[seg_first_item].slot = -1;
+          segs[seg] = SegInfo{0, 1};
+        } else {
+          for (int i = 0; i < pieces; ++i) items[seg_first_item + i].slot = n_slots + i;
+          segs[seg] = SegInfo{n_slots, pieces};
+          n_slots += pieces;
+        }
+        ++seg;
+        pos = 0;
+        while (seg < n_segs && cache->seg_len[seg] == 0) { segs[seg] = SegInfo{0, 0}; ++seg; }
+        seg_first_item = n_items;
+      }
+    }
+  }
+  cta_begin[num_ctas] = n_items;
+  if (seg != n_segs) return CATEKV_ERR_INVALID_ARG;  // cannot happen: quota * num_ctas >= total
+  hdr->magic = kPlanMagic;
+  hdr->num_ctas = num_ctas;
+  hdr->n_segs = n_segs;
+  hdr->n_items = n_items;
+  hdr->n_slots = n_slots;
+  hdr->tile = kTile;
+  hdr->total_rows = total;
+  if (plan_dev)
+    CATEKV_CUDA_TRY(cudaMemcpyAsync(plan_dev, plan_host, L.bytes, cudaMemcpyHostToDevice, (cudaStream_t)stream));
+  return CATEKV_OK;
+}
+
+extern "C" int catekv_decode_attn(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
+                                  int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
+                                  size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+  int rc = check_cache(cache);
+  if (rc) return rc;
+  if (!q || !out || !plan_host || !plan_dev || !ws) return CATEKV_ERR_INVALID_ARG;
+  if (Hq <= 0 || Hq % cache->Hkv != 0) return CATEKV_ERR_INVALID_ARG;
+  const int G = Hq / cache->Hkv;
+  if (G > kMaxG) return CATEKV_ERR_UNSUPPORTED;
+  if (out_dtype != CATEKV_OUT_BF16 && out_dtype != CATEKV_OUT_FP32) return CATEKV_ERR_UNSUPPORTED;
+  if (!(sm_scale >= 0.f) || isinf(sm_scale)) return CATEKV_ERR_INVALID_ARG;
+  const PlanHeader* hdr = (const PlanHeader*)plan_host;
+  const int n_segs = cache->B * cache->Hkv;
+  if (plan_bytes < sizeof(PlanHeader) || hdr->magic != kPlanMagic || hdr->n_segs != n_segs || hdr->num_ctas <= 0 ||
+      hdr->tile != kTile)
+    return CATEKV_ERR_INVALID_ARG;
+  const PlanLayout L = plan_layout(n_segs, hdr->num_ctas);
+  if (plan_bytes < L.bytes) return CATEKV_ERR_WORKSPACE;
+  size_t off_lse = 0;
+  if (ws_bytes < ws_layout(n_segs, hdr->num_ctas, &off_lse)) return CATEKV_ERR_WORKSPACE;
+
+  static bool attr_set[64] = {};
+  int dev = 0;
+  CATEKV_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  const uint8_t* pd = (const uint8_t*)plan_dev;
+  DecodeArgs a;
+  a.k_pool = (const uint8_t*)cache->k_pool;
+  a.v_pool = (const uint8_t*)cache->v_pool;
+  a.seg_off = cache->seg_off_dev;
+  a.seg_len = cache->seg_len_dev;
+  a.q = (const uint16_t*)q;
+  a.Hq = Hq;
+  a.Hkv = cache->Hkv;
+  a.G = G;
+  a.scale_log2 = (sm_scale == 0.f ? 1.0f / sqrtf((float)kD) : sm_scale) * 1.4426950408889634f;
+  a.cta_item_begin = (const int32_t*)(pd + L.off_cta);
+  a.items = (const WorkItem*)(pd + L.off_items);
+  a.part_o = (float*)ws;
+  a.part_lse = (float*)((uint8_t*)ws + off_lse);
+  a.out = out;
+  a.out_fp32 = out_dtype == CATEKV_OUT_FP32;
+  a.lse_out = lse_out;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (hdr->n_items > 0) {
+    decode_partial_kernel<<<hdr->num_ctas, kDecodeThreads, kDecodeSmem, st>>>(a);
+    CATEKV_CUDA_TRY(cudaGetLastError());
+  }
+  CombineArgs ca;
+  ca.seg_info = (const SegInfo*)(pd + L.off_seg);
+  ca.part_o = a.part_o;
+  ca.part_lse = a.part_lse;
+  ca.out = out;
+  ca.lse_out = lse_out;
+  ca.Hq = Hq;
+  ca.Hkv = cache->Hkv;
+  ca.G = G;
+  ca.out_fp32 = a.out_fp32;
+  decode_combine_kernel<<<dim3(n_segs, G), kD, 0, st>>>(ca);
+  CATEKV_CUDA_TRY(cudaGetLastError());
+  return CATEKV_OK;
+}

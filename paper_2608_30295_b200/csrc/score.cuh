@@ -1,0 +1,38 @@
+// Observation-window scoring shared by catekv_select_compact (Algorithm 1, token criticality)
+// and catekv_head_cv (Eq. 1): softmax(Q_win K^T / sqrt(d)) over a key range, per query head
+// of the group, reduced either to column sums (C_j) or to the group-mean matrix (A_ij).
+#pragma once
+
+#include "common.cuh"
+
+namespace catekv {
+
+// One (sequence, KV head) to score: keys [j_begin, j_end) of a sequence of n tokens.
+struct ScoreJob {
+  int32_t b, h, n, j_begin, j_end, reserved;
+};
+
+struct ScoreArgs {
+  const uint16_t* q_win;  // [B, Hq, L_obs, d]
+  const uint16_t* k;      // element strides sb, sh, st; d contiguous
+  int64_t sb, sh, st;
+  const ScoreJob* jobs;   // device
+  int32_t n_jobs, Hq, G, L_obs, causal;
+  float scale_log2;       // log2(e) / sqrt(d)
+  int32_t keys_per_cta;   // multiple of 64
+  int32_t n_chunks;       // grid.x: ceil(max key range / keys_per_cta)
+  float2* stats_part;     // [n_jobs][n_chunks * key_groups][rows_pad]  (row max in log2 domain, row sum)
+  float2* stats;          // [n_jobs][rows_pad]                        (row max, 1 / row sum)
+  float* out;             // column sums C[job][j - j_begin] or matrix A[job][i][j - j_begin]
+  int64_t out_job_stride, out_row_stride;
+};
+
+enum ScoreMode { kScoreStats = 0, kScoreColsum = 1, kScoreMatrix = 2 };
+
+// rows_pad = G * (16 * n_it), n_it = 2 for L_obs <= 32, 4 for L_obs <= 64
+int score_rows_pad(int G, int L_obs);
+int score_key_groups(int L_obs);
+// Enqueue: pass 1 (row max / sum partials), their merge, and pass 2 (column sums or matrix).
+int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream);
+
+}  // namespace catekv

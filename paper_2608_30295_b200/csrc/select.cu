@@ -1,0 +1,399 @@
+// Prefill-end selection (Algorithm 1, pre-filling stage): window scores -> pooling -> per-KV-head
+// top-k with lowest-index tie-break -> ascending kept list -> gather of K/V rows into the
+// head's segment of the pool.
+#include <math.h>
+
+#include <vector>
+
+#include "radix.cuh"
+#include "score.cuh"
+
+namespace catekv {
+
+struct SelSeg {
+  int32_t n;         // tokens of the sequence
+  int32_t keep_all;  // 1: straight copy of all n rows
+  int32_t job;       // scoring job index, -1 if none (keep_all, or nothing to select)
+  int32_t k_sel;     // candidates (tokens, or chunks in CHUNK mode) to select
+  int32_t n_pool;    // pooled entries (candidate tokens, or chunks)
+  int32_t cand_end;  // candidates are tokens [sink, cand_end)
+  int32_t len_ub;    // upper bound of the kept length (exact except for a short last chunk)
+  int32_t reserved;
+};
+
+struct TopkArgs {
+  const SelSeg* segs;
+  const float* C;       // [n_jobs][c_stride] criticality of tokens [0, n - L_obs)
+  float* P;             // [n_jobs][c_stride] pooled scores (scratch)
+  int64_t c_stride;
+  int32_t* idx;         // [n_segs][idx_stride] kept indices (scratch)
+  int64_t idx_stride;
+  int32_t* seg_len_dev;
+  int32_t sink, local, L_obs, pool_mode, pool_param;
+};
+
+constexpr int kTopkThreads = 1024;
+
+// Block-wide exclusive scan of a packed pair (lo 32 bits, hi 32 bits) over 1024 threads.
+__device__ __forceinline__ unsigned long long block_excl_scan(unsigned long long v, unsigned long long* s_warp,
+                                                              unsigned long long& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned long long x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  if (lane == 31) s_warp[warp] = x;
+  __syncthreads();
+  if (warp == 0) {
+    unsigned long long w = s_warp[lane], ws = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long y = __shfl_up_sync(0xffffffffu, ws, o);
+      if (lane >= o) ws += y;
+    }
+    s_warp[lane] = ws - w;            // exclusive prefix of the warp totals
+    if (lane == 31) s_warp[32] = ws;  // grand total
+  }
+  __syncthreads();
+  const unsigned long long res = s_warp[warp] + x - v;
+  total = s_warp[32];
+  __syncthreads();  // s_warp is reused by the next call
+  return res;
+}
+
+// One CTA per segment that selects: pooling, radix select of the k-th largest pooled score,
+// ordered compaction into the ascending kept list.
+__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
+  const int seg = blockIdx.x;
+  const SelSeg s = a.segs[seg];
+  if (s.keep_all) return;
+  __shared__ unsigned int hist[256];
+  __shared__ unsigned long long s_warp[33];
+  __shared__ unsigned int s_pair[2];
+  const int tid = threadIdx.x;
+  int32_t* idx = a.idx + (size_t)seg * a.idx_stride;
+  const int S = a.sink;
+  int n_sel_tokens = 0;
+
+  if (s.k_sel > 0) {
+    const float* C = a.C + (size_t)s.job * a.c_stride;
+    float* P = a.P + (size_t)s.job * a.c_stride;
+    const int n_sc = s.n - a.L_obs;
+    // ---- pooling
+    if (a.pool_mode == CATEKV_POOL_NONE) {
+      for (int c = tid; c < s.n_pool; c += kTopkThreads) P[c] = C[S + c];
+    } else if (a.pool_mode == CATEKV_POOL_SLIDING) {
+      const int half = (a.pool_param - 1) / 2;
+      for (int c = tid; c < s.n_pool; c += kTopkThreads) {
+        const int j = S + c;
+        const int lo = max(0, j - half), hi = min(n_sc - 1, j + half);
+        float m = C[lo];
+        for (int u = lo + 1; u <= hi; ++u) m = fmaxf(m, C[u]);
+        P[c] = m;
+      }
+    } else {
+      const int cs = a.pool_param;
+      for (int c = tid; c < s.n_pool; c += kTopkThreads) {
+        const int lo = S + c * cs, hi = min(lo + cs, s.cand_end);
+        float m = C[lo];
+        for (int u = lo + 1; u < hi; ++u) m = fmaxf(m, C[u]);
+        P[c] = m;
+      }
+    }
+    __syncthreads();
+    // ---- radix select of the k_sel-th largest pooled score
+    const unsigned int* Pb = reinterpret_cast<const unsigned int*>(P);
+    unsigned int thr, need_eq;  // threshold bits; entries equal to it that are taken (lowest index first)
+    block_radix_select([&](int c) { return Pb[c]; }, s.n_pool, (unsigned int)s.k_sel, hist, s_pair, thr, need_eq);
+    // ---- ordered compaction
+    unsigned long long run = 0;  // packed: low = entries above the threshold so far, high = entries equal to it
+    const int cs = a.pool_mode == CATEKV_POOL_CHUNK ? a.pool_param : 1;
+    for (int base = 0; base < s.n_pool; base += kTopkThreads) {
+      const int c = base + tid;
+      unsigned int v = 0;
+      bool gt = false, eq = false;
+      if (c < s.n_pool) {
+        v = Pb[c];
+        gt = v > thr;
+        eq = v == thr;
+      }
+      unsigned long long tot;
+      const unsigned long long ex =
+          run + block_excl_scan((unsigned long long)gt | ((unsigned long long)eq << 32), s_warp, tot);
+      const unsigned int gt_before = (unsigned int)(ex & 0xffffffffu), eq_before = (unsigned int)(ex >> 32);
+      if (gt || (eq && eq_before < need_eq)) {
+        const unsigned int rank = gt_before + min(eq_before, need_eq);
+        if (cs == 1) {
+          idx[S + rank] = S + c;
+        } else {
+          const int lo = S + c * cs, hi = min(lo + cs, s.cand_end);
+          for (int u = lo; u < hi; ++u) idx[S + rank * cs + (u - lo)] = u;
+        }
+      }
+      run += tot;
+    }
+    // selected tokens: whole chunks, except that the last chunk of the range may be short
+    n_sel_tokens = s.k_sel * cs;
+    if (cs > 1) {
+      const int last = s.n_pool - 1;
+      const int last_sz = s.cand_end - (S + last * cs);
+      const unsigned int vl = Pb[last];
+      // the last chunk is taken iff it is above the threshold, or ties with it and is within the quota of ties
+      const unsigned int eq_total = (unsigned int)(run >> 32);
+      const bool last_taken = vl > thr || (vl == thr && eq_total <= need_eq);
+      if (last_taken) n_sel_tokens -= cs - last_sz;
+    }
+  }
+  for (int i = tid; i < S; i += kTopkThreads) idx[i] = i;
+  for (int i = tid; i < a.local; i += kTopkThreads) idx[S + n_sel_tokens + i] = s.n - a.local + i;
+  if (tid == 0) a.seg_len_dev[seg] = S + n_sel_tokens + a.local;
+}
+
+// keep_all segments: seg_len = n
+__global__ void set_full_len_kernel(const SelSeg* segs, int32_t* seg_len_dev, int n_segs) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_segs && segs[i].keep_all) seg_len_dev[i] = segs[i].n;
+}
+
+struct GatherArgs {
+  const SelSeg* segs;
+  const int32_t* idx;
+  int64_t idx_stride;
+  const uint8_t* k;
+  const uint8_t* v;
+  int64_t sb, sh, st;  // byte strides
+  uint8_t* k_pool;
+  uint8_t* v_pool;
+  const int32_t* seg_off;
+  const int32_t* seg_len_dev;
+  int32_t* idx_out;
+  int64_t idx_out_stride;
+  int32_t Hkv;
+};
+
+constexpr int kGatherRowsPerBlock = 64;
+
+// One warp per kept row: lanes 0-15 move the K row, lanes 16-31 the V row (16 bytes each).
+__global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
+  const int seg = blockIdx.y;
+  const SelSeg s = a.segs[seg];
+  const int len = a.seg_len_dev[seg];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = seg / a.Hkv, h = seg % a.Hkv;
+  const int64_t off = a.seg_off[seg];
+  const uint8_t* src_base = (lane < 16 ? a.k : a.v) + b * a.sb + h * a.sh + (lane & 15) * 16;
+  uint8_t* dst_base = (lane < 16 ? a.k_pool : a.v_pool) + off * kRowBytes + (lane & 15) * 16;
+  const int r0 = blockIdx.x * kGatherRowsPerBlock;
+#pragma unroll 4
+  for (int i = warp; i < kGatherRowsPerBlock; i += 8) {
+    const int r = r0 + i;
+    if (r >= len) break;
+    const int tok = s.keep_all ? r : a.idx[(size_t)seg * a.idx_stride + r];
+    const uint4 val = __ldg(reinterpret_cast<const uint4*>(src_base + (int64_t)tok * a.st));
+    *reinterpret_cast<uint4*>(dst_base + (int64_t)r * kRowBytes) = val;
+    if (a.idx_out && lane == 0) a.idx_out[(size_t)seg * a.idx_out_stride + r] = tok;
+  }
+}
+
+static int keys_per_cta_for(int n_segs, int n_sc_max) {
+  // the smallest power-of-two multiple of 256 keys that keeps the grid within 8 CTAs per SM
+  int kp = 256;
+  while ((long)n_segs * ((n_sc_max + kp - 1) / kp) > 148 * 8 && kp < (1 << 30)) kp *= 2;
+  return kp;
+}
+
+struct SelWs {
+  size_t off_segs, off_jobs, off_part, off_stats, off_C, off_P, off_idx, bytes;
+  int keys_per_cta, n_chunks, rows_pad, kgroups;
+  int64_t c_stride, idx_stride;
+};
+static SelWs sel_ws_layout(int n_segs, int G, int n_max, int L_obs) {
+  SelWs w;
+  const int n_sc = n_max > L_obs ? n_max - L_obs : 1;
+  w.keys_per_cta = keys_per_cta_for(n_segs, n_sc);
+  w.n_chunks = (n_sc + w.keys_per_cta - 1) / w.keys_per_cta;
+  w.rows_pad = score_rows_pad(G, L_obs);
+  w.kgroups = score_key_groups(L_obs);
+  w.c_stride = (int64_t)align_up((size_t)n_sc, 64);
+  w.idx_stride = (int64_t)align_up((size_t)n_max, 64);
+  size_t o = 0;
+  w.off_segs = o; o = align_up(o + sizeof(SelSeg) * (size_t)n_segs, 256);
+  w.off_jobs = o; o = align_up(o + sizeof(ScoreJob) * (size_t)n_segs, 256);
+  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 8 ? n_segs : 148 * 8) * w.kgroups * w.rows_pad, 256);
+  w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * w.rows_pad, 256);
+  w.off_C = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.c_stride, 256);
+  w.off_P = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.c_stride, 256);
+  w.off_idx = o; o = align_up(o + sizeof(int32_t) * (size_t)n_segs * w.idx_stride, 256);
+  w.bytes = o;
+  return w;
+}
+
+}  // namespace catekv
+
+using namespace catekv;
+
+extern "C" size_t catekv_select_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t n_max, int32_t L_obs) {
+  if (B <= 0 || Hq <= 0 || Hkv <= 0 || n_max <= 0 || L_obs <= 0 || Hq % Hkv) return 0;
+  return sel_ws_layout(B * Hkv, Hq / Hkv, n_max, L_obs).bytes;
+}
+
+extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache* cache, int32_t* idx_out,
+                                     int64_t idx_stride, void* ws, size_t ws_bytes, catekv_stream stream) {
+  if (!p || !cache || !ws) return CATEKV_ERR_INVALID_ARG;
+  if (p->B <= 0 || p->Hq <= 0 || p->Hkv <= 0 || p->Hq % p->Hkv) return CATEKV_ERR_INVALID_ARG;
+  if (p->d != kD) return CATEKV_ERR_UNSUPPORTED;
+  const int G = p->Hq / p->Hkv;
+  if (G > kMaxG) return CATEKV_ERR_UNSUPPORTED;
+  if (p->L_obs < 1 || p->sink < 0 || p->local < p->L_obs || p->budget_consistent < 0) return CATEKV_ERR_INVALID_ARG;
+  if (p->L_obs > 64) return CATEKV_ERR_UNSUPPORTED;
+  if (!(p->eta_adaptive >= 0.f)) return CATEKV_ERR_INVALID_ARG;
+  if (p->pool_mode == CATEKV_POOL_CHUNK) {
+    if (p->pool_param < 1) return CATEKV_ERR_INVALID_ARG;
+  } else if (p->pool_mode == CATEKV_POOL_SLIDING) {
+    if (p->pool_param < 1 || p->pool_param % 2 == 0) return CATEKV_ERR_INVALID_ARG;
+  } else if (p->pool_mode != CATEKV_POOL_NONE) {
+    return CATEKV_ERR_UNSUPPORTED;
+  }
+  if (!p->q_win || !p->k || !p->v || !p->seq_len || !p->head_mask) return CATEKV_ERR_INVALID_ARG;
+  if (cache->B != p->B || cache->Hkv != p->Hkv || cache->d != kD) return CATEKV_ERR_INVALID_ARG;
+  if (!cache->k_pool || !cache->v_pool || !cache->seg_off_dev || !cache->seg_len_dev || !cache->seg_off ||
+      !cache->seg_cap || !cache->seg_len)
+    return CATEKV_ERR_INVALID_ARG;
+  const int n_segs = p->B * p->Hkv;
+  int n_max = 0;
+  for (int b = 0; b < p->B; ++b) {
+    if (p->seq_len[b] < 1) return CATEKV_ERR_INVALID_ARG;
+    n_max = p->seq_len[b] > n_max ? p->seq_len[b] : n_max;
+  }
+  if (idx_out && idx_stride < n_max) return CATEKV_ERR_INVALID_ARG;
+  const SelWs W = sel_ws_layout(n_segs, G, n_max, p->L_obs);
+  if (ws_bytes < W.bytes) return CATEKV_ERR_WORKSPACE;
+
+  // ---- per-segment decisions, all on the host
+  std::vector<SelSeg> segs(n_segs);
+  std::vector<ScoreJob> jobs;
+  std::vector<int32_t> new_len(n_segs);
+  bool need_readback = false;
+  int max_len_ub = 0, n_sc_jobs_max = 0;
+  const int S = p->sink, Lc = p->local;
+  for (int b = 0; b < p->B; ++b) {
+    const int n = p->seq_len[b];
+    for (int h = 0; h < p->Hkv; ++h) {
+      const int sgi = b * p->Hkv + h;
+      SelSeg s = {};
+      s.n = n;
+      s.job = -1;
+      int64_t T;
+      if (p->head_mask[sgi]) T = p->budget_consistent;
+      else T = p->eta_adaptive >= 1.f ? n : (int64_t)floor((double)p->eta_adaptive * (double)n);
+      if (T >= n || (int64_t)S + Lc >= n) {
+        s.keep_all = 1;
+        s.len_ub = n;
+      } else {
+        s.cand_end = n - Lc;
+        const int ncand = s.cand_end - S;
+        const int k_rest = (int)(T - S - Lc > 0 ? T - S - Lc : 0);
+        int sel_tokens;
+        if (p->pool_mode == CATEKV_POOL_CHUNK) {
+          const int cs = p->pool_param;
+          s.n_pool = (ncand + cs - 1) / cs;
+          s.k_sel = k_rest / cs;
+          sel_tokens = s.k_sel * cs;
+          if (s.k_sel > 0 && ncand % cs != 0) need_readback = true;
+        } else {
+          s.n_pool = ncand;
+          s.k_sel = k_rest;
+          sel_tokens = k_rest;
+        }
+        s.len_ub = S + sel_tokens + Lc;
+        if (s.k_sel > 0) {
+          s.job = (int)jobs.size();
+          jobs.push_back(ScoreJob{b, h, n, 0, n - p->L_obs, 0});
+          n_sc_jobs_max = n - p->L_obs > n_sc_jobs_max ? n - p->L_obs : n_sc_jobs_max;
+        }
+      }
+      if (s.len_ub > cache->seg_cap[sgi]) return CATEKV_ERR_CAPACITY;
+      max_len_ub = s.len_ub > max_len_ub ? s.len_ub : max_len_ub;
+      new_len[sgi] = s.len_ub;
+      segs[sgi] = s;
+    }
+  }
+
+  cudaStream_t st = (cudaStream_t)stream;
+  uint8_t* w8 = (uint8_t*)ws;
+  SelSeg* d_segs = (SelSeg*)(w8 + W.off_segs);
+  ScoreJob* d_jobs = (ScoreJob*)(w8 + W.off_jobs);
+  CATEKV_CUDA_TRY(cudaMemcpyAsync(d_segs, segs.data(), sizeof(SelSeg) * n_segs, cudaMemcpyHostToDevice, st));
+  if (!jobs.empty()) {
+    CATEKV_CUDA_TRY(cudaMemcpyAsync(d_jobs, jobs.data(), sizeof(ScoreJob) * jobs.size(), cudaMemcpyHostToDevice, st));
+    ScoreArgs sa = {};
+    sa.q_win = (const uint16_t*)p->q_win;
+    sa.k = (const uint16_t*)p->k;
+    sa.sb = p->kv_stride_b;
+    sa.sh = p->kv_stride_h;
+    sa.st = p->kv_stride_t;
+    sa.jobs = d_jobs;
+    sa.n_jobs = (int)jobs.size();
+    sa.Hq = p->Hq;
+    sa.G = G;
+    sa.L_obs = p->L_obs;
+    sa.causal = 0;  // every scored key precedes every window query
+    sa.scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
+    sa.keys_per_cta = W.keys_per_cta;
+    sa.n_chunks = (n_sc_jobs_max + W.keys_per_cta - 1) / W.keys_per_cta;
+    sa.stats_part = (float2*)(w8 + W.off_part);
+    sa.stats = (float2*)(w8 + W.off_stats);
+    sa.out = (float*)(w8 + W.off_C);
+    sa.out_job_stride = W.c_stride;
+    sa.out_row_stride = 0;
+    int rc = score_launch(sa, kScoreColsum, st);
+    if (rc) return rc;
+  }
+  TopkArgs ta;
+  ta.segs = d_segs;
+  ta.C = (const float*)(w8 + W.off_C);
+  ta.P = (float*)(w8 + W.off_P);
+  ta.c_stride = W.c_stride;
+  ta.idx = (int32_t*)(w8 + W.off_idx);
+  ta.idx_stride = W.idx_stride;
+  ta.seg_len_dev = cache->seg_len_dev;
+  ta.sink = S;
+  ta.local = Lc;
+  ta.L_obs = p->L_obs;
+  ta.pool_mode = p->pool_mode;
+  ta.pool_param = p->pool_param;
+  topk_kernel<<<n_segs, kTopkThreads, 0, st>>>(ta);
+  CATEKV_CUDA_TRY(cudaGetLastError());
+  set_full_len_kernel<<<(n_segs + 255) / 256, 256, 0, st>>>(d_segs, cache->seg_len_dev, n_segs);
+  CATEKV_CUDA_TRY(cudaGetLastError());
+
+  GatherArgs ga;
+  ga.segs = d_segs;
+  ga.idx = ta.idx;
+  ga.idx_stride = W.idx_stride;
+  ga.k = (const uint8_t*)p->k;
+  ga.v = (const uint8_t*)p->v;
+  ga.sb = p->kv_stride_b * 2;
+  ga.sh = p->kv_stride_h * 2;
+  ga.st = p->kv_stride_t * 2;
+  ga.k_pool = (uint8_t*)cache->k_pool;
+  ga.v_pool = (uint8_t*)cache->v_pool;
+  ga.seg_off = cache->seg_off_dev;
+  ga.seg_len_dev = cache->seg_len_dev;
+  ga.idx_out = idx_out;
+  ga.idx_out_stride = idx_stride;
+  ga.Hkv = p->Hkv;
+  gather_kernel<<<dim3((max_len_ub + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock, n_segs), 256, 0, st>>>(ga);
+  CATEKV_CUDA_TRY(cudaGetLastError());
+
+  if (need_readback) {
+    // a short last chunk makes the kept length depend on the scores: fetch the device's lengths
+    CATEKV_CUDA_TRY(cudaMemcpyAsync(cache->seg_len, cache->seg_len_dev, sizeof(int32_t) * n_segs, cudaMemcpyDeviceToHost, st));
+    CATEKV_CUDA_TRY(cudaStreamSynchronize(st));
+  } else {
+    for (int i = 0; i < n_segs; ++i) cache->seg_len[i] = new_len[i];
+  }
+  return CATEKV_OK;
+}

@@ -1,0 +1,101 @@
+"""Shared helpers of the library tests: loading oracle caches onto the device and error metrics."""
+import math
+
+import numpy as np
+import torch
+
+from oracle import catekv_oracle as orc
+from workloads import synth
+
+# Tolerances (bf16 inputs, fp32 accumulation): relative L2 <= 1e-3 and max-abs <= 1e-2 on attention
+# outputs.  The fp32 output is compared with the oracle's fp64 result, the bf16 output with the oracle's
+# result rounded to bf16 (rounding alone costs ~1.7e-3 relative L2, so like is compared with like).
+REL_L2 = 1e-3
+MAX_ABS = 1e-2
+TIE_BAND = 1e-4  # relative gap below which the k-th / (k+1)-th pooled scores count as tied
+
+
+def rel_l2(got, ref):
+    got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    den = np.linalg.norm(ref)
+    return float(np.linalg.norm(got - ref) / (den if den > 0 else 1.0))
+
+
+def max_abs(got, ref):
+    return float(np.max(np.abs(np.asarray(got, dtype=np.float64) - np.asarray(ref, dtype=np.float64)))) if np.size(ref) else 0.0
+
+
+def device_cache_from_oracle(ck, ocache, max_new, device="cuda"):
+    """Copy an oracle HybridCache into a device Cache (rows written by torch copies)."""
+    lens = ocache.lengths()
+    cache = ck.Cache(ocache.B, ocache.Hkv, lens, max_new, device)
+    for i in range(ocache.B * ocache.Hkv):
+        L = int(lens[i])
+        if L:
+            o = int(cache.seg_off[i])
+            cache.k_pool[o:o + L] = synth.from_bits(ocache.k_rows[i], device)
+            cache.v_pool[o:o + L] = synth.from_bits(ocache.v_rows[i], device)
+    cache.set_lengths(lens)
+    return cache
+
+
+def random_cache(B, Hkv, lens, seed, d=128):
+    """An oracle cache with random rows of the given lengths [B*Hkv]."""
+    oc = orc.HybridCache(B, Hkv, d)
+    for i, L in enumerate(lens):
+        oc.k_rows.append(synth.bits(synth.randn_bf16((int(L), d), "cpu", seed, "k", i)))
+        oc.v_rows.append(synth.bits(synth.randn_bf16((int(L), d), "cpu", seed, "v", i)))
+    return oc
+
+
+def check_attention(out_f32, out_bf16, lse, ref, ref_lse, where=""):
+    """ref: oracle fp64 [.., d]; NaN rows of ref are skipped."""
+    ok = ~np.isnan(ref).any(axis=-1)
+    r = ref[ok]
+    if out_f32 is not None:
+        g = out_f32.detach().cpu().double().numpy()[ok]
+        assert rel_l2(g, r) <= REL_L2, (where, "fp32 rel-L2", rel_l2(g, r))
+        assert max_abs(g, r) <= MAX_ABS, (where, "fp32 max-abs", max_abs(g, r))
+    if out_bf16 is not None:
+        g = orc.bf16_to_f64(synth.bits(out_bf16))[ok]
+        rb = orc.bf16_to_f64(orc.f64_to_bf16(r))
+        assert rel_l2(g, rb) <= REL_L2, (where, "bf16 rel-L2", rel_l2(g, rb))
+        assert max_abs(g, rb) <= MAX_ABS, (where, "bf16 max-abs", max_abs(g, rb))
+    if lse is not None:
+        gl = lse.detach().cpu().double().numpy()[ok]
+        rl = ref_lse[ok]
+        fin = np.isfinite(rl)
+        assert np.array_equal(np.isfinite(gl), fin), where
+        assert np.all(np.abs(gl[fin] - rl[fin]) <= 1e-3), (where, "lse", np.abs(gl[fin] - rl[fin]).max())
+
+
+def check_indices_band(got_idx, C, n, S, Lc, T, mode, param, where=""):
+    """Band-aware comparison of a kept list with the oracle's selection.
+
+    The oracle's pooled scores P (fp64) define the k-th largest value P_k.  The list must be strictly
+    ascending, hold the sink and local tokens, have the oracle's length, contain every candidate with
+    P > P_k (1 + band) and nothing with P < P_k (1 - band).  Returns True when the oracle's gap around
+    the threshold is wide enough that the comparison was bit-exact.
+    """
+    want = orc.select_indices(C, n, S, Lc, T, mode, param)
+    got = np.asarray(got_idx, dtype=np.int64)
+    assert got.shape == want.shape, (where, got.shape, want.shape)
+    assert np.all(np.diff(got) > 0), where
+    if np.array_equal(got, want):
+        return True
+    assert T < n and S + Lc < n, where
+    cand_end = n - Lc
+    P = orc.pool_scores(C, S, cand_end, mode, param)
+    cs = param if mode == orc.POOL_CHUNK else 1
+    k_sel = max(0, T - S - Lc) // cs
+    order = np.sort(P)[::-1]
+    Pk = order[k_sel - 1]
+    assert list(got[:S]) == list(range(S)) and list(got[-Lc:]) == list(range(n - Lc, n)), where
+    mid = got[S:len(got) - Lc]
+    units = np.unique((mid - S) // cs)
+    must = np.nonzero(P > Pk * (1 + TIE_BAND))[0]
+    may = np.nonzero(P >= Pk * (1 - TIE_BAND))[0]
+    assert set(must.tolist()) <= set(units.tolist()), (where, "missing clear winners")
+    assert set(units.tolist()) <= set(may.tolist()), (where, "took a clear loser")
+    assert len(units) == k_sel, where
+    return False

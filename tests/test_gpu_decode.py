@@ -1,0 +1,126 @@
+"""GPU parity: catekv_append / catekv_decode_plan / catekv_decode_attn against the CPU oracle."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import catekv_oracle as orc
+from workloads import synth
+import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ck():
+    import paper_2608_30295_b200 as pkg
+    assert torch.cuda.is_available()
+    return pkg.binding
+
+
+def _run_decode(ck, oc, q_bits, num_ctas, max_new=0, scale=0.0):
+    cache = H.device_cache_from_oracle(ck, oc, max_new)
+    plan = ck.DecodePlan(cache, num_ctas)
+    ck.catekv_decode_plan(cache, plan)
+    q = synth.from_bits(q_bits, "cuda")
+    B, Hq, d = q.shape
+    o32 = torch.full((B, Hq, d), float("nan"), dtype=torch.float32, device="cuda")
+    o16 = torch.full((B, Hq, d), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device="cuda")
+    ck.catekv_decode_attn(cache, q, plan, o32, lse, sm_scale=scale)
+    ck.catekv_decode_attn(cache, q, plan, o16, None, sm_scale=scale)
+    torch.cuda.synchronize()
+    return cache, plan, o32, o16, lse
+
+
+@pytest.mark.parametrize("G", [1, 4, 7, 8])
+@pytest.mark.parametrize("num_ctas", [1, 5, 296])
+def test_decode_ragged_lengths(ck, G, num_ctas):
+    # odd lengths around the 16-row MMA block and the 64-row tile, an empty list, one long list
+    lens = [0, 1, 15, 16, 17, 63, 64, 65, 255, 257, 1000, 3]
+    B, Hkv = 3, 4
+    oc = H.random_cache(B, Hkv, lens, seed=100 + G)
+    q = synth.bits(synth.randn_bf16((B, Hkv * G, 128), "cpu", 200 + G, "q"))
+    ref, ref_lse = orc.decode_attention(oc, q)
+    _, _, o32, o16, lse = _run_decode(ck, oc, q, num_ctas)
+    H.check_attention(o32, o16, lse, ref, ref_lse, f"G={G} ctas={num_ctas}")
+    # the empty segment gives exact zeros and -inf
+    assert torch.all(o32[0, :G] == 0) and torch.all(torch.isinf(lse[0, :G]))
+    assert not torch.isnan(o32).any() and not torch.isnan(o16.float()).any()
+
+
+def test_decode_brute_force_one_head_64_tokens(ck):
+    oc = H.random_cache(1, 1, [64], seed=7)
+    q = synth.bits(synth.randn_bf16((1, 1, 128), "cpu", 7, "q1"))
+    ref, ref_lse = orc.decode_attention(oc, q)
+    for ctas in (1, 3):
+        _, _, o32, o16, lse = _run_decode(ck, oc, q, ctas)
+        H.check_attention(o32, o16, lse, ref, ref_lse)
+
+
+def test_decode_scale_and_peaked_softmax(ck):
+    # a large logit scale makes the softmax one-hot: exercises the running max
+    oc = H.random_cache(1, 2, [777, 130], seed=9)
+    q = synth.bits(synth.randn_bf16((1, 8, 128), "cpu", 9, "q"))
+    for scale in (1.0, 0.01):
+        ref, ref_lse = orc.decode_attention(oc, q, scale=scale)
+        _, _, o32, o16, lse = _run_decode(ck, oc, q, 11, scale=scale)
+        H.check_attention(o32, o16, lse, ref, ref_lse, f"scale={scale}")
+
+
+def test_decode_split_invariance(ck):
+    # the result may not depend on how the rows are cut into CTA ranges (up to fp32 merge rounding)
+    lens = [5000, 40, 2048, 911]
+    oc = H.random_cache(1, 4, lens, seed=11)
+    q = synth.bits(synth.randn_bf16((1, 16, 128), "cpu", 11, "q"))
+    outs = [_run_decode(ck, oc, q, n)[2].cpu().double().numpy() for n in (1, 2, 64, 500)]
+    for o in outs[1:]:
+        assert H.rel_l2(o, outs[0]) < 2e-6
+
+
+def test_append_then_decode_with_stale_plan(ck):
+    w = synth.scaled(synth.WORKLOADS["cfg0"], n=512, B=2)
+    lens = [100, 128, 1, 0, 300, 64, 17, 255]
+    oc = H.random_cache(2, 4, lens, seed=13)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=20)
+    plan = ck.DecodePlan(cache, 9)
+    ck.catekv_decode_plan(cache, plan)  # built once; the lists then grow under it
+    out = torch.empty((2, 16, 128), dtype=torch.float32, device="cuda")
+    for step in range(20):
+        kn = synth.randn_bf16((2, 4, 128), "cpu", 13, "kn", step)
+        vn = synth.randn_bf16((2, 4, 128), "cpu", 13, "vn", step)
+        q = synth.randn_bf16((2, 16, 128), "cpu", 13, "q", step)
+        ck.catekv_append(cache, kn.cuda(), vn.cuda())
+        oc.append(synth.bits(kn), synth.bits(vn))
+        ck.catekv_decode_attn(cache, q.cuda(), plan, out)
+        if step in (0, 1, 19):
+            ref, _ = orc.decode_attention(oc, synth.bits(q))
+            H.check_attention(out, None, None, ref, None, f"step {step}")
+    torch.cuda.synchronize()
+    assert list(cache.seg_len) == [l + 20 for l in lens]
+    assert cache.seg_len_dev.cpu().tolist() == [l + 20 for l in lens]
+    # pool bytes: the appended rows sit right after the old ones
+    for i in range(8):
+        o, L = int(cache.seg_off[i]), lens[i] + 20
+        assert np.array_equal(synth.bits(cache.k_pool[o:o + L]), oc.k_rows[i])
+        assert np.array_equal(synth.bits(cache.v_pool[o:o + L]), oc.v_rows[i])
+    # one more append overflows the 128-aligned capacity of some segment: refused, nothing changes
+    full = [i for i in range(8) if cache.seg_len[i] == cache.seg_cap[i]]
+    if not full:
+        while all(cache.seg_len[i] < cache.seg_cap[i] for i in range(8)):
+            ck.catekv_append(cache, kn.cuda(), vn.cuda())
+    before = cache.seg_len.copy()
+    with pytest.raises(ck.CatekvError) as e:
+        ck.catekv_append(cache, kn.cuda(), vn.cuda())
+    assert e.value.code == ck.ERR_CAPACITY
+    torch.cuda.synchronize()
+    assert np.array_equal(cache.seg_len, before) and cache.seg_len_dev.cpu().tolist() == before.tolist()
+
+
+def test_decode_is_deterministic(ck):
+    oc = H.random_cache(2, 4, [700, 64, 1500, 3, 90, 400, 2000, 128], seed=17)
+    q = synth.bits(synth.randn_bf16((2, 16, 128), "cpu", 17, "q"))
+    a = _run_decode(ck, oc, q, 40)
+    b = _run_decode(ck, oc, q, 40)
+    assert torch.equal(a[2], b[2]) and torch.equal(a[3], b[3]) and torch.equal(a[4], b[4])

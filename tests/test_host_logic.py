@@ -1,0 +1,197 @@
+"""CPU tests of the library's host side: exports, layout, plan, validation, classification.
+
+No kernel is launched: every call either is host-only or fails its argument checks first."""
+import ctypes as C
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import catekv_oracle as orc
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def ck():
+    from paper_2608_30295_b200 import build
+    build.build()
+    from paper_2608_30295_b200 import binding
+    return binding
+
+
+def test_library_exports_every_declared_symbol(ck):
+    hdr = open(os.path.join(ROOT, "include", "catekv.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(catekv_[a-z_0-9]+)\s*\(", hdr))
+    assert len(declared) >= 15
+    lib = C.CDLL(ck.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(ck.EXPORTS)
+    assert ck.catekv_version() == 1000
+    assert ck._lib.catekv_error_string(-3) == b"segment capacity exceeded"
+
+
+def test_cache_layout(ck):
+    off, cap, total = ck.catekv_cache_layout(2, 3, [0, 1, 127, 128, 129, 1000], 16)
+    assert list(cap) == [128, 128, 256, 256, 256, 1024]
+    assert list(off) == [0, 128, 256, 512, 768, 1024]
+    assert total == 2048
+    with pytest.raises(ck.CatekvError) as e:
+        ck.catekv_cache_layout(1, 2, [5, -1], 0)
+    assert e.value.code == ck.ERR_INVALID_ARG
+
+
+def _host_cache(ck, B, Hkv, lens, max_new=0):
+    off, cap, total = ck.catekv_cache_layout(B, Hkv, lens, max_new)
+    seg_len = np.array(lens, dtype=np.int32)
+    keep = (off, cap, seg_len)
+    fake = 0x10000  # non-null stand-ins for device pointers; nothing dereferences them in these tests
+    st = ck.CacheStruct(B, Hkv, 128, 0, total, fake, fake, fake, fake, off.ctypes.data, cap.ctypes.data,
+                        seg_len.ctypes.data)
+    return st, keep
+
+
+def _plan(ck, lens, B, Hkv, num_ctas):
+    st, keep = _host_cache(ck, B, Hkv, lens)
+    nbytes = ck._lib.catekv_decode_plan_bytes(B, Hkv, num_ctas)
+    buf = np.zeros(nbytes, dtype=np.uint8)
+    rc = ck._lib.catekv_decode_plan(C.byref(st), num_ctas, buf.ctypes.data, None, nbytes, None)
+    assert rc == 0
+    hdr = buf[:32].view(np.int32)
+    n_items, n_slots = int(hdr[3]), int(hdr[4])
+    off_cta = 32
+    off_items = (off_cta + 4 * (num_ctas + 1) + 15) // 16 * 16
+    off_seg = off_items + 16 * (num_ctas + B * Hkv)
+    cta = buf[off_cta:off_cta + 4 * (num_ctas + 1)].view(np.int32)
+    items = buf[off_items:off_items + 16 * n_items].view(np.int32).reshape(-1, 4)
+    segs = buf[off_seg:off_seg + 8 * B * Hkv].view(np.int32).reshape(-1, 2)
+    return cta, items, segs, n_slots
+
+
+@pytest.mark.parametrize("lens,num_ctas", [
+    ([1024, 1024, 32768, 32768, 1024, 32768, 1024, 32768], 296),
+    ([0, 5, 0, 17, 300, 1], 4),
+    ([100], 7),
+    ([0, 0], 3),
+    ([64, 64, 64, 64], 2),
+    (list(np.random.default_rng(5).integers(0, 5000, size=48)), 37),
+])
+def test_decode_plan_covers_every_row_once_and_balances(ck, lens, num_ctas):
+    lens = [int(x) for x in lens]
+    n = len(lens)
+    cta, items, segs, n_slots = _plan(ck, lens, 1, n, num_ctas)
+    assert cta[0] == 0 and np.all(np.diff(cta) >= 0) and cta[-1] == len(items)
+    # every segment's rows are covered exactly once, in order, by consecutive items
+    pos = {s: 0 for s in range(n)}
+    pieces = {s: [] for s in range(n)}
+    for i, (seg, t0, t1, slot) in enumerate(items):
+        assert t0 == pos[seg]
+        end = lens[seg] if t1 < 0 else t1
+        assert end > t0
+        pos[seg] = end
+        pieces[seg].append((i, t1, slot))
+    for s in range(n):
+        assert pos[s] == lens[s]
+        sb, npieces = segs[s]
+        assert npieces == len(pieces[s])
+        if npieces:
+            assert pieces[s][-1][1] == -1  # the last piece follows the live length
+            assert all(t1 >= 0 for (_, t1, _) in pieces[s][:-1])
+        if npieces == 1:
+            assert pieces[s][0][2] == -1
+        elif npieces > 1:
+            assert [sl for (_, _, sl) in pieces[s]] == list(range(sb, sb + npieces))
+    assert n_slots == sum(len(p) for p in pieces.values() if len(p) > 1)
+    # balance: no CTA gets more than an equal share rounded up to 16 rows
+    total = sum(lens)
+    quota = max(16, -(-(-(-total // num_ctas)) // 16) * 16)
+    for c in range(num_ctas):
+        rows = 0
+        for seg, t0, t1, _ in items[cta[c]:cta[c + 1]]:
+            rows += (lens[seg] if t1 < 0 else t1) - t0
+        assert rows <= quota
+
+
+def test_append_capacity_is_checked_before_launch(ck):
+    st, keep = _host_cache(ck, 1, 2, [128, 5], 0)  # segment 0 is exactly full
+    rc = ck._lib.catekv_append(C.byref(st), 0x10000, 0x10000, None)
+    assert rc == ck.ERR_CAPACITY
+    assert list(keep[2]) == [128, 5]  # host mirror untouched
+    assert ck._lib.catekv_append(C.byref(st), None, 0x10000, None) == ck.ERR_INVALID_ARG
+
+
+def test_decode_attn_argument_checks(ck):
+    st, keep = _host_cache(ck, 1, 2, [10, 10])
+    nbytes = ck._lib.catekv_decode_plan_bytes(1, 2, 4)
+    buf = np.zeros(nbytes, dtype=np.uint8)
+    assert ck._lib.catekv_decode_plan(C.byref(st), 4, buf.ctypes.data, None, nbytes, None) == 0
+    f = 0x10000
+    call = lambda **kw: ck._lib.catekv_decode_attn(
+        C.byref(st), kw.get("q", f), kw.get("Hq", 8), kw.get("scale", 0.0), f, kw.get("dt", 0), None,
+        kw.get("ph", buf.ctypes.data), f, kw.get("pb", nbytes), f, kw.get("wsb", 1 << 30), None)
+    assert call(q=None) == ck.ERR_INVALID_ARG
+    assert call(Hq=7) == ck.ERR_INVALID_ARG          # not a multiple of Hkv
+    assert call(Hq=18) == ck.ERR_UNSUPPORTED         # G = 9
+    assert call(dt=5) == ck.ERR_UNSUPPORTED
+    assert call(scale=-1.0) == ck.ERR_INVALID_ARG
+    assert call(wsb=16) == ck.ERR_WORKSPACE
+    assert call(pb=8) == ck.ERR_INVALID_ARG
+    junk = np.zeros(nbytes, dtype=np.uint8)
+    assert call(ph=junk.ctypes.data) == ck.ERR_INVALID_ARG   # not a plan
+    st2, keep2 = _host_cache(ck, 1, 2, [10, 10])
+    st2.d = 64
+    assert ck._lib.catekv_decode_plan(C.byref(st2), 4, buf.ctypes.data, None, nbytes, None) == ck.ERR_UNSUPPORTED
+    assert ck._lib.catekv_decode_plan(C.byref(st), 4, buf.ctypes.data, None, 8, None) == ck.ERR_WORKSPACE
+
+
+def test_select_argument_checks(ck):
+    st, keep = _host_cache(ck, 1, 2, [64, 200], 0)
+    seq = np.array([200], dtype=np.int32)
+    mask = np.array([1, 0], dtype=np.uint8)
+    f = 0x10000
+
+    def call(**kw):
+        p = ck.SelectParams(1, kw.get("Hq", 8), 2, kw.get("d", 128), kw.get("L_obs", 16), 4, kw.get("local", 16),
+                            kw.get("budget", 64), kw.get("eta", 1.0), kw.get("mode", 0), kw.get("param", 0), 0,
+                            f, f, f, 0, 0, 128, seq.ctypes.data, mask.ctypes.data)
+        return ck._lib.catekv_select_compact(C.byref(p), C.byref(st), None, 0, f, kw.get("wsb", 1 << 40), None)
+
+    assert call(local=8) == ck.ERR_INVALID_ARG       # local window shorter than the observation window
+    assert call(d=64) == ck.ERR_UNSUPPORTED
+    assert call(Hq=18) == ck.ERR_UNSUPPORTED
+    assert call(L_obs=65, local=65) == ck.ERR_UNSUPPORTED
+    assert call(mode=2, param=4) == ck.ERR_INVALID_ARG  # even window
+    assert call(mode=1, param=0) == ck.ERR_INVALID_ARG
+    assert call(mode=9) == ck.ERR_UNSUPPORTED
+    assert call(wsb=64) == ck.ERR_WORKSPACE
+    assert call(budget=150) == ck.ERR_CAPACITY       # 150 kept rows do not fit segment 0 (capacity 128)
+    assert list(keep[2]) == [64, 200]
+
+
+def test_head_cv_argument_checks(ck):
+    seq = np.array([100], dtype=np.int32)
+    f = 0x10000
+    call = lambda **kw: ck._lib.catekv_head_cv(f, f, 0, 0, 128, seq.ctypes.data, 1, kw.get("Hq", 8), 2, kw.get("d", 128),
+                                               kw.get("L_obs", 16), kw.get("L_init", 4), kw.get("L_rec", 4),
+                                               kw.get("k", 0.99), 1.0, 1, f, f, kw.get("wsb", 1 << 40), None)
+    assert call(d=64) == ck.ERR_UNSUPPORTED
+    assert call(k=1.5) == ck.ERR_INVALID_ARG
+    assert call(L_init=60, L_rec=40) == ck.ERR_INVALID_ARG   # no column left
+    assert call(L_obs=128) == ck.ERR_UNSUPPORTED
+    assert call(wsb=8) == ck.ERR_WORKSPACE
+    assert ck.catekv_head_cv_workspace_bytes(1, 8, 2, 100, 16, 60, 40) == 0
+
+
+def test_classify_heads_matches_oracle(ck):
+    rng = np.random.default_rng(30)
+    for N, H, r in [(8, 112, 0.5), (3, 4, 0.5), (5, 16, 0.4), (1, 7, 0.3), (4, 9, 0.0), (4, 9, 1.0)]:
+        cv = rng.random((N, H)).astype(np.float32)
+        want = orc.static_head_mask(cv.astype(np.float64), float(np.float32(r)))
+        got = ck.catekv_classify_heads(cv, r)
+        assert np.array_equal(got, want), (N, H, r)
+    cv = np.array([[9, 1, 8, 2], [9, 7, 1, 2], [9, 1, 8, 2]], dtype=np.float32)
+    assert list(ck.catekv_classify_heads(cv, 0.5)) == [1, 0, 1, 0]
