@@ -1,0 +1,484 @@
+#!/usr/bin/env python
+"""Benchmark of the CateKV hot path on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--workload cfg3] [--impl reference]
+
+A "step" is one decode step of the whole model on one batch: for every layer,
+catekv_append of the token's K/V followed by catekv_decode_attn over the hybrid
+per-head caches.  The caches are produced, before the timed region, by the
+library's own prefill-end path (catekv_select_compact over seeded synthetic
+prefill K/V, one layer at a time), which is timed and reported separately, as
+is catekv_head_cv.  `value` is decode throughput in tokens/s (batch tokens per
+step / step time) with everything resident in HBM; `e2e` repeats the
+measurement with the step's q / k_new / v_new coming from pinned host memory
+and the outputs copied back, inside the timed region.
+
+One JSON line is printed by rank 0.  With --gpus N > 1 (under torchrun) every
+rank runs an independent replica of the workload (the path has no exchange
+step); the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "hybrid decode attention throughput (tokens/s = batch / (layers x layer-step time))"
+UNIT = "tokens/s"
+ROW_BYTES = 512  # one kept token of one KV head: 256 B of K + 256 B of V
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi sampling in the background; started before and stopped after a timed region."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        try:
+            os.unlink(self.file.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------
+# building the model's caches through the library's prefill-end path
+# ------------------------------------------------------------------------------------------
+def expected_lengths(w, mask):
+    from workloads import synth  # noqa: F401
+    lens = []
+    for b in range(w.B):
+        for h in range(w.Hkv):
+            if mask[b, h]:
+                T = w.budget
+            else:
+                T = w.n if w.eta >= 1.0 else int(math.floor(float(np.float32(w.eta)) * w.n))
+            lens.append(w.n if (T >= w.n or w.sink + w.local >= w.n) else max(T, w.sink + w.local))
+    return lens
+
+
+def build_model(ck, w, dev, max_new, layers=None, time_select=True):
+    """Caches and plans of `layers` layers via catekv_select_compact.  Returns (layer list, select ms/layer)."""
+    import torch
+    from workloads import synth
+    n_layers = w.layers if layers is None else layers
+    num_ctas = ck.catekv_decode_num_ctas()
+    out, sel_ms = [], []
+    ws = torch.empty(ck.catekv_select_workspace_bytes(w.B, w.Hq, w.Hkv, w.n, w.L_obs), dtype=torch.uint8, device=dev)
+    for l in range(n_layers):
+        p = synth.prefill_layer(w, l, dev)
+        mask = p["head_mask"]
+        cache = ck.Cache(w.B, w.Hkv, expected_lengths(w, mask), max_new, dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        ck.catekv_select_compact(p["q_win"], p["k"], p["v"], p["seq_len"], mask, cache, w.budget, w.eta, w.sink,
+                                 w.local, w.pool_mode, w.pool_param, ws=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        sel_ms.append(e0.elapsed_time(e1))
+        plan = ck.DecodePlan(cache, num_ctas)
+        ck.catekv_decode_plan(cache, plan)
+        out.append({"cache": cache, "plan": plan, "mask": mask})
+        del p
+    torch.cuda.synchronize()
+    return out, sel_ms
+
+
+def make_step_inputs(w, n_layers, dev, n_sets=2):
+    """A few sets of per-step inputs for all layers: q [L,B,Hq,d], k_new, v_new [L,B,Hkv,d]."""
+    import torch
+    from workloads import synth
+    sets = []
+    for s in range(n_sets):
+        q = synth.randn_bf16((n_layers, w.B, w.Hq, w.d), dev, w.seed, "bench_q", s)
+        kn = synth.randn_bf16((n_layers, w.B, w.Hkv, w.d), dev, w.seed, "bench_kn", s)
+        vn = synth.randn_bf16((n_layers, w.B, w.Hkv, w.d), dev, w.seed, "bench_vn", s)
+        sets.append((q, kn, vn))
+    return sets
+
+
+def decode_step(ck, model, q, kn, vn, out):
+    for l, m in enumerate(model):
+        ck.catekv_append(m["cache"], kn[l], vn[l])
+        ck.catekv_decode_attn(m["cache"], q[l], m["plan"], out[l])
+
+
+def kept_bytes(model):
+    return [int(m["cache"].seg_len.sum()) * ROW_BYTES for m in model]
+
+
+def time_decode(ck, w, model, dev, steps, warmup, barrier=None):
+    """Device-resident timing: returns ms per step (CUDA events on the launching stream)."""
+    import torch
+    L = len(model)
+    sets = make_step_inputs(w, L, dev)
+    out = torch.empty((L, w.B, w.Hq, w.d), dtype=torch.bfloat16, device=dev)
+    for i in range(warmup):
+        decode_step(ck, model, *sets[i % len(sets)], out)
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        decode_step(ck, model, *sets[i % len(sets)], out)
+    e1.record()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    return e0.elapsed_time(e1) / steps
+
+
+def time_kernels(ck, w, model, dev, steps):
+    """Per-kernel durations over the same steps: events around the partials kernel of every launch."""
+    import torch
+    L = len(model)
+    sets = make_step_inputs(w, L, dev)
+    out = torch.empty((L, w.B, w.Hq, w.d), dtype=torch.bfloat16, device=dev)
+    ev = []
+    for i in range(steps):
+        q, kn, vn = sets[i % len(sets)]
+        for l, m in enumerate(model):
+            ck.catekv_append(m["cache"], kn[l], vn[l])
+            a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            a.record()
+            ck.catekv_decode_partials(m["cache"], q[l], m["plan"], out[l])
+            b.record()
+            ck.catekv_decode_combine(m["cache"], q[l], m["plan"], out[l])
+            c.record()
+            ev.append((a, b, c))
+    torch.cuda.synchronize()
+    part = [a.elapsed_time(b) * 1e3 for a, b, _ in ev]
+    comb = [b.elapsed_time(c) * 1e3 for _, b, c in ev]
+    return float(np.mean(part)), float(np.median(part)), float(np.mean(comb))
+
+
+def time_e2e(ck, w, model, dev, steps, warmup, barrier=None):
+    """Same step through the public API with host buffers: H2D of q/k_new/v_new and D2H of the outputs inside
+    the timed region."""
+    import torch
+    L = len(model)
+    host_sets = []
+    for q, kn, vn in make_step_inputs(w, L, "cpu"):
+        host_sets.append((q.pin_memory(), kn.pin_memory(), vn.pin_memory()))
+    dq = torch.empty((L, w.B, w.Hq, w.d), dtype=torch.bfloat16, device=dev)
+    dk = torch.empty((L, w.B, w.Hkv, w.d), dtype=torch.bfloat16, device=dev)
+    dv = torch.empty_like(dk)
+    out = torch.empty_like(dq)
+    hout = torch.empty((L, w.B, w.Hq, w.d), dtype=torch.bfloat16).pin_memory()
+
+    def step(i):
+        q, kn, vn = host_sets[i % len(host_sets)]
+        dq.copy_(q, non_blocking=True)
+        dk.copy_(kn, non_blocking=True)
+        dv.copy_(vn, non_blocking=True)
+        decode_step(ck, model, dq, dk, dv, out)
+        hout.copy_(out, non_blocking=True)
+        torch.cuda.current_stream().synchronize()  # the caller needs the outputs before the next token
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    h2d = sum(t.numel() * t.element_size() for t in host_sets[0])
+    d2h = hout.numel() * hout.element_size()
+    return e0.elapsed_time(e1) / steps, h2d, d2h
+
+
+def time_head_cv(ck, dev):
+    """catekv_head_cv on configs[4]'s calibration shape: 8 prompts x 16K tokens, one layer (4 KV heads, G = 7)."""
+    import torch
+    from workloads import synth
+    w = synth.WORKLOADS["cfg4"]
+    n = 16384
+    qs, ks = [], []
+    types = np.array([1, 0, 1, 0], dtype=np.uint8)
+    for pr in range(8):
+        q, k = synth.calibration_prompt(w, 0, pr, n, types, dev)
+        qs.append(q), ks.append(k)
+    q, k = torch.cat(qs), torch.cat(ks)
+    seq = [n] * 8
+    ws = torch.empty(ck.catekv_head_cv_workspace_bytes(8, w.Hq, w.Hkv, n, w.L_obs, 128, 32), dtype=torch.uint8,
+                     device=dev)
+    for _ in range(2):
+        ck.catekv_head_cv(q, k, seq, 128, 32, 0.99, 1.0, True, ws=ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(3):
+        ck.catekv_head_cv(q, k, seq, 128, 32, 0.99, 1.0, True, ws=ws)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / 3
+
+
+# ------------------------------------------------------------------------------------------
+# the oracle, timed as it stands, on a bounded sample
+# ------------------------------------------------------------------------------------------
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return int(max(n)) if n else 1
+    except Exception:
+        return 1
+
+
+def oracle_sample_rate(w, target_s=15.0, seed_rows=200_000):
+    """Times oracle.decode_attention on synthetic segments; returns (rows per second, sample description,
+    seconds spent).  The sample grows until about target_s seconds of CPU work have been done."""
+    from oracle import catekv_oracle as orc
+    from workloads import synth
+    G = w.G
+    rows_done, t_done = 0, 0.0
+    seg_rows = min(w.n, 65536)
+    i = 0
+    while True:
+        oc = orc.HybridCache(1, 1, w.d)
+        oc.k_rows.append(synth.bits(synth.randn_bf16((seg_rows, w.d), "cpu", w.seed, "ok", i)))
+        oc.v_rows.append(synth.bits(synth.randn_bf16((seg_rows, w.d), "cpu", w.seed, "ov", i)))
+        q = synth.bits(synth.randn_bf16((1, G, w.d), "cpu", w.seed, "oq", i))
+        t0 = time.perf_counter()
+        orc.decode_attention(oc, q)
+        t_done += time.perf_counter() - t0
+        rows_done += seg_rows
+        i += 1
+        if t_done >= target_s or i >= 400:
+            break
+    desc = f"{i} segments of {seg_rows} rows x {G} query heads (one KV head each), oracle.decode_attention"
+    return rows_done / t_done, desc, t_done
+
+
+def workload_rows_per_layer_step(w):
+    """Expected kept rows of one layer-step (mean over the seeded masks of all layers)."""
+    from workloads import synth
+    tot = 0
+    for l in range(w.layers):
+        tot += sum(expected_lengths(w, synth.head_mask(w, l)))
+    return tot / w.layers
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the same metric; each step is a bounded sample, extrapolated."""
+    from workloads import synth
+    w = synth.WORKLOADS[args.workload]
+    rows = workload_rows_per_layer_step(w)
+    vals = []
+    per = 4.0 if args.steps > 3 else 10.0
+    for i in range(args.warmup + args.steps):
+        rate, desc, spent = oracle_sample_rate(w, target_s=per if i >= args.warmup else 1.0)
+        if i >= args.warmup:
+            vals.append(rate)
+    rate = float(np.mean(vals))
+    t_layer = rows / rate
+    value = w.B / (w.layers * t_layer)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": w.layers * t_layer * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "note": "CPU oracle (numpy fp64) timed on a bounded sample and extrapolated "
+                   "by rows; not the target"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                         "sample": desc + f", {rate:.3e} rows/s"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg3", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the other configs, head_cv and the oracle timing")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2608_30295_b200 as pkg
+    ck = pkg.binding
+    from workloads import synth
+
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    barrier = None
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+        barrier = lambda: dist.barrier()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    peaks, peak_src = measured_peaks()
+    w = synth.WORKLOADS[args.workload]
+    n_layers = args.layers or w.layers
+    total_steps = 3 * (args.warmup + args.steps) + 8
+    model, sel_ms = build_model(ck, w, dev, max_new=total_steps, layers=n_layers)
+
+    vis = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
+    sampler = ClockSampler(vis[local_rank] if local_rank < len(vis) else local_rank)
+    sampler.start()
+    ms = max_over_ranks(time_decode(ck, w, model, dev, args.steps, args.warmup, barrier))
+    clocks = sampler.stop()
+    bytes_per_layer = float(np.mean(kept_bytes(model)))
+    part_us, part_med_us, comb_us = time_kernels(ck, w, model, dev, max(2, min(args.steps, 5)))
+    ms_e2e, h2d, d2h = time_e2e(ck, w, model, dev, args.steps, args.warmup, barrier)
+    ms_e2e = max_over_ranks(ms_e2e)
+
+    scale_layers = w.layers / n_layers  # only != 1 when --layers is used for profiling
+    value = world * w.B / (ms * scale_layers * 1e-3)
+    e2e_value = world * w.B / (ms_e2e * scale_layers * 1e-3)
+    achieved = bytes_per_layer / (part_us * 1e-6) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": w.name, "layers": n_layers, "batch": w.B, "context": w.n, "q_heads": w.Hq,
+                   "kv_heads": w.Hkv, "head_dim": w.d, "budget_consistent": w.budget, "eta_adaptive": w.eta,
+                   "window": w.L_obs, "replicas": world,
+                   "l2": "no flush: per-layer working set %.0f MB x %d layers, far above the 126 MB L2"
+                         % (bytes_per_layer / 1e6, n_layers),
+                   "step": "one decode token of the whole model: per layer catekv_append + catekv_decode_attn"},
+        "us_per_layer_step": ms * 1e3 / n_layers,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src, "traffic": None,
+                     "kernel": "decode_partial_kernel", "bytes_per_launch": bytes_per_layer,
+                     "us_per_launch": part_us, "us_per_launch_median": part_med_us,
+                     "frac_of_8TBs": achieved / 8000.0, "combine_us": comb_us},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": ms_e2e},
+        "gpu_launches": args.steps * n_layers * (2 + (1 if any(ck.plan_header(m["plan"])["n_slots"] for m in model) else 0)),
+        "clocks": clocks,
+        "select_compact": {"ms_per_layer": float(np.mean(sel_ms[1:] or sel_ms)), "layers": n_layers},
+    }
+    del model
+    torch.cuda.empty_cache()
+
+    if rank == 0 and not args.no_extras:
+        # the other configurations, decode only, a few layers each (parity-test cases, reported for context)
+        table = {}
+        for name in ("cfg1", "cfg2", "cfg4"):
+            if name == w.name:
+                continue
+            wo = synth.WORKLOADS[name]
+            nl = min(wo.layers, 8)
+            mo, so = build_model(ck, wo, dev, max_new=64, layers=nl)
+            t = time_decode(ck, wo, mo, dev, 10, 3)
+            pu, pm, cu = time_kernels(ck, wo, mo, dev, 3)
+            by = float(np.mean(kept_bytes(mo)))
+            table[name] = {"layers_timed": nl, "us_per_layer_step": t * 1e3 / nl, "partials_us": pu,
+                           "bytes_per_layer_step": by, "hbm_gbs": by / (pu * 1e-6) / 1e9,
+                           "frac_of_measured": by / (pu * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                           "select_ms_per_layer": float(np.mean(so[1:] or so))}
+            del mo
+            torch.cuda.empty_cache()
+        line["other_configs"] = table
+        line["head_cv"] = {"ms": time_head_cv(ck, dev), "shape": "8 prompts x 16384 tokens, 28q/4kv, window 64"}
+        rate, desc, spent = oracle_sample_rate(w, target_s=15.0)
+        rows = bytes_per_layer / ROW_BYTES
+        line["cpu_baseline"] = {"value": w.B / (w.layers * rows / rate), "unit": UNIT, "cores": oracle_threads(),
+                                "kind": "oracle", "sample": desc + f" ({spent:.1f} s, {rate:.3e} rows/s), "
+                                "extrapolated by rows to the full step"}
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -218,6 +218,20 @@ int catekv_decode_attn(const catekv_cache* cache, const void* q, int32_t Hq, flo
                        int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                        size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream);
 
+/*
+ * The two phases of catekv_decode_attn as separate calls, with the same arguments: the split-KV
+ * attention partials (every CTA range of the plan: online softmax over its rows; a segment that
+ * fits one range is written to `out` directly) and the combine pass (log-sum-exp merge of the
+ * partials of every segment that was cut).  catekv_decode_attn is exactly partials then combine
+ * on one stream; the split exists so that a caller can time or overlap the phases.
+ */
+int catekv_decode_partials(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
+                           int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
+                           size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream);
+int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
+                          int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
+                          size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -72,6 +72,8 @@ def _load():
         "catekv_decode_workspace_bytes": (sz, [i32, i32, i32]),
         "catekv_decode_plan": (C.c_int, [C.POINTER(CacheStruct), i32, vp, vp, sz, vp]),
         "catekv_decode_attn": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
+        "catekv_decode_partials": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
+        "catekv_decode_combine": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -176,8 +178,7 @@ def plan_header(plan: DecodePlan) -> dict:
             "tile": int(h[5]), "total_rows": int(plan.host[24:32].numpy().view(np.int64)[0])}
 
 
-def catekv_decode_attn(cache: Cache, q: torch.Tensor, plan: DecodePlan, out: torch.Tensor,
-                       lse_out: Optional[torch.Tensor] = None, sm_scale: float = 0.0):
+def _decode_call(fn, name, cache, q, plan, out, lse_out, sm_scale):
     assert q.is_contiguous() and out.is_contiguous() and q.dtype == torch.bfloat16
     Hq = q.shape[1]
     if out.dtype == torch.bfloat16:
@@ -186,9 +187,23 @@ def catekv_decode_attn(cache: Cache, q: torch.Tensor, plan: DecodePlan, out: tor
         od = OUT_FP32
     else:
         raise TypeError("out must be bf16 or fp32")
-    _check(_lib.catekv_decode_attn(C.byref(cache.struct), q.data_ptr(), Hq, sm_scale, out.data_ptr(), od,
-                                   _dev_ptr(lse_out), plan.host.data_ptr(), plan.dev.data_ptr(), plan.bytes,
-                                   plan.ws.data_ptr(), plan.ws_bytes, _stream()), "catekv_decode_attn")
+    _check(fn(C.byref(cache.struct), q.data_ptr(), Hq, sm_scale, out.data_ptr(), od, _dev_ptr(lse_out),
+              plan.host.data_ptr(), plan.dev.data_ptr(), plan.bytes, plan.ws.data_ptr(), plan.ws_bytes, _stream()), name)
+
+
+def catekv_decode_attn(cache: Cache, q: torch.Tensor, plan: DecodePlan, out: torch.Tensor,
+                       lse_out: Optional[torch.Tensor] = None, sm_scale: float = 0.0):
+    _decode_call(_lib.catekv_decode_attn, "catekv_decode_attn", cache, q, plan, out, lse_out, sm_scale)
+
+
+def catekv_decode_partials(cache: Cache, q: torch.Tensor, plan: DecodePlan, out: torch.Tensor,
+                           lse_out: Optional[torch.Tensor] = None, sm_scale: float = 0.0):
+    _decode_call(_lib.catekv_decode_partials, "catekv_decode_partials", cache, q, plan, out, lse_out, sm_scale)
+
+
+def catekv_decode_combine(cache: Cache, q: torch.Tensor, plan: DecodePlan, out: torch.Tensor,
+                          lse_out: Optional[torch.Tensor] = None, sm_scale: float = 0.0):
+    _decode_call(_lib.catekv_decode_combine, "catekv_decode_combine", cache, q, plan, out, lse_out, sm_scale)
 
 
 def catekv_select_workspace_bytes(B, Hq, Hkv, n_max, L_obs) -> int:

@@ -483,13 +483,21 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
   int n_items = 0, n_slots = 0;
   int seg = 0;
   int32_t pos = 0;  // next unassigned row of `seg`
-  while (seg < n_segs && cache->seg_len[seg] == 0) { segs[seg] = SegInfo{0, 0}; ++seg; }
-  int seg_first_item = n_items;
+  int seg_first_item = 0;
   for (int c = 0; c < num_ctas; ++c) {
     cta_begin[c] = n_items;
     int64_t room = quota;
-    while (room > 0 && seg < n_segs) {
+    while (seg < n_segs) {
       const int32_t len = cache->seg_len[seg];
+      if (len == 0) {
+        // an empty segment still gets one (direct) item, so that the plan stays valid once it grows
+        items[n_items++] = WorkItem{seg, 0, -1, -1};
+        segs[seg] = SegInfo{0, 1};
+        ++seg;
+        seg_first_item = n_items;
+        continue;
+      }
+      if (room <= 0) break;
       const int32_t take = (int32_t)((int64_t)(len - pos) < room ? (len - pos) : room);
       items[n_items++] = WorkItem{seg, pos, pos + take, 0};
       pos += take;
@@ -508,7 +516,6 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
         }
         ++seg;
         pos = 0;
-        while (seg < n_segs && cache->seg_len[seg] == 0) { segs[seg] = SegInfo{0, 0}; ++seg; }
         seg_first_item = n_items;
       }
     }
@@ -527,9 +534,10 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
   return CATEKV_OK;
 }
 
-extern "C" int catekv_decode_attn(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
-                                  int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
-                                  size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+// phases: 1 = attention partials, 2 = combine, 3 = both
+static int decode_launch(int phases, const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
+                         int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
+                         size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
   int rc = check_cache(cache);
   if (rc) return rc;
   if (!q || !out || !plan_host || !plan_dev || !ws) return CATEKV_ERR_INVALID_ARG;
@@ -548,47 +556,73 @@ extern "C" int catekv_decode_attn(const catekv_cache* cache, const void* q, int3
   size_t off_lse = 0;
   if (ws_bytes < ws_layout(n_segs, hdr->num_ctas, &off_lse)) return CATEKV_ERR_WORKSPACE;
 
-  static bool attr_set[64] = {};
-  int dev = 0;
-  CATEKV_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
-    if (dev >= 0 && dev < 64) attr_set[dev] = true;
-  }
   const uint8_t* pd = (const uint8_t*)plan_dev;
-  DecodeArgs a;
-  a.k_pool = (const uint8_t*)cache->k_pool;
-  a.v_pool = (const uint8_t*)cache->v_pool;
-  a.seg_off = cache->seg_off_dev;
-  a.seg_len = cache->seg_len_dev;
-  a.q = (const uint16_t*)q;
-  a.Hq = Hq;
-  a.Hkv = cache->Hkv;
-  a.G = G;
-  a.scale_log2 = (sm_scale == 0.f ? 1.0f / sqrtf((float)kD) : sm_scale) * 1.4426950408889634f;
-  a.cta_item_begin = (const int32_t*)(pd + L.off_cta);
-  a.items = (const WorkItem*)(pd + L.off_items);
-  a.part_o = (float*)ws;
-  a.part_lse = (float*)((uint8_t*)ws + off_lse);
-  a.out = out;
-  a.out_fp32 = out_dtype == CATEKV_OUT_FP32;
-  a.lse_out = lse_out;
   cudaStream_t st = (cudaStream_t)stream;
-  if (hdr->n_items > 0) {
+  float* part_o = (float*)ws;
+  float* part_lse = (float*)((uint8_t*)ws + off_lse);
+  const int out_fp32 = out_dtype == CATEKV_OUT_FP32;
+  if ((phases & 1) && hdr->n_items > 0) {
+    static bool attr_set[64] = {};
+    int dev = 0;
+    CATEKV_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+      CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
+      if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    DecodeArgs a;
+    a.k_pool = (const uint8_t*)cache->k_pool;
+    a.v_pool = (const uint8_t*)cache->v_pool;
+    a.seg_off = cache->seg_off_dev;
+    a.seg_len = cache->seg_len_dev;
+    a.q = (const uint16_t*)q;
+    a.Hq = Hq;
+    a.Hkv = cache->Hkv;
+    a.G = G;
+    a.scale_log2 = (sm_scale == 0.f ? 1.0f / sqrtf((float)kD) : sm_scale) * 1.4426950408889634f;
+    a.cta_item_begin = (const int32_t*)(pd + L.off_cta);
+    a.items = (const WorkItem*)(pd + L.off_items);
+    a.part_o = part_o;
+    a.part_lse = part_lse;
+    a.out = out;
+    a.out_fp32 = out_fp32;
+    a.lse_out = lse_out;
     decode_partial_kernel<<<hdr->num_ctas, kDecodeThreads, kDecodeSmem, st>>>(a);
     CATEKV_CUDA_TRY(cudaGetLastError());
   }
-  CombineArgs ca;
-  ca.seg_info = (const SegInfo*)(pd + L.off_seg);
-  ca.part_o = a.part_o;
-  ca.part_lse = a.part_lse;
-  ca.out = out;
-  ca.lse_out = lse_out;
-  ca.Hq = Hq;
-  ca.Hkv = cache->Hkv;
-  ca.G = G;
-  ca.out_fp32 = a.out_fp32;
-  decode_combine_kernel<<<dim3(n_segs, G), kD, 0, st>>>(ca);
-  CATEKV_CUDA_TRY(cudaGetLastError());
+  if ((phases & 2) && hdr->n_slots > 0) {
+    CombineArgs ca;
+    ca.seg_info = (const SegInfo*)(pd + L.off_seg);
+    ca.part_o = part_o;
+    ca.part_lse = part_lse;
+    ca.out = out;
+    ca.lse_out = lse_out;
+    ca.Hq = Hq;
+    ca.Hkv = cache->Hkv;
+    ca.G = G;
+    ca.out_fp32 = out_fp32;
+    decode_combine_kernel<<<dim3(n_segs, G), kD, 0, st>>>(ca);
+    CATEKV_CUDA_TRY(cudaGetLastError());
+  }
   return CATEKV_OK;
+}
+
+extern "C" int catekv_decode_attn(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
+                                  int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
+                                  size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+  return decode_launch(3, cache, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
+                       ws_bytes, stream);
+}
+
+extern "C" int catekv_decode_partials(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
+                                      int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
+                                      size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+  return decode_launch(1, cache, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
+                       ws_bytes, stream);
+}
+
+extern "C" int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
+                                     int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
+                                     size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+  return decode_launch(2, cache, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
+                       ws_bytes, stream);
 }
