@@ -232,6 +232,36 @@ int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, 
                           int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                           size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream);
 
+/*
+ * catekv_decode_attn for callers that cannot hand over scratch memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, same arithmetic, same results.)
+ *
+ * Who needs it: hosts that take all of the GPU's memory for themselves at start-up and give a
+ * plugin no allocator afterwards (an inference server with a pre-sized arena, a sandboxed
+ * extension), and code on a request path where an allocation would stall the whole device
+ * (cudaMalloc and cudaFree synchronise it) or fail because nothing is left.  Such callers still
+ * own the inputs, the cache, the plan and `out`; what they lack is a place for the split-KV
+ * partials.  Here those live in a fixed array of CATEKV_NOALLOC_SCRATCH_BYTES (4 MiB) that is
+ * part of the library image: every GPU that loads the library carries it until the process
+ * exits, whether or not this function is ever called.
+ *
+ * The call allocates and frees nothing, on the device or through any library.  Its arguments are
+ * those of catekv_decode_attn minus ws / ws_bytes.  A plan whose partials do not fit
+ * - (num_ctas + B*Hkv) * 4128 bytes > CATEKV_NOALLOC_SCRATCH_BYTES, i.e. more than 1016 slots -
+ * is refused with CATEKV_ERR_WORKSPACE before anything is launched; build the plan with fewer
+ * CTAs or use catekv_decode_attn.
+ *
+ * The first call on a device looks up the array's device address (with that device current) and
+ * keeps it; make that first call outside any stream capture.  All calls of a process share the
+ * one array per GPU: nothing in it has to start at zero and it keeps whatever the last call left,
+ * but two calls whose kernels overlap on the same GPU (different streams, or different threads)
+ * would overwrite each other's partials - keep them on one stream or otherwise ordered.
+ */
+#define CATEKV_NOALLOC_SCRATCH_BYTES (4u << 20)
+int catekv_decode_attn_noalloc(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
+                               int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
+                               size_t plan_bytes, catekv_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

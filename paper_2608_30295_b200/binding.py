@@ -74,6 +74,7 @@ def _load():
         "catekv_decode_attn": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
         "catekv_decode_partials": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
         "catekv_decode_combine": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
+        "catekv_decode_attn_noalloc": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -204,6 +205,27 @@ def catekv_decode_partials(cache: Cache, q: torch.Tensor, plan: DecodePlan, out:
 def catekv_decode_combine(cache: Cache, q: torch.Tensor, plan: DecodePlan, out: torch.Tensor,
                           lse_out: Optional[torch.Tensor] = None, sm_scale: float = 0.0):
     _decode_call(_lib.catekv_decode_combine, "catekv_decode_combine", cache, q, plan, out, lse_out, sm_scale)
+
+
+NOALLOC_SCRATCH_BYTES = 4 << 20
+
+
+def catekv_decode_attn_noalloc(cache: Cache, q: torch.Tensor, plan: DecodePlan, out: torch.Tensor,
+                               lse_out: Optional[torch.Tensor] = None, sm_scale: float = 0.0):
+    """catekv_decode_attn with the partials in the library's own fixed 4 MiB array instead of plan.ws: for
+    callers that may not allocate device memory (a host that owns the whole GPU arena, or a request path that
+    cannot afford cudaMalloc's device-wide synchronisation).  Nothing is allocated by this call; plans with
+    more than 1016 partial slots are refused (ERR_WORKSPACE).  Calls share the array: keep them ordered."""
+    assert q.is_contiguous() and out.is_contiguous() and q.dtype == torch.bfloat16
+    if out.dtype == torch.bfloat16:
+        od = OUT_BF16
+    elif out.dtype == torch.float32:
+        od = OUT_FP32
+    else:
+        raise TypeError("out must be bf16 or fp32")
+    _check(_lib.catekv_decode_attn_noalloc(C.byref(cache.struct), q.data_ptr(), q.shape[1], sm_scale,
+                                           out.data_ptr(), od, _dev_ptr(lse_out), plan.host.data_ptr(),
+                                           plan.dev.data_ptr(), plan.bytes, _stream()), "catekv_decode_attn_noalloc")
 
 
 def catekv_select_workspace_bytes(B, Hq, Hkv, n_max, L_obs) -> int:

@@ -626,3 +626,31 @@ extern "C" int catekv_decode_combine(const catekv_cache* cache, const void* q, i
   return decode_launch(2, cache, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
                        ws_bytes, stream);
 }
+
+// ------------------------------------------------------------------------------------------
+// Decode attention without caller-provided scratch
+// ------------------------------------------------------------------------------------------
+// The split-KV partials of this variant live in a fixed array inside the library image instead of
+// a caller workspace.  In host code the array's name only stands for the symbol; the address the
+// kernels need is looked up once per device.
+static __device__ __align__(256) unsigned char g_decode_noalloc_scratch[CATEKV_NOALLOC_SCRATCH_BYTES];
+
+extern "C" int catekv_decode_attn_noalloc(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale,
+                                          void* out, int32_t out_dtype, float* lse_out, const void* plan_host,
+                                          const void* plan_dev, size_t plan_bytes, catekv_stream stream) {
+  static void* scratch_of_device[64] = {};
+  int dev = 0;
+  CATEKV_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return CATEKV_ERR_UNSUPPORTED;
+  if (!scratch_of_device[dev]) {
+    // first call on this device (which is current): resolve the device address of the array
+    void* p = nullptr;
+    CATEKV_CUDA_TRY(cudaGetSymbolAddress(&p, g_decode_noalloc_scratch));
+    if (!p) return CATEKV_ERR_CUDA;
+    scratch_of_device[dev] = p;
+  }
+  // decode_launch checks the plan and returns CATEKV_ERR_WORKSPACE when the partials of this plan
+  // (num_ctas + B*Hkv slots) do not fit the fixed array
+  return decode_launch(3, cache, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes,
+                       scratch_of_device[dev], (size_t)CATEKV_NOALLOC_SCRATCH_BYTES, stream);
+}
