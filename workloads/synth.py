@@ -95,13 +95,15 @@ def randn_bf16(shape, device, *parts) -> torch.Tensor:
 
 def head_mask(w: Workload, layer: int) -> np.ndarray:
     """[B, Hkv] uint8, 1 = consistent.  The share of consistent heads of a
-    sequence is drawn in [consistent_lo, consistent_hi]; which heads is a
-    seeded permutation."""
+    sequence is drawn in [consistent_lo, consistent_hi]; share * Hkv is rounded
+    stochastically to a head count (so the share holds on average over
+    layers); which heads is a seeded permutation."""
     rng = _rng(w.seed, "mask", layer)
     m = np.zeros((w.B, w.Hkv), dtype=np.uint8)
     for b in range(w.B):
         frac = w.consistent_lo + (w.consistent_hi - w.consistent_lo) * rng.random()
-        cnt = int(round(frac * w.Hkv))
+        x = frac * w.Hkv
+        cnt = int(math.floor(x)) + (1 if rng.random() < x - math.floor(x) else 0)
         m[b, rng.permutation(w.Hkv)[:cnt]] = 1
     return m
 
