@@ -168,25 +168,58 @@ def decode_step(ck, model, q, kn, vn, out):
         ck.catekv_decode_attn(m["cache"], q[l], m["plan"], out[l])
 
 
+def capture_step(ck, model, q, kn, vn, out):
+    """One decode step of the whole model as a CUDA graph.  Capturing runs the library's host code (which
+    advances the host length mirrors) but not the kernels, so the graph is replayed once right away; every
+    later replay is preceded by catekv_cache_advance."""
+    import torch
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            decode_step(ck, model, q, kn, vn, out)
+    torch.cuda.current_stream().wait_stream(s)
+    g.replay()
+    return g
+
+
+def replay_step(ck, model, g):
+    for m in model:
+        ck.catekv_cache_advance(m["cache"], 1)
+    g.replay()
+
+
 def kept_bytes(model):
     return [int(m["cache"].seg_len.sum()) * ROW_BYTES for m in model]
 
 
-def time_decode(ck, w, model, dev, steps, warmup, barrier=None):
-    """Device-resident timing: returns ms per step (CUDA events on the launching stream)."""
+def time_decode(ck, w, model, dev, steps, warmup, barrier=None, graph=True):
+    """Device-resident timing: returns ms per step (CUDA events on the launching stream).  With `graph` the
+    step's launches are captured once per input set and replayed."""
     import torch
     L = len(model)
     sets = make_step_inputs(w, L, dev)
     out = torch.empty((L, w.B, w.Hq, w.d), dtype=torch.bfloat16, device=dev)
+    decode_step(ck, model, *sets[0], out)  # first launch of every kernel happens outside any capture
+    torch.cuda.synchronize()
+    graphs = [capture_step(ck, model, *st, out) for st in sets] if graph else None
+
+    def step(i):
+        if graph:
+            replay_step(ck, model, graphs[i % len(graphs)])
+        else:
+            decode_step(ck, model, *sets[i % len(sets)], out)
+
     for i in range(warmup):
-        decode_step(ck, model, *sets[i % len(sets)], out)
+        step(i)
     torch.cuda.synchronize()
     if barrier:
         barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(steps):
-        decode_step(ck, model, *sets[i % len(sets)], out)
+        step(i)
     e1.record()
     torch.cuda.synchronize()
     if barrier:
@@ -218,7 +251,7 @@ def time_kernels(ck, w, model, dev, steps):
     return float(np.mean(part)), float(np.median(part)), float(np.mean(comb))
 
 
-def time_e2e(ck, w, model, dev, steps, warmup, barrier=None):
+def time_e2e(ck, w, model, dev, steps, warmup, barrier=None, graph=True):
     """Same step through the public API with host buffers: H2D of q/k_new/v_new and D2H of the outputs inside
     the timed region."""
     import torch
@@ -232,12 +265,19 @@ def time_e2e(ck, w, model, dev, steps, warmup, barrier=None):
     out = torch.empty_like(dq)
     hout = torch.empty((L, w.B, w.Hq, w.d), dtype=torch.bfloat16).pin_memory()
 
+    decode_step(ck, model, dq, dk, dv, out)
+    torch.cuda.synchronize()
+    g = capture_step(ck, model, dq, dk, dv, out) if graph else None
+
     def step(i):
         q, kn, vn = host_sets[i % len(host_sets)]
         dq.copy_(q, non_blocking=True)
         dk.copy_(kn, non_blocking=True)
         dv.copy_(vn, non_blocking=True)
-        decode_step(ck, model, dq, dk, dv, out)
+        if graph:
+            replay_step(ck, model, g)
+        else:
+            decode_step(ck, model, dq, dk, dv, out)
         hout.copy_(out, non_blocking=True)
         torch.cuda.current_stream().synchronize()  # the caller needs the outputs before the next token
 
@@ -369,6 +409,8 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying "
+                    "a captured CUDA graph of the step")
     ap.add_argument("--no-extras", action="store_true", help="skip the other configs, head_cv and the oracle timing")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -406,17 +448,18 @@ def main():
     peaks, peak_src = measured_peaks()
     w = synth.WORKLOADS[args.workload]
     n_layers = args.layers or w.layers
-    total_steps = 3 * (args.warmup + args.steps) + 8
+    total_steps = 3 * (args.warmup + args.steps) + 16
+    graph = not args.no_graph
     model, sel_ms = build_model(ck, w, dev, max_new=total_steps, layers=n_layers)
 
     vis = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
     sampler = ClockSampler(vis[local_rank] if local_rank < len(vis) else local_rank)
     sampler.start()
-    ms = max_over_ranks(time_decode(ck, w, model, dev, args.steps, args.warmup, barrier))
+    ms = max_over_ranks(time_decode(ck, w, model, dev, args.steps, args.warmup, barrier, graph))
     clocks = sampler.stop()
     bytes_per_layer = float(np.mean(kept_bytes(model)))
     part_us, part_med_us, comb_us = time_kernels(ck, w, model, dev, max(2, min(args.steps, 5)))
-    ms_e2e, h2d, d2h = time_e2e(ck, w, model, dev, args.steps, args.warmup, barrier)
+    ms_e2e, h2d, d2h = time_e2e(ck, w, model, dev, args.steps, args.warmup, barrier, graph)
     ms_e2e = max_over_ranks(ms_e2e)
 
     scale_layers = w.layers / n_layers  # only != 1 when --layers is used for profiling
@@ -432,7 +475,8 @@ def main():
                    "window": w.L_obs, "replicas": world,
                    "l2": "no flush: per-layer working set %.0f MB x %d layers, far above the 126 MB L2"
                          % (bytes_per_layer / 1e6, n_layers),
-                   "step": "one decode token of the whole model: per layer catekv_append + catekv_decode_attn"},
+                   "step": "one decode token of the whole model: per layer catekv_append + catekv_decode_attn",
+                   "launch": "CUDA graph replay of the step" if graph else "host launches"},
         "us_per_layer_step": ms * 1e3 / n_layers,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src, "traffic": None,
@@ -456,7 +500,7 @@ def main():
                 continue
             wo = synth.WORKLOADS[name]
             nl = min(wo.layers, 8)
-            mo, so = build_model(ck, wo, dev, max_new=64, layers=nl)
+            mo, so = build_model(ck, wo, dev, max_new=96, layers=nl)
             t = time_decode(ck, wo, mo, dev, 10, 3)
             pu, pm, cu = time_kernels(ck, wo, mo, dev, 3)
             by = float(np.mean(kept_bytes(mo)))

@@ -180,6 +180,14 @@ int catekv_select_compact(const catekv_select_params* p, catekv_cache* cache, in
 int catekv_append(catekv_cache* cache, const void* k_new, const void* v_new, catekv_stream stream);
 
 /*
+ * Host mirror only: record that n_tokens appends have run (or are about to run) on the device without
+ * the library's host code seeing them - the case of a caller who captured catekv_append in a CUDA
+ * graph and replays it.  Call it before each replay: it checks every segment's capacity
+ * (CATEKV_ERR_CAPACITY, nothing changed) and then adds n_tokens to cache->seg_len.  Launches nothing.
+ */
+int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens);
+
+/*
  * Work-balanced split-KV schedule for catekv_decode_attn.
  *
  * The rows of all segments, laid end to end, are cut into num_ctas near-equal

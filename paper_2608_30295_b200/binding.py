@@ -67,6 +67,7 @@ def _load():
         "catekv_select_workspace_bytes": (sz, [i32, i32, i32, i32, i32]),
         "catekv_select_compact": (C.c_int, [C.POINTER(SelectParams), C.POINTER(CacheStruct), vp, i64, vp, sz, vp]),
         "catekv_append": (C.c_int, [C.POINTER(CacheStruct), vp, vp, vp]),
+        "catekv_cache_advance": (C.c_int, [C.POINTER(CacheStruct), i32]),
         "catekv_decode_num_ctas": (C.c_int, []),
         "catekv_decode_plan_bytes": (sz, [i32, i32, i32]),
         "catekv_decode_workspace_bytes": (sz, [i32, i32, i32]),
@@ -149,6 +150,11 @@ def catekv_append(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor):
     _check(_lib.catekv_append(C.byref(cache.struct), k_new.data_ptr(), v_new.data_ptr(), _stream()), "catekv_append")
 
 
+def catekv_cache_advance(cache: Cache, n_tokens: int = 1):
+    """Host mirror only: account for appends that a replayed CUDA graph performs on the device."""
+    _check(_lib.catekv_cache_advance(C.byref(cache.struct), n_tokens), "catekv_cache_advance")
+
+
 def catekv_decode_num_ctas() -> int:
     n = _lib.catekv_decode_num_ctas()
     if n < 0:
@@ -174,9 +180,10 @@ def catekv_decode_plan(cache: Cache, plan: DecodePlan):
 
 
 def plan_header(plan: DecodePlan) -> dict:
-    h = plan.host[:32].numpy().view(np.int32)
+    h = plan.host[:48].numpy().view(np.int32)
     return {"num_ctas": int(h[1]), "n_segs": int(h[2]), "n_items": int(h[3]), "n_slots": int(h[4]),
-            "tile": int(h[5]), "total_rows": int(plan.host[24:32].numpy().view(np.int64)[0])}
+            "tile": int(h[5]), "total_rows": int(plan.host[24:32].numpy().view(np.int64)[0]),
+            "max_pieces": int(h[11])}
 
 
 def _decode_call(fn, name, cache, q, plan, out, lse_out, sm_scale):

@@ -34,15 +34,26 @@ struct PlanHeader {
   int32_t n_slots;
   int32_t tile;
   int64_t total_rows;
+  int32_t off_cta, off_items, off_seg;  // byte offsets of the three tables
+  int32_t max_pieces;                   // most pieces any segment was cut into
 };
-static_assert(sizeof(PlanHeader) == 32, "plan header layout");
+static_assert(sizeof(PlanHeader) == 48, "plan header layout");
 
-struct WorkItem {
+struct WorkItem {  // 32 bytes
   int32_t seg;
-  int32_t t0;    // first row of the piece, relative to the segment
-  int32_t t1;    // one past the last row; -1 = up to the segment's current length (last piece)
-  int32_t slot;  // partial slot, or -1 when the piece is the whole segment (final output written directly)
+  int32_t t0;        // first row of the piece, relative to the segment
+  int32_t t1;        // one past its last row at plan time
+  int32_t slot;      // partial slot, or -1 when the piece is the whole segment (final output written directly)
+  int64_t row_base;  // pool row of t0 (segment offset + t0)
+  int32_t last;      // 1: last piece of its segment; it also covers rows [t1, current length)
+  int32_t reserved;
 };
+static_assert(sizeof(WorkItem) == 32, "work item layout");
+struct CtaHeader {  // 48 bytes: the CTA's item range and a copy of its first item (one load starts the stream)
+  int32_t item_begin, item_end, reserved0, reserved1;
+  WorkItem first;
+};
+static_assert(sizeof(CtaHeader) == 48, "cta header layout");
 struct SegInfo {
   int32_t slot_begin;
   int32_t n_pieces;
@@ -56,7 +67,7 @@ static PlanLayout plan_layout(int n_segs, int num_ctas) {
   PlanLayout L;
   L.n_items_cap = num_ctas + n_segs;
   L.off_cta = sizeof(PlanHeader);
-  L.off_items = align_up(L.off_cta + sizeof(int32_t) * (size_t)(num_ctas + 1), 16);
+  L.off_items = align_up(L.off_cta + sizeof(CtaHeader) * (size_t)num_ctas, 32);
   L.off_seg = L.off_items + sizeof(WorkItem) * (size_t)L.n_items_cap;
   L.bytes = align_up(L.off_seg + sizeof(SegInfo) * (size_t)n_segs, 16);
   return L;
@@ -81,7 +92,7 @@ struct DecodeArgs {
   const uint16_t* q;  // [B, Hq, d]
   int32_t Hq, Hkv, G;
   float scale_log2;  // sm_scale * log2(e)
-  const int32_t* cta_item_begin;
+  const CtaHeader* ctas;
   const WorkItem* items;
   float* part_o;    // [slots, 8, 128]
   float* part_lse;  // [slots, 8], log2 domain
@@ -96,31 +107,90 @@ constexpr int kMergeRegs = 36;                         // 32 accumulators + m0, 
 constexpr int kMergeSlotBytes = kMergeRegs * 32 * 4;
 constexpr int kDecodeSmem = kStages * (kStageBytes + kQSlotBytes) + 2 * kMergeSlotBytes;
 
+// A piece is streamed as tiles of its plan-time rows [t0, t1), followed - for the last piece of a
+// segment - by tiles of the rows appended since the plan was built, [t1, live length).  The live length
+// is loaded when the item is read but first used only after the plan-time tiles have been issued, so
+// the stream never waits for that load.
 struct ItemCursor {
-  int seg, t0, t1, ntiles, slot;
-  int64_t row_base;  // first pool row of the piece
+  int seg, t0, t1, slot, last;
+  int np;            // tiles of the plan-time rows
+  int live;          // current segment length (meaningful if last)
+  int64_t row_base;
 };
 
-__device__ __forceinline__ ItemCursor read_item(const DecodeArgs& a, int it) {
-  const int4 w = __ldg(reinterpret_cast<const int4*>(a.items) + it);
+__device__ __forceinline__ ItemCursor make_cursor(const DecodeArgs& a, const WorkItem& w) {
   ItemCursor c;
-  c.seg = w.x;
-  c.t0 = w.y;
-  c.t1 = (w.z < 0) ? __ldg(a.seg_len + w.x) : w.z;
-  c.slot = w.w;
-  const int rows = c.t1 - c.t0;
-  c.ntiles = rows > 0 ? (rows + kTile - 1) / kTile : 1;
-  c.row_base = (int64_t)__ldg(a.seg_off + w.x) + c.t0;
+  c.seg = w.seg;
+  c.t0 = w.t0;
+  c.t1 = w.t1;
+  c.slot = w.slot;
+  c.last = w.last;
+  c.row_base = w.row_base;
+  c.np = (w.t1 - w.t0 + kTile - 1) / kTile;
+  c.live = w.last ? __ldg(a.seg_len + w.seg) : w.t1;
   return c;
 }
+__device__ __forceinline__ ItemCursor read_item(const DecodeArgs& a, int it) {
+  const int4* p = reinterpret_cast<const int4*>(a.items + it);
+  const int4 x = __ldg(p), y = __ldg(p + 1);
+  WorkItem w;
+  w.seg = x.x; w.t0 = x.y; w.t1 = x.z; w.slot = x.w;
+  w.row_base = (int64_t)(((uint64_t)(uint32_t)y.y << 32) | (uint32_t)y.x);
+  w.last = y.z; w.reserved = 0;
+  return make_cursor(a, w);
+}
+// tiles of the item: plan-time tiles plus tiles of the appended rows; at least one
+__device__ __forceinline__ int item_tiles(const ItemCursor& c) {
+  const int extra = c.live - c.t1;
+  const int ne = extra > 0 ? (extra + kTile - 1) / kTile : 0;
+  return max(1, c.np + ne);
+}
+// first row (relative to the segment) and number of valid rows of tile i
+__device__ __forceinline__ void tile_rows(const ItemCursor& c, int i, int& start, int& nvalid) {
+  if (i < c.np) {
+    start = c.t0 + i * kTile;
+    nvalid = c.t1 - start;
+  } else {
+    start = c.t1 + (i - c.np) * kTile;
+    nvalid = c.live - start;
+  }
+}
+
+#ifdef CATEKV_TRACE
+__device__ unsigned long long g_trace[4096 * 4];
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+#define CATEKV_STAMP(i) do { if (threadIdx.x == 0) g_trace[blockIdx.x * 4 + (i)] = gtime(); } while (0)
+#else
+#define CATEKV_STAMP(i) do { } while (0)
+#endif
 
 __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int item_begin = a.cta_item_begin[blockIdx.x];
-  const int item_end = a.cta_item_begin[blockIdx.x + 1];
-  if (item_begin >= item_end) return;
+  CATEKV_STAMP(0);
+  pdl_launch_dependents();
+  int item_begin, item_end;
+  ItemCursor pc;
+  {
+    // the plan was uploaded by a copy that precedes the previous kernel: it may be read before the wait
+    const int4* hp = reinterpret_cast<const int4*>(a.ctas + blockIdx.x);
+    const int4 h0 = __ldg(hp), x = __ldg(hp + 1), y = __ldg(hp + 2);
+    pdl_wait();  // from here on: lengths, queries and cache rows written by earlier kernels
+    item_begin = h0.x;
+    item_end = h0.y;
+    if (item_begin >= item_end) return;
+    WorkItem w;
+    w.seg = x.x; w.t0 = x.y; w.t1 = x.z; w.slot = x.w;
+    w.row_base = (int64_t)(((uint64_t)(uint32_t)y.y << 32) | (uint32_t)y.x);
+    w.last = y.z; w.reserved = 0;
+    pc = make_cursor(a, w);
+  }
+  const ItemCursor first = pc;
 
   const uint32_t s_stage = smem_u32(smem);
   const uint32_t s_q = s_stage + kStages * kStageBytes;
@@ -128,12 +198,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
 
   // ---- producer: issues one tile (and the item's queries with its first tile) per call
   int p_item = item_begin, p_tile = 0, p_seq = 0;
-  ItemCursor pc = read_item(a, p_item);
   auto issue = [&]() {
     if (p_item < item_end) {
       const uint32_t sb = s_stage + (p_seq % kStages) * kStageBytes;
-      const int rows_left = pc.t1 - pc.t0 - p_tile * kTile;
-      const int64_t row0 = pc.row_base + (int64_t)p_tile * kTile;
+      int start, rows_left;
+      tile_rows(pc, p_tile, start, rows_left);
+      const int64_t row0 = pc.row_base + (start - pc.t0);
 #pragma unroll
       for (int i = 0; i < (kTile * 16) / kDecodeThreads; ++i) {
         const int id = tid + i * kDecodeThreads;
@@ -154,7 +224,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
         cp_async16(qb + r * kRowBytes + c * 16, src, ok);
       }
       ++p_seq;
-      if (++p_tile == pc.ntiles) {
+      // the plan-time tiles need no look at the live length; only past them is it consulted
+      if (++p_tile >= pc.np && p_tile >= item_tiles(pc)) {
         p_tile = 0;
         if (++p_item < item_end) pc = read_item(a, p_item);
       }
@@ -167,16 +238,17 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
 
   int seq = 0;
   for (int c_item = item_begin; c_item < item_end; ++c_item) {
-    const ItemCursor cc = read_item(a, c_item);
+    const ItemCursor cc = c_item == item_begin ? first : read_item(a, c_item);
     uint32_t qf[8][2];
     float o[8][4];
 #pragma unroll
     for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
-    for (int tile = 0; tile < cc.ntiles; ++tile, ++seq) {
+    for (int tile = 0; tile < cc.np || tile < item_tiles(cc); ++tile, ++seq) {
       cp_async_wait<kStages - 2>();
       __syncthreads();
+      if (seq == 0) CATEKV_STAMP(1);
       issue();
       if (tile == 0) {
         const uint8_t* qs = smem + kStages * kStageBytes + ((c_item - item_begin) % kStages) * kQSlotBytes;
@@ -186,7 +258,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
           qf[ks][1] = *reinterpret_cast<const uint32_t*>(qs + g * kRowBytes + (ks * 16 + 8 + 2 * t) * 2);
         }
       }
-      const int nvalid = cc.t1 - cc.t0 - tile * kTile;  // valid rows of this tile (may exceed kTile)
+      int tstart, nvalid;  // valid rows of this tile (may exceed kTile)
+      tile_rows(cc, tile, tstart, nvalid);
       const int row0 = warp * 16;
       if (row0 >= nvalid) continue;  // warp-uniform: this warp's 16 rows are all padding
       const uint32_t kb = s_stage + (seq % kStages) * kStageBytes;
@@ -255,6 +328,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     }
 
     // ---- end of the piece: finish the row sums, merge the four warps, write the result
+    if (c_item == item_end - 1) CATEKV_STAMP(2);
 #pragma unroll
     for (int sh = 4; sh <= 16; sh <<= 1) {
       l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
@@ -345,7 +419,14 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     }
   }
   cp_async_wait<0>();
+  CATEKV_STAMP(3);
 }
+
+#ifdef CATEKV_TRACE
+extern "C" int catekv_debug_trace(unsigned long long* host_out, int n_ctas) {
+  return (int)cudaMemcpyFromSymbol(host_out, g_trace, sizeof(unsigned long long) * 4 * n_ctas);
+}
+#endif
 
 // ------------------------------------------------------------------------------------------
 // Combine: merge the partials of every segment that was cut into several pieces
@@ -359,29 +440,67 @@ struct CombineArgs {
   int32_t Hq, Hkv, G, out_fp32;
 };
 
+// One CTA per (segment, query head of the group).  The LSEs of the pieces are loaded in parallel, the
+// four warps each sum a quarter of the pieces (a lane owns four consecutive d, so a piece is one
+// 512-byte row per warp-load and many loads are in flight), then the warps are summed in a fixed order.
 __global__ void __launch_bounds__(kD) decode_combine_kernel(const CombineArgs a) {
-  const int seg = blockIdx.x, hd = blockIdx.y, dI = threadIdx.x;
-  const SegInfo si = a.seg_info[seg];
-  if (si.n_pieces == 1) return;  // written directly by the attention kernel
-  const int b = seg / a.Hkv, h = seg % a.Hkv;
-  const size_t oidx = ((size_t)b * a.Hq + (size_t)h * a.G + hd) * kD + dI;
-  float acc = 0.f, wsum = 0.f, M = -INFINITY;
-  for (int p = 0; p < si.n_pieces; ++p) M = fmaxf(M, a.part_lse[(size_t)(si.slot_begin + p) * kMaxG + hd]);
+  const int seg = blockIdx.x, hd = blockIdx.y;
+  pdl_launch_dependents();
+  const SegInfo si = a.seg_info[seg];  // plan data: older than the previous kernel
+  pdl_wait();
+  if (si.n_pieces <= 1) return;  // written directly by the attention kernel
+  __shared__ float s_red[4];
+  __shared__ float4 s_acc[4][32];
+  __shared__ float s_w[4];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const float* lse = a.part_lse + (size_t)si.slot_begin * kMaxG + hd;
+  // max of the pieces' LSEs
+  float m = -INFINITY;
+  for (int p = tid; p < si.n_pieces; p += kD) m = fmaxf(m, lse[(size_t)p * kMaxG]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if (lane == 0) s_red[warp] = m;
+  __syncthreads();
+  const float M = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float wsum = 0.f;
   if (M > -INFINITY) {
-    for (int p = 0; p < si.n_pieces; ++p) {
-      const size_t s = (size_t)(si.slot_begin + p);
-      const float w = exp2f(a.part_lse[s * kMaxG + hd] - M);
-      acc += w * a.part_o[s * (kMaxG * kD) + hd * kD + dI];
+    const float* po = a.part_o + ((size_t)si.slot_begin * kMaxG + hd) * kD + lane * 4;
+#pragma unroll 4
+    for (int p = warp; p < si.n_pieces; p += 4) {
+      const float w = exp2f(lse[(size_t)p * kMaxG] - M);
+      const float4 v = *reinterpret_cast<const float4*>(po + (size_t)p * (kMaxG * kD));
+      acc.x += w * v.x;
+      acc.y += w * v.y;
+      acc.z += w * v.z;
+      acc.w += w * v.w;
       wsum += w;
     }
-    acc /= wsum;
   }
-  if (a.out_fp32)
-    reinterpret_cast<float*>(a.out)[oidx] = acc;
-  else
-    reinterpret_cast<__nv_bfloat16*>(a.out)[oidx] = __float2bfloat16_rn(acc);
-  if (a.lse_out && dI == 0)
-    a.lse_out[(size_t)b * a.Hq + h * a.G + hd] = (M > -INFINITY) ? (M + log2f(wsum)) * 0.6931471805599453f : -INFINITY;
+  s_acc[warp][lane] = acc;
+  if (lane == 0) s_w[warp] = wsum;
+  __syncthreads();
+  if (warp == 0) {
+    const float W = ((s_w[0] + s_w[1]) + s_w[2]) + s_w[3];
+    const float inv = W > 0.f ? 1.f / W : 0.f;
+    float4 r;
+    r.x = (((s_acc[0][lane].x + s_acc[1][lane].x) + s_acc[2][lane].x) + s_acc[3][lane].x) * inv;
+    r.y = (((s_acc[0][lane].y + s_acc[1][lane].y) + s_acc[2][lane].y) + s_acc[3][lane].y) * inv;
+    r.z = (((s_acc[0][lane].z + s_acc[1][lane].z) + s_acc[2][lane].z) + s_acc[3][lane].z) * inv;
+    r.w = (((s_acc[0][lane].w + s_acc[1][lane].w) + s_acc[2][lane].w) + s_acc[3][lane].w) * inv;
+    const int b = seg / a.Hkv, h = seg % a.Hkv;
+    const size_t obase = ((size_t)b * a.Hq + (size_t)h * a.G + hd) * kD;
+    if (a.out_fp32) {
+      reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + obase)[lane] = r;
+    } else {
+      uint2 pk;
+      pk.x = pack_bf16(r.x, r.y);
+      pk.y = pack_bf16(r.z, r.w);
+      reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(a.out) + obase)[lane] = pk;
+    }
+    if (a.lse_out && lane == 0)
+      a.lse_out[(size_t)b * a.Hq + h * a.G + hd] = W > 0.f ? (M + log2f(W)) * 0.6931471805599453f : -INFINITY;
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -392,6 +511,8 @@ __global__ void __launch_bounds__(128) append_kernel(uint8_t* k_pool, uint8_t* v
                                                      int n_segs) {
   const int seg = blockIdx.x * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
+  pdl_launch_dependents();
+  pdl_wait();
   if (seg >= n_segs) return;
   const int len = seg_len[seg];
   const int64_t row = (int64_t)seg_off[seg] + len;
@@ -425,11 +546,21 @@ extern "C" int catekv_append(catekv_cache* cache, const void* k_new, const void*
     if (cache->seg_len[s] < 0) return CATEKV_ERR_INVALID_ARG;
     if (cache->seg_len[s] + 1 > cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
   }
-  append_kernel<<<(n + 3) / 4, 128, 0, (cudaStream_t)stream>>>(
-      (uint8_t*)cache->k_pool, (uint8_t*)cache->v_pool, cache->seg_off_dev, cache->seg_len_dev,
-      (const uint8_t*)k_new, (const uint8_t*)v_new, n);
-  CATEKV_CUDA_TRY(cudaGetLastError());
+  CATEKV_CUDA_TRY(launch_pdl(append_kernel, dim3((n + 3) / 4), dim3(128), 0, (cudaStream_t)stream,
+                             (uint8_t*)cache->k_pool, (uint8_t*)cache->v_pool, cache->seg_off_dev, cache->seg_len_dev,
+                             (const uint8_t*)k_new, (const uint8_t*)v_new, n));
   for (int s = 0; s < n; ++s) cache->seg_len[s] += 1;
+  return CATEKV_OK;
+}
+
+extern "C" int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens) {
+  int rc = check_cache(cache);
+  if (rc) return rc;
+  if (n_tokens < 0) return CATEKV_ERR_INVALID_ARG;
+  const int n = cache->B * cache->Hkv;
+  for (int s = 0; s < n; ++s)
+    if ((int64_t)cache->seg_len[s] + n_tokens > cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+  for (int s = 0; s < n; ++s) cache->seg_len[s] += n_tokens;
   return CATEKV_OK;
 }
 
@@ -470,8 +601,9 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
     total += cache->seg_len[s];
   }
   uint8_t* base = (uint8_t*)plan_host;
+  memset(base, 0, L.bytes);
   PlanHeader* hdr = (PlanHeader*)base;
-  int32_t* cta_begin = (int32_t*)(base + L.off_cta);
+  CtaHeader* ctas = (CtaHeader*)(base + L.off_cta);
   WorkItem* items = (WorkItem*)(base + L.off_items);
   SegInfo* segs = (SegInfo*)(base + L.off_seg);
 
@@ -480,18 +612,18 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
   quota = (quota + kSplitAlign - 1) / kSplitAlign * kSplitAlign;
   if (quota < kSplitAlign) quota = kSplitAlign;
 
-  int n_items = 0, n_slots = 0;
+  int n_items = 0, n_slots = 0, max_pieces = 1;
   int seg = 0;
   int32_t pos = 0;  // next unassigned row of `seg`
   int seg_first_item = 0;
   for (int c = 0; c < num_ctas; ++c) {
-    cta_begin[c] = n_items;
+    ctas[c].item_begin = n_items;
     int64_t room = quota;
     while (seg < n_segs) {
       const int32_t len = cache->seg_len[seg];
       if (len == 0) {
         // an empty segment still gets one (direct) item, so that the plan stays valid once it grows
-        items[n_items++] = WorkItem{seg, 0, -1, -1};
+        items[n_items++] = WorkItem{seg, 0, 0, -1, (int64_t)cache->seg_off[seg], 1, 0};
         segs[seg] = SegInfo{0, 1};
         ++seg;
         seg_first_item = n_items;
@@ -499,13 +631,13 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
       }
       if (room <= 0) break;
       const int32_t take = (int32_t)((int64_t)(len - pos) < room ? (len - pos) : room);
-      items[n_items++] = WorkItem{seg, pos, pos + take, 0};
+      items[n_items++] = WorkItem{seg, pos, pos + take, 0, (int64_t)cache->seg_off[seg] + pos, 0, 0};
       pos += take;
       room -= take;
       if (pos == len) {
         // segment finished: fix up its pieces
         const int pieces = n_items - seg_first_item;
-        items[n_items - 1].t1 = -1;  // the last piece follows the segment's current length
+        items[n_items - 1].last = 1;  // the last piece follows the segment's current length
         if (pieces == 1) {
           items[seg_first_item].slot = -1;
           segs[seg] = SegInfo{0, 1};
@@ -513,15 +645,18 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
           for (int i = 0; i < pieces; ++i) items[seg_first_item + i].slot = n_slots + i;
           segs[seg] = SegInfo{n_slots, pieces};
           n_slots += pieces;
+          max_pieces = pieces > max_pieces ? pieces : max_pieces;
         }
         ++seg;
         pos = 0;
         seg_first_item = n_items;
       }
     }
+    ctas[c].item_end = n_items;
   }
-  cta_begin[num_ctas] = n_items;
   if (seg != n_segs) return CATEKV_ERR_INVALID_ARG;  // cannot happen: quota * num_ctas >= total
+  for (int c = 0; c < num_ctas; ++c)
+    if (ctas[c].item_begin < ctas[c].item_end) ctas[c].first = items[ctas[c].item_begin];
   hdr->magic = kPlanMagic;
   hdr->num_ctas = num_ctas;
   hdr->n_segs = n_segs;
@@ -529,6 +664,10 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
   hdr->n_slots = n_slots;
   hdr->tile = kTile;
   hdr->total_rows = total;
+  hdr->off_cta = (int32_t)L.off_cta;
+  hdr->off_items = (int32_t)L.off_items;
+  hdr->off_seg = (int32_t)L.off_seg;
+  hdr->max_pieces = max_pieces;
   if (plan_dev)
     CATEKV_CUDA_TRY(cudaMemcpyAsync(plan_dev, plan_host, L.bytes, cudaMemcpyHostToDevice, (cudaStream_t)stream));
   return CATEKV_OK;
@@ -579,15 +718,14 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* q, i
     a.Hkv = cache->Hkv;
     a.G = G;
     a.scale_log2 = (sm_scale == 0.f ? 1.0f / sqrtf((float)kD) : sm_scale) * 1.4426950408889634f;
-    a.cta_item_begin = (const int32_t*)(pd + L.off_cta);
+    a.ctas = (const CtaHeader*)(pd + L.off_cta);
     a.items = (const WorkItem*)(pd + L.off_items);
     a.part_o = part_o;
     a.part_lse = part_lse;
     a.out = out;
     a.out_fp32 = out_fp32;
     a.lse_out = lse_out;
-    decode_partial_kernel<<<hdr->num_ctas, kDecodeThreads, kDecodeSmem, st>>>(a);
-    CATEKV_CUDA_TRY(cudaGetLastError());
+    CATEKV_CUDA_TRY(launch_pdl(decode_partial_kernel, dim3(hdr->num_ctas), dim3(kDecodeThreads), kDecodeSmem, st, a));
   }
   if ((phases & 2) && hdr->n_slots > 0) {
     CombineArgs ca;
@@ -600,8 +738,7 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* q, i
     ca.Hkv = cache->Hkv;
     ca.G = G;
     ca.out_fp32 = out_fp32;
-    decode_combine_kernel<<<dim3(n_segs, G), kD, 0, st>>>(ca);
-    CATEKV_CUDA_TRY(cudaGetLastError());
+    CATEKV_CUDA_TRY(launch_pdl(decode_combine_kernel, dim3(n_segs, G), dim3(kD), 0, st, ca));
   }
   return CATEKV_OK;
 }

@@ -77,8 +77,8 @@ struct CvWs {
 };
 static CvWs cv_ws_layout(int n_segs, int G, int m_max, int L_obs) {
   CvWs w;
-  int kp = 256;
-  while ((long)n_segs * ((m_max + kp - 1) / kp) > 148 * 8 && kp < (1 << 30)) kp *= 2;
+  int kp = 512;
+  while ((long)n_segs * ((m_max + kp - 1) / kp) > 148 * 4 && kp < (1 << 30)) kp *= 2;
   w.keys_per_cta = kp;
   w.n_chunks = (m_max + kp - 1) / kp;
   w.rows_pad = score_rows_pad(G, L_obs);

@@ -227,26 +227,33 @@ __global__ void __launch_bounds__(kScoreThreads) score_kernel(const ScoreArgs a)
 }
 
 // Merge the per-CTA row partials: stats[job][row] = (max, 1 / sum); padding rows get (0, 0).
-__global__ void score_stats_merge_kernel(const ScoreArgs a, int rows_it, int kgroups) {
+// One warp per row: the lanes stride over the partials, then merge pairwise.
+__global__ void __launch_bounds__(256) score_stats_merge_kernel(const ScoreArgs a, int rows_it, int kgroups) {
   const int jobi = blockIdx.y;
   const int rows_pad = a.G * rows_it;
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
   if (r >= rows_pad) return;
   const ScoreJob job = a.jobs[jobi];
-  float2 res = make_float2(0.f, 0.f);
+  float m = -INFINITY, l = 0.f;
   if (r % rows_it < a.L_obs) {
     const int used = (job.j_end - job.j_begin + a.keys_per_cta - 1) / a.keys_per_cta;
-    float m = -INFINITY, l = 0.f;
-    for (int c = 0; c < used * kgroups; ++c) {
+    for (int c = lane; c < used * kgroups; c += 32) {
       const float2 p = a.stats_part[((size_t)jobi * a.n_chunks * kgroups + c) * rows_pad + r];
       if (p.x == -INFINITY) continue;
       const float mn = fmaxf(m, p.x);
       l = l * ((m == -INFINITY) ? 0.f : exp2f(m - mn)) + p.y * exp2f(p.x - mn);
       m = mn;
     }
-    res = (l > 0.f) ? make_float2(m, 1.f / l) : make_float2(0.f, 0.f);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, m, o), ol = __shfl_xor_sync(0xffffffffu, l, o);
+      const float mn = fmaxf(m, om);
+      l = l * ((m == -INFINITY) ? 0.f : exp2f(m - mn)) + ol * ((om == -INFINITY) ? 0.f : exp2f(om - mn));
+      m = mn;
+    }
   }
-  a.stats[(size_t)jobi * rows_pad + r] = res;
+  if (lane == 0) a.stats[(size_t)jobi * rows_pad + r] = (l > 0.f) ? make_float2(m, 1.f / l) : make_float2(0.f, 0.f);
 }
 
 template <int MODE, int N_IT>
@@ -267,7 +274,7 @@ int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream) {
   if (rc) return rc;
   const int rows_it = small ? 32 : 64;
   const int rows_pad = a.G * rows_it;
-  score_stats_merge_kernel<<<dim3((rows_pad + 127) / 128, a.n_jobs), 128, 0, stream>>>(a, rows_it, score_key_groups(a.L_obs));
+  score_stats_merge_kernel<<<dim3((rows_pad + 7) / 8, a.n_jobs), 256, 0, stream>>>(a, rows_it, score_key_groups(a.L_obs));
   CATEKV_CUDA_TRY(cudaGetLastError());
   if (out_mode == kScoreColsum)
     return small ? launch_one<kScoreColsum, 2>(a, stream) : launch_one<kScoreColsum, 4>(a, stream);

@@ -198,9 +198,9 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
 }
 
 static int keys_per_cta_for(int n_segs, int n_sc_max) {
-  // the smallest power-of-two multiple of 256 keys that keeps the grid within 8 CTAs per SM
-  int kp = 256;
-  while ((long)n_segs * ((n_sc_max + kp - 1) / kp) > 148 * 8 && kp < (1 << 30)) kp *= 2;
+  // the smallest power-of-two multiple of 512 keys that keeps the grid within 4 CTAs per SM
+  int kp = 512;
+  while ((long)n_segs * ((n_sc_max + kp - 1) / kp) > 148 * 4 && kp < (1 << 30)) kp *= 2;
   return kp;
 }
 

@@ -61,13 +61,22 @@ def _plan(ck, lens, B, Hkv, num_ctas):
     buf = np.zeros(nbytes, dtype=np.uint8)
     rc = ck._lib.catekv_decode_plan(C.byref(st), num_ctas, buf.ctypes.data, None, nbytes, None)
     assert rc == 0
-    hdr = buf[:32].view(np.int32)
+    hdr = buf[:48].view(np.int32)
     n_items, n_slots = int(hdr[3]), int(hdr[4])
-    off_cta = 32
-    off_items = (off_cta + 4 * (num_ctas + 1) + 15) // 16 * 16
-    off_seg = off_items + 16 * (num_ctas + B * Hkv)
-    cta = buf[off_cta:off_cta + 4 * (num_ctas + 1)].view(np.int32)
-    items = buf[off_items:off_items + 16 * n_items].view(np.int32).reshape(-1, 4)
+    off_cta, off_items, off_seg = int(hdr[8]), int(hdr[9]), int(hdr[10])
+    ch = buf[off_cta:off_cta + 48 * num_ctas].view(np.int32).reshape(num_ctas, 12)
+    cta = np.concatenate([ch[:, 0], ch[-1:, 1]])
+    assert np.array_equal(ch[1:, 0], ch[:-1, 1])  # consecutive item ranges
+    raw = buf[off_items:off_items + 32 * n_items].view(np.int32).reshape(-1, 8)
+    seg_off = keep[0]
+    for c in range(num_ctas):  # the inline copy of the CTA's first item
+        if ch[c, 0] < ch[c, 1]:
+            assert np.array_equal(ch[c, 4:12], raw[ch[c, 0]])
+    for r in raw:  # pool row of the piece's first row
+        assert int(r[4:6].view(np.int64)[0]) == int(seg_off[r[0]]) + int(r[1])
+    # (seg, t0, t1 or -1 for the piece that follows the live length, slot)
+    items = np.stack([raw[:, 0], raw[:, 1], np.where(raw[:, 6] == 1, -1, raw[:, 2]), raw[:, 3]], axis=1) \
+        if n_items else np.zeros((0, 4), dtype=np.int32)
     segs = buf[off_seg:off_seg + 8 * B * Hkv].view(np.int32).reshape(-1, 2)
     return cta, items, segs, n_slots
 
