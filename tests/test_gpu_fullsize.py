@@ -1,0 +1,168 @@
+"""GPU parity at the full sizes of the five configurations, in the launch configuration bench.py times
+(plan over SMs x resident CTAs, caches built by catekv_select_compact).  The oracle is run on sampled
+(sequence, KV head) cells: their prefill rows and kept lists are copied back and checked one by one."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import catekv_oracle as orc
+from workloads import synth
+import helpers as H
+import bench
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ck():
+    import paper_2608_30295_b200 as pkg
+    assert torch.cuda.is_available()
+    return pkg.binding
+
+
+def _build_layer(ck, w, layer, max_new):
+    p = synth.prefill_layer(w, layer, "cuda")
+    mask = p["head_mask"]
+    cache = ck.Cache(w.B, w.Hkv, bench.expected_lengths(w, mask), max_new, "cuda")
+    idx = torch.full((w.B * w.Hkv, w.n), -1, dtype=torch.int32, device="cuda")
+    ck.catekv_select_compact(p["q_win"], p["k"], p["v"], p["seq_len"], mask, cache, w.budget, w.eta, w.sink, w.local,
+                             w.pool_mode, w.pool_param, idx_out=idx)
+    torch.cuda.synchronize()
+    return p, mask, cache, idx
+
+
+def _check_selection_cells(w, p, mask, cache, idx, cells):
+    """Selected indices (band-aware) and segment bytes of the sampled cells; returns oracle caches of the cells
+    built from the device's own kept lists."""
+    eta32 = float(np.float32(w.eta))
+    oc = orc.HybridCache(w.B, w.Hkv, w.d)
+    oc.k_rows = [np.zeros((0, w.d), dtype=np.uint16)] * (w.B * w.Hkv)
+    oc.v_rows = [np.zeros((0, w.d), dtype=np.uint16)] * (w.B * w.Hkv)
+    dev_len = cache.seg_len_dev.cpu().numpy()
+    assert np.array_equal(dev_len, cache.seg_len)
+    for (b, h) in cells:
+        i = b * w.Hkv + h
+        L = int(cache.seg_len[i])
+        got = idx[i, :L].cpu().numpy()
+        k = synth.bits(p["k"][b, h])
+        v = synth.bits(p["v"][b, h])
+        T = orc.token_budget(w.n, bool(mask[b, h]), w.budget, eta32)
+        if T >= w.n:
+            assert np.array_equal(got, np.arange(w.n))
+        else:
+            qw = synth.bits(p["q_win"][b, h * w.G:(h + 1) * w.G])
+            C = orc.window_scores(qw, k, w.L_obs)
+            H.check_indices_band(got, C, w.n, w.sink, w.local, T, w.pool_mode, w.pool_param, f"{w.name} b{b} h{h}")
+            assert L == min(w.n, T) or w.pool_mode == orc.POOL_CHUNK
+            # every planted heavy key is far above the threshold
+            assert set(p["heavy"][b, h]) <= set(got.tolist())
+        o = int(cache.seg_off[i])
+        assert np.array_equal(synth.bits(cache.k_pool[o:o + L]), k[got])
+        assert np.array_equal(synth.bits(cache.v_pool[o:o + L]), v[got])
+        oc.k_rows[i] = k[got]
+        oc.v_rows[i] = v[got]
+    return oc
+
+
+def _decode_steps(ck, w, layer, mask, cache, oc, cells, n_steps, check_steps):
+    plan = ck.DecodePlan(cache, ck.catekv_decode_num_ctas())
+    ck.catekv_decode_plan(cache, plan)
+    o32 = torch.empty((w.B, w.Hq, w.d), dtype=torch.float32, device="cuda")
+    o16 = torch.empty((w.B, w.Hq, w.d), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((w.B, w.Hq), dtype=torch.float32, device="cuda")
+    for step in range(n_steps):
+        q, kn, vn = synth.decode_inputs(w, layer, step, "cuda", mask)
+        ck.catekv_append(cache, kn, vn)
+        knb, vnb = synth.bits(kn), synth.bits(vn)
+        for (b, h) in cells:
+            i = b * w.Hkv + h
+            oc.k_rows[i] = np.concatenate([oc.k_rows[i], knb[b, h][None]])
+            oc.v_rows[i] = np.concatenate([oc.v_rows[i], vnb[b, h][None]])
+        if step in check_steps:
+            ck.catekv_decode_attn(cache, q, plan, o32, lse)
+            ck.catekv_decode_attn(cache, q, plan, o16)
+            ref, ref_lse = orc.decode_attention(oc, synth.bits(q), cells=cells)
+            H.check_attention(o32, o16, lse, ref, ref_lse, f"{w.name} layer {layer} step {step}")
+
+
+def _pick_cells(mask, want):
+    """Up to `want` cells, alternating consistent and adaptive heads across sequences."""
+    cons = [(b, h) for b in range(mask.shape[0]) for h in range(mask.shape[1]) if mask[b, h]]
+    adap = [(b, h) for b in range(mask.shape[0]) for h in range(mask.shape[1]) if not mask[b, h]]
+    rng = np.random.default_rng(int(mask.sum()) + 7)
+    rng.shuffle(cons), rng.shuffle(adap)
+    out = []
+    while len(out) < want and (cons or adap):
+        if cons:
+            out.append(cons.pop())
+        if adap and len(out) < want:
+            out.append(adap.pop())
+    return out
+
+
+def test_cfg1_32k_two_layers_steps_0_1_127(ck):
+    w = synth.WORKLOADS["cfg1"]
+    for layer in (0, 17):
+        p, mask, cache, idx = _build_layer(ck, w, layer, w.decode_steps)
+        cells = _pick_cells(mask, 4)
+        oc = _check_selection_cells(w, p, mask, cache, idx, cells)
+        del p, idx
+        _decode_steps(ck, w, layer, mask, cache, oc, cells, 128, {0, 1, 127})
+        assert np.all(cache.seg_len_dev.cpu().numpy() == cache.seg_len)
+
+
+def test_cfg2_128k_adaptive_keeps_90_percent(ck):
+    w = synth.WORKLOADS["cfg2"]
+    p, mask, cache, idx = _build_layer(ck, w, 3, 8)
+    lens = cache.seg_len.reshape(w.B, w.Hkv)
+    assert set(np.unique(lens[mask == 1])) <= {2048} and set(np.unique(lens[mask == 0])) == {117964}
+    cells = _pick_cells(mask, 3)
+    oc = _check_selection_cells(w, p, mask, cache, idx, cells)
+    del p, idx
+    _decode_steps(ck, w, 3, mask, cache, oc, cells, 3, {0, 1, 2})
+
+
+def test_cfg3_batch16_ragged_masks(ck):
+    w = synth.WORKLOADS["cfg3"]
+    p, mask, cache, idx = _build_layer(ck, w, 5, 8)
+    per_seq = mask.sum(axis=1)
+    assert per_seq.min() >= 3 and per_seq.max() <= 6 and len(set(per_seq.tolist())) > 1  # 40-70 % of 8 heads
+    cells = _pick_cells(mask, 4)
+    assert len({b for b, _ in cells}) >= 3
+    oc = _check_selection_cells(w, p, mask, cache, idx, cells)
+    del p, idx
+    _decode_steps(ck, w, 5, mask, cache, oc, cells, 2, {0, 1})
+
+
+def test_cfg4_qwen_gqa7_chunks(ck):
+    w = synth.WORKLOADS["cfg4"]
+    p, mask, cache, idx = _build_layer(ck, w, 2, 8)
+    cells = _pick_cells(mask, 2)
+    oc = _check_selection_cells(w, p, mask, cache, idx, cells)
+    del p, idx
+    _decode_steps(ck, w, 2, mask, cache, oc, cells, 2, {0, 1})
+
+
+def test_cfg4_head_mask_from_calibration_prompts(ck):
+    # 8 calibration prompts of 16K tokens; the library's scores and vote must reproduce the oracle's mask
+    w = synth.WORKLOADS["cfg4"]
+    layers, prompts, n = 4, 8, 16384
+    L_init, L_rec = 2048 // 32, 2048 // 128
+    rng = np.random.default_rng(44)
+    types = np.stack([rng.permutation(np.array([1, 1, 0, 0], dtype=np.uint8)) for _ in range(layers)])
+    got = np.zeros((prompts, layers * w.Hkv), dtype=np.float32)
+    want = np.zeros((prompts, layers * w.Hkv))
+    for l in range(layers):
+        qs, ks = zip(*[synth.calibration_prompt(w, l, pr, n, types[l], "cuda") for pr in range(prompts)])
+        q, k = torch.cat(qs), torch.cat(ks)
+        cv = ck.catekv_head_cv(q, k, [n] * prompts, L_init, L_rec, 0.99, 1.0, True).cpu().numpy()
+        got[:, l * w.Hkv:(l + 1) * w.Hkv] = cv
+        ref = orc.head_cv(synth.bits(q), synth.bits(k), [n] * prompts, w.L_obs, L_init, L_rec,
+                          float(np.float32(0.99)), 1.0, True)
+        want[:, l * w.Hkv:(l + 1) * w.Hkv] = ref
+    np.testing.assert_allclose(got, want, rtol=1e-3)
+    m = ck.catekv_classify_heads(got, 0.5)
+    assert np.array_equal(m, orc.static_head_mask(want, 0.5))
+    assert np.array_equal(m, types.reshape(-1))
