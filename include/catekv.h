@@ -24,7 +24,8 @@
  *   - Kernels are enqueued on the caller's stream (a cudaStream_t passed as
  *     void*); calls do not synchronise unless stated.
  *   - bf16 values are raw 16-bit patterns.  The head dimension d is the
- *     contiguous inner dimension and must be 128.  Hq / Hkv = G <= 8.
+ *     contiguous inner dimension and must be 128.  Hq / Hkv = G <= 8; where an
+ *     observation window is involved, G * L_obs <= 512.
  *   - A "segment" is the cached list of one (sequence b, KV head h), index
  *     b * Hkv + h.  All segments of a layer live in two pools, k_pool and
  *     v_pool, each [total_rows, d] bf16; segment s owns rows

@@ -71,8 +71,8 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
 }
 
 struct CvWs {
-  size_t off_segs, off_jobs, off_part, off_stats, off_A, bytes;
-  int keys_per_cta, n_chunks, rows_pad, kgroups;
+  size_t off_status, off_segs, off_jobs, off_part, off_stats, off_A, bytes;
+  int keys_per_cta, n_chunks;
   int64_t row_stride;
 };
 static CvWs cv_ws_layout(int n_segs, int G, int m_max, int L_obs) {
@@ -81,14 +81,13 @@ static CvWs cv_ws_layout(int n_segs, int G, int m_max, int L_obs) {
   while ((long)n_segs * ((m_max + kp - 1) / kp) > 148 * 4 && kp < (1 << 30)) kp *= 2;
   w.keys_per_cta = kp;
   w.n_chunks = (m_max + kp - 1) / kp;
-  w.rows_pad = score_rows_pad(G, L_obs);
-  w.kgroups = score_key_groups(L_obs);
   w.row_stride = (int64_t)align_up((size_t)m_max, 64);
   size_t o = 0;
+  w.off_status = o; o = 256;
   w.off_segs = o; o = align_up(o + sizeof(CvSeg) * (size_t)n_segs, 256);
   w.off_jobs = o; o = align_up(o + sizeof(ScoreJob) * (size_t)n_segs, 256);
-  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 8 ? n_segs : 148 * 8) * w.kgroups * w.rows_pad, 256);
-  w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * w.rows_pad, 256);
+  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 4 ? n_segs : 148 * 4) * kScoreMaxRows, 256);
+  w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * kScoreMaxRows, 256);
   w.off_A = o; o = align_up(o + sizeof(float) * (size_t)n_segs * L_obs * w.row_stride, 256);
   w.bytes = o;
   return w;
@@ -116,7 +115,7 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   const int G = Hq / Hkv;
   if (G > kMaxG) return CATEKV_ERR_UNSUPPORTED;
   if (L_obs < 1 || L_init < 0 || L_rec < 0) return CATEKV_ERR_INVALID_ARG;
-  if (L_obs > 64) return CATEKV_ERR_UNSUPPORTED;
+  if (G * L_obs > kScoreMaxRows) return CATEKV_ERR_UNSUPPORTED;
   if (!(quantile_k >= 0.f && quantile_k <= 1.f) || !(alpha >= 0.f) || isinf(alpha)) return CATEKV_ERR_INVALID_ARG;
   const int n_segs = B * Hkv;
   int m_max = 0;
@@ -143,6 +142,7 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   }
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* w8 = (uint8_t*)ws;
+  CATEKV_CUDA_TRY(cudaMemsetAsync(w8 + W.off_status, 0, 256, st));
   CATEKV_CUDA_TRY(cudaMemcpyAsync(w8 + W.off_segs, segs.data(), sizeof(CvSeg) * n_segs, cudaMemcpyHostToDevice, st));
   CATEKV_CUDA_TRY(cudaMemcpyAsync(w8 + W.off_jobs, jobs.data(), sizeof(ScoreJob) * n_segs, cudaMemcpyHostToDevice, st));
   ScoreArgs sa = {};
@@ -162,6 +162,7 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   sa.n_chunks = W.n_chunks;
   sa.stats_part = (float2*)(w8 + W.off_part);
   sa.stats = (float2*)(w8 + W.off_stats);
+  sa.status = (int32_t*)(w8 + W.off_status);
   sa.out = (float*)(w8 + W.off_A);
   sa.out_job_stride = (int64_t)L_obs * W.row_stride;
   sa.out_row_stride = W.row_stride;

@@ -1,284 +1,375 @@
-// Observation-window scoring kernels (first version: mma.sync tensor-core tiles).
+// Observation-window scoring on the 5th-generation tensor cores (tcgen05 + TMEM).
 //
-// A CTA scores `keys_per_cta` keys of one (sequence, KV head) against the L_obs window queries
-// of all G query heads of the group.  The queries (G * L_obs rows) sit in swizzled shared
-// memory for the CTA's lifetime; 64-key tiles of K stream through a two-stage cp.async
-// pipeline.  Warp w owns one 16-row slice of the window (i-tile) and a group of key columns of
-// the tile, and loops over the G heads, so that sums over heads and over window rows stay in
-// registers.  Two passes over K: row max / row sum (online, merged over CTAs by a small
-// kernel), then exp(s - max) / sum reduced to column sums (selection) or to the group-mean
-// matrix (head identification).
+// A CTA scores `keys_per_cta` keys of one (sequence, KV head) against the R = G * L_obs window
+// query rows of the group (row r = i * G + g: window row i of the group's g-th query head).
+// Q stays in shared memory for the CTA's lifetime, 128-key tiles of K stream through two
+// cp.async stages, both in the K-major SWIZZLE_128B layout the UMMA descriptors expect.
+//
+//   pass 1 (row statistics)   D[128 rows x 128 keys] = Q_rows . K_tile^T   (M = rows, N = keys)
+//       every thread owns one query row (one TMEM lane): running max and sum of exp2 over the
+//       keys are thread-local.  Partials per CTA, merged by a small kernel.
+//   pass 2 (column sums / group-mean matrix)
+//                             D[128 keys x R rows]   = K_tile . Q^T        (M = keys, N = rows)
+//       the same two shared-memory tiles with the operand roles swapped: now every thread owns
+//       one key, so C_j = sum_r exp2(x_rj - m_r) / l_r and A_ij = mean_g (...) are thread-local
+//       sums over TMEM columns and the global writes are coalesced over keys.
+//
+// One elected thread issues tcgen05.mma (8 k-steps of 16 per 128-wide head dim) and commits to an
+// mbarrier; accumulators are double- or quad-buffered in TMEM so that the MMAs of the next unit
+// run under the exp2 epilogue of the current one.  Every mbarrier wait is bounded: on expiry the
+// CTA records a status word, drains its copies, frees its TMEM and returns.
 #include <math.h>
 
 #include "score.cuh"
 
 namespace catekv {
 
-constexpr int kScoreThreads = 256;
-constexpr int kScoreWarps = 8;
-constexpr int kKeyTile = 64;
+constexpr int kScThreads = 128;
+constexpr int kKeyTile = 128;                       // keys per tile
+constexpr int kKBlockBytes = kKeyTile * 128;        // one 64-element k-block of a K tile
+constexpr int kKStageBytes = 2 * kKBlockBytes;      // K tile: 128 keys x 128 dims bf16
+constexpr uint32_t kSpinLimit = 1u << 22;
 
-int score_rows_pad(int G, int L_obs) { return G * (L_obs <= 32 ? 32 : 64); }
-int score_key_groups(int L_obs) { return kScoreWarps / (L_obs <= 32 ? 2 : 4); }
+struct ScoreShape {
+  int R;         // query rows
+  int MT;        // 128-row M tiles of pass 1
+  int q_rows;    // rows of the Q region in shared memory (MT * 128)
+  int NH, NW;    // pass 2: N halves and their width (multiple of 16)
+  int nslot1, la1, cols1;  // pass 1: TMEM slots of 128 columns, issue look-ahead, allocated columns
+  int slotw2, cols2;       // pass 2: 2 slots of slotw2 columns
+};
 
-template <int MODE, int N_IT>
-__global__ void __launch_bounds__(kScoreThreads) score_kernel(const ScoreArgs a) {
-  constexpr int ROWS_IT = N_IT * 16;          // padded window rows per head
-  constexpr int KG = kScoreWarps / N_IT;      // key groups per tile
-  constexpr int NP = 4 / KG;                  // 16-key pairs per warp per tile (N_IT=2 -> 1, N_IT=4 -> 2)
-  extern __shared__ __align__(128) uint8_t smem[];
+static ScoreShape score_shape(int G, int L_obs) {
+  ScoreShape s;
+  s.R = G * L_obs;
+  s.MT = (s.R + 127) / 128;
+  s.q_rows = s.MT * 128;
+  const int rp = (s.R + 15) / 16 * 16;
+  s.NH = rp <= 256 ? 1 : 2;
+  s.NW = s.NH == 1 ? rp : ((rp / 2 + 15) / 16 * 16);
+  s.nslot1 = s.MT >= 3 ? 4 : 2;
+  s.la1 = s.MT >= 3 ? 2 : 1;
+  s.cols1 = s.nslot1 * 128;
+  s.slotw2 = (s.NW + 31) / 32 * 32;
+  int c = 32;
+  while (c < 2 * s.slotw2) c *= 2;
+  s.cols2 = c;
+  return s;
+}
+
+// ---- tcgen05 / mbarrier wrappers ----------------------------------------------------------
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+  // K-major, SWIZZLE_128B: rows of 128 bytes, 8-row groups 1024 bytes apart
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)1 << 16;               // leading byte offset: unused for this layout
+  d |= (uint64_t)(1024 >> 4) << 32;     // stride byte offset
+  d |= (uint64_t)1 << 46;               // descriptor version
+  d |= (uint64_t)2 << 61;               // SWIZZLE_128B
+  return d;
+}
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int M, int N) {
+  // D = f32, A = B = bf16, both K-major
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(tmem_d),
+      "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+// bounded wait for a phase of an mbarrier; false if it never completed
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done = 0;
+  for (uint32_t it = 0; it < kSpinLimit && !done; ++it)
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+  return done != 0;
+}
+// 32 consecutive TMEM columns of this thread's lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// offset of the 16-byte chunk c (0..15) of row r inside a two-k-block SW128 region of `rows` rows
+__device__ __forceinline__ uint32_t sw128_off(int r, int c, int rows) {
+  return (uint32_t)((c >> 3) * rows * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kScThreads) score_tc_kernel(const ScoreArgs a, const ScoreShape sh) {
+  extern __shared__ uint8_t smem_raw[];
   const ScoreJob job = a.jobs[blockIdx.y];
   const int j_lo = job.j_begin + blockIdx.x * a.keys_per_cta;
   if (j_lo >= job.j_end) return;
   const int j_hi = min(job.j_end, j_lo + a.keys_per_cta);
   const int n_tiles = (j_hi - j_lo + kKeyTile - 1) / kKeyTile;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = lane >> 2, t = lane & 3;
-  const int it = warp % N_IT, kg = warp / N_IT;
-  const int rows_pad = a.G * ROWS_IT;
+  const int tid = threadIdx.x, warp = tid >> 5;
 
-  const uint32_t s_q = smem_u32(smem);
-  const uint32_t s_k = s_q + rows_pad * kRowBytes;
-  float2* s_stats = reinterpret_cast<float2*>(smem + rows_pad * kRowBytes + 2 * kKeyTile * kRowBytes);
-  float* s_col = reinterpret_cast<float*>(s_stats + rows_pad);  // [N_IT][64] per-i-tile column sums of the tile
+  // ---- shared memory carve-up (1024-byte aligned for the 128-byte swizzle)
+  const uint32_t s_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (s_base - smem_u32(smem_raw));
+  const uint32_t q_block = (uint32_t)sh.q_rows * 128;  // one k-block of Q
+  const uint32_t s_q = s_base;
+  const uint32_t s_k = s_q + 2 * q_block;
+  float* s_f = reinterpret_cast<float*>(smem + 2 * q_block + 2 * kKStageBytes);  // pass 1: (m, l)[MT][128]; pass 2: m'[R]
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_f + 2 * 4 * 128);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 4);
 
-  // ---- stage the group's window queries (rows >= L_obs zero) and, for pass 2, the row stats
-  for (int id = tid; id < rows_pad * 16; id += kScoreThreads) {
+  constexpr bool kStats = MODE == kScoreStats;
+  const int UPT = kStats ? sh.MT : sh.NH;          // MMA units per key tile
+  const int NSLOT = kStats ? sh.nslot1 : 2;
+  const int LA = kStats ? sh.la1 : 1;
+  const int slot_w = kStats ? 128 : sh.slotw2;
+  const int n_cols = kStats ? sh.cols1 : sh.cols2;
+  const int U = n_tiles * UPT;
+
+  // ---- stage Q (row r = i * G + g) and the first two K tiles
+  for (int id = tid; id < sh.q_rows * 16; id += kScThreads) {
     const int r = id >> 4, c = id & 15;
-    const int gh = r / ROWS_IT, i = r % ROWS_IT;
-    const int ok = i < a.L_obs ? 16 : 0;
-    const uint16_t* src = a.q_win + (((int64_t)job.b * a.Hq + job.h * a.G + gh) * a.L_obs + (ok ? i : 0)) * kD + c * 8;
-    cp_async16(s_q + tile_off(r, c), src, ok);
-  }
-  if (MODE != kScoreStats) {
-    const float2* st = a.stats + (size_t)blockIdx.y * rows_pad;
-    for (int r = tid; r < rows_pad; r += kScoreThreads) s_stats[r] = st[r];
+    const int i = r / a.G, g = r - i * a.G;
+    const int ok = r < sh.R ? 16 : 0;
+    const uint16_t* src = a.q_win + (((int64_t)job.b * a.Hq + job.h * a.G + (ok ? g : 0)) * a.L_obs + (ok ? i : 0)) * kD + c * 8;
+    cp_async16(s_q + sw128_off(r, c, sh.q_rows), src, ok);
   }
   const uint16_t* kbase = a.k + (int64_t)job.b * a.sb + (int64_t)job.h * a.sh;
-  auto issue = [&](int tile) {
+  auto load_tile = [&](int tile) {
     if (tile < n_tiles) {
-      const uint32_t sb = s_k + (tile & 1) * (kKeyTile * kRowBytes);
+      const uint32_t sb = s_k + (tile & 1) * kKStageBytes;
       const int j0 = j_lo + tile * kKeyTile;
-#pragma unroll
-      for (int i = 0; i < (kKeyTile * 16) / kScoreThreads; ++i) {
-        const int id = tid + i * kScoreThreads;
+#pragma unroll 4
+      for (int id = tid; id < kKeyTile * 16; id += kScThreads) {
         const int r = id >> 4, c = id & 15;
         const int ok = (j0 + r) < j_hi ? 16 : 0;
-        cp_async16(sb + tile_off(r, c), kbase + (int64_t)(ok ? j0 + r : job.j_begin) * a.st + c * 8, ok);
+        cp_async16(sb + sw128_off(r, c, kKeyTile), kbase + (int64_t)(ok ? j0 + r : job.j_begin) * a.st + c * 8, ok);
       }
     }
     cp_async_commit();
   };
-  issue(0);
-
-  // pass-1 state: running max / sum of the rows (it*16 + g) and (+8) of every head
-  float rm[kMaxG][2], rl[kMaxG][2];
-#pragma unroll
-  for (int gh = 0; gh < kMaxG; ++gh) rm[gh][0] = rm[gh][1] = -INFINITY, rl[gh][0] = rl[gh][1] = 0.f;
-  const int row_lo = it * 16 + g, row_hi = row_lo + 8;  // window rows of this thread
-  const float inv_g = 1.f / (float)a.G;
-  // causal: window row i sits at position n - L_obs + i and sees keys j <= that position
-  const int lim_lo = a.causal ? job.n - a.L_obs + row_lo : 0x7fffffff;
-  const int lim_hi = a.causal ? job.n - a.L_obs + row_hi : 0x7fffffff;
-
-  for (int tile = 0; tile < n_tiles; ++tile) {
-    cp_async_wait<0>();
-    __syncthreads();
-    issue(tile + 1);
-    const uint32_t kb = s_k + (tile & 1) * (kKeyTile * kRowBytes);
-    const int j0 = j_lo + tile * kKeyTile;
-#pragma unroll
-    for (int p = 0; p < NP; ++p) {
-      const int key0 = (kg * NP + p) * 16;  // first key of the pair inside the tile
-      if (j0 + key0 >= j_hi) continue;      // warp-uniform: padding columns
-      uint32_t bf[8][4];
-      {
-        const int r = key0 + (lane & 7) + ((lane >> 4) & 1) * 8;
-        const int cadd = (lane >> 3) & 1;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) ldmatrix_x4(bf[ks], kb + tile_off(r, ks * 2 + cadd));
-      }
-      // keys held by this thread: n-tile 0 -> key0 + 2t, +1 ; n-tile 1 -> key0 + 8 + 2t, +1
-      const int jA = j0 + key0 + 2 * t, jB = jA + 8;
-      float acc[2][4];  // pass 2: sum over heads of the probabilities, C-fragment layout per n-tile
-#pragma unroll
-      for (int i = 0; i < 2; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
-#pragma unroll
-      for (int gh = 0; gh < kMaxG; ++gh) {
-        if (gh >= a.G) break;
-        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-        {
-          const int r = gh * ROWS_IT + it * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-          const int cadd = lane >> 4;
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            uint32_t af[4];
-            ldmatrix_x4(af, s_q + tile_off(r, ks * 2 + cadd));
-            mma_bf16_16816(s0, af, bf[ks][0], bf[ks][1]);
-            mma_bf16_16816(s1, af, bf[ks][2], bf[ks][3]);
-          }
-        }
-        // logits in the log2 domain; masked entries are -inf
-        float x[2][4];
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-          const float* s = nt ? s1 : s0;
-          const int j = nt ? jB : jA;
-          x[nt][0] = (j < j_hi && j <= lim_lo) ? s[0] * a.scale_log2 : -INFINITY;
-          x[nt][1] = (j + 1 < j_hi && j + 1 <= lim_lo) ? s[1] * a.scale_log2 : -INFINITY;
-          x[nt][2] = (j < j_hi && j <= lim_hi) ? s[2] * a.scale_log2 : -INFINITY;
-          x[nt][3] = (j + 1 < j_hi && j + 1 <= lim_hi) ? s[3] * a.scale_log2 : -INFINITY;
-        }
-        if (MODE == kScoreStats) {
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {  // row_lo, row_hi
-            const float e0 = x[0][2 * half], e1 = x[0][2 * half + 1], e2 = x[1][2 * half], e3 = x[1][2 * half + 1];
-            const float mx = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
-            if (mx > rm[gh][half]) {  // the running max rises only a few times per row
-              rl[gh][half] *= fast_exp2(rm[gh][half] - mx);
-              rm[gh][half] = mx;
-            }
-            if (rm[gh][half] > -INFINITY) {
-              const float m = rm[gh][half];
-              rl[gh][half] += fast_exp2(e0 - m) + fast_exp2(e1 - m) + fast_exp2(e2 - m) + fast_exp2(e3 - m);
-            }
-          }
-        } else {
-          const float2 st_lo = s_stats[gh * ROWS_IT + row_lo], st_hi = s_stats[gh * ROWS_IT + row_hi];
-#pragma unroll
-          for (int nt = 0; nt < 2; ++nt) {
-            acc[nt][0] += fast_exp2(x[nt][0] - st_lo.x) * st_lo.y;
-            acc[nt][1] += fast_exp2(x[nt][1] - st_lo.x) * st_lo.y;
-            acc[nt][2] += fast_exp2(x[nt][2] - st_hi.x) * st_hi.y;
-            acc[nt][3] += fast_exp2(x[nt][3] - st_hi.x) * st_hi.y;
-          }
-        }
-      }
-      if (MODE == kScoreColsum) {
-        // sum over this warp's 16 window rows, then over warps through shared memory
-        float c0 = acc[0][0] + acc[0][2], c1 = acc[0][1] + acc[0][3];
-        float c2 = acc[1][0] + acc[1][2], c3 = acc[1][1] + acc[1][3];
-#pragma unroll
-        for (int sh = 4; sh <= 16; sh <<= 1) {
-          c0 += __shfl_xor_sync(0xffffffffu, c0, sh);
-          c1 += __shfl_xor_sync(0xffffffffu, c1, sh);
-          c2 += __shfl_xor_sync(0xffffffffu, c2, sh);
-          c3 += __shfl_xor_sync(0xffffffffu, c3, sh);
-        }
-        if (g == 0) {  // each (i-tile, key) has one writer: the sum over i-tiles below runs in a fixed order
-          float* sc = s_col + it * kKeyTile + key0;
-          sc[2 * t] = c0;
-          sc[2 * t + 1] = c1;
-          sc[8 + 2 * t] = c2;
-          sc[8 + 2 * t + 1] = c3;
-        }
-      } else if (MODE == kScoreMatrix) {
-        float* A = a.out + (size_t)blockIdx.y * a.out_job_stride;
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-          const int j = nt ? jB : jA;
-          if (row_lo < a.L_obs) {
-            if (j < j_hi) A[(size_t)row_lo * a.out_row_stride + (j - job.j_begin)] = acc[nt][0] * inv_g;
-            if (j + 1 < j_hi) A[(size_t)row_lo * a.out_row_stride + (j + 1 - job.j_begin)] = acc[nt][1] * inv_g;
-          }
-          if (row_hi < a.L_obs) {
-            if (j < j_hi) A[(size_t)row_hi * a.out_row_stride + (j - job.j_begin)] = acc[nt][2] * inv_g;
-            if (j + 1 < j_hi) A[(size_t)row_hi * a.out_row_stride + (j + 1 - job.j_begin)] = acc[nt][3] * inv_g;
-          }
-        }
-      }
+  load_tile(0);
+  load_tile(1);
+  if (kStats) {
+    for (int i = tid; i < 4 * 128; i += kScThreads) {
+      s_f[2 * i] = -INFINITY;
+      s_f[2 * i + 1] = 0.f;
     }
-    if (MODE == kScoreColsum) {
-      __syncthreads();
-      if (tid < kKeyTile) {
-        const int j = j0 + tid;
-        float c = 0.f;
-#pragma unroll
-        for (int i = 0; i < N_IT; ++i) c += s_col[i * kKeyTile + tid];
-        if (j < j_hi) a.out[(size_t)blockIdx.y * a.out_job_stride + (j - job.j_begin)] = c * inv_g;
-      }
-      // the next tile's partial sums are written after the next iteration's barrier
+  } else {
+    // m'_r = m_r + log2(l_r): exp2(x - m'_r) is the normalised probability; rows without mass get +inf (-> 0)
+    const float2* st = a.stats + (size_t)blockIdx.y * kScoreMaxRows;
+    for (int r = tid; r < sh.R; r += kScThreads) {
+      const float2 v = st[r];
+      s_f[r] = v.y > 0.f ? v.x + log2f(v.y) : INFINITY;
     }
+  }
+  if (tid == 0) {
+    for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(smem_u32(s_bar + i)));
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(s_tmem)), "r"(n_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
   cp_async_wait<0>();
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
 
-  if (MODE == kScoreStats) {
-    // per-row partials of this warp: merge the four lanes of a quad, lane t == 0 writes
-    float2* outp = a.stats_part + ((size_t)blockIdx.y * a.n_chunks * KG + (size_t)blockIdx.x * KG + kg) * rows_pad;
+  const uint32_t idesc = kStats ? umma_idesc_bf16(128, 128) : umma_idesc_bf16(128, sh.NW);
+  auto issue_unit = [&](int v) {  // thread 0 only
+    const int tile = v / UPT, sub = v - tile * UPT;
+    const uint32_t sk = s_k + (tile & 1) * kKStageBytes;
+    const uint32_t d = tmem + (uint32_t)((v % NSLOT) * slot_w);
 #pragma unroll
-    for (int gh = 0; gh < kMaxG; ++gh) {
-      if (gh >= a.G) break;
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        float m = rm[gh][half], l = rl[gh][half];
-#pragma unroll
-        for (int sh = 1; sh <= 2; sh <<= 1) {
-          const float om = __shfl_xor_sync(0xffffffffu, m, sh), ol = __shfl_xor_sync(0xffffffffu, l, sh);
-          const float mn = fmaxf(m, om);
-          const float sa = (m == -INFINITY) ? 0.f : fast_exp2(m - mn);
-          const float sb2 = (om == -INFINITY) ? 0.f : fast_exp2(om - mn);
-          l = l * sa + ol * sb2;
-          m = mn;
-        }
-        if (t == 0) outp[gh * ROWS_IT + it * 16 + g + half * 8] = make_float2(m, l);
-      }
+    for (int kk = 0; kk < 8; ++kk) {
+      const uint32_t koff = (kk & 3) * 32;
+      const uint32_t aq = s_q + (kk >> 2) * q_block + koff;
+      const uint32_t ak = sk + (kk >> 2) * kKBlockBytes + koff;
+      if (kStats)  // D[rows x keys]: A = Q rows of this M tile, B = K tile
+        umma_bf16(d, umma_desc_sw128(aq + sub * 128 * 128), umma_desc_sw128(ak), idesc, kk ? 1u : 0u);
+      else         // D[keys x rows]: A = K tile, B = Q rows of this half
+        umma_bf16(d, umma_desc_sw128(ak), umma_desc_sw128(aq + sub * sh.NW * 128), idesc, kk ? 1u : 0u);
     }
+    umma_commit(smem_u32(s_bar + (v % NSLOT)));
+  };
+  if (tid == 0)
+    for (int v = 0; v < LA && v < U; ++v) issue_unit(v);
+
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+  const float inv_g = 1.f / (float)a.G;
+  float col_acc = 0.f;  // pass 2: this key's sum over rows (colsum) or over the heads of one window row (matrix)
+  bool alive = true;
+
+  for (int u = 0; u < U; ++u) {
+    const int tile = u / UPT, sub = u - tile * UPT;
+    const int v = u + LA;
+    if (sub == 0 && tile >= 1) load_tile(tile + 1);  // into the stage of tile - 1, whose MMAs have been waited for
+    if (v < U && v % UPT == 0) {                     // the tile of unit v must have landed before its MMAs are issued
+      cp_async_wait<0>();
+      fence_async_smem();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (tid == 0 && v < U) issue_unit(v);
+    alive = __syncthreads_and(mbar_wait(smem_u32(s_bar + (u % NSLOT)), (uint32_t)((u / NSLOT) & 1)));
+    if (!alive) break;
+    tc_fence_after();
+    const uint32_t tbase = tmem + lane_base + (uint32_t)((u % NSLOT) * slot_w);
+    const int j0 = j_lo + tile * kKeyTile;
+
+    if (kStats) {
+      // this thread's query row
+      const int r = sub * 128 + tid;
+      const int i = r / a.G;
+      const int lim = a.causal ? job.n - a.L_obs + i : 0x7fffffff;  // last key this window row sees
+      float m = s_f[2 * r], l = s_f[2 * r + 1];
+      const int jmax = min(j_hi - 1, lim);  // keys j <= jmax are live
+#pragma unroll 1
+      for (int c0 = 0; c0 < kKeyTile; c0 += 32) {
+        if (j0 + c0 >= j_hi) break;  // uniform: the rest of the tile is padding
+        float x[32];
+        tmem_ld32(tbase + c0, x);
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          x[c] = (j0 + c0 + c <= jmax) ? x[c] * a.scale_log2 : -INFINITY;
+          mx = fmaxf(mx, x[c]);
+        }
+        if (mx > m) {
+          l *= fast_exp2(m - mx);
+          m = mx;
+        }
+        if (m > -INFINITY) {
+          float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            s0 += fast_exp2(x[c] - m);
+            s1 += fast_exp2(x[c + 1] - m);
+          }
+          l += s0 + s1;
+        }
+      }
+      s_f[2 * r] = m;
+      s_f[2 * r + 1] = l;
+    } else {
+      // this thread's key
+      const int j = j0 + tid;
+      const int r_begin = sub * sh.NW, r_end = min(sh.R, r_begin + sh.NW);
+      if (sub == 0) col_acc = 0.f;
+      int i = r_begin / a.G, g = r_begin - i * a.G;
+      float* A = a.out + (size_t)blockIdx.y * a.out_job_stride;
+#pragma unroll 1
+      for (int c0 = 0; r_begin + c0 < r_end; c0 += 32) {
+        float x[32];
+        tmem_ld32(tbase + c0, x);
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const int r = r_begin + c0 + c;
+          if (r < r_end) {
+            const bool seen = !a.causal || j <= job.n - a.L_obs + i;
+            const float p = seen ? fast_exp2(x[c] * a.scale_log2 - s_f[r]) : 0.f;
+            col_acc += p;
+            if (++g == a.G) {
+              if (MODE == kScoreMatrix) {
+                if (j < j_hi) A[(size_t)i * a.out_row_stride + (j - job.j_begin)] = col_acc * inv_g;
+                col_acc = 0.f;
+              }
+              g = 0;
+              ++i;
+            }
+          }
+        }
+      }
+      if (MODE == kScoreColsum && sub == UPT - 1 && j < j_hi) A[j - job.j_begin] = col_acc * inv_g;
+    }
+  }
+
+  // ---- drain, release TMEM
+  cp_async_wait<0>();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(n_cols) : "memory");
+  if (!alive) {
+    if (tid == 0) atomicExch(a.status, 1);
+    return;
+  }
+  if (kStats) {
+    float2* outp = a.stats_part + ((size_t)blockIdx.y * a.n_chunks + blockIdx.x) * kScoreMaxRows;
+    for (int r = tid; r < sh.R; r += kScThreads) outp[r] = make_float2(s_f[2 * r], s_f[2 * r + 1]);
   }
 }
 
-// Merge the per-CTA row partials: stats[job][row] = (max, 1 / sum); padding rows get (0, 0).
-// One warp per row: the lanes stride over the partials, then merge pairwise.
-__global__ void __launch_bounds__(256) score_stats_merge_kernel(const ScoreArgs a, int rows_it, int kgroups) {
+// Merge the per-CTA row partials: stats[job][row] = (max, sum).  One warp per row.
+__global__ void __launch_bounds__(256) score_stats_merge_kernel(const ScoreArgs a, int R) {
   const int jobi = blockIdx.y;
-  const int rows_pad = a.G * rows_it;
   const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  if (r >= rows_pad) return;
+  if (r >= R) return;
   const ScoreJob job = a.jobs[jobi];
+  const int used = (job.j_end - job.j_begin + a.keys_per_cta - 1) / a.keys_per_cta;
   float m = -INFINITY, l = 0.f;
-  if (r % rows_it < a.L_obs) {
-    const int used = (job.j_end - job.j_begin + a.keys_per_cta - 1) / a.keys_per_cta;
-    for (int c = lane; c < used * kgroups; c += 32) {
-      const float2 p = a.stats_part[((size_t)jobi * a.n_chunks * kgroups + c) * rows_pad + r];
-      if (p.x == -INFINITY) continue;
-      const float mn = fmaxf(m, p.x);
-      l = l * ((m == -INFINITY) ? 0.f : exp2f(m - mn)) + p.y * exp2f(p.x - mn);
-      m = mn;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float om = __shfl_xor_sync(0xffffffffu, m, o), ol = __shfl_xor_sync(0xffffffffu, l, o);
-      const float mn = fmaxf(m, om);
-      l = l * ((m == -INFINITY) ? 0.f : exp2f(m - mn)) + ol * ((om == -INFINITY) ? 0.f : exp2f(om - mn));
-      m = mn;
-    }
+  for (int c = lane; c < used; c += 32) {
+    const float2 p = a.stats_part[((size_t)jobi * a.n_chunks + c) * kScoreMaxRows + r];
+    if (p.x == -INFINITY) continue;
+    const float mn = fmaxf(m, p.x);
+    l = l * ((m == -INFINITY) ? 0.f : exp2f(m - mn)) + p.y * exp2f(p.x - mn);
+    m = mn;
   }
-  if (lane == 0) a.stats[(size_t)jobi * rows_pad + r] = (l > 0.f) ? make_float2(m, 1.f / l) : make_float2(0.f, 0.f);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o), ol = __shfl_xor_sync(0xffffffffu, l, o);
+    const float mn = fmaxf(m, om);
+    l = l * ((m == -INFINITY) ? 0.f : exp2f(m - mn)) + ol * ((om == -INFINITY) ? 0.f : exp2f(om - mn));
+    m = mn;
+  }
+  if (lane == 0) a.stats[(size_t)jobi * kScoreMaxRows + r] = make_float2(m, l);
 }
 
-template <int MODE, int N_IT>
-static int launch_one(const ScoreArgs& a, cudaStream_t stream) {
-  const int rows_pad = a.G * N_IT * 16;
-  const size_t smem = (size_t)rows_pad * kRowBytes + 2 * kKeyTile * kRowBytes + rows_pad * sizeof(float2) +
-                      N_IT * kKeyTile * sizeof(float);
-  CATEKV_CUDA_TRY(cudaFuncSetAttribute(score_kernel<MODE, N_IT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  score_kernel<MODE, N_IT><<<dim3(a.n_chunks, a.n_jobs), kScoreThreads, smem, stream>>>(a);
+static size_t score_smem_bytes(const ScoreShape& sh) {
+  return 1024 + 2 * (size_t)sh.q_rows * 128 + 2 * kKStageBytes + 2 * 4 * 128 * sizeof(float) + 4 * sizeof(uint64_t) + 16;
+}
+
+template <int MODE>
+static int launch_one(const ScoreArgs& a, const ScoreShape& sh, cudaStream_t stream) {
+  const size_t smem = score_smem_bytes(sh);
+  CATEKV_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  score_tc_kernel<MODE><<<dim3(a.n_chunks, a.n_jobs), kScThreads, smem, stream>>>(a, sh);
   CATEKV_CUDA_TRY(cudaGetLastError());
   return CATEKV_OK;
 }
 
 int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream) {
   if (a.n_jobs <= 0 || a.n_chunks <= 0) return CATEKV_OK;
-  const bool small = a.L_obs <= 32;
-  int rc = small ? launch_one<kScoreStats, 2>(a, stream) : launch_one<kScoreStats, 4>(a, stream);
+  if (a.G * a.L_obs > kScoreMaxRows || a.keys_per_cta % kKeyTile || !a.status) return CATEKV_ERR_UNSUPPORTED;
+  const ScoreShape sh = score_shape(a.G, a.L_obs);
+  int rc = launch_one<kScoreStats>(a, sh, stream);
   if (rc) return rc;
-  const int rows_it = small ? 32 : 64;
-  const int rows_pad = a.G * rows_it;
-  score_stats_merge_kernel<<<dim3((rows_pad + 7) / 8, a.n_jobs), 256, 0, stream>>>(a, rows_it, score_key_groups(a.L_obs));
+  score_stats_merge_kernel<<<dim3((sh.R + 7) / 8, a.n_jobs), 256, 0, stream>>>(a, sh.R);
   CATEKV_CUDA_TRY(cudaGetLastError());
-  if (out_mode == kScoreColsum)
-    return small ? launch_one<kScoreColsum, 2>(a, stream) : launch_one<kScoreColsum, 4>(a, stream);
-  return small ? launch_one<kScoreMatrix, 2>(a, stream) : launch_one<kScoreMatrix, 4>(a, stream);
+  return out_mode == kScoreColsum ? launch_one<kScoreColsum>(a, sh, stream) : launch_one<kScoreMatrix>(a, sh, stream);
 }
 
 }  // namespace catekv

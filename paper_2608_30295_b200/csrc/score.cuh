@@ -19,19 +19,18 @@ struct ScoreArgs {
   const ScoreJob* jobs;   // device
   int32_t n_jobs, Hq, G, L_obs, causal;
   float scale_log2;       // log2(e) / sqrt(d)
-  int32_t keys_per_cta;   // multiple of 64
+  int32_t keys_per_cta;   // multiple of 128
   int32_t n_chunks;       // grid.x: ceil(max key range / keys_per_cta)
-  float2* stats_part;     // [n_jobs][n_chunks * key_groups][rows_pad]  (row max in log2 domain, row sum)
-  float2* stats;          // [n_jobs][rows_pad]                        (row max, 1 / row sum)
+  float2* stats_part;     // [n_jobs][n_chunks][kScoreMaxRows]  per-CTA (row max in the log2 domain, row sum)
+  float2* stats;          // [n_jobs][kScoreMaxRows]            merged (row max, row sum)
+  int32_t* status;        // device word, set to 1 if a tensor-core wait ever expired (never in a healthy run)
   float* out;             // column sums C[job][j - j_begin] or matrix A[job][i][j - j_begin]
   int64_t out_job_stride, out_row_stride;
 };
 
 enum ScoreMode { kScoreStats = 0, kScoreColsum = 1, kScoreMatrix = 2 };
 
-// rows_pad = G * (16 * n_it), n_it = 2 for L_obs <= 32, 4 for L_obs <= 64
-int score_rows_pad(int G, int L_obs);
-int score_key_groups(int L_obs);
+constexpr int kScoreMaxRows = 512;  // G * L_obs may not exceed this (8 heads x 64 window rows)
 // Enqueue: pass 1 (row max / sum partials), their merge, and pass 2 (column sums or matrix).
 int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream);
 

@@ -205,8 +205,8 @@ static int keys_per_cta_for(int n_segs, int n_sc_max) {
 }
 
 struct SelWs {
-  size_t off_segs, off_jobs, off_part, off_stats, off_C, off_P, off_idx, bytes;
-  int keys_per_cta, n_chunks, rows_pad, kgroups;
+  size_t off_status, off_segs, off_jobs, off_part, off_stats, off_C, off_P, off_idx, bytes;
+  int keys_per_cta, n_chunks;
   int64_t c_stride, idx_stride;
 };
 static SelWs sel_ws_layout(int n_segs, int G, int n_max, int L_obs) {
@@ -214,15 +214,14 @@ static SelWs sel_ws_layout(int n_segs, int G, int n_max, int L_obs) {
   const int n_sc = n_max > L_obs ? n_max - L_obs : 1;
   w.keys_per_cta = keys_per_cta_for(n_segs, n_sc);
   w.n_chunks = (n_sc + w.keys_per_cta - 1) / w.keys_per_cta;
-  w.rows_pad = score_rows_pad(G, L_obs);
-  w.kgroups = score_key_groups(L_obs);
   w.c_stride = (int64_t)align_up((size_t)n_sc, 64);
   w.idx_stride = (int64_t)align_up((size_t)n_max, 64);
   size_t o = 0;
+  w.off_status = o; o = 256;
   w.off_segs = o; o = align_up(o + sizeof(SelSeg) * (size_t)n_segs, 256);
   w.off_jobs = o; o = align_up(o + sizeof(ScoreJob) * (size_t)n_segs, 256);
-  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 8 ? n_segs : 148 * 8) * w.kgroups * w.rows_pad, 256);
-  w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * w.rows_pad, 256);
+  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 4 ? n_segs : 148 * 4) * kScoreMaxRows, 256);
+  w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * kScoreMaxRows, 256);
   w.off_C = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.c_stride, 256);
   w.off_P = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.c_stride, 256);
   w.off_idx = o; o = align_up(o + sizeof(int32_t) * (size_t)n_segs * w.idx_stride, 256);
@@ -247,7 +246,7 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   const int G = p->Hq / p->Hkv;
   if (G > kMaxG) return CATEKV_ERR_UNSUPPORTED;
   if (p->L_obs < 1 || p->sink < 0 || p->local < p->L_obs || p->budget_consistent < 0) return CATEKV_ERR_INVALID_ARG;
-  if (p->L_obs > 64) return CATEKV_ERR_UNSUPPORTED;
+  if (G * p->L_obs > kScoreMaxRows) return CATEKV_ERR_UNSUPPORTED;
   if (!(p->eta_adaptive >= 0.f)) return CATEKV_ERR_INVALID_ARG;
   if (p->pool_mode == CATEKV_POOL_CHUNK) {
     if (p->pool_param < 1) return CATEKV_ERR_INVALID_ARG;
@@ -325,6 +324,7 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   uint8_t* w8 = (uint8_t*)ws;
   SelSeg* d_segs = (SelSeg*)(w8 + W.off_segs);
   ScoreJob* d_jobs = (ScoreJob*)(w8 + W.off_jobs);
+  CATEKV_CUDA_TRY(cudaMemsetAsync(w8 + W.off_status, 0, 256, st));
   CATEKV_CUDA_TRY(cudaMemcpyAsync(d_segs, segs.data(), sizeof(SelSeg) * n_segs, cudaMemcpyHostToDevice, st));
   if (!jobs.empty()) {
     CATEKV_CUDA_TRY(cudaMemcpyAsync(d_jobs, jobs.data(), sizeof(ScoreJob) * jobs.size(), cudaMemcpyHostToDevice, st));
@@ -345,6 +345,7 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
     sa.n_chunks = (n_sc_jobs_max + W.keys_per_cta - 1) / W.keys_per_cta;
     sa.stats_part = (float2*)(w8 + W.off_part);
     sa.stats = (float2*)(w8 + W.off_stats);
+    sa.status = (int32_t*)(w8 + W.off_status);
     sa.out = (float*)(w8 + W.off_C);
     sa.out_job_stride = W.c_stride;
     sa.out_row_stride = 0;

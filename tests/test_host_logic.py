@@ -173,7 +173,7 @@ def test_select_argument_checks(ck):
     assert call(local=8) == ck.ERR_INVALID_ARG       # local window shorter than the observation window
     assert call(d=64) == ck.ERR_UNSUPPORTED
     assert call(Hq=18) == ck.ERR_UNSUPPORTED
-    assert call(L_obs=65, local=65) == ck.ERR_UNSUPPORTED
+    assert call(L_obs=129, local=129) == ck.ERR_UNSUPPORTED  # G * L_obs = 516 > 512
     assert call(mode=2, param=4) == ck.ERR_INVALID_ARG  # even window
     assert call(mode=1, param=0) == ck.ERR_INVALID_ARG
     assert call(mode=9) == ck.ERR_UNSUPPORTED
@@ -191,7 +191,7 @@ def test_head_cv_argument_checks(ck):
     assert call(d=64) == ck.ERR_UNSUPPORTED
     assert call(k=1.5) == ck.ERR_INVALID_ARG
     assert call(L_init=60, L_rec=40) == ck.ERR_INVALID_ARG   # no column left
-    assert call(L_obs=128) == ck.ERR_UNSUPPORTED
+    assert call(L_obs=129) == ck.ERR_UNSUPPORTED
     assert call(wsb=8) == ck.ERR_WORKSPACE
     assert ck.catekv_head_cv_workspace_bytes(1, 8, 2, 100, 16, 60, 40) == 0
 
