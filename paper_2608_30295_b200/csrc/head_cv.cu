@@ -86,7 +86,7 @@ static CvWs cv_ws_layout(int n_segs, int G, int m_max, int L_obs) {
   w.off_status = o; o = 256;
   w.off_segs = o; o = align_up(o + sizeof(CvSeg) * (size_t)n_segs, 256);
   w.off_jobs = o; o = align_up(o + sizeof(ScoreJob) * (size_t)n_segs, 256);
-  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 4 ? n_segs : 148 * 4) * kScoreMaxRows, 256);
+  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 4 ? n_segs : 148 * 4) * 2 * kScoreMaxRows, 256);
   w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * kScoreMaxRows, 256);
   w.off_A = o; o = align_up(o + sizeof(float) * (size_t)n_segs * L_obs * w.row_stride, 256);
   w.bytes = o;

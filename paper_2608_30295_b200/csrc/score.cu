@@ -24,7 +24,7 @@
 
 namespace catekv {
 
-constexpr int kScThreads = 128;
+constexpr int kScThreads = 256;                    // 8 warps: two per TMEM lane quarter, each takes half the columns
 constexpr int kKeyTile = 128;                       // keys per tile
 constexpr int kKBlockBytes = kKeyTile * 128;        // one 64-element k-block of a K tile
 constexpr int kKStageBytes = 2 * kKBlockBytes;      // K tile: 128 keys x 128 dims bf16
@@ -44,9 +44,13 @@ static ScoreShape score_shape(int G, int L_obs) {
   s.R = G * L_obs;
   s.MT = (s.R + 127) / 128;
   s.q_rows = s.MT * 128;
-  const int rp = (s.R + 15) / 16 * 16;
-  s.NH = rp <= 256 ? 1 : 2;
-  s.NW = s.NH == 1 ? rp : ((rp / 2 + 15) / 16 * 16);
+  // pass 2 splits the R rows into NH halves of NW columns: a multiple of 16 (UMMA N) and of G (so that the
+  // G heads of one window row never straddle two halves)
+  int unit = 16;
+  while (unit % G) unit += 16;
+  s.NH = (s.R + unit - 1) / unit * unit <= 256 ? 1 : 2;
+  s.NW = ((s.R + s.NH - 1) / s.NH + unit - 1) / unit * unit;
+  if (s.NH * s.NW > s.q_rows) s.q_rows = (s.NH * s.NW + 7) / 8 * 8;
   s.nslot1 = s.MT >= 3 ? 4 : 2;
   s.la1 = s.MT >= 3 ? 2 : 1;
   s.cols1 = s.nslot1 * 128;
@@ -134,7 +138,7 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const ScoreArgs a,
   const uint32_t s_q = s_base;
   const uint32_t s_k = s_q + 2 * q_block;
   float* s_f = reinterpret_cast<float*>(smem + 2 * q_block + 2 * kKStageBytes);  // pass 1: (m, l)[MT][128]; pass 2: m'[R]
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_f + 2 * 4 * 128);
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_f + 4 * kScoreMaxRows);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 4);
 
   constexpr bool kStats = MODE == kScoreStats;
@@ -170,7 +174,7 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const ScoreArgs a,
   load_tile(0);
   load_tile(1);
   if (kStats) {
-    for (int i = tid; i < 4 * 128; i += kScThreads) {
+    for (int i = tid; i < 2 * kScoreMaxRows; i += kScThreads) {
       s_f[2 * i] = -INFINITY;
       s_f[2 * i + 1] = 0.f;
     }
@@ -217,9 +221,13 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const ScoreArgs a,
   if (tid == 0)
     for (int v = 0; v < LA && v < U; ++v) issue_unit(v);
 
-  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+  // warp w reads TMEM lanes 32 * (w % 4) ...; warps 0-3 take the first half of a unit's columns, warps 4-7 the second
+  const int lane_row = (warp & 3) * 32 + (tid & 31);  // this thread's TMEM lane: a query row (pass 1) or a key (pass 2)
+  const int half = warp >> 2;
+  const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
   const float inv_g = 1.f / (float)a.G;
-  float col_acc = 0.f;  // pass 2: this key's sum over rows (colsum) or over the heads of one window row (matrix)
+  float* s_col = s_f + kScoreMaxRows;  // pass 2: [2][128] per-half sums of a key
+  float col_acc = 0.f;                 // pass 2, column sums: this key's sum over this thread's rows of the tile
   bool alive = true;
 
   for (int u = 0; u < U; ++u) {
@@ -241,69 +249,105 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const ScoreArgs a,
     const int j0 = j_lo + tile * kKeyTile;
 
     if (kStats) {
-      // this thread's query row
-      const int r = sub * 128 + tid;
+      // this thread's query row, keys [64 * half, 64 * half + 64) of the tile
+      const int r = sub * 128 + lane_row;
       const int i = r / a.G;
       const int lim = a.causal ? job.n - a.L_obs + i : 0x7fffffff;  // last key this window row sees
-      float m = s_f[2 * r], l = s_f[2 * r + 1];
-      const int jmax = min(j_hi - 1, lim);  // keys j <= jmax are live
+      const int jmax = min(j_hi - 1, lim);                          // keys j <= jmax are live
+      float m = s_f[2 * (half * kScoreMaxRows + r)], l = s_f[2 * (half * kScoreMaxRows + r) + 1];
 #pragma unroll 1
-      for (int c0 = 0; c0 < kKeyTile; c0 += 32) {
+      for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 32) {
         if (j0 + c0 >= j_hi) break;  // uniform: the rest of the tile is padding
         float x[32];
         tmem_ld32(tbase + c0, x);
-        float mx = -INFINITY;
+        if (j0 + c0 + 31 > jmax) {  // tail of the key range or the causal edge: mask entry by entry
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          x[c] = (j0 + c0 + c <= jmax) ? x[c] * a.scale_log2 : -INFINITY;
-          mx = fmaxf(mx, x[c]);
+          for (int c = 0; c < 32; ++c) x[c] = (j0 + c0 + c <= jmax) ? x[c] : -INFINITY;
         }
+        float mx = x[0];
+#pragma unroll
+        for (int c = 1; c < 32; ++c) mx = fmaxf(mx, x[c]);
+        mx *= a.scale_log2;  // the scale is positive: the max commutes with it
         if (mx > m) {
           l *= fast_exp2(m - mx);
           m = mx;
         }
         if (m > -INFINITY) {
-          float s0 = 0.f, s1 = 0.f;
+          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-          for (int c = 0; c < 32; c += 2) {
-            s0 += fast_exp2(x[c] - m);
-            s1 += fast_exp2(x[c + 1] - m);
+          for (int c = 0; c < 32; c += 4) {
+            s0 += fast_exp2(fmaf(x[c], a.scale_log2, -m));
+            s1 += fast_exp2(fmaf(x[c + 1], a.scale_log2, -m));
+            s2 += fast_exp2(fmaf(x[c + 2], a.scale_log2, -m));
+            s3 += fast_exp2(fmaf(x[c + 3], a.scale_log2, -m));
           }
-          l += s0 + s1;
+          l += (s0 + s1) + (s2 + s3);
         }
       }
-      s_f[2 * r] = m;
-      s_f[2 * r + 1] = l;
+      s_f[2 * (half * kScoreMaxRows + r)] = m;
+      s_f[2 * (half * kScoreMaxRows + r) + 1] = l;
     } else {
-      // this thread's key
-      const int j = j0 + tid;
+      // this thread's key; the unit's rows [r_begin, r_end) are cut, at a multiple of G, between the two halves
+      const int j = j0 + lane_row;
       const int r_begin = sub * sh.NW, r_end = min(sh.R, r_begin + sh.NW);
-      if (sub == 0) col_acc = 0.f;
-      int i = r_begin / a.G, g = r_begin - i * a.G;
-      float* A = a.out + (size_t)blockIdx.y * a.out_job_stride;
+      // column sums cut at a multiple of 32 columns, the matrix at a multiple of G (whole window rows per thread)
+      const int cut = MODE == kScoreColsum ? min(r_end, r_begin + ((r_end - r_begin) / 2 + 31) / 32 * 32)
+                                           : r_begin + ((r_end - r_begin) / 2 / a.G) * a.G;
+      const int r0 = half ? cut : r_begin, r1 = half ? r_end : cut;
+      if (MODE == kScoreColsum) {
+        if (sub == 0) col_acc = 0.f;
+        float c0s = 0.f, c1s = 0.f, c2s = 0.f, c3s = 0.f;
 #pragma unroll 1
-      for (int c0 = 0; r_begin + c0 < r_end; c0 += 32) {
-        float x[32];
-        tmem_ld32(tbase + c0, x);
+        for (int rr = r0; rr < r1; rr += 32) {
+          float x[32];
+          tmem_ld32(tbase + (rr - r_begin), x);
+          if (rr + 32 <= r1) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const int r = r_begin + c0 + c;
-          if (r < r_end) {
-            const bool seen = !a.causal || j <= job.n - a.L_obs + i;
-            const float p = seen ? fast_exp2(x[c] * a.scale_log2 - s_f[r]) : 0.f;
-            col_acc += p;
-            if (++g == a.G) {
-              if (MODE == kScoreMatrix) {
-                if (j < j_hi) A[(size_t)i * a.out_row_stride + (j - job.j_begin)] = col_acc * inv_g;
-                col_acc = 0.f;
+            for (int c = 0; c < 32; c += 4) {
+              const float4 mm = *reinterpret_cast<const float4*>(s_f + rr + c);  // rr is a multiple of 16
+              c0s += fast_exp2(fmaf(x[c], a.scale_log2, -mm.x));
+              c1s += fast_exp2(fmaf(x[c + 1], a.scale_log2, -mm.y));
+              c2s += fast_exp2(fmaf(x[c + 2], a.scale_log2, -mm.z));
+              c3s += fast_exp2(fmaf(x[c + 3], a.scale_log2, -mm.w));
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c)
+              if (rr + c < r1) c0s += fast_exp2(fmaf(x[c], a.scale_log2, -s_f[rr + c]));
+          }
+        }
+        col_acc += (c0s + c1s) + (c2s + c3s);
+        if (sub == UPT - 1) {
+          s_col[half * 128 + lane_row] = col_acc;
+          __syncthreads();
+          if (half == 0 && j < j_hi)
+            a.out[(size_t)blockIdx.y * a.out_job_stride + (j - job.j_begin)] = (s_col[lane_row] + s_col[128 + lane_row]) * inv_g;
+          // s_col is rewritten one tile later, after several barriers
+        }
+      } else {
+        // group-mean matrix: rows come in runs of G heads per window row; r0 is a multiple of G
+        float* A = a.out + (size_t)blockIdx.y * a.out_job_stride;
+        int i = r0 / a.G, g = 0;
+        float acc = 0.f;
+#pragma unroll 1
+        for (int rr = r0; rr < r1; rr += 32) {
+          float x[32];
+          tmem_ld32(tbase + (rr - r_begin), x);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            if (rr + c < r1) {
+              const bool seen = !a.causal || j <= job.n - a.L_obs + i;
+              acc += seen ? fast_exp2(fmaf(x[c], a.scale_log2, -s_f[rr + c])) : 0.f;
+              if (++g == a.G) {
+                if (j < j_hi) A[(size_t)i * a.out_row_stride + (j - job.j_begin)] = acc * inv_g;
+                acc = 0.f;
+                g = 0;
+                ++i;
               }
-              g = 0;
-              ++i;
             }
           }
         }
       }
-      if (MODE == kScoreColsum && sub == UPT - 1 && j < j_hi) A[j - job.j_begin] = col_acc * inv_g;
     }
   }
 
@@ -317,8 +361,10 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const ScoreArgs a,
     return;
   }
   if (kStats) {
-    float2* outp = a.stats_part + ((size_t)blockIdx.y * a.n_chunks + blockIdx.x) * kScoreMaxRows;
-    for (int r = tid; r < sh.R; r += kScThreads) outp[r] = make_float2(s_f[2 * r], s_f[2 * r + 1]);
+    // two partials per CTA and row: one per column half
+    float2* outp = a.stats_part + ((size_t)blockIdx.y * a.n_chunks + blockIdx.x) * (2 * kScoreMaxRows);
+    for (int r = tid; r < 2 * kScoreMaxRows; r += kScThreads)
+      if ((r & (kScoreMaxRows - 1)) < sh.R) outp[r] = make_float2(s_f[2 * r], s_f[2 * r + 1]);
   }
 }
 
@@ -331,8 +377,8 @@ __global__ void __launch_bounds__(256) score_stats_merge_kernel(const ScoreArgs 
   const ScoreJob job = a.jobs[jobi];
   const int used = (job.j_end - job.j_begin + a.keys_per_cta - 1) / a.keys_per_cta;
   float m = -INFINITY, l = 0.f;
-  for (int c = lane; c < used; c += 32) {
-    const float2 p = a.stats_part[((size_t)jobi * a.n_chunks + c) * kScoreMaxRows + r];
+  for (int c = lane; c < 2 * used; c += 32) {
+    const float2 p = a.stats_part[((size_t)jobi * a.n_chunks + (c >> 1)) * (2 * kScoreMaxRows) + (c & 1) * kScoreMaxRows + r];
     if (p.x == -INFINITY) continue;
     const float mn = fmaxf(m, p.x);
     l = l * ((m == -INFINITY) ? 0.f : exp2f(m - mn)) + p.y * exp2f(p.x - mn);
@@ -349,7 +395,7 @@ __global__ void __launch_bounds__(256) score_stats_merge_kernel(const ScoreArgs 
 }
 
 static size_t score_smem_bytes(const ScoreShape& sh) {
-  return 1024 + 2 * (size_t)sh.q_rows * 128 + 2 * kKStageBytes + 2 * 4 * 128 * sizeof(float) + 4 * sizeof(uint64_t) + 16;
+  return 1024 + 2 * (size_t)sh.q_rows * 128 + 2 * kKStageBytes + 4 * kScoreMaxRows * sizeof(float) + 4 * sizeof(uint64_t) + 16;
 }
 
 template <int MODE>

@@ -220,7 +220,7 @@ static SelWs sel_ws_layout(int n_segs, int G, int n_max, int L_obs) {
   w.off_status = o; o = 256;
   w.off_segs = o; o = align_up(o + sizeof(SelSeg) * (size_t)n_segs, 256);
   w.off_jobs = o; o = align_up(o + sizeof(ScoreJob) * (size_t)n_segs, 256);
-  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 4 ? n_segs : 148 * 4) * kScoreMaxRows, 256);
+  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 4 ? n_segs : 148 * 4) * 2 * kScoreMaxRows, 256);
   w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * kScoreMaxRows, 256);
   w.off_C = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.c_stride, 256);
   w.off_P = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.c_stride, 256);
