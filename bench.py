@@ -162,10 +162,16 @@ def make_step_inputs(w, n_layers, dev, n_sets=2):
     return sets
 
 
+FUSED = True  # per layer: catekv_append_decode_attn (one attention launch) instead of catekv_append + catekv_decode_attn
+
+
 def decode_step(ck, model, q, kn, vn, out):
     for l, m in enumerate(model):
-        ck.catekv_append(m["cache"], kn[l], vn[l])
-        ck.catekv_decode_attn(m["cache"], q[l], m["plan"], out[l])
+        if FUSED:
+            ck.catekv_append_decode_attn(m["cache"], kn[l], vn[l], q[l], m["plan"], out[l])
+        else:
+            ck.catekv_append(m["cache"], kn[l], vn[l])
+            ck.catekv_decode_attn(m["cache"], q[l], m["plan"], out[l])
 
 
 def capture_step(ck, model, q, kn, vn, out):
@@ -411,6 +417,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying "
                     "a captured CUDA graph of the step")
+    ap.add_argument("--no-fused", action="store_true", help="catekv_append + catekv_decode_attn as two calls per layer")
     ap.add_argument("--no-extras", action="store_true", help="skip the other configs, head_cv and the oracle timing")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -450,6 +457,8 @@ def main():
     n_layers = args.layers or w.layers
     total_steps = 3 * (args.warmup + args.steps) + 16
     graph = not args.no_graph
+    global FUSED
+    FUSED = not args.no_fused
     model, sel_ms = build_model(ck, w, dev, max_new=total_steps, layers=n_layers)
 
     vis = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
@@ -475,7 +484,9 @@ def main():
                    "window": w.L_obs, "replicas": world,
                    "l2": "no flush: per-layer working set %.0f MB x %d layers, far above the 126 MB L2"
                          % (bytes_per_layer / 1e6, n_layers),
-                   "step": "one decode token of the whole model: per layer catekv_append + catekv_decode_attn",
+                   "step": "one decode token of the whole model: per layer " +
+                           ("catekv_append_decode_attn (append fused into the attention launch)" if FUSED
+                            else "catekv_append + catekv_decode_attn"),
                    "launch": "CUDA graph replay of the step" if graph else "host launches"},
         "us_per_layer_step": ms * 1e3 / n_layers,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -485,7 +496,8 @@ def main():
                      "frac_of_8TBs": achieved / 8000.0, "combine_us": comb_us},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e},
-        "gpu_launches": args.steps * n_layers * (2 + (1 if any(ck.plan_header(m["plan"])["n_slots"] for m in model) else 0)),
+        "gpu_launches": args.steps * n_layers * ((1 if FUSED else 2) +
+                                                 (1 if any(ck.plan_header(m["plan"])["n_slots"] for m in model) else 0)),
         "clocks": clocks,
         "select_compact": {"ms_per_layer": float(np.mean(sel_ms[1:] or sel_ms)), "layers": n_layers},
     }

@@ -222,6 +222,11 @@ int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, void* plan_h
  *   lse_out  device float [B, Hq] or NULL: natural-log sum of exp(logits); -inf if empty
  *   plan_host / plan_dev  the plan built by catekv_decode_plan for this cache
  *   ws       device scratch of at least catekv_decode_workspace_bytes(...)
+ *
+ * Ordering: the kernels use programmatic dependent launch.  They wait for all earlier work of the
+ * stream before they read lengths, queries or appended rows, but they may request cache rows that
+ * were valid when the plan was built while the previous kernel is still finishing.  Such rows must
+ * therefore not be rewritten (by catekv_select_compact, say) between catekv_decode_plan and this call.
  */
 int catekv_decode_attn(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
                        int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
@@ -240,6 +245,17 @@ int catekv_decode_partials(const catekv_cache* cache, const void* q, int32_t Hq,
 int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
                           int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                           size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream);
+
+/*
+ * catekv_append followed by catekv_decode_attn, as one call with one attention launch: the CTA that
+ * owns the end of a segment takes the decoded token's row from k_new / v_new, attends to it and stores
+ * it in the pool; seg_len grows by one (device and host mirror).  Same results as the two calls.
+ * CATEKV_ERR_CAPACITY (nothing launched) if any segment is full.
+ */
+int catekv_append_decode_attn(catekv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t Hq,
+                              float sm_scale, void* out, int32_t out_dtype, float* lse_out, const void* plan_host,
+                              const void* plan_dev, size_t plan_bytes, void* ws, size_t ws_bytes,
+                              catekv_stream stream);
 
 /*
  * catekv_decode_attn for callers that cannot hand over scratch memory.  (The paper has no

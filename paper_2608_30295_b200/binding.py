@@ -75,6 +75,8 @@ def _load():
         "catekv_decode_attn": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
         "catekv_decode_partials": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
         "catekv_decode_combine": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
+        "catekv_append_decode_attn": (C.c_int, [C.POINTER(CacheStruct), vp, vp, vp, i32, f32, vp, i32, vp, vp, vp, sz,
+                                                vp, sz, vp]),
         "catekv_decode_attn_noalloc": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp]),
     }
     for name, (res, args) in sig.items():
@@ -212,6 +214,18 @@ def catekv_decode_partials(cache: Cache, q: torch.Tensor, plan: DecodePlan, out:
 def catekv_decode_combine(cache: Cache, q: torch.Tensor, plan: DecodePlan, out: torch.Tensor,
                           lse_out: Optional[torch.Tensor] = None, sm_scale: float = 0.0):
     _decode_call(_lib.catekv_decode_combine, "catekv_decode_combine", cache, q, plan, out, lse_out, sm_scale)
+
+
+def catekv_append_decode_attn(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor, q: torch.Tensor,
+                              plan: DecodePlan, out: torch.Tensor, lse_out: Optional[torch.Tensor] = None,
+                              sm_scale: float = 0.0):
+    assert q.is_contiguous() and out.is_contiguous() and k_new.is_contiguous() and v_new.is_contiguous()
+    od = OUT_BF16 if out.dtype == torch.bfloat16 else OUT_FP32
+    assert out.dtype in (torch.bfloat16, torch.float32) and q.dtype == torch.bfloat16
+    _check(_lib.catekv_append_decode_attn(C.byref(cache.struct), k_new.data_ptr(), v_new.data_ptr(), q.data_ptr(),
+                                          q.shape[1], sm_scale, out.data_ptr(), od, _dev_ptr(lse_out),
+                                          plan.host.data_ptr(), plan.dev.data_ptr(), plan.bytes, plan.ws.data_ptr(),
+                                          plan.ws_bytes, _stream()), "catekv_append_decode_attn")
 
 
 NOALLOC_SCRATCH_BYTES = 4 << 20

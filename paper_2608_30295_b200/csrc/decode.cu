@@ -85,10 +85,12 @@ static size_t ws_layout(int n_segs, int num_ctas, size_t* off_lse) {
 // Attention partials
 // ------------------------------------------------------------------------------------------
 struct DecodeArgs {
-  const uint8_t* k_pool;
-  const uint8_t* v_pool;
+  uint8_t* k_pool;
+  uint8_t* v_pool;
   const int32_t* seg_off;
-  const int32_t* seg_len;
+  int32_t* seg_len;
+  const uint8_t* k_new;  // fused append: this step's [B*Hkv, d] rows, else null
+  const uint8_t* v_new;
   const uint16_t* q;  // [B, Hq, d]
   int32_t Hq, Hkv, G;
   float scale_log2;  // sm_scale * log2(e)
@@ -114,11 +116,13 @@ constexpr int kDecodeSmem = kStages * (kStageBytes + kQSlotBytes) + 2 * kMergeSl
 struct ItemCursor {
   int seg, t0, t1, slot, last;
   int np;            // tiles of the plan-time rows
-  int live;          // current segment length (meaningful if last)
+  int live;          // rows to attend to: current segment length (plus the row being appended), if last
+  int new_row;       // fused append: the segment-relative row that comes from k_new / v_new, else -1
   int64_t row_base;
 };
 
-__device__ __forceinline__ ItemCursor make_cursor(const DecodeArgs& a, const WorkItem& w) {
+// the part of a cursor that needs only the plan
+__device__ __forceinline__ ItemCursor plan_cursor(const WorkItem& w) {
   ItemCursor c;
   c.seg = w.seg;
   c.t0 = w.t0;
@@ -127,17 +131,31 @@ __device__ __forceinline__ ItemCursor make_cursor(const DecodeArgs& a, const Wor
   c.last = w.last;
   c.row_base = w.row_base;
   c.np = (w.t1 - w.t0 + kTile - 1) / kTile;
-  c.live = w.last ? __ldg(a.seg_len + w.seg) : w.t1;
+  c.live = w.t1;
+  c.new_row = -1;
   return c;
 }
-__device__ __forceinline__ ItemCursor read_item(const DecodeArgs& a, int it) {
-  const int4* p = reinterpret_cast<const int4*>(a.items + it);
-  const int4 x = __ldg(p), y = __ldg(p + 1);
+// the part that reads what earlier kernels wrote: the live length (a plain load: with a fused append this
+// kernel itself updates the length when it is done with the segment)
+__device__ __forceinline__ void live_cursor(const DecodeArgs& a, ItemCursor& c) {
+  if (c.last) {
+    const int len = *reinterpret_cast<const volatile int32_t*>(a.seg_len + c.seg);
+    c.new_row = a.k_new ? len : -1;
+    c.live = a.k_new ? len + 1 : len;
+  }
+}
+__device__ __forceinline__ WorkItem unpack_item(const int4& x, const int4& y) {
   WorkItem w;
   w.seg = x.x; w.t0 = x.y; w.t1 = x.z; w.slot = x.w;
   w.row_base = (int64_t)(((uint64_t)(uint32_t)y.y << 32) | (uint32_t)y.x);
   w.last = y.z; w.reserved = 0;
-  return make_cursor(a, w);
+  return w;
+}
+__device__ __forceinline__ ItemCursor read_item(const DecodeArgs& a, int it) {
+  const int4* p = reinterpret_cast<const int4*>(a.items + it);
+  ItemCursor c = plan_cursor(unpack_item(__ldg(p), __ldg(p + 1)));
+  live_cursor(a, c);
+  return c;
 }
 // tiles of the item: plan-time tiles plus tiles of the appended rows; at least one
 __device__ __forceinline__ int item_tiles(const ItemCursor& c) {
@@ -180,61 +198,87 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     // the plan was uploaded by a copy that precedes the previous kernel: it may be read before the wait
     const int4* hp = reinterpret_cast<const int4*>(a.ctas + blockIdx.x);
     const int4 h0 = __ldg(hp), x = __ldg(hp + 1), y = __ldg(hp + 2);
-    pdl_wait();  // from here on: lengths, queries and cache rows written by earlier kernels
     item_begin = h0.x;
     item_end = h0.y;
     if (item_begin >= item_end) return;
-    WorkItem w;
-    w.seg = x.x; w.t0 = x.y; w.t1 = x.z; w.slot = x.w;
-    w.row_base = (int64_t)(((uint64_t)(uint32_t)y.y << 32) | (uint32_t)y.x);
-    w.last = y.z; w.reserved = 0;
-    pc = make_cursor(a, w);
+    pc = plan_cursor(unpack_item(x, y));
   }
-  const ItemCursor first = pc;
 
   const uint32_t s_stage = smem_u32(smem);
   const uint32_t s_q = s_stage + kStages * kStageBytes;
   float* merge = reinterpret_cast<float*>(smem + kStages * (kStageBytes + kQSlotBytes));
 
-  // ---- producer: issues one tile (and the item's queries with its first tile) per call
+  // ---- producer
   int p_item = item_begin, p_tile = 0, p_seq = 0;
-  auto issue = [&]() {
-    if (p_item < item_end) {
-      const uint32_t sb = s_stage + (p_seq % kStages) * kStageBytes;
-      int start, rows_left;
-      tile_rows(pc, p_tile, start, rows_left);
-      const int64_t row0 = pc.row_base + (start - pc.t0);
+  auto issue_tile = [&]() {  // tile p_tile of the producer's item into stage p_seq % kStages
+    const uint32_t sb = s_stage + (p_seq % kStages) * kStageBytes;
+    int start, rows_left;
+    tile_rows(pc, p_tile, start, rows_left);
+    const int64_t row0 = pc.row_base + (start - pc.t0);
+    const int new_r = pc.new_row - start;  // tile row that is being appended by this call, if in [0, kTile)
 #pragma unroll
-      for (int i = 0; i < (kTile * 16) / kDecodeThreads; ++i) {
-        const int id = tid + i * kDecodeThreads;
-        const int r = id >> 4, c = id & 15;
-        const int ok = r < rows_left ? 16 : 0;
-        const int64_t goff = (ok ? row0 + r : 0) * kRowBytes + c * 16;  // padding rows read nothing
-        const uint32_t so = tile_off(r, c);
+    for (int i = 0; i < (kTile * 16) / kDecodeThreads; ++i) {
+      const int id = tid + i * kDecodeThreads;
+      const int r = id >> 4, c = id & 15;
+      const int ok = r < rows_left ? 16 : 0;
+      const int64_t goff = (ok ? row0 + r : 0) * kRowBytes + c * 16;  // padding rows read nothing
+      const uint32_t so = tile_off(r, c);
+      if (ok && r == new_r && pc.new_row >= 0) {  // only inside the tile's valid rows (never in a plan-time tile)
+        // the decoded token's row: attend to it from k_new / v_new and store it in the pool
+        const size_t noff = (size_t)pc.seg * kRowBytes + c * 16;
+        cp_async16(sb + so, a.k_new + noff, 16);
+        cp_async16(sb + kTile * kRowBytes + so, a.v_new + noff, 16);
+        *reinterpret_cast<uint4*>(a.k_pool + goff) = *reinterpret_cast<const uint4*>(a.k_new + noff);
+        *reinterpret_cast<uint4*>(a.v_pool + goff) = *reinterpret_cast<const uint4*>(a.v_new + noff);
+      } else {
         cp_async16(sb + so, a.k_pool + goff, ok);
         cp_async16(sb + kTile * kRowBytes + so, a.v_pool + goff, ok);
       }
-      if (p_tile == 0) {
-        // the group's G query rows; heads >= G are zero-filled
-        const uint32_t qb = s_q + ((p_item - item_begin) % kStages) * kQSlotBytes;
-        const int b = pc.seg / a.Hkv, h = pc.seg % a.Hkv;
-        const int r = tid >> 4, c = tid & 15;  // 128 threads = 8 rows x 16 chunks
-        const int ok = r < a.G ? 16 : 0;
-        const uint16_t* src = a.q + ((int64_t)b * a.Hq + h * a.G + (ok ? r : 0)) * kD + c * 8;
-        cp_async16(qb + r * kRowBytes + c * 16, src, ok);
-      }
-      ++p_seq;
-      // the plan-time tiles need no look at the live length; only past them is it consulted
-      if (++p_tile >= pc.np && p_tile >= item_tiles(pc)) {
-        p_tile = 0;
-        if (++p_item < item_end) pc = read_item(a, p_item);
-      }
+    }
+  };
+  auto issue_q = [&](int ordinal, int seg) {  // the group's G query rows; heads >= G are zero-filled
+    const uint32_t qb = s_q + (ordinal % kStages) * kQSlotBytes;
+    const int b = seg / a.Hkv, h = seg % a.Hkv;
+    const int r = tid >> 4, c = tid & 15;  // 128 threads = 8 rows x 16 chunks
+    const int ok = r < a.G ? 16 : 0;
+    const uint16_t* src = a.q + ((int64_t)b * a.Hq + h * a.G + (ok ? r : 0)) * kD + c * 8;
+    cp_async16(qb + r * kRowBytes + c * 16, src, ok);
+  };
+  auto advance = [&]() {  // after a tile was issued; the plan-time tiles need no look at the live length
+    ++p_seq;
+    if (++p_tile >= pc.np && p_tile >= item_tiles(pc)) {
+      p_tile = 0;
+      if (++p_item < item_end) pc = read_item(a, p_item);
+    }
+  };
+  auto issue = [&]() {  // one tile (with the item's queries if it is the item's first) = one commit group
+    if (p_item < item_end) {
+      issue_tile();
+      if (p_tile == 0 && p_item != item_begin) issue_q(p_item - item_begin, pc.seg);
+      advance();
     }
     cp_async_commit();
   };
 
-#pragma unroll
-  for (int s = 0; s < kStages - 1; ++s) issue();
+  // Rows that were valid when the plan was built are older than anything the previous kernel of the stream
+  // may still be writing (an append writes behind them): the first tiles are requested before the wait.
+  const int pre = min(kStages - 1, pc.np);
+  for (int s = 0; s < pre; ++s) {
+    issue_tile();
+    ++p_seq;
+    ++p_tile;
+    cp_async_commit();
+  }
+  pdl_wait();  // from here on: lengths, queries and rows written by earlier kernels
+  live_cursor(a, pc);
+  const ItemCursor first = pc;
+  issue_q(0, pc.seg);
+  if (p_tile >= pc.np && p_tile >= item_tiles(pc)) {
+    p_tile = 0;
+    if (++p_item < item_end) pc = read_item(a, p_item);
+  }
+  for (int s = pre; s < kStages - 1; ++s) issue();
+  if (pre == kStages - 1) cp_async_commit();  // the queries of the first item form a group of their own
 
   int seq = 0;
   for (int c_item = item_begin; c_item < item_end; ++c_item) {
@@ -246,7 +290,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
     for (int tile = 0; tile < cc.np || tile < item_tiles(cc); ++tile, ++seq) {
-      cp_async_wait<kStages - 2>();
+      if (seq == 0)
+        cp_async_wait<0>();  // first tile and the first item's queries (whichever group they are in)
+      else
+        cp_async_wait<kStages - 2>();
       __syncthreads();
       if (seq == 0) CATEKV_STAMP(1);
       issue();
@@ -329,6 +376,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
 
     // ---- end of the piece: finish the row sums, merge the four warps, write the result
     if (c_item == item_end - 1) CATEKV_STAMP(2);
+    if (cc.new_row >= 0 && tid == 0) a.seg_len[cc.seg] = cc.live;  // fused append: the segment has grown by one row
 #pragma unroll
     for (int sh = 4; sh <= 16; sh <<= 1) {
       l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
@@ -674,7 +722,8 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
 }
 
 // phases: 1 = attention partials, 2 = combine, 3 = both
-static int decode_launch(int phases, const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
+static int decode_launch(int phases, const catekv_cache* cache, const void* k_new, const void* v_new, const void* q,
+                         int32_t Hq, float sm_scale, void* out,
                          int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                          size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
   int rc = check_cache(cache);
@@ -709,8 +758,10 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* q, i
       if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     DecodeArgs a;
-    a.k_pool = (const uint8_t*)cache->k_pool;
-    a.v_pool = (const uint8_t*)cache->v_pool;
+    a.k_pool = (uint8_t*)cache->k_pool;
+    a.v_pool = (uint8_t*)cache->v_pool;
+    a.k_new = (const uint8_t*)k_new;
+    a.v_new = (const uint8_t*)v_new;
     a.seg_off = cache->seg_off_dev;
     a.seg_len = cache->seg_len_dev;
     a.q = (const uint16_t*)q;
@@ -746,22 +797,41 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* q, i
 extern "C" int catekv_decode_attn(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
                                   int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                                   size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
-  return decode_launch(3, cache, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
+  return decode_launch(3, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
                        ws_bytes, stream);
 }
 
 extern "C" int catekv_decode_partials(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
                                       int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                                       size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
-  return decode_launch(1, cache, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
+  return decode_launch(1, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
                        ws_bytes, stream);
 }
 
 extern "C" int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
                                      int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                                      size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
-  return decode_launch(2, cache, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
+  return decode_launch(2, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
                        ws_bytes, stream);
+}
+
+extern "C" int catekv_append_decode_attn(catekv_cache* cache, const void* k_new, const void* v_new, const void* q,
+                                         int32_t Hq, float sm_scale, void* out, int32_t out_dtype, float* lse_out,
+                                         const void* plan_host, const void* plan_dev, size_t plan_bytes, void* ws,
+                                         size_t ws_bytes, catekv_stream stream) {
+  int rc = check_cache(cache);
+  if (rc) return rc;
+  if (!k_new || !v_new) return CATEKV_ERR_INVALID_ARG;
+  const int n = cache->B * cache->Hkv;
+  for (int s = 0; s < n; ++s) {
+    if (cache->seg_len[s] < 0) return CATEKV_ERR_INVALID_ARG;
+    if (cache->seg_len[s] + 1 > cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+  }
+  rc = decode_launch(3, cache, k_new, v_new, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev,
+                     plan_bytes, ws, ws_bytes, stream);
+  if (rc) return rc;
+  for (int s = 0; s < n; ++s) cache->seg_len[s] += 1;
+  return CATEKV_OK;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -788,6 +858,6 @@ extern "C" int catekv_decode_attn_noalloc(const catekv_cache* cache, const void*
   }
   // decode_launch checks the plan and returns CATEKV_ERR_WORKSPACE when the partials of this plan
   // (num_ctas + B*Hkv slots) do not fit the fixed array
-  return decode_launch(3, cache, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes,
+  return decode_launch(3, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes,
                        scratch_of_device[dev], (size_t)CATEKV_NOALLOC_SCRATCH_BYTES, stream);
 }

@@ -107,30 +107,37 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     const unsigned int* Pb = reinterpret_cast<const unsigned int*>(P);
     unsigned int thr, need_eq;  // threshold bits; entries equal to it that are taken (lowest index first)
     block_radix_select([&](int c) { return Pb[c]; }, s.n_pool, (unsigned int)s.k_sel, hist, s_pair, thr, need_eq);
-    // ---- ordered compaction
+    // ---- ordered compaction, four consecutive entries per thread and step
     unsigned long long run = 0;  // packed: low = entries above the threshold so far, high = entries equal to it
     const int cs = a.pool_mode == CATEKV_POOL_CHUNK ? a.pool_param : 1;
-    for (int base = 0; base < s.n_pool; base += kTopkThreads) {
-      const int c = base + tid;
-      unsigned int v = 0;
-      bool gt = false, eq = false;
-      if (c < s.n_pool) {
-        v = Pb[c];
-        gt = v > thr;
-        eq = v == thr;
+    for (int base = 0; base < s.n_pool; base += 4 * kTopkThreads) {
+      const int c4 = base + tid * 4;
+      unsigned int v[4];
+      bool gt[4], eq[4];
+      unsigned long long mine = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        v[e] = (c4 + e < s.n_pool) ? Pb[c4 + e] : 0u;
+        gt[e] = (c4 + e < s.n_pool) && v[e] > thr;
+        eq[e] = (c4 + e < s.n_pool) && v[e] == thr;
+        mine += (unsigned long long)gt[e] | ((unsigned long long)eq[e] << 32);
       }
       unsigned long long tot;
-      const unsigned long long ex =
-          run + block_excl_scan((unsigned long long)gt | ((unsigned long long)eq << 32), s_warp, tot);
-      const unsigned int gt_before = (unsigned int)(ex & 0xffffffffu), eq_before = (unsigned int)(ex >> 32);
-      if (gt || (eq && eq_before < need_eq)) {
-        const unsigned int rank = gt_before + min(eq_before, need_eq);
-        if (cs == 1) {
-          idx[S + rank] = S + c;
-        } else {
-          const int lo = S + c * cs, hi = min(lo + cs, s.cand_end);
-          for (int u = lo; u < hi; ++u) idx[S + rank * cs + (u - lo)] = u;
+      unsigned long long ex = run + block_excl_scan(mine, s_warp, tot);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const unsigned int gt_before = (unsigned int)(ex & 0xffffffffu), eq_before = (unsigned int)(ex >> 32);
+        if (gt[e] || (eq[e] && eq_before < need_eq)) {
+          const unsigned int rank = gt_before + min(eq_before, need_eq);
+          const int c = c4 + e;
+          if (cs == 1) {
+            idx[S + rank] = S + c;
+          } else {
+            const int lo = S + c * cs, hi = min(lo + cs, s.cand_end);
+            for (int u = lo; u < hi; ++u) idx[S + rank * cs + (u - lo)] = u;
+          }
         }
+        ex += (unsigned long long)gt[e] | ((unsigned long long)eq[e] << 32);
       }
       run += tot;
     }

@@ -124,3 +124,46 @@ def test_decode_is_deterministic(ck):
     a = _run_decode(ck, oc, q, 40)
     b = _run_decode(ck, oc, q, 40)
     assert torch.equal(a[2], b[2]) and torch.equal(a[3], b[3]) and torch.equal(a[4], b[4])
+
+
+def test_fused_append_decode_matches_oracle_and_two_call_path(ck):
+    lens = [100, 128, 1, 0, 300, 64, 17, 255, 63, 2000, 0, 5]
+    oc = H.random_cache(3, 4, lens, seed=19)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=24)
+    ref_cache = H.device_cache_from_oracle(ck, oc, max_new=24)
+    plan = ck.DecodePlan(cache, 13)
+    ck.catekv_decode_plan(cache, plan)
+    plan2 = ck.DecodePlan(ref_cache, 13)
+    ck.catekv_decode_plan(ref_cache, plan2)
+    out = torch.empty((3, 28, 128), dtype=torch.float32, device="cuda")
+    out2 = torch.empty_like(out)
+    lse = torch.empty((3, 28), dtype=torch.float32, device="cuda")
+    for step in range(24):
+        kn = synth.randn_bf16((3, 4, 128), "cuda", 19, "kn", step)
+        vn = synth.randn_bf16((3, 4, 128), "cuda", 19, "vn", step)
+        q = synth.randn_bf16((3, 28, 128), "cuda", 19, "q", step)
+        ck.catekv_append_decode_attn(cache, kn, vn, q, plan, out, lse)
+        ck.catekv_append(ref_cache, kn, vn)
+        ck.catekv_decode_attn(ref_cache, q, plan2, out2)
+        oc.append(synth.bits(kn), synth.bits(vn))
+        assert torch.equal(out, out2), step  # same kernel, same arithmetic
+        if step in (0, 1, 23):
+            ref, ref_lse = orc.decode_attention(oc, synth.bits(q))
+            H.check_attention(out, None, lse, ref, ref_lse, f"fused step {step}")
+    torch.cuda.synchronize()
+    assert list(cache.seg_len) == [l + 24 for l in lens]
+    assert cache.seg_len_dev.cpu().tolist() == [l + 24 for l in lens]
+    for i in range(12):
+        o, L = int(cache.seg_off[i]), lens[i] + 24
+        assert np.array_equal(synth.bits(cache.k_pool[o:o + L]), oc.k_rows[i])
+        assert np.array_equal(synth.bits(cache.v_pool[o:o + L]), oc.v_rows[i])
+    # a full segment refuses the fused call too, before anything is launched
+    while all(cache.seg_len[i] < cache.seg_cap[i] for i in range(12)):
+        ck.catekv_append(cache, kn, vn)
+    before = cache.seg_len.copy()
+    out.fill_(7.0)
+    with pytest.raises(ck.CatekvError) as e:
+        ck.catekv_append_decode_attn(cache, kn, vn, q, plan, out)
+    assert e.value.code == ck.ERR_CAPACITY
+    torch.cuda.synchronize()
+    assert np.array_equal(cache.seg_len, before) and torch.all(out == 7.0)
