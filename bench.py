@@ -418,6 +418,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying "
                     "a captured CUDA graph of the step")
     ap.add_argument("--no-fused", action="store_true", help="catekv_append + catekv_decode_attn as two calls per layer")
+    ap.add_argument("--select-only", action="store_true", help="run only the prefill-end path (catekv_select_compact) "
+                    "for --layers layers and print its time; used for profiling that path on a small case")
     ap.add_argument("--no-extras", action="store_true", help="skip the other configs, head_cv and the oracle timing")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -460,6 +462,10 @@ def main():
     global FUSED
     FUSED = not args.no_fused
     model, sel_ms = build_model(ck, w, dev, max_new=total_steps, layers=n_layers)
+    if args.select_only:
+        if rank == 0:
+            print(json.dumps({"workload": w.name, "layers": n_layers, "select_compact_ms_per_layer": sel_ms}))
+        return
 
     vis = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
     sampler = ClockSampler(vis[local_rank] if local_rank < len(vis) else local_rank)

@@ -488,54 +488,70 @@ struct CombineArgs {
   int32_t Hq, Hkv, G, out_fp32;
 };
 
-// One CTA per (segment, query head of the group).  The LSEs of the pieces are loaded in parallel, the
-// four warps each sum a quarter of the pieces (a lane owns four consecutive d, so a piece is one
-// 512-byte row per warp-load and many loads are in flight), then the warps are summed in a fixed order.
-__global__ void __launch_bounds__(kD) decode_combine_kernel(const CombineArgs a) {
+// One CTA of 8 warps per (segment, query head of the group).  The kernel is a chain of dependent memory
+// round trips, so it is arranged to have few of them: every warp finds the maximum LSE by itself (no
+// barrier), then sums its eighth of the pieces with all of its loads in flight at once (a lane owns four
+// consecutive d, a piece is one 512-byte row per warp-load); the warps are summed in a fixed order.
+constexpr int kCombineWarps = 8;
+__global__ void __launch_bounds__(kCombineWarps * 32) decode_combine_kernel(const CombineArgs a) {
   const int seg = blockIdx.x, hd = blockIdx.y;
   pdl_launch_dependents();
   const SegInfo si = a.seg_info[seg];  // plan data: older than the previous kernel
   pdl_wait();
   if (si.n_pieces <= 1) return;  // written directly by the attention kernel
-  __shared__ float s_red[4];
-  __shared__ float4 s_acc[4][32];
-  __shared__ float s_w[4];
+  __shared__ float4 s_acc[kCombineWarps][32];
+  __shared__ float s_w[kCombineWarps];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n = si.n_pieces;
   const float* lse = a.part_lse + (size_t)si.slot_begin * kMaxG + hd;
-  // max of the pieces' LSEs
-  float m = -INFINITY;
-  for (int p = tid; p < si.n_pieces; p += kD) m = fmaxf(m, lse[(size_t)p * kMaxG]);
+  float M = -INFINITY;
+  for (int p = lane; p < n; p += 32) M = fmaxf(M, lse[(size_t)p * kMaxG]);
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  if (lane == 0) s_red[warp] = m;
-  __syncthreads();
-  const float M = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float wsum = 0.f;
   if (M > -INFINITY) {
     const float* po = a.part_o + ((size_t)si.slot_begin * kMaxG + hd) * kD + lane * 4;
-#pragma unroll 4
-    for (int p = warp; p < si.n_pieces; p += 4) {
-      const float w = exp2f(lse[(size_t)p * kMaxG] - M);
-      const float4 v = *reinterpret_cast<const float4*>(po + (size_t)p * (kMaxG * kD));
-      acc.x += w * v.x;
-      acc.y += w * v.y;
-      acc.z += w * v.z;
-      acc.w += w * v.w;
-      wsum += w;
+    for (int p0 = warp; p0 < n; p0 += kCombineWarps * 8) {
+      float4 v[8];
+      float w[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int p = p0 + u * kCombineWarps;
+        const bool ok = p < n;
+        v[u] = ok ? *reinterpret_cast<const float4*>(po + (size_t)p * (kMaxG * kD)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        w[u] = ok ? lse[(size_t)p * kMaxG] : -INFINITY;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float e = exp2f(w[u] - M);
+        acc.x += e * v[u].x;
+        acc.y += e * v[u].y;
+        acc.z += e * v[u].z;
+        acc.w += e * v[u].w;
+        wsum += e;
+      }
     }
   }
   s_acc[warp][lane] = acc;
   if (lane == 0) s_w[warp] = wsum;
   __syncthreads();
   if (warp == 0) {
-    const float W = ((s_w[0] + s_w[1]) + s_w[2]) + s_w[3];
+    float W = 0.f;
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int wv = 0; wv < kCombineWarps; ++wv) {
+      W += s_w[wv];
+      r.x += s_acc[wv][lane].x;
+      r.y += s_acc[wv][lane].y;
+      r.z += s_acc[wv][lane].z;
+      r.w += s_acc[wv][lane].w;
+    }
     const float inv = W > 0.f ? 1.f / W : 0.f;
-    float4 r;
-    r.x = (((s_acc[0][lane].x + s_acc[1][lane].x) + s_acc[2][lane].x) + s_acc[3][lane].x) * inv;
-    r.y = (((s_acc[0][lane].y + s_acc[1][lane].y) + s_acc[2][lane].y) + s_acc[3][lane].y) * inv;
-    r.z = (((s_acc[0][lane].z + s_acc[1][lane].z) + s_acc[2][lane].z) + s_acc[3][lane].z) * inv;
-    r.w = (((s_acc[0][lane].w + s_acc[1][lane].w) + s_acc[2][lane].w) + s_acc[3][lane].w) * inv;
+    r.x *= inv;
+    r.y *= inv;
+    r.z *= inv;
+    r.w *= inv;
     const int b = seg / a.Hkv, h = seg % a.Hkv;
     const size_t obase = ((size_t)b * a.Hq + (size_t)h * a.G + hd) * kD;
     if (a.out_fp32) {
@@ -789,7 +805,7 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* k_ne
     ca.Hkv = cache->Hkv;
     ca.G = G;
     ca.out_fp32 = out_fp32;
-    CATEKV_CUDA_TRY(launch_pdl(decode_combine_kernel, dim3(n_segs, G), dim3(kD), 0, st, ca));
+    CATEKV_CUDA_TRY(launch_pdl(decode_combine_kernel, dim3(n_segs, G), dim3(kCombineWarps * 32), 0, st, ca));
   }
   return CATEKV_OK;
 }
