@@ -118,8 +118,9 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   if (G * L_obs > kScoreMaxRows) return CATEKV_ERR_UNSUPPORTED;
   if (!(quantile_k >= 0.f && quantile_k <= 1.f) || !(alpha >= 0.f) || isinf(alpha)) return CATEKV_ERR_INVALID_ARG;
   const int n_segs = B * Hkv;
-  int m_max = 0;
+  int m_max = 0, n_max_tokens = 0;
   for (int b = 0; b < B; ++b) {
+    n_max_tokens = seq_len[b] > n_max_tokens ? seq_len[b] : n_max_tokens;
     const int64_t m = (int64_t)seq_len[b] - L_init - L_rec;
     if (m < 1 || seq_len[b] < L_obs) return CATEKV_ERR_INVALID_ARG;
     if (m * L_obs > INT32_MAX) return CATEKV_ERR_UNSUPPORTED;
@@ -154,6 +155,9 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   sa.jobs = (const ScoreJob*)(w8 + W.off_jobs);
   sa.n_jobs = n_segs;
   sa.Hq = Hq;
+  sa.B = B;
+  sa.Hkv = Hkv;
+  sa.n_max = n_max_tokens;
   sa.G = G;
   sa.L_obs = L_obs;
   sa.causal = causal ? 1 : 0;

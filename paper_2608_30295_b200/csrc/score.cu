@@ -1,9 +1,10 @@
-// Observation-window scoring on the 5th-generation tensor cores (tcgen05 + TMEM).
+// Observation-window scoring on the 5th-generation tensor cores (TMA + tcgen05 + TMEM).
 //
 // A CTA scores `keys_per_cta` keys of one (sequence, KV head) against the R = G * L_obs window
 // query rows of the group (row r = i * G + g: window row i of the group's g-th query head).
-// Q stays in shared memory for the CTA's lifetime, 128-key tiles of K stream through two
-// cp.async stages, both in the K-major SWIZZLE_128B layout the UMMA descriptors expect.
+// Q stays in shared memory for the CTA's lifetime; 128-key tiles of K are fetched by TMA
+// (cp.async.bulk.tensor, two 64-column boxes per tile) straight into the K-major SWIZZLE_128B
+// layout the UMMA descriptors expect, two stages deep.
 //
 //   pass 1 (row statistics)   D[128 rows x 128 keys] = Q_rows . K_tile^T   (M = rows, N = keys)
 //       every thread owns one query row (one TMEM lane): running max and sum of exp2 over the
@@ -14,17 +15,23 @@
 //       one key, so C_j = sum_r exp2(x_rj - m_r) / l_r and A_ij = mean_g (...) are thread-local
 //       sums over TMEM columns and the global writes are coalesced over keys.
 //
-// One elected thread issues tcgen05.mma (8 k-steps of 16 per 128-wide head dim) and commits to an
-// mbarrier; accumulators are double- or quad-buffered in TMEM so that the MMAs of the next unit
-// run under the exp2 epilogue of the current one.  Every mbarrier wait is bounded: on expiry the
-// CTA records a status word, drains its copies, frees its TMEM and returns.
+// Warp roles: warp 8 (one elected lane) waits for a K tile, issues the eight k-steps of
+// tcgen05.mma per unit and commits them to an mbarrier; warps 0-7 are the epilogue (two per
+// TMEM lane quarter, each half of a unit's columns): they wait for the unit, read the
+// accumulators with tcgen05.ld, do the exp2 arithmetic and hand the TMEM slot back.  The thread
+// that observes the last unit of a tile complete re-arms that tile's stage with the next TMA
+// load.  There is no CTA-wide barrier in the main loop.  Every mbarrier wait is bounded: on
+// expiry the thread raises a CTA-wide abort flag (which ends all other waits early) and a status
+// word in the workspace; the CTA then frees its TMEM and returns.
+#include <cuda.h>
 #include <math.h>
 
 #include "score.cuh"
 
 namespace catekv {
 
-constexpr int kScThreads = 256;                    // 8 warps: two per TMEM lane quarter, each takes half the columns
+constexpr int kEpiThreads = 256;                   // 8 epilogue warps: two per TMEM lane quarter, each takes half the columns
+constexpr int kScThreads = kEpiThreads + 32;       // + the TMA / MMA warp
 constexpr int kKeyTile = 128;                       // keys per tile
 constexpr int kKBlockBytes = kKeyTile * 128;        // one 64-element k-block of a K tile
 constexpr int kKStageBytes = 2 * kKBlockBytes;      // K tile: 128 keys x 128 dims bf16
@@ -89,16 +96,34 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
-// bounded wait for a phase of an mbarrier; false if it never completed
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  uint32_t done = 0;
-  for (uint32_t it = 0; it < kSpinLimit && !done; ++it)
+// Bounded wait for a phase of an mbarrier.  Returns false if it never completed or if another thread of
+// the CTA has given up (abort flag), in which case the flag is (also) raised by this thread.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    uint32_t done;
     asm volatile(
         "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
         : "=r"(done)
         : "r"(bar), "r"(parity)
         : "memory");
-  return done != 0;
+    if (done) return true;
+    if ((it & 255u) == 255u && *abort_flag) break;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+// one 64-column x 128-row box of K (rank-4 map: d, token, head, sequence) into shared memory
+__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* map, int d0, int j0, int h, int b, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n" ::"r"(dst),
+      "l"(map), "r"(d0), "r"(j0), "r"(h), "r"(b), "r"(bar)
+      : "memory");
 }
 // 32 consecutive TMEM columns of this thread's lane
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
@@ -122,14 +147,15 @@ __device__ __forceinline__ uint32_t sw128_off(int r, int c, int rows) {
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(kScThreads) score_tc_kernel(const ScoreArgs a, const ScoreShape sh) {
+__global__ void __launch_bounds__(kScThreads) score_tc_kernel(const __grid_constant__ CUtensorMap k_map, const ScoreArgs a,
+                                                              const ScoreShape sh) {
   extern __shared__ uint8_t smem_raw[];
   const ScoreJob job = a.jobs[blockIdx.y];
   const int j_lo = job.j_begin + blockIdx.x * a.keys_per_cta;
   if (j_lo >= job.j_end) return;
   const int j_hi = min(job.j_end, j_lo + a.keys_per_cta);
   const int n_tiles = (j_hi - j_lo + kKeyTile - 1) / kKeyTile;
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   // ---- shared memory carve-up (1024-byte aligned for the 128-byte swizzle)
   const uint32_t s_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -137,19 +163,20 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const ScoreArgs a,
   const uint32_t q_block = (uint32_t)sh.q_rows * 128;  // one k-block of Q
   const uint32_t s_q = s_base;
   const uint32_t s_k = s_q + 2 * q_block;
-  float* s_f = reinterpret_cast<float*>(smem + 2 * q_block + 2 * kKStageBytes);  // pass 1: (m, l)[MT][128]; pass 2: m'[R]
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_f + 4 * kScoreMaxRows);
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 4);
+  float* s_f = reinterpret_cast<float*>(smem + 2 * q_block + 2 * kKStageBytes);  // pass 1: (m, l)[2][512]; pass 2: m'[R]
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_f + 4 * kScoreMaxRows);         // full[2], done[4], free[4]
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 10);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  const uint32_t bar_full = smem_u32(s_bar), bar_done = smem_u32(s_bar + 2), bar_free = smem_u32(s_bar + 6);
 
   constexpr bool kStats = MODE == kScoreStats;
   const int UPT = kStats ? sh.MT : sh.NH;          // MMA units per key tile
   const int NSLOT = kStats ? sh.nslot1 : 2;
-  const int LA = kStats ? sh.la1 : 1;
   const int slot_w = kStats ? 128 : sh.slotw2;
   const int n_cols = kStats ? sh.cols1 : sh.cols2;
   const int U = n_tiles * UPT;
 
-  // ---- stage Q (row r = i * G + g) and the first two K tiles
+  // ---- set-up: Q (row r = i * G + g) by cp.async from all threads, barriers, TMEM
   for (int id = tid; id < sh.q_rows * 16; id += kScThreads) {
     const int r = id >> 4, c = id & 15;
     const int i = r / a.G, g = r - i * a.G;
@@ -157,22 +184,7 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const ScoreArgs a,
     const uint16_t* src = a.q_win + (((int64_t)job.b * a.Hq + job.h * a.G + (ok ? g : 0)) * a.L_obs + (ok ? i : 0)) * kD + c * 8;
     cp_async16(s_q + sw128_off(r, c, sh.q_rows), src, ok);
   }
-  const uint16_t* kbase = a.k + (int64_t)job.b * a.sb + (int64_t)job.h * a.sh;
-  auto load_tile = [&](int tile) {
-    if (tile < n_tiles) {
-      const uint32_t sb = s_k + (tile & 1) * kKStageBytes;
-      const int j0 = j_lo + tile * kKeyTile;
-#pragma unroll 4
-      for (int id = tid; id < kKeyTile * 16; id += kScThreads) {
-        const int r = id >> 4, c = id & 15;
-        const int ok = (j0 + r) < j_hi ? 16 : 0;
-        cp_async16(sb + sw128_off(r, c, kKeyTile), kbase + (int64_t)(ok ? j0 + r : job.j_begin) * a.st + c * 8, ok);
-      }
-    }
-    cp_async_commit();
-  };
-  load_tile(0);
-  load_tile(1);
+  cp_async_commit();
   if (kStats) {
     for (int i = tid; i < 2 * kScoreMaxRows; i += kScThreads) {
       s_f[2 * i] = -INFINITY;
@@ -187,176 +199,188 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const ScoreArgs a,
     }
   }
   if (tid == 0) {
-    for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(smem_u32(s_bar + i)));
+    *s_abort = 0;
+    for (int i = 0; i < 2; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar_full + 8 * i));
+    for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar_done + 8 * i));
+    for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 8;\n" ::"r"(bar_free + 8 * i));  // one arrival per epilogue warp
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
-  if (warp == 0) {
+  if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(s_tmem)), "r"(n_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
   cp_async_wait<0>();
-  fence_async_smem();
+  fence_async_smem();  // Q was written through the generic proxy; the MMAs read it through the async proxy
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
 
-  const uint32_t idesc = kStats ? umma_idesc_bf16(128, 128) : umma_idesc_bf16(128, sh.NW);
-  auto issue_unit = [&](int v) {  // thread 0 only
-    const int tile = v / UPT, sub = v - tile * UPT;
-    const uint32_t sk = s_k + (tile & 1) * kKStageBytes;
-    const uint32_t d = tmem + (uint32_t)((v % NSLOT) * slot_w);
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-      const uint32_t koff = (kk & 3) * 32;
-      const uint32_t aq = s_q + (kk >> 2) * q_block + koff;
-      const uint32_t ak = sk + (kk >> 2) * kKBlockBytes + koff;
-      if (kStats)  // D[rows x keys]: A = Q rows of this M tile, B = K tile
-        umma_bf16(d, umma_desc_sw128(aq + sub * 128 * 128), umma_desc_sw128(ak), idesc, kk ? 1u : 0u);
-      else         // D[keys x rows]: A = K tile, B = Q rows of this half
-        umma_bf16(d, umma_desc_sw128(ak), umma_desc_sw128(aq + sub * sh.NW * 128), idesc, kk ? 1u : 0u);
-    }
-    umma_commit(smem_u32(s_bar + (v % NSLOT)));
+  // K tile `tile` -> stage tile & 1: two boxes of 64 columns (one k-block each), 32 KB on the stage's barrier
+  auto load_tile = [&](int tile) {
+    const uint32_t sb = s_k + (tile & 1) * kKStageBytes;
+    const uint32_t bar = bar_full + 8 * (tile & 1);
+    mbar_expect_tx(bar, kKStageBytes);
+    tma_load_box(sb, &k_map, 0, j_lo + tile * kKeyTile, job.h, job.b, bar);
+    tma_load_box(sb + kKBlockBytes, &k_map, 64, j_lo + tile * kKeyTile, job.h, job.b, bar);
   };
-  if (tid == 0)
-    for (int v = 0; v < LA && v < U; ++v) issue_unit(v);
 
-  // warp w reads TMEM lanes 32 * (w % 4) ...; warps 0-3 take the first half of a unit's columns, warps 4-7 the second
-  const int lane_row = (warp & 3) * 32 + (tid & 31);  // this thread's TMEM lane: a query row (pass 1) or a key (pass 2)
-  const int half = warp >> 2;
-  const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-  const float inv_g = 1.f / (float)a.G;
-  float* s_col = s_f + kScoreMaxRows;  // pass 2: [2][128] per-half sums of a key
-  float col_acc = 0.f;                 // pass 2, column sums: this key's sum over this thread's rows of the tile
-  bool alive = true;
-
-  for (int u = 0; u < U; ++u) {
-    const int tile = u / UPT, sub = u - tile * UPT;
-    const int v = u + LA;
-    if (sub == 0 && tile >= 1) load_tile(tile + 1);  // into the stage of tile - 1, whose MMAs have been waited for
-    if (v < U && v % UPT == 0) {                     // the tile of unit v must have landed before its MMAs are issued
-      cp_async_wait<0>();
-      fence_async_smem();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    if (tid == 0 && v < U) issue_unit(v);
-    alive = __syncthreads_and(mbar_wait(smem_u32(s_bar + (u % NSLOT)), (uint32_t)((u / NSLOT) & 1)));
-    if (!alive) break;
-    tc_fence_after();
-    const uint32_t tbase = tmem + lane_base + (uint32_t)((u % NSLOT) * slot_w);
-    const int j0 = j_lo + tile * kKeyTile;
-
-    if (kStats) {
-      // this thread's query row, keys [64 * half, 64 * half + 64) of the tile
-      const int r = sub * 128 + lane_row;
-      const int i = r / a.G;
-      const int lim = a.causal ? job.n - a.L_obs + i : 0x7fffffff;  // last key this window row sees
-      const int jmax = min(j_hi - 1, lim);                          // keys j <= jmax are live
-      float m = s_f[2 * (half * kScoreMaxRows + r)], l = s_f[2 * (half * kScoreMaxRows + r) + 1];
-#pragma unroll 1
-      for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 32) {
-        if (j0 + c0 >= j_hi) break;  // uniform: the rest of the tile is padding
-        float x[32];
-        tmem_ld32(tbase + c0, x);
-        if (j0 + c0 + 31 > jmax) {  // tail of the key range or the causal edge: mask entry by entry
+  if (warp == 8) {
+    // ================= TMA + MMA issue: one elected lane =================
+    if (lane == 0) {
+      for (int tl = 0; tl < 2 && tl < n_tiles; ++tl) load_tile(tl);
+      const uint32_t idesc = kStats ? umma_idesc_bf16(128, 128) : umma_idesc_bf16(128, sh.NW);
+      for (int v = 0; v < U; ++v) {
+        const int tile = v / UPT, sub = v - tile * UPT;
+        if (sub == 0 && !mbar_wait(bar_full + 8 * (tile & 1), (uint32_t)((tile >> 1) & 1), s_abort)) break;
+        if (v >= NSLOT && !mbar_wait(bar_free + 8 * (v % NSLOT), (uint32_t)(((v / NSLOT) - 1) & 1), s_abort)) break;
+        tc_fence_after();
+        const uint32_t sk = s_k + (tile & 1) * kKStageBytes;
+        const uint32_t d = tmem + (uint32_t)((v % NSLOT) * slot_w);
 #pragma unroll
-          for (int c = 0; c < 32; ++c) x[c] = (j0 + c0 + c <= jmax) ? x[c] : -INFINITY;
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint32_t koff = (kk & 3) * 32;
+          const uint32_t aq = s_q + (kk >> 2) * q_block + koff;
+          const uint32_t ak = sk + (kk >> 2) * kKBlockBytes + koff;
+          if (kStats)  // D[rows x keys]: A = Q rows of this M tile, B = K tile
+            umma_bf16(d, umma_desc_sw128(aq + sub * 128 * 128), umma_desc_sw128(ak), idesc, kk ? 1u : 0u);
+          else         // D[keys x rows]: A = K tile, B = Q rows of this half
+            umma_bf16(d, umma_desc_sw128(ak), umma_desc_sw128(aq + sub * sh.NW * 128), idesc, kk ? 1u : 0u);
         }
-        float mx = x[0];
-#pragma unroll
-        for (int c = 1; c < 32; ++c) mx = fmaxf(mx, x[c]);
-        mx *= a.scale_log2;  // the scale is positive: the max commutes with it
-        if (mx > m) {
-          l *= fast_exp2(m - mx);
-          m = mx;
-        }
-        if (m > -INFINITY) {
-          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-          for (int c = 0; c < 32; c += 4) {
-            s0 += fast_exp2(fmaf(x[c], a.scale_log2, -m));
-            s1 += fast_exp2(fmaf(x[c + 1], a.scale_log2, -m));
-            s2 += fast_exp2(fmaf(x[c + 2], a.scale_log2, -m));
-            s3 += fast_exp2(fmaf(x[c + 3], a.scale_log2, -m));
-          }
-          l += (s0 + s1) + (s2 + s3);
-        }
+        umma_commit(bar_done + 8 * (v % NSLOT));
       }
-      s_f[2 * (half * kScoreMaxRows + r)] = m;
-      s_f[2 * (half * kScoreMaxRows + r) + 1] = l;
-    } else {
-      // this thread's key; the unit's rows [r_begin, r_end) are cut, at a multiple of G, between the two halves
-      const int j = j0 + lane_row;
-      const int r_begin = sub * sh.NW, r_end = min(sh.R, r_begin + sh.NW);
-      // column sums cut at a multiple of 32 columns, the matrix at a multiple of G (whole window rows per thread)
-      const int cut = MODE == kScoreColsum ? min(r_end, r_begin + ((r_end - r_begin) / 2 + 31) / 32 * 32)
-                                           : r_begin + ((r_end - r_begin) / 2 / a.G) * a.G;
-      const int r0 = half ? cut : r_begin, r1 = half ? r_end : cut;
-      if (MODE == kScoreColsum) {
-        if (sub == 0) col_acc = 0.f;
-        float c0s = 0.f, c1s = 0.f, c2s = 0.f, c3s = 0.f;
+    }
+    __syncwarp();
+  } else {
+    // ================= epilogue warps =================
+    // warp w reads TMEM lanes 32 * (w % 4) ...; warps 0-3 take the first half of a unit's columns, warps 4-7 the second
+    const int lane_row = (warp & 3) * 32 + lane;  // this thread's TMEM lane: a query row (pass 1) or a key (pass 2)
+    const int half = warp >> 2;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const float inv_g = 1.f / (float)a.G;
+    float col_acc = 0.f;  // pass 2, column sums: this key's sum over this thread's rows of the tile
+
+    for (int u = 0; u < U; ++u) {
+      const int tile = u / UPT, sub = u - tile * UPT;
+      if (!mbar_wait(bar_done + 8 * (u % NSLOT), (uint32_t)((u / NSLOT) & 1), s_abort)) break;
+      tc_fence_after();
+      // the MMAs of this tile have read its stage: re-arm the stage with the tile after next
+      if (tid == 0 && sub == UPT - 1 && tile + 2 < n_tiles) load_tile(tile + 2);
+      const uint32_t tbase = tmem + lane_base + (uint32_t)((u % NSLOT) * slot_w);
+      const int j0 = j_lo + tile * kKeyTile;
+
+      if (kStats) {
+        // this thread's query row, keys [64 * half, 64 * half + 64) of the tile
+        const int r = sub * 128 + lane_row;
+        const int i = r / a.G;
+        const int lim = a.causal ? job.n - a.L_obs + i : 0x7fffffff;  // last key this window row sees
+        const int jmax = min(j_hi - 1, lim);                          // keys j <= jmax are live
+        float m = s_f[2 * (half * kScoreMaxRows + r)], l = s_f[2 * (half * kScoreMaxRows + r) + 1];
 #pragma unroll 1
-        for (int rr = r0; rr < r1; rr += 32) {
+        for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 32) {
+          if (j0 + c0 >= j_hi) break;  // uniform: the rest of the tile is padding
           float x[32];
-          tmem_ld32(tbase + (rr - r_begin), x);
-          if (rr + 32 <= r1) {
+          tmem_ld32(tbase + c0, x);
+          if (j0 + c0 + 31 > jmax) {  // tail of the key range or the causal edge: mask entry by entry
+#pragma unroll
+            for (int c = 0; c < 32; ++c) x[c] = (j0 + c0 + c <= jmax) ? x[c] : -INFINITY;
+          }
+          float mx = x[0];
+#pragma unroll
+          for (int c = 1; c < 32; ++c) mx = fmaxf(mx, x[c]);
+          mx *= a.scale_log2;  // the scale is positive: the max commutes with it
+          if (mx > m) {
+            l *= fast_exp2(m - mx);
+            m = mx;
+          }
+          if (m > -INFINITY) {
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
             for (int c = 0; c < 32; c += 4) {
-              const float4 mm = *reinterpret_cast<const float4*>(s_f + rr + c);  // rr is a multiple of 16
-              c0s += fast_exp2(fmaf(x[c], a.scale_log2, -mm.x));
-              c1s += fast_exp2(fmaf(x[c + 1], a.scale_log2, -mm.y));
-              c2s += fast_exp2(fmaf(x[c + 2], a.scale_log2, -mm.z));
-              c3s += fast_exp2(fmaf(x[c + 3], a.scale_log2, -mm.w));
+              s0 += fast_exp2(fmaf(x[c], a.scale_log2, -m));
+              s1 += fast_exp2(fmaf(x[c + 1], a.scale_log2, -m));
+              s2 += fast_exp2(fmaf(x[c + 2], a.scale_log2, -m));
+              s3 += fast_exp2(fmaf(x[c + 3], a.scale_log2, -m));
             }
-          } else {
-#pragma unroll
-            for (int c = 0; c < 32; ++c)
-              if (rr + c < r1) c0s += fast_exp2(fmaf(x[c], a.scale_log2, -s_f[rr + c]));
+            l += (s0 + s1) + (s2 + s3);
           }
         }
-        col_acc += (c0s + c1s) + (c2s + c3s);
-        if (sub == UPT - 1) {
-          s_col[half * 128 + lane_row] = col_acc;
-          __syncthreads();
-          if (half == 0 && j < j_hi)
-            a.out[(size_t)blockIdx.y * a.out_job_stride + (j - job.j_begin)] = (s_col[lane_row] + s_col[128 + lane_row]) * inv_g;
-          // s_col is rewritten one tile later, after several barriers
-        }
+        s_f[2 * (half * kScoreMaxRows + r)] = m;
+        s_f[2 * (half * kScoreMaxRows + r) + 1] = l;
       } else {
-        // group-mean matrix: rows come in runs of G heads per window row; r0 is a multiple of G
-        float* A = a.out + (size_t)blockIdx.y * a.out_job_stride;
-        int i = r0 / a.G, g = 0;
-        float acc = 0.f;
+        // this thread's key; the unit's rows [r_begin, r_end) are cut between the two halves: at a multiple of 32
+        // columns for the column sums, at a multiple of G for the matrix (whole window rows per thread)
+        const int j = j0 + lane_row;
+        const int r_begin = sub * sh.NW, r_end = min(sh.R, r_begin + sh.NW);
+        const int cut = MODE == kScoreColsum ? min(r_end, r_begin + ((r_end - r_begin) / 2 + 31) / 32 * 32)
+                                             : r_begin + ((r_end - r_begin) / 2 / a.G) * a.G;
+        const int r0 = half ? cut : r_begin, r1 = half ? r_end : cut;
+        if (MODE == kScoreColsum) {
+          if (sub == 0) col_acc = 0.f;
+          float c0s = 0.f, c1s = 0.f, c2s = 0.f, c3s = 0.f;
 #pragma unroll 1
-        for (int rr = r0; rr < r1; rr += 32) {
-          float x[32];
-          tmem_ld32(tbase + (rr - r_begin), x);
+          for (int rr = r0; rr < r1; rr += 32) {
+            float x[32];
+            tmem_ld32(tbase + (rr - r_begin), x);
+            if (rr + 32 <= r1) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            if (rr + c < r1) {
-              const bool seen = !a.causal || j <= job.n - a.L_obs + i;
-              acc += seen ? fast_exp2(fmaf(x[c], a.scale_log2, -s_f[rr + c])) : 0.f;
-              if (++g == a.G) {
-                if (j < j_hi) A[(size_t)i * a.out_row_stride + (j - job.j_begin)] = acc * inv_g;
-                acc = 0.f;
-                g = 0;
-                ++i;
+              for (int c = 0; c < 32; c += 4) {
+                const float4 mm = *reinterpret_cast<const float4*>(s_f + rr + c);  // rr is a multiple of 16
+                c0s += fast_exp2(fmaf(x[c], a.scale_log2, -mm.x));
+                c1s += fast_exp2(fmaf(x[c + 1], a.scale_log2, -mm.y));
+                c2s += fast_exp2(fmaf(x[c + 2], a.scale_log2, -mm.z));
+                c3s += fast_exp2(fmaf(x[c + 3], a.scale_log2, -mm.w));
+              }
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (rr + c < r1) c0s += fast_exp2(fmaf(x[c], a.scale_log2, -s_f[rr + c]));
+            }
+          }
+          col_acc += (c0s + c1s) + (c2s + c3s);
+          // the two threads of a key add their shares to the zero-initialised output: 0 + x + y is the same
+          // in either order, so the result does not depend on timing
+          if (sub == UPT - 1 && j < j_hi)
+            atomicAdd(a.out + (size_t)blockIdx.y * a.out_job_stride + (j - job.j_begin), col_acc * inv_g);
+        } else {
+          // group-mean matrix: rows come in runs of G heads per window row; r0 is a multiple of G
+          float* A = a.out + (size_t)blockIdx.y * a.out_job_stride;
+          int i = r0 / a.G, g = 0;
+          float acc = 0.f;
+#pragma unroll 1
+          for (int rr = r0; rr < r1; rr += 32) {
+            float x[32];
+            tmem_ld32(tbase + (rr - r_begin), x);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              if (rr + c < r1) {
+                const bool seen = !a.causal || j <= job.n - a.L_obs + i;
+                acc += seen ? fast_exp2(fmaf(x[c], a.scale_log2, -s_f[rr + c])) : 0.f;
+                if (++g == a.G) {
+                  if (j < j_hi) A[(size_t)i * a.out_row_stride + (j - job.j_begin)] = acc * inv_g;
+                  acc = 0.f;
+                  g = 0;
+                  ++i;
+                }
               }
             }
           }
         }
       }
+      // hand the TMEM slot back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_free + 8 * (u % NSLOT));
     }
   }
 
-  // ---- drain, release TMEM
-  cp_async_wait<0>();
+  // ---- release TMEM (after an abort: first give copies that may still be in flight time to land)
+  if (*s_abort)
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(n_cols) : "memory");
-  if (!alive) {
+  if (warp == 8) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(n_cols) : "memory");
+  if (*s_abort) {
     if (tid == 0) atomicExch(a.status, 1);
     return;
   }
@@ -395,14 +419,47 @@ __global__ void __launch_bounds__(256) score_stats_merge_kernel(const ScoreArgs 
 }
 
 static size_t score_smem_bytes(const ScoreShape& sh) {
-  return 1024 + 2 * (size_t)sh.q_rows * 128 + 2 * kKStageBytes + 4 * kScoreMaxRows * sizeof(float) + 4 * sizeof(uint64_t) + 16;
+  return 1024 + 2 * (size_t)sh.q_rows * 128 + 2 * kKStageBytes + 4 * kScoreMaxRows * sizeof(float) + 10 * sizeof(uint64_t) + 16;
+}
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup (libcuda is not linked)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// K as a rank-4 tensor (d, token, head, sequence) with the caller's strides; box = 64 columns x 128 tokens,
+// 128-byte swizzle, out-of-range tokens read as zero
+static int make_k_map(const ScoreArgs& a, CUtensorMap* map) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return CATEKV_ERR_CUDA;
+  if (((uintptr_t)a.k & 15) || (a.st * 2) % 16 || (a.sh * 2) % 16 || (a.sb * 2) % 16 || a.st <= 0) return CATEKV_ERR_UNSUPPORTED;
+  const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)a.n_max, (cuuint64_t)a.Hkv, (cuuint64_t)a.B};
+  const cuuint64_t strides[3] = {(cuuint64_t)a.st * 2, (cuuint64_t)(a.Hkv > 1 ? a.sh : a.st * a.n_max) * 2,
+                                 (cuuint64_t)(a.B > 1 ? a.sb : (a.Hkv > 1 ? a.sh * a.Hkv : a.st * a.n_max)) * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)kKeyTile, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<uint16_t*>(a.k), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? CATEKV_OK : CATEKV_ERR_UNSUPPORTED;
 }
 
 template <int MODE>
-static int launch_one(const ScoreArgs& a, const ScoreShape& sh, cudaStream_t stream) {
+static int launch_one(const ScoreArgs& a, const ScoreShape& sh, const CUtensorMap& map, cudaStream_t stream) {
   const size_t smem = score_smem_bytes(sh);
   CATEKV_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  score_tc_kernel<MODE><<<dim3(a.n_chunks, a.n_jobs), kScThreads, smem, stream>>>(a, sh);
+  score_tc_kernel<MODE><<<dim3(a.n_chunks, a.n_jobs), kScThreads, smem, stream>>>(map, a, sh);
   CATEKV_CUDA_TRY(cudaGetLastError());
   return CATEKV_OK;
 }
@@ -411,11 +468,19 @@ int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream) {
   if (a.n_jobs <= 0 || a.n_chunks <= 0) return CATEKV_OK;
   if (a.G * a.L_obs > kScoreMaxRows || a.keys_per_cta % kKeyTile || !a.status) return CATEKV_ERR_UNSUPPORTED;
   const ScoreShape sh = score_shape(a.G, a.L_obs);
-  int rc = launch_one<kScoreStats>(a, sh, stream);
+  CUtensorMap map;
+  int rc = make_k_map(a, &map);
+  if (rc) return rc;
+  rc = launch_one<kScoreStats>(a, sh, map, stream);
   if (rc) return rc;
   score_stats_merge_kernel<<<dim3((sh.R + 7) / 8, a.n_jobs), 256, 0, stream>>>(a, sh.R);
   CATEKV_CUDA_TRY(cudaGetLastError());
-  return out_mode == kScoreColsum ? launch_one<kScoreColsum>(a, sh, stream) : launch_one<kScoreMatrix>(a, sh, stream);
+  if (out_mode == kScoreColsum) {
+    // the two epilogue threads of a key add their shares into a zeroed vector
+    CATEKV_CUDA_TRY(cudaMemsetAsync(a.out, 0, sizeof(float) * (size_t)a.n_jobs * a.out_job_stride, stream));
+    return launch_one<kScoreColsum>(a, sh, map, stream);
+  }
+  return launch_one<kScoreMatrix>(a, sh, map, stream);
 }
 
 }  // namespace catekv

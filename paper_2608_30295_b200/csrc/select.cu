@@ -344,6 +344,9 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
     sa.jobs = d_jobs;
     sa.n_jobs = (int)jobs.size();
     sa.Hq = p->Hq;
+    sa.B = p->B;
+    sa.Hkv = p->Hkv;
+    sa.n_max = n_max;
     sa.G = G;
     sa.L_obs = p->L_obs;
     sa.causal = 0;  // every scored key precedes every window query
