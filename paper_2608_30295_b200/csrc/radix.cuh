@@ -19,14 +19,24 @@ __device__ __forceinline__ void block_radix_select(Load load, int n, unsigned in
     const unsigned int pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
     if (tid < 256) hist[tid] = 0;
     __syncthreads();
-    for (int c0 = 0; c0 < n; c0 += nthr) {  // whole warps stay in the loop: the vote below needs them
-      const int c = c0 + tid;
-      const unsigned int v = c < n ? load(c) : 0u;
-      const bool in = c < n && (v & pmask) == prefix;
-      // lanes with the same digit elect one of them to add their count (scores cluster in a few bins)
-      const unsigned int dgt = in ? ((v >> shift) & 0xffu) : 0x100u;
-      const unsigned int peers = __match_any_sync(0xffffffffu, dgt);
-      if (in && (threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[dgt], (unsigned int)__popc(peers));
+    for (int c0 = 0; c0 < n; c0 += 4 * nthr) {  // whole warps stay in the loop: the vote below needs them
+      // four independent loads in flight per thread
+      unsigned int v[4];
+      bool in[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int c = c0 + e * nthr + tid;
+        v[e] = c < n ? load(c) : 0u;
+        in[e] = c < n;
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool hit = in[e] && (v[e] & pmask) == prefix;
+        // lanes with the same digit elect one of them to add their count (scores cluster in a few bins)
+        const unsigned int dgt = hit ? ((v[e] >> shift) & 0xffu) : 0x100u;
+        const unsigned int peers = __match_any_sync(0xffffffffu, dgt);
+        if (hit && (threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[dgt], (unsigned int)__popc(peers));
+      }
     }
     __syncthreads();
     if (tid == 0) {

@@ -81,25 +81,56 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     const float* C = a.C + (size_t)s.job * a.c_stride;
     float* P = a.P + (size_t)s.job * a.c_stride;
     const int n_sc = s.n - a.L_obs;
-    // ---- pooling
+    // ---- pooling (four entries per thread and step, so that several loads are in flight)
+    const float* __restrict__ Cr = C;
+    float* __restrict__ Pw = P;
     if (a.pool_mode == CATEKV_POOL_NONE) {
-      for (int c = tid; c < s.n_pool; c += kTopkThreads) P[c] = C[S + c];
+      for (int c0 = tid; c0 < s.n_pool; c0 += 4 * kTopkThreads) {
+        float vv[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) vv[e] = (c0 + e * kTopkThreads < s.n_pool) ? Cr[S + c0 + e * kTopkThreads] : 0.f;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (c0 + e * kTopkThreads < s.n_pool) Pw[c0 + e * kTopkThreads] = vv[e];
+      }
     } else if (a.pool_mode == CATEKV_POOL_SLIDING) {
       const int half = (a.pool_param - 1) / 2;
-      for (int c = tid; c < s.n_pool; c += kTopkThreads) {
-        const int j = S + c;
-        const int lo = max(0, j - half), hi = min(n_sc - 1, j + half);
-        float m = C[lo];
-        for (int u = lo + 1; u <= hi; ++u) m = fmaxf(m, C[u]);
-        P[c] = m;
+      for (int c0 = tid; c0 < s.n_pool; c0 += 4 * kTopkThreads) {
+        float mm[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int c = c0 + e * kTopkThreads;
+          mm[e] = 0.f;
+          if (c < s.n_pool) {
+            const int j = S + c;
+            const int lo = max(0, j - half), hi = min(n_sc - 1, j + half);
+            float m = Cr[lo];
+            for (int u = lo + 1; u <= hi; ++u) m = fmaxf(m, Cr[u]);
+            mm[e] = m;
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (c0 + e * kTopkThreads < s.n_pool) Pw[c0 + e * kTopkThreads] = mm[e];
       }
     } else {
       const int cs = a.pool_param;
-      for (int c = tid; c < s.n_pool; c += kTopkThreads) {
-        const int lo = S + c * cs, hi = min(lo + cs, s.cand_end);
-        float m = C[lo];
-        for (int u = lo + 1; u < hi; ++u) m = fmaxf(m, C[u]);
-        P[c] = m;
+      for (int c0 = tid; c0 < s.n_pool; c0 += 4 * kTopkThreads) {
+        float mm[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int c = c0 + e * kTopkThreads;
+          mm[e] = 0.f;
+          if (c < s.n_pool) {
+            const int lo = S + c * cs, hi = min(lo + cs, s.cand_end);
+            float m = Cr[lo];
+            for (int u = lo + 1; u < hi; ++u) m = fmaxf(m, Cr[u]);
+            mm[e] = m;
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (c0 + e * kTopkThreads < s.n_pool) Pw[c0 + e * kTopkThreads] = mm[e];
       }
     }
     __syncthreads();
