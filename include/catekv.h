@@ -147,7 +147,7 @@ typedef struct catekv_select_params {
   const void* v;             /* device bf16 prefill values */
   int64_t kv_stride_b, kv_stride_h, kv_stride_t; /* element strides of k and v; d contiguous */
   const int32_t* seq_len;    /* host [B]: n of each sequence */
-  const uint8_t* head_mask;  /* host [B*Hkv]: 1 = consistent, 0 = adaptive */
+  const uint8_t* head_mask;  /* host [B*Hkv]: 0 = adaptive, 1 = consistent, 2 = streaming (T = sink + local; Section 4.2.4) */
 } catekv_select_params;
 
 /*
@@ -245,6 +245,16 @@ int catekv_decode_partials(const catekv_cache* cache, const void* q, int32_t Hq,
 int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
                           int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                           size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream);
+
+/*
+ * Attention recall of the kept rows (Section 3.4, the recall curves of the consistent / streaming / Quest /
+ * top-k patterns): for each query head, the share of the full softmax mass that falls on the rows its hybrid
+ * list keeps, recall = exp(lse_kept - lse_full), 0 for an empty list.  lse_kept is the lse_out of a
+ * catekv_decode_attn call over the hybrid cache, lse_full that of a call with the same queries over a cache
+ * that keeps every token.  All three arrays: device float [n].
+ */
+int catekv_attention_recall(const float* lse_kept, const float* lse_full, float* recall, int32_t n,
+                            catekv_stream stream);
 
 /*
  * catekv_append followed by catekv_decode_attn, as one call with one attention launch: the CTA that

@@ -22,6 +22,9 @@ What each function follows
                                       grows by the decoded token.
 * attention, decode_attention       : Algorithm 1, "Attention(q, k, v)"; the
                                       plain softmax-attention definition.
+* attention_recall                  : Section 3.4 (attention weight recall of a
+                                      kept set, Fig. 4).
+* token_budget (streaming type)     : Section 4.2.4 (sink + recent heads).
 
 Parity pins: every function above is pinned by tests that do not re-use it
 (pure-Python brute force, closed forms, hand-worked examples, library
@@ -221,9 +224,18 @@ def pool_scores(C: np.ndarray, S: int, cand_end: int, mode: int, param: int) -> 
     raise ValueError("pool mode")
 
 
-def token_budget(n: int, consistent: bool, budget_consistent: int, eta_adaptive: float) -> int:
-    """T of the head: b for a consistent head, floor(eta * n) for an adaptive one."""
-    if consistent:
+HEAD_ADAPTIVE, HEAD_CONSISTENT, HEAD_STREAMING = 0, 1, 2
+
+
+def token_budget(n: int, head_type: int, budget_consistent: int, eta_adaptive: float, sink: int = 0,
+                 local: int = 0) -> int:
+    """T of the head: b for a consistent head (1), floor(eta * n) for an adaptive one (0), and sink + local for a
+    streaming head (2: attention sinks and recent tokens only, the head type of the DuoAttention comparison in
+    Section 4.2.4)."""
+    head_type = int(head_type)
+    if head_type == HEAD_STREAMING:
+        return int(sink) + int(local)
+    if head_type == HEAD_CONSISTENT:
         return int(budget_consistent)
     if eta_adaptive >= 1.0:
         return n
@@ -285,7 +297,7 @@ def select_compact(qwin_bits: np.ndarray, k_bits: np.ndarray, v_bits: np.ndarray
             if want is not None and (b, h) not in want:
                 idx = np.zeros(0, dtype=np.int64)
             else:
-                T = token_budget(n, bool(head_mask[b, h]), budget_consistent, eta_adaptive)
+                T = token_budget(n, int(head_mask[b, h]), budget_consistent, eta_adaptive, S, Lc)
                 if T >= n or S + Lc >= n:
                     idx = np.arange(n, dtype=np.int64)
                 else:
@@ -394,6 +406,15 @@ def static_head_mask(cv: np.ndarray, r: float) -> np.ndarray:
     for h in order[: H - n_adapt]:
         mask[h] = 1
     return mask
+
+
+def attention_recall(q: np.ndarray, K: np.ndarray, kept: np.ndarray, scale: float) -> float:
+    """Attention recall of a kept set (Section 3.4, the recall curves): the share of the full softmax mass
+    of one decode query that falls on the kept tokens, sum_{j in kept} softmax(scale * K q)_j."""
+    s = (K @ q) * scale
+    p = np.exp(s - s.max())
+    p /= p.sum()
+    return float(p[np.asarray(kept, dtype=np.int64)].sum())
 
 
 def kept_fraction(r: float, eta: float, budget: int, n: int) -> float:

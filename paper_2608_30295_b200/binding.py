@@ -77,6 +77,7 @@ def _load():
         "catekv_decode_combine": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp, sz, vp]),
         "catekv_append_decode_attn": (C.c_int, [C.POINTER(CacheStruct), vp, vp, vp, i32, f32, vp, i32, vp, vp, vp, sz,
                                                 vp, sz, vp]),
+        "catekv_attention_recall": (C.c_int, [vp, vp, vp, i32, vp]),
         "catekv_decode_attn_noalloc": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp]),
     }
     for name, (res, args) in sig.items():
@@ -226,6 +227,16 @@ def catekv_append_decode_attn(cache: Cache, k_new: torch.Tensor, v_new: torch.Te
                                           q.shape[1], sm_scale, out.data_ptr(), od, _dev_ptr(lse_out),
                                           plan.host.data_ptr(), plan.dev.data_ptr(), plan.bytes, plan.ws.data_ptr(),
                                           plan.ws_bytes, _stream()), "catekv_append_decode_attn")
+
+
+def catekv_attention_recall(lse_kept: torch.Tensor, lse_full: torch.Tensor) -> torch.Tensor:
+    """-> recall float32, same shape: exp(lse_kept - lse_full), computed on the device."""
+    assert lse_kept.is_contiguous() and lse_full.is_contiguous() and lse_kept.shape == lse_full.shape
+    assert lse_kept.dtype == torch.float32 and lse_full.dtype == torch.float32
+    out = torch.empty_like(lse_kept)
+    _check(_lib.catekv_attention_recall(lse_kept.data_ptr(), lse_full.data_ptr(), out.data_ptr(), lse_kept.numel(),
+                                        _stream()), "catekv_attention_recall")
+    return out
 
 
 NOALLOC_SCRATCH_BYTES = 4 << 20

@@ -617,6 +617,23 @@ extern "C" int catekv_append(catekv_cache* cache, const void* k_new, const void*
   return CATEKV_OK;
 }
 
+// recall = exp(lse_kept - lse_full): the share of the full attention mass that falls on the kept rows
+__global__ void recall_kernel(const float* lse_kept, const float* lse_full, float* recall, int n) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) recall[i] = (lse_kept[i] == -INFINITY) ? 0.f : expf(lse_kept[i] - lse_full[i]);
+}
+
+extern "C" int catekv_attention_recall(const float* lse_kept, const float* lse_full, float* recall, int32_t n,
+                                       catekv_stream stream) {
+  if (!lse_kept || !lse_full || !recall || n < 0) return CATEKV_ERR_INVALID_ARG;
+  if (n == 0) return CATEKV_OK;
+  CATEKV_CUDA_TRY(launch_pdl(recall_kernel, dim3((n + 255) / 256), dim3(256), 0, (cudaStream_t)stream, lse_kept, lse_full,
+                             recall, (int)n));
+  return CATEKV_OK;
+}
+
 extern "C" int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens) {
   int rc = check_cache(cache);
   if (rc) return rc;

@@ -323,7 +323,9 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
       s.n = n;
       s.job = -1;
       int64_t T;
-      if (p->head_mask[sgi]) T = p->budget_consistent;
+      if (p->head_mask[sgi] > 2) return CATEKV_ERR_INVALID_ARG;
+      if (p->head_mask[sgi] == 2) T = (int64_t)S + Lc;  // streaming head: sinks and recent tokens only
+      else if (p->head_mask[sgi] == 1) T = p->budget_consistent;
       else T = p->eta_adaptive >= 1.f ? n : (int64_t)floor((double)p->eta_adaptive * (double)n);
       if (T >= n || (int64_t)S + Lc >= n) {
         s.keep_all = 1;

@@ -174,3 +174,41 @@ def test_select_full_budget_equals_full_attention(ck):
     ref = np.stack([orc.attention(orc.bf16_to_f64(qb[0, hq]), orc.bf16_to_f64(k[0, hq // 4]),
                                   orc.bf16_to_f64(v[0, hq // 4]), 1 / math.sqrt(128))[0] for hq in range(8)])
     H.check_attention(out[0], None, None, ref, None)
+
+
+def test_streaming_heads_and_attention_recall(ck):
+    # three head types in one launch; recall of each kept set against the oracle's definition
+    w = synth.scaled(synth.WORKLOADS["cfg0"], n=3000, Hq=24, Hkv=6)
+    p = synth.prefill_layer(w, 6)
+    mask = np.array([[2, 1, 0, 1, 2, 0]], dtype=np.uint8)
+    lens = [w.sink + w.local, 256, w.n, 256, w.sink + w.local, w.n]
+    cache = ck.Cache(1, 6, lens, 4, "cuda")
+    full = ck.Cache(1, 6, [w.n] * 6, 4, "cuda")
+    idx = torch.full((6, w.n), -1, dtype=torch.int32, device="cuda")
+    args = (p["q_win"].cuda(), p["k"].cuda(), p["v"].cuda(), p["seq_len"])
+    ck.catekv_select_compact(*args, mask, cache, 256, 1.0, w.sink, w.local, orc.POOL_SLIDING, 7, idx_out=idx)
+    ck.catekv_select_compact(*args, np.zeros((1, 6), dtype=np.uint8), full, 256, 1.0, w.sink, w.local, orc.POOL_NONE, 0)
+    torch.cuda.synchronize()
+    assert list(cache.seg_len) == lens and list(full.seg_len) == [w.n] * 6
+    idx = idx.cpu().numpy()
+    for h in (0, 4):
+        assert list(idx[h, :lens[h]]) == list(range(w.sink)) + list(range(w.n - w.local, w.n))
+    q, _, _ = synth.decode_inputs(w, 6, 0, "cpu", (mask == 1).astype(np.uint8))
+    plan, plan_f = ck.DecodePlan(cache, 8), ck.DecodePlan(full, 8)
+    ck.catekv_decode_plan(cache, plan)
+    ck.catekv_decode_plan(full, plan_f)
+    out = torch.empty((1, 24, 128), dtype=torch.float32, device="cuda")
+    lse_k = torch.empty((1, 24), dtype=torch.float32, device="cuda")
+    lse_f = torch.empty_like(lse_k)
+    ck.catekv_decode_attn(cache, q.cuda(), plan, out, lse_k)
+    ck.catekv_decode_attn(full, q.cuda(), plan_f, out, lse_f)
+    rec = ck.catekv_attention_recall(lse_k, lse_f).cpu().numpy()[0]
+    kb, qb = synth.bits(p["k"]), synth.bits(q)
+    for hq in range(24):
+        h = hq // 4
+        want = orc.attention_recall(orc.bf16_to_f64(qb[0, hq]), orc.bf16_to_f64(kb[0, h]), idx[h, :lens[h]],
+                                    1 / math.sqrt(128))
+        assert rec[hq] == pytest.approx(want, rel=2e-3, abs=1e-6), (hq, rec[hq], want)
+    assert np.allclose(rec[8:12], 1.0, atol=1e-4) and np.allclose(rec[20:24], 1.0, atol=1e-4)  # adaptive: everything kept
+    # consistent heads lean on their planted keys: they recall more mass than the streaming heads of this input
+    assert rec[4:8].mean() > rec[0:4].mean()

@@ -194,3 +194,43 @@ def test_kept_fraction_matches_paper(golden_dir):
     assert sum(lens) / (5 * n) == pytest.approx(orc.kept_fraction(0.4, 1.0, 256, n))
     assert orc.token_budget(1000, False, 64, 0.9) == 900
     assert orc.token_budget(1001, False, 64, 0.9) == 900
+
+
+def test_streaming_head_keeps_sink_and_recent_only():
+    # third head type (Section 4.2.4): budget = sink + local, no top-k slot
+    assert orc.token_budget(5000, orc.HEAD_STREAMING, 256, 0.9, 4, 64) == 68
+    assert orc.token_budget(5000, orc.HEAD_CONSISTENT, 256, 0.9, 4, 64) == 256
+    assert orc.token_budget(5000, orc.HEAD_ADAPTIVE, 256, 0.9, 4, 64) == 4500
+    w = synth.scaled(synth.WORKLOADS["cfg0"], n=600, Hq=12, Hkv=3)
+    p = synth.prefill_layer(w, 0)
+    mask = np.array([[2, 1, 0]], dtype=np.uint8)
+    cache, idx = orc.select_compact(synth.bits(p["q_win"]), synth.bits(p["k"]), synth.bits(p["v"]), p["seq_len"], mask,
+                                    128, 1.0, w.sink, w.local, w.L_obs, orc.POOL_NONE, 0)
+    assert list(idx[0]) == list(range(4)) + list(range(600 - 64, 600))
+    assert len(idx[1]) == 128 and len(idx[2]) == 600
+
+
+def test_attention_recall_pins(golden_dir):
+    # hand example: full weights [1,2,4,2,1,1]/11, kept {0,1,2,5} -> 8/11
+    l = [0.0, math.log(2), math.log(4), math.log(2), 0.0, 0.0]
+    K = np.array([[x, 0.0] for x in l])
+    q = np.array([1.0, 0.0])
+    assert orc.attention_recall(q, K, [0, 1, 2, 5], 1.0) == pytest.approx(8 / 11, rel=1e-14)
+    assert orc.attention_recall(q, K, list(range(6)), 1.0) == pytest.approx(1.0, rel=1e-14)
+    # identical keys: recall = |kept| / n
+    K2 = np.tile(np.array([[0.3, -0.7]]), (10, 1))
+    assert orc.attention_recall(q, K2, [1, 5, 9], 1.0) == pytest.approx(0.3, rel=1e-14)
+    # recall = exp(lse_kept - lse_full), the identity the device path uses; and additivity over disjoint sets
+    rng = np.random.default_rng(50)
+    K3, q3 = rng.standard_normal((200, 16)), rng.standard_normal(16)
+    kept = np.sort(rng.choice(200, 40, replace=False))
+    rest = np.setdiff1d(np.arange(200), kept)
+    _, lse_k = orc.attention(q3, K3[kept], K3[kept], 0.25)
+    _, lse_f = orc.attention(q3, K3, K3, 0.25)
+    r = orc.attention_recall(q3, K3, kept, 0.25)
+    assert r == pytest.approx(math.exp(lse_k - lse_f), rel=1e-12)
+    assert r + orc.attention_recall(q3, K3, rest, 0.25) == pytest.approx(1.0, rel=1e-12)
+    # brute force with Python floats
+    s = [0.25 * sum(float(a) * float(b) for a, b in zip(K3[j], q3)) for j in range(200)]
+    Z = math.fsum(math.exp(x) for x in s)
+    assert r == pytest.approx(math.fsum(math.exp(s[j]) for j in kept) / Z, rel=1e-12)
