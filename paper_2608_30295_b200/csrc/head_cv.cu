@@ -16,8 +16,8 @@ struct CvSeg {
 
 struct CvArgs {
   const CvSeg* segs;
-  const float* A;  // [n_segs][L_obs][row_stride]
-  int64_t seg_stride, row_stride;
+  const float* A;  // [n_segs][L_obs * m], dense
+  int64_t seg_stride;
   int32_t L_obs;
   float alpha;
   float* cv_out;
@@ -37,15 +37,14 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
   const unsigned int* Ab = reinterpret_cast<const unsigned int*>(A);
   const int m = s.m;
   const int N = a.L_obs * m;
-  const int64_t rs = a.row_stride;
   unsigned int thr, need_eq;
-  block_radix_select([&](int e) { return Ab[(size_t)(e / m) * rs + (e % m)]; }, N, (unsigned int)s.need, hist, s_pair,
-                     thr, need_eq);
+  block_radix_select([&](int e) { return Ab[e]; }, N, (unsigned int)s.need, hist, s_pair, thr, need_eq);
   const float phi = __uint_as_float(thr) * a.alpha;
   unsigned long long sum = 0, sum2 = 0;
   for (int j = threadIdx.x; j < m; j += kCvThreads) {
     unsigned int c = 0;
-    for (int i = 0; i < a.L_obs; ++i) c += A[(size_t)i * rs + j] >= phi ? 1u : 0u;
+#pragma unroll 8
+    for (int i = 0; i < a.L_obs; ++i) c += A[(size_t)i * m + j] >= phi ? 1u : 0u;
     sum += c;
     sum2 += (unsigned long long)c * c;
   }
@@ -169,14 +168,12 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   sa.status = (int32_t*)(w8 + W.off_status);
   sa.out = (float*)(w8 + W.off_A);
   sa.out_job_stride = (int64_t)L_obs * W.row_stride;
-  sa.out_row_stride = W.row_stride;
   int rc = score_launch(sa, kScoreMatrix, st);
   if (rc) return rc;
   CvArgs ca;
   ca.segs = (const CvSeg*)(w8 + W.off_segs);
   ca.A = sa.out;
   ca.seg_stride = sa.out_job_stride;
-  ca.row_stride = W.row_stride;
   ca.L_obs = L_obs;
   ca.alpha = alpha;
   ca.cv_out = cv_out;

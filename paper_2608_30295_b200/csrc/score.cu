@@ -343,8 +343,10 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const __grid_const
           if (sub == UPT - 1 && j < j_hi)
             atomicAdd(a.out + (size_t)blockIdx.y * a.out_job_stride + (j - job.j_begin), col_acc * inv_g);
         } else {
-          // group-mean matrix: rows come in runs of G heads per window row; r0 is a multiple of G
+          // group-mean matrix, stored densely ([L_obs][m], m = the job's key range): rows come in runs of G heads per
+          // window row; r0 is a multiple of G
           float* A = a.out + (size_t)blockIdx.y * a.out_job_stride;
+          const int m_cols = job.j_end - job.j_begin;
           int i = r0 / a.G, g = 0;
           float acc = 0.f;
 #pragma unroll 1
@@ -357,7 +359,7 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const __grid_const
                 const bool seen = !a.causal || j <= job.n - a.L_obs + i;
                 acc += seen ? fast_exp2(fmaf(x[c], a.scale_log2, -s_f[rr + c])) : 0.f;
                 if (++g == a.G) {
-                  if (j < j_hi) A[(size_t)i * a.out_row_stride + (j - job.j_begin)] = acc * inv_g;
+                  if (j < j_hi) A[(size_t)i * m_cols + (j - job.j_begin)] = acc * inv_g;
                   acc = 0.f;
                   g = 0;
                   ++i;

@@ -25,8 +25,8 @@ struct ScoreArgs {
   float2* stats_part;     // [n_jobs][n_chunks][kScoreMaxRows]  per-CTA (row max in the log2 domain, row sum)
   float2* stats;          // [n_jobs][kScoreMaxRows]            merged (row max, row sum)
   int32_t* status;        // device word, set to 1 if a tensor-core wait ever expired (never in a healthy run)
-  float* out;             // column sums C[job][j - j_begin] or matrix A[job][i][j - j_begin]
-  int64_t out_job_stride, out_row_stride;
+  float* out;             // column sums C[job][j - j_begin], or the dense matrix A[job][i * m + (j - j_begin)], m = j_end - j_begin
+  int64_t out_job_stride;
 };
 
 enum ScoreMode { kScoreStats = 0, kScoreColsum = 1, kScoreMatrix = 2 };

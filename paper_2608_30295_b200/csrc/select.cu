@@ -391,7 +391,6 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
     sa.status = (int32_t*)(w8 + W.off_status);
     sa.out = (float*)(w8 + W.off_C);
     sa.out_job_stride = W.c_stride;
-    sa.out_row_stride = 0;
     int rc = score_launch(sa, kScoreColsum, st);
     if (rc) return rc;
   }
