@@ -25,6 +25,12 @@ What each function follows
 * attention_recall                  : Section 3.4 (attention weight recall of a
                                       kept set, Fig. 4).
 * token_budget (streaming type)     : Section 4.2.4 (sink + recent heads).
+* retrieval_metadata, retrieval_scores, retrieve_indices
+                                    : Algorithm 1, decoding stage, "Retrival(q,
+                                      cache)" in its query-aware form on adaptive
+                                      heads, with the page criterion of Quest that
+                                      the paper combines with (Section 4.2.2,
+                                      appendix B.2.2; chunk size 8).
 
 Parity pins: every function above is pinned by tests that do not re-use it
 (pure-Python brute force, closed forms, hand-worked examples, library
@@ -415,6 +421,60 @@ def attention_recall(q: np.ndarray, K: np.ndarray, kept: np.ndarray, scale: floa
     p = np.exp(s - s.max())
     p /= p.sum()
     return float(p[np.asarray(kept, dtype=np.int64)].sum())
+
+
+# --------------------------------------------------------------------------
+# Query-aware retrieval on adaptive heads (Algorithm 1: "Retrival(q, cache)")
+# --------------------------------------------------------------------------
+def retrieval_metadata(k_bits: np.ndarray, cs: int):
+    """Per chunk of cs consecutive cached rows: the element-wise maximum and minimum of the keys.
+    k_bits [len, d] -> (kmax, kmin), each [ceil(len / cs), d] float64 (values are bf16 values)."""
+    K = bf16_to_f64(k_bits)
+    L = K.shape[0]
+    nch = (L + cs - 1) // cs
+    kmax = np.empty((nch, K.shape[1]))
+    kmin = np.empty((nch, K.shape[1]))
+    for c in range(nch):
+        blk = K[c * cs:min((c + 1) * cs, L)]
+        kmax[c] = blk.max(axis=0)
+        kmin[c] = blk.min(axis=0)
+    return kmax, kmin
+
+
+def retrieval_scores(q_group: np.ndarray, kmax: np.ndarray, kmin: np.ndarray) -> np.ndarray:
+    """Upper bound of q.k over the rows of every chunk, per query head sum_d max(q_d kmin_d, q_d kmax_d), and the
+    group's score as the maximum over its G query heads.  q_group [G, d] float64 -> [n_chunks]."""
+    s = np.full(kmax.shape[0], -np.inf)
+    for g in range(q_group.shape[0]):
+        q = q_group[g][None, :]
+        s = np.maximum(s, np.maximum(q * kmin, q * kmax).sum(axis=1))
+    return s
+
+
+def retrieve_indices(scores: np.ndarray, n: int, S: int, Lc: int, budget: int, cs: int) -> np.ndarray:
+    """Rows a retrieval head attends to in one step, ascending.
+
+    Chunks start at row 0.  The chunks that hold the first S rows and every chunk from the one holding row
+    n - Lc on are always taken; of the chunks in between, the floor((budget - forced rows) / cs) with the largest
+    score, ties to the lowest index.  budget >= n (or no chunk in between) takes every row.
+    """
+    S2 = (S + cs - 1) // cs * cs                 # sink rows, rounded up to whole chunks
+    cand_end = max(0, (n - Lc)) // cs * cs       # first row of the always-taken tail
+    if budget >= n or cand_end <= S2:
+        return np.arange(n, dtype=np.int64)
+    forced = S2 + (n - cand_end)
+    n_pool = (cand_end - S2) // cs
+    k_sel = max(0, (budget - forced) // cs)
+    if k_sel >= n_pool:
+        return np.arange(n, dtype=np.int64)
+    P = scores[S2 // cs: cand_end // cs]
+    order = np.argsort(-P, kind="stable")[:k_sel]
+    rows = [np.arange(S2, dtype=np.int64)]
+    for c in np.sort(order):
+        lo = S2 + int(c) * cs
+        rows.append(np.arange(lo, lo + cs, dtype=np.int64))
+    rows.append(np.arange(cand_end, n, dtype=np.int64))
+    return np.concatenate(rows)
 
 
 def kept_fraction(r: float, eta: float, budget: int, n: int) -> float:
