@@ -246,6 +246,44 @@ int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, 
                           int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                           size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream);
 
+/* ---------------------------------------------------------------- query-aware retrieval */
+
+/*
+ * Algorithm 1, decoding stage: "k, v = Retrival(q, cache)" on adaptive heads in its query-aware form, with the
+ * page criterion of Quest (the retrieval method the paper combines with, chunk size 8; Section 4.2.2 and
+ * appendix B.2.2).  The full list of a retrieval head stays in `cache`; every step a subset of its rows is
+ * gathered into the same segment of a second, small cache (`step_cache`, same B and Hkv) on which
+ * catekv_decode_attn then runs unchanged.
+ *
+ *   metadata  per chunk of chunk_size consecutive cached rows (chunks start at row 0 of a segment) the
+ *             element-wise maximum and minimum of the keys: device bf16 [total_rows / chunk_size][2][d].
+ *             chunk_size must divide 128.  catekv_retrieval_build fills it for all current rows of all
+ *             segments; catekv_retrieval_append folds in the row that the preceding catekv_append (or
+ *             catekv_append_decode_attn) stored, k_new being that call's k_new.
+ *   score     bound(c) = max over the group's G query heads of sum_d max(q_d kmin_d, q_d kmax_d), an upper
+ *             bound of q.k over the chunk's rows (fp32).
+ *   select    (segments with retrieval_mask[s] != 0 and more than `budget` rows) the chunks holding the first
+ *             `sink` rows and every chunk from the one holding row len - local on are always taken; of the
+ *             chunks in between the floor((budget - forced rows) / chunk_size) with the largest bound, ties to
+ *             the lowest chunk.  Other segments are copied whole.
+ *   gather    the taken rows, ascending, K and V; step_cache->seg_len (device and host) is set; the kept
+ *             length depends only on the lengths and the parameters, never on the scores.
+ *
+ *   q         device bf16 [B, Hq, d], this step's queries
+ *   idx_out   device int32 [B*Hkv, idx_stride] or NULL: the rows taken from each segment
+ *   ws        device scratch of at least catekv_retrieve_workspace_bytes(B, Hkv, longest segment)
+ * Errors: CATEKV_ERR_CAPACITY if a kept list does not fit its segment of step_cache (nothing launched).
+ */
+size_t catekv_retrieval_meta_bytes(const catekv_cache* cache, int32_t chunk_size);
+int catekv_retrieval_build(const catekv_cache* cache, int32_t chunk_size, void* meta, catekv_stream stream);
+int catekv_retrieval_append(const catekv_cache* cache, int32_t chunk_size, const void* k_new, void* meta,
+                            catekv_stream stream);
+size_t catekv_retrieve_workspace_bytes(int32_t B, int32_t Hkv, int32_t max_len);
+int catekv_retrieve_compact(const catekv_cache* cache, const void* meta, int32_t chunk_size, const void* q, int32_t Hq,
+                            const uint8_t* retrieval_mask, int32_t budget, int32_t sink, int32_t local,
+                            catekv_cache* step_cache, int32_t* idx_out, int64_t idx_stride, void* ws, size_t ws_bytes,
+                            catekv_stream stream);
+
 /*
  * Attention recall of the kept rows (Section 3.4, the recall curves of the consistent / streaming / Quest /
  * top-k patterns): for each query head, the share of the full softmax mass that falls on the rows its hybrid

@@ -78,6 +78,12 @@ def _load():
         "catekv_append_decode_attn": (C.c_int, [C.POINTER(CacheStruct), vp, vp, vp, i32, f32, vp, i32, vp, vp, vp, sz,
                                                 vp, sz, vp]),
         "catekv_attention_recall": (C.c_int, [vp, vp, vp, i32, vp]),
+        "catekv_retrieval_meta_bytes": (sz, [C.POINTER(CacheStruct), i32]),
+        "catekv_retrieval_build": (C.c_int, [C.POINTER(CacheStruct), i32, vp, vp]),
+        "catekv_retrieval_append": (C.c_int, [C.POINTER(CacheStruct), i32, vp, vp, vp]),
+        "catekv_retrieve_workspace_bytes": (sz, [i32, i32, i32]),
+        "catekv_retrieve_compact": (C.c_int, [C.POINTER(CacheStruct), vp, i32, vp, i32, vp, i32, i32, i32,
+                                              C.POINTER(CacheStruct), vp, i64, vp, sz, vp]),
         "catekv_decode_attn_noalloc": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp]),
     }
     for name, (res, args) in sig.items():
@@ -237,6 +243,41 @@ def catekv_attention_recall(lse_kept: torch.Tensor, lse_full: torch.Tensor) -> t
     _check(_lib.catekv_attention_recall(lse_kept.data_ptr(), lse_full.data_ptr(), out.data_ptr(), lse_kept.numel(),
                                         _stream()), "catekv_attention_recall")
     return out
+
+
+def catekv_retrieval_meta(cache: Cache, chunk_size: int) -> torch.Tensor:
+    """An uninitialised metadata buffer of the right size for `cache` (memory only)."""
+    n = _lib.catekv_retrieval_meta_bytes(C.byref(cache.struct), chunk_size)
+    if n == 0:
+        raise CatekvError(ERR_UNSUPPORTED, "catekv_retrieval_meta_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=cache.device)
+
+
+def catekv_retrieval_build(cache: Cache, chunk_size: int, meta: torch.Tensor):
+    _check(_lib.catekv_retrieval_build(C.byref(cache.struct), chunk_size, meta.data_ptr(), _stream()),
+           "catekv_retrieval_build")
+
+
+def catekv_retrieval_append(cache: Cache, chunk_size: int, k_new: torch.Tensor, meta: torch.Tensor):
+    assert k_new.is_contiguous()
+    _check(_lib.catekv_retrieval_append(C.byref(cache.struct), chunk_size, k_new.data_ptr(), meta.data_ptr(), _stream()),
+           "catekv_retrieval_append")
+
+
+def catekv_retrieve_compact(cache: Cache, meta: torch.Tensor, chunk_size: int, q: torch.Tensor, retrieval_mask,
+                            budget: int, sink: int, local: int, step_cache: Cache,
+                            idx_out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None):
+    assert q.is_contiguous() and q.dtype == torch.bfloat16
+    retrieval_mask = np.ascontiguousarray(retrieval_mask, dtype=np.uint8).reshape(-1)
+    if ws is None:
+        ws = torch.empty(_lib.catekv_retrieve_workspace_bytes(cache.B, cache.Hkv, int(cache.seg_len.max())),
+                         dtype=torch.uint8, device=cache.device)
+    stride = 0 if idx_out is None else idx_out.stride(0)
+    _check(_lib.catekv_retrieve_compact(C.byref(cache.struct), meta.data_ptr(), chunk_size, q.data_ptr(), q.shape[1],
+                                        _np_ptr(retrieval_mask), budget, sink, local, C.byref(step_cache.struct),
+                                        _dev_ptr(idx_out), stride, ws.data_ptr(), ws.numel(), _stream()),
+           "catekv_retrieve_compact")
+    return ws
 
 
 NOALLOC_SCRATCH_BYTES = 4 << 20

@@ -7,30 +7,9 @@
 
 #include "radix.cuh"
 #include "score.cuh"
+#include "select.cuh"
 
 namespace catekv {
-
-struct SelSeg {
-  int32_t n;         // tokens of the sequence
-  int32_t keep_all;  // 1: straight copy of all n rows
-  int32_t job;       // scoring job index, -1 if none (keep_all, or nothing to select)
-  int32_t k_sel;     // candidates (tokens, or chunks in CHUNK mode) to select
-  int32_t n_pool;    // pooled entries (candidate tokens, or chunks)
-  int32_t cand_end;  // candidates are tokens [sink, cand_end)
-  int32_t len_ub;    // upper bound of the kept length (exact except for a short last chunk)
-  int32_t reserved;
-};
-
-struct TopkArgs {
-  const SelSeg* segs;
-  const float* C;       // [n_jobs][c_stride] criticality of tokens [0, n - L_obs)
-  float* P;             // [n_jobs][c_stride] pooled scores (scratch)
-  int64_t c_stride;
-  int32_t* idx;         // [n_segs][idx_stride] kept indices (scratch)
-  int64_t idx_stride;
-  int32_t* seg_len_dev;
-  int32_t sink, local, L_obs, pool_mode, pool_param;
-};
 
 constexpr int kTopkThreads = 1024;
 
@@ -84,7 +63,9 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     // ---- pooling (four entries per thread and step, so that several loads are in flight)
     const float* __restrict__ Cr = C;
     float* __restrict__ Pw = P;
-    if (a.pool_mode == CATEKV_POOL_NONE) {
+    if (a.pool_mode == kPoolPrescored) {
+      // P was filled by the caller's scoring kernel
+    } else if (a.pool_mode == CATEKV_POOL_NONE) {
       for (int c0 = tid; c0 < s.n_pool; c0 += 4 * kTopkThreads) {
         float vv[4];
 #pragma unroll
@@ -140,7 +121,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     block_radix_select([&](int c) { return Pb[c]; }, s.n_pool, (unsigned int)s.k_sel, hist, s_pair, thr, need_eq);
     // ---- ordered compaction, four consecutive entries per thread and step
     unsigned long long run = 0;  // packed: low = entries above the threshold so far, high = entries equal to it
-    const int cs = a.pool_mode == CATEKV_POOL_CHUNK ? a.pool_param : 1;
+    const int cs = (a.pool_mode == CATEKV_POOL_CHUNK || a.pool_mode == kPoolPrescored) ? a.pool_param : 1;
     for (int base = 0; base < s.n_pool; base += 4 * kTopkThreads) {
       const int c4 = base + tid * 4;
       unsigned int v[4];
@@ -185,8 +166,9 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     }
   }
   for (int i = tid; i < S; i += kTopkThreads) idx[i] = i;
-  for (int i = tid; i < a.local; i += kTopkThreads) idx[S + n_sel_tokens + i] = s.n - a.local + i;
-  if (tid == 0) a.seg_len_dev[seg] = S + n_sel_tokens + a.local;
+  const int n_tail = s.n - s.cand_end;  // the always-kept most recent tokens
+  for (int i = tid; i < n_tail; i += kTopkThreads) idx[S + n_sel_tokens + i] = s.cand_end + i;
+  if (tid == 0) a.seg_len_dev[seg] = S + n_sel_tokens + n_tail;
 }
 
 // keep_all segments: seg_len = n
@@ -194,22 +176,6 @@ __global__ void set_full_len_kernel(const SelSeg* segs, int32_t* seg_len_dev, in
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n_segs && segs[i].keep_all) seg_len_dev[i] = segs[i].n;
 }
-
-struct GatherArgs {
-  const SelSeg* segs;
-  const int32_t* idx;
-  int64_t idx_stride;
-  const uint8_t* k;
-  const uint8_t* v;
-  int64_t sb, sh, st;  // byte strides
-  uint8_t* k_pool;
-  uint8_t* v_pool;
-  const int32_t* seg_off;
-  const int32_t* seg_len_dev;
-  int32_t* idx_out;
-  int64_t idx_out_stride;
-  int32_t Hkv;
-};
 
 constexpr int kGatherRowsPerBlock = 64;
 
@@ -221,7 +187,8 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = seg / a.Hkv, h = seg % a.Hkv;
   const int64_t off = a.seg_off[seg];
-  const uint8_t* src_base = (lane < 16 ? a.k : a.v) + b * a.sb + h * a.sh + (lane & 15) * 16;
+  const uint8_t* src_base = (lane < 16 ? a.k : a.v) + (lane & 15) * 16 +
+                            (a.src_seg_off ? (int64_t)a.src_seg_off[seg] * a.st : b * a.sb + h * a.sh);
   uint8_t* dst_base = (lane < 16 ? a.k_pool : a.v_pool) + off * kRowBytes + (lane & 15) * 16;
   const int r0 = blockIdx.x * kGatherRowsPerBlock;
 #pragma unroll 4
@@ -233,6 +200,23 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
     *reinterpret_cast<uint4*>(dst_base + (int64_t)r * kRowBytes) = val;
     if (a.idx_out && lane == 0) a.idx_out[(size_t)seg * a.idx_out_stride + r] = tok;
   }
+}
+
+int launch_topk(const TopkArgs& a, int n_segs, cudaStream_t stream) {
+  topk_kernel<<<n_segs, kTopkThreads, 0, stream>>>(a);
+  CATEKV_CUDA_TRY(cudaGetLastError());
+  return CATEKV_OK;
+}
+int launch_set_full_len(const SelSeg* segs, int32_t* seg_len_dev, int n_segs, cudaStream_t stream) {
+  set_full_len_kernel<<<(n_segs + 255) / 256, 256, 0, stream>>>(segs, seg_len_dev, n_segs);
+  CATEKV_CUDA_TRY(cudaGetLastError());
+  return CATEKV_OK;
+}
+int launch_gather(const GatherArgs& a, int max_len, int n_segs, cudaStream_t stream) {
+  if (max_len <= 0) return CATEKV_OK;
+  gather_kernel<<<dim3((max_len + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock, n_segs), 256, 0, stream>>>(a);
+  CATEKV_CUDA_TRY(cudaGetLastError());
+  return CATEKV_OK;
 }
 
 static int keys_per_cta_for(int n_segs, int n_sc_max) {
@@ -403,7 +387,6 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   ta.idx_stride = W.idx_stride;
   ta.seg_len_dev = cache->seg_len_dev;
   ta.sink = S;
-  ta.local = Lc;
   ta.L_obs = p->L_obs;
   ta.pool_mode = p->pool_mode;
   ta.pool_param = p->pool_param;
@@ -428,6 +411,7 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   ga.idx_out = idx_out;
   ga.idx_out_stride = idx_stride;
   ga.Hkv = p->Hkv;
+  ga.src_seg_off = nullptr;
   gather_kernel<<<dim3((max_len_ub + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock, n_segs), 256, 0, st>>>(ga);
   CATEKV_CUDA_TRY(cudaGetLastError());
 

@@ -1,0 +1,55 @@
+// Structures and launchers shared by the prefill-end selection (catekv_select_compact) and the per-step
+// query-aware retrieval (catekv_retrieve_compact): top-k over pooled scores and the row gather.
+#pragma once
+
+#include "common.cuh"
+
+namespace catekv {
+
+constexpr int kPoolPrescored = 3;  // internal pool mode: P already holds one score per chunk of pool_param tokens
+
+struct SelSeg {
+  int32_t n;         // tokens of the sequence
+  int32_t keep_all;  // 1: straight copy of all n rows
+  int32_t job;       // scoring job index, -1 if none (keep_all, or nothing to select)
+  int32_t k_sel;     // candidates (tokens, or chunks in CHUNK mode) to select
+  int32_t n_pool;    // pooled entries (candidate tokens, or chunks)
+  int32_t cand_end;  // candidates are tokens [sink, cand_end)
+  int32_t len_ub;    // upper bound of the kept length (exact except for a short last chunk)
+  int32_t reserved;
+};
+
+struct TopkArgs {
+  const SelSeg* segs;
+  const float* C;       // [n_jobs][c_stride] criticality of tokens [0, n - L_obs)
+  float* P;             // [n_jobs][c_stride] pooled scores (scratch)
+  int64_t c_stride;
+  int32_t* idx;         // [n_segs][idx_stride] kept indices (scratch)
+  int64_t idx_stride;
+  int32_t* seg_len_dev;
+  int32_t sink, L_obs, pool_mode, pool_param;  // the always-kept tail of a segment is [cand_end, n)
+};
+
+struct GatherArgs {
+  const SelSeg* segs;
+  const int32_t* idx;
+  int64_t idx_stride;
+  const uint8_t* k;
+  const uint8_t* v;
+  int64_t sb, sh, st;  // byte strides
+  const int32_t* src_seg_off;  // if set: the source row of token t of segment s is src_seg_off[s] + t (sb, sh unused)
+  uint8_t* k_pool;
+  uint8_t* v_pool;
+  const int32_t* seg_off;
+  const int32_t* seg_len_dev;
+  int32_t* idx_out;
+  int64_t idx_out_stride;
+  int32_t Hkv;
+};
+
+
+int launch_topk(const TopkArgs& a, int n_segs, cudaStream_t stream);
+int launch_set_full_len(const SelSeg* segs, int32_t* seg_len_dev, int n_segs, cudaStream_t stream);
+int launch_gather(const GatherArgs& a, int max_len, int n_segs, cudaStream_t stream);
+
+}  // namespace catekv

@@ -1,0 +1,156 @@
+"""GPU parity: query-aware retrieval on adaptive heads (metadata, chunk selection, gathered attention)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import catekv_oracle as orc
+from workloads import synth
+import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ck():
+    import paper_2608_30295_b200 as pkg
+    assert torch.cuda.is_available()
+    return pkg.binding
+
+
+def _meta_of(ck, cache, meta, cs, seg, n_chunks):
+    c0 = int(cache.seg_off[seg]) // cs
+    m = synth.bits(meta.view(torch.bfloat16).view(-1, 2, 128)[c0:c0 + n_chunks])
+    return orc.bf16_to_f64(m[:, 0]), orc.bf16_to_f64(m[:, 1])
+
+
+def _check_selection(got, scores, n, S, Lc, budget, cs, where):
+    """Band-aware comparison of the retrieved rows with the oracle (fp32 bounds against fp64 bounds)."""
+    want = orc.retrieve_indices(scores, n, S, Lc, budget, cs)
+    assert got.shape == want.shape, (where, got.shape, want.shape)
+    assert np.all(np.diff(got) > 0), where
+    if np.array_equal(got, want):
+        return True
+    S2 = (S + cs - 1) // cs * cs
+    cand_end = (n - Lc) // cs * cs
+    P = scores[S2 // cs: cand_end // cs]
+    k_sel = (budget - S2 - (n - cand_end)) // cs
+    Pk = np.sort(P)[::-1][k_sel - 1]
+    tol = 1e-4 * max(1.0, abs(Pk))
+    mid = got[S2:len(got) - (n - cand_end)]
+    units = np.unique((mid - S2) // cs)
+    assert len(units) == k_sel, where
+    assert set(np.nonzero(P > Pk + tol)[0].tolist()) <= set(units.tolist()), (where, "missing clear winners")
+    assert set(units.tolist()) <= set(np.nonzero(P >= Pk - tol)[0].tolist()), (where, "took a clear loser")
+    return False
+
+
+@pytest.mark.parametrize("cs,G", [(8, 4), (8, 7), (16, 1), (1, 2)])
+def test_retrieval_matches_oracle(ck, cs, G):
+    lens = [700, 64, 2049, 5, 1300, 0]
+    B, Hkv = 2, 3
+    oc = H.random_cache(B, Hkv, lens, seed=70 + cs)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=8)
+    meta = ck.catekv_retrieval_meta(cache, cs)
+    ck.catekv_retrieval_build(cache, cs, meta)
+    torch.cuda.synchronize()
+    # metadata: bit-exact element-wise extremes
+    for s, L in enumerate(lens):
+        if L:
+            kmax, kmin = orc.retrieval_metadata(oc.k_rows[s], cs)
+            gmax, gmin = _meta_of(ck, cache, meta, cs, s, kmax.shape[0])
+            assert np.array_equal(gmax, kmax) and np.array_equal(gmin, kmin), s
+    q = synth.randn_bf16((B, Hkv * G, 128), "cuda", 71, "q", cs)
+    qb = orc.bf16_to_f64(synth.bits(q))
+    mask = np.array([1, 1, 1, 1, 0, 1], dtype=np.uint8)
+    budget, sink, local = 256, 4, 32
+    want_len = []
+    for s, L in enumerate(lens):
+        if mask[s] and L > budget:
+            want_len.append(len(orc.retrieve_indices(np.zeros((L + cs - 1) // cs), L, sink, local, budget, cs)))
+        else:
+            want_len.append(L)
+    step = ck.Cache(B, Hkv, want_len, 0, "cuda")
+    idx = torch.full((B * Hkv, max(lens)), -1, dtype=torch.int32, device="cuda")
+    ck.catekv_retrieve_compact(cache, meta, cs, q, mask, budget, sink, local, step, idx_out=idx)
+    torch.cuda.synchronize()
+    assert list(step.seg_len) == want_len and step.seg_len_dev.cpu().tolist() == want_len
+    idx = idx.cpu().numpy()
+    soc = orc.HybridCache(B, Hkv, 128)
+    for s, L in enumerate(lens):
+        got = idx[s, :want_len[s]].astype(np.int64)
+        if mask[s] and L > budget:
+            kmax, kmin = orc.retrieval_metadata(oc.k_rows[s], cs)
+            b, h = divmod(s, Hkv)
+            scores = orc.retrieval_scores(qb[b, h * G:(h + 1) * G], kmax, kmin)
+            _check_selection(got, scores, L, sink, local, budget, cs, f"seg {s}")
+        else:
+            assert np.array_equal(got, np.arange(L))
+        o = int(step.seg_off[s])
+        assert np.array_equal(synth.bits(step.k_pool[o:o + want_len[s]]), oc.k_rows[s][got])
+        assert np.array_equal(synth.bits(step.v_pool[o:o + want_len[s]]), oc.v_rows[s][got])
+        soc.k_rows.append(oc.k_rows[s][got])
+        soc.v_rows.append(oc.v_rows[s][got])
+    # attention over the step cache == oracle attention over the retrieved rows
+    plan = ck.DecodePlan(step, 12)
+    ck.catekv_decode_plan(step, plan)
+    out = torch.empty((B, Hkv * G, 128), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, Hkv * G), dtype=torch.float32, device="cuda")
+    ck.catekv_decode_attn(step, q, plan, out, lse)
+    ref, ref_lse = orc.decode_attention(soc, synth.bits(q))
+    H.check_attention(out, None, lse, ref, ref_lse, f"cs={cs} G={G}")
+
+
+def test_retrieval_metadata_follows_appends(ck):
+    cs = 8
+    lens = [100, 7, 0, 64]
+    oc = H.random_cache(1, 4, lens, seed=75)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=20)
+    meta = ck.catekv_retrieval_meta(cache, cs)
+    ck.catekv_retrieval_build(cache, cs, meta)
+    for step in range(20):
+        kn = synth.randn_bf16((1, 4, 128), "cuda", 75, "kn", step)
+        vn = synth.randn_bf16((1, 4, 128), "cuda", 75, "vn", step)
+        ck.catekv_append(cache, kn, vn)
+        ck.catekv_retrieval_append(cache, cs, kn, meta)
+        oc.append(synth.bits(kn), synth.bits(vn))
+    torch.cuda.synchronize()
+    for s in range(4):
+        kmax, kmin = orc.retrieval_metadata(oc.k_rows[s], cs)
+        gmax, gmin = _meta_of(ck, cache, meta, cs, s, kmax.shape[0])
+        assert np.array_equal(gmax, kmax) and np.array_equal(gmin, kmin), s
+
+
+def test_retrieval_finds_loud_keys_and_budget_covers_all(ck):
+    # quiet keys plus a few loud ones on the direction the queries lean on: all loud rows are retrieved
+    rng = np.random.default_rng(76)
+    n, G = 4096, 4
+    c = rng.standard_normal(128)
+    c /= np.linalg.norm(c)
+    K = 0.05 * rng.standard_normal((n, 128))
+    loud = np.sort(rng.choice(np.arange(16, n - 80), 12, replace=False))
+    K[loud] += 3.0 * c
+    oc = orc.HybridCache(1, 1, 128)
+    oc.k_rows.append(orc.f64_to_bf16(K))
+    oc.v_rows.append(orc.f64_to_bf16(rng.standard_normal((n, 128))))
+    cache = H.device_cache_from_oracle(ck, oc, 0)
+    meta = ck.catekv_retrieval_meta(cache, 8)
+    ck.catekv_retrieval_build(cache, 8, meta)
+    q = synth.from_bits(orc.f64_to_bf16(0.1 * rng.standard_normal((1, G, 128)) + 3.0 * c), "cuda")
+    step = ck.Cache(1, 1, [n], 0, "cuda")
+    idx = torch.full((1, n), -1, dtype=torch.int32, device="cuda")
+    ck.catekv_retrieve_compact(cache, meta, 8, q, [1], 256, 4, 64, step, idx_out=idx)
+    torch.cuda.synchronize()
+    got = idx[0, :int(step.seg_len[0])].cpu().numpy()
+    assert len(got) == 256 and set(loud.tolist()) <= set(got.tolist())
+    # a budget at or above the length takes every row, as does an unmasked segment
+    for mask, budget in (([1], n), ([0], 64)):
+        ck.catekv_retrieve_compact(cache, meta, 8, q, mask, budget, 4, 64, step, idx_out=idx)
+        torch.cuda.synchronize()
+        assert int(step.seg_len[0]) == n and torch.equal(idx[0].cpu(), torch.arange(n, dtype=torch.int32))
+    # a step cache that is too small is refused before anything runs
+    small = ck.Cache(1, 1, [128], 0, "cuda")
+    with pytest.raises(ck.CatekvError) as e:
+        ck.catekv_retrieve_compact(cache, meta, 8, q, [1], 256, 4, 64, small)
+    assert e.value.code == ck.ERR_CAPACITY
