@@ -11,8 +11,6 @@
 //              catekv_decode_attn then runs unchanged
 #include <math.h>
 
-#include <vector>
-
 #include "select.cuh"
 
 namespace catekv {
@@ -77,56 +75,154 @@ struct RetJob {
   int32_t n_pool;      // candidate chunks
 };
 
-// One warp per candidate chunk; a lane owns four d of both extremes and of the G query rows.
-__global__ void __launch_bounds__(256) retrieval_score_kernel(const RetJob* jobs, const uint8_t* meta, const uint16_t* q, int Hq,
-                                                              int G, float* P, int64_t p_stride) {
-  const RetJob job = jobs[blockIdx.y];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // q+ = max(q, 0), q- = min(q, 0) of the group's heads, this lane's four d
-  float qp[kMaxG][4], qn[kMaxG][4];
-#pragma unroll
-  for (int g = 0; g < kMaxG; ++g) {
-    uint2 w = make_uint2(0u, 0u);
-    if (g < G) w = *reinterpret_cast<const uint2*>(q + ((int64_t)job.b * Hq + job.h * G + g) * kD + lane * 4);
-    const float v[4] = {bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y)};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) qp[g][e] = fmaxf(v[e], 0.f), qn[g][e] = fminf(v[e], 0.f);
-  }
-  for (int c = blockIdx.x * 8 + warp; c < job.n_pool; c += gridDim.x * 8) {
-    const uint8_t* src = meta + ((int64_t)job.chunk0 + c) * (2 * kRowBytes) + lane * 8;
-    const uint2 a = *reinterpret_cast<const uint2*>(src), b = *reinterpret_cast<const uint2*>(src + kRowBytes);
-    const float mx[4] = {bf16_lo(a.x), bf16_hi(a.x), bf16_lo(a.y), bf16_hi(a.y)};
-    const float mn[4] = {bf16_lo(b.x), bf16_hi(b.x), bf16_lo(b.y), bf16_hi(b.y)};
-    float best = -INFINITY;
-#pragma unroll
-    for (int g = 0; g < kMaxG; ++g) {
-      if (g < G) {
-        float s = 0.f;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) s = fmaf(qp[g][e], mx[e], fmaf(qn[g][e], mn[e], s));
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        best = fmaxf(best, s);
-      }
-    }
-    if (lane == 0) P[(size_t)blockIdx.y * p_stride + c] = best;
-  }
-}
-
 // Monotone map of arbitrary finite floats to non-negative floats whose bit patterns order the same way as the
 // values (what the radix select of the top-k kernel needs): flip so that larger values get larger unsigned
-// patterns, then clear the sign by halving the range.  Ties are preserved (it is injective on 31 bits after the
-// least significant bit is dropped, so values one ulp apart may merge: within the parity tolerance band).
-__global__ void monotone_key_kernel(float* P, int64_t n) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const uint32_t u = __float_as_uint(P[i]);
+// patterns, then clear the sign by halving the range.  Values one ulp apart may merge into a tie: within the
+// parity tolerance band.
+__device__ __forceinline__ float monotone_key(float x) {
+  const uint32_t u = __float_as_uint(x);
   const uint32_t k = (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // unsigned order == float order
-  P[i] = __uint_as_float(k >> 1);                                 // non-negative finite float pattern
+  return __uint_as_float(k >> 1);                                 // non-negative pattern
+}
+
+// bound(c, g) = [kmax_c | kmin_c] . [max(q_g, 0) | min(q_g, 0)]: a [chunks x 256] x [256 x 8 heads] product, so the
+// tensor cores take it (mma.m16n8k16, chunks are M, the group's heads N = 8).  A CTA streams 64-chunk tiles of the
+// metadata (32 KB, contiguous) through a 3-stage cp.async pipeline into XOR-swizzled shared memory; each of its 4
+// warps owns 16 chunks of a tile, takes the maximum over the heads and writes one score per chunk.
+constexpr int kRsTile = 64, kRsThreads = 128, kRsStages = 3;
+constexpr int kRsRowBytes = 2 * kRowBytes;                 // one chunk: 256 bf16
+constexpr int kRsStageBytes = kRsTile * kRsRowBytes;
+constexpr int kRsSmem = kRsStages * kRsStageBytes + kMaxG * kRsRowBytes;
+__device__ __forceinline__ uint32_t rs_off(int row, int piece) {  // 16-byte piece (0..31) of a 512-byte row
+  return (uint32_t)(row * kRsRowBytes + ((piece ^ (row & 7)) << 4));
+}
+
+__global__ void __launch_bounds__(kRsThreads, 2) retrieval_score_kernel(const RetJob* jobs, const uint8_t* meta, const uint16_t* q,
+                                                                        int Hq, int G, float* P, int64_t p_stride) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const RetJob job = jobs[blockIdx.y];
+  if (job.n_pool == 0) return;  // this segment selects nothing
+  // this CTA's chunks: an equal share, in whole tiles
+  const int tiles_total = (job.n_pool + kRsTile - 1) / kRsTile;
+  const int tiles_per = (tiles_total + gridDim.x - 1) / gridDim.x;
+  const int tile_lo = blockIdx.x * tiles_per, tile_hi = min(tiles_total, tile_lo + tiles_per);
+  if (tile_lo >= tile_hi) return;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const uint32_t s_stage = smem_u32(smem);
+  uint16_t* s_q = reinterpret_cast<uint16_t*>(smem + kRsStages * kRsStageBytes);  // [8][256]: max(q,0) | min(q,0)
+  const uint8_t* src0 = meta + (int64_t)job.chunk0 * kRsRowBytes;
+  auto issue = [&](int tile) {
+    if (tile < tile_hi) {
+      const uint32_t sb = s_stage + ((tile - tile_lo) % kRsStages) * kRsStageBytes;
+      const int c0 = tile * kRsTile;
+#pragma unroll
+      for (int i = 0; i < (kRsTile * 32) / kRsThreads; ++i) {
+        const int id = tid + i * kRsThreads;
+        const int r = id >> 5, pc = id & 31;
+        const int ok = (c0 + r) < job.n_pool ? 16 : 0;
+        cp_async16(sb + rs_off(r, pc), src0 + (int64_t)(ok ? c0 + r : 0) * kRsRowBytes + pc * 16, ok);
+      }
+    }
+    cp_async_commit();
+  };
+  issue(tile_lo);
+  issue(tile_lo + 1);
+  // the group's queries, split by sign (exact in bf16); heads >= G are zero
+  for (int i = tid; i < kMaxG * kD; i += kRsThreads) {
+    const int hd = i / kD, e = i % kD;
+    uint16_t v = 0;
+    if (hd < G) v = q[((int64_t)job.b * Hq + job.h * G + hd) * kD + e];
+    const bool neg = v & 0x8000u;
+    s_q[hd * 256 + e] = neg ? 0 : v;
+    s_q[hd * 256 + 128 + e] = neg ? v : 0;
+  }
+  __syncthreads();
+  uint32_t qf[16][2];
+#pragma unroll
+  for (int ks = 0; ks < 16; ++ks) {
+    qf[ks][0] = *reinterpret_cast<const uint32_t*>(s_q + g * 256 + ks * 16 + 2 * t);
+    qf[ks][1] = *reinterpret_cast<const uint32_t*>(s_q + g * 256 + ks * 16 + 8 + 2 * t);
+  }
+  for (int tile = tile_lo; tile < tile_hi; ++tile) {
+    cp_async_wait<kRsStages - 2>();
+    __syncthreads();
+    issue(tile + kRsStages - 1);
+    const uint32_t sb = s_stage + ((tile - tile_lo) % kRsStages) * kRsStageBytes;
+    const int row0 = warp * 16;
+    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb2[4] = {0.f, 0.f, 0.f, 0.f};
+    const int r = row0 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    const int padd = lane >> 4;
+#pragma unroll
+    for (int ks = 0; ks < 16; ks += 2) {
+      uint32_t af[4];
+      ldmatrix_x4(af, sb + rs_off(r, ks * 2 + padd));
+      mma_bf16_16816(sa, af, qf[ks][0], qf[ks][1]);
+      ldmatrix_x4(af, sb + rs_off(r, ks * 2 + 2 + padd));
+      mma_bf16_16816(sb2, af, qf[ks + 1][0], qf[ks + 1][1]);
+    }
+    // c0, c1: chunk row0 + g, heads 2t, 2t+1;  c2, c3: chunk row0 + g + 8
+    float lo = fmaxf(2 * t < G ? sa[0] + sb2[0] : -INFINITY, 2 * t + 1 < G ? sa[1] + sb2[1] : -INFINITY);
+    float hi = fmaxf(2 * t < G ? sa[2] + sb2[2] : -INFINITY, 2 * t + 1 < G ? sa[3] + sb2[3] : -INFINITY);
+#pragma unroll
+    for (int o = 1; o <= 2; o <<= 1) {
+      lo = fmaxf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (t == 0) {
+      const int c = tile * kRsTile + row0 + g;
+      if (c < job.n_pool) P[(size_t)blockIdx.y * p_stride + c] = monotone_key(lo);
+      if (c + 8 < job.n_pool) P[(size_t)blockIdx.y * p_stride + c + 8] = monotone_key(hi);
+    }
+  }
+  cp_async_wait<0>();
+}
+
+// Per-segment decisions (what to keep, how many chunks to select) from the device's own lengths, so that a step
+// needs no host-to-device copy.  The host makes the same decisions from its mirror for the capacity check.
+struct RetParams {
+  int32_t cs, budget, sink2 /* sink rounded up to whole chunks */, local, Hkv;
+};
+__host__ __device__ inline SelSeg retrieval_decide(int n, bool enabled, const RetParams& p) {
+  SelSeg d = {};
+  d.n = n;
+  d.job = -1;
+  d.keep_all = 1;
+  d.len_ub = n;
+  if (enabled && p.budget < n) {
+    const int cand_end = (n - p.local > 0 ? n - p.local : 0) / p.cs * p.cs;  // first row of the always-taken tail
+    if (cand_end > p.sink2) {
+      const int forced = p.sink2 + (n - cand_end);
+      const int n_pool = (cand_end - p.sink2) / p.cs;
+      const int k_sel = p.budget - forced > 0 ? (p.budget - forced) / p.cs : 0;
+      if (k_sel < n_pool) {
+        d.keep_all = 0;
+        d.cand_end = cand_end;
+        d.n_pool = n_pool;
+        d.k_sel = k_sel;
+        d.len_ub = forced + k_sel * p.cs;
+      }
+    }
+  }
+  return d;
+}
+__global__ void retrieval_plan_kernel(const int32_t* seg_len, const int32_t* seg_off, const uint8_t* mask, RetParams p,
+                                      SelSeg* segs, RetJob* jobs, int n_segs) {
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= n_segs) return;
+  SelSeg d = retrieval_decide(seg_len[s], mask[s] != 0, p);
+  RetJob j = {s / p.Hkv, s % p.Hkv, 0, 0};
+  if (!d.keep_all && d.k_sel > 0) {
+    d.job = s;  // job slot = segment index
+    j.chunk0 = seg_off[s] / p.cs + p.sink2 / p.cs;
+    j.n_pool = d.n_pool;
+  }
+  segs[s] = d;
+  jobs[s] = j;
 }
 
 struct RetWs {
-  size_t off_segs, off_jobs, off_srcoff, off_P, off_idx, bytes;
+  size_t off_segs, off_jobs, off_mask, off_P, off_idx, bytes;
   int64_t p_stride, idx_stride;
 };
 static RetWs ret_ws_layout(int n_segs, int max_len) {
@@ -136,7 +232,7 @@ static RetWs ret_ws_layout(int n_segs, int max_len) {
   size_t o = 0;
   w.off_segs = o; o = align_up(o + sizeof(SelSeg) * (size_t)n_segs, 256);
   w.off_jobs = o; o = align_up(o + sizeof(RetJob) * (size_t)n_segs, 256);
-  w.off_srcoff = o; o = align_up(o + sizeof(int32_t) * (size_t)n_segs, 256);
+  w.off_mask = o; o = align_up(o + (size_t)n_segs, 256);
   w.off_P = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.p_stride, 256);
   w.off_idx = o; o = align_up(o + sizeof(int32_t) * (size_t)n_segs * w.idx_stride, 256);
   w.bytes = o;
@@ -221,59 +317,44 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
   const RetWs W = ret_ws_layout(n_segs, max_len);
   if (ws_bytes < W.bytes) return CATEKV_ERR_WORKSPACE;
 
-  const int S2 = (sink + cs - 1) / cs * cs;  // sink rows rounded up to whole chunks
-  std::vector<SelSeg> segs(n_segs);
-  std::vector<RetJob> jobs;
-  std::vector<int32_t> new_len(n_segs);
+  RetParams rp;
+  rp.cs = cs;
+  rp.budget = budget;
+  rp.sink2 = (sink + cs - 1) / cs * cs;  // sink rows rounded up to whole chunks
+  rp.local = local;
+  rp.Hkv = cache->Hkv;
+  const int S2 = rp.sink2;
   int max_out = 0, max_pool = 0;
+  bool any_job = false;
   for (int s = 0; s < n_segs; ++s) {
-    const int n = cache->seg_len[s];
-    SelSeg d = {};
-    d.n = n;
-    d.job = -1;
-    d.keep_all = 1;
-    d.len_ub = n;
-    if (retrieval_mask[s] && budget < n) {
-      const int cand_end = (n - local > 0 ? n - local : 0) / cs * cs;  // first row of the always-taken tail
-      if (cand_end > S2) {
-        const int forced = S2 + (n - cand_end);
-        const int n_pool = (cand_end - S2) / cs;
-        const int k_sel = budget - forced > 0 ? (budget - forced) / cs : 0;
-        if (k_sel < n_pool) {
-          d.keep_all = 0;
-          d.cand_end = cand_end;
-          d.n_pool = n_pool;
-          d.k_sel = k_sel;
-          d.len_ub = forced + k_sel * cs;
-          if (k_sel > 0) {
-            d.job = (int)jobs.size();
-            jobs.push_back(RetJob{s / cache->Hkv, s % cache->Hkv, cache->seg_off[s] / cs + S2 / cs, n_pool});
-            max_pool = n_pool > max_pool ? n_pool : max_pool;
-          }
-        }
-      }
-    }
+    const SelSeg d = retrieval_decide(cache->seg_len[s], retrieval_mask[s] != 0, rp);
     if (d.len_ub > step_cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
     max_out = d.len_ub > max_out ? d.len_ub : max_out;
-    new_len[s] = d.len_ub;
-    segs[s] = d;
+    if (!d.keep_all && d.k_sel > 0) {
+      any_job = true;
+      max_pool = d.n_pool > max_pool ? d.n_pool : max_pool;
+    }
   }
 
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* w8 = (uint8_t*)ws;
   SelSeg* d_segs = (SelSeg*)(w8 + W.off_segs);
   RetJob* d_jobs = (RetJob*)(w8 + W.off_jobs);
+  uint8_t* d_mask = w8 + W.off_mask;
   float* P = (float*)(w8 + W.off_P);
-  CATEKV_CUDA_TRY(cudaMemcpyAsync(d_segs, segs.data(), sizeof(SelSeg) * n_segs, cudaMemcpyHostToDevice, st));
-  if (!jobs.empty()) {
-    CATEKV_CUDA_TRY(cudaMemcpyAsync(d_jobs, jobs.data(), sizeof(RetJob) * jobs.size(), cudaMemcpyHostToDevice, st));
-    int gx = (max_pool + 7) / 8;
-    if (gx > 512) gx = 512;  // warps stride over the chunks
-    retrieval_score_kernel<<<dim3(gx, (unsigned)jobs.size()), 256, 0, st>>>(d_jobs, (const uint8_t*)meta, (const uint16_t*)q, Hq, G,
-                                                                            P, W.p_stride);
-    CATEKV_CUDA_TRY(cudaGetLastError());
-    const int64_t np = (int64_t)jobs.size() * W.p_stride;
-    monotone_key_kernel<<<(unsigned)((np + 255) / 256), 256, 0, st>>>(P, np);
+  // the mask is the only table that comes from the host (n_segs bytes)
+  CATEKV_CUDA_TRY(cudaMemcpyAsync(d_mask, retrieval_mask, (size_t)n_segs, cudaMemcpyHostToDevice, st));
+  retrieval_plan_kernel<<<(n_segs + 127) / 128, 128, 0, st>>>(cache->seg_len_dev, cache->seg_off_dev, d_mask, rp, d_segs, d_jobs,
+                                                              n_segs);
+  CATEKV_CUDA_TRY(cudaGetLastError());
+  if (any_job) {
+    // a few 64-chunk tiles per CTA, enough CTAs to fill the machine
+    int gx = (max_pool + 8 * kRsTile - 1) / (8 * kRsTile);
+    if (gx > 64) gx = 64;
+    if (gx < 1) gx = 1;
+    CATEKV_CUDA_TRY(cudaFuncSetAttribute(retrieval_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRsSmem));
+    retrieval_score_kernel<<<dim3(gx, (unsigned)n_segs), kRsThreads, kRsSmem, st>>>(d_jobs, (const uint8_t*)meta, (const uint16_t*)q,
+                                                                                     Hq, G, P, W.p_stride);
     CATEKV_CUDA_TRY(cudaGetLastError());
   }
   TopkArgs ta;
@@ -311,6 +392,6 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
   ga.Hkv = cache->Hkv;
   rc = launch_gather(ga, max_out, n_segs, st);
   if (rc) return rc;
-  for (int s = 0; s < n_segs; ++s) step_cache->seg_len[s] = new_len[s];
+  for (int s = 0; s < n_segs; ++s) step_cache->seg_len[s] = retrieval_decide(cache->seg_len[s], retrieval_mask[s] != 0, rp).len_ub;
   return CATEKV_OK;
 }
