@@ -332,6 +332,54 @@ def time_head_cv(ck, dev):
     return e0.elapsed_time(e1) / 3
 
 
+def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8):
+    """Decode step with query-aware retrieval on the adaptive heads (budget rows per adaptive head, chunk size 8):
+    per layer catekv_append + catekv_retrieval_append + catekv_retrieve_compact + catekv_decode_attn over the
+    per-step cache.  Host launches.  Returns (us per layer-step, attended bytes per layer-step)."""
+    import torch
+    from workloads import synth
+    model, _ = build_model(ck, w, dev, max_new=steps + 8, layers=n_layers)
+    num_ctas = ck.catekv_decode_num_ctas()
+    q = synth.randn_bf16((n_layers, w.B, w.Hq, w.d), dev, w.seed, "ret_q")
+    kn = synth.randn_bf16((n_layers, w.B, w.Hkv, w.d), dev, w.seed, "ret_kn")
+    vn = synth.randn_bf16((n_layers, w.B, w.Hkv, w.d), dev, w.seed, "ret_vn")
+    out = torch.empty((w.B, w.Hq, w.d), dtype=torch.bfloat16, device=dev)
+    for l, m in enumerate(model):
+        c = m["cache"]
+        m["meta"] = ck.catekv_retrieval_meta(c, cs)
+        ck.catekv_retrieval_build(c, cs, m["meta"])
+        m["rmask"] = (m["mask"].reshape(-1) == 0).astype(np.uint8)
+        slens = [min(int(L), budget + 2 * cs + w.local) if m["rmask"][i] else int(L) + steps + 8
+                 for i, L in enumerate(c.seg_len)]
+        m["step"] = ck.Cache(w.B, w.Hkv, slens, 0, dev)
+        m["ws"] = torch.empty(ck._lib.catekv_retrieve_workspace_bytes(w.B, w.Hkv, int(c.seg_len.max()) + steps + 8),
+                              dtype=torch.uint8, device=dev)
+        ck.catekv_retrieve_compact(c, m["meta"], cs, q[l], m["rmask"], budget, w.sink, w.local, m["step"], ws=m["ws"])
+        m["splan"] = ck.DecodePlan(m["step"], num_ctas)
+        ck.catekv_decode_plan(m["step"], m["splan"])
+
+    def step():
+        for l, m in enumerate(model):
+            ck.catekv_append(m["cache"], kn[l], vn[l])
+            ck.catekv_retrieval_append(m["cache"], cs, kn[l], m["meta"])
+            ck.catekv_retrieve_compact(m["cache"], m["meta"], cs, q[l], m["rmask"], budget, w.sink, w.local, m["step"],
+                                       ws=m["ws"])
+            ck.catekv_decode_attn(m["step"], q[l], m["splan"], out)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    attended = float(np.mean([int(m["step"].seg_len.sum()) * ROW_BYTES for m in model]))
+    meta_bytes = float(np.mean([int(m["cache"].seg_len[m["rmask"] == 1].sum()) // cs * 512 for m in model]))
+    return e0.elapsed_time(e1) * 1e3 / (steps * n_layers), attended, meta_bytes
+
+
 # ------------------------------------------------------------------------------------------
 # the oracle, timed as it stands, on a bounded sample
 # ------------------------------------------------------------------------------------------
@@ -535,6 +583,10 @@ def main():
             torch.cuda.empty_cache()
         line["other_configs"] = table
         line["head_cv"] = {"ms": time_head_cv(ck, dev), "shape": "8 prompts x 16384 tokens, 28q/4kv, window 64"}
+        ru, ra, rm = time_retrieval(ck, w, dev)
+        line["retrieval"] = {"us_per_layer_step": ru, "attended_bytes_per_layer_step": ra,
+                             "metadata_bytes_per_layer_step": rm, "budget_rows": 1024, "chunk": 8,
+                             "note": "query-aware retrieval on the adaptive heads of the same workload (host launches)"}
         rate, desc, spent = oracle_sample_rate(w, target_s=15.0)
         rows = bytes_per_layer / ROW_BYTES
         line["cpu_baseline"] = {"value": w.B / (w.layers * rows / rate), "unit": UNIT, "cores": oracle_threads(),

@@ -166,3 +166,51 @@ def test_cfg4_head_mask_from_calibration_prompts(ck):
     m = ck.catekv_classify_heads(got, 0.5)
     assert np.array_equal(m, orc.static_head_mask(want, 0.5))
     assert np.array_equal(m, types.reshape(-1))
+
+
+def test_cfg2_retrieval_on_adaptive_heads(ck):
+    # configs[2] shape: adaptive heads (117 964 rows) answer a decode query from 2048 retrieved rows, chunk size 8
+    w = synth.WORKLOADS["cfg2"]
+    p, mask, cache, idx = _build_layer(ck, w, 3, 8)
+    cs, budget = 8, 2048
+    meta = ck.catekv_retrieval_meta(cache, cs)
+    ck.catekv_retrieval_build(cache, cs, meta)
+    q, kn, vn = synth.decode_inputs(w, 3, 0, "cuda", mask)
+    ck.catekv_append(cache, kn, vn)
+    ck.catekv_retrieval_append(cache, cs, kn, meta)
+    rmask = (mask.reshape(-1) == 0).astype(np.uint8)
+    lens = [int(L) for L in cache.seg_len]
+    slens = [len(orc.retrieve_indices(np.zeros((L + cs - 1) // cs), L, w.sink, w.local, budget, cs)) if rmask[i] else L
+             for i, L in enumerate(lens)]
+    step = ck.Cache(w.B, w.Hkv, slens, 0, "cuda")
+    ridx = torch.full((w.B * w.Hkv, max(lens)), -1, dtype=torch.int32, device="cuda")
+    ck.catekv_retrieve_compact(cache, meta, cs, q, rmask, budget, w.sink, w.local, step, idx_out=ridx)
+    torch.cuda.synchronize()
+    assert list(step.seg_len) == slens
+    cells = [int(i) for i in np.nonzero(rmask)[0][:2]] + [int(np.nonzero(rmask == 0)[0][0])]
+    qb = orc.bf16_to_f64(synth.bits(q))
+    soc = orc.HybridCache(w.B, w.Hkv, w.d)
+    soc.k_rows = [np.zeros((0, w.d), dtype=np.uint16)] * (w.B * w.Hkv)
+    soc.v_rows = [np.zeros((0, w.d), dtype=np.uint16)] * (w.B * w.Hkv)
+    for s in cells:
+        o, L = int(cache.seg_off[s]), lens[s]
+        krows, vrows = synth.bits(cache.k_pool[o:o + L]), synth.bits(cache.v_pool[o:o + L])
+        got = ridx[s, :slens[s]].cpu().numpy().astype(np.int64)
+        if rmask[s]:
+            kmax, kmin = orc.retrieval_metadata(krows, cs)
+            scores = orc.retrieval_scores(qb[0, s * w.G:(s + 1) * w.G], kmax, kmin)
+            want = orc.retrieve_indices(scores, L, w.sink, w.local, budget, cs)
+            assert got.shape == want.shape and np.all(np.diff(got) > 0)
+            # fp32 bounds against fp64 bounds: the sets may differ only among near-ties
+            assert len(np.setdiff1d(got, want)) <= 0.02 * len(want)
+        else:
+            assert np.array_equal(got, np.arange(L))
+        so = int(step.seg_off[s])
+        assert np.array_equal(synth.bits(step.k_pool[so:so + slens[s]]), krows[got])
+        soc.k_rows[s], soc.v_rows[s] = krows[got], vrows[got]
+    plan = ck.DecodePlan(step, ck.catekv_decode_num_ctas())
+    ck.catekv_decode_plan(step, plan)
+    out = torch.empty((w.B, w.Hq, w.d), dtype=torch.float32, device="cuda")
+    ck.catekv_decode_attn(step, q, plan, out)
+    ref, _ = orc.decode_attention(soc, synth.bits(q), cells=[(0, s) for s in cells])
+    H.check_attention(out, None, None, ref, None, "cfg2 retrieval")
