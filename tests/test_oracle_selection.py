@@ -215,7 +215,8 @@ def test_attention_recall_pins(golden_dir):
     l = [0.0, math.log(2), math.log(4), math.log(2), 0.0, 0.0]
     K = np.array([[x, 0.0] for x in l])
     q = np.array([1.0, 0.0])
-    assert orc.attention_recall(q, K, [0, 1, 2, 5], 1.0) == pytest.approx(8 / 11, rel=1e-14)
+    g = _golden(golden_dir, "hand_examples.txt")
+    assert orc.attention_recall(q, K, [0, 1, 2, 5], 1.0) == pytest.approx(float(Fraction(g["recall_kept"][0])), rel=1e-14)
     assert orc.attention_recall(q, K, list(range(6)), 1.0) == pytest.approx(1.0, rel=1e-14)
     # identical keys: recall = |kept| / n
     K2 = np.tile(np.array([[0.3, -0.7]]), (10, 1))
