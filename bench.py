@@ -39,6 +39,17 @@ UNIT = "tokens/s"
 ROW_BYTES = 512  # one kept token of one KV head: 256 B of K + 256 B of V
 
 
+def max_over_ranks(x: float, device=None) -> float:
+    """Maximum of a per-rank time over all ranks of the default process group (identity without one)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return x
+    t = torch.tensor([x], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -495,13 +506,6 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(dev))
         barrier = lambda: dist.barrier()
 
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
     peaks, peak_src = measured_peaks()
     w = synth.WORKLOADS[args.workload]
     n_layers = args.layers or w.layers
@@ -518,12 +522,12 @@ def main():
     vis = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
     sampler = ClockSampler(vis[local_rank] if local_rank < len(vis) else local_rank)
     sampler.start()
-    ms = max_over_ranks(time_decode(ck, w, model, dev, args.steps, args.warmup, barrier, graph))
+    ms = max_over_ranks(time_decode(ck, w, model, dev, args.steps, args.warmup, barrier, graph), dev)
     clocks = sampler.stop()
     bytes_per_layer = float(np.mean(kept_bytes(model)))
     part_us, part_med_us, comb_us = time_kernels(ck, w, model, dev, max(2, min(args.steps, 5)))
     ms_e2e, h2d, d2h = time_e2e(ck, w, model, dev, args.steps, args.warmup, barrier, graph)
-    ms_e2e = max_over_ranks(ms_e2e)
+    ms_e2e = max_over_ranks(ms_e2e, dev)
 
     scale_layers = w.layers / n_layers  # only != 1 when --layers is used for profiling
     value = world * w.B / (ms * scale_layers * 1e-3)

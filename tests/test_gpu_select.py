@@ -84,7 +84,7 @@ def test_select_cfg0_all_modes(ck, mode, param):
     _check_against_oracle(ck, w, p, p["head_mask"], w.budget, 1.0, mode, param)
 
 
-@pytest.mark.parametrize("Hq,Hkv,L_obs", [(8, 8, 16), (28, 4, 64), (16, 2, 48), (6, 2, 7)])
+@pytest.mark.parametrize("Hq,Hkv,L_obs", [(8, 8, 16), (28, 4, 64), (16, 2, 48), (6, 2, 7), (16, 2, 64), (10, 2, 50)])
 def test_select_shapes_and_adaptive_eta(ck, Hq, Hkv, L_obs):
     w = synth.scaled(synth.WORKLOADS["cfg0"], Hq=Hq, Hkv=Hkv, L_obs=L_obs, n=1500, B=2)
     p = synth.prefill_layer(w, 1)
