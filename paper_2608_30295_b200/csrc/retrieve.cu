@@ -369,7 +369,7 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
   ta.L_obs = 0;
   ta.pool_mode = kPoolPrescored;
   ta.pool_param = cs;
-  rc = launch_topk(ta, n_segs, st);
+  rc = launch_topk(ta, n_segs, max_pool, st);
   if (rc) return rc;
   rc = launch_set_full_len(d_segs, step_cache->seg_len_dev, n_segs, st);
   if (rc) return rc;

@@ -5,9 +5,13 @@
 
 #include <vector>
 
+#include <cooperative_groups.h>
+
 #include "radix.cuh"
 #include "score.cuh"
 #include "select.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace catekv {
 
@@ -42,15 +46,25 @@ __device__ __forceinline__ unsigned long long block_excl_scan(unsigned long long
   return res;
 }
 
-// One CTA per segment that selects: pooling, radix select of the k-th largest pooled score,
-// ordered compaction into the ascending kept list.
+// One thread-block cluster of CL CTAs (1 or 8) per segment that selects: pooling, radix select of the k-th largest
+// pooled score, ordered compaction into the ascending kept list.  Every CTA owns a contiguous share of the pooled
+// entries.  The CTAs meet only through distributed shared memory: the per-pass digit histograms and the per-CTA
+// (greater, equal) totals are read from the peers' shared memory, every CTA derives the same decisions from them.
+template <int CL>
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
-  const int seg = blockIdx.x;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int seg = blockIdx.x / CL;
+  const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
   const SelSeg s = a.segs[seg];
-  if (s.keep_all) return;
+  if (s.keep_all) return;  // the whole cluster leaves
   __shared__ unsigned int hist[256];
+  __shared__ unsigned int hsum[256];
   __shared__ unsigned long long s_warp[33];
   __shared__ unsigned int s_pair[2];
+  __shared__ unsigned long long s_tot;  // this CTA's (greater, equal) totals, read by its peers
+  auto cluster_sync = [&]() {
+    if (CL > 1) cluster.sync(); else __syncthreads();
+  };
   const int tid = threadIdx.x;
   int32_t* idx = a.idx + (size_t)seg * a.idx_stride;
   const int S = a.sink;
@@ -60,78 +74,145 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     const float* C = a.C + (size_t)s.job * a.c_stride;
     float* P = a.P + (size_t)s.job * a.c_stride;
     const int n_sc = s.n - a.L_obs;
+    // this CTA's share of the pooled entries (a multiple of 4 entries, so that 4-entry steps stay aligned)
+    const int per = ((s.n_pool + CL - 1) / CL + 3) / 4 * 4;
+    const int lo = min(s.n_pool, rank * per), hi = min(s.n_pool, lo + per);
     // ---- pooling (four entries per thread and step, so that several loads are in flight)
     const float* __restrict__ Cr = C;
     float* __restrict__ Pw = P;
     if (a.pool_mode == kPoolPrescored) {
       // P was filled by the caller's scoring kernel
     } else if (a.pool_mode == CATEKV_POOL_NONE) {
-      for (int c0 = tid; c0 < s.n_pool; c0 += 4 * kTopkThreads) {
+      for (int c0 = lo + tid; c0 < hi; c0 += 4 * kTopkThreads) {
         float vv[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) vv[e] = (c0 + e * kTopkThreads < s.n_pool) ? Cr[S + c0 + e * kTopkThreads] : 0.f;
+        for (int e = 0; e < 4; ++e) vv[e] = (c0 + e * kTopkThreads < hi) ? Cr[S + c0 + e * kTopkThreads] : 0.f;
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-          if (c0 + e * kTopkThreads < s.n_pool) Pw[c0 + e * kTopkThreads] = vv[e];
+          if (c0 + e * kTopkThreads < hi) Pw[c0 + e * kTopkThreads] = vv[e];
       }
     } else if (a.pool_mode == CATEKV_POOL_SLIDING) {
       const int half = (a.pool_param - 1) / 2;
-      for (int c0 = tid; c0 < s.n_pool; c0 += 4 * kTopkThreads) {
+      for (int c0 = lo + tid; c0 < hi; c0 += 4 * kTopkThreads) {
         float mm[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int c = c0 + e * kTopkThreads;
           mm[e] = 0.f;
-          if (c < s.n_pool) {
+          if (c < hi) {
             const int j = S + c;
-            const int lo = max(0, j - half), hi = min(n_sc - 1, j + half);
-            float m = Cr[lo];
-            for (int u = lo + 1; u <= hi; ++u) m = fmaxf(m, Cr[u]);
+            const int l2 = max(0, j - half), h2 = min(n_sc - 1, j + half);
+            float m = Cr[l2];
+            for (int u = l2 + 1; u <= h2; ++u) m = fmaxf(m, Cr[u]);
             mm[e] = m;
           }
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-          if (c0 + e * kTopkThreads < s.n_pool) Pw[c0 + e * kTopkThreads] = mm[e];
+          if (c0 + e * kTopkThreads < hi) Pw[c0 + e * kTopkThreads] = mm[e];
       }
     } else {
       const int cs = a.pool_param;
-      for (int c0 = tid; c0 < s.n_pool; c0 += 4 * kTopkThreads) {
+      for (int c0 = lo + tid; c0 < hi; c0 += 4 * kTopkThreads) {
         float mm[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int c = c0 + e * kTopkThreads;
           mm[e] = 0.f;
-          if (c < s.n_pool) {
-            const int lo = S + c * cs, hi = min(lo + cs, s.cand_end);
-            float m = Cr[lo];
-            for (int u = lo + 1; u < hi; ++u) m = fmaxf(m, Cr[u]);
+          if (c < hi) {
+            const int l2 = S + c * cs, h2 = min(l2 + cs, s.cand_end);
+            float m = Cr[l2];
+            for (int u = l2 + 1; u < h2; ++u) m = fmaxf(m, Cr[u]);
             mm[e] = m;
           }
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-          if (c0 + e * kTopkThreads < s.n_pool) Pw[c0 + e * kTopkThreads] = mm[e];
+          if (c0 + e * kTopkThreads < hi) Pw[c0 + e * kTopkThreads] = mm[e];
       }
     }
-    __syncthreads();
-    // ---- radix select of the k_sel-th largest pooled score
+    __syncthreads();  // a CTA reads back only its own share of P
+    // ---- radix select of the k_sel-th largest pooled score: 8 bits per pass from the top (scores are >= 0, so
+    // their bit patterns order as integers); the histograms of the CTAs are summed through distributed shared memory
     const unsigned int* Pb = reinterpret_cast<const unsigned int*>(P);
-    unsigned int thr, need_eq;  // threshold bits; entries equal to it that are taken (lowest index first)
-    block_radix_select([&](int c) { return Pb[c]; }, s.n_pool, (unsigned int)s.k_sel, hist, s_pair, thr, need_eq);
+    unsigned int prefix = 0, need = (unsigned int)s.k_sel;
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      const unsigned int pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+      if (tid < 256) hist[tid] = 0;
+      __syncthreads();
+      for (int c0 = lo; c0 < hi; c0 += 4 * kTopkThreads) {  // whole warps stay in the loop: the vote needs them
+        unsigned int v[4];
+        bool in[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int c = c0 + e * kTopkThreads + tid;
+          in[e] = c < hi;
+          v[e] = in[e] ? Pb[c] : 0u;
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const bool hit = in[e] && (v[e] & pmask) == prefix;
+          // lanes with the same digit elect one of them to add their count (scores cluster in a few bins)
+          const unsigned int dgt = hit ? ((v[e] >> shift) & 0xffu) : 0x100u;
+          const unsigned int peers = __match_any_sync(0xffffffffu, dgt);
+          if (hit && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[dgt], (unsigned int)__popc(peers));
+        }
+      }
+      cluster_sync();  // all histograms complete
+      if (tid < 256) {
+        unsigned int t = 0;
+#pragma unroll
+        for (int r = 0; r < CL; ++r) t += CL > 1 ? *cluster.map_shared_rank(&hist[tid], r) : hist[tid];
+        hsum[tid] = t;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        unsigned int cum = 0;
+        int dsel = 0;
+        for (int dgt = 255; dgt >= 0; --dgt) {
+          if (cum + hsum[dgt] >= need) { dsel = dgt; break; }
+          cum += hsum[dgt];
+        }
+        s_pair[0] = prefix | ((unsigned int)dsel << shift);
+        s_pair[1] = need - cum;
+      }
+      cluster_sync();  // decision visible; the peers are done reading this CTA's histogram
+      prefix = s_pair[0];
+      need = s_pair[1];
+    }
+    const unsigned int thr = prefix, need_eq = need;  // threshold bits; ties taken (lowest index first)
+    // ---- (greater, equal) counts of every CTA's share -> where this CTA's selected entries start
+    unsigned long long mine_tot = 0;
+    for (int c = lo + tid; c < hi; c += kTopkThreads) {
+      const unsigned int v = Pb[c];
+      mine_tot += (unsigned long long)(v > thr) | ((unsigned long long)(v == thr) << 32);
+    }
+    {
+      unsigned long long tot;
+      block_excl_scan(mine_tot, s_warp, tot);
+      if (tid == 0) s_tot = tot;
+    }
+    cluster_sync();
+    unsigned long long run = 0, all = 0;  // packed: low = entries above the threshold, high = entries equal to it
+#pragma unroll
+    for (int r = 0; r < CL; ++r) {
+      const unsigned long long t = CL > 1 ? *cluster.map_shared_rank(&s_tot, r) : s_tot;
+      if (r < rank) run += t;
+      all += t;
+    }
     // ---- ordered compaction, four consecutive entries per thread and step
-    unsigned long long run = 0;  // packed: low = entries above the threshold so far, high = entries equal to it
     const int cs = (a.pool_mode == CATEKV_POOL_CHUNK || a.pool_mode == kPoolPrescored) ? a.pool_param : 1;
-    for (int base = 0; base < s.n_pool; base += 4 * kTopkThreads) {
+    for (int base = lo; base < hi; base += 4 * kTopkThreads) {
       const int c4 = base + tid * 4;
       unsigned int v[4];
       bool gt[4], eq[4];
       unsigned long long mine = 0;
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        v[e] = (c4 + e < s.n_pool) ? Pb[c4 + e] : 0u;
-        gt[e] = (c4 + e < s.n_pool) && v[e] > thr;
-        eq[e] = (c4 + e < s.n_pool) && v[e] == thr;
+        v[e] = (c4 + e < hi) ? Pb[c4 + e] : 0u;
+        gt[e] = (c4 + e < hi) && v[e] > thr;
+        eq[e] = (c4 + e < hi) && v[e] == thr;
         mine += (unsigned long long)gt[e] | ((unsigned long long)eq[e] << 32);
       }
       unsigned long long tot;
@@ -140,13 +221,13 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
       for (int e = 0; e < 4; ++e) {
         const unsigned int gt_before = (unsigned int)(ex & 0xffffffffu), eq_before = (unsigned int)(ex >> 32);
         if (gt[e] || (eq[e] && eq_before < need_eq)) {
-          const unsigned int rank = gt_before + min(eq_before, need_eq);
+          const unsigned int rnk = gt_before + min(eq_before, need_eq);
           const int c = c4 + e;
           if (cs == 1) {
-            idx[S + rank] = S + c;
+            idx[S + rnk] = S + c;
           } else {
-            const int lo = S + c * cs, hi = min(lo + cs, s.cand_end);
-            for (int u = lo; u < hi; ++u) idx[S + rank * cs + (u - lo)] = u;
+            const int l2 = S + c * cs, h2 = min(l2 + cs, s.cand_end);
+            for (int u = l2; u < h2; ++u) idx[S + rnk * cs + (u - l2)] = u;
           }
         }
         ex += (unsigned long long)gt[e] | ((unsigned long long)eq[e] << 32);
@@ -158,17 +239,20 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     if (cs > 1) {
       const int last = s.n_pool - 1;
       const int last_sz = s.cand_end - (S + last * cs);
-      const unsigned int vl = Pb[last];
+      const unsigned int vl = Pb[last];  // written by the last CTA before the cluster barriers above
       // the last chunk is taken iff it is above the threshold, or ties with it and is within the quota of ties
-      const unsigned int eq_total = (unsigned int)(run >> 32);
+      const unsigned int eq_total = (unsigned int)(all >> 32);
       const bool last_taken = vl > thr || (vl == thr && eq_total <= need_eq);
       if (last_taken) n_sel_tokens -= cs - last_sz;
     }
+    cluster_sync();  // no CTA leaves while a peer may still read its shared memory
   }
-  for (int i = tid; i < S; i += kTopkThreads) idx[i] = i;
-  const int n_tail = s.n - s.cand_end;  // the always-kept most recent tokens
-  for (int i = tid; i < n_tail; i += kTopkThreads) idx[S + n_sel_tokens + i] = s.cand_end + i;
-  if (tid == 0) a.seg_len_dev[seg] = S + n_sel_tokens + n_tail;
+  if (rank == 0) {
+    for (int i = tid; i < S; i += kTopkThreads) idx[i] = i;
+    const int n_tail = s.n - s.cand_end;  // the always-kept most recent tokens
+    for (int i = tid; i < n_tail; i += kTopkThreads) idx[S + n_sel_tokens + i] = s.cand_end + i;
+    if (tid == 0) a.seg_len_dev[seg] = S + n_sel_tokens + n_tail;
+  }
 }
 
 // keep_all segments: seg_len = n
@@ -202,9 +286,25 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
   }
 }
 
-int launch_topk(const TopkArgs& a, int n_segs, cudaStream_t stream) {
-  topk_kernel<<<n_segs, kTopkThreads, 0, stream>>>(a);
-  CATEKV_CUDA_TRY(cudaGetLastError());
+int launch_topk(const TopkArgs& a, int n_segs, int max_pool, cudaStream_t stream) {
+  if (max_pool < 16384) {  // short lists: one CTA per segment
+    topk_kernel<1><<<n_segs, kTopkThreads, 0, stream>>>(a);
+    CATEKV_CUDA_TRY(cudaGetLastError());
+    return CATEKV_OK;
+  }
+  // long lists: a cluster of 8 CTAs per segment
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_segs * 8);
+  cfg.blockDim = dim3(kTopkThreads);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 8;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  CATEKV_CUDA_TRY(cudaLaunchKernelEx(&cfg, topk_kernel<8>, a));
   return CATEKV_OK;
 }
 int launch_set_full_len(const SelSeg* segs, int32_t* seg_len_dev, int n_segs, cudaStream_t stream) {
@@ -390,8 +490,12 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   ta.L_obs = p->L_obs;
   ta.pool_mode = p->pool_mode;
   ta.pool_param = p->pool_param;
-  topk_kernel<<<n_segs, kTopkThreads, 0, st>>>(ta);
-  CATEKV_CUDA_TRY(cudaGetLastError());
+  {
+    int max_pool = 0;
+    for (const SelSeg& sg : segs) max_pool = sg.n_pool > max_pool ? sg.n_pool : max_pool;
+    int rc2 = launch_topk(ta, n_segs, max_pool, st);
+    if (rc2) return rc2;
+  }
   set_full_len_kernel<<<(n_segs + 255) / 256, 256, 0, st>>>(d_segs, cache->seg_len_dev, n_segs);
   CATEKV_CUDA_TRY(cudaGetLastError());
 

@@ -48,7 +48,7 @@ struct GatherArgs {
 };
 
 
-int launch_topk(const TopkArgs& a, int n_segs, cudaStream_t stream);
+int launch_topk(const TopkArgs& a, int n_segs, int max_pool, cudaStream_t stream);  // max_pool: longest pooled list
 int launch_set_full_len(const SelSeg* segs, int32_t* seg_len_dev, int n_segs, cudaStream_t stream);
 int launch_gather(const GatherArgs& a, int max_len, int n_segs, cudaStream_t stream);
 
