@@ -85,7 +85,7 @@ static CvWs cv_ws_layout(int n_segs, int G, int m_max, int L_obs) {
   w.off_status = o; o = 256;
   w.off_segs = o; o = align_up(o + sizeof(CvSeg) * (size_t)n_segs, 256);
   w.off_jobs = o; o = align_up(o + sizeof(ScoreJob) * (size_t)n_segs, 256);
-  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 4 ? n_segs : 148 * 4) * 2 * kScoreMaxRows, 256);
+  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs + 148 * 4) * 2 * kScoreMaxRows, 256);
   w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * kScoreMaxRows, 256);
   w.off_A = o; o = align_up(o + sizeof(float) * (size_t)n_segs * L_obs * w.row_stride, 256);
   w.bytes = o;
@@ -161,8 +161,8 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   sa.L_obs = L_obs;
   sa.causal = causal ? 1 : 0;
   sa.scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
-  sa.keys_per_cta = W.keys_per_cta;
-  sa.n_chunks = W.n_chunks;
+  sa.keys_per_cta = score_keys_per_cta(n_segs, m_max);
+  sa.n_chunks = (m_max + sa.keys_per_cta - 1) / sa.keys_per_cta;
   sa.stats_part = (float2*)(w8 + W.off_part);
   sa.stats = (float2*)(w8 + W.off_stats);
   sa.status = (int32_t*)(w8 + W.off_status);

@@ -466,6 +466,15 @@ static int launch_one(const ScoreArgs& a, const ScoreShape& sh, const CUtensorMa
   return CATEKV_OK;
 }
 
+int score_keys_per_cta(int n_jobs, int max_keys) {
+  if (n_jobs < 1) n_jobs = 1;
+  int chunks = (296 + n_jobs / 2) / n_jobs;  // about 296 CTAs in all
+  if (chunks < 1) chunks = 1;
+  int kp = ((max_keys + chunks - 1) / chunks + kKeyTile - 1) / kKeyTile * kKeyTile;
+  if (kp < 4 * kKeyTile) kp = 4 * kKeyTile;  // at least a few tiles per CTA: the queries are staged once per CTA
+  return kp;
+}
+
 int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream) {
   if (a.n_jobs <= 0 || a.n_chunks <= 0) return CATEKV_OK;
   if (a.G * a.L_obs > kScoreMaxRows || a.keys_per_cta % kKeyTile || !a.status) return CATEKV_ERR_UNSUPPORTED;

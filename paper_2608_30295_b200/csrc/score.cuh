@@ -32,6 +32,9 @@ struct ScoreArgs {
 enum ScoreMode { kScoreStats = 0, kScoreColsum = 1, kScoreMatrix = 2 };
 
 constexpr int kScoreMaxRows = 512;  // G * L_obs may not exceed this (8 heads x 64 window rows)
+// Keys per CTA for n_jobs jobs of at most max_keys keys: a multiple of 128 chosen so that the grid is close to two
+// CTAs per SM in whole waves (never more than 592 CTAs unless there are more jobs than that).
+int score_keys_per_cta(int n_jobs, int max_keys);
 // Enqueue: pass 1 (row max / sum partials), their merge, and pass 2 (column sums or matrix).
 int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream);
 

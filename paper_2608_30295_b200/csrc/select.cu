@@ -342,7 +342,7 @@ static SelWs sel_ws_layout(int n_segs, int G, int n_max, int L_obs) {
   w.off_status = o; o = 256;
   w.off_segs = o; o = align_up(o + sizeof(SelSeg) * (size_t)n_segs, 256);
   w.off_jobs = o; o = align_up(o + sizeof(ScoreJob) * (size_t)n_segs, 256);
-  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs > 148 * 4 ? n_segs : 148 * 4) * 2 * kScoreMaxRows, 256);
+  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs + 148 * 4) * 2 * kScoreMaxRows, 256);
   w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * kScoreMaxRows, 256);
   w.off_C = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.c_stride, 256);
   w.off_P = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.c_stride, 256);
@@ -468,8 +468,8 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
     sa.L_obs = p->L_obs;
     sa.causal = 0;  // every scored key precedes every window query
     sa.scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
-    sa.keys_per_cta = W.keys_per_cta;
-    sa.n_chunks = (n_sc_jobs_max + W.keys_per_cta - 1) / W.keys_per_cta;
+    sa.keys_per_cta = score_keys_per_cta((int)jobs.size(), n_sc_jobs_max);
+    sa.n_chunks = (n_sc_jobs_max + sa.keys_per_cta - 1) / sa.keys_per_cta;  // jobs * chunks <= 592 + jobs: fits the partials
     sa.stats_part = (float2*)(w8 + W.off_part);
     sa.stats = (float2*)(w8 + W.off_stats);
     sa.status = (int32_t*)(w8 + W.off_status);
