@@ -479,6 +479,8 @@ def main():
     ap.add_argument("--no-fused", action="store_true", help="catekv_append + catekv_decode_attn as two calls per layer")
     ap.add_argument("--select-only", action="store_true", help="run only the prefill-end path (catekv_select_compact) "
                     "for --layers layers and print its time; used for profiling that path on a small case")
+    ap.add_argument("--retrieval-only", action="store_true", help="run only the query-aware retrieval decode step "
+                    "(small case for profiling; use with --workload and --layers)")
     ap.add_argument("--no-extras", action="store_true", help="skip the other configs, head_cv and the oracle timing")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -513,6 +515,12 @@ def main():
     graph = not args.no_graph
     global FUSED
     FUSED = not args.no_fused
+    if args.retrieval_only:
+        ru, ra, rm = time_retrieval(ck, w, dev, n_layers=n_layers, steps=args.steps)
+        if rank == 0:
+            print(json.dumps({"workload": w.name, "layers": n_layers, "retrieval_us_per_layer_step": ru,
+                              "attended_bytes_per_layer_step": ra, "metadata_bytes_per_layer_step": rm}))
+        return
     model, sel_ms = build_model(ck, w, dev, max_new=total_steps, layers=n_layers)
     if args.select_only:
         if rank == 0:
