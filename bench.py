@@ -343,13 +343,14 @@ def time_head_cv(ck, dev):
     return e0.elapsed_time(e1) / 3
 
 
-def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8):
+def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8, graph=True):
     """Decode step with query-aware retrieval on the adaptive heads (budget rows per adaptive head, chunk size 8):
     per layer catekv_append + catekv_retrieval_append + catekv_retrieve_compact + catekv_decode_attn over the
-    per-step cache.  Host launches.  Returns (us per layer-step, attended bytes per layer-step)."""
+    per-step cache, replayed as a CUDA graph of the step (graph=False: host launches).
+    Returns (us per layer-step, attended bytes per layer-step, metadata bytes per layer-step)."""
     import torch
     from workloads import synth
-    model, _ = build_model(ck, w, dev, max_new=steps + 8, layers=n_layers)
+    model, _ = build_model(ck, w, dev, max_new=steps + 16, layers=n_layers)
     num_ctas = ck.catekv_decode_num_ctas()
     q = synth.randn_bf16((n_layers, w.B, w.Hq, w.d), dev, w.seed, "ret_q")
     kn = synth.randn_bf16((n_layers, w.B, w.Hkv, w.d), dev, w.seed, "ret_kn")
@@ -360,10 +361,10 @@ def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8):
         m["meta"] = ck.catekv_retrieval_meta(c, cs)
         ck.catekv_retrieval_build(c, cs, m["meta"])
         m["rmask"] = (m["mask"].reshape(-1) == 0).astype(np.uint8)
-        slens = [min(int(L), budget + 2 * cs + w.local) if m["rmask"][i] else int(L) + steps + 8
+        slens = [min(int(L), budget + 2 * cs + w.local) if m["rmask"][i] else int(L) + steps + 16
                  for i, L in enumerate(c.seg_len)]
         m["step"] = ck.Cache(w.B, w.Hkv, slens, 0, dev)
-        m["ws"] = torch.empty(ck._lib.catekv_retrieve_workspace_bytes(w.B, w.Hkv, int(c.seg_len.max()) + steps + 8),
+        m["ws"] = torch.empty(ck._lib.catekv_retrieve_workspace_bytes(w.B, w.Hkv, int(c.seg_cap.max())),
                               dtype=torch.uint8, device=dev)
         ck.catekv_retrieve_compact(c, m["meta"], cs, q[l], m["rmask"], budget, w.sink, w.local, m["step"], ws=m["ws"])
         m["splan"] = ck.DecodePlan(m["step"], num_ctas)
@@ -377,13 +378,28 @@ def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8):
                                        ws=m["ws"])
             ck.catekv_decode_attn(m["step"], q[l], m["splan"], out)
 
+    run = step
+    if graph:
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                step()  # runs the host code (the length mirrors advance), launches nothing
+        torch.cuda.current_stream().wait_stream(side)
+        g.replay()
+
+        def run():
+            for m in model:
+                ck.catekv_cache_advance(m["cache"], 1)
+            g.replay()
     for _ in range(3):
-        step()
+        run()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(steps):
-        step()
+        run()
     e1.record()
     torch.cuda.synchronize()
     attended = float(np.mean([int(m["step"].seg_len.sum()) * ROW_BYTES for m in model]))
@@ -516,7 +532,7 @@ def main():
     global FUSED
     FUSED = not args.no_fused
     if args.retrieval_only:
-        ru, ra, rm = time_retrieval(ck, w, dev, n_layers=n_layers, steps=args.steps)
+        ru, ra, rm = time_retrieval(ck, w, dev, n_layers=n_layers, steps=args.steps, graph=graph)
         if rank == 0:
             print(json.dumps({"workload": w.name, "layers": n_layers, "retrieval_us_per_layer_step": ru,
                               "attended_bytes_per_layer_step": ra, "metadata_bytes_per_layer_step": rm}))
@@ -598,7 +614,7 @@ def main():
         ru, ra, rm = time_retrieval(ck, w, dev)
         line["retrieval"] = {"us_per_layer_step": ru, "attended_bytes_per_layer_step": ra,
                              "metadata_bytes_per_layer_step": rm, "budget_rows": 1024, "chunk": 8,
-                             "note": "query-aware retrieval on the adaptive heads of the same workload (host launches)"}
+                             "note": "query-aware retrieval on the adaptive heads of the same workload (CUDA graph replay of the step)"}
         rate, desc, spent = oracle_sample_rate(w, target_s=15.0)
         rows = bytes_per_layer / ROW_BYTES
         line["cpu_baseline"] = {"value": w.B / (w.layers * rows / rate), "unit": UNIT, "cores": oracle_threads(),

@@ -197,9 +197,12 @@ int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens);
  * every CTA evenly.  The plan is built on the host from cache->seg_len, stored
  * in plan_host and copied to plan_dev (cudaMemcpyAsync on `stream`; plan_host
  * must stay untouched until that copy has run - use pinned memory to make it
- * asynchronous).  A plan stays valid while segments only grow (append): the
- * last item of a segment reads the current length on the device; rebuild it
- * now and then to restore balance.
+ * asynchronous).  A plan stays valid while the segments' lengths change within
+ * their capacities: every item reads the current length on the device, the last
+ * item of a segment follows rows appended since (append), and rows behind a length
+ * that has shrunk (a per-step cache refilled by catekv_retrieve_compact) are left
+ * out; rebuild it now and then to restore balance.  catekv_append_decode_attn
+ * alone needs lengths that are not below the plan's (ERR_INVALID_ARG otherwise).
  *
  * catekv_decode_num_ctas: SM count * resident CTAs per SM of the decode kernel
  * on the current device (a CUDA query); < 0 on error.
@@ -271,8 +274,14 @@ int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, 
  *
  *   q         device bf16 [B, Hq, d], this step's queries
  *   idx_out   device int32 [B*Hkv, idx_stride] or NULL: the rows taken from each segment
- *   ws        device scratch of at least catekv_retrieve_workspace_bytes(B, Hkv, longest segment)
- * Errors: CATEKV_ERR_CAPACITY if a kept list does not fit its segment of step_cache (nothing launched).
+ *   ws        device scratch of at least catekv_retrieve_workspace_bytes(B, Hkv, largest seg_cap of `cache`)
+ * Errors: CATEKV_ERR_CAPACITY if a kept list does not fit its segment of step_cache (nothing launched);
+ * CATEKV_ERR_UNSUPPORTED for more than 2048 segments (the mask travels in the kernel arguments).
+ * The call copies nothing from the host and takes every per-segment decision on the device from the device's
+ * lengths; launch shapes follow the capacities.  A step (append, metadata append, this call, attention over
+ * step_cache with a plan built once) can therefore be captured in a CUDA graph and replayed while the caches
+ * grow; step_cache->seg_len on the host is then the value of the captured call (an upper bound: the kept
+ * length moves within one chunk as the source grows).
  */
 size_t catekv_retrieval_meta_bytes(const catekv_cache* cache, int32_t chunk_size);
 int catekv_retrieval_build(const catekv_cache* cache, int32_t chunk_size, void* meta, catekv_stream stream);

@@ -270,7 +270,7 @@ def catekv_retrieve_compact(cache: Cache, meta: torch.Tensor, chunk_size: int, q
     assert q.is_contiguous() and q.dtype == torch.bfloat16
     retrieval_mask = np.ascontiguousarray(retrieval_mask, dtype=np.uint8).reshape(-1)
     if ws is None:
-        ws = torch.empty(_lib.catekv_retrieve_workspace_bytes(cache.B, cache.Hkv, int(cache.seg_len.max())),
+        ws = torch.empty(_lib.catekv_retrieve_workspace_bytes(cache.B, cache.Hkv, int(cache.seg_cap.max())),
                          dtype=torch.uint8, device=cache.device)
     stride = 0 if idx_out is None else idx_out.stride(0)
     _check(_lib.catekv_retrieve_compact(C.byref(cache.struct), meta.data_ptr(), chunk_size, q.data_ptr(), q.shape[1],

@@ -57,6 +57,8 @@ static_assert(sizeof(CtaHeader) == 48, "cta header layout");
 struct SegInfo {
   int32_t slot_begin;
   int32_t n_pieces;
+  int32_t plan_len;  // rows the segment held when the plan was built
+  int32_t reserved;
 };
 
 struct PlanLayout {
@@ -138,10 +140,12 @@ __device__ __forceinline__ ItemCursor plan_cursor(const WorkItem& w) {
 // the part that reads what earlier kernels wrote: the live length (a plain load: with a fused append this
 // kernel itself updates the length when it is done with the segment)
 __device__ __forceinline__ void live_cursor(const DecodeArgs& a, ItemCursor& c) {
+  const int len = *reinterpret_cast<const volatile int32_t*>(a.seg_len + c.seg);
   if (c.last) {
-    const int len = *reinterpret_cast<const volatile int32_t*>(a.seg_len + c.seg);
     c.new_row = a.k_new ? len : -1;
     c.live = a.k_new ? len + 1 : len;
+  } else {
+    c.live = min(c.t1, len);  // a segment that has shrunk since the plan was built: attend only to what it holds
   }
 }
 __device__ __forceinline__ WorkItem unpack_item(const int4& x, const int4& y) {
@@ -167,7 +171,7 @@ __device__ __forceinline__ int item_tiles(const ItemCursor& c) {
 __device__ __forceinline__ void tile_rows(const ItemCursor& c, int i, int& start, int& nvalid) {
   if (i < c.np) {
     start = c.t0 + i * kTile;
-    nvalid = c.t1 - start;
+    nvalid = min(c.t1, c.live) - start;  // <= 0: the whole tile lies behind the live length
   } else {
     start = c.t1 + (i - c.np) * kTile;
     nvalid = c.live - start;
@@ -705,7 +709,7 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
       if (len == 0) {
         // an empty segment still gets one (direct) item, so that the plan stays valid once it grows
         items[n_items++] = WorkItem{seg, 0, 0, -1, (int64_t)cache->seg_off[seg], 1, 0};
-        segs[seg] = SegInfo{0, 1};
+        segs[seg] = SegInfo{0, 1, 0, 0};
         ++seg;
         seg_first_item = n_items;
         continue;
@@ -721,10 +725,10 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
         items[n_items - 1].last = 1;  // the last piece follows the segment's current length
         if (pieces == 1) {
           items[seg_first_item].slot = -1;
-          segs[seg] = SegInfo{0, 1};
+          segs[seg] = SegInfo{0, 1, len, 0};
         } else {
           for (int i = 0; i < pieces; ++i) items[seg_first_item + i].slot = n_slots + i;
-          segs[seg] = SegInfo{n_slots, pieces};
+          segs[seg] = SegInfo{n_slots, pieces, len, 0};
           n_slots += pieces;
           max_pieces = pieces > max_pieces ? pieces : max_pieces;
         }
@@ -859,6 +863,19 @@ extern "C" int catekv_append_decode_attn(catekv_cache* cache, const void* k_new,
   for (int s = 0; s < n; ++s) {
     if (cache->seg_len[s] < 0) return CATEKV_ERR_INVALID_ARG;
     if (cache->seg_len[s] + 1 > cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+  }
+  // The appended row must lie behind every row the plan knows: the kernel requests plan-time tiles before it
+  // may look at the lengths.  (catekv_decode_attn, without the append, also takes segments that have shrunk.)
+  if (plan_host && plan_bytes >= sizeof(PlanHeader)) {
+    const PlanHeader* hdr = (const PlanHeader*)plan_host;
+    if (hdr->magic == kPlanMagic && hdr->n_segs == n && hdr->num_ctas > 0) {
+      const PlanLayout L = plan_layout(n, hdr->num_ctas);
+      if (plan_bytes >= L.bytes) {
+        const SegInfo* si = (const SegInfo*)((const uint8_t*)plan_host + L.off_seg);
+        for (int s = 0; s < n; ++s)
+          if (cache->seg_len[s] < si[s].plan_len) return CATEKV_ERR_INVALID_ARG;
+      }
+    }
   }
   rc = decode_launch(3, cache, k_new, v_new, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev,
                      plan_bytes, ws, ws_bytes, stream);

@@ -69,11 +69,40 @@ __global__ void __launch_bounds__(128) meta_append_kernel(const int32_t* seg_off
 }
 
 // ---- chunk scores ----------------------------------------------------------------------------
-struct RetJob {
-  int32_t b, h;        // sequence and KV head
-  int32_t chunk0;      // global index of the first candidate chunk
-  int32_t n_pool;      // candidate chunks
+
+// Per-segment decisions (what to keep, how many chunks to select) are taken on the device from its own lengths,
+// by the scoring kernel itself: a step needs no host-to-device copy and can be captured in a CUDA graph.  The
+// host makes the same decisions from its mirror for the capacity check.
+struct RetParams {
+  int32_t cs, budget, sink2 /* sink rounded up to whole chunks */, local, Hkv;
 };
+constexpr int kRetMaxSegs = 2048;
+struct RetMask {  // which segments retrieve, one bit each; travels by value in the kernel arguments
+  uint32_t w[kRetMaxSegs / 32];
+};
+__host__ __device__ inline SelSeg retrieval_decide(int n, bool enabled, const RetParams& p) {
+  SelSeg d = {};
+  d.n = n;
+  d.job = -1;
+  d.keep_all = 1;
+  d.len_ub = n;
+  if (enabled && p.budget < n) {
+    const int cand_end = (n - p.local > 0 ? n - p.local : 0) / p.cs * p.cs;  // first row of the always-taken tail
+    if (cand_end > p.sink2) {
+      const int forced = p.sink2 + (n - cand_end);
+      const int n_pool = (cand_end - p.sink2) / p.cs;
+      const int k_sel = p.budget - forced > 0 ? (p.budget - forced) / p.cs : 0;
+      if (k_sel < n_pool) {
+        d.keep_all = 0;
+        d.cand_end = cand_end;
+        d.n_pool = n_pool;
+        d.k_sel = k_sel;
+        d.len_ub = forced + k_sel * p.cs;
+      }
+    }
+  }
+  return d;
+}
 
 // Monotone map of arbitrary finite floats to non-negative floats whose bit patterns order the same way as the
 // values (what the radix select of the top-k kernel needs): flip so that larger values get larger unsigned
@@ -97,11 +126,36 @@ __device__ __forceinline__ uint32_t rs_off(int row, int piece) {  // 16-byte pie
   return (uint32_t)(row * kRsRowBytes + ((piece ^ (row & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(kRsThreads, 2) retrieval_score_kernel(const RetJob* jobs, const uint8_t* meta, const uint16_t* q,
-                                                                        int Hq, int G, float* P, int64_t p_stride) {
+struct RetScoreArgs {
+  RetParams p;
+  RetMask mask;
+  const int32_t* seg_len;  // the source cache's lengths and offsets
+  const int32_t* seg_off;
+  const uint8_t* meta;
+  const uint16_t* q;
+  int32_t Hq, G;
+  float* P;
+  int64_t p_stride;
+  SelSeg* segs;  // out: the decision per segment, for the top-k and gather kernels that follow
+};
+struct RetJobView {
+  int32_t b, h, chunk0 /* global index of the first candidate chunk */, n_pool /* candidate chunks */;
+};
+
+__global__ void __launch_bounds__(kRsThreads, 2) retrieval_score_kernel(const RetScoreArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  const RetJob job = jobs[blockIdx.y];
-  if (job.n_pool == 0) return;  // this segment selects nothing
+  const int seg = blockIdx.y;
+  SelSeg d = retrieval_decide(a.seg_len[seg], (a.mask.w[seg >> 5] >> (seg & 31)) & 1u, a.p);
+  const bool scores = !d.keep_all && d.k_sel > 0;
+  if (scores) d.job = seg;  // score row = segment index
+  if (blockIdx.x == 0 && threadIdx.x == 0) a.segs[seg] = d;
+  if (!scores) return;  // this segment selects nothing
+  const RetJobView job = {seg / a.p.Hkv, seg % a.p.Hkv, a.seg_off[seg] / a.p.cs + a.p.sink2 / a.p.cs, d.n_pool};
+  const uint8_t* meta = a.meta;
+  const uint16_t* q = a.q;
+  const int Hq = a.Hq, G = a.G;
+  float* P = a.P;
+  const int64_t p_stride = a.p_stride;
   // this CTA's chunks: an equal share, in whole tiles
   const int tiles_total = (job.n_pool + kRsTile - 1) / kRsTile;
   const int tiles_per = (tiles_total + gridDim.x - 1) / gridDim.x;
@@ -178,51 +232,8 @@ __global__ void __launch_bounds__(kRsThreads, 2) retrieval_score_kernel(const Re
   cp_async_wait<0>();
 }
 
-// Per-segment decisions (what to keep, how many chunks to select) from the device's own lengths, so that a step
-// needs no host-to-device copy.  The host makes the same decisions from its mirror for the capacity check.
-struct RetParams {
-  int32_t cs, budget, sink2 /* sink rounded up to whole chunks */, local, Hkv;
-};
-__host__ __device__ inline SelSeg retrieval_decide(int n, bool enabled, const RetParams& p) {
-  SelSeg d = {};
-  d.n = n;
-  d.job = -1;
-  d.keep_all = 1;
-  d.len_ub = n;
-  if (enabled && p.budget < n) {
-    const int cand_end = (n - p.local > 0 ? n - p.local : 0) / p.cs * p.cs;  // first row of the always-taken tail
-    if (cand_end > p.sink2) {
-      const int forced = p.sink2 + (n - cand_end);
-      const int n_pool = (cand_end - p.sink2) / p.cs;
-      const int k_sel = p.budget - forced > 0 ? (p.budget - forced) / p.cs : 0;
-      if (k_sel < n_pool) {
-        d.keep_all = 0;
-        d.cand_end = cand_end;
-        d.n_pool = n_pool;
-        d.k_sel = k_sel;
-        d.len_ub = forced + k_sel * p.cs;
-      }
-    }
-  }
-  return d;
-}
-__global__ void retrieval_plan_kernel(const int32_t* seg_len, const int32_t* seg_off, const uint8_t* mask, RetParams p,
-                                      SelSeg* segs, RetJob* jobs, int n_segs) {
-  const int s = blockIdx.x * blockDim.x + threadIdx.x;
-  if (s >= n_segs) return;
-  SelSeg d = retrieval_decide(seg_len[s], mask[s] != 0, p);
-  RetJob j = {s / p.Hkv, s % p.Hkv, 0, 0};
-  if (!d.keep_all && d.k_sel > 0) {
-    d.job = s;  // job slot = segment index
-    j.chunk0 = seg_off[s] / p.cs + p.sink2 / p.cs;
-    j.n_pool = d.n_pool;
-  }
-  segs[s] = d;
-  jobs[s] = j;
-}
-
 struct RetWs {
-  size_t off_segs, off_jobs, off_mask, off_P, off_idx, bytes;
+  size_t off_segs, off_P, off_idx, bytes;
   int64_t p_stride, idx_stride;
 };
 static RetWs ret_ws_layout(int n_segs, int max_len) {
@@ -231,8 +242,6 @@ static RetWs ret_ws_layout(int n_segs, int max_len) {
   w.idx_stride = w.p_stride;
   size_t o = 0;
   w.off_segs = o; o = align_up(o + sizeof(SelSeg) * (size_t)n_segs, 256);
-  w.off_jobs = o; o = align_up(o + sizeof(RetJob) * (size_t)n_segs, 256);
-  w.off_mask = o; o = align_up(o + (size_t)n_segs, 256);
   w.off_P = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.p_stride, 256);
   w.off_idx = o; o = align_up(o + sizeof(int32_t) * (size_t)n_segs * w.idx_stride, 256);
   w.bytes = o;
@@ -308,53 +317,61 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
   if (G > kMaxG) return CATEKV_ERR_UNSUPPORTED;
   const int n_segs = cache->B * cache->Hkv;
   const int cs = chunk_size;
-  int max_len = 0;
+  if (n_segs > kRetMaxSegs) return CATEKV_ERR_UNSUPPORTED;
+  // Launch shapes and the scratch layout follow the capacities, not the current lengths: the same launches stay
+  // valid while the caches grow, so a captured step can be replayed.
+  int max_len = 0, max_cap = 0, max_step_cap = 0;
   for (int s = 0; s < n_segs; ++s) {
     if (cache->seg_len[s] < 0 || cache->seg_len[s] > cache->seg_cap[s]) return CATEKV_ERR_INVALID_ARG;
     max_len = cache->seg_len[s] > max_len ? cache->seg_len[s] : max_len;
+    max_cap = cache->seg_cap[s] > max_cap ? cache->seg_cap[s] : max_cap;
+    max_step_cap = step_cache->seg_cap[s] > max_step_cap ? step_cache->seg_cap[s] : max_step_cap;
   }
   if (idx_out && idx_stride < max_len) return CATEKV_ERR_INVALID_ARG;
-  const RetWs W = ret_ws_layout(n_segs, max_len);
+  const RetWs W = ret_ws_layout(n_segs, max_cap);
   if (ws_bytes < W.bytes) return CATEKV_ERR_WORKSPACE;
 
-  RetParams rp;
+  RetScoreArgs sa = {};
+  RetParams& rp = sa.p;
   rp.cs = cs;
   rp.budget = budget;
   rp.sink2 = (sink + cs - 1) / cs * cs;  // sink rows rounded up to whole chunks
   rp.local = local;
   rp.Hkv = cache->Hkv;
   const int S2 = rp.sink2;
-  int max_out = 0, max_pool = 0;
-  bool any_job = false;
   for (int s = 0; s < n_segs; ++s) {
     const SelSeg d = retrieval_decide(cache->seg_len[s], retrieval_mask[s] != 0, rp);
     if (d.len_ub > step_cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
-    max_out = d.len_ub > max_out ? d.len_ub : max_out;
-    if (!d.keep_all && d.k_sel > 0) {
-      any_job = true;
-      max_pool = d.n_pool > max_pool ? d.n_pool : max_pool;
-    }
+    if (retrieval_mask[s]) sa.mask.w[s >> 5] |= 1u << (s & 31);
   }
+  const int max_pool = max_cap / cs;  // bound of the candidate chunks of a segment
 
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* w8 = (uint8_t*)ws;
   SelSeg* d_segs = (SelSeg*)(w8 + W.off_segs);
-  RetJob* d_jobs = (RetJob*)(w8 + W.off_jobs);
-  uint8_t* d_mask = w8 + W.off_mask;
   float* P = (float*)(w8 + W.off_P);
-  // the mask is the only table that comes from the host (n_segs bytes)
-  CATEKV_CUDA_TRY(cudaMemcpyAsync(d_mask, retrieval_mask, (size_t)n_segs, cudaMemcpyHostToDevice, st));
-  retrieval_plan_kernel<<<(n_segs + 127) / 128, 128, 0, st>>>(cache->seg_len_dev, cache->seg_off_dev, d_mask, rp, d_segs, d_jobs,
-                                                              n_segs);
-  CATEKV_CUDA_TRY(cudaGetLastError());
-  if (any_job) {
+  {
     // a few 64-chunk tiles per CTA, enough CTAs to fill the machine
     int gx = (max_pool + 8 * kRsTile - 1) / (8 * kRsTile);
     if (gx > 64) gx = 64;
     if (gx < 1) gx = 1;
-    CATEKV_CUDA_TRY(cudaFuncSetAttribute(retrieval_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRsSmem));
-    retrieval_score_kernel<<<dim3(gx, (unsigned)n_segs), kRsThreads, kRsSmem, st>>>(d_jobs, (const uint8_t*)meta, (const uint16_t*)q,
-                                                                                     Hq, G, P, W.p_stride);
+    static bool attr_set[64] = {};
+    int dev = 0;
+    CATEKV_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+      CATEKV_CUDA_TRY(cudaFuncSetAttribute(retrieval_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRsSmem));
+      if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    sa.seg_len = cache->seg_len_dev;
+    sa.seg_off = cache->seg_off_dev;
+    sa.meta = (const uint8_t*)meta;
+    sa.q = (const uint16_t*)q;
+    sa.Hq = Hq;
+    sa.G = G;
+    sa.P = P;
+    sa.p_stride = W.p_stride;
+    sa.segs = d_segs;
+    retrieval_score_kernel<<<dim3(gx, (unsigned)n_segs), kRsThreads, kRsSmem, st>>>(sa);
     CATEKV_CUDA_TRY(cudaGetLastError());
   }
   TopkArgs ta;
@@ -370,8 +387,6 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
   ta.pool_mode = kPoolPrescored;
   ta.pool_param = cs;
   rc = launch_topk(ta, n_segs, max_pool, st);
-  if (rc) return rc;
-  rc = launch_set_full_len(d_segs, step_cache->seg_len_dev, n_segs, st);
   if (rc) return rc;
   GatherArgs ga;
   ga.segs = d_segs;
@@ -390,7 +405,7 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
   ga.idx_out = idx_out;
   ga.idx_out_stride = idx_stride;
   ga.Hkv = cache->Hkv;
-  rc = launch_gather(ga, max_out, n_segs, st);
+  rc = launch_gather(ga, max_step_cap, n_segs, st);
   if (rc) return rc;
   for (int s = 0; s < n_segs; ++s) step_cache->seg_len[s] = retrieval_decide(cache->seg_len[s], retrieval_mask[s] != 0, rp).len_ub;
   return CATEKV_OK;

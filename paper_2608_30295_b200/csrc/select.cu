@@ -62,6 +62,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
   __shared__ unsigned long long s_warp[33];
   __shared__ unsigned int s_pair[2];
   __shared__ unsigned long long s_tot;  // this CTA's (greater, equal) totals, read by its peers
+  extern __shared__ unsigned int stage[];  // a.stage_entries words: this CTA's share of the pooled scores
   auto cluster_sync = [&]() {
     if (CL > 1) cluster.sync(); else __syncthreads();
   };
@@ -132,9 +133,24 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
       }
     }
     __syncthreads();  // a CTA reads back only its own share of P
+    // The share is read six more times (four digit passes, the counts, the compaction): from shared memory if it
+    // fits the staging area the launch provided, else from global memory (L2).
+    const unsigned int* Pg = reinterpret_cast<const unsigned int*>(P);
+    const bool staged = hi - lo <= a.stage_entries;
+    if (staged) {
+      for (int c0 = lo + tid; c0 < hi; c0 += 4 * kTopkThreads) {  // four loads in flight
+        unsigned int vv[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) vv[e] = (c0 + e * kTopkThreads < hi) ? Pg[c0 + e * kTopkThreads] : 0u;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (c0 + e * kTopkThreads < hi) stage[c0 + e * kTopkThreads - lo] = vv[e];
+      }
+      __syncthreads();
+    }
+    const unsigned int* Pb = staged ? stage - lo : Pg;  // Pb[c], lo <= c < hi
     // ---- radix select of the k_sel-th largest pooled score: 8 bits per pass from the top (scores are >= 0, so
     // their bit patterns order as integers); the histograms of the CTAs are summed through distributed shared memory
-    const unsigned int* Pb = reinterpret_cast<const unsigned int*>(P);
     unsigned int prefix = 0, need = (unsigned int)s.k_sel;
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
@@ -167,16 +183,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
         hsum[tid] = t;
       }
       __syncthreads();
-      if (tid == 0) {
-        unsigned int cum = 0;
-        int dsel = 0;
-        for (int dgt = 255; dgt >= 0; --dgt) {
-          if (cum + hsum[dgt] >= need) { dsel = dgt; break; }
-          cum += hsum[dgt];
-        }
-        s_pair[0] = prefix | ((unsigned int)dsel << shift);
-        s_pair[1] = need - cum;
-      }
+      if (tid < 32) radix_pick_digit(hsum, need, prefix, shift, s_pair);
       cluster_sync();  // decision visible; the peers are done reading this CTA's histogram
       prefix = s_pair[0];
       need = s_pair[1];
@@ -239,7 +246,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     if (cs > 1) {
       const int last = s.n_pool - 1;
       const int last_sz = s.cand_end - (S + last * cs);
-      const unsigned int vl = Pb[last];  // written by the last CTA before the cluster barriers above
+      const unsigned int vl = Pg[last];  // written by the last CTA before the cluster barriers above
       // the last chunk is taken iff it is above the threshold, or ties with it and is within the quota of ties
       const unsigned int eq_total = (unsigned int)(all >> 32);
       const bool last_taken = vl > thr || (vl == thr && eq_total <= need_eq);
@@ -255,19 +262,14 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
   }
 }
 
-// keep_all segments: seg_len = n
-__global__ void set_full_len_kernel(const SelSeg* segs, int32_t* seg_len_dev, int n_segs) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n_segs && segs[i].keep_all) seg_len_dev[i] = segs[i].n;
-}
-
 constexpr int kGatherRowsPerBlock = 64;
 
 // One warp per kept row: lanes 0-15 move the K row, lanes 16-31 the V row (16 bytes each).
 __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
   const int seg = blockIdx.y;
   const SelSeg s = a.segs[seg];
-  const int len = a.seg_len_dev[seg];
+  const int len = s.keep_all ? s.n : a.seg_len_dev[seg];  // a straight copy keeps all n rows
+  if (s.keep_all && blockIdx.x == 0 && threadIdx.x == 0) a.seg_len_dev[seg] = s.n;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = seg / a.Hkv, h = seg % a.Hkv;
   const int64_t off = a.seg_off[seg];
@@ -286,9 +288,24 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
   }
 }
 
-int launch_topk(const TopkArgs& a, int n_segs, int max_pool, cudaStream_t stream) {
-  if (max_pool < 16384) {  // short lists: one CTA per segment
-    topk_kernel<1><<<n_segs, kTopkThreads, 0, stream>>>(a);
+constexpr int kTopkStageMax = 16384;  // pooled entries a CTA may stage in shared memory (64 KB)
+
+int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, cudaStream_t stream) {
+  static bool attr_set[64] = {};
+  int dev = 0;
+  CATEKV_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkStageMax * 4));
+    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkStageMax * 4));
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  TopkArgs a = a0;
+  const int CL = max_pool <= kTopkStageMax ? 1 : 8;  // lists that one CTA can stage: one CTA per segment
+  const int share = ((max_pool + CL - 1) / CL + 3) / 4 * 4;
+  a.stage_entries = share <= kTopkStageMax ? share : 0;  // longer shares are read from global memory
+  const size_t smem = (size_t)a.stage_entries * 4;
+  if (CL == 1) {
+    topk_kernel<1><<<n_segs, kTopkThreads, smem, stream>>>(a);
     CATEKV_CUDA_TRY(cudaGetLastError());
     return CATEKV_OK;
   }
@@ -296,6 +313,7 @@ int launch_topk(const TopkArgs& a, int n_segs, int max_pool, cudaStream_t stream
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_segs * 8);
   cfg.blockDim = dim3(kTopkThreads);
+  cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -307,14 +325,10 @@ int launch_topk(const TopkArgs& a, int n_segs, int max_pool, cudaStream_t stream
   CATEKV_CUDA_TRY(cudaLaunchKernelEx(&cfg, topk_kernel<8>, a));
   return CATEKV_OK;
 }
-int launch_set_full_len(const SelSeg* segs, int32_t* seg_len_dev, int n_segs, cudaStream_t stream) {
-  set_full_len_kernel<<<(n_segs + 255) / 256, 256, 0, stream>>>(segs, seg_len_dev, n_segs);
-  CATEKV_CUDA_TRY(cudaGetLastError());
-  return CATEKV_OK;
-}
 int launch_gather(const GatherArgs& a, int max_len, int n_segs, cudaStream_t stream) {
-  if (max_len <= 0) return CATEKV_OK;
-  gather_kernel<<<dim3((max_len + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock, n_segs), 256, 0, stream>>>(a);
+  // at least one block per segment: block 0 also records the length of a straight copy
+  const int gx = max_len > 0 ? (max_len + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock : 1;
+  gather_kernel<<<dim3(gx, n_segs), 256, 0, stream>>>(a);
   CATEKV_CUDA_TRY(cudaGetLastError());
   return CATEKV_OK;
 }
@@ -496,9 +510,6 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
     int rc2 = launch_topk(ta, n_segs, max_pool, st);
     if (rc2) return rc2;
   }
-  set_full_len_kernel<<<(n_segs + 255) / 256, 256, 0, st>>>(d_segs, cache->seg_len_dev, n_segs);
-  CATEKV_CUDA_TRY(cudaGetLastError());
-
   GatherArgs ga;
   ga.segs = d_segs;
   ga.idx = ta.idx;
@@ -516,8 +527,10 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   ga.idx_out_stride = idx_stride;
   ga.Hkv = p->Hkv;
   ga.src_seg_off = nullptr;
-  gather_kernel<<<dim3((max_len_ub + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock, n_segs), 256, 0, st>>>(ga);
-  CATEKV_CUDA_TRY(cudaGetLastError());
+  {
+    int rc2 = launch_gather(ga, max_len_ub, n_segs, st);
+    if (rc2) return rc2;
+  }
 
   if (need_readback) {
     // a short last chunk makes the kept length depend on the scores: fetch the device's lengths

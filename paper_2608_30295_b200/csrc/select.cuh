@@ -28,6 +28,7 @@ struct TopkArgs {
   int64_t idx_stride;
   int32_t* seg_len_dev;
   int32_t sink, L_obs, pool_mode, pool_param;  // the always-kept tail of a segment is [cand_end, n)
+  int32_t stage_entries;  // set by launch_topk: pooled entries per CTA that the dynamic shared memory holds
 };
 
 struct GatherArgs {
@@ -41,7 +42,7 @@ struct GatherArgs {
   uint8_t* k_pool;
   uint8_t* v_pool;
   const int32_t* seg_off;
-  const int32_t* seg_len_dev;
+  int32_t* seg_len_dev;  // kept length per segment: read for selecting segments, written for keep_all ones
   int32_t* idx_out;
   int64_t idx_out_stride;
   int32_t Hkv;
@@ -49,7 +50,6 @@ struct GatherArgs {
 
 
 int launch_topk(const TopkArgs& a, int n_segs, int max_pool, cudaStream_t stream);  // max_pool: longest pooled list
-int launch_set_full_len(const SelSeg* segs, int32_t* seg_len_dev, int n_segs, cudaStream_t stream);
 int launch_gather(const GatherArgs& a, int max_len, int n_segs, cudaStream_t stream);
 
 }  // namespace catekv

@@ -118,6 +118,42 @@ def test_append_then_decode_with_stale_plan(ck):
     assert np.array_equal(cache.seg_len, before) and cache.seg_len_dev.cpu().tolist() == before.tolist()
 
 
+@pytest.mark.parametrize("num_ctas", [1, 9, 40])
+def test_decode_with_stale_plan_after_segments_shrank(ck, num_ctas):
+    """A plan built for longer lists stays valid when lists get shorter (a per-step cache that is refilled with
+    fewer rows): rows behind the live length are left out, whole pieces included; a list cut to nothing gives 0."""
+    lens = [700, 64, 1500, 3, 90, 400, 2000, 128]
+    new_lens = [693, 64, 130, 0, 1, 399, 1999, 17]  # by a few rows, across piece boundaries, to one row, to nothing
+    oc = H.random_cache(2, 4, lens, seed=23)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=8)
+    plan = ck.DecodePlan(cache, num_ctas)
+    ck.catekv_decode_plan(cache, plan)
+    cache.set_lengths(new_lens)
+    short = orc.HybridCache(2, 4, 128)
+    for i, L in enumerate(new_lens):
+        short.k_rows.append(oc.k_rows[i][:L])
+        short.v_rows.append(oc.v_rows[i][:L])
+    q = synth.randn_bf16((2, 16, 128), "cpu", 23, "q")
+    o32 = torch.full((2, 16, 128), float("nan"), dtype=torch.float32, device="cuda")
+    lse = torch.full((2, 16), float("nan"), dtype=torch.float32, device="cuda")
+    ck.catekv_decode_attn(cache, q.cuda(), plan, o32, lse)
+    torch.cuda.synchronize()
+    ref, ref_lse = orc.decode_attention(short, synth.bits(q))
+    H.check_attention(o32, None, lse, ref, ref_lse, "shrunk")
+    assert torch.all(o32[0, 12:16] == 0)  # the emptied list (sequence 0, KV head 3)
+    # the fused append needs lengths that are not below the plan's
+    kn = synth.randn_bf16((2, 4, 128), "cuda", 23, "kn")
+    with pytest.raises(ck.CatekvError) as e:
+        ck.catekv_append_decode_attn(cache, kn, kn, q.cuda(), plan, o32, lse)
+    assert e.value.code == ck.ERR_INVALID_ARG
+    # grown back (and beyond): the same plan again
+    cache.set_lengths(lens)
+    ck.catekv_decode_attn(cache, q.cuda(), plan, o32, lse)
+    torch.cuda.synchronize()
+    ref, ref_lse = orc.decode_attention(oc, synth.bits(q))
+    H.check_attention(o32, None, lse, ref, ref_lse, "restored")
+
+
 def test_decode_is_deterministic(ck):
     oc = H.random_cache(2, 4, [700, 64, 1500, 3, 90, 400, 2000, 128], seed=17)
     q = synth.bits(synth.randn_bf16((2, 16, 128), "cpu", 17, "q"))

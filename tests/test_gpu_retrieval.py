@@ -154,3 +154,75 @@ def test_retrieval_finds_loud_keys_and_budget_covers_all(ck):
     with pytest.raises(ck.CatekvError) as e:
         ck.catekv_retrieve_compact(cache, meta, 8, q, [1], 256, 4, 64, small)
     assert e.value.code == ck.ERR_CAPACITY
+
+
+def test_retrieval_step_replayed_as_cuda_graph(ck):
+    """append + metadata append + retrieve + attention captured once and replayed while the lists grow: the kept
+    lengths move within a chunk under a decode plan that was built once, and every step matches the oracle."""
+    cs, G, B, Hkv = 8, 4, 2, 2
+    lens = [900, 300, 1500, 40]
+    budget, sink, local = 256, 4, 32
+    steps = 11  # crosses a chunk boundary of every list
+    oc = H.random_cache(B, Hkv, lens, seed=81)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=steps + 2)
+    meta = ck.catekv_retrieval_meta(cache, cs)
+    ck.catekv_retrieval_build(cache, cs, meta)
+    mask = np.array([1, 1, 1, 0], dtype=np.uint8)
+    step_cache = ck.Cache(B, Hkv, [budget + 2 * cs if mask[s] and L > budget else L + steps + 2
+                                   for s, L in enumerate(lens)], 0, "cuda")
+    q = torch.empty((B, Hkv * G, 128), dtype=torch.bfloat16, device="cuda")
+    kn = torch.empty((B, Hkv, 128), dtype=torch.bfloat16, device="cuda")
+    vn = torch.empty_like(kn)
+    out = torch.empty((B, Hkv * G, 128), dtype=torch.float32, device="cuda")
+    idx = torch.full((B * Hkv, max(lens) + steps + 2), -1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(ck._lib.catekv_retrieve_workspace_bytes(B, Hkv, int(cache.seg_cap.max())), dtype=torch.uint8,
+                     device="cuda")
+    ck.catekv_retrieve_compact(cache, meta, cs, q.zero_(), mask, budget, sink, local, step_cache, ws=ws)
+    plan = ck.DecodePlan(step_cache, 7)
+    ck.catekv_decode_plan(step_cache, plan)  # once, from the lengths of this first fill
+
+    def one_step():
+        ck.catekv_append(cache, kn, vn)
+        ck.catekv_retrieval_append(cache, cs, kn, meta)
+        ck.catekv_retrieve_compact(cache, meta, cs, q, mask, budget, sink, local, step_cache, idx_out=idx, ws=ws)
+        ck.catekv_decode_attn(step_cache, q, plan, out)
+
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            one_step()  # host code only: the host mirror of `cache` advances by one row
+    torch.cuda.current_stream().wait_stream(side)
+    seen_lens = set()
+    for t in range(steps):
+        q.copy_(synth.randn_bf16((B, Hkv * G, 128), "cuda", 81, "q", t))
+        kn.copy_(synth.randn_bf16((B, Hkv, 128), "cuda", 81, "kn", t))
+        vn.copy_(synth.randn_bf16((B, Hkv, 128), "cuda", 81, "vn", t))
+        if t:
+            ck.catekv_cache_advance(cache, 1)
+        g.replay()
+        torch.cuda.synchronize()
+        oc.append(synth.bits(kn), synth.bits(vn))
+        qb = orc.bf16_to_f64(synth.bits(q))
+        got_len = step_cache.seg_len_dev.cpu().tolist()
+        got_idx = idx.cpu().numpy()
+        soc = orc.HybridCache(B, Hkv, 128)
+        for s in range(B * Hkv):
+            L = lens[s] + t + 1
+            got = got_idx[s, :got_len[s]].astype(np.int64)
+            if mask[s] and L > budget:
+                kmax, kmin = orc.retrieval_metadata(oc.k_rows[s], cs)
+                b, h = divmod(s, Hkv)
+                scores = orc.retrieval_scores(qb[b, h * G:(h + 1) * G], kmax, kmin)
+                _check_selection(got, scores, L, sink, local, budget, cs, f"step {t} seg {s}")
+            else:
+                assert np.array_equal(got, np.arange(L)), (t, s)
+            soc.k_rows.append(oc.k_rows[s][got])
+            soc.v_rows.append(oc.v_rows[s][got])
+        seen_lens.add(got_len[0])
+        ref, _ = orc.decode_attention(soc, synth.bits(q))
+        H.check_attention(out, None, None, ref, None, f"graph step {t}")
+    assert len(seen_lens) > 1  # the kept length did move under the plan
+    assert list(cache.seg_len) == [L + steps for L in lens] == cache.seg_len_dev.cpu().tolist()

@@ -77,7 +77,7 @@ def _plan(ck, lens, B, Hkv, num_ctas):
     # (seg, t0, t1 or -1 for the piece that follows the live length, slot)
     items = np.stack([raw[:, 0], raw[:, 1], np.where(raw[:, 6] == 1, -1, raw[:, 2]), raw[:, 3]], axis=1) \
         if n_items else np.zeros((0, 4), dtype=np.int32)
-    segs = buf[off_seg:off_seg + 8 * B * Hkv].view(np.int32).reshape(-1, 2)
+    segs = buf[off_seg:off_seg + 16 * B * Hkv].view(np.int32).reshape(-1, 4)
     return cta, items, segs, n_slots
 
 
@@ -105,7 +105,8 @@ def test_decode_plan_covers_every_row_once_and_balances(ck, lens, num_ctas):
         pieces[seg].append((i, t1, slot))
     for s in range(n):
         assert pos[s] == lens[s]
-        sb, npieces = segs[s]
+        sb, npieces, plan_len, _ = segs[s]
+        assert plan_len == lens[s]
         assert npieces == len(pieces[s])
         assert npieces >= 1
         if npieces:
