@@ -71,10 +71,16 @@ __device__ __forceinline__ void block_radix_select(Load load, int n, unsigned in
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const bool hit = in[e] && (v[e] & pmask) == prefix;
-        // lanes with the same digit elect one of them to add their count (scores cluster in a few bins)
+        // a warp whose lanes all fall in one bin (the common case in the top digit: scores share their exponent)
+        // adds once; otherwise every hit adds for itself, the digits being spread over the bins
         const unsigned int dgt = hit ? ((v[e] >> shift) & 0xffu) : 0x100u;
-        const unsigned int peers = __match_any_sync(0xffffffffu, dgt);
-        if (hit && (threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[dgt], (unsigned int)__popc(peers));
+        int same;
+        __match_all_sync(0xffffffffu, dgt, &same);
+        if (same) {
+          if (hit && (threadIdx.x & 31) == 0) atomicAdd(&hist[dgt], 32u);
+        } else if (hit) {
+          atomicAdd(&hist[dgt], 1u);
+        }
       }
     }
     __syncthreads();

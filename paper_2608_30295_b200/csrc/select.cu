@@ -17,6 +17,20 @@ namespace catekv {
 
 constexpr int kTopkThreads = 1024;
 
+#ifdef CATEKV_TOPK_TRACE
+__device__ unsigned long long g_topk_trace[64 * 16];
+#define TOPK_STAMP(i)                                                                       \
+  do {                                                                                      \
+    if (threadIdx.x == 0 && blockIdx.x < 64) {                                              \
+      unsigned long long t_;                                                                \
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                                 \
+      g_topk_trace[blockIdx.x * 16 + (i)] = t_;                                             \
+    }                                                                                       \
+  } while (0)
+#else
+#define TOPK_STAMP(i)
+#endif
+
 // Block-wide exclusive scan of a packed pair (lo 32 bits, hi 32 bits) over 1024 threads.
 __device__ __forceinline__ unsigned long long block_excl_scan(unsigned long long v, unsigned long long* s_warp,
                                                               unsigned long long& total) {
@@ -57,10 +71,12 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
   const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
   const SelSeg s = a.segs[seg];
   if (s.keep_all) return;  // the whole cluster leaves
+  TOPK_STAMP(0);
   __shared__ unsigned int hist[256];
   __shared__ unsigned int hsum[256];
   __shared__ unsigned long long s_warp[33];
   __shared__ unsigned int s_pair[2];
+  __shared__ unsigned int s_mm[2];  // smallest and largest bit pattern of this CTA's share
   __shared__ unsigned long long s_tot;  // this CTA's (greater, equal) totals, read by its peers
   extern __shared__ unsigned int stage[];  // a.stage_entries words: this CTA's share of the pooled scores
   auto cluster_sync = [&]() {
@@ -133,46 +149,81 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
       }
     }
     __syncthreads();  // a CTA reads back only its own share of P
-    // The share is read six more times (four digit passes, the counts, the compaction): from shared memory if it
-    // fits the staging area the launch provided, else from global memory (L2).
+    // The share is read several more times (digit passes, counts, compaction): from shared memory if it fits the
+    // staging area the launch provided (entry i of the share at word i + i / 32: the pad keeps both the strided
+    // sweeps of the digit passes and the per-thread runs of the compaction free of bank conflicts), else from
+    // global memory (L2).  The same sweep finds the smallest and largest bit pattern.
     const unsigned int* Pg = reinterpret_cast<const unsigned int*>(P);
-    const bool staged = hi - lo <= a.stage_entries;
-    if (staged) {
-      for (int c0 = lo + tid; c0 < hi; c0 += 4 * kTopkThreads) {  // four loads in flight
-        unsigned int vv[4];
+    const int n_loc = hi - lo;
+    const bool staged = n_loc <= a.stage_entries;
+    auto sp = [](int i) { return i + (i >> 5); };
+    unsigned int vmin = 0xffffffffu, vmax = 0u;
+    for (int i0 = tid; i0 < n_loc; i0 += 4 * kTopkThreads) {  // four loads in flight
+      unsigned int vv[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) vv[e] = (c0 + e * kTopkThreads < hi) ? Pg[c0 + e * kTopkThreads] : 0u;
+      for (int e = 0; e < 4; ++e) vv[e] = (i0 + e * kTopkThreads < n_loc) ? Pg[lo + i0 + e * kTopkThreads] : 0u;
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if (c0 + e * kTopkThreads < hi) stage[c0 + e * kTopkThreads - lo] = vv[e];
-      }
-      __syncthreads();
+      for (int e = 0; e < 4; ++e)
+        if (i0 + e * kTopkThreads < n_loc) {
+          if (staged) stage[sp(i0 + e * kTopkThreads)] = vv[e];
+          vmin = min(vmin, vv[e]);
+          vmax = max(vmax, vv[e]);
+        }
     }
-    const unsigned int* Pb = staged ? stage - lo : Pg;  // Pb[c], lo <= c < hi
-    // ---- radix select of the k_sel-th largest pooled score: 8 bits per pass from the top (scores are >= 0, so
-    // their bit patterns order as integers); the histograms of the CTAs are summed through distributed shared memory
-    unsigned int prefix = 0, need = (unsigned int)s.k_sel;
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      const unsigned int pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+    if (tid == 0) {
+      s_mm[0] = 0xffffffffu;
+      s_mm[1] = 0u;
+    }
+    __syncthreads();
+    vmin = __reduce_min_sync(0xffffffffu, vmin);
+    vmax = __reduce_max_sync(0xffffffffu, vmax);
+    if ((tid & 31) == 0) {
+      atomicMin(&s_mm[0], vmin);
+      atomicMax(&s_mm[1], vmax);
+    }
+    cluster_sync();  // staging complete; every CTA's extremes are in its shared memory
+    unsigned int gmin = 0xffffffffu, gmax = 0u;
+#pragma unroll
+    for (int r = 0; r < CL; ++r) {
+      gmin = min(gmin, CL > 1 ? *cluster.map_shared_rank(&s_mm[0], r) : s_mm[0]);
+      gmax = max(gmax, CL > 1 ? *cluster.map_shared_rank(&s_mm[1], r) : s_mm[1]);
+    }
+    auto ldp = [&](int i) { return staged ? stage[sp(i)] : Pg[lo + i]; };  // entry i of this CTA's share
+    TOPK_STAMP(1);
+    // ---- radix select of the k_sel-th largest pooled score (scores are >= 0, so their bit patterns order as
+    // integers).  The bits above the highest bit in which the extremes differ are common to all entries and become
+    // the prefix; the nb bits below are resolved from the top, up to 8 per pass, with the CTAs' histograms summed
+    // through distributed shared memory.  Scores within a factor of two of one another need three passes.
+    int nb = 32 - __clz(gmin ^ gmax);  // 0: all entries are equal
+    unsigned int prefix = nb >= 32 ? 0u : (gmax >> nb) << nb, need = (unsigned int)s.k_sel;
+    int pass_no = 0;
+    while (nb > 0) {
+      const int wbits = min(8, nb);
+      const int shift = nb - wbits;
+      const unsigned int dmask = (1u << wbits) - 1u;
+      const unsigned int pmask = shift + wbits >= 32 ? 0u : (0xffffffffu << (shift + wbits));
       if (tid < 256) hist[tid] = 0;
       __syncthreads();
-      for (int c0 = lo; c0 < hi; c0 += 4 * kTopkThreads) {  // whole warps stay in the loop: the vote needs them
+      for (int i0 = 0; i0 < n_loc; i0 += 4 * kTopkThreads) {  // whole warps stay in the loop: the vote needs them
         unsigned int v[4];
         bool in[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const int c = c0 + e * kTopkThreads + tid;
-          in[e] = c < hi;
-          v[e] = in[e] ? Pb[c] : 0u;
+          const int i = i0 + e * kTopkThreads + tid;
+          in[e] = i < n_loc;
+          v[e] = in[e] ? ldp(i) : 0u;
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const bool hit = in[e] && (v[e] & pmask) == prefix;
-          // lanes with the same digit elect one of them to add their count (scores cluster in a few bins)
-          const unsigned int dgt = hit ? ((v[e] >> shift) & 0xffu) : 0x100u;
-          const unsigned int peers = __match_any_sync(0xffffffffu, dgt);
-          if (hit && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[dgt], (unsigned int)__popc(peers));
+          // a warp whose lanes all fall in one bin adds once; otherwise every hit adds for itself
+          const unsigned int dgt = hit ? ((v[e] >> shift) & dmask) : 0x100u;
+          const unsigned int d0 = __shfl_sync(0xffffffffu, dgt, 0);
+          if (__all_sync(0xffffffffu, dgt == d0)) {
+            if (hit && (tid & 31) == 0) atomicAdd(&hist[dgt], 32u);
+          } else if (hit) {
+            atomicAdd(&hist[dgt], 1u);
+          }
         }
       }
       cluster_sync();  // all histograms complete
@@ -187,60 +238,95 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
       cluster_sync();  // decision visible; the peers are done reading this CTA's histogram
       prefix = s_pair[0];
       need = s_pair[1];
+      nb = shift;
+      TOPK_STAMP(2 + pass_no);
+      ++pass_no;
     }
     const unsigned int thr = prefix, need_eq = need;  // threshold bits; ties taken (lowest index first)
-    // ---- (greater, equal) counts of every CTA's share -> where this CTA's selected entries start
-    unsigned long long mine_tot = 0;
-    for (int c = lo + tid; c < hi; c += kTopkThreads) {
-      const unsigned int v = Pb[c];
-      mine_tot += (unsigned long long)(v > thr) | ((unsigned long long)(v == thr) << 32);
-    }
-    {
-      unsigned long long tot;
-      block_excl_scan(mine_tot, s_warp, tot);
-      if (tid == 0) s_tot = tot;
-    }
-    cluster_sync();
-    unsigned long long run = 0, all = 0;  // packed: low = entries above the threshold, high = entries equal to it
-#pragma unroll
-    for (int r = 0; r < CL; ++r) {
-      const unsigned long long t = CL > 1 ? *cluster.map_shared_rank(&s_tot, r) : s_tot;
-      if (r < rank) run += t;
-      all += t;
-    }
-    // ---- ordered compaction, four consecutive entries per thread and step
+    // ---- ordered compaction.  A thread owns a run of consecutive entries of the share (staged) or, per step of
+    // 4096 entries, four consecutive ones (from global memory): it counts its entries above and at the threshold,
+    // an exclusive scan over the block (plus the totals of the CTAs before this one) says where its selected
+    // entries go, and it writes them in order.
     const int cs = (a.pool_mode == CATEKV_POOL_CHUNK || a.pool_mode == kPoolPrescored) ? a.pool_param : 1;
-    for (int base = lo; base < hi; base += 4 * kTopkThreads) {
-      const int c4 = base + tid * 4;
-      unsigned int v[4];
-      bool gt[4], eq[4];
+    auto emit = [&](int c, unsigned int rnk) {  // pooled entry c of the segment is the rnk-th selected one
+      if (cs == 1) {
+        idx[S + rnk] = S + c;
+      } else {
+        const int l2 = S + c * cs, h2 = min(l2 + cs, s.cand_end);
+        for (int u = l2; u < h2; ++u) idx[S + rnk * cs + (u - l2)] = u;
+      }
+    };
+    unsigned long long all = 0;  // packed: low = entries above the threshold, high = entries equal to it
+    if (staged) {
+      const int E = (n_loc + kTopkThreads - 1) / kTopkThreads;
+      const int r0 = min(n_loc, tid * E), r1 = min(n_loc, r0 + E);
       unsigned long long mine = 0;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        v[e] = (c4 + e < hi) ? Pb[c4 + e] : 0u;
-        gt[e] = (c4 + e < hi) && v[e] > thr;
-        eq[e] = (c4 + e < hi) && v[e] == thr;
-        mine += (unsigned long long)gt[e] | ((unsigned long long)eq[e] << 32);
+      for (int i = r0; i < r1; ++i) {
+        const unsigned int v = stage[sp(i)];
+        mine += (unsigned long long)(v > thr) | ((unsigned long long)(v == thr) << 32);
       }
       unsigned long long tot;
-      unsigned long long ex = run + block_excl_scan(mine, s_warp, tot);
+      unsigned long long ex = block_excl_scan(mine, s_warp, tot);
+      if (tid == 0) s_tot = tot;
+      cluster_sync();
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const unsigned int gt_before = (unsigned int)(ex & 0xffffffffu), eq_before = (unsigned int)(ex >> 32);
-        if (gt[e] || (eq[e] && eq_before < need_eq)) {
-          const unsigned int rnk = gt_before + min(eq_before, need_eq);
-          const int c = c4 + e;
-          if (cs == 1) {
-            idx[S + rnk] = S + c;
-          } else {
-            const int l2 = S + c * cs, h2 = min(l2 + cs, s.cand_end);
-            for (int u = l2; u < h2; ++u) idx[S + rnk * cs + (u - l2)] = u;
-          }
-        }
-        ex += (unsigned long long)gt[e] | ((unsigned long long)eq[e] << 32);
+      for (int r = 0; r < CL; ++r) {
+        const unsigned long long t = CL > 1 ? *cluster.map_shared_rank(&s_tot, r) : s_tot;
+        if (r < rank) ex += t;
+        all += t;
       }
-      run += tot;
+      TOPK_STAMP(6);
+      for (int i = r0; i < r1; ++i) {
+        const unsigned int v = stage[sp(i)];
+        const bool gt = v > thr, eq = v == thr;
+        const unsigned int gt_before = (unsigned int)(ex & 0xffffffffu), eq_before = (unsigned int)(ex >> 32);
+        if (gt || (eq && eq_before < need_eq)) emit(lo + i, gt_before + min(eq_before, need_eq));
+        ex += (unsigned long long)gt | ((unsigned long long)eq << 32);
+      }
+    } else {
+      unsigned long long mine_tot = 0;
+      for (int c = lo + tid; c < hi; c += kTopkThreads) {
+        const unsigned int v = Pg[c];
+        mine_tot += (unsigned long long)(v > thr) | ((unsigned long long)(v == thr) << 32);
+      }
+      {
+        unsigned long long tot;
+        block_excl_scan(mine_tot, s_warp, tot);
+        if (tid == 0) s_tot = tot;
+      }
+      cluster_sync();
+      unsigned long long run = 0;
+#pragma unroll
+      for (int r = 0; r < CL; ++r) {
+        const unsigned long long t = CL > 1 ? *cluster.map_shared_rank(&s_tot, r) : s_tot;
+        if (r < rank) run += t;
+        all += t;
+      }
+      TOPK_STAMP(6);
+      for (int base = lo; base < hi; base += 4 * kTopkThreads) {
+        const int c4 = base + tid * 4;
+        unsigned int v[4];
+        bool gt[4], eq[4];
+        unsigned long long mine = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          v[e] = (c4 + e < hi) ? Pg[c4 + e] : 0u;
+          gt[e] = (c4 + e < hi) && v[e] > thr;
+          eq[e] = (c4 + e < hi) && v[e] == thr;
+          mine += (unsigned long long)gt[e] | ((unsigned long long)eq[e] << 32);
+        }
+        unsigned long long tot;
+        unsigned long long ex = run + block_excl_scan(mine, s_warp, tot);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const unsigned int gt_before = (unsigned int)(ex & 0xffffffffu), eq_before = (unsigned int)(ex >> 32);
+          if (gt[e] || (eq[e] && eq_before < need_eq)) emit(c4 + e, gt_before + min(eq_before, need_eq));
+          ex += (unsigned long long)gt[e] | ((unsigned long long)eq[e] << 32);
+        }
+        run += tot;
+      }
     }
+    TOPK_STAMP(7);
     // selected tokens: whole chunks, except that the last chunk of the range may be short
     n_sel_tokens = s.k_sel * cs;
     if (cs > 1) {
@@ -260,6 +346,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     for (int i = tid; i < n_tail; i += kTopkThreads) idx[S + n_sel_tokens + i] = s.cand_end + i;
     if (tid == 0) a.seg_len_dev[seg] = S + n_sel_tokens + n_tail;
   }
+  TOPK_STAMP(8);
 }
 
 constexpr int kGatherRowsPerBlock = 64;
@@ -288,22 +375,30 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
   }
 }
 
-constexpr int kTopkStageMax = 16384;  // pooled entries a CTA may stage in shared memory (64 KB)
+constexpr int kTopkStageMax = 32768;  // pooled entries a CTA may stage in shared memory (132 KB with the padding)
+
+#ifdef CATEKV_TOPK_TRACE
+}  // namespace catekv
+extern "C" int catekv_debug_topk_trace(unsigned long long* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, catekv::g_topk_trace, sizeof(unsigned long long) * 64 * 16);
+}
+namespace catekv {
+#endif
 
 int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, cudaStream_t stream) {
   static bool attr_set[64] = {};
   int dev = 0;
   CATEKV_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkStageMax * 4));
-    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkStageMax * 4));
+    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (kTopkStageMax + kTopkStageMax / 32 + 1) * 4));
+    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (kTopkStageMax + kTopkStageMax / 32 + 1) * 4));
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
   TopkArgs a = a0;
-  const int CL = max_pool <= kTopkStageMax ? 1 : 8;  // lists that one CTA can stage: one CTA per segment
+  const int CL = max_pool <= 16384 ? 1 : 8;  // short lists: one CTA per segment
   const int share = ((max_pool + CL - 1) / CL + 3) / 4 * 4;
   a.stage_entries = share <= kTopkStageMax ? share : 0;  // longer shares are read from global memory
-  const size_t smem = (size_t)a.stage_entries * 4;
+  const size_t smem = (size_t)(a.stage_entries + a.stage_entries / 32 + 1) * 4;
   if (CL == 1) {
     topk_kernel<1><<<n_segs, kTopkThreads, smem, stream>>>(a);
     CATEKV_CUDA_TRY(cudaGetLastError());
