@@ -343,10 +343,11 @@ def time_head_cv(ck, dev):
     return e0.elapsed_time(e1) / 3
 
 
-def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8, graph=True):
+def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8, graph=True, gather=False):
     """Decode step with query-aware retrieval on the adaptive heads (budget rows per adaptive head, chunk size 8):
-    per layer catekv_append + catekv_retrieval_append + catekv_retrieve_compact + catekv_decode_attn over the
-    per-step cache, replayed as a CUDA graph of the step (graph=False: host launches).
+    per layer catekv_append + catekv_retrieval_append + catekv_retrieve_select + catekv_decode_attn_indexed
+    (attention in place through the index lists), replayed as a CUDA graph of the step (graph=False: host
+    launches).  gather=True: catekv_retrieve_compact into a per-step cache + catekv_decode_attn instead.
     Returns (us per layer-step, attended bytes per layer-step, metadata bytes per layer-step)."""
     import torch
     from workloads import synth
@@ -361,22 +362,36 @@ def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8, graph=Tru
         m["meta"] = ck.catekv_retrieval_meta(c, cs)
         ck.catekv_retrieval_build(c, cs, m["meta"])
         m["rmask"] = (m["mask"].reshape(-1) == 0).astype(np.uint8)
-        slens = [min(int(L), budget + 2 * cs + w.local) if m["rmask"][i] else int(L) + steps + 16
-                 for i, L in enumerate(c.seg_len)]
-        m["step"] = ck.Cache(w.B, w.Hkv, slens, 0, dev)
         m["ws"] = torch.empty(ck._lib.catekv_retrieve_workspace_bytes(w.B, w.Hkv, int(c.seg_cap.max())),
                               dtype=torch.uint8, device=dev)
-        ck.catekv_retrieve_compact(c, m["meta"], cs, q[l], m["rmask"], budget, w.sink, w.local, m["step"], ws=m["ws"])
-        m["splan"] = ck.DecodePlan(m["step"], num_ctas)
-        ck.catekv_decode_plan(m["step"], m["splan"])
+        m["lens"] = ck.catekv_retrieve_lengths(c, cs, m["rmask"], budget, w.sink, w.local)
+        if gather:
+            slens = [min(int(L), budget + 2 * cs + w.local) if m["rmask"][i] else int(L) + steps + 16
+                     for i, L in enumerate(c.seg_len)]
+            m["step"] = ck.Cache(w.B, w.Hkv, slens, 0, dev)
+            ck.catekv_retrieve_compact(c, m["meta"], cs, q[l], m["rmask"], budget, w.sink, w.local, m["step"],
+                                       ws=m["ws"])
+            m["splan"] = ck.DecodePlan(m["step"], num_ctas)
+            ck.catekv_decode_plan(m["step"], m["splan"])
+        else:
+            m["idx"] = torch.zeros((w.B * w.Hkv, budget + 2 * cs + w.local), dtype=torch.int32, device=dev)
+            m["sel"] = torch.zeros(w.B * w.Hkv, dtype=torch.int32, device=dev)
+            m["view"] = ck.CacheView(c, m["lens"])
+            m["splan"] = ck.DecodePlan(m["view"], num_ctas)
+            ck.catekv_decode_plan(m["view"], m["splan"])
 
     def step():
         for l, m in enumerate(model):
             ck.catekv_append(m["cache"], kn[l], vn[l])
             ck.catekv_retrieval_append(m["cache"], cs, kn[l], m["meta"])
-            ck.catekv_retrieve_compact(m["cache"], m["meta"], cs, q[l], m["rmask"], budget, w.sink, w.local, m["step"],
-                                       ws=m["ws"])
-            ck.catekv_decode_attn(m["step"], q[l], m["splan"], out)
+            if gather:
+                ck.catekv_retrieve_compact(m["cache"], m["meta"], cs, q[l], m["rmask"], budget, w.sink, w.local,
+                                           m["step"], ws=m["ws"])
+                ck.catekv_decode_attn(m["step"], q[l], m["splan"], out)
+            else:
+                ck.catekv_retrieve_select(m["cache"], m["meta"], cs, q[l], m["rmask"], budget, w.sink, w.local,
+                                          m["idx"], m["sel"], ws=m["ws"])
+                ck.catekv_decode_attn_indexed(m["cache"], m["idx"], m["sel"], q[l], m["splan"], out)
 
     run = step
     if graph:
@@ -402,7 +417,7 @@ def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8, graph=Tru
         run()
     e1.record()
     torch.cuda.synchronize()
-    attended = float(np.mean([int(m["step"].seg_len.sum()) * ROW_BYTES for m in model]))
+    attended = float(np.mean([int(m["lens"].sum()) * ROW_BYTES for m in model]))
     meta_bytes = float(np.mean([int(m["cache"].seg_len[m["rmask"] == 1].sum()) // cs * 512 for m in model]))
     return e0.elapsed_time(e1) * 1e3 / (steps * n_layers), attended, meta_bytes
 
@@ -497,6 +512,8 @@ def main():
                     "for --layers layers and print its time; used for profiling that path on a small case")
     ap.add_argument("--retrieval-only", action="store_true", help="run only the query-aware retrieval decode step "
                     "(small case for profiling; use with --workload and --layers)")
+    ap.add_argument("--retrieval-gather", action="store_true", help="with --retrieval-only: the gather path "
+                    "(catekv_retrieve_compact into a per-step cache) instead of attention in place")
     ap.add_argument("--no-extras", action="store_true", help="skip the other configs, head_cv and the oracle timing")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -532,7 +549,8 @@ def main():
     global FUSED
     FUSED = not args.no_fused
     if args.retrieval_only:
-        ru, ra, rm = time_retrieval(ck, w, dev, n_layers=n_layers, steps=args.steps, graph=graph)
+        ru, ra, rm = time_retrieval(ck, w, dev, n_layers=n_layers, steps=args.steps, graph=graph,
+                                    gather=args.retrieval_gather)
         if rank == 0:
             print(json.dumps({"workload": w.name, "layers": n_layers, "retrieval_us_per_layer_step": ru,
                               "attended_bytes_per_layer_step": ra, "metadata_bytes_per_layer_step": rm}))
@@ -614,7 +632,8 @@ def main():
         ru, ra, rm = time_retrieval(ck, w, dev)
         line["retrieval"] = {"us_per_layer_step": ru, "attended_bytes_per_layer_step": ra,
                              "metadata_bytes_per_layer_step": rm, "budget_rows": 1024, "chunk": 8,
-                             "note": "query-aware retrieval on the adaptive heads of the same workload (CUDA graph replay of the step)"}
+                             "note": "query-aware retrieval on the adaptive heads of the same workload: per layer append, metadata "
+                                     "append, catekv_retrieve_select, catekv_decode_attn_indexed; CUDA graph replay of the step"}
         rate, desc, spent = oracle_sample_rate(w, target_s=15.0)
         rows = bytes_per_layer / ROW_BYTES
         line["cpu_baseline"] = {"value": w.B / (w.layers * rows / rate), "unit": UNIT, "cores": oracle_threads(),

@@ -294,6 +294,34 @@ int catekv_retrieve_compact(const catekv_cache* cache, const void* meta, int32_t
                             catekv_stream stream);
 
 /*
+ * The same retrieval without the copy: catekv_retrieve_select stops after the chunk selection and leaves, per
+ * segment, the ascending list of the rows to attend to; catekv_decode_attn_indexed then reads those rows in
+ * place, straight from `cache` (the same split-KV kernel, each 256-byte row addressed through the list), and
+ * the whole list of every segment that retrieves nothing.  No per-step cache, no gather traffic.
+ *
+ *   idx      device int32 [B*Hkv, idx_stride]: rows (relative to the segment) of the segments that retrieve;
+ *            idx_stride must hold the longest kept list (catekv_retrieve_lengths)
+ *   sel_len  device int32 [B*Hkv]: the kept length of a segment that retrieves, -1 for a segment that is
+ *            attended to as a whole (mask 0, or not longer than the budget)
+ *   catekv_retrieve_lengths: host only; lens_out[s] = rows segment s will be attended over for these
+ *            parameters and the current host lengths.  A decode plan for catekv_decode_attn_indexed is built by
+ *            catekv_decode_plan from a cache descriptor whose host seg_len array holds these lengths (same
+ *            pools, offsets and capacities); like every plan it stays valid while the lengths move.
+ *   The other arguments, the errors and the CUDA-graph property are those of catekv_retrieve_compact and
+ *   catekv_decode_attn.  catekv_decode_attn_indexed requests no rows before the preceding kernel has finished
+ *   (the lists are that kernel's output).
+ */
+int catekv_retrieve_select(const catekv_cache* cache, const void* meta, int32_t chunk_size, const void* q, int32_t Hq,
+                           const uint8_t* retrieval_mask, int32_t budget, int32_t sink, int32_t local, int32_t* idx,
+                           int64_t idx_stride, int32_t* sel_len, void* ws, size_t ws_bytes, catekv_stream stream);
+int catekv_retrieve_lengths(const catekv_cache* cache, int32_t chunk_size, const uint8_t* retrieval_mask, int32_t budget,
+                            int32_t sink, int32_t local, int32_t* lens_out);
+int catekv_decode_attn_indexed(const catekv_cache* cache, const int32_t* idx, int64_t idx_stride, const int32_t* sel_len,
+                               const void* q, int32_t Hq, float sm_scale, void* out, int32_t out_dtype, float* lse_out,
+                               const void* plan_host, const void* plan_dev, size_t plan_bytes, void* ws, size_t ws_bytes,
+                               catekv_stream stream);
+
+/*
  * Attention recall of the kept rows (Section 3.4, the recall curves of the consistent / streaming / Quest /
  * top-k patterns): for each query head, the share of the full softmax mass that falls on the rows its hybrid
  * list keeps, recall = exp(lse_kept - lse_full), 0 for an empty list.  lse_kept is the lse_out of a

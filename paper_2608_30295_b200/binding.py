@@ -84,6 +84,11 @@ def _load():
         "catekv_retrieve_workspace_bytes": (sz, [i32, i32, i32]),
         "catekv_retrieve_compact": (C.c_int, [C.POINTER(CacheStruct), vp, i32, vp, i32, vp, i32, i32, i32,
                                               C.POINTER(CacheStruct), vp, i64, vp, sz, vp]),
+        "catekv_retrieve_select": (C.c_int, [C.POINTER(CacheStruct), vp, i32, vp, i32, vp, i32, i32, i32, vp, i64, vp,
+                                             vp, sz, vp]),
+        "catekv_retrieve_lengths": (C.c_int, [C.POINTER(CacheStruct), i32, vp, i32, i32, i32, vp]),
+        "catekv_decode_attn_indexed": (C.c_int, [C.POINTER(CacheStruct), vp, i64, vp, vp, i32, f32, vp, i32, vp, vp, vp,
+                                                 sz, vp, sz, vp]),
         "catekv_decode_attn_noalloc": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp]),
     }
     for name, (res, args) in sig.items():
@@ -278,6 +283,62 @@ def catekv_retrieve_compact(cache: Cache, meta: torch.Tensor, chunk_size: int, q
                                         _dev_ptr(idx_out), stride, ws.data_ptr(), ws.numel(), _stream()),
            "catekv_retrieve_compact")
     return ws
+
+
+def catekv_retrieve_lengths(cache: Cache, chunk_size: int, retrieval_mask, budget: int, sink: int, local: int):
+    """Host only: rows every segment is attended over under query-aware retrieval with these parameters."""
+    retrieval_mask = np.ascontiguousarray(retrieval_mask, dtype=np.uint8).reshape(-1)
+    lens = np.zeros(cache.B * cache.Hkv, dtype=np.int32)
+    _check(_lib.catekv_retrieve_lengths(C.byref(cache.struct), chunk_size, _np_ptr(retrieval_mask), budget, sink,
+                                        local, _np_ptr(lens)), "catekv_retrieve_lengths")
+    return lens
+
+
+class CacheView:
+    """The pools, offsets and capacities of `cache` under other host lengths: what catekv_decode_plan needs to
+    plan catekv_decode_attn_indexed (lens = catekv_retrieve_lengths).  Memory only; shares the device arrays."""
+
+    def __init__(self, cache: Cache, lens):
+        self.B, self.Hkv, self.d, self.device = cache.B, cache.Hkv, cache.d, cache.device
+        self.base = cache
+        self.seg_off, self.seg_cap = cache.seg_off, cache.seg_cap
+        self.seg_len = np.ascontiguousarray(lens, dtype=np.int32).reshape(-1).copy()
+        b = cache.struct
+        self.struct = CacheStruct(b.B, b.Hkv, b.d, 0, b.total_rows, b.k_pool, b.v_pool, b.seg_off_dev, b.seg_len_dev,
+                                  b.seg_off, b.seg_cap, _np_ptr(self.seg_len))
+
+
+def catekv_retrieve_select(cache: Cache, meta: torch.Tensor, chunk_size: int, q: torch.Tensor, retrieval_mask,
+                           budget: int, sink: int, local: int, idx: torch.Tensor, sel_len: torch.Tensor,
+                           ws: Optional[torch.Tensor] = None):
+    assert q.is_contiguous() and q.dtype == torch.bfloat16
+    assert idx.dtype == torch.int32 and sel_len.dtype == torch.int32 and idx.stride(1) == 1
+    retrieval_mask = np.ascontiguousarray(retrieval_mask, dtype=np.uint8).reshape(-1)
+    if ws is None:
+        ws = torch.empty(_lib.catekv_retrieve_workspace_bytes(cache.B, cache.Hkv, int(cache.seg_cap.max())),
+                         dtype=torch.uint8, device=cache.device)
+    _check(_lib.catekv_retrieve_select(C.byref(cache.struct), meta.data_ptr(), chunk_size, q.data_ptr(), q.shape[1],
+                                       _np_ptr(retrieval_mask), budget, sink, local, idx.data_ptr(), idx.stride(0),
+                                       sel_len.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "catekv_retrieve_select")
+    return ws
+
+
+def catekv_decode_attn_indexed(cache: Cache, idx: torch.Tensor, sel_len: torch.Tensor, q: torch.Tensor,
+                               plan: DecodePlan, out: torch.Tensor, lse_out: Optional[torch.Tensor] = None,
+                               sm_scale: float = 0.0):
+    assert q.is_contiguous() and out.is_contiguous() and q.dtype == torch.bfloat16
+    assert idx.dtype == torch.int32 and sel_len.dtype == torch.int32 and idx.stride(1) == 1
+    if out.dtype == torch.bfloat16:
+        od = OUT_BF16
+    elif out.dtype == torch.float32:
+        od = OUT_FP32
+    else:
+        raise TypeError("out must be bf16 or fp32")
+    _check(_lib.catekv_decode_attn_indexed(C.byref(cache.struct), idx.data_ptr(), idx.stride(0), sel_len.data_ptr(),
+                                           q.data_ptr(), q.shape[1], sm_scale, out.data_ptr(), od, _dev_ptr(lse_out),
+                                           plan.host.data_ptr(), plan.dev.data_ptr(), plan.bytes, plan.ws.data_ptr(),
+                                           plan.ws_bytes, _stream()), "catekv_decode_attn_indexed")
 
 
 NOALLOC_SCRATCH_BYTES = 4 << 20

@@ -93,6 +93,11 @@ struct DecodeArgs {
   int32_t* seg_len;
   const uint8_t* k_new;  // fused append: this step's [B*Hkv, d] rows, else null
   const uint8_t* v_new;
+  // indexed variant only: segment s attends to the rows idx[s * idx_stride + 0 .. sel_len[s]) of its list (ascending
+  // row numbers relative to the segment) if sel_len[s] >= 0, to its whole list if sel_len[s] < 0
+  const int32_t* idx;
+  int64_t idx_stride;
+  const int32_t* sel_len;
   const uint16_t* q;  // [B, Hq, d]
   int32_t Hq, Hkv, G;
   float scale_log2;  // sm_scale * log2(e)
@@ -120,6 +125,7 @@ struct ItemCursor {
   int np;            // tiles of the plan-time rows
   int live;          // rows to attend to: current segment length (plus the row being appended), if last
   int new_row;       // fused append: the segment-relative row that comes from k_new / v_new, else -1
+  int indexed;       // indexed variant: the item's rows are taken through the index list
   int64_t row_base;
 };
 
@@ -135,15 +141,24 @@ __device__ __forceinline__ ItemCursor plan_cursor(const WorkItem& w) {
   c.np = (w.t1 - w.t0 + kTile - 1) / kTile;
   c.live = w.t1;
   c.new_row = -1;
+  c.indexed = 0;
   return c;
 }
 // the part that reads what earlier kernels wrote: the live length (a plain load: with a fused append this
 // kernel itself updates the length when it is done with the segment)
+template <bool kIndexed>
 __device__ __forceinline__ void live_cursor(const DecodeArgs& a, ItemCursor& c) {
-  const int len = *reinterpret_cast<const volatile int32_t*>(a.seg_len + c.seg);
+  int len;
+  if (kIndexed) {
+    const int sel = *reinterpret_cast<const volatile int32_t*>(a.sel_len + c.seg);
+    c.indexed = sel >= 0;
+    len = sel >= 0 ? sel : *reinterpret_cast<const volatile int32_t*>(a.seg_len + c.seg);
+  } else {
+    len = *reinterpret_cast<const volatile int32_t*>(a.seg_len + c.seg);
+  }
   if (c.last) {
-    c.new_row = a.k_new ? len : -1;
-    c.live = a.k_new ? len + 1 : len;
+    c.new_row = (!kIndexed && a.k_new) ? len : -1;
+    c.live = (!kIndexed && a.k_new) ? len + 1 : len;
   } else {
     c.live = min(c.t1, len);  // a segment that has shrunk since the plan was built: attend only to what it holds
   }
@@ -155,10 +170,11 @@ __device__ __forceinline__ WorkItem unpack_item(const int4& x, const int4& y) {
   w.last = y.z; w.reserved = 0;
   return w;
 }
+template <bool kIndexed>
 __device__ __forceinline__ ItemCursor read_item(const DecodeArgs& a, int it) {
   const int4* p = reinterpret_cast<const int4*>(a.items + it);
   ItemCursor c = plan_cursor(unpack_item(__ldg(p), __ldg(p + 1)));
-  live_cursor(a, c);
+  live_cursor<kIndexed>(a, c);
   return c;
 }
 // tiles of the item: plan-time tiles plus tiles of the appended rows; at least one
@@ -190,6 +206,7 @@ __device__ __forceinline__ unsigned long long gtime() {
 #define CATEKV_STAMP(i) do { } while (0)
 #endif
 
+template <bool kIndexed>
 __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -225,7 +242,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       const int id = tid + i * kDecodeThreads;
       const int r = id >> 4, c = id & 15;
       const int ok = r < rows_left ? 16 : 0;
-      const int64_t goff = (ok ? row0 + r : 0) * kRowBytes + c * 16;  // padding rows read nothing
+      int64_t grow = ok ? row0 + r : 0;  // padding rows read nothing
+      if (kIndexed && pc.indexed && ok)
+        grow = (pc.row_base - pc.t0) + __ldg(a.idx + (int64_t)pc.seg * a.idx_stride + start + r);
+      const int64_t goff = grow * kRowBytes + c * 16;
       const uint32_t so = tile_off(r, c);
       if (ok && r == new_r && pc.new_row >= 0) {  // only inside the tile's valid rows (never in a plan-time tile)
         // the decoded token's row: attend to it from k_new / v_new and store it in the pool
@@ -252,7 +272,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     ++p_seq;
     if (++p_tile >= pc.np && p_tile >= item_tiles(pc)) {
       p_tile = 0;
-      if (++p_item < item_end) pc = read_item(a, p_item);
+      if (++p_item < item_end) pc = read_item<kIndexed>(a, p_item);
     }
   };
   auto issue = [&]() {  // one tile (with the item's queries if it is the item's first) = one commit group
@@ -266,7 +286,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
 
   // Rows that were valid when the plan was built are older than anything the previous kernel of the stream
   // may still be writing (an append writes behind them): the first tiles are requested before the wait.
-  const int pre = min(kStages - 1, pc.np);
+  // (not in the indexed variant: its rows are named by the index list, which the preceding kernel writes)
+  const int pre = kIndexed ? 0 : min(kStages - 1, pc.np);
   for (int s = 0; s < pre; ++s) {
     issue_tile();
     ++p_seq;
@@ -274,19 +295,19 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     cp_async_commit();
   }
   pdl_wait();  // from here on: lengths, queries and rows written by earlier kernels
-  live_cursor(a, pc);
+  live_cursor<kIndexed>(a, pc);
   const ItemCursor first = pc;
   issue_q(0, pc.seg);
   if (p_tile >= pc.np && p_tile >= item_tiles(pc)) {
     p_tile = 0;
-    if (++p_item < item_end) pc = read_item(a, p_item);
+    if (++p_item < item_end) pc = read_item<kIndexed>(a, p_item);
   }
   for (int s = pre; s < kStages - 1; ++s) issue();
   if (pre == kStages - 1) cp_async_commit();  // the queries of the first item form a group of their own
 
   int seq = 0;
   for (int c_item = item_begin; c_item < item_end; ++c_item) {
-    const ItemCursor cc = c_item == item_begin ? first : read_item(a, c_item);
+    const ItemCursor cc = c_item == item_begin ? first : read_item<kIndexed>(a, c_item);
     uint32_t qf[8][2];
     float o[8][4];
 #pragma unroll
@@ -652,11 +673,11 @@ extern "C" int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens) {
 extern "C" int catekv_decode_num_ctas(void) {
   int dev = 0, sms = 0, per_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return CATEKV_ERR_CUDA;
-  cudaError_t e = cudaFuncSetAttribute(decode_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
+  cudaError_t e = cudaFuncSetAttribute(decode_partial_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
   if (e != cudaSuccess) { set_cuda_error(e); return CATEKV_ERR_CUDA; }
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) { set_cuda_error(e); return CATEKV_ERR_CUDA; }
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_partial_kernel, kDecodeThreads, kDecodeSmem);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_partial_kernel<false>, kDecodeThreads, kDecodeSmem);
   if (e != cudaSuccess) { set_cuda_error(e); return CATEKV_ERR_CUDA; }
   if (per_sm < 1) per_sm = 1;
   return sms * per_sm;
@@ -759,10 +780,17 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
 }
 
 // phases: 1 = attention partials, 2 = combine, 3 = both
+struct IndexList {  // indexed attention: see DecodeArgs
+  const int32_t* idx;
+  int64_t idx_stride;
+  const int32_t* sel_len;
+};
+
 static int decode_launch(int phases, const catekv_cache* cache, const void* k_new, const void* v_new, const void* q,
                          int32_t Hq, float sm_scale, void* out,
                          int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
-                         size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+                         size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream,
+                         const IndexList* il = nullptr) {
   int rc = check_cache(cache);
   if (rc) return rc;
   if (!q || !out || !plan_host || !plan_dev || !ws) return CATEKV_ERR_INVALID_ARG;
@@ -791,7 +819,8 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* k_ne
     int dev = 0;
     CATEKV_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-      CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
+      CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
+      CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
       if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     DecodeArgs a;
@@ -813,7 +842,13 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* k_ne
     a.out = out;
     a.out_fp32 = out_fp32;
     a.lse_out = lse_out;
-    CATEKV_CUDA_TRY(launch_pdl(decode_partial_kernel, dim3(hdr->num_ctas), dim3(kDecodeThreads), kDecodeSmem, st, a));
+    a.idx = il ? il->idx : nullptr;
+    a.idx_stride = il ? il->idx_stride : 0;
+    a.sel_len = il ? il->sel_len : nullptr;
+    if (il)
+      CATEKV_CUDA_TRY(launch_pdl(decode_partial_kernel<true>, dim3(hdr->num_ctas), dim3(kDecodeThreads), kDecodeSmem, st, a));
+    else
+      CATEKV_CUDA_TRY(launch_pdl(decode_partial_kernel<false>, dim3(hdr->num_ctas), dim3(kDecodeThreads), kDecodeSmem, st, a));
   }
   if ((phases & 2) && hdr->n_slots > 0) {
     CombineArgs ca;
@@ -836,6 +871,16 @@ extern "C" int catekv_decode_attn(const catekv_cache* cache, const void* q, int3
                                   size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
   return decode_launch(3, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
                        ws_bytes, stream);
+}
+
+extern "C" int catekv_decode_attn_indexed(const catekv_cache* cache, const int32_t* idx, int64_t idx_stride,
+                                          const int32_t* sel_len, const void* q, int32_t Hq, float sm_scale, void* out,
+                                          int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
+                                          size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+  if (!idx || !sel_len || idx_stride < 0) return CATEKV_ERR_INVALID_ARG;
+  const IndexList il = {idx, idx_stride, sel_len};
+  return decode_launch(3, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
+                       ws_bytes, stream, &il);
 }
 
 extern "C" int catekv_decode_partials(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,

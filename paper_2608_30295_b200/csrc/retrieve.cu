@@ -301,17 +301,23 @@ extern "C" size_t catekv_retrieve_workspace_bytes(int32_t B, int32_t Hkv, int32_
   return ret_ws_layout(B * Hkv, max_len).bytes;
 }
 
-extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* meta, int32_t chunk_size, const void* q,
-                                       int32_t Hq, const uint8_t* retrieval_mask, int32_t budget, int32_t sink, int32_t local,
-                                       catekv_cache* step_cache, int32_t* idx_out, int64_t idx_stride, void* ws,
-                                       size_t ws_bytes, catekv_stream stream) {
+// Scoring and chunk selection, then either the gather into step_cache (catekv_retrieve_compact) or, with
+// step_cache == NULL, just the index lists and kept lengths for catekv_decode_attn_indexed (catekv_retrieve_select).
+static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t chunk_size, const void* q,
+                         int32_t Hq, const uint8_t* retrieval_mask, int32_t budget, int32_t sink, int32_t local,
+                         catekv_cache* step_cache, int32_t* idx_out, int64_t idx_stride, int32_t* sel_len, void* ws,
+                         size_t ws_bytes, catekv_stream stream) {
   int rc = check_cache_r(cache);
   if (rc) return rc;
-  rc = check_cache_r(step_cache);
-  if (rc) return rc;
+  if (step_cache) {
+    rc = check_cache_r(step_cache);
+    if (rc) return rc;
+    if (step_cache->B != cache->B || step_cache->Hkv != cache->Hkv) return CATEKV_ERR_INVALID_ARG;
+  } else if (!idx_out || !sel_len) {
+    return CATEKV_ERR_INVALID_ARG;
+  }
   if (!meta || !q || !retrieval_mask || !ws) return CATEKV_ERR_INVALID_ARG;
   if (!chunk_size_ok(chunk_size)) return CATEKV_ERR_UNSUPPORTED;
-  if (step_cache->B != cache->B || step_cache->Hkv != cache->Hkv) return CATEKV_ERR_INVALID_ARG;
   if (Hq <= 0 || Hq % cache->Hkv || budget < 0 || sink < 0 || local < 0) return CATEKV_ERR_INVALID_ARG;
   const int G = Hq / cache->Hkv;
   if (G > kMaxG) return CATEKV_ERR_UNSUPPORTED;
@@ -325,9 +331,9 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
     if (cache->seg_len[s] < 0 || cache->seg_len[s] > cache->seg_cap[s]) return CATEKV_ERR_INVALID_ARG;
     max_len = cache->seg_len[s] > max_len ? cache->seg_len[s] : max_len;
     max_cap = cache->seg_cap[s] > max_cap ? cache->seg_cap[s] : max_cap;
-    max_step_cap = step_cache->seg_cap[s] > max_step_cap ? step_cache->seg_cap[s] : max_step_cap;
+    if (step_cache) max_step_cap = step_cache->seg_cap[s] > max_step_cap ? step_cache->seg_cap[s] : max_step_cap;
   }
-  if (idx_out && idx_stride < max_len) return CATEKV_ERR_INVALID_ARG;
+  if (step_cache && idx_out && idx_stride < max_len) return CATEKV_ERR_INVALID_ARG;
   const RetWs W = ret_ws_layout(n_segs, max_cap);
   if (ws_bytes < W.bytes) return CATEKV_ERR_WORKSPACE;
 
@@ -341,7 +347,8 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
   const int S2 = rp.sink2;
   for (int s = 0; s < n_segs; ++s) {
     const SelSeg d = retrieval_decide(cache->seg_len[s], retrieval_mask[s] != 0, rp);
-    if (d.len_ub > step_cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+    if (step_cache && d.len_ub > step_cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+    if (!step_cache && !d.keep_all && d.len_ub > idx_stride) return CATEKV_ERR_INVALID_ARG;  // its index list must fit
     if (retrieval_mask[s]) sa.mask.w[s >> 5] |= 1u << (s & 31);
   }
   const int max_pool = max_cap / cs;  // bound of the candidate chunks of a segment
@@ -374,20 +381,22 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
     retrieval_score_kernel<<<dim3(gx, (unsigned)n_segs), kRsThreads, kRsSmem, st>>>(sa);
     CATEKV_CUDA_TRY(cudaGetLastError());
   }
-  TopkArgs ta;
+  TopkArgs ta = {};
   ta.segs = d_segs;
   ta.C = P;
   ta.P = P;
   ta.c_stride = W.p_stride;
-  ta.idx = (int32_t*)(w8 + W.off_idx);
-  ta.idx_stride = W.idx_stride;
-  ta.seg_len_dev = step_cache->seg_len_dev;
+  ta.idx = step_cache ? (int32_t*)(w8 + W.off_idx) : idx_out;
+  ta.idx_stride = step_cache ? W.idx_stride : idx_stride;
+  ta.seg_len_dev = step_cache ? step_cache->seg_len_dev : sel_len;
+  ta.mark_keep_all = step_cache ? 0 : 1;  // select only: a segment that keeps all rows gets the length -1
   ta.sink = S2;
   ta.L_obs = 0;
   ta.pool_mode = kPoolPrescored;
   ta.pool_param = cs;
   rc = launch_topk(ta, n_segs, max_pool, st);
   if (rc) return rc;
+  if (!step_cache) return CATEKV_OK;
   GatherArgs ga;
   ga.segs = d_segs;
   ga.idx = ta.idx;
@@ -408,5 +417,39 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
   rc = launch_gather(ga, max_step_cap, n_segs, st);
   if (rc) return rc;
   for (int s = 0; s < n_segs; ++s) step_cache->seg_len[s] = retrieval_decide(cache->seg_len[s], retrieval_mask[s] != 0, rp).len_ub;
+  return CATEKV_OK;
+}
+
+extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* meta, int32_t chunk_size, const void* q,
+                                       int32_t Hq, const uint8_t* retrieval_mask, int32_t budget, int32_t sink, int32_t local,
+                                       catekv_cache* step_cache, int32_t* idx_out, int64_t idx_stride, void* ws,
+                                       size_t ws_bytes, catekv_stream stream) {
+  if (!step_cache) return CATEKV_ERR_INVALID_ARG;
+  return retrieve_impl(cache, meta, chunk_size, q, Hq, retrieval_mask, budget, sink, local, step_cache, idx_out, idx_stride,
+                       nullptr, ws, ws_bytes, stream);
+}
+
+extern "C" int catekv_retrieve_select(const catekv_cache* cache, const void* meta, int32_t chunk_size, const void* q,
+                                      int32_t Hq, const uint8_t* retrieval_mask, int32_t budget, int32_t sink, int32_t local,
+                                      int32_t* idx, int64_t idx_stride, int32_t* sel_len, void* ws, size_t ws_bytes,
+                                      catekv_stream stream) {
+  return retrieve_impl(cache, meta, chunk_size, q, Hq, retrieval_mask, budget, sink, local, nullptr, idx, idx_stride, sel_len,
+                       ws, ws_bytes, stream);
+}
+
+extern "C" int catekv_retrieve_lengths(const catekv_cache* cache, int32_t chunk_size, const uint8_t* retrieval_mask,
+                                       int32_t budget, int32_t sink, int32_t local, int32_t* lens_out) {
+  int rc = check_cache_r(cache);
+  if (rc) return rc;
+  if (!retrieval_mask || !lens_out || budget < 0 || sink < 0 || local < 0) return CATEKV_ERR_INVALID_ARG;
+  if (!chunk_size_ok(chunk_size)) return CATEKV_ERR_UNSUPPORTED;
+  RetParams rp;
+  rp.cs = chunk_size;
+  rp.budget = budget;
+  rp.sink2 = (sink + chunk_size - 1) / chunk_size * chunk_size;
+  rp.local = local;
+  rp.Hkv = cache->Hkv;
+  const int n_segs = cache->B * cache->Hkv;
+  for (int s = 0; s < n_segs; ++s) lens_out[s] = retrieval_decide(cache->seg_len[s], retrieval_mask[s] != 0, rp).len_ub;
   return CATEKV_OK;
 }

@@ -70,7 +70,10 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
   const int seg = blockIdx.x / CL;
   const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
   const SelSeg s = a.segs[seg];
-  if (s.keep_all) return;  // the whole cluster leaves
+  if (s.keep_all) {  // the whole cluster leaves
+    if (a.mark_keep_all && rank == 0 && threadIdx.x == 0) a.seg_len_dev[seg] = -1;
+    return;
+  }
   TOPK_STAMP(0);
   __shared__ unsigned int hist[256];
   __shared__ unsigned int hsum[256];
@@ -587,7 +590,7 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
     int rc = score_launch(sa, kScoreColsum, st);
     if (rc) return rc;
   }
-  TopkArgs ta;
+  TopkArgs ta = {};
   ta.segs = d_segs;
   ta.C = (const float*)(w8 + W.off_C);
   ta.P = (float*)(w8 + W.off_P);

@@ -28,6 +28,7 @@ struct TopkArgs {
   int64_t idx_stride;
   int32_t* seg_len_dev;
   int32_t sink, L_obs, pool_mode, pool_param;  // the always-kept tail of a segment is [cand_end, n)
+  int32_t mark_keep_all;  // 1: a keep_all segment gets seg_len_dev = -1 ("the whole list") instead of being skipped
   int32_t stage_entries;  // set by launch_topk: pooled entries per CTA that the dynamic shared memory holds
 };
 

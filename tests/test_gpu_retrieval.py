@@ -156,7 +156,8 @@ def test_retrieval_finds_loud_keys_and_budget_covers_all(ck):
     assert e.value.code == ck.ERR_CAPACITY
 
 
-def test_retrieval_step_replayed_as_cuda_graph(ck):
+@pytest.mark.parametrize("indexed", [False, True])
+def test_retrieval_step_replayed_as_cuda_graph(ck, indexed):
     """append + metadata append + retrieve + attention captured once and replayed while the lists grow: the kept
     lengths move within a chunk under a decode plan that was built once, and every step matches the oracle."""
     cs, G, B, Hkv = 8, 4, 2, 2
@@ -177,15 +178,25 @@ def test_retrieval_step_replayed_as_cuda_graph(ck):
     idx = torch.full((B * Hkv, max(lens) + steps + 2), -1, dtype=torch.int32, device="cuda")
     ws = torch.empty(ck._lib.catekv_retrieve_workspace_bytes(B, Hkv, int(cache.seg_cap.max())), dtype=torch.uint8,
                      device="cuda")
-    ck.catekv_retrieve_compact(cache, meta, cs, q.zero_(), mask, budget, sink, local, step_cache, ws=ws)
-    plan = ck.DecodePlan(step_cache, 7)
-    ck.catekv_decode_plan(step_cache, plan)  # once, from the lengths of this first fill
+    sel = torch.full((B * Hkv,), -99, dtype=torch.int32, device="cuda")
+    if indexed:
+        view = ck.CacheView(cache, ck.catekv_retrieve_lengths(cache, cs, mask, budget, sink, local))
+        plan = ck.DecodePlan(view, 7)
+        ck.catekv_decode_plan(view, plan)  # once, from the lengths before the first step
+    else:
+        ck.catekv_retrieve_compact(cache, meta, cs, q.zero_(), mask, budget, sink, local, step_cache, ws=ws)
+        plan = ck.DecodePlan(step_cache, 7)
+        ck.catekv_decode_plan(step_cache, plan)  # once, from the lengths of this first fill
 
     def one_step():
         ck.catekv_append(cache, kn, vn)
         ck.catekv_retrieval_append(cache, cs, kn, meta)
-        ck.catekv_retrieve_compact(cache, meta, cs, q, mask, budget, sink, local, step_cache, idx_out=idx, ws=ws)
-        ck.catekv_decode_attn(step_cache, q, plan, out)
+        if indexed:
+            ck.catekv_retrieve_select(cache, meta, cs, q, mask, budget, sink, local, idx, sel, ws=ws)
+            ck.catekv_decode_attn_indexed(cache, idx, sel, q, plan, out)
+        else:
+            ck.catekv_retrieve_compact(cache, meta, cs, q, mask, budget, sink, local, step_cache, idx_out=idx, ws=ws)
+            ck.catekv_decode_attn(step_cache, q, plan, out)
 
     g = torch.cuda.CUDAGraph()
     side = torch.cuda.Stream()
@@ -206,12 +217,16 @@ def test_retrieval_step_replayed_as_cuda_graph(ck):
         torch.cuda.synchronize()
         oc.append(synth.bits(kn), synth.bits(vn))
         qb = orc.bf16_to_f64(synth.bits(q))
-        got_len = step_cache.seg_len_dev.cpu().tolist()
+        got_len = sel.cpu().tolist() if indexed else step_cache.seg_len_dev.cpu().tolist()
         got_idx = idx.cpu().numpy()
         soc = orc.HybridCache(B, Hkv, 128)
         for s in range(B * Hkv):
             L = lens[s] + t + 1
-            got = got_idx[s, :got_len[s]].astype(np.int64)
+            if indexed and not (mask[s] and L > budget):
+                assert got_len[s] == -1
+                got = np.arange(L)
+            else:
+                got = got_idx[s, :got_len[s]].astype(np.int64)
             if mask[s] and L > budget:
                 kmax, kmin = orc.retrieval_metadata(oc.k_rows[s], cs)
                 b, h = divmod(s, Hkv)
@@ -226,3 +241,68 @@ def test_retrieval_step_replayed_as_cuda_graph(ck):
         H.check_attention(out, None, None, ref, None, f"graph step {t}")
     assert len(seen_lens) > 1  # the kept length did move under the plan
     assert list(cache.seg_len) == [L + steps for L in lens] == cache.seg_len_dev.cpu().tolist()
+
+
+@pytest.mark.parametrize("cs,G,num_ctas", [(8, 4, 12), (8, 7, 296), (16, 1, 3), (1, 2, 12)])
+def test_retrieve_select_and_indexed_attention(ck, cs, G, num_ctas):
+    """Retrieval without the copy: index lists + attention in place == oracle == the gather path bit for bit."""
+    lens = [700, 64, 2049, 5, 1300, 0]
+    B, Hkv = 2, 3
+    oc = H.random_cache(B, Hkv, lens, seed=90 + cs)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=8)
+    meta = ck.catekv_retrieval_meta(cache, cs)
+    ck.catekv_retrieval_build(cache, cs, meta)
+    q = synth.randn_bf16((B, Hkv * G, 128), "cuda", 91, "q", cs)
+    qb = orc.bf16_to_f64(synth.bits(q))
+    mask = np.array([1, 1, 1, 1, 0, 1], dtype=np.uint8)
+    budget, sink, local = 256, 4, 32
+    want = ck.catekv_retrieve_lengths(cache, cs, mask, budget, sink, local)
+    for s, L in enumerate(lens):
+        if mask[s] and L > budget:
+            assert want[s] == len(orc.retrieve_indices(np.zeros((L + cs - 1) // cs), L, sink, local, budget, cs))
+        else:
+            assert want[s] == L
+    idx = torch.full((B * Hkv, int(want.max()) + 3), -7, dtype=torch.int32, device="cuda")
+    sel = torch.full((B * Hkv,), -99, dtype=torch.int32, device="cuda")
+    ck.catekv_retrieve_select(cache, meta, cs, q, mask, budget, sink, local, idx, sel)
+    torch.cuda.synchronize()
+    got_sel = sel.cpu().tolist()
+    soc = orc.HybridCache(B, Hkv, 128)
+    for s, L in enumerate(lens):
+        if mask[s] and L > budget:
+            assert got_sel[s] == want[s]
+            got = idx[s, :want[s]].cpu().numpy().astype(np.int64)
+            kmax, kmin = orc.retrieval_metadata(oc.k_rows[s], cs)
+            b, h = divmod(s, Hkv)
+            scores = orc.retrieval_scores(qb[b, h * G:(h + 1) * G], kmax, kmin)
+            _check_selection(got, scores, L, sink, local, budget, cs, f"seg {s}")
+            assert torch.all(idx[s, want[s]:] == -7)  # nothing written behind the list
+        else:
+            assert got_sel[s] == -1 and torch.all(idx[s] == -7)
+            got = np.arange(L)
+        soc.k_rows.append(oc.k_rows[s][got])
+        soc.v_rows.append(oc.v_rows[s][got])
+    view = ck.CacheView(cache, want)
+    plan = ck.DecodePlan(view, num_ctas)
+    ck.catekv_decode_plan(view, plan)
+    out = torch.full((B, Hkv * G, 128), float("nan"), dtype=torch.float32, device="cuda")
+    lse = torch.full((B, Hkv * G), float("nan"), dtype=torch.float32, device="cuda")
+    ck.catekv_decode_attn_indexed(cache, idx, sel, q, plan, out, lse)
+    o16 = torch.full((B, Hkv * G, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ck.catekv_decode_attn_indexed(cache, idx, sel, q, plan, o16)
+    ref, ref_lse = orc.decode_attention(soc, synth.bits(q))
+    H.check_attention(out, o16, lse, ref, ref_lse, f"indexed cs={cs} G={G}")
+    # the gather path attends to the same rows in the same order under the same split: identical bits
+    step = ck.Cache(B, Hkv, want, 0, "cuda")
+    ck.catekv_retrieve_compact(cache, meta, cs, q, mask, budget, sink, local, step)
+    plan2 = ck.DecodePlan(step, num_ctas)
+    ck.catekv_decode_plan(step, plan2)
+    out2 = torch.empty_like(out)
+    lse2 = torch.empty_like(lse)
+    ck.catekv_decode_attn(step, q, plan2, out2, lse2)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2) and torch.equal(lse, lse2)
+    # an index row that is too short for a kept list is refused before anything runs
+    with pytest.raises(ck.CatekvError) as e:
+        ck.catekv_retrieve_select(cache, meta, cs, q, mask, budget, sink, local, idx[:, :100].contiguous(), sel)
+    assert e.value.code == ck.ERR_INVALID_ARG
