@@ -459,6 +459,31 @@ def oracle_sample_rate(w, target_s=15.0, seed_rows=200_000):
     return rows_done / t_done, desc, t_done
 
 
+def oracle_extra_timings(w):
+    """The oracle at one thread (a 3 s sample of decode_attention) and one KV head's prefill-end selection
+    (oracle.select_indices on the workload's shape: window scores, pooling, top-k) at all cores."""
+    from oracle import catekv_oracle as orc
+    from workloads import synth
+    out = {}
+    try:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            rate1, _, _ = oracle_sample_rate(w, target_s=3.0)
+        out["rows_per_s_1thread"] = rate1
+    except Exception as e:  # threadpoolctl missing: report the reason, keep the line
+        out["rows_per_s_1thread"] = None
+        out["note_1thread"] = repr(e)
+    n = min(w.n, 65536)
+    qwin = synth.bits(synth.randn_bf16((w.G, w.L_obs, w.d), "cpu", w.seed, "osq"))
+    k = synth.bits(synth.randn_bf16((n, w.d), "cpu", w.seed, "osk"))
+    t0 = time.perf_counter()
+    C = orc.window_scores(qwin, k, w.L_obs)
+    orc.select_indices(C, n, w.sink, w.local, w.budget, w.pool_mode, w.pool_param)
+    out["select_one_head_s"] = time.perf_counter() - t0
+    out["select_shape"] = f"{w.G} x {w.L_obs} window queries, {n} keys, budget {w.budget}"
+    return out
+
+
 def workload_rows_per_layer_step(w):
     """Expected kept rows of one layer-step (mean over the seeded masks of all layers)."""
     from workloads import synth
@@ -639,6 +664,7 @@ def main():
         line["cpu_baseline"] = {"value": w.B / (w.layers * rows / rate), "unit": UNIT, "cores": oracle_threads(),
                                 "kind": "oracle", "sample": desc + f" ({spent:.1f} s, {rate:.3e} rows/s), "
                                 "extrapolated by rows to the full step"}
+        line["cpu_baseline"].update(oracle_extra_timings(w))
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

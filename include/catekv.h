@@ -189,6 +189,17 @@ int catekv_append(catekv_cache* cache, const void* k_new, const void* v_new, cat
 int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens);
 
 /*
+ * Growth beyond the capacity a cache was laid out with (Section 4.4.3 keeps generating for as long as the
+ * request runs; the paper sizes its caches up front and has no counterpart to this call).  The caller lays out
+ * a second cache with larger capacities (catekv_cache_layout with a larger max_new), and this call copies the
+ * seg_len valid rows of every segment of `src` to the start of the same segment of `dst` and sets dst's lengths
+ * (device and host mirror).  src is left untouched; plans and retrieval metadata are per cache and must be
+ * rebuilt for dst.  CATEKV_ERR_CAPACITY (nothing launched) if a segment of src does not fit its segment of dst;
+ * CATEKV_ERR_INVALID_ARG if the two caches differ in B or Hkv or share a pool.
+ */
+int catekv_cache_regrow(const catekv_cache* src, catekv_cache* dst, catekv_stream stream);
+
+/*
  * Work-balanced split-KV schedule for catekv_decode_attn.
  *
  * The rows of all segments, laid end to end, are cut into num_ctas near-equal

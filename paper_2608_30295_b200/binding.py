@@ -68,6 +68,7 @@ def _load():
         "catekv_select_compact": (C.c_int, [C.POINTER(SelectParams), C.POINTER(CacheStruct), vp, i64, vp, sz, vp]),
         "catekv_append": (C.c_int, [C.POINTER(CacheStruct), vp, vp, vp]),
         "catekv_cache_advance": (C.c_int, [C.POINTER(CacheStruct), i32]),
+        "catekv_cache_regrow": (C.c_int, [C.POINTER(CacheStruct), C.POINTER(CacheStruct), vp]),
         "catekv_decode_num_ctas": (C.c_int, []),
         "catekv_decode_plan_bytes": (sz, [i32, i32, i32]),
         "catekv_decode_workspace_bytes": (sz, [i32, i32, i32]),
@@ -167,6 +168,13 @@ def catekv_append(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor):
 def catekv_cache_advance(cache: Cache, n_tokens: int = 1):
     """Host mirror only: account for appends that a replayed CUDA graph performs on the device."""
     _check(_lib.catekv_cache_advance(C.byref(cache.struct), n_tokens), "catekv_cache_advance")
+
+
+def catekv_cache_regrow(src: Cache, max_new: int) -> Cache:
+    """A new cache with room for max_new more rows per segment, holding src's rows (device copy)."""
+    dst = Cache(src.B, src.Hkv, src.seg_len, max_new, src.device, src.d)
+    _check(_lib.catekv_cache_regrow(C.byref(src.struct), C.byref(dst.struct), _stream()), "catekv_cache_regrow")
+    return dst
 
 
 def catekv_decode_num_ctas() -> int:

@@ -670,6 +670,52 @@ extern "C" int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens) {
   return CATEKV_OK;
 }
 
+// Growth: every segment's valid rows move to the same segment of a cache with larger capacities.  One warp per
+// row (lanes 0-15 the K row, 16-31 the V row); block 0 of a segment records its length.
+namespace catekv {
+constexpr int kRegrowRowsPerBlock = 64;
+__global__ void __launch_bounds__(256) regrow_kernel(const uint8_t* sk, const uint8_t* sv, const int32_t* s_off,
+                                                     const int32_t* s_len, uint8_t* dk, uint8_t* dv, const int32_t* d_off,
+                                                     int32_t* d_len) {
+  const int seg = blockIdx.y;
+  const int len = s_len[seg];
+  if (blockIdx.x == 0 && threadIdx.x == 0) d_len[seg] = len;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint8_t* src = (lane < 16 ? sk : sv) + (int64_t)s_off[seg] * kRowBytes + (lane & 15) * 16;
+  uint8_t* dst = (lane < 16 ? dk : dv) + (int64_t)d_off[seg] * kRowBytes + (lane & 15) * 16;
+  const int r0 = blockIdx.x * kRegrowRowsPerBlock;
+#pragma unroll 4
+  for (int i = warp; i < kRegrowRowsPerBlock; i += 8) {
+    const int r = r0 + i;
+    if (r >= len) break;
+    *reinterpret_cast<uint4*>(dst + (int64_t)r * kRowBytes) = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)r * kRowBytes));
+  }
+}
+}  // namespace catekv
+
+extern "C" int catekv_cache_regrow(const catekv_cache* src, catekv_cache* dst, catekv_stream stream) {
+  int rc = check_cache(src);
+  if (rc) return rc;
+  rc = check_cache(dst);
+  if (rc) return rc;
+  if (src->B != dst->B || src->Hkv != dst->Hkv) return CATEKV_ERR_INVALID_ARG;
+  if (src->k_pool == dst->k_pool || src->v_pool == dst->v_pool) return CATEKV_ERR_INVALID_ARG;
+  const int n = src->B * src->Hkv;
+  int max_len = 0;
+  for (int s = 0; s < n; ++s) {
+    if (src->seg_len[s] < 0 || src->seg_len[s] > src->seg_cap[s]) return CATEKV_ERR_INVALID_ARG;
+    if (src->seg_len[s] > dst->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+    max_len = src->seg_len[s] > max_len ? src->seg_len[s] : max_len;
+  }
+  const int gx = max_len > 0 ? (max_len + kRegrowRowsPerBlock - 1) / kRegrowRowsPerBlock : 1;
+  regrow_kernel<<<dim3(gx, n), 256, 0, (cudaStream_t)stream>>>((const uint8_t*)src->k_pool, (const uint8_t*)src->v_pool,
+                                                               src->seg_off_dev, src->seg_len_dev, (uint8_t*)dst->k_pool,
+                                                               (uint8_t*)dst->v_pool, dst->seg_off_dev, dst->seg_len_dev);
+  CATEKV_CUDA_TRY(cudaGetLastError());
+  for (int s = 0; s < n; ++s) dst->seg_len[s] = src->seg_len[s];
+  return CATEKV_OK;
+}
+
 extern "C" int catekv_decode_num_ctas(void) {
   int dev = 0, sms = 0, per_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return CATEKV_ERR_CUDA;

@@ -358,8 +358,13 @@ static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t ch
   SelSeg* d_segs = (SelSeg*)(w8 + W.off_segs);
   float* P = (float*)(w8 + W.off_P);
   {
-    // a few 64-chunk tiles per CTA, enough CTAs to fill the machine
-    int gx = (max_pool + 8 * kRsTile - 1) / (8 * kRsTile);
+    // CTAs per segment: about two waves of resident CTAs (2 per SM) over the segments that retrieve, so that a
+    // CTA streams many 64-chunk tiles through its pipeline; never more CTAs than tiles
+    int n_ret = 0;
+    for (int s = 0; s < n_segs; ++s) n_ret += retrieval_mask[s] != 0;
+    const int tiles = (max_pool + kRsTile - 1) / kRsTile;
+    int gx = n_ret > 0 ? (4 * 148 + n_ret - 1) / n_ret : 1;
+    if (gx > tiles) gx = tiles;
     if (gx > 64) gx = 64;
     if (gx < 1) gx = 1;
     static bool attr_set[64] = {};

@@ -154,6 +154,40 @@ def test_decode_with_stale_plan_after_segments_shrank(ck, num_ctas):
     H.check_attention(o32, None, lse, ref, ref_lse, "restored")
 
 
+def test_cache_regrow_lets_full_segments_keep_growing(ck):
+    lens = [100, 128, 1, 0, 300, 64, 17, 255]
+    oc = H.random_cache(2, 4, lens, seed=29)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=0)  # capacities round_up(len, 128): some are full
+    kn = synth.randn_bf16((2, 4, 128), "cuda", 29, "kn")
+    vn = synth.randn_bf16((2, 4, 128), "cuda", 29, "vn")
+    with pytest.raises(ck.CatekvError) as e:
+        ck.catekv_append(cache, kn, vn)
+    assert e.value.code == ck.ERR_CAPACITY
+    big = ck.catekv_cache_regrow(cache, max_new=40)
+    torch.cuda.synchronize()
+    assert list(big.seg_len) == lens == big.seg_len_dev.cpu().tolist()
+    for i, L in enumerate(lens):
+        o = int(big.seg_off[i])
+        assert np.array_equal(synth.bits(big.k_pool[o:o + L]), oc.k_rows[i])
+        assert np.array_equal(synth.bits(big.v_pool[o:o + L]), oc.v_rows[i])
+    plan = ck.DecodePlan(big, 11)
+    ck.catekv_decode_plan(big, plan)
+    out = torch.empty((2, 16, 128), dtype=torch.float32, device="cuda")
+    for step in range(40):
+        kn = synth.randn_bf16((2, 4, 128), "cuda", 29, "kn", step)
+        vn = synth.randn_bf16((2, 4, 128), "cuda", 29, "vn", step)
+        q = synth.randn_bf16((2, 16, 128), "cuda", 29, "q", step)
+        ck.catekv_append_decode_attn(big, kn, vn, q, plan, out)
+        oc.append(synth.bits(kn), synth.bits(vn))
+    ref, _ = orc.decode_attention(oc, synth.bits(q))
+    H.check_attention(out, None, None, ref, None, "after regrow")
+    # a destination that is too small, or the cache itself, is refused
+    small = ck.Cache(2, 4, [8] * 8, 0, "cuda")
+    for dst, code in ((small, ck.ERR_CAPACITY), (big, ck.ERR_INVALID_ARG)):
+        rc = ck._lib.catekv_cache_regrow(ck.C.byref(big.struct), ck.C.byref(dst.struct), None)
+        assert rc == code
+
+
 def test_decode_is_deterministic(ck):
     oc = H.random_cache(2, 4, [700, 64, 1500, 3, 90, 400, 2000, 128], seed=17)
     q = synth.bits(synth.randn_bf16((2, 16, 128), "cpu", 17, "q"))
