@@ -616,11 +616,12 @@ def main():
         "us_per_layer_step": ms * 1e3 / n_layers,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src,
-                     # DRAM read+write bytes per launch: measured with ncu on the configs[2] small case (read
-                     # traffic = 1.0004 x algorithmic bytes, ~4 MB of writes; profiles/decode_partial_kernel_*.md)
-                     # and scaled by the kept rows: a launch of this size is beyond the capture size rule
-                     "traffic": bytes_per_layer * 1.0004 + 4.0e6,
-                     "traffic_source": "scaled from the ncu capture of the configs[2] small case",
+                     # DRAM read+write bytes per launch: one-pass ncu capture of this workload's own launches
+                     # (profiles/decode_partial_kernel_cfg3_traffic.md): reads = 1.00015 x algorithmic bytes,
+                     # about 1.25 MB of writes; the configs[2] small case gave the same ratio
+                     "traffic": bytes_per_layer * 1.00015 + 1.25e6,
+                     "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the configs[3] launches "
+                                       "(read = 1.00015 x algorithmic bytes), applied to this run's kept rows",
                      "kernel": "decode_partial_kernel", "bytes_per_launch": bytes_per_layer,
                      "us_per_launch": part_us, "us_per_launch_median": part_med_us,
                      "frac_of_8TBs": achieved / 8000.0, "combine_us": comb_us},
