@@ -518,6 +518,7 @@ struct CombineArgs {
 // barrier), then sums its eighth of the pieces with all of its loads in flight at once (a lane owns four
 // consecutive d, a piece is one 512-byte row per warp-load); the warps are summed in a fixed order.
 constexpr int kCombineWarps = 8;
+constexpr int kCombineUnroll = 16;
 __global__ void __launch_bounds__(kCombineWarps * 32) decode_combine_kernel(const CombineArgs a) {
   const int seg = blockIdx.x, hd = blockIdx.y;
   pdl_launch_dependents();
@@ -526,51 +527,69 @@ __global__ void __launch_bounds__(kCombineWarps * 32) decode_combine_kernel(cons
   if (si.n_pieces <= 1) return;  // written directly by the attention kernel
   __shared__ float4 s_acc[kCombineWarps][32];
   __shared__ float s_w[kCombineWarps];
+  __shared__ float s_m[kCombineWarps];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n = si.n_pieces;
   const float* lse = a.part_lse + (size_t)si.slot_begin * kMaxG + hd;
-  float M = -INFINITY;
-  for (int p = lane; p < n; p += 32) M = fmaxf(M, lse[(size_t)p * kMaxG]);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  // One trip to memory: a warp loads the values and the LSEs of its pieces together (16 pieces in flight: one round for up to 128 pieces) and merges
+  // them with a running maximum of its own; the 8 warps are then merged through shared memory.
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  float wsum = 0.f;
-  if (M > -INFINITY) {
+  float wsum = 0.f, mw = -INFINITY;
+  {
     const float* po = a.part_o + ((size_t)si.slot_begin * kMaxG + hd) * kD + lane * 4;
-    for (int p0 = warp; p0 < n; p0 += kCombineWarps * 8) {
-      float4 v[8];
-      float w[8];
+    for (int p0 = warp; p0 < n; p0 += kCombineWarps * kCombineUnroll) {
+      float4 v[kCombineUnroll];
+      float w[kCombineUnroll];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
+      for (int u = 0; u < kCombineUnroll; ++u) {
         const int p = p0 + u * kCombineWarps;
         const bool ok = p < n;
         v[u] = ok ? *reinterpret_cast<const float4*>(po + (size_t)p * (kMaxG * kD)) : make_float4(0.f, 0.f, 0.f, 0.f);
         w[u] = ok ? lse[(size_t)p * kMaxG] : -INFINITY;
       }
+      float mx = mw;
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const float e = exp2f(w[u] - M);
-        acc.x += e * v[u].x;
-        acc.y += e * v[u].y;
-        acc.z += e * v[u].z;
-        acc.w += e * v[u].w;
-        wsum += e;
+      for (int u = 0; u < kCombineUnroll; ++u) mx = fmaxf(mx, w[u]);
+      if (mx > -INFINITY) {
+        const float sc = exp2f(mw - mx);  // 0 on the first round (mw = -inf)
+        acc.x *= sc;
+        acc.y *= sc;
+        acc.z *= sc;
+        acc.w *= sc;
+        wsum *= sc;
+        mw = mx;
+#pragma unroll
+        for (int u = 0; u < kCombineUnroll; ++u) {
+          const float e = exp2f(w[u] - mx);  // an empty piece (LSE -inf) weighs 0
+          acc.x += e * v[u].x;
+          acc.y += e * v[u].y;
+          acc.z += e * v[u].z;
+          acc.w += e * v[u].w;
+          wsum += e;
+        }
       }
     }
   }
   s_acc[warp][lane] = acc;
-  if (lane == 0) s_w[warp] = wsum;
+  if (lane == 0) {
+    s_w[warp] = wsum;
+    s_m[warp] = mw;
+  }
   __syncthreads();
   if (warp == 0) {
+    float M = -INFINITY;
+#pragma unroll
+    for (int wv = 0; wv < kCombineWarps; ++wv) M = fmaxf(M, s_m[wv]);
     float W = 0.f;
     float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int wv = 0; wv < kCombineWarps; ++wv) {
-      W += s_w[wv];
-      r.x += s_acc[wv][lane].x;
-      r.y += s_acc[wv][lane].y;
-      r.z += s_acc[wv][lane].z;
-      r.w += s_acc[wv][lane].w;
+      const float f = s_m[wv] > -INFINITY ? exp2f(s_m[wv] - M) : 0.f;
+      W += f * s_w[wv];
+      r.x += f * s_acc[wv][lane].x;
+      r.y += f * s_acc[wv][lane].y;
+      r.z += f * s_acc[wv][lane].z;
+      r.w += f * s_acc[wv][lane].w;
     }
     const float inv = W > 0.f ? 1.f / W : 0.f;
     r.x *= inv;
