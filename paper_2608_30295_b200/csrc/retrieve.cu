@@ -50,6 +50,8 @@ __global__ void __launch_bounds__(128) meta_append_kernel(const int32_t* seg_off
                                                           uint8_t* meta, int cs, int n_segs) {
   const int seg = blockIdx.x * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
+  pdl_launch_dependents();
+  pdl_wait();  // the length and k_new come from earlier kernels of the stream
   if (seg >= n_segs) return;
   const int r = seg_len[seg] - 1;
   if (r < 0) return;
@@ -145,6 +147,8 @@ struct RetJobView {
 __global__ void __launch_bounds__(kRsThreads, 2) retrieval_score_kernel(const RetScoreArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int seg = blockIdx.y;
+  pdl_launch_dependents();
+  pdl_wait();  // lengths, metadata and queries come from earlier kernels of the stream
   SelSeg d = retrieval_decide(a.seg_len[seg], (a.mask.w[seg >> 5] >> (seg & 31)) & 1u, a.p);
   const bool scores = !d.keep_all && d.k_sel > 0;
   if (scores) d.job = seg;  // score row = segment index
@@ -290,9 +294,8 @@ extern "C" int catekv_retrieval_append(const catekv_cache* cache, int32_t chunk_
   if (!meta || !k_new) return CATEKV_ERR_INVALID_ARG;
   if (!chunk_size_ok(chunk_size)) return CATEKV_ERR_UNSUPPORTED;
   const int n_segs = cache->B * cache->Hkv;
-  meta_append_kernel<<<(n_segs + 3) / 4, 128, 0, (cudaStream_t)stream>>>(cache->seg_off_dev, cache->seg_len_dev,
-                                                                           (const uint8_t*)k_new, (uint8_t*)meta, chunk_size, n_segs);
-  CATEKV_CUDA_TRY(cudaGetLastError());
+  CATEKV_CUDA_TRY(launch_pdl(meta_append_kernel, dim3((n_segs + 3) / 4), dim3(128), 0, (cudaStream_t)stream,
+                             cache->seg_off_dev, cache->seg_len_dev, (const uint8_t*)k_new, (uint8_t*)meta, chunk_size, n_segs));
   return CATEKV_OK;
 }
 
@@ -358,12 +361,12 @@ static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t ch
   SelSeg* d_segs = (SelSeg*)(w8 + W.off_segs);
   float* P = (float*)(w8 + W.off_P);
   {
-    // CTAs per segment: about two waves of resident CTAs (2 per SM) over the segments that retrieve, so that a
-    // CTA streams many 64-chunk tiles through its pipeline; never more CTAs than tiles
+    // CTAs per segment: one wave of resident CTAs (2 per SM) over the segments that retrieve, so that a CTA
+    // streams many 64-chunk tiles through its pipeline and no partial wave trails; never more CTAs than tiles
     int n_ret = 0;
     for (int s = 0; s < n_segs; ++s) n_ret += retrieval_mask[s] != 0;
     const int tiles = (max_pool + kRsTile - 1) / kRsTile;
-    int gx = n_ret > 0 ? (4 * 148 + n_ret - 1) / n_ret : 1;
+    int gx = n_ret > 0 ? (2 * 148) / n_ret : 1;
     if (gx > tiles) gx = tiles;
     if (gx > 64) gx = 64;
     if (gx < 1) gx = 1;
@@ -383,8 +386,7 @@ static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t ch
     sa.P = P;
     sa.p_stride = W.p_stride;
     sa.segs = d_segs;
-    retrieval_score_kernel<<<dim3(gx, (unsigned)n_segs), kRsThreads, kRsSmem, st>>>(sa);
-    CATEKV_CUDA_TRY(cudaGetLastError());
+    CATEKV_CUDA_TRY(launch_pdl(retrieval_score_kernel, dim3(gx, (unsigned)n_segs), dim3(kRsThreads), kRsSmem, st, sa));
   }
   TopkArgs ta = {};
   ta.segs = d_segs;

@@ -69,6 +69,8 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
   cg::cluster_group cluster = cg::this_cluster();
   const int seg = blockIdx.x / CL;
   const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
+  pdl_launch_dependents();
+  pdl_wait();  // the decisions and the scores come from earlier kernels of the stream
   const SelSeg s = a.segs[seg];
   if (s.keep_all) {  // the whole cluster leaves
     if (a.mark_keep_all && rank == 0 && threadIdx.x == 0) a.seg_len_dev[seg] = -1;
@@ -403,8 +405,7 @@ int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, cudaStream_t strea
   a.stage_entries = share <= kTopkStageMax ? share : 0;  // longer shares are read from global memory
   const size_t smem = (size_t)(a.stage_entries + a.stage_entries / 32 + 1) * 4;
   if (CL == 1) {
-    topk_kernel<1><<<n_segs, kTopkThreads, smem, stream>>>(a);
-    CATEKV_CUDA_TRY(cudaGetLastError());
+    CATEKV_CUDA_TRY(launch_pdl(topk_kernel<1>, dim3(n_segs), dim3(kTopkThreads), smem, stream, a));
     return CATEKV_OK;
   }
   // long lists: a cluster of 8 CTAs per segment
@@ -413,13 +414,15 @@ int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, cudaStream_t strea
   cfg.blockDim = dim3(kTopkThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 8;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   CATEKV_CUDA_TRY(cudaLaunchKernelEx(&cfg, topk_kernel<8>, a));
   return CATEKV_OK;
 }
