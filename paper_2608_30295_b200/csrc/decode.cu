@@ -231,6 +231,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
 
   // ---- producer
   int p_item = item_begin, p_tile = 0, p_seq = 0;
+  int ix[(kTile * 16) / kDecodeThreads];  // indexed variant: see load_idx
   auto issue_tile = [&]() {  // tile p_tile of the producer's item into stage p_seq % kStages
     const uint32_t sb = s_stage + (p_seq % kStages) * kStageBytes;
     int start, rows_left;
@@ -243,8 +244,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       const int r = id >> 4, c = id & 15;
       const int ok = r < rows_left ? 16 : 0;
       int64_t grow = ok ? row0 + r : 0;  // padding rows read nothing
-      if (kIndexed && pc.indexed && ok)
-        grow = (pc.row_base - pc.t0) + __ldg(a.idx + (int64_t)pc.seg * a.idx_stride + start + r);
+      if (kIndexed && pc.indexed && ok) grow = (pc.row_base - pc.t0) + ix[i];
       const int64_t goff = grow * kRowBytes + c * 16;
       const uint32_t so = tile_off(r, c);
       if (ok && r == new_r && pc.new_row >= 0) {  // only inside the tile's valid rows (never in a plan-time tile)
@@ -257,6 +257,20 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       } else {
         cp_async16(sb + so, a.k_pool + goff, ok);
         cp_async16(sb + kTile * kRowBytes + so, a.v_pool + goff, ok);
+      }
+    }
+  };
+  // indexed variant: the list entries of this thread's 8 rows of the producer's next tile, fetched one tile
+  // ahead (right after the previous tile was issued) so that their latency is off the issue path
+  auto load_idx = [&]() {
+    if (kIndexed && p_item < item_end && pc.indexed) {
+      int start, rows_left;
+      tile_rows(pc, p_tile, start, rows_left);
+      const int32_t* src = a.idx + (int64_t)pc.seg * a.idx_stride + start;
+#pragma unroll
+      for (int i = 0; i < (kTile * 16) / kDecodeThreads; ++i) {
+        const int r = (tid + i * kDecodeThreads) >> 4;
+        ix[i] = r < rows_left ? __ldg(src + r) : 0;
       }
     }
   };
@@ -274,6 +288,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       p_tile = 0;
       if (++p_item < item_end) pc = read_item<kIndexed>(a, p_item);
     }
+    load_idx();
   };
   auto issue = [&]() {  // one tile (with the item's queries if it is the item's first) = one commit group
     if (p_item < item_end) {
@@ -302,6 +317,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     p_tile = 0;
     if (++p_item < item_end) pc = read_item<kIndexed>(a, p_item);
   }
+  load_idx();
   for (int s = pre; s < kStages - 1; ++s) issue();
   if (pre == kStages - 1) cp_async_commit();  // the queries of the first item form a group of their own
 
