@@ -345,7 +345,7 @@ def time_head_cv(ck, dev):
 
 def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8, graph=True, gather=False):
     """Decode step with query-aware retrieval on the adaptive heads (budget rows per adaptive head, chunk size 8):
-    per layer catekv_append + catekv_retrieval_append + catekv_retrieve_select + catekv_decode_attn_indexed
+    per layer catekv_append_retrieval + catekv_retrieve_select + catekv_decode_attn_indexed
     (attention in place through the index lists), replayed as a CUDA graph of the step (graph=False: host
     launches).  gather=True: catekv_retrieve_compact into a per-step cache + catekv_decode_attn instead.
     Returns (us per layer-step, attended bytes per layer-step, metadata bytes per layer-step)."""
@@ -382,8 +382,7 @@ def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8, graph=Tru
 
     def step():
         for l, m in enumerate(model):
-            ck.catekv_append(m["cache"], kn[l], vn[l])
-            ck.catekv_retrieval_append(m["cache"], cs, kn[l], m["meta"])
+            ck.catekv_append_retrieval(m["cache"], kn[l], vn[l], cs, m["meta"])
             if gather:
                 ck.catekv_retrieve_compact(m["cache"], m["meta"], cs, q[l], m["rmask"], budget, w.sink, w.local,
                                            m["step"], ws=m["ws"])
@@ -658,8 +657,8 @@ def main():
         ru, ra, rm = time_retrieval(ck, w, dev)
         line["retrieval"] = {"us_per_layer_step": ru, "attended_bytes_per_layer_step": ra,
                              "metadata_bytes_per_layer_step": rm, "budget_rows": 1024, "chunk": 8,
-                             "note": "query-aware retrieval on the adaptive heads of the same workload: per layer append, metadata "
-                                     "append, catekv_retrieve_select, catekv_decode_attn_indexed; CUDA graph replay of the step"}
+                             "note": "query-aware retrieval on the adaptive heads of the same workload: per layer "
+                                     "catekv_append_retrieval, catekv_retrieve_select, catekv_decode_attn_indexed; CUDA graph replay of the step"}
         rate, desc, spent = oracle_sample_rate(w, target_s=15.0)
         rows = bytes_per_layer / ROW_BYTES
         line["cpu_baseline"] = {"value": w.B / (w.layers * rows / rate), "unit": UNIT, "cores": oracle_threads(),

@@ -298,6 +298,9 @@ size_t catekv_retrieval_meta_bytes(const catekv_cache* cache, int32_t chunk_size
 int catekv_retrieval_build(const catekv_cache* cache, int32_t chunk_size, void* meta, catekv_stream stream);
 int catekv_retrieval_append(const catekv_cache* cache, int32_t chunk_size, const void* k_new, void* meta,
                             catekv_stream stream);
+/* catekv_append and catekv_retrieval_append in one launch (same checks and errors as catekv_append). */
+int catekv_append_retrieval(catekv_cache* cache, const void* k_new, const void* v_new, int32_t chunk_size, void* meta,
+                            catekv_stream stream);
 size_t catekv_retrieve_workspace_bytes(int32_t B, int32_t Hkv, int32_t max_len);
 int catekv_retrieve_compact(const catekv_cache* cache, const void* meta, int32_t chunk_size, const void* q, int32_t Hq,
                             const uint8_t* retrieval_mask, int32_t budget, int32_t sink, int32_t local,

@@ -82,6 +82,7 @@ def _load():
         "catekv_retrieval_meta_bytes": (sz, [C.POINTER(CacheStruct), i32]),
         "catekv_retrieval_build": (C.c_int, [C.POINTER(CacheStruct), i32, vp, vp]),
         "catekv_retrieval_append": (C.c_int, [C.POINTER(CacheStruct), i32, vp, vp, vp]),
+        "catekv_append_retrieval": (C.c_int, [C.POINTER(CacheStruct), vp, vp, i32, vp, vp]),
         "catekv_retrieve_workspace_bytes": (sz, [i32, i32, i32]),
         "catekv_retrieve_compact": (C.c_int, [C.POINTER(CacheStruct), vp, i32, vp, i32, vp, i32, i32, i32,
                                               C.POINTER(CacheStruct), vp, i64, vp, sz, vp]),
@@ -291,6 +292,13 @@ def catekv_retrieve_compact(cache: Cache, meta: torch.Tensor, chunk_size: int, q
                                         _dev_ptr(idx_out), stride, ws.data_ptr(), ws.numel(), _stream()),
            "catekv_retrieve_compact")
     return ws
+
+
+def catekv_append_retrieval(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor, chunk_size: int,
+                            meta: torch.Tensor):
+    assert k_new.is_contiguous() and v_new.is_contiguous()
+    _check(_lib.catekv_append_retrieval(C.byref(cache.struct), k_new.data_ptr(), v_new.data_ptr(), chunk_size,
+                                        meta.data_ptr(), _stream()), "catekv_append_retrieval")
 
 
 def catekv_retrieve_lengths(cache: Cache, chunk_size: int, retrieval_mask, budget: int, sink: int, local: int):

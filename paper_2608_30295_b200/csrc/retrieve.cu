@@ -45,18 +45,9 @@ __global__ void __launch_bounds__(256) meta_build_kernel(const uint8_t* k_pool, 
   *reinterpret_cast<uint2*>(dst + kRowBytes) = make_uint2(pack_bf16(mn[0], mn[1]), pack_bf16(mn[2], mn[3]));
 }
 
-// After an append: fold the newest row (index len - 1) into its chunk.  One warp per segment.
-__global__ void __launch_bounds__(128) meta_append_kernel(const int32_t* seg_off, const int32_t* seg_len, const uint8_t* k_new,
-                                                          uint8_t* meta, int cs, int n_segs) {
-  const int seg = blockIdx.x * 4 + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  pdl_launch_dependents();
-  pdl_wait();  // the length and k_new come from earlier kernels of the stream
-  if (seg >= n_segs) return;
-  const int r = seg_len[seg] - 1;
-  if (r < 0) return;
-  const uint2 w = *reinterpret_cast<const uint2*>(k_new + (size_t)seg * kRowBytes + lane * 8);
-  uint8_t* dst = meta + ((int64_t)seg_off[seg] / cs + r / cs) * (2 * kRowBytes) + lane * 8;
+// Fold row r of a segment (its key given as this lane's 8 bytes, w) into the metadata of its chunk.
+__device__ __forceinline__ void meta_fold_row(uint8_t* meta, int64_t seg_row0, int r, int cs, int lane, uint2 w) {
+  uint8_t* dst = meta + (seg_row0 / cs + r / cs) * (2 * kRowBytes) + lane * 8;
   if (r % cs == 0) {
     *reinterpret_cast<uint2*>(dst) = w;
     *reinterpret_cast<uint2*>(dst + kRowBytes) = w;
@@ -70,7 +61,41 @@ __global__ void __launch_bounds__(128) meta_append_kernel(const int32_t* seg_off
   }
 }
 
-// ---- chunk scores ----------------------------------------------------------------------------
+// After an append: fold the newest row (index len - 1) into its chunk.  One warp per segment.
+__global__ void __launch_bounds__(128) meta_append_kernel(const int32_t* seg_off, const int32_t* seg_len, const uint8_t* k_new,
+                                                          uint8_t* meta, int cs, int n_segs) {
+  const int seg = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  pdl_launch_dependents();
+  pdl_wait();  // the length and k_new come from earlier kernels of the stream
+  if (seg >= n_segs) return;
+  const int r = seg_len[seg] - 1;
+  if (r < 0) return;
+  const uint2 w = *reinterpret_cast<const uint2*>(k_new + (size_t)seg * kRowBytes + lane * 8);
+  meta_fold_row(meta, seg_off[seg], r, cs, lane, w);
+}
+
+// The append and the metadata update in one launch.  One warp per segment: lanes 0-15 store the K row, lanes
+// 16-31 the V row (16 bytes each), all 32 fold the key into its chunk, lane 0 bumps the length.
+__global__ void __launch_bounds__(128) append_meta_kernel(uint8_t* k_pool, uint8_t* v_pool, const int32_t* seg_off,
+                                                          int32_t* seg_len, const uint8_t* k_new, const uint8_t* v_new,
+                                                          uint8_t* meta, int cs, int n_segs) {
+  const int seg = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  pdl_launch_dependents();
+  pdl_wait();
+  if (seg >= n_segs) return;
+  const int len = seg_len[seg];
+  const int64_t row0 = seg_off[seg];
+  const int c = lane & 15;
+  const uint8_t* src = (lane < 16 ? k_new : v_new) + (size_t)seg * kRowBytes + c * 16;
+  uint8_t* dst = (lane < 16 ? k_pool : v_pool) + (row0 + len) * kRowBytes + c * 16;
+  *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+  const uint2 w = *reinterpret_cast<const uint2*>(k_new + (size_t)seg * kRowBytes + lane * 8);
+  meta_fold_row(meta, row0, len, cs, lane, w);
+  __syncwarp();
+  if (lane == 0) seg_len[seg] = len + 1;
+}
 
 // Per-segment decisions (what to keep, how many chunks to select) are taken on the device from its own lengths,
 // by the scoring kernel itself: a step needs no host-to-device copy and can be captured in a CUDA graph.  The
@@ -296,6 +321,24 @@ extern "C" int catekv_retrieval_append(const catekv_cache* cache, int32_t chunk_
   const int n_segs = cache->B * cache->Hkv;
   CATEKV_CUDA_TRY(launch_pdl(meta_append_kernel, dim3((n_segs + 3) / 4), dim3(128), 0, (cudaStream_t)stream,
                              cache->seg_off_dev, cache->seg_len_dev, (const uint8_t*)k_new, (uint8_t*)meta, chunk_size, n_segs));
+  return CATEKV_OK;
+}
+
+extern "C" int catekv_append_retrieval(catekv_cache* cache, const void* k_new, const void* v_new, int32_t chunk_size,
+                                       void* meta, catekv_stream stream) {
+  int rc = check_cache_r(cache);
+  if (rc) return rc;
+  if (!meta || !k_new || !v_new) return CATEKV_ERR_INVALID_ARG;
+  if (!chunk_size_ok(chunk_size)) return CATEKV_ERR_UNSUPPORTED;
+  const int n_segs = cache->B * cache->Hkv;
+  for (int s = 0; s < n_segs; ++s) {
+    if (cache->seg_len[s] < 0) return CATEKV_ERR_INVALID_ARG;
+    if (cache->seg_len[s] + 1 > cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+  }
+  CATEKV_CUDA_TRY(launch_pdl(append_meta_kernel, dim3((n_segs + 3) / 4), dim3(128), 0, (cudaStream_t)stream,
+                             (uint8_t*)cache->k_pool, (uint8_t*)cache->v_pool, cache->seg_off_dev, cache->seg_len_dev,
+                             (const uint8_t*)k_new, (const uint8_t*)v_new, (uint8_t*)meta, chunk_size, n_segs));
+  for (int s = 0; s < n_segs; ++s) cache->seg_len[s] += 1;
   return CATEKV_OK;
 }
 

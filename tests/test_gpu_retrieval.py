@@ -102,7 +102,8 @@ def test_retrieval_matches_oracle(ck, cs, G):
     H.check_attention(out, None, lse, ref, ref_lse, f"cs={cs} G={G}")
 
 
-def test_retrieval_metadata_follows_appends(ck):
+@pytest.mark.parametrize("one_launch", [False, True])
+def test_retrieval_metadata_follows_appends(ck, one_launch):
     cs = 8
     lens = [100, 7, 0, 64]
     oc = H.random_cache(1, 4, lens, seed=75)
@@ -112,10 +113,18 @@ def test_retrieval_metadata_follows_appends(ck):
     for step in range(20):
         kn = synth.randn_bf16((1, 4, 128), "cuda", 75, "kn", step)
         vn = synth.randn_bf16((1, 4, 128), "cuda", 75, "vn", step)
-        ck.catekv_append(cache, kn, vn)
-        ck.catekv_retrieval_append(cache, cs, kn, meta)
+        if one_launch:
+            ck.catekv_append_retrieval(cache, kn, vn, cs, meta)
+        else:
+            ck.catekv_append(cache, kn, vn)
+            ck.catekv_retrieval_append(cache, cs, kn, meta)
         oc.append(synth.bits(kn), synth.bits(vn))
     torch.cuda.synchronize()
+    assert list(cache.seg_len) == [L + 20 for L in lens] == cache.seg_len_dev.cpu().tolist()
+    for s in range(4):
+        o, L = int(cache.seg_off[s]), lens[s] + 20
+        assert np.array_equal(synth.bits(cache.k_pool[o:o + L]), oc.k_rows[s])
+        assert np.array_equal(synth.bits(cache.v_pool[o:o + L]), oc.v_rows[s])
     for s in range(4):
         kmax, kmin = orc.retrieval_metadata(oc.k_rows[s], cs)
         gmax, gmin = _meta_of(ck, cache, meta, cs, s, kmax.shape[0])
@@ -189,8 +198,11 @@ def test_retrieval_step_replayed_as_cuda_graph(ck, indexed):
         ck.catekv_decode_plan(step_cache, plan)  # once, from the lengths of this first fill
 
     def one_step():
-        ck.catekv_append(cache, kn, vn)
-        ck.catekv_retrieval_append(cache, cs, kn, meta)
+        if indexed:  # the one-launch form of the two appends
+            ck.catekv_append_retrieval(cache, kn, vn, cs, meta)
+        else:
+            ck.catekv_append(cache, kn, vn)
+            ck.catekv_retrieval_append(cache, cs, kn, meta)
         if indexed:
             ck.catekv_retrieve_select(cache, meta, cs, q, mask, budget, sink, local, idx, sel, ws=ws)
             ck.catekv_decode_attn_indexed(cache, idx, sel, q, plan, out)
