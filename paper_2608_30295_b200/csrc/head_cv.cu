@@ -4,8 +4,12 @@
 
 #include <vector>
 
+#include <cooperative_groups.h>
+
 #include "radix.cuh"
 #include "score.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace catekv {
 
@@ -24,31 +28,124 @@ struct CvArgs {
 };
 
 constexpr int kCvThreads = 1024;
+constexpr int kCvCluster = 8;
 
-// One CTA per (sequence, KV head): Phi = alpha * percentile element (Eq. 2), C_j = #{i: A_ij >= Phi}
-// (Eq. 3), cv = std_pop(C) / mean(C) (Eq. 4) from exact integer sums.
+// One thread-block cluster of 8 CTAs per (sequence, KV head): Phi = alpha * percentile element (Eq. 2),
+// C_j = #{i: A_ij >= Phi} (Eq. 3), cv = std_pop(C) / mean(C) (Eq. 4) from exact integer sums.
+// The percentile element is found by a radix select on the bit patterns (entries are >= 0): every CTA owns a
+// contiguous share of the flat matrix; the bits above the highest bit in which the smallest and largest entry
+// differ are common, the rest is resolved 8 bits per pass with the CTAs' histograms summed through distributed
+// shared memory.  For the counts every CTA owns a range of columns; the sums meet in CTA 0.
 __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
-  const int seg = blockIdx.x;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int seg = blockIdx.x / kCvCluster;
+  const int rank = (int)cluster.block_rank();
   const CvSeg s = a.segs[seg];
   __shared__ unsigned int hist[256];
+  __shared__ unsigned int hsum[256];
   __shared__ unsigned int s_pair[2];
+  __shared__ unsigned int s_mm[2];
   __shared__ unsigned long long red[2][32];
+  __shared__ unsigned long long s_sums[2];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* A = a.A + (size_t)seg * a.seg_stride;
   const unsigned int* Ab = reinterpret_cast<const unsigned int*>(A);
   const int m = s.m;
   const int N = a.L_obs * m;
-  unsigned int thr, need_eq;
-  block_radix_select([&](int e) { return Ab[e]; }, N, (unsigned int)s.need, hist, s_pair, thr, need_eq);
-  const float phi = __uint_as_float(thr) * a.alpha;
+  const int per = ((N + kCvCluster - 1) / kCvCluster + 3) / 4 * 4;
+  const int lo = min(N, rank * per), hi = min(N, lo + per);
+
+  // ---- extremes of the bit patterns
+  unsigned int vmin = 0xffffffffu, vmax = 0u;
+  for (int c0 = lo + tid; c0 < hi; c0 += 4 * kCvThreads) {  // four loads in flight
+    unsigned int v[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = (c0 + e * kCvThreads < hi) ? Ab[c0 + e * kCvThreads] : 0u;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (c0 + e * kCvThreads < hi) {
+        vmin = min(vmin, v[e]);
+        vmax = max(vmax, v[e]);
+      }
+  }
+  if (tid == 0) {
+    s_mm[0] = 0xffffffffu;
+    s_mm[1] = 0u;
+  }
+  __syncthreads();
+  vmin = __reduce_min_sync(0xffffffffu, vmin);
+  vmax = __reduce_max_sync(0xffffffffu, vmax);
+  if (lane == 0) {
+    atomicMin(&s_mm[0], vmin);
+    atomicMax(&s_mm[1], vmax);
+  }
+  cluster.sync();
+  unsigned int gmin = 0xffffffffu, gmax = 0u;
+#pragma unroll
+  for (int r = 0; r < kCvCluster; ++r) {
+    gmin = min(gmin, *cluster.map_shared_rank(&s_mm[0], r));
+    gmax = max(gmax, *cluster.map_shared_rank(&s_mm[1], r));
+  }
+
+  // ---- radix select of the need-th largest entry
+  int nb = 32 - __clz(gmin ^ gmax);  // 0: all entries are equal
+  unsigned int prefix = nb >= 32 ? 0u : (gmax >> nb) << nb, need = (unsigned int)s.need;
+  while (nb > 0) {
+    const int wbits = min(8, nb);
+    const int shift = nb - wbits;
+    const unsigned int dmask = (1u << wbits) - 1u;
+    const unsigned int pmask = shift + wbits >= 32 ? 0u : (0xffffffffu << (shift + wbits));
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    for (int c0 = lo; c0 < hi; c0 += 4 * kCvThreads) {  // whole warps stay in the loop: the vote needs them
+      unsigned int v[4];
+      bool in[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int c = c0 + e * kCvThreads + tid;
+        in[e] = c < hi;
+        v[e] = in[e] ? Ab[c] : 0u;
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool hit = in[e] && (v[e] & pmask) == prefix;
+        // a warp whose lanes all fall in one bin adds once; otherwise every hit adds for itself
+        const unsigned int dgt = hit ? ((v[e] >> shift) & dmask) : 0x100u;
+        const unsigned int d0 = __shfl_sync(0xffffffffu, dgt, 0);
+        if (__all_sync(0xffffffffu, dgt == d0)) {
+          if (hit && lane == 0) atomicAdd(&hist[dgt], 32u);
+        } else if (hit) {
+          atomicAdd(&hist[dgt], 1u);
+        }
+      }
+    }
+    cluster.sync();  // all histograms complete
+    if (tid < 256) {
+      unsigned int t = 0;
+#pragma unroll
+      for (int r = 0; r < kCvCluster; ++r) t += *cluster.map_shared_rank(&hist[tid], r);
+      hsum[tid] = t;
+    }
+    __syncthreads();
+    if (tid < 32) radix_pick_digit(hsum, need, prefix, shift, s_pair);
+    cluster.sync();  // decision visible; the peers are done reading this CTA's histogram
+    prefix = s_pair[0];
+    need = s_pair[1];
+    nb = shift;
+  }
+  const float phi = __uint_as_float(prefix) * a.alpha;
+
+  // ---- column counts over this CTA's columns
+  const int cper = (m + kCvCluster - 1) / kCvCluster;
+  const int j_lo = min(m, rank * cper), j_hi = min(m, j_lo + cper);
   unsigned long long sum = 0, sum2 = 0;
-  for (int j = threadIdx.x; j < m; j += kCvThreads) {
+  for (int j = j_lo + tid; j < j_hi; j += kCvThreads) {
     unsigned int c = 0;
 #pragma unroll 8
     for (int i = 0; i < a.L_obs; ++i) c += A[(size_t)i * m + j] >= phi ? 1u : 0u;
     sum += c;
     sum2 += (unsigned long long)c * c;
   }
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     sum += __shfl_xor_sync(0xffffffffu, sum, o);
@@ -56,9 +153,19 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
   }
   if (lane == 0) { red[0][warp] = sum; red[1][warp] = sum2; }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (tid == 0) {
     unsigned long long S1 = 0, S2 = 0;
     for (int w = 0; w < kCvThreads / 32; ++w) { S1 += red[0][w]; S2 += red[1][w]; }
+    s_sums[0] = S1;
+    s_sums[1] = S2;
+  }
+  cluster.sync();
+  if (rank == 0 && tid == 0) {
+    unsigned long long S1 = 0, S2 = 0;
+    for (int r = 0; r < kCvCluster; ++r) {
+      S1 += *cluster.map_shared_rank(&s_sums[0], r);
+      S2 += *cluster.map_shared_rank(&s_sums[1], r);
+    }
     // std_pop / mean = sqrt(m * sum(C^2) - (sum C)^2) / sum C
     double cv = 0.0;
     if (S1 > 0) {
@@ -67,6 +174,7 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
     }
     a.cv_out[seg] = (float)cv;
   }
+  cluster.sync();  // no CTA leaves while CTA 0 may still read its sums
 }
 
 struct CvWs {
@@ -177,7 +285,17 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   ca.L_obs = L_obs;
   ca.alpha = alpha;
   ca.cv_out = cv_out;
-  cv_kernel<<<n_segs, kCvThreads, 0, st>>>(ca);
-  CATEKV_CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_segs * kCvCluster);
+  cfg.blockDim = dim3(kCvThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kCvCluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  CATEKV_CUDA_TRY(cudaLaunchKernelEx(&cfg, cv_kernel, ca));
   return CATEKV_OK;
 }
