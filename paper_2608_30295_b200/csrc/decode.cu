@@ -782,10 +782,13 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
   const int n_segs = cache->B * cache->Hkv;
   const PlanLayout L = plan_layout(n_segs, num_ctas);
   if (plan_bytes < L.bytes) return CATEKV_ERR_WORKSPACE;
-  int64_t total = 0;
+  // The CTA that owns the end of a segment also streams the rows appended since the plan was built, one more
+  // tile: every non-empty segment's end is charged one tile of rows, so that those CTAs get fewer plan-time rows.
+  int64_t total = 0, charged = 0;
   for (int s = 0; s < n_segs; ++s) {
     if (cache->seg_len[s] < 0 || cache->seg_len[s] > cache->seg_cap[s]) return CATEKV_ERR_INVALID_ARG;
     total += cache->seg_len[s];
+    charged += cache->seg_len[s] + (cache->seg_len[s] > 0 ? kTile : 0);
   }
   uint8_t* base = (uint8_t*)plan_host;
   memset(base, 0, L.bytes);
@@ -794,8 +797,8 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
   WorkItem* items = (WorkItem*)(base + L.off_items);
   SegInfo* segs = (SegInfo*)(base + L.off_seg);
 
-  // rows per CTA: an equal share of all rows, rounded up to the split alignment
-  int64_t quota = (total + num_ctas - 1) / num_ctas;
+  // rows per CTA: an equal share of all (charged) rows, rounded up to the split alignment
+  int64_t quota = (charged + num_ctas - 1) / num_ctas;
   quota = (quota + kSplitAlign - 1) / kSplitAlign * kSplitAlign;
   if (quota < kSplitAlign) quota = kSplitAlign;
 
@@ -837,11 +840,12 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
         ++seg;
         pos = 0;
         seg_first_item = n_items;
+        room -= kTile;  // the tile of appended rows
       }
     }
     ctas[c].item_end = n_items;
   }
-  if (seg != n_segs) return CATEKV_ERR_INVALID_ARG;  // cannot happen: quota * num_ctas >= total
+  if (seg != n_segs) return CATEKV_ERR_INVALID_ARG;  // cannot happen: quota * num_ctas >= the charged rows
   for (int c = 0; c < num_ctas; ++c)
     if (ctas[c].item_begin < ctas[c].item_end) ctas[c].first = items[ctas[c].item_begin];
   hdr->magic = kPlanMagic;

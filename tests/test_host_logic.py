@@ -117,14 +117,16 @@ def test_decode_plan_covers_every_row_once_and_balances(ck, lens, num_ctas):
         elif npieces > 1:
             assert [sl for (_, _, sl) in pieces[s]] == list(range(sb, sb + npieces))
     assert n_slots == sum(len(p) for p in pieces.values() if len(p) > 1)
-    # balance: no CTA gets more than an equal share rounded up to 16 rows
-    total = sum(lens)
-    quota = max(16, -(-(-(-total // num_ctas)) // 16) * 16)
+    # balance: every non-empty segment's end is charged one tile (64 rows: the tile of rows appended later);
+    # no CTA gets more than an equal share of the charged rows rounded up to 16 (a charge may overshoot it)
+    charged = sum(lens) + 64 * sum(1 for x in lens if x > 0)
+    quota = max(16, -(-(-(-charged // num_ctas)) // 16) * 16)
     for c in range(num_ctas):
-        rows = 0
+        rows = ends = 0
         for seg, t0, t1, _ in items[cta[c]:cta[c + 1]]:
             rows += (lens[seg] if t1 < 0 else t1) - t0
-        assert rows <= quota
+            ends += 1 if (t1 < 0 and lens[seg] > 0) else 0
+        assert rows <= quota and rows + 64 * ends <= quota + 64
 
 
 def test_append_capacity_is_checked_before_launch(ck):
