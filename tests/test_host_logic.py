@@ -117,16 +117,17 @@ def test_decode_plan_covers_every_row_once_and_balances(ck, lens, num_ctas):
         elif npieces > 1:
             assert [sl for (_, _, sl) in pieces[s]] == list(range(sb, sb + npieces))
     assert n_slots == sum(len(p) for p in pieces.values() if len(p) > 1)
-    # balance: every non-empty segment's end is charged one tile (64 rows: the tile of rows appended later);
+    # balance: every non-empty segment's end is charged 384 rows (the extra work of the CTA that owns it);
     # no CTA gets more than an equal share of the charged rows rounded up to 16 (a charge may overshoot it)
-    charged = sum(lens) + 64 * sum(1 for x in lens if x > 0)
+    charge = 384
+    charged = sum(lens) + charge * sum(1 for x in lens if x > 0)
     quota = max(16, -(-(-(-charged // num_ctas)) // 16) * 16)
     for c in range(num_ctas):
         rows = ends = 0
         for seg, t0, t1, _ in items[cta[c]:cta[c + 1]]:
             rows += (lens[seg] if t1 < 0 else t1) - t0
             ends += 1 if (t1 < 0 and lens[seg] > 0) else 0
-        assert rows <= quota and rows + 64 * ends <= quota + 64
+        assert rows <= quota and rows + charge * ends <= quota + charge
 
 
 def test_append_capacity_is_checked_before_launch(ck):
