@@ -112,7 +112,7 @@ struct DecodeArgs {
 
 constexpr int kStageBytes = 2 * kTile * kRowBytes;     // K tile + V tile
 constexpr int kQSlotBytes = kMaxG * kRowBytes;         // 8 query rows
-constexpr int kSegEndCharge = 384;                     // plan: rows charged to the CTA that owns a segment's end
+constexpr int kSegEndCharge = 320;                     // plan: rows charged to the CTA that owns a segment's end
 constexpr int kMergeRegs = 36;                         // 32 accumulators + m0, m1, l0, l1
 constexpr int kMergeSlotBytes = kMergeRegs * 32 * 4;
 constexpr int kDecodeSmem = kStages * (kStageBytes + kQSlotBytes) + 2 * kMergeSlotBytes;
@@ -786,8 +786,9 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
   // The CTA that owns the end of a segment does more than stream rows: it streams one more tile (the rows appended
   // since the plan was built), stores the appended row, and finishes one piece and starts the next (merge of the
   // warps, output, the next group's queries).  Every non-empty segment's end is therefore charged kSegEndCharge
-  // rows, so that those CTAs get fewer plan-time rows and do not finish last (measured: configs[1] 19.7 -> 17.2 us
-  // and configs[2] 36.3 -> 34.1 us per layer-step between a charge of 64 and of 384 rows; flat beyond).
+  // rows, so that those CTAs get fewer plan-time rows and do not finish last.  Measured per-CTA stream times put
+  // the cost of a segment end at 290-330 rows' worth of streaming; between a charge of 64 and of 320 rows
+  // configs[1] went from 19.7 to 17.3 us and configs[2] from 36.3 to 34.2 us per layer-step (flat from 256 to 512).
   int64_t total = 0, charged = 0;
   for (int s = 0; s < n_segs; ++s) {
     if (cache->seg_len[s] < 0 || cache->seg_len[s] > cache->seg_cap[s]) return CATEKV_ERR_INVALID_ARG;
