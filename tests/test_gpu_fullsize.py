@@ -214,3 +214,60 @@ def test_cfg2_retrieval_on_adaptive_heads(ck):
     ck.catekv_decode_attn(step, q, plan, out)
     ref, _ = orc.decode_attention(soc, synth.bits(q), cells=[(0, s) for s in cells])
     H.check_attention(out, None, None, ref, None, "cfg2 retrieval")
+
+
+def test_cfg3_retrieval_in_place_as_the_bench_runs_it(ck):
+    # configs[3] shape, the retrieval step bench.py times: 1024 rows per adaptive head, chunk size 8, one-launch
+    # append, index lists, attention in place under a plan over all resident CTAs
+    w = synth.WORKLOADS["cfg3"]
+    layer, cs, budget = 7, 8, 1024
+    p, mask, cache, idx = _build_layer(ck, w, layer, 8)
+    del p, idx
+    meta = ck.catekv_retrieval_meta(cache, cs)
+    ck.catekv_retrieval_build(cache, cs, meta)
+    rmask = (mask.reshape(-1) == 0).astype(np.uint8)
+    n_segs = w.B * w.Hkv
+    ridx = torch.full((n_segs, budget + 2 * cs + w.local), -1, dtype=torch.int32, device="cuda")
+    sel = torch.full((n_segs,), -99, dtype=torch.int32, device="cuda")
+    view = ck.CacheView(cache, ck.catekv_retrieve_lengths(cache, cs, rmask, budget, w.sink, w.local))
+    plan = ck.DecodePlan(view, ck.catekv_decode_num_ctas())
+    ck.catekv_decode_plan(view, plan)
+    out = torch.empty((w.B, w.Hq, w.d), dtype=torch.float32, device="cuda")
+    lse = torch.empty((w.B, w.Hq), dtype=torch.float32, device="cuda")
+    for step in range(2):
+        q, kn, vn = synth.decode_inputs(w, layer, step, "cuda", mask)
+        ck.catekv_append_retrieval(cache, kn, vn, cs, meta)
+        ck.catekv_retrieve_select(cache, meta, cs, q, rmask, budget, w.sink, w.local, ridx, sel)
+        ck.catekv_decode_attn_indexed(cache, ridx, sel, q, plan, out, lse)
+    torch.cuda.synchronize()
+    lens = [int(L) for L in cache.seg_len]
+    got_sel = sel.cpu().tolist()
+    want_len = ck.catekv_retrieve_lengths(cache, cs, rmask, budget, w.sink, w.local)
+    ret = np.nonzero(rmask)[0]
+    cells = [int(ret[0]), int(ret[len(ret) // 2]), int(ret[-1]), int(np.nonzero(rmask == 0)[0][3])]
+    qb = orc.bf16_to_f64(synth.bits(q))
+    soc = orc.HybridCache(w.B, w.Hkv, w.d)
+    soc.k_rows = [np.zeros((0, w.d), dtype=np.uint16)] * n_segs
+    soc.v_rows = [np.zeros((0, w.d), dtype=np.uint16)] * n_segs
+    for s in cells:
+        o, L = int(cache.seg_off[s]), lens[s]
+        krows, vrows = synth.bits(cache.k_pool[o:o + L]), synth.bits(cache.v_pool[o:o + L])
+        b, h = divmod(s, w.Hkv)
+        if rmask[s]:
+            assert got_sel[s] == want_len[s] and want_len[s] <= budget
+            got = ridx[s, :got_sel[s]].cpu().numpy().astype(np.int64)
+            kmax, kmin = orc.retrieval_metadata(krows, cs)
+            # the metadata the device keeps, appended rows included
+            c0 = o // cs
+            m = synth.bits(meta.view(torch.bfloat16).view(-1, 2, 128)[c0:c0 + kmax.shape[0]])
+            assert np.array_equal(orc.bf16_to_f64(m[:, 0]), kmax) and np.array_equal(orc.bf16_to_f64(m[:, 1]), kmin)
+            scores = orc.retrieval_scores(qb[b, h * w.G:(h + 1) * w.G], kmax, kmin)
+            want = orc.retrieve_indices(scores, L, w.sink, w.local, budget, cs)
+            assert got.shape == want.shape and np.all(np.diff(got) > 0)
+            assert len(np.setdiff1d(got, want)) <= 0.02 * len(want)  # fp32 against fp64 bounds: near-ties only
+        else:
+            assert got_sel[s] == -1
+            got = np.arange(L)
+        soc.k_rows[s], soc.v_rows[s] = krows[got], vrows[got]
+    ref, ref_lse = orc.decode_attention(soc, synth.bits(q), cells=[divmod(s, w.Hkv) for s in cells])
+    H.check_attention(out, None, lse, ref, ref_lse, "cfg3 retrieval in place")
