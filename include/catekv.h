@@ -62,6 +62,28 @@ extern "C" {
 
 typedef void* catekv_stream; /* cudaStream_t */
 
+#define CATEKV_PAGE_ROWS 64 /* rows of an overflow page */
+
+/*
+ * Overflow pages of a cache: room for segments to grow past the capacity they were laid out with, without moving
+ * what they hold (the paper sizes its caches up front and has no counterpart).  Row r of segment s lives in the
+ * cache's own pools while r < seg_cap[s]; beyond that, row seg_cap[s] + 64 p + i is row 64 table[s][p] + i of the
+ * overflow pools.  Pages are handed out by catekv_pages_reserve (host bump allocator) and never move or return.
+ * All arrays are allocated by the caller; table and table_dev start out filled with -1, seg_pages with 0.
+ */
+typedef struct catekv_pages {
+  int32_t max_pages;   /* table entries per segment */
+  int32_t n_pages;     /* pages of the overflow pools */
+  int32_t next_free;   /* host: pages handed out so far (start at 0) */
+  int32_t reserved;
+  void* k_ovf;         /* device, bf16 [n_pages * 64, d] */
+  void* v_ovf;         /* device, bf16 [n_pages * 64, d] */
+  int32_t* table_dev;  /* device [B*Hkv, max_pages] */
+  int32_t* table;      /* host   [B*Hkv, max_pages], mirror of table_dev */
+  int32_t* seg_pages;  /* host   [B*Hkv], pages handed to each segment */
+  const int32_t* seg_cap_dev; /* device [B*Hkv], copy of the cache's seg_cap */
+} catekv_pages;
+
 /* Hybrid per-head KV cache of one layer (Section 1; Section 3.2 last paragraph). */
 typedef struct catekv_cache {
   int32_t B;              /* sequences */
@@ -76,6 +98,11 @@ typedef struct catekv_cache {
   const int32_t* seg_off;     /* host   [B*Hkv] */
   const int32_t* seg_cap;     /* host   [B*Hkv] */
   int32_t* seg_len;           /* host   [B*Hkv], mirror of seg_len_dev kept by the library's calls */
+  catekv_pages* pages;        /* overflow pages, or NULL.  With pages a segment may hold up to
+                                 seg_cap + 64 * seg_pages rows; catekv_append, catekv_cache_advance,
+                                 catekv_decode_plan, catekv_decode_attn / _partials / _combine,
+                                 catekv_append_decode_attn and catekv_cache_regrow (as the source) follow them;
+                                 every other call refuses such a cache with CATEKV_ERR_UNSUPPORTED */
 } catekv_cache;
 
 /* Version of this ABI (major * 1000 + minor). */
@@ -187,6 +214,17 @@ int catekv_append(catekv_cache* cache, const void* k_new, const void* v_new, cat
  * (CATEKV_ERR_CAPACITY, nothing changed) and then adds n_tokens to cache->seg_len.  Launches nothing.
  */
 int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens);
+
+/*
+ * Paged growth.  Makes sure that every segment can take n_new more rows: segments whose capacity
+ * (seg_cap + 64 * seg_pages) is short get further overflow pages, the new table entries are copied to the device
+ * on `stream` (from cache->pages->table: leave it untouched until that copy has run).  Host bookkeeping only
+ * besides that copy; nothing is launched.  CATEKV_ERR_CAPACITY (nothing changed) if the overflow pools or a
+ * segment's table row run out; CATEKV_ERR_INVALID_ARG if the cache has no pages.  Decode plans built before
+ * stay valid.  catekv_cache_regrow with such a cache as the source gathers base rows and pages into one
+ * contiguous segment again.
+ */
+int catekv_pages_reserve(catekv_cache* cache, int32_t n_new, catekv_stream stream);
 
 /*
  * Growth beyond the capacity a cache was laid out with (Section 4.4.3 keeps generating for as long as the

@@ -32,11 +32,20 @@ class CatekvError(RuntimeError):
         super().__init__(f"{where}: {msg} [{code}]")
 
 
+class PagesStruct(C.Structure):
+    _fields_ = [("max_pages", C.c_int32), ("n_pages", C.c_int32), ("next_free", C.c_int32), ("reserved", C.c_int32),
+                ("k_ovf", C.c_void_p), ("v_ovf", C.c_void_p), ("table_dev", C.c_void_p), ("table", C.c_void_p),
+                ("seg_pages", C.c_void_p), ("seg_cap_dev", C.c_void_p)]
+
+
 class CacheStruct(C.Structure):
     _fields_ = [("B", C.c_int32), ("Hkv", C.c_int32), ("d", C.c_int32), ("reserved", C.c_int32),
                 ("total_rows", C.c_int64), ("k_pool", C.c_void_p), ("v_pool", C.c_void_p),
                 ("seg_off_dev", C.c_void_p), ("seg_len_dev", C.c_void_p),
-                ("seg_off", C.c_void_p), ("seg_cap", C.c_void_p), ("seg_len", C.c_void_p)]
+                ("seg_off", C.c_void_p), ("seg_cap", C.c_void_p), ("seg_len", C.c_void_p),
+                ("pages", C.POINTER(PagesStruct))]
+
+PAGE_ROWS = 64
 
 
 class SelectParams(C.Structure):
@@ -69,6 +78,7 @@ def _load():
         "catekv_append": (C.c_int, [C.POINTER(CacheStruct), vp, vp, vp]),
         "catekv_cache_advance": (C.c_int, [C.POINTER(CacheStruct), i32]),
         "catekv_cache_regrow": (C.c_int, [C.POINTER(CacheStruct), C.POINTER(CacheStruct), vp]),
+        "catekv_pages_reserve": (C.c_int, [C.POINTER(CacheStruct), i32, vp]),
         "catekv_decode_num_ctas": (C.c_int, []),
         "catekv_decode_plan_bytes": (sz, [i32, i32, i32]),
         "catekv_decode_workspace_bytes": (sz, [i32, i32, i32]),
@@ -150,7 +160,26 @@ class Cache:
         self.seg_len_dev = torch.zeros(B * Hkv, dtype=torch.int32, device=device)
         self.struct = CacheStruct(B, Hkv, d, 0, self.total_rows, self.k_pool.data_ptr(), self.v_pool.data_ptr(),
                                   self.seg_off_dev.data_ptr(), self.seg_len_dev.data_ptr(),
-                                  _np_ptr(self.seg_off), _np_ptr(self.seg_cap), _np_ptr(self.seg_len))
+                                  _np_ptr(self.seg_off), _np_ptr(self.seg_cap), _np_ptr(self.seg_len), None)
+        self.pages = None
+
+    def attach_pages(self, n_pages: int, max_pages: int):
+        """Give the cache overflow pools of n_pages pages of 64 rows (memory only; catekv_pages_reserve hands
+        the pages out).  The segments keep what they hold."""
+        n = self.B * self.Hkv
+        pg = type("Pages", (), {})()
+        pg.k_ovf = torch.empty((max(n_pages, 1) * PAGE_ROWS, self.d), dtype=torch.bfloat16, device=self.device)
+        pg.v_ovf = torch.empty_like(pg.k_ovf)
+        pg.table = np.full((n, max_pages), -1, dtype=np.int32)
+        pg.table_dev = torch.full((n, max_pages), -1, dtype=torch.int32, device=self.device)
+        pg.seg_pages = np.zeros(n, dtype=np.int32)
+        pg.seg_cap_dev = torch.from_numpy(self.seg_cap).to(self.device)
+        pg.struct = PagesStruct(max_pages, n_pages, 0, 0, pg.k_ovf.data_ptr(), pg.v_ovf.data_ptr(),
+                                pg.table_dev.data_ptr(), _np_ptr(pg.table), _np_ptr(pg.seg_pages),
+                                pg.seg_cap_dev.data_ptr())
+        self.pages = pg
+        self.struct.pages = C.pointer(pg.struct)
+        return pg
 
     def set_lengths(self, lens):
         """Set host mirror and device lengths (used when rows are written by the caller)."""
@@ -169,6 +198,11 @@ def catekv_append(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor):
 def catekv_cache_advance(cache: Cache, n_tokens: int = 1):
     """Host mirror only: account for appends that a replayed CUDA graph performs on the device."""
     _check(_lib.catekv_cache_advance(C.byref(cache.struct), n_tokens), "catekv_cache_advance")
+
+
+def catekv_pages_reserve(cache: Cache, n_new: int):
+    """Make sure every segment can take n_new more rows (hands out overflow pages where the capacity is short)."""
+    _check(_lib.catekv_pages_reserve(C.byref(cache.struct), n_new, _stream()), "catekv_pages_reserve")
 
 
 def catekv_cache_regrow(src: Cache, max_new: int) -> Cache:
@@ -321,7 +355,7 @@ class CacheView:
         self.seg_len = np.ascontiguousarray(lens, dtype=np.int32).reshape(-1).copy()
         b = cache.struct
         self.struct = CacheStruct(b.B, b.Hkv, b.d, 0, b.total_rows, b.k_pool, b.v_pool, b.seg_off_dev, b.seg_len_dev,
-                                  b.seg_off, b.seg_cap, _np_ptr(self.seg_len))
+                                  b.seg_off, b.seg_cap, _np_ptr(self.seg_len), None)
 
 
 def catekv_retrieve_select(cache: Cache, meta: torch.Tensor, chunk_size: int, q: torch.Tensor, retrieval_mask,

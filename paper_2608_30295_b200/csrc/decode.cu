@@ -46,7 +46,7 @@ struct WorkItem {  // 32 bytes
   int32_t slot;      // partial slot, or -1 when the piece is the whole segment (final output written directly)
   int64_t row_base;  // pool row of t0 (segment offset + t0)
   int32_t last;      // 1: last piece of its segment; it also covers rows [t1, current length)
-  int32_t reserved;
+  int32_t cap;       // capacity of the segment in the cache's own pools (rows from there on live in overflow pages)
 };
 static_assert(sizeof(WorkItem) == 32, "work item layout");
 struct CtaHeader {  // 48 bytes: the CTA's item range and a copy of its first item (one load starts the stream)
@@ -98,6 +98,12 @@ struct DecodeArgs {
   const int32_t* idx;
   int64_t idx_stride;
   const int32_t* sel_len;
+  // paged variant only: row r >= cap of segment s is row 64 * page_table[s * max_pages + (r - cap) / 64] + (r - cap) % 64
+  // of the overflow pools
+  uint8_t* k_ovf;
+  uint8_t* v_ovf;
+  const int32_t* page_table;
+  int32_t max_pages;
   const uint16_t* q;  // [B, Hq, d]
   int32_t Hq, Hkv, G;
   float scale_log2;  // sm_scale * log2(e)
@@ -121,12 +127,14 @@ constexpr int kDecodeSmem = kStages * (kStageBytes + kQSlotBytes) + 2 * kMergeSl
 // segment - by tiles of the rows appended since the plan was built, [t1, live length).  The live length
 // is loaded when the item is read but first used only after the plan-time tiles have been issued, so
 // the stream never waits for that load.
+constexpr int kModePlain = 0, kModeIndexed = 1, kModePaged = 2;  // instantiations of the attention kernel
 struct ItemCursor {
   int seg, t0, t1, slot, last;
   int np;            // tiles of the plan-time rows
   int live;          // rows to attend to: current segment length (plus the row being appended), if last
   int new_row;       // fused append: the segment-relative row that comes from k_new / v_new, else -1
   int indexed;       // indexed variant: the item's rows are taken through the index list
+  int cap;           // paged variant: rows from here on live in overflow pages
   int64_t row_base;
 };
 
@@ -143,12 +151,14 @@ __device__ __forceinline__ ItemCursor plan_cursor(const WorkItem& w) {
   c.live = w.t1;
   c.new_row = -1;
   c.indexed = 0;
+  c.cap = w.cap;
   return c;
 }
 // the part that reads what earlier kernels wrote: the live length (a plain load: with a fused append this
 // kernel itself updates the length when it is done with the segment)
-template <bool kIndexed>
+template <int kMode>
 __device__ __forceinline__ void live_cursor(const DecodeArgs& a, ItemCursor& c) {
+  constexpr bool kIndexed = kMode == kModeIndexed;
   int len;
   if (kIndexed) {
     const int sel = *reinterpret_cast<const volatile int32_t*>(a.sel_len + c.seg);
@@ -168,14 +178,14 @@ __device__ __forceinline__ WorkItem unpack_item(const int4& x, const int4& y) {
   WorkItem w;
   w.seg = x.x; w.t0 = x.y; w.t1 = x.z; w.slot = x.w;
   w.row_base = (int64_t)(((uint64_t)(uint32_t)y.y << 32) | (uint32_t)y.x);
-  w.last = y.z; w.reserved = 0;
+  w.last = y.z; w.cap = y.w;
   return w;
 }
-template <bool kIndexed>
+template <int kMode>
 __device__ __forceinline__ ItemCursor read_item(const DecodeArgs& a, int it) {
   const int4* p = reinterpret_cast<const int4*>(a.items + it);
   ItemCursor c = plan_cursor(unpack_item(__ldg(p), __ldg(p + 1)));
-  live_cursor<kIndexed>(a, c);
+  live_cursor<kMode>(a, c);
   return c;
 }
 // tiles of the item: plan-time tiles plus tiles of the appended rows; at least one
@@ -207,8 +217,10 @@ __device__ __forceinline__ unsigned long long gtime() {
 #define CATEKV_STAMP(i) do { } while (0)
 #endif
 
-template <bool kIndexed>
+template <int kMode>
 __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const DecodeArgs a) {
+  constexpr bool kIndexed = kMode == kModeIndexed;
+  constexpr bool kPaged = kMode == kModePaged;
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -245,7 +257,16 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       const int r = id >> 4, c = id & 15;
       const int ok = r < rows_left ? 16 : 0;
       int64_t grow = ok ? row0 + r : 0;  // padding rows read nothing
+      uint8_t* kp = a.k_pool;
+      uint8_t* vp = a.v_pool;
       if (kIndexed && pc.indexed && ok) grow = (pc.row_base - pc.t0) + ix[i];
+      if (kPaged && ok && start + r >= pc.cap) {  // the row lives in an overflow page
+        const int o = start + r - pc.cap;
+        const int page = __ldg(a.page_table + (int64_t)pc.seg * a.max_pages + (o >> 6));
+        grow = (int64_t)page * 64 + (o & 63);
+        kp = a.k_ovf;
+        vp = a.v_ovf;
+      }
       const int64_t goff = grow * kRowBytes + c * 16;
       const uint32_t so = tile_off(r, c);
       if (ok && r == new_r && pc.new_row >= 0) {  // only inside the tile's valid rows (never in a plan-time tile)
@@ -253,11 +274,11 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
         const size_t noff = (size_t)pc.seg * kRowBytes + c * 16;
         cp_async16(sb + so, a.k_new + noff, 16);
         cp_async16(sb + kTile * kRowBytes + so, a.v_new + noff, 16);
-        *reinterpret_cast<uint4*>(a.k_pool + goff) = *reinterpret_cast<const uint4*>(a.k_new + noff);
-        *reinterpret_cast<uint4*>(a.v_pool + goff) = *reinterpret_cast<const uint4*>(a.v_new + noff);
+        *reinterpret_cast<uint4*>(kp + goff) = *reinterpret_cast<const uint4*>(a.k_new + noff);
+        *reinterpret_cast<uint4*>(vp + goff) = *reinterpret_cast<const uint4*>(a.v_new + noff);
       } else {
-        cp_async16(sb + so, a.k_pool + goff, ok);
-        cp_async16(sb + kTile * kRowBytes + so, a.v_pool + goff, ok);
+        cp_async16(sb + so, kp + goff, ok);
+        cp_async16(sb + kTile * kRowBytes + so, vp + goff, ok);
       }
     }
   };
@@ -287,7 +308,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     ++p_seq;
     if (++p_tile >= pc.np && p_tile >= item_tiles(pc)) {
       p_tile = 0;
-      if (++p_item < item_end) pc = read_item<kIndexed>(a, p_item);
+      if (++p_item < item_end) pc = read_item<kMode>(a, p_item);
     }
     load_idx();
   };
@@ -311,12 +332,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     cp_async_commit();
   }
   pdl_wait();  // from here on: lengths, queries and rows written by earlier kernels
-  live_cursor<kIndexed>(a, pc);
+  live_cursor<kMode>(a, pc);
   const ItemCursor first = pc;
   issue_q(0, pc.seg);
   if (p_tile >= pc.np && p_tile >= item_tiles(pc)) {
     p_tile = 0;
-    if (++p_item < item_end) pc = read_item<kIndexed>(a, p_item);
+    if (++p_item < item_end) pc = read_item<kMode>(a, p_item);
   }
   load_idx();
   for (int s = pre; s < kStages - 1; ++s) issue();
@@ -324,7 +345,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
 
   int seq = 0;
   for (int c_item = item_begin; c_item < item_end; ++c_item) {
-    const ItemCursor cc = c_item == item_begin ? first : read_item<kIndexed>(a, c_item);
+    const ItemCursor cc = c_item == item_begin ? first : read_item<kMode>(a, c_item);
     uint32_t qf[8][2];
     float o[8][4];
 #pragma unroll
@@ -631,16 +652,41 @@ __global__ void __launch_bounds__(kCombineWarps * 32) decode_combine_kernel(cons
 // ------------------------------------------------------------------------------------------
 // Append
 // ------------------------------------------------------------------------------------------
+struct PageArgs {  // overflow pages of a cache (all null / 0 without pages)
+  uint8_t* k_ovf;
+  uint8_t* v_ovf;
+  const int32_t* table;
+  const int32_t* seg_cap;
+  int32_t max_pages;
+};
+static PageArgs page_args(const catekv_cache* c) {
+  PageArgs p = {nullptr, nullptr, nullptr, nullptr, 0};
+  if (c->pages) {
+    p.k_ovf = (uint8_t*)c->pages->k_ovf;
+    p.v_ovf = (uint8_t*)c->pages->v_ovf;
+    p.table = c->pages->table_dev;
+    p.seg_cap = c->pages->seg_cap_dev;
+    p.max_pages = c->pages->max_pages;
+  }
+  return p;
+}
+
 __global__ void __launch_bounds__(128) append_kernel(uint8_t* k_pool, uint8_t* v_pool, const int32_t* seg_off,
                                                      int32_t* seg_len, const uint8_t* k_new, const uint8_t* v_new,
-                                                     int n_segs) {
+                                                     int n_segs, const PageArgs pg) {
   const int seg = blockIdx.x * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   pdl_launch_dependents();
   pdl_wait();
   if (seg >= n_segs) return;
   const int len = seg_len[seg];
-  const int64_t row = (int64_t)seg_off[seg] + len;
+  int64_t row = (int64_t)seg_off[seg] + len;
+  if (pg.table && len >= pg.seg_cap[seg]) {  // the row goes to an overflow page
+    const int o = len - pg.seg_cap[seg];
+    row = (int64_t)pg.table[(int64_t)seg * pg.max_pages + (o >> 6)] * 64 + (o & 63);
+    k_pool = pg.k_ovf;
+    v_pool = pg.v_ovf;
+  }
   const int c = lane & 15;
   const uint8_t* src = (lane < 16 ? k_new : v_new) + (size_t)seg * kRowBytes + c * 16;
   uint8_t* dst = (lane < 16 ? k_pool : v_pool) + row * kRowBytes + c * 16;
@@ -655,7 +701,16 @@ static int check_cache(const catekv_cache* c) {
   if (c->d != kD) return CATEKV_ERR_UNSUPPORTED;
   if (!c->k_pool || !c->v_pool || !c->seg_off_dev || !c->seg_len_dev || !c->seg_off || !c->seg_cap || !c->seg_len)
     return CATEKV_ERR_INVALID_ARG;
+  if (c->pages) {
+    const catekv_pages* p = c->pages;
+    if (p->max_pages <= 0 || p->n_pages < 0 || p->next_free < 0 || p->next_free > p->n_pages) return CATEKV_ERR_INVALID_ARG;
+    if (!p->k_ovf || !p->v_ovf || !p->table_dev || !p->table || !p->seg_pages || !p->seg_cap_dev) return CATEKV_ERR_INVALID_ARG;
+  }
   return CATEKV_OK;
+}
+// rows segment s can hold: its own capacity plus the overflow pages it has been given
+static inline int64_t seg_capacity(const catekv_cache* c, int s) {
+  return (int64_t)c->seg_cap[s] + (c->pages ? (int64_t)c->pages->seg_pages[s] * CATEKV_PAGE_ROWS : 0);
 }
 
 }  // namespace catekv
@@ -669,11 +724,11 @@ extern "C" int catekv_append(catekv_cache* cache, const void* k_new, const void*
   const int n = cache->B * cache->Hkv;
   for (int s = 0; s < n; ++s) {
     if (cache->seg_len[s] < 0) return CATEKV_ERR_INVALID_ARG;
-    if (cache->seg_len[s] + 1 > cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+    if (cache->seg_len[s] + 1 > seg_capacity(cache, s)) return CATEKV_ERR_CAPACITY;
   }
   CATEKV_CUDA_TRY(launch_pdl(append_kernel, dim3((n + 3) / 4), dim3(128), 0, (cudaStream_t)stream,
                              (uint8_t*)cache->k_pool, (uint8_t*)cache->v_pool, cache->seg_off_dev, cache->seg_len_dev,
-                             (const uint8_t*)k_new, (const uint8_t*)v_new, n));
+                             (const uint8_t*)k_new, (const uint8_t*)v_new, n, page_args(cache)));
   for (int s = 0; s < n; ++s) cache->seg_len[s] += 1;
   return CATEKV_OK;
 }
@@ -701,7 +756,7 @@ extern "C" int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens) {
   if (n_tokens < 0) return CATEKV_ERR_INVALID_ARG;
   const int n = cache->B * cache->Hkv;
   for (int s = 0; s < n; ++s)
-    if ((int64_t)cache->seg_len[s] + n_tokens > cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+    if ((int64_t)cache->seg_len[s] + n_tokens > seg_capacity(cache, s)) return CATEKV_ERR_CAPACITY;
   for (int s = 0; s < n; ++s) cache->seg_len[s] += n_tokens;
   return CATEKV_OK;
 }
@@ -712,22 +767,59 @@ namespace catekv {
 constexpr int kRegrowRowsPerBlock = 64;
 __global__ void __launch_bounds__(256) regrow_kernel(const uint8_t* sk, const uint8_t* sv, const int32_t* s_off,
                                                      const int32_t* s_len, uint8_t* dk, uint8_t* dv, const int32_t* d_off,
-                                                     int32_t* d_len) {
+                                                     int32_t* d_len, const PageArgs pg) {
   const int seg = blockIdx.y;
   const int len = s_len[seg];
   if (blockIdx.x == 0 && threadIdx.x == 0) d_len[seg] = len;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint8_t* src = (lane < 16 ? sk : sv) + (int64_t)s_off[seg] * kRowBytes + (lane & 15) * 16;
+  const uint8_t* ovf = (lane < 16 ? pg.k_ovf : pg.v_ovf) + (lane & 15) * 16;
+  const int cap = pg.table ? pg.seg_cap[seg] : 0x7fffffff;  // rows from here on come from the source's overflow pages
   uint8_t* dst = (lane < 16 ? dk : dv) + (int64_t)d_off[seg] * kRowBytes + (lane & 15) * 16;
   const int r0 = blockIdx.x * kRegrowRowsPerBlock;
 #pragma unroll 4
   for (int i = warp; i < kRegrowRowsPerBlock; i += 8) {
     const int r = r0 + i;
     if (r >= len) break;
-    *reinterpret_cast<uint4*>(dst + (int64_t)r * kRowBytes) = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)r * kRowBytes));
+    const uint8_t* from = src + (int64_t)r * kRowBytes;
+    if (r >= cap) {
+      const int o = r - cap;
+      from = ovf + ((int64_t)pg.table[(int64_t)seg * pg.max_pages + (o >> 6)] * 64 + (o & 63)) * kRowBytes;
+    }
+    *reinterpret_cast<uint4*>(dst + (int64_t)r * kRowBytes) = __ldg(reinterpret_cast<const uint4*>(from));
   }
 }
 }  // namespace catekv
+
+extern "C" int catekv_pages_reserve(catekv_cache* cache, int32_t n_new, catekv_stream stream) {
+  int rc = check_cache(cache);
+  if (rc) return rc;
+  if (!cache->pages || n_new < 0) return CATEKV_ERR_INVALID_ARG;
+  catekv_pages* p = cache->pages;
+  const int n = cache->B * cache->Hkv;
+  // first pass: what is needed, nothing changed yet
+  int64_t extra = 0;
+  for (int s = 0; s < n; ++s) {
+    if (cache->seg_len[s] < 0 || cache->seg_len[s] > seg_capacity(cache, s)) return CATEKV_ERR_INVALID_ARG;
+    const int64_t over = (int64_t)cache->seg_len[s] + n_new - cache->seg_cap[s];
+    const int64_t want = over > 0 ? (over + CATEKV_PAGE_ROWS - 1) / CATEKV_PAGE_ROWS : 0;
+    if (want > p->max_pages) return CATEKV_ERR_CAPACITY;
+    if (want > p->seg_pages[s]) extra += want - p->seg_pages[s];
+  }
+  if (extra > (int64_t)p->n_pages - p->next_free) return CATEKV_ERR_CAPACITY;
+  for (int s = 0; s < n; ++s) {
+    const int64_t over = (int64_t)cache->seg_len[s] + n_new - cache->seg_cap[s];
+    const int want = over > 0 ? (int)((over + CATEKV_PAGE_ROWS - 1) / CATEKV_PAGE_ROWS) : 0;
+    const int have = p->seg_pages[s];
+    if (want <= have) continue;
+    int32_t* row = p->table + (size_t)s * p->max_pages;
+    for (int q = have; q < want; ++q) row[q] = p->next_free++;
+    p->seg_pages[s] = want;
+    CATEKV_CUDA_TRY(cudaMemcpyAsync(p->table_dev + (size_t)s * p->max_pages + have, row + have,
+                                    sizeof(int32_t) * (size_t)(want - have), cudaMemcpyHostToDevice, (cudaStream_t)stream));
+  }
+  return CATEKV_OK;
+}
 
 extern "C" int catekv_cache_regrow(const catekv_cache* src, catekv_cache* dst, catekv_stream stream) {
   int rc = check_cache(src);
@@ -736,17 +828,19 @@ extern "C" int catekv_cache_regrow(const catekv_cache* src, catekv_cache* dst, c
   if (rc) return rc;
   if (src->B != dst->B || src->Hkv != dst->Hkv) return CATEKV_ERR_INVALID_ARG;
   if (src->k_pool == dst->k_pool || src->v_pool == dst->v_pool) return CATEKV_ERR_INVALID_ARG;
+  if (dst->pages) return CATEKV_ERR_UNSUPPORTED;  // the destination is one contiguous segment per (sequence, head)
   const int n = src->B * src->Hkv;
   int max_len = 0;
   for (int s = 0; s < n; ++s) {
-    if (src->seg_len[s] < 0 || src->seg_len[s] > src->seg_cap[s]) return CATEKV_ERR_INVALID_ARG;
+    if (src->seg_len[s] < 0 || src->seg_len[s] > seg_capacity(src, s)) return CATEKV_ERR_INVALID_ARG;
     if (src->seg_len[s] > dst->seg_cap[s]) return CATEKV_ERR_CAPACITY;
     max_len = src->seg_len[s] > max_len ? src->seg_len[s] : max_len;
   }
   const int gx = max_len > 0 ? (max_len + kRegrowRowsPerBlock - 1) / kRegrowRowsPerBlock : 1;
   regrow_kernel<<<dim3(gx, n), 256, 0, (cudaStream_t)stream>>>((const uint8_t*)src->k_pool, (const uint8_t*)src->v_pool,
                                                                src->seg_off_dev, src->seg_len_dev, (uint8_t*)dst->k_pool,
-                                                               (uint8_t*)dst->v_pool, dst->seg_off_dev, dst->seg_len_dev);
+                                                               (uint8_t*)dst->v_pool, dst->seg_off_dev, dst->seg_len_dev,
+                                                               page_args(src));
   CATEKV_CUDA_TRY(cudaGetLastError());
   for (int s = 0; s < n; ++s) dst->seg_len[s] = src->seg_len[s];
   return CATEKV_OK;
@@ -755,11 +849,11 @@ extern "C" int catekv_cache_regrow(const catekv_cache* src, catekv_cache* dst, c
 extern "C" int catekv_decode_num_ctas(void) {
   int dev = 0, sms = 0, per_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return CATEKV_ERR_CUDA;
-  cudaError_t e = cudaFuncSetAttribute(decode_partial_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
+  cudaError_t e = cudaFuncSetAttribute(decode_partial_kernel<kModePlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
   if (e != cudaSuccess) { set_cuda_error(e); return CATEKV_ERR_CUDA; }
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) { set_cuda_error(e); return CATEKV_ERR_CUDA; }
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_partial_kernel<false>, kDecodeThreads, kDecodeSmem);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_partial_kernel<kModePlain>, kDecodeThreads, kDecodeSmem);
   if (e != cudaSuccess) { set_cuda_error(e); return CATEKV_ERR_CUDA; }
   if (per_sm < 1) per_sm = 1;
   return sms * per_sm;
@@ -791,7 +885,7 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
   // configs[1] went from 19.7 to 17.3 us and configs[2] from 36.3 to 34.2 us per layer-step (flat from 256 to 512).
   int64_t total = 0, charged = 0;
   for (int s = 0; s < n_segs; ++s) {
-    if (cache->seg_len[s] < 0 || cache->seg_len[s] > cache->seg_cap[s]) return CATEKV_ERR_INVALID_ARG;
+    if (cache->seg_len[s] < 0 || cache->seg_len[s] > seg_capacity(cache, s)) return CATEKV_ERR_INVALID_ARG;
     total += cache->seg_len[s];
     charged += cache->seg_len[s] + (cache->seg_len[s] > 0 ? kSegEndCharge : 0);
   }
@@ -818,7 +912,7 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
       const int32_t len = cache->seg_len[seg];
       if (len == 0) {
         // an empty segment still gets one (direct) item, so that the plan stays valid once it grows
-        items[n_items++] = WorkItem{seg, 0, 0, -1, (int64_t)cache->seg_off[seg], 1, 0};
+        items[n_items++] = WorkItem{seg, 0, 0, -1, (int64_t)cache->seg_off[seg], 1, cache->seg_cap[seg]};
         segs[seg] = SegInfo{0, 1, 0, 0};
         ++seg;
         seg_first_item = n_items;
@@ -826,7 +920,7 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
       }
       if (room <= 0) break;
       const int32_t take = (int32_t)((int64_t)(len - pos) < room ? (len - pos) : room);
-      items[n_items++] = WorkItem{seg, pos, pos + take, 0, (int64_t)cache->seg_off[seg] + pos, 0, 0};
+      items[n_items++] = WorkItem{seg, pos, pos + take, 0, (int64_t)cache->seg_off[seg] + pos, 0, cache->seg_cap[seg]};
       pos += take;
       room -= take;
       if (pos == len) {
@@ -909,8 +1003,9 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* k_ne
     int dev = 0;
     CATEKV_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-      CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
-      CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
+      CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<kModePlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
+      CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<kModeIndexed>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
+      CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<kModePaged>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
       if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     DecodeArgs a;
@@ -935,10 +1030,17 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* k_ne
     a.idx = il ? il->idx : nullptr;
     a.idx_stride = il ? il->idx_stride : 0;
     a.sel_len = il ? il->sel_len : nullptr;
+    const PageArgs pg = page_args(cache);
+    a.k_ovf = pg.k_ovf;
+    a.v_ovf = pg.v_ovf;
+    a.page_table = pg.table;
+    a.max_pages = pg.max_pages;
     if (il)
-      CATEKV_CUDA_TRY(launch_pdl(decode_partial_kernel<true>, dim3(hdr->num_ctas), dim3(kDecodeThreads), kDecodeSmem, st, a));
+      CATEKV_CUDA_TRY(launch_pdl(decode_partial_kernel<kModeIndexed>, dim3(hdr->num_ctas), dim3(kDecodeThreads), kDecodeSmem, st, a));
+    else if (cache->pages)
+      CATEKV_CUDA_TRY(launch_pdl(decode_partial_kernel<kModePaged>, dim3(hdr->num_ctas), dim3(kDecodeThreads), kDecodeSmem, st, a));
     else
-      CATEKV_CUDA_TRY(launch_pdl(decode_partial_kernel<false>, dim3(hdr->num_ctas), dim3(kDecodeThreads), kDecodeSmem, st, a));
+      CATEKV_CUDA_TRY(launch_pdl(decode_partial_kernel<kModePlain>, dim3(hdr->num_ctas), dim3(kDecodeThreads), kDecodeSmem, st, a));
   }
   if ((phases & 2) && hdr->n_slots > 0) {
     CombineArgs ca;
@@ -968,6 +1070,7 @@ extern "C" int catekv_decode_attn_indexed(const catekv_cache* cache, const int32
                                           int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                                           size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
   if (!idx || !sel_len || idx_stride < 0) return CATEKV_ERR_INVALID_ARG;
+  if (cache && cache->pages) return CATEKV_ERR_UNSUPPORTED;
   const IndexList il = {idx, idx_stride, sel_len};
   return decode_launch(3, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
                        ws_bytes, stream, &il);
@@ -997,7 +1100,7 @@ extern "C" int catekv_append_decode_attn(catekv_cache* cache, const void* k_new,
   const int n = cache->B * cache->Hkv;
   for (int s = 0; s < n; ++s) {
     if (cache->seg_len[s] < 0) return CATEKV_ERR_INVALID_ARG;
-    if (cache->seg_len[s] + 1 > cache->seg_cap[s]) return CATEKV_ERR_CAPACITY;
+    if (cache->seg_len[s] + 1 > seg_capacity(cache, s)) return CATEKV_ERR_CAPACITY;
   }
   // The appended row must lie behind every row the plan knows: the kernel requests plan-time tiles before it
   // may look at the lengths.  (catekv_decode_attn, without the append, also takes segments that have shrunk.)

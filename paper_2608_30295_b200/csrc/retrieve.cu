@@ -280,7 +280,7 @@ static RetWs ret_ws_layout(int n_segs, int max_len) {
 static int check_cache_r(const catekv_cache* c) {
   if (!c) return CATEKV_ERR_INVALID_ARG;
   if (c->B <= 0 || c->Hkv <= 0) return CATEKV_ERR_INVALID_ARG;
-  if (c->d != kD) return CATEKV_ERR_UNSUPPORTED;
+  if (c->d != kD || c->pages) return CATEKV_ERR_UNSUPPORTED;  // retrieval walks contiguous segments
   if (!c->k_pool || !c->v_pool || !c->seg_off_dev || !c->seg_len_dev || !c->seg_off || !c->seg_cap || !c->seg_len)
     return CATEKV_ERR_INVALID_ARG;
   return CATEKV_OK;

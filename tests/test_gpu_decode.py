@@ -188,6 +188,81 @@ def test_cache_regrow_lets_full_segments_keep_growing(ck):
         assert rc == code
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_paged_growth_past_the_laid_out_capacity(ck, fused):
+    """Segments outgrow their capacity into overflow pages: appends land there, attention reads base rows and
+    pages under plans built before and after the growth, and a regrow gathers everything back."""
+    lens = [100, 128, 1, 0, 300, 64, 17, 255]
+    B, Hkv, G = 2, 4, 4
+    oc = H.random_cache(B, Hkv, lens, seed=31)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=0)  # capacities round_up(len, 128): two segments are full
+    steps = 150  # up to three pages per segment
+    kn = synth.randn_bf16((B, Hkv, 128), "cuda", 31, "kn")
+    vn = synth.randn_bf16((B, Hkv, 128), "cuda", 31, "vn")
+    with pytest.raises(ck.CatekvError) as e:
+        ck.catekv_append(cache, kn, vn)
+    assert e.value.code == ck.ERR_CAPACITY
+    pg = cache.attach_pages(n_pages=24, max_pages=3)
+    with pytest.raises(ck.CatekvError) as e:  # pages attached but none handed out yet
+        ck.catekv_append(cache, kn, vn)
+    assert e.value.code == ck.ERR_CAPACITY
+    with pytest.raises(ck.CatekvError) as e:  # more than the pools hold: refused, nothing changed
+        ck.catekv_pages_reserve(cache, 64 * 3 + 129)
+    assert e.value.code == ck.ERR_CAPACITY and pg.struct.next_free == 0 and not pg.seg_pages.any()
+    plan = ck.DecodePlan(cache, 9)
+    ck.catekv_decode_plan(cache, plan)  # before any growth
+    out = torch.empty((B, Hkv * G, 128), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, Hkv * G), dtype=torch.float32, device="cuda")
+    for step in range(steps):
+        if step % 50 == 0:
+            ck.catekv_pages_reserve(cache, 50)  # in instalments: later pages join the earlier ones
+        kn = synth.randn_bf16((B, Hkv, 128), "cuda", 31, "kn", step)
+        vn = synth.randn_bf16((B, Hkv, 128), "cuda", 31, "vn", step)
+        q = synth.randn_bf16((B, Hkv * G, 128), "cuda", 31, "q", step)
+        if fused:
+            ck.catekv_append_decode_attn(cache, kn, vn, q, plan, out, lse)
+        else:
+            ck.catekv_append(cache, kn, vn)
+            ck.catekv_decode_attn(cache, q, plan, out, lse)
+        oc.append(synth.bits(kn), synth.bits(vn))
+        if step in (0, 27, 28, 63, 64, 65, 149):
+            ref, ref_lse = orc.decode_attention(oc, synth.bits(q))
+            H.check_attention(out, None, lse, ref, ref_lse, f"paged step {step}")
+        if step == 90:
+            ck.catekv_decode_plan(cache, plan)  # a plan whose plan-time rows lie in pages
+    torch.cuda.synchronize()
+    assert list(cache.seg_len) == [L + steps for L in lens] == cache.seg_len_dev.cpu().tolist()
+    want_pages = [max(0, -(-(L + steps - int(c)) // 64)) for L, c in zip(lens, cache.seg_cap)]
+    assert list(pg.seg_pages) == want_pages and pg.struct.next_free == sum(want_pages)
+    assert np.array_equal(pg.table_dev.cpu().numpy(), pg.table)
+    used = pg.table[pg.table >= 0]
+    assert len(set(used.tolist())) == len(used) == sum(want_pages)  # every page handed out once
+    # rows: base part in the cache's pools, the rest in the pages of the table
+    for i, L0 in enumerate(lens):
+        cap, L = int(cache.seg_cap[i]), L0 + steps
+        o = int(cache.seg_off[i])
+        assert np.array_equal(synth.bits(cache.k_pool[o:o + min(L, cap)]), oc.k_rows[i][:cap])
+        for p_i in range(want_pages[i]):
+            r0 = cap + 64 * p_i
+            nrows = min(64, L - r0)
+            page = int(pg.table[i, p_i])
+            assert np.array_equal(synth.bits(pg.k_ovf[page * 64:page * 64 + nrows]), oc.k_rows[i][r0:r0 + nrows])
+            assert np.array_equal(synth.bits(pg.v_ovf[page * 64:page * 64 + nrows]), oc.v_rows[i][r0:r0 + nrows])
+    # the table row of a segment is full: one row more is refused
+    with pytest.raises(ck.CatekvError) as e:
+        ck.catekv_pages_reserve(cache, 64 * 3)
+    assert e.value.code == ck.ERR_CAPACITY
+    # gather everything back into one contiguous cache
+    big = ck.catekv_cache_regrow(cache, max_new=8)
+    torch.cuda.synchronize()
+    for i, L0 in enumerate(lens):
+        o, L = int(big.seg_off[i]), L0 + steps
+        assert np.array_equal(synth.bits(big.k_pool[o:o + L]), oc.k_rows[i])
+        assert np.array_equal(synth.bits(big.v_pool[o:o + L]), oc.v_rows[i])
+    # calls that walk contiguous segments refuse a paged cache
+    assert ck._lib.catekv_retrieval_meta_bytes(ck.C.byref(cache.struct), 8) == 0
+
+
 def test_decode_is_deterministic(ck):
     oc = H.random_cache(2, 4, [700, 64, 1500, 3, 90, 400, 2000, 128], seed=17)
     q = synth.bits(synth.randn_bf16((2, 16, 128), "cpu", 17, "q"))
