@@ -100,7 +100,7 @@ typedef struct catekv_cache {
   int32_t* seg_len;           /* host   [B*Hkv], mirror of seg_len_dev kept by the library's calls */
   catekv_pages* pages;        /* overflow pages, or NULL.  With pages a segment may hold up to
                                  seg_cap + 64 * seg_pages rows; catekv_append, catekv_cache_advance,
-                                 catekv_decode_plan, catekv_decode_attn / _partials / _combine,
+                                 catekv_decode_plan, catekv_decode_attn / _partials / _combine / _noalloc,
                                  catekv_append_decode_attn and catekv_cache_regrow (as the source) follow them;
                                  every other call refuses such a cache with CATEKV_ERR_UNSUPPORTED */
 } catekv_cache;

@@ -251,6 +251,14 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     tile_rows(pc, p_tile, start, rows_left);
     const int64_t row0 = pc.row_base + (start - pc.t0);
     const int new_r = pc.new_row - start;  // tile row that is being appended by this call, if in [0, kTile)
+    // paged variant: a tile touches at most two overflow pages; their table entries are read once, together
+    int pg0 = 0, page0 = 0, page1 = 0;
+    if (kPaged && start + kTile > pc.cap && rows_left > 0) {
+      pg0 = max(0, start - pc.cap) >> 6;
+      const int32_t* row = a.page_table + (int64_t)pc.seg * a.max_pages;
+      page0 = __ldg(row + min(pg0, a.max_pages - 1));
+      page1 = __ldg(row + min(pg0 + 1, a.max_pages - 1));
+    }
 #pragma unroll
     for (int i = 0; i < (kTile * 16) / kDecodeThreads; ++i) {
       const int id = tid + i * kDecodeThreads;
@@ -262,8 +270,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       if (kIndexed && pc.indexed && ok) grow = (pc.row_base - pc.t0) + ix[i];
       if (kPaged && ok && start + r >= pc.cap) {  // the row lives in an overflow page
         const int o = start + r - pc.cap;
-        const int page = __ldg(a.page_table + (int64_t)pc.seg * a.max_pages + (o >> 6));
-        grow = (int64_t)page * 64 + (o & 63);
+        grow = (int64_t)((o >> 6) == pg0 ? page0 : page1) * 64 + (o & 63);
         kp = a.k_ovf;
         vp = a.v_ovf;
       }
