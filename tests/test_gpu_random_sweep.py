@@ -102,3 +102,99 @@ def test_random_select(ck, seed):
                 H.check_indices_band(got, C, nb, sink, local, T, mode, param, where)
             o = int(cache.seg_off[i])
             assert np.array_equal(kp[o:o + L], k[b, h][got]) and np.array_equal(vp[o:o + L], v[b, h][got]), where
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_paged_growth_equals_plain_cache(ck, seed):
+    """The same rows, once in a cache with room and once spilling into overflow pages: identical bits, and the oracle."""
+    rng = np.random.default_rng(7000 + seed)
+    B, Hkv = int(rng.integers(1, 4)), int(rng.integers(1, 5))
+    G = int(rng.choice([1, 2, 4, 7, 8]))
+    kinds = rng.integers(0, 4, size=B * Hkv)
+    lens = [int({0: 0, 1: rng.integers(1, 70), 2: rng.integers(70, 700), 3: rng.integers(700, 3000)}[k]) for k in kinds]
+    steps = int(rng.integers(1, 140))
+    num_ctas = int(rng.choice([1, 3, 17, 296]))
+    fused = bool(rng.integers(0, 2))
+    oc = H.random_cache(B, Hkv, lens, seed=7100 + seed)
+    plain = H.device_cache_from_oracle(ck, oc, max_new=steps)
+    paged = H.device_cache_from_oracle(ck, oc, max_new=int(rng.integers(0, 3)))  # almost no room of its own
+    paged.attach_pages(n_pages=B * Hkv * 4, max_pages=4)
+    plans = []
+    for c in (plain, paged):
+        p = ck.DecodePlan(c, num_ctas)
+        ck.catekv_decode_plan(c, p)
+        plans.append(p)
+    outs = [torch.empty((B, Hkv * G, 128), dtype=torch.float32, device="cuda") for _ in range(2)]
+    lses = [torch.empty((B, Hkv * G), dtype=torch.float32, device="cuda") for _ in range(2)]
+    replan = int(rng.integers(0, steps))
+    for st in range(steps):
+        if st % 32 == 0:
+            ck.catekv_pages_reserve(paged, min(32, steps - st))
+        kn = synth.randn_bf16((B, Hkv, 128), "cuda", 7200 + seed, "kn", st)
+        vn = synth.randn_bf16((B, Hkv, 128), "cuda", 7200 + seed, "vn", st)
+        q = synth.randn_bf16((B, Hkv * G, 128), "cuda", 7200 + seed, "q", st)
+        for c, p, o, l in zip((plain, paged), plans, outs, lses):
+            if fused:
+                ck.catekv_append_decode_attn(c, kn, vn, q, p, o, l)
+            else:
+                ck.catekv_append(c, kn, vn)
+                ck.catekv_decode_attn(c, q, p, o, l)
+        oc.append(synth.bits(kn), synth.bits(vn))
+        assert torch.equal(outs[0], outs[1]) and torch.equal(lses[0], lses[1]), (seed, st)
+        if st == replan:
+            for c, p in zip((plain, paged), plans):
+                ck.catekv_decode_plan(c, p)
+    ref, ref_lse = orc.decode_attention(oc, synth.bits(q))
+    H.check_attention(outs[1], None, lses[1], ref, ref_lse, f"paged seed {seed} lens {lens} steps {steps}")
+    assert paged.seg_len_dev.cpu().tolist() == [l + steps for l in lens]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_retrieval_in_place_equals_gather(ck, seed):
+    rng = np.random.default_rng(8000 + seed)
+    B, Hkv = int(rng.integers(1, 3)), int(rng.integers(1, 4))
+    G = int(rng.choice([1, 2, 4, 7]))
+    cs = int(rng.choice([1, 4, 8, 16]))
+    lens = [int(rng.integers(0, 3000)) for _ in range(B * Hkv)]
+    budget = int(rng.integers(64, 600))
+    sink, local = int(rng.integers(0, 9)), int(rng.integers(0, 48))
+    mask = rng.integers(0, 2, size=B * Hkv).astype(np.uint8)
+    num_ctas = int(rng.choice([1, 5, 296]))
+    oc = H.random_cache(B, Hkv, lens, seed=8100 + seed)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=2)
+    meta = ck.catekv_retrieval_meta(cache, cs)
+    ck.catekv_retrieval_build(cache, cs, meta)
+    kn = synth.randn_bf16((B, Hkv, 128), "cuda", 8200 + seed, "kn")
+    vn = synth.randn_bf16((B, Hkv, 128), "cuda", 8200 + seed, "vn")
+    q = synth.randn_bf16((B, Hkv * G, 128), "cuda", 8200 + seed, "q")
+    ck.catekv_append_retrieval(cache, kn, vn, cs, meta)
+    oc.append(synth.bits(kn), synth.bits(vn))
+    want = ck.catekv_retrieve_lengths(cache, cs, mask, budget, sink, local)
+    idx = torch.full((B * Hkv, max(int(want.max()), 1)), -1, dtype=torch.int32, device="cuda")
+    sel = torch.empty(B * Hkv, dtype=torch.int32, device="cuda")
+    ck.catekv_retrieve_select(cache, meta, cs, q, mask, budget, sink, local, idx, sel)
+    view = ck.CacheView(cache, want)
+    plan = ck.DecodePlan(view, num_ctas)
+    ck.catekv_decode_plan(view, plan)
+    out = torch.empty((B, Hkv * G, 128), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, Hkv * G), dtype=torch.float32, device="cuda")
+    ck.catekv_decode_attn_indexed(cache, idx, sel, q, plan, out, lse)
+    step = ck.Cache(B, Hkv, want, 0, "cuda")
+    gidx = torch.full((B * Hkv, max(max(lens) + 1, 1)), -1, dtype=torch.int32, device="cuda")
+    ck.catekv_retrieve_compact(cache, meta, cs, q, mask, budget, sink, local, step, idx_out=gidx)
+    plan2 = ck.DecodePlan(step, num_ctas)
+    ck.catekv_decode_plan(step, plan2)
+    out2, lse2 = torch.empty_like(out), torch.empty_like(lse)
+    ck.catekv_decode_attn(step, q, plan2, out2, lse2)
+    torch.cuda.synchronize()
+    assert list(step.seg_len) == list(want)
+    assert torch.equal(out, out2) and torch.equal(lse, lse2), seed
+    # the oracle on the device's own lists
+    soc = orc.HybridCache(B, Hkv, 128)
+    g = gidx.cpu().numpy()
+    for s in range(B * Hkv):
+        rows = g[s, :want[s]].astype(np.int64)
+        soc.k_rows.append(oc.k_rows[s][rows])
+        soc.v_rows.append(oc.v_rows[s][rows])
+    ref, ref_lse = orc.decode_attention(soc, synth.bits(q))
+    H.check_attention(out, None, lse, ref, ref_lse, f"retrieval seed {seed} lens {lens} cs {cs} budget {budget}")
