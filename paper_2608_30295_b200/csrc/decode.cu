@@ -1,5 +1,5 @@
-// Decoding stage of Algorithm 1: append, work-balanced split-KV schedule, attention partials
-// and the combine pass, for per-(sequence, KV head) variable-length caches.
+// Decoding stage of Algorithm 1: the split-KV attention partials and the combine pass over per-(sequence, KV head)
+// variable-length caches (the schedule is built in plan.cu, the lists grow in cache.cu).
 //
 // The attention kernel is a memory-bound stream over the K and V rows of the cache.  Each CTA
 // owns a contiguous range of the rows of all segments laid end to end (so short consistent
@@ -10,78 +10,10 @@
 // warp in fp32, and P enters the P.V product as a bf16 hi + lo pair so that no precision of
 // the fp32 probabilities is lost.
 #include <math.h>
-#include <string.h>
 
-#include "common.cuh"
+#include "decode.cuh"
 
 namespace catekv {
-
-// ------------------------------------------------------------------------------------------
-// Plan (host)
-// ------------------------------------------------------------------------------------------
-constexpr uint32_t kPlanMagic = 0x43544B56u;  // "CTKV"
-constexpr int kTile = 64;                     // rows per pipeline stage
-constexpr int kDecodeWarps = kTile / 16;
-constexpr int kDecodeThreads = kDecodeWarps * 32;
-constexpr int kStages = 3;
-constexpr int kSplitAlign = 16;               // CTA ranges are cut at multiples of this many rows
-
-struct PlanHeader {
-  uint32_t magic;
-  int32_t num_ctas;
-  int32_t n_segs;
-  int32_t n_items;
-  int32_t n_slots;
-  int32_t tile;
-  int64_t total_rows;
-  int32_t off_cta, off_items, off_seg;  // byte offsets of the three tables
-  int32_t max_pieces;                   // most pieces any segment was cut into
-};
-static_assert(sizeof(PlanHeader) == 48, "plan header layout");
-
-struct WorkItem {  // 32 bytes
-  int32_t seg;
-  int32_t t0;        // first row of the piece, relative to the segment
-  int32_t t1;        // one past its last row at plan time
-  int32_t slot;      // partial slot, or -1 when the piece is the whole segment (final output written directly)
-  int64_t row_base;  // pool row of t0 (segment offset + t0)
-  int32_t last;      // 1: last piece of its segment; it also covers rows [t1, current length)
-  int32_t cap;       // capacity of the segment in the cache's own pools (rows from there on live in overflow pages)
-};
-static_assert(sizeof(WorkItem) == 32, "work item layout");
-struct CtaHeader {  // 48 bytes: the CTA's item range and a copy of its first item (one load starts the stream)
-  int32_t item_begin, item_end, reserved0, reserved1;
-  WorkItem first;
-};
-static_assert(sizeof(CtaHeader) == 48, "cta header layout");
-struct SegInfo {
-  int32_t slot_begin;
-  int32_t n_pieces;
-  int32_t plan_len;  // rows the segment held when the plan was built
-  int32_t reserved;
-};
-
-struct PlanLayout {
-  size_t off_cta, off_items, off_seg, bytes;
-  int n_items_cap;
-};
-static PlanLayout plan_layout(int n_segs, int num_ctas) {
-  PlanLayout L;
-  L.n_items_cap = num_ctas + n_segs;
-  L.off_cta = sizeof(PlanHeader);
-  L.off_items = align_up(L.off_cta + sizeof(CtaHeader) * (size_t)num_ctas, 32);
-  L.off_seg = L.off_items + sizeof(WorkItem) * (size_t)L.n_items_cap;
-  L.bytes = align_up(L.off_seg + sizeof(SegInfo) * (size_t)n_segs, 16);
-  return L;
-}
-
-constexpr size_t kPartOBytes = (size_t)kMaxG * kD * sizeof(float);  // one partial: 8 heads x 128 floats
-static size_t ws_layout(int n_segs, int num_ctas, size_t* off_lse) {
-  size_t slots = (size_t)num_ctas + n_segs;
-  size_t o = slots * kPartOBytes;
-  if (off_lse) *off_lse = o;
-  return o + slots * kMaxG * sizeof(float);
-}
 
 // ------------------------------------------------------------------------------------------
 // Attention partials
@@ -118,7 +50,6 @@ struct DecodeArgs {
 
 constexpr int kStageBytes = 2 * kTile * kRowBytes;     // K tile + V tile
 constexpr int kQSlotBytes = kMaxG * kRowBytes;         // 8 query rows
-constexpr int kSegEndCharge = 320;                     // plan: rows charged to the CTA that owns a segment's end
 constexpr int kMergeRegs = 36;                         // 32 accumulators + m0, m1, l0, l1
 constexpr int kMergeSlotBytes = kMergeRegs * 32 * 4;
 constexpr int kDecodeSmem = kStages * (kStageBytes + kQSlotBytes) + 2 * kMergeSlotBytes;
@@ -656,202 +587,9 @@ __global__ void __launch_bounds__(kCombineWarps * 32) decode_combine_kernel(cons
   }
 }
 
-// ------------------------------------------------------------------------------------------
-// Append
-// ------------------------------------------------------------------------------------------
-struct PageArgs {  // overflow pages of a cache (all null / 0 without pages)
-  uint8_t* k_ovf;
-  uint8_t* v_ovf;
-  const int32_t* table;
-  const int32_t* seg_cap;
-  int32_t max_pages;
-};
-static PageArgs page_args(const catekv_cache* c) {
-  PageArgs p = {nullptr, nullptr, nullptr, nullptr, 0};
-  if (c->pages) {
-    p.k_ovf = (uint8_t*)c->pages->k_ovf;
-    p.v_ovf = (uint8_t*)c->pages->v_ovf;
-    p.table = c->pages->table_dev;
-    p.seg_cap = c->pages->seg_cap_dev;
-    p.max_pages = c->pages->max_pages;
-  }
-  return p;
-}
-
-__global__ void __launch_bounds__(128) append_kernel(uint8_t* k_pool, uint8_t* v_pool, const int32_t* seg_off,
-                                                     int32_t* seg_len, const uint8_t* k_new, const uint8_t* v_new,
-                                                     int n_segs, const PageArgs pg) {
-  const int seg = blockIdx.x * 4 + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  pdl_launch_dependents();
-  pdl_wait();
-  if (seg >= n_segs) return;
-  const int len = seg_len[seg];
-  int64_t row = (int64_t)seg_off[seg] + len;
-  if (pg.table && len >= pg.seg_cap[seg]) {  // the row goes to an overflow page
-    const int o = len - pg.seg_cap[seg];
-    row = (int64_t)pg.table[(int64_t)seg * pg.max_pages + (o >> 6)] * 64 + (o & 63);
-    k_pool = pg.k_ovf;
-    v_pool = pg.v_ovf;
-  }
-  const int c = lane & 15;
-  const uint8_t* src = (lane < 16 ? k_new : v_new) + (size_t)seg * kRowBytes + c * 16;
-  uint8_t* dst = (lane < 16 ? k_pool : v_pool) + row * kRowBytes + c * 16;
-  *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
-  __syncwarp();
-  if (lane == 0) seg_len[seg] = len + 1;
-}
-
-static int check_cache(const catekv_cache* c) {
-  if (!c) return CATEKV_ERR_INVALID_ARG;
-  if (c->B <= 0 || c->Hkv <= 0 || c->total_rows < 0) return CATEKV_ERR_INVALID_ARG;
-  if (c->d != kD) return CATEKV_ERR_UNSUPPORTED;
-  if (!c->k_pool || !c->v_pool || !c->seg_off_dev || !c->seg_len_dev || !c->seg_off || !c->seg_cap || !c->seg_len)
-    return CATEKV_ERR_INVALID_ARG;
-  if (c->pages) {
-    const catekv_pages* p = c->pages;
-    if (p->max_pages <= 0 || p->n_pages < 0 || p->next_free < 0 || p->next_free > p->n_pages) return CATEKV_ERR_INVALID_ARG;
-    if (!p->k_ovf || !p->v_ovf || !p->table_dev || !p->table || !p->seg_pages || !p->seg_cap_dev) return CATEKV_ERR_INVALID_ARG;
-  }
-  return CATEKV_OK;
-}
-// rows segment s can hold: its own capacity plus the overflow pages it has been given
-static inline int64_t seg_capacity(const catekv_cache* c, int s) {
-  return (int64_t)c->seg_cap[s] + (c->pages ? (int64_t)c->pages->seg_pages[s] * CATEKV_PAGE_ROWS : 0);
-}
-
 }  // namespace catekv
 
 using namespace catekv;
-
-extern "C" int catekv_append(catekv_cache* cache, const void* k_new, const void* v_new, catekv_stream stream) {
-  int rc = check_cache(cache);
-  if (rc) return rc;
-  if (!k_new || !v_new) return CATEKV_ERR_INVALID_ARG;
-  const int n = cache->B * cache->Hkv;
-  for (int s = 0; s < n; ++s) {
-    if (cache->seg_len[s] < 0) return CATEKV_ERR_INVALID_ARG;
-    if (cache->seg_len[s] + 1 > seg_capacity(cache, s)) return CATEKV_ERR_CAPACITY;
-  }
-  CATEKV_CUDA_TRY(launch_pdl(append_kernel, dim3((n + 3) / 4), dim3(128), 0, (cudaStream_t)stream,
-                             (uint8_t*)cache->k_pool, (uint8_t*)cache->v_pool, cache->seg_off_dev, cache->seg_len_dev,
-                             (const uint8_t*)k_new, (const uint8_t*)v_new, n, page_args(cache)));
-  for (int s = 0; s < n; ++s) cache->seg_len[s] += 1;
-  return CATEKV_OK;
-}
-
-// recall = exp(lse_kept - lse_full): the share of the full attention mass that falls on the kept rows
-__global__ void recall_kernel(const float* lse_kept, const float* lse_full, float* recall, int n) {
-  pdl_launch_dependents();
-  pdl_wait();
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) recall[i] = (lse_kept[i] == -INFINITY) ? 0.f : expf(lse_kept[i] - lse_full[i]);
-}
-
-extern "C" int catekv_attention_recall(const float* lse_kept, const float* lse_full, float* recall, int32_t n,
-                                       catekv_stream stream) {
-  if (!lse_kept || !lse_full || !recall || n < 0) return CATEKV_ERR_INVALID_ARG;
-  if (n == 0) return CATEKV_OK;
-  CATEKV_CUDA_TRY(launch_pdl(recall_kernel, dim3((n + 255) / 256), dim3(256), 0, (cudaStream_t)stream, lse_kept, lse_full,
-                             recall, (int)n));
-  return CATEKV_OK;
-}
-
-extern "C" int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens) {
-  int rc = check_cache(cache);
-  if (rc) return rc;
-  if (n_tokens < 0) return CATEKV_ERR_INVALID_ARG;
-  const int n = cache->B * cache->Hkv;
-  for (int s = 0; s < n; ++s)
-    if ((int64_t)cache->seg_len[s] + n_tokens > seg_capacity(cache, s)) return CATEKV_ERR_CAPACITY;
-  for (int s = 0; s < n; ++s) cache->seg_len[s] += n_tokens;
-  return CATEKV_OK;
-}
-
-// Growth: every segment's valid rows move to the same segment of a cache with larger capacities.  One warp per
-// row (lanes 0-15 the K row, 16-31 the V row); block 0 of a segment records its length.
-namespace catekv {
-constexpr int kRegrowRowsPerBlock = 64;
-__global__ void __launch_bounds__(256) regrow_kernel(const uint8_t* sk, const uint8_t* sv, const int32_t* s_off,
-                                                     const int32_t* s_len, uint8_t* dk, uint8_t* dv, const int32_t* d_off,
-                                                     int32_t* d_len, const PageArgs pg) {
-  const int seg = blockIdx.y;
-  const int len = s_len[seg];
-  if (blockIdx.x == 0 && threadIdx.x == 0) d_len[seg] = len;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint8_t* src = (lane < 16 ? sk : sv) + (int64_t)s_off[seg] * kRowBytes + (lane & 15) * 16;
-  const uint8_t* ovf = (lane < 16 ? pg.k_ovf : pg.v_ovf) + (lane & 15) * 16;
-  const int cap = pg.table ? pg.seg_cap[seg] : 0x7fffffff;  // rows from here on come from the source's overflow pages
-  uint8_t* dst = (lane < 16 ? dk : dv) + (int64_t)d_off[seg] * kRowBytes + (lane & 15) * 16;
-  const int r0 = blockIdx.x * kRegrowRowsPerBlock;
-#pragma unroll 4
-  for (int i = warp; i < kRegrowRowsPerBlock; i += 8) {
-    const int r = r0 + i;
-    if (r >= len) break;
-    const uint8_t* from = src + (int64_t)r * kRowBytes;
-    if (r >= cap) {
-      const int o = r - cap;
-      from = ovf + ((int64_t)pg.table[(int64_t)seg * pg.max_pages + (o >> 6)] * 64 + (o & 63)) * kRowBytes;
-    }
-    *reinterpret_cast<uint4*>(dst + (int64_t)r * kRowBytes) = __ldg(reinterpret_cast<const uint4*>(from));
-  }
-}
-}  // namespace catekv
-
-extern "C" int catekv_pages_reserve(catekv_cache* cache, int32_t n_new, catekv_stream stream) {
-  int rc = check_cache(cache);
-  if (rc) return rc;
-  if (!cache->pages || n_new < 0) return CATEKV_ERR_INVALID_ARG;
-  catekv_pages* p = cache->pages;
-  const int n = cache->B * cache->Hkv;
-  // first pass: what is needed, nothing changed yet
-  int64_t extra = 0;
-  for (int s = 0; s < n; ++s) {
-    if (cache->seg_len[s] < 0 || cache->seg_len[s] > seg_capacity(cache, s)) return CATEKV_ERR_INVALID_ARG;
-    const int64_t over = (int64_t)cache->seg_len[s] + n_new - cache->seg_cap[s];
-    const int64_t want = over > 0 ? (over + CATEKV_PAGE_ROWS - 1) / CATEKV_PAGE_ROWS : 0;
-    if (want > p->max_pages) return CATEKV_ERR_CAPACITY;
-    if (want > p->seg_pages[s]) extra += want - p->seg_pages[s];
-  }
-  if (extra > (int64_t)p->n_pages - p->next_free) return CATEKV_ERR_CAPACITY;
-  for (int s = 0; s < n; ++s) {
-    const int64_t over = (int64_t)cache->seg_len[s] + n_new - cache->seg_cap[s];
-    const int want = over > 0 ? (int)((over + CATEKV_PAGE_ROWS - 1) / CATEKV_PAGE_ROWS) : 0;
-    const int have = p->seg_pages[s];
-    if (want <= have) continue;
-    int32_t* row = p->table + (size_t)s * p->max_pages;
-    for (int q = have; q < want; ++q) row[q] = p->next_free++;
-    p->seg_pages[s] = want;
-    CATEKV_CUDA_TRY(cudaMemcpyAsync(p->table_dev + (size_t)s * p->max_pages + have, row + have,
-                                    sizeof(int32_t) * (size_t)(want - have), cudaMemcpyHostToDevice, (cudaStream_t)stream));
-  }
-  return CATEKV_OK;
-}
-
-extern "C" int catekv_cache_regrow(const catekv_cache* src, catekv_cache* dst, catekv_stream stream) {
-  int rc = check_cache(src);
-  if (rc) return rc;
-  rc = check_cache(dst);
-  if (rc) return rc;
-  if (src->B != dst->B || src->Hkv != dst->Hkv) return CATEKV_ERR_INVALID_ARG;
-  if (src->k_pool == dst->k_pool || src->v_pool == dst->v_pool) return CATEKV_ERR_INVALID_ARG;
-  if (dst->pages) return CATEKV_ERR_UNSUPPORTED;  // the destination is one contiguous segment per (sequence, head)
-  const int n = src->B * src->Hkv;
-  int max_len = 0;
-  for (int s = 0; s < n; ++s) {
-    if (src->seg_len[s] < 0 || src->seg_len[s] > seg_capacity(src, s)) return CATEKV_ERR_INVALID_ARG;
-    if (src->seg_len[s] > dst->seg_cap[s]) return CATEKV_ERR_CAPACITY;
-    max_len = src->seg_len[s] > max_len ? src->seg_len[s] : max_len;
-  }
-  const int gx = max_len > 0 ? (max_len + kRegrowRowsPerBlock - 1) / kRegrowRowsPerBlock : 1;
-  regrow_kernel<<<dim3(gx, n), 256, 0, (cudaStream_t)stream>>>((const uint8_t*)src->k_pool, (const uint8_t*)src->v_pool,
-                                                               src->seg_off_dev, src->seg_len_dev, (uint8_t*)dst->k_pool,
-                                                               (uint8_t*)dst->v_pool, dst->seg_off_dev, dst->seg_len_dev,
-                                                               page_args(src));
-  CATEKV_CUDA_TRY(cudaGetLastError());
-  for (int s = 0; s < n; ++s) dst->seg_len[s] = src->seg_len[s];
-  return CATEKV_OK;
-}
 
 extern "C" int catekv_decode_num_ctas(void) {
   int dev = 0, sms = 0, per_sm = 0;
@@ -864,110 +602,6 @@ extern "C" int catekv_decode_num_ctas(void) {
   if (e != cudaSuccess) { set_cuda_error(e); return CATEKV_ERR_CUDA; }
   if (per_sm < 1) per_sm = 1;
   return sms * per_sm;
-}
-
-extern "C" size_t catekv_decode_plan_bytes(int32_t B, int32_t Hkv, int32_t num_ctas) {
-  if (B <= 0 || Hkv <= 0 || num_ctas <= 0) return 0;
-  return plan_layout(B * Hkv, num_ctas).bytes;
-}
-
-extern "C" size_t catekv_decode_workspace_bytes(int32_t B, int32_t Hkv, int32_t num_ctas) {
-  if (B <= 0 || Hkv <= 0 || num_ctas <= 0) return 0;
-  return ws_layout(B * Hkv, num_ctas, nullptr);
-}
-
-extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, void* plan_host, void* plan_dev,
-                                  size_t plan_bytes, catekv_stream stream) {
-  int rc = check_cache(cache);
-  if (rc) return rc;
-  if (num_ctas <= 0 || !plan_host) return CATEKV_ERR_INVALID_ARG;
-  const int n_segs = cache->B * cache->Hkv;
-  const PlanLayout L = plan_layout(n_segs, num_ctas);
-  if (plan_bytes < L.bytes) return CATEKV_ERR_WORKSPACE;
-  // The CTA that owns the end of a segment does more than stream rows: it streams one more tile (the rows appended
-  // since the plan was built), stores the appended row, and finishes one piece and starts the next (merge of the
-  // warps, output, the next group's queries).  Every non-empty segment's end is therefore charged kSegEndCharge
-  // rows, so that those CTAs get fewer plan-time rows and do not finish last.  Measured per-CTA stream times put
-  // the cost of a segment end at 290-330 rows' worth of streaming; between a charge of 64 and of 320 rows
-  // configs[1] went from 19.7 to 17.3 us and configs[2] from 36.3 to 34.2 us per layer-step (flat from 256 to 512).
-  int64_t total = 0, charged = 0;
-  for (int s = 0; s < n_segs; ++s) {
-    if (cache->seg_len[s] < 0 || cache->seg_len[s] > seg_capacity(cache, s)) return CATEKV_ERR_INVALID_ARG;
-    total += cache->seg_len[s];
-    charged += cache->seg_len[s] + (cache->seg_len[s] > 0 ? kSegEndCharge : 0);
-  }
-  uint8_t* base = (uint8_t*)plan_host;
-  memset(base, 0, L.bytes);
-  PlanHeader* hdr = (PlanHeader*)base;
-  CtaHeader* ctas = (CtaHeader*)(base + L.off_cta);
-  WorkItem* items = (WorkItem*)(base + L.off_items);
-  SegInfo* segs = (SegInfo*)(base + L.off_seg);
-
-  // rows per CTA: an equal share of all (charged) rows, rounded up to the split alignment
-  int64_t quota = (charged + num_ctas - 1) / num_ctas;
-  quota = (quota + kSplitAlign - 1) / kSplitAlign * kSplitAlign;
-  if (quota < kSplitAlign) quota = kSplitAlign;
-
-  int n_items = 0, n_slots = 0, max_pieces = 1;
-  int seg = 0;
-  int32_t pos = 0;  // next unassigned row of `seg`
-  int seg_first_item = 0;
-  for (int c = 0; c < num_ctas; ++c) {
-    ctas[c].item_begin = n_items;
-    int64_t room = quota;
-    while (seg < n_segs) {
-      const int32_t len = cache->seg_len[seg];
-      if (len == 0) {
-        // an empty segment still gets one (direct) item, so that the plan stays valid once it grows
-        items[n_items++] = WorkItem{seg, 0, 0, -1, (int64_t)cache->seg_off[seg], 1, cache->seg_cap[seg]};
-        segs[seg] = SegInfo{0, 1, 0, 0};
-        ++seg;
-        seg_first_item = n_items;
-        continue;
-      }
-      if (room <= 0) break;
-      const int32_t take = (int32_t)((int64_t)(len - pos) < room ? (len - pos) : room);
-      items[n_items++] = WorkItem{seg, pos, pos + take, 0, (int64_t)cache->seg_off[seg] + pos, 0, cache->seg_cap[seg]};
-      pos += take;
-      room -= take;
-      if (pos == len) {
-        // segment finished: fix up its pieces
-        const int pieces = n_items - seg_first_item;
-        items[n_items - 1].last = 1;  // the last piece follows the segment's current length
-        if (pieces == 1) {
-          items[seg_first_item].slot = -1;
-          segs[seg] = SegInfo{0, 1, len, 0};
-        } else {
-          for (int i = 0; i < pieces; ++i) items[seg_first_item + i].slot = n_slots + i;
-          segs[seg] = SegInfo{n_slots, pieces, len, 0};
-          n_slots += pieces;
-          max_pieces = pieces > max_pieces ? pieces : max_pieces;
-        }
-        ++seg;
-        pos = 0;
-        seg_first_item = n_items;
-        room -= kSegEndCharge;
-      }
-    }
-    ctas[c].item_end = n_items;
-  }
-  if (seg != n_segs) return CATEKV_ERR_INVALID_ARG;  // cannot happen: quota * num_ctas >= the charged rows
-  for (int c = 0; c < num_ctas; ++c)
-    if (ctas[c].item_begin < ctas[c].item_end) ctas[c].first = items[ctas[c].item_begin];
-  hdr->magic = kPlanMagic;
-  hdr->num_ctas = num_ctas;
-  hdr->n_segs = n_segs;
-  hdr->n_items = n_items;
-  hdr->n_slots = n_slots;
-  hdr->tile = kTile;
-  hdr->total_rows = total;
-  hdr->off_cta = (int32_t)L.off_cta;
-  hdr->off_items = (int32_t)L.off_items;
-  hdr->off_seg = (int32_t)L.off_seg;
-  hdr->max_pieces = max_pieces;
-  if (plan_dev)
-    CATEKV_CUDA_TRY(cudaMemcpyAsync(plan_dev, plan_host, L.bytes, cudaMemcpyHostToDevice, (cudaStream_t)stream));
-  return CATEKV_OK;
 }
 
 // phases: 1 = attention partials, 2 = combine, 3 = both
