@@ -54,14 +54,16 @@ constexpr int kMergeRegs = 36;                         // 32 accumulators + m0, 
 constexpr int kMergeSlotBytes = kMergeRegs * 32 * 4;
 constexpr int kDecodeSmem = kStages * (kStageBytes + kQSlotBytes) + 2 * kMergeSlotBytes;
 
-// A piece is streamed as tiles of its plan-time rows [t0, t1), followed - for the last piece of a
-// segment - by tiles of the rows appended since the plan was built, [t1, live length).  The live length
-// is loaded when the item is read but first used only after the plan-time tiles have been issued, so
-// the stream never waits for that load.
+// A piece is streamed as 64-row tiles of its rows [t0, live): live is t1 for an inner piece of a segment (or less,
+// if the segment has shrunk) and the segment's current length for its last piece, which so also covers the rows
+// appended since the plan was built - they continue the piece's last, partly filled plan-time tile.  The live
+// length is loaded when the item is read but first used only after the tiles that hold nothing but plan-time rows
+// (np of them: these may be requested before the dependency wait) have been issued, so the stream never waits
+// for that load.
 constexpr int kModePlain = 0, kModeIndexed = 1, kModePaged = 2;  // instantiations of the attention kernel
 struct ItemCursor {
   int seg, t0, t1, slot, last;
-  int np;            // tiles of the plan-time rows
+  int np;            // leading tiles that hold only plan-time rows
   int live;          // rows to attend to: current segment length (plus the row being appended), if last
   int new_row;       // fused append: the segment-relative row that comes from k_new / v_new, else -1
   int indexed;       // indexed variant: the item's rows are taken through the index list
@@ -78,7 +80,8 @@ __device__ __forceinline__ ItemCursor plan_cursor(const WorkItem& w) {
   c.slot = w.slot;
   c.last = w.last;
   c.row_base = w.row_base;
-  c.np = (w.t1 - w.t0 + kTile - 1) / kTile;
+  // tiles of plan-time rows only; the last piece's partly filled tile is left to the live length
+  c.np = w.last ? (w.t1 - w.t0) / kTile : (w.t1 - w.t0 + kTile - 1) / kTile;
   c.live = w.t1;
   c.new_row = -1;
   c.indexed = 0;
@@ -119,21 +122,15 @@ __device__ __forceinline__ ItemCursor read_item(const DecodeArgs& a, int it) {
   live_cursor<kMode>(a, c);
   return c;
 }
-// tiles of the item: plan-time tiles plus tiles of the appended rows; at least one
+// tiles of the item's live rows; at least one
 __device__ __forceinline__ int item_tiles(const ItemCursor& c) {
-  const int extra = c.live - c.t1;
-  const int ne = extra > 0 ? (extra + kTile - 1) / kTile : 0;
-  return max(1, c.np + ne);
+  return max(1, (c.live - c.t0 + kTile - 1) / kTile);
 }
-// first row (relative to the segment) and number of valid rows of tile i
+// first row (relative to the segment) and number of valid rows of tile i (may exceed kTile, or be <= 0 for a tile
+// that lies behind the live length)
 __device__ __forceinline__ void tile_rows(const ItemCursor& c, int i, int& start, int& nvalid) {
-  if (i < c.np) {
-    start = c.t0 + i * kTile;
-    nvalid = min(c.t1, c.live) - start;  // <= 0: the whole tile lies behind the live length
-  } else {
-    start = c.t1 + (i - c.np) * kTile;
-    nvalid = c.live - start;
-  }
+  start = c.t0 + i * kTile;
+  nvalid = c.live - start;
 }
 
 #ifdef CATEKV_TRACE
@@ -207,7 +204,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       }
       const int64_t goff = grow * kRowBytes + c * 16;
       const uint32_t so = tile_off(r, c);
-      if (ok && r == new_r && pc.new_row >= 0) {  // only inside the tile's valid rows (never in a plan-time tile)
+      if (ok && r == new_r && pc.new_row >= 0) {  // only inside the tile's valid rows (never in one of the np tiles)
         // the decoded token's row: attend to it from k_new / v_new and store it in the pool
         const size_t noff = (size_t)pc.seg * kRowBytes + c * 16;
         cp_async16(sb + so, a.k_new + noff, 16);

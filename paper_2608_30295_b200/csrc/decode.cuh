@@ -16,7 +16,7 @@ constexpr int kDecodeWarps = kTile / 16;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kStages = 3;
 constexpr int kSplitAlign = 16;               // CTA ranges are cut at multiples of this many rows
-constexpr int kSegEndCharge = 320;            // rows charged to the CTA that owns a segment's end (see catekv_decode_plan)
+constexpr int kSegEndCharge = 256;            // rows charged to the CTA that owns a segment's end (see catekv_decode_plan)
 
 struct PlanHeader {
   uint32_t magic;

@@ -21,12 +21,13 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
   const int n_segs = cache->B * cache->Hkv;
   const PlanLayout L = plan_layout(n_segs, num_ctas);
   if (plan_bytes < L.bytes) return CATEKV_ERR_WORKSPACE;
-  // The CTA that owns the end of a segment does more than stream rows: it streams one more tile (the rows appended
-  // since the plan was built), stores the appended row, and finishes one piece and starts the next (merge of the
-  // warps, output, the next group's queries).  Every non-empty segment's end is therefore charged kSegEndCharge
-  // rows, so that those CTAs get fewer plan-time rows and do not finish last.  Measured per-CTA stream times put
-  // the cost of a segment end at 290-330 rows' worth of streaming; between a charge of 64 and of 320 rows
-  // configs[1] went from 19.7 to 17.3 us and configs[2] from 36.3 to 34.2 us per layer-step (flat from 256 to 512).
+  // The CTA that owns the end of a segment does more than stream rows: its last tile also takes the rows appended
+  // since the plan was built, it stores the appended row, and it finishes one piece and starts the next (merge of
+  // the warps, output, the next group's queries) while nothing new is issued.  Every non-empty segment's end is
+  // therefore charged kSegEndCharge rows, so that those CTAs get fewer plan-time rows and do not finish last.
+  // Measured per-CTA stream times put the cost of a segment end at 250-330 rows' worth of streaming; between a
+  // charge of 64 and of 256 rows configs[1] went from 19.7 to 17.1 us and configs[2] from 36.3 to 34.0 us per
+  // layer-step (flat from 256 to 512).
   int64_t total = 0, charged = 0;
   for (int s = 0; s < n_segs; ++s) {
     if (cache->seg_len[s] < 0 || cache->seg_len[s] > seg_capacity(cache, s)) return CATEKV_ERR_INVALID_ARG;

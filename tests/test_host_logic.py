@@ -117,9 +117,9 @@ def test_decode_plan_covers_every_row_once_and_balances(ck, lens, num_ctas):
         elif npieces > 1:
             assert [sl for (_, _, sl) in pieces[s]] == list(range(sb, sb + npieces))
     assert n_slots == sum(len(p) for p in pieces.values() if len(p) > 1)
-    # balance: every non-empty segment's end is charged 320 rows (the extra work of the CTA that owns it);
+    # balance: every non-empty segment's end is charged 256 rows (the extra work of the CTA that owns it);
     # no CTA gets more than an equal share of the charged rows rounded up to 16 (a charge may overshoot it)
-    charge = 320
+    charge = 256
     charged = sum(lens) + charge * sum(1 for x in lens if x > 0)
     quota = max(16, -(-(-(-charged // num_ctas)) // 16) * 16)
     for c in range(num_ctas):
