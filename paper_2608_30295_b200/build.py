@@ -30,7 +30,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-shared", "-Xcompiler", "-fPIC", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3",
            "-std=c++17", "-DCATEKV_BUILD", "-I", os.path.join(ROOT, "include"),
-           "-I", os.path.join(HERE, "csrc"), "-o", LIB]
+           "-I", os.path.join(HERE, "csrc"), "-o", LIB, "-ldl"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += sources()

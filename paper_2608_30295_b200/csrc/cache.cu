@@ -35,6 +35,7 @@ __global__ void __launch_bounds__(128) append_kernel(uint8_t* k_pool, uint8_t* v
 using namespace catekv;
 
 extern "C" int catekv_append(catekv_cache* cache, const void* k_new, const void* v_new, catekv_stream stream) {
+  CATEKV_API_RANGE();
   int rc = check_cache(cache);
   if (rc) return rc;
   if (!k_new || !v_new) return CATEKV_ERR_INVALID_ARG;
@@ -60,6 +61,7 @@ __global__ void recall_kernel(const float* lse_kept, const float* lse_full, floa
 
 extern "C" int catekv_attention_recall(const float* lse_kept, const float* lse_full, float* recall, int32_t n,
                                        catekv_stream stream) {
+  CATEKV_API_RANGE();
   if (!lse_kept || !lse_full || !recall || n < 0) return CATEKV_ERR_INVALID_ARG;
   if (n == 0) return CATEKV_OK;
   CATEKV_CUDA_TRY(launch_pdl(recall_kernel, dim3((n + 255) / 256), dim3(256), 0, (cudaStream_t)stream, lse_kept, lse_full,
@@ -109,6 +111,7 @@ __global__ void __launch_bounds__(256) regrow_kernel(const uint8_t* sk, const ui
 }  // namespace catekv
 
 extern "C" int catekv_pages_reserve(catekv_cache* cache, int32_t n_new, catekv_stream stream) {
+  CATEKV_API_RANGE();
   int rc = check_cache(cache);
   if (rc) return rc;
   if (!cache->pages || n_new < 0) return CATEKV_ERR_INVALID_ARG;
@@ -139,6 +142,7 @@ extern "C" int catekv_pages_reserve(catekv_cache* cache, int32_t n_new, catekv_s
 }
 
 extern "C" int catekv_cache_regrow(const catekv_cache* src, catekv_cache* dst, catekv_stream stream) {
+  CATEKV_API_RANGE();
   int rc = check_cache(src);
   if (rc) return rc;
   rc = check_cache(dst);

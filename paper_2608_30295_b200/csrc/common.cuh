@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "catekv.h"
 
 namespace catekv {
@@ -44,6 +46,15 @@ static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 b
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
+
+// ---- host: an NVTX range per entry point (named after the function; costs nothing without a profiler attached)
+struct ApiRange {
+  explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+  ~ApiRange() { nvtxRangePop(); }
+  ApiRange(const ApiRange&) = delete;
+  ApiRange& operator=(const ApiRange&) = delete;
+};
+#define CATEKV_API_RANGE() ::catekv::ApiRange catekv_api_range_(__func__)
 
 // ---- device: programmatic dependent launch ------------------------------------------------
 // Let the next kernel of the stream be scheduled (it still waits, in pdl_wait, for this grid to finish).

@@ -699,6 +699,7 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* k_ne
 extern "C" int catekv_decode_attn(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
                                   int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                                   size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+  CATEKV_API_RANGE();
   return decode_launch(3, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
                        ws_bytes, stream);
 }
@@ -707,6 +708,7 @@ extern "C" int catekv_decode_attn_indexed(const catekv_cache* cache, const int32
                                           const int32_t* sel_len, const void* q, int32_t Hq, float sm_scale, void* out,
                                           int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                                           size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+  CATEKV_API_RANGE();
   if (!idx || !sel_len || idx_stride < 0) return CATEKV_ERR_INVALID_ARG;
   if (cache && cache->pages) return CATEKV_ERR_UNSUPPORTED;
   const IndexList il = {idx, idx_stride, sel_len};
@@ -717,6 +719,7 @@ extern "C" int catekv_decode_attn_indexed(const catekv_cache* cache, const int32
 extern "C" int catekv_decode_partials(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
                                       int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                                       size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+  CATEKV_API_RANGE();
   return decode_launch(1, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
                        ws_bytes, stream);
 }
@@ -724,6 +727,7 @@ extern "C" int catekv_decode_partials(const catekv_cache* cache, const void* q, 
 extern "C" int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale, void* out,
                                      int32_t out_dtype, float* lse_out, const void* plan_host, const void* plan_dev,
                                      size_t plan_bytes, void* ws, size_t ws_bytes, catekv_stream stream) {
+  CATEKV_API_RANGE();
   return decode_launch(2, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes, ws,
                        ws_bytes, stream);
 }
@@ -732,6 +736,7 @@ extern "C" int catekv_append_decode_attn(catekv_cache* cache, const void* k_new,
                                          int32_t Hq, float sm_scale, void* out, int32_t out_dtype, float* lse_out,
                                          const void* plan_host, const void* plan_dev, size_t plan_bytes, void* ws,
                                          size_t ws_bytes, catekv_stream stream) {
+  CATEKV_API_RANGE();
   int rc = check_cache(cache);
   if (rc) return rc;
   if (!k_new || !v_new) return CATEKV_ERR_INVALID_ARG;
@@ -771,6 +776,7 @@ static __device__ __align__(256) unsigned char g_decode_noalloc_scratch[CATEKV_N
 extern "C" int catekv_decode_attn_noalloc(const catekv_cache* cache, const void* q, int32_t Hq, float sm_scale,
                                           void* out, int32_t out_dtype, float* lse_out, const void* plan_host,
                                           const void* plan_dev, size_t plan_bytes, catekv_stream stream) {
+  CATEKV_API_RANGE();
   static void* scratch_of_device[64] = {};
   int dev = 0;
   CATEKV_CUDA_TRY(cudaGetDevice(&dev));

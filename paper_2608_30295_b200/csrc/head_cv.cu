@@ -216,6 +216,7 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
                               int64_t k_stride_t, const int32_t* seq_len, int32_t B, int32_t Hq, int32_t Hkv,
                               int32_t d, int32_t L_obs, int32_t L_init, int32_t L_rec, float quantile_k, float alpha,
                               int32_t causal, float* cv_out, void* ws, size_t ws_bytes, catekv_stream stream) {
+  CATEKV_API_RANGE();
   if (!q_win || !k || !seq_len || !cv_out || !ws) return CATEKV_ERR_INVALID_ARG;
   if (B <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv) return CATEKV_ERR_INVALID_ARG;
   if (d != kD) return CATEKV_ERR_UNSUPPORTED;

@@ -15,6 +15,7 @@ extern "C" size_t catekv_decode_workspace_bytes(int32_t B, int32_t Hkv, int32_t 
 
 extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, void* plan_host, void* plan_dev,
                                   size_t plan_bytes, catekv_stream stream) {
+  CATEKV_API_RANGE();
   int rc = check_cache(cache);
   if (rc) return rc;
   if (num_ctas <= 0 || !plan_host) return CATEKV_ERR_INVALID_ARG;

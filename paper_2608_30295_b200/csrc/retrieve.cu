@@ -297,6 +297,7 @@ extern "C" size_t catekv_retrieval_meta_bytes(const catekv_cache* cache, int32_t
 }
 
 extern "C" int catekv_retrieval_build(const catekv_cache* cache, int32_t chunk_size, void* meta, catekv_stream stream) {
+  CATEKV_API_RANGE();
   int rc = check_cache_r(cache);
   if (rc) return rc;
   if (!meta) return CATEKV_ERR_INVALID_ARG;
@@ -314,6 +315,7 @@ extern "C" int catekv_retrieval_build(const catekv_cache* cache, int32_t chunk_s
 
 extern "C" int catekv_retrieval_append(const catekv_cache* cache, int32_t chunk_size, const void* k_new, void* meta,
                                        catekv_stream stream) {
+  CATEKV_API_RANGE();
   int rc = check_cache_r(cache);
   if (rc) return rc;
   if (!meta || !k_new) return CATEKV_ERR_INVALID_ARG;
@@ -326,6 +328,7 @@ extern "C" int catekv_retrieval_append(const catekv_cache* cache, int32_t chunk_
 
 extern "C" int catekv_append_retrieval(catekv_cache* cache, const void* k_new, const void* v_new, int32_t chunk_size,
                                        void* meta, catekv_stream stream) {
+  CATEKV_API_RANGE();
   int rc = check_cache_r(cache);
   if (rc) return rc;
   if (!meta || !k_new || !v_new) return CATEKV_ERR_INVALID_ARG;
@@ -474,6 +477,7 @@ extern "C" int catekv_retrieve_compact(const catekv_cache* cache, const void* me
                                        int32_t Hq, const uint8_t* retrieval_mask, int32_t budget, int32_t sink, int32_t local,
                                        catekv_cache* step_cache, int32_t* idx_out, int64_t idx_stride, void* ws,
                                        size_t ws_bytes, catekv_stream stream) {
+  CATEKV_API_RANGE();
   if (!step_cache) return CATEKV_ERR_INVALID_ARG;
   return retrieve_impl(cache, meta, chunk_size, q, Hq, retrieval_mask, budget, sink, local, step_cache, idx_out, idx_stride,
                        nullptr, ws, ws_bytes, stream);
@@ -483,6 +487,7 @@ extern "C" int catekv_retrieve_select(const catekv_cache* cache, const void* met
                                       int32_t Hq, const uint8_t* retrieval_mask, int32_t budget, int32_t sink, int32_t local,
                                       int32_t* idx, int64_t idx_stride, int32_t* sel_len, void* ws, size_t ws_bytes,
                                       catekv_stream stream) {
+  CATEKV_API_RANGE();
   return retrieve_impl(cache, meta, chunk_size, q, Hq, retrieval_mask, budget, sink, local, nullptr, idx, idx_stride, sel_len,
                        ws, ws_bytes, stream);
 }

@@ -477,6 +477,7 @@ extern "C" size_t catekv_select_workspace_bytes(int32_t B, int32_t Hq, int32_t H
 
 extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache* cache, int32_t* idx_out,
                                      int64_t idx_stride, void* ws, size_t ws_bytes, catekv_stream stream) {
+  CATEKV_API_RANGE();
   if (!p || !cache || !ws) return CATEKV_ERR_INVALID_ARG;
   if (p->B <= 0 || p->Hq <= 0 || p->Hkv <= 0 || p->Hq % p->Hkv) return CATEKV_ERR_INVALID_ARG;
   if (p->d != kD) return CATEKV_ERR_UNSUPPORTED;
