@@ -209,3 +209,78 @@ def test_classify_heads_matches_oracle(ck):
         assert np.array_equal(got, want), (N, H, r)
     cv = np.array([[9, 1, 8, 2], [9, 7, 1, 2], [9, 1, 8, 2]], dtype=np.float32)
     assert list(ck.catekv_classify_heads(cv, 0.5)) == [1, 0, 1, 0]
+
+
+def test_retrieve_lengths_match_the_oracle_selection_sizes(ck):
+    from oracle import catekv_oracle as orc
+    rng = np.random.default_rng(11)
+    for _ in range(40):
+        n_segs = int(rng.integers(1, 7))
+        lens = [int(rng.integers(0, 3000)) for _ in range(n_segs)]
+        cs = int(rng.choice([1, 2, 4, 8, 16, 32]))
+        budget, sink, local = int(rng.integers(0, 1200)), int(rng.integers(0, 20)), int(rng.integers(0, 100))
+        mask = rng.integers(0, 2, size=n_segs).astype(np.uint8)
+        st, keep = _host_cache(ck, 1, n_segs, lens)
+        got = np.zeros(n_segs, dtype=np.int32)
+        rc = ck._lib.catekv_retrieve_lengths(C.byref(st), cs, mask.ctypes.data, budget, sink, local, got.ctypes.data)
+        assert rc == 0
+        for s, L in enumerate(lens):
+            want = len(orc.retrieve_indices(np.zeros((L + cs - 1) // cs), L, sink, local, budget, cs)) if mask[s] else L
+            assert got[s] == want, (lens, cs, budget, sink, local, s)
+    assert ck._lib.catekv_retrieve_lengths(C.byref(st), 3, mask.ctypes.data, 10, 0, 0, got.ctypes.data) == ck.ERR_UNSUPPORTED
+
+
+def _pages(ck, st, n_segs, n_pages, max_pages):
+    table = np.full((n_segs, max_pages), -1, dtype=np.int32)
+    seg_pages = np.zeros(n_segs, dtype=np.int32)
+    fake = 0x10000
+    pg = ck.PagesStruct(max_pages, n_pages, 0, 0, fake, fake, fake, table.ctypes.data, seg_pages.ctypes.data, fake)
+    st.pages = C.pointer(pg)
+    return pg, table, seg_pages
+
+
+def test_pages_bookkeeping_without_a_device(ck):
+    # the paths of catekv_pages_reserve that copy nothing: refusals, and requests the capacity already covers
+    st, keep = _host_cache(ck, 1, 3, [128, 5, 200], 0)  # capacities 128, 128, 256
+    assert ck._lib.catekv_pages_reserve(C.byref(st), 1, None) == ck.ERR_INVALID_ARG  # no pages attached
+    pg, table, seg_pages = _pages(ck, st, 3, n_pages=2, max_pages=2)
+    assert ck._lib.catekv_pages_reserve(C.byref(st), 0, None) == 0
+    assert ck._lib.catekv_pages_reserve(C.byref(st), -1, None) == ck.ERR_INVALID_ARG
+    # 129 more rows: segment 0 would need 3 pages (> max_pages); 100 more rows: 2 + 0 + 1 pages > the 2 of the pools
+    for n_new in (129, 100):
+        assert ck._lib.catekv_pages_reserve(C.byref(st), n_new, None) == ck.ERR_CAPACITY
+        assert pg.next_free == 0 and not seg_pages.any() and (table == -1).all()
+    # capacity seen by the other host checks: appends are refused while no page has been handed out
+    assert ck._lib.catekv_append(C.byref(st), 0x10000, 0x10000, None) == ck.ERR_CAPACITY
+    assert ck._lib.catekv_cache_advance(C.byref(st), 1) == ck.ERR_CAPACITY
+    # with a page per segment on the books (as catekv_pages_reserve would leave them) 64 more rows fit
+    seg_pages[:] = 1
+    table[:, 0] = [0, 1, 2]
+    pg.n_pages, pg.next_free = 3, 3
+    assert ck._lib.catekv_cache_advance(C.byref(st), 64) == 0
+    assert list(keep[2]) == [192, 69, 264]
+    assert ck._lib.catekv_cache_advance(C.byref(st), 1) == ck.ERR_CAPACITY  # segment 0 is full again
+    # plans accept lengths beyond the segment's own capacity and carry that capacity in every work item
+    nbytes = ck._lib.catekv_decode_plan_bytes(1, 3, 4)
+    buf = np.zeros(nbytes, dtype=np.uint8)
+    assert ck._lib.catekv_decode_plan(C.byref(st), 4, buf.ctypes.data, None, nbytes, None) == 0
+    hdr = buf[:48].view(np.int32)
+    raw = buf[int(hdr[9]):int(hdr[9]) + 32 * int(hdr[3])].view(np.int32).reshape(-1, 8)
+    assert all(int(r[7]) == int(keep[1][r[0]]) for r in raw)
+    # calls that walk contiguous segments refuse the paged cache
+    assert ck._lib.catekv_retrieval_meta_bytes(C.byref(st), 8) == 0
+    got = np.zeros(3, dtype=np.int32)
+    m = np.ones(3, dtype=np.uint8)
+    assert ck._lib.catekv_retrieve_lengths(C.byref(st), 8, m.ctypes.data, 64, 0, 0, got.ctypes.data) == ck.ERR_UNSUPPORTED
+
+
+def test_fused_append_refuses_lengths_below_the_plan(ck):
+    st, keep = _host_cache(ck, 1, 2, [300, 40], 8)
+    nbytes = ck._lib.catekv_decode_plan_bytes(1, 2, 3)
+    buf = np.zeros(nbytes, dtype=np.uint8)
+    assert ck._lib.catekv_decode_plan(C.byref(st), 3, buf.ctypes.data, None, nbytes, None) == 0
+    keep[2][0] = 299  # the list has shrunk since
+    f = 0x10000
+    rc = ck._lib.catekv_append_decode_attn(C.byref(st), f, f, f, 8, 0.0, f, 0, None, buf.ctypes.data, f, nbytes, f, 1 << 30,
+                                           None)
+    assert rc == ck.ERR_INVALID_ARG and list(keep[2]) == [299, 40]
