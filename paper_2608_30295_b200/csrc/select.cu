@@ -223,8 +223,9 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
           const bool hit = in[e] && (v[e] & pmask) == prefix;
           // a warp whose lanes all fall in one bin adds once; otherwise every hit adds for itself
           const unsigned int dgt = hit ? ((v[e] >> shift) & dmask) : 0x100u;
-          const unsigned int d0 = __shfl_sync(0xffffffffu, dgt, 0);
-          if (__all_sync(0xffffffffu, dgt == d0)) {
+          int same;
+          __match_all_sync(0xffffffffu, dgt, &same);
+          if (same) {
             if (hit && (tid & 31) == 0) atomicAdd(&hist[dgt], 32u);
           } else if (hit) {
             atomicAdd(&hist[dgt], 1u);
