@@ -88,18 +88,14 @@ __device__ __forceinline__ ItemCursor plan_cursor(const WorkItem& w) {
   c.cap = w.cap;
   return c;
 }
-// the part that reads what earlier kernels wrote: the live length (a plain load: with a fused append this
-// kernel itself updates the length when it is done with the segment)
+// the part that depends on what earlier kernels wrote: the live length (with a fused append this kernel itself
+// updates the length when it is done with the segment); len and sel are the loaded seg_len / sel_len entries
 template <int kMode>
-__device__ __forceinline__ void live_cursor(const DecodeArgs& a, ItemCursor& c) {
+__device__ __forceinline__ void apply_live(const DecodeArgs& a, ItemCursor& c, int len, int sel) {
   constexpr bool kIndexed = kMode == kModeIndexed;
-  int len;
   if (kIndexed) {
-    const int sel = *reinterpret_cast<const volatile int32_t*>(a.sel_len + c.seg);
     c.indexed = sel >= 0;
-    len = sel >= 0 ? sel : *reinterpret_cast<const volatile int32_t*>(a.seg_len + c.seg);
-  } else {
-    len = *reinterpret_cast<const volatile int32_t*>(a.seg_len + c.seg);
+    if (sel >= 0) len = sel;
   }
   if (c.last) {
     c.new_row = (!kIndexed && a.k_new) ? len : -1;
@@ -108,6 +104,18 @@ __device__ __forceinline__ void live_cursor(const DecodeArgs& a, ItemCursor& c) 
     c.live = min(c.t1, len);  // a segment that has shrunk since the plan was built: attend only to what it holds
   }
 }
+template <int kMode>
+__device__ __forceinline__ void live_cursor(const DecodeArgs& a, ItemCursor& c) {
+  const int len = *reinterpret_cast<const volatile int32_t*>(a.seg_len + c.seg);
+  const int sel = kMode == kModeIndexed ? *reinterpret_cast<const volatile int32_t*>(a.sel_len + c.seg) : -1;
+  apply_live<kMode>(a, c, len, sel);
+}
+// What the cursor of the next piece is made of, requested one piece ahead: a piece change then finds the values in
+// registers instead of waiting for two dependent loads while no tile is being issued.
+struct NextItem {
+  int4 x, y;
+  int len, sel;
+};
 __device__ __forceinline__ WorkItem unpack_item(const int4& x, const int4& y) {
   WorkItem w;
   w.seg = x.x; w.t0 = x.y; w.t1 = x.z; w.slot = x.w;
@@ -115,11 +123,19 @@ __device__ __forceinline__ WorkItem unpack_item(const int4& x, const int4& y) {
   w.last = y.z; w.cap = y.w;
   return w;
 }
+// item `it` belongs to segment `seg` (pieces after a CTA's first belong to consecutive segments)
 template <int kMode>
-__device__ __forceinline__ ItemCursor read_item(const DecodeArgs& a, int it) {
+__device__ __forceinline__ void fetch_next(const DecodeArgs& a, int it, int seg, NextItem& n) {
   const int4* p = reinterpret_cast<const int4*>(a.items + it);
-  ItemCursor c = plan_cursor(unpack_item(__ldg(p), __ldg(p + 1)));
-  live_cursor<kMode>(a, c);
+  n.x = __ldg(p);
+  n.y = __ldg(p + 1);
+  n.len = *reinterpret_cast<const volatile int32_t*>(a.seg_len + seg);
+  n.sel = kMode == kModeIndexed ? *reinterpret_cast<const volatile int32_t*>(a.sel_len + seg) : -1;
+}
+template <int kMode>
+__device__ __forceinline__ ItemCursor make_cursor(const DecodeArgs& a, const NextItem& n) {
+  ItemCursor c = plan_cursor(unpack_item(n.x, n.y));
+  apply_live<kMode>(a, c, n.len, n.sel);
   return c;
 }
 // tiles of the item's live rows; at least one
@@ -150,6 +166,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
   constexpr bool kIndexed = kMode == kModeIndexed;
   constexpr bool kPaged = kMode == kModePaged;
   extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ ItemCursor s_ring[4];  // cursors of the pieces the producer has started, for the consumer
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
   CATEKV_STAMP(0);
@@ -239,12 +256,21 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     const uint16_t* src = a.q + ((int64_t)b * a.Hq + h * a.G + (ok ? r : 0)) * kD + c * 8;
     cp_async16(qb + r * kRowBytes + c * 16, src, ok);
   };
+  // The producer moves on to the next piece: its cursor comes from the values requested one piece ahead, is handed
+  // to the consumer through a small ring in shared memory (the consumer gets there at least one barrier later and
+  // at most kStages - 1 tiles, hence pieces, behind), and the piece after it is requested.
+  NextItem nxt;
+  auto next_item = [&]() {
+    p_tile = 0;
+    if (++p_item < item_end) {
+      pc = make_cursor<kMode>(a, nxt);
+      if (tid == 0) s_ring[(p_item - item_begin) & 3] = pc;
+      if (p_item + 1 < item_end) fetch_next<kMode>(a, p_item + 1, pc.seg + 1, nxt);
+    }
+  };
   auto advance = [&]() {  // after a tile was issued; the plan-time tiles need no look at the live length
     ++p_seq;
-    if (++p_tile >= pc.np && p_tile >= item_tiles(pc)) {
-      p_tile = 0;
-      if (++p_item < item_end) pc = read_item<kMode>(a, p_item);
-    }
+    if (++p_tile >= pc.np && p_tile >= item_tiles(pc)) next_item();
     load_idx();
   };
   auto issue = [&]() {  // one tile (with the item's queries if it is the item's first) = one commit group
@@ -269,18 +295,16 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
   pdl_wait();  // from here on: lengths, queries and rows written by earlier kernels
   live_cursor<kMode>(a, pc);
   const ItemCursor first = pc;
+  if (item_begin + 1 < item_end) fetch_next<kMode>(a, item_begin + 1, pc.seg + 1, nxt);
   issue_q(0, pc.seg);
-  if (p_tile >= pc.np && p_tile >= item_tiles(pc)) {
-    p_tile = 0;
-    if (++p_item < item_end) pc = read_item<kMode>(a, p_item);
-  }
+  if (p_tile >= pc.np && p_tile >= item_tiles(pc)) next_item();
   load_idx();
   for (int s = pre; s < kStages - 1; ++s) issue();
   if (pre == kStages - 1) cp_async_commit();  // the queries of the first item form a group of their own
 
   int seq = 0;
   for (int c_item = item_begin; c_item < item_end; ++c_item) {
-    const ItemCursor cc = c_item == item_begin ? first : read_item<kMode>(a, c_item);
+    const ItemCursor cc = c_item == item_begin ? first : s_ring[(c_item - item_begin) & 3];
     uint32_t qf[8][2];
     float o[8][4];
 #pragma unroll
