@@ -649,6 +649,9 @@ def main():
             table[name] = {"layers_timed": nl, "us_per_layer_step": t * 1e3 / nl, "partials_us": pu,
                            "bytes_per_layer_step": by, "hbm_gbs": by / (pu * 1e-6) / 1e9,
                            "frac_of_measured": by / (pu * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                           # the whole replayed layer-step (attention + combine, append fused) against the same bytes
+                           "step_hbm_gbs": by / (t * 1e-3 / nl) / 1e9,
+                           "step_frac_of_measured": by / (t * 1e-3 / nl) / 1e9 / peaks["hbm_gbs"],
                            "select_ms_per_layer": float(np.mean(so[1:] or so))}
             del mo
             torch.cuda.empty_cache()
