@@ -405,11 +405,11 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
     }
 #pragma unroll
-    for (int round = 0; round < 2; ++round) {
-      const int stride = 1 << round;                       // 1, then 2
-      const bool writer = (warp & (2 * stride - 1)) == stride;  // round 0: warps 1,3; round 1: warp 2
-      const bool reader = (warp & (2 * stride - 1)) == 0;       // round 0: warps 0,2; round 1: warp 0
-      float* mb = merge + (warp >> (round + 1)) * (kMergeRegs * 32);
+    for (int lvl = 0; lvl < 2; ++lvl) {
+      const int stride = 1 << lvl;                       // 1, then 2
+      const bool writer = (warp & (2 * stride - 1)) == stride;  // level 0: warps 1,3; level 1: warp 2
+      const bool reader = (warp & (2 * stride - 1)) == 0;       // level 0: warps 0,2; level 1: warp 0
+      float* mb = merge + (warp >> (lvl + 1)) * (kMergeRegs * 32);
       if (writer) {
 #pragma unroll
         for (int i = 0; i < 8; ++i)
@@ -441,7 +441,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
         m0 = mn0;
         m1 = mn1;
       }
-      if (round == 0) __syncthreads();  // slot 0 is rewritten by warp 2 in the next round
+      if (lvl == 0) __syncthreads();  // slot 0 is rewritten by warp 2 at the next level
     }
     if (warp == 0) {
       // stage the normalised [8 heads x 128] block in shared memory, then write whole rows
