@@ -510,10 +510,10 @@ struct CombineArgs {
   int32_t Hq, Hkv, G, out_fp32;
 };
 
-// One CTA of 8 warps per (segment, query head of the group).  The kernel is a chain of dependent memory
-// round trips, so it is arranged to have few of them: every warp finds the maximum LSE by itself (no
-// barrier), then sums its eighth of the pieces with all of its loads in flight at once (a lane owns four
-// consecutive d, a piece is one 512-byte row per warp-load); the warps are summed in a fixed order.
+// One CTA of 8 warps per (segment, query head of the group).  The kernel is a chain of dependent trips to
+// memory, so it is arranged to have one: a warp loads the values and the LSEs of its eighth of the pieces at
+// once (a lane owns four consecutive d, a piece is one 512-byte row per warp-load) and merges them under a
+// running maximum of its own; the warps are then merged through shared memory in a fixed order.
 constexpr int kCombineWarps = 8;
 constexpr int kCombineUnroll = 16;
 __global__ void __launch_bounds__(kCombineWarps * 32) decode_combine_kernel(const CombineArgs a) {
@@ -528,7 +528,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32) decode_combine_kernel(cons
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n = si.n_pieces;
   const float* lse = a.part_lse + (size_t)si.slot_begin * kMaxG + hd;
-  // One trip to memory: a warp loads the values and the LSEs of its pieces together (16 pieces in flight: one round for up to 128 pieces) and merges
+  // One trip to memory: a warp loads the values and the LSEs of its pieces together (16 pieces in flight: a single pass for up to 128 pieces) and merges
   // them with a running maximum of its own; the 8 warps are then merged through shared memory.
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float wsum = 0.f, mw = -INFINITY;
@@ -548,7 +548,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32) decode_combine_kernel(cons
 #pragma unroll
       for (int u = 0; u < kCombineUnroll; ++u) mx = fmaxf(mx, w[u]);
       if (mx > -INFINITY) {
-        const float sc = exp2f(mw - mx);  // 0 on the first round (mw = -inf)
+        const float sc = exp2f(mw - mx);  // 0 on the first pass (mw = -inf)
         acc.x *= sc;
         acc.y *= sc;
         acc.z *= sc;
