@@ -270,6 +270,7 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   sa.G = G;
   sa.L_obs = L_obs;
   sa.causal = causal ? 1 : 0;
+  sa.g_major = L_obs == 64 ? 1 : 0;  // the paper's window: head-major rows make the group mean a register sum
   sa.scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
   sa.keys_per_cta = score_keys_per_cta(n_segs, m_max);
   sa.n_chunks = (m_max + sa.keys_per_cta - 1) / sa.keys_per_cta;

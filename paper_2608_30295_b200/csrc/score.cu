@@ -147,7 +147,7 @@ __device__ __forceinline__ uint32_t sw128_off(int r, int c, int rows) {
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(kScThreads) score_tc_kernel(const __grid_constant__ CUtensorMap k_map, const ScoreArgs a,
+__global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_constant__ CUtensorMap k_map, const ScoreArgs a,
                                                               const ScoreShape sh) {
   extern __shared__ uint8_t smem_raw[];
   const ScoreJob job = a.jobs[blockIdx.y];
@@ -176,10 +176,17 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const __grid_const
   const int n_cols = kStats ? sh.cols1 : sh.cols2;
   const int U = n_tiles * UPT;
 
-  // ---- set-up: Q (row r = i * G + g) by cp.async from all threads, barriers, TMEM
+  // ---- set-up: Q (row r = i * G + g, or g * L_obs + i) by cp.async from all threads, barriers, TMEM
   for (int id = tid; id < sh.q_rows * 16; id += kScThreads) {
     const int r = id >> 4, c = id & 15;
-    const int i = r / a.G, g = r - i * a.G;
+    int i, g;
+    if (a.g_major) {
+      g = r / a.L_obs;
+      i = r - g * a.L_obs;
+    } else {
+      i = r / a.G;
+      g = r - i * a.G;
+    }
     const int ok = r < sh.R ? 16 : 0;
     const uint16_t* src = a.q_win + (((int64_t)job.b * a.Hq + job.h * a.G + (ok ? g : 0)) * a.L_obs + (ok ? i : 0)) * kD + c * 8;
     cp_async16(s_q + sw128_off(r, c, sh.q_rows), src, ok);
@@ -259,6 +266,7 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const __grid_const
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float inv_g = 1.f / (float)a.G;
     float col_acc = 0.f;  // pass 2, column sums: this key's sum over this thread's rows of the tile
+    float macc[32];       // pass 2, head-major matrix: this key's entries of this thread's 32 window rows
 
     for (int u = 0; u < U; ++u) {
       const int tile = u / UPT, sub = u - tile * UPT;
@@ -272,7 +280,7 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const __grid_const
       if (kStats) {
         // this thread's query row, keys [64 * half, 64 * half + 64) of the tile
         const int r = sub * 128 + lane_row;
-        const int i = r / a.G;
+        const int i = a.g_major ? r % a.L_obs : r / a.G;
         const int lim = a.causal ? job.n - a.L_obs + i : 0x7fffffff;  // last key this window row sees
         const int jmax = min(j_hi - 1, lim);                          // keys j <= jmax are live
         float m = s_f[2 * (half * kScoreMaxRows + r)], l = s_f[2 * (half * kScoreMaxRows + r) + 1];
@@ -342,6 +350,48 @@ __global__ void __launch_bounds__(kScThreads) score_tc_kernel(const __grid_const
           // in either order, so the result does not depend on timing
           if (sub == UPT - 1 && j < j_hi)
             atomicAdd(a.out + (size_t)blockIdx.y * a.out_job_stride + (j - job.j_begin), col_acc * inv_g);
+        } else if (a.g_major) {
+          // group-mean matrix with head-major rows and L_obs = 64: this thread owns the window rows 32 * half + c
+          // (c = 0..31) of its key; head g's logits for them are the 32 TMEM columns from g * 64 + 32 * half on, so
+          // the mean over the heads is a register accumulation without any bookkeeping
+          float* A = a.out + (size_t)blockIdx.y * a.out_job_stride;
+          const int m_cols = job.j_end - job.j_begin;
+          if (sub == 0) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) macc[c] = 0.f;
+          }
+          const int i_min = j - (job.n - a.L_obs);  // causal: window row i sees key j iff i >= i_min
+          const bool edge = a.causal && __any_sync(0xffffffffu, i_min > half * 32);
+#pragma unroll 1
+          for (int gg = 0; gg < a.G; ++gg) {
+            const int col = gg * 64 + half * 32;
+            if (col < r_begin || col >= r_end) continue;  // another unit's columns
+            float x[32];
+            tmem_ld32(tbase + (col - r_begin), x);
+#pragma unroll
+            for (int c = 0; c < 32; c += 4) {
+              const float4 mm = *reinterpret_cast<const float4*>(s_f + col + c);
+              float e0 = fast_exp2(fmaf(x[c], a.scale_log2, -mm.x));
+              float e1 = fast_exp2(fmaf(x[c + 1], a.scale_log2, -mm.y));
+              float e2 = fast_exp2(fmaf(x[c + 2], a.scale_log2, -mm.z));
+              float e3 = fast_exp2(fmaf(x[c + 3], a.scale_log2, -mm.w));
+              if (edge) {
+                const int i0 = half * 32 + c;
+                e0 = i0 >= i_min ? e0 : 0.f;
+                e1 = i0 + 1 >= i_min ? e1 : 0.f;
+                e2 = i0 + 2 >= i_min ? e2 : 0.f;
+                e3 = i0 + 3 >= i_min ? e3 : 0.f;
+              }
+              macc[c] += e0;
+              macc[c + 1] += e1;
+              macc[c + 2] += e2;
+              macc[c + 3] += e3;
+            }
+          }
+          if (sub == UPT - 1 && j < j_hi) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) A[(size_t)(half * 32 + c) * m_cols + (j - job.j_begin)] = macc[c] * inv_g;
+          }
         } else {
           // group-mean matrix, stored densely ([L_obs][m], m = the job's key range): rows come in runs of G heads per
           // window row; r0 is a multiple of G
@@ -478,6 +528,7 @@ int score_keys_per_cta(int n_jobs, int max_keys) {
 int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream) {
   if (a.n_jobs <= 0 || a.n_chunks <= 0) return CATEKV_OK;
   if (a.G * a.L_obs > kScoreMaxRows || a.keys_per_cta % kKeyTile || !a.status) return CATEKV_ERR_UNSUPPORTED;
+  if (a.g_major && (a.L_obs != 64 || out_mode != kScoreMatrix)) return CATEKV_ERR_UNSUPPORTED;
   const ScoreShape sh = score_shape(a.G, a.L_obs);
   CUtensorMap map;
   int rc = make_k_map(a, &map);

@@ -18,6 +18,7 @@ struct ScoreArgs {
   int64_t sb, sh, st;
   const ScoreJob* jobs;   // device
   int32_t n_jobs, Hq, G, L_obs, causal;
+  int32_t g_major;        // row order of the window queries: 0: r = i * G + g; 1: r = g * L_obs + i (matrix mode, L_obs = 64)
   int32_t B, Hkv, n_max;  // extents of k (sequences, KV heads, tokens) for the TMA descriptor
   float scale_log2;       // log2(e) / sqrt(d)
   int32_t keys_per_cta;   // multiple of 128
