@@ -34,6 +34,8 @@ def _cv_both(ck, q, k, seq_len, L_obs, L_init, L_rec, kq, alpha, causal):
     (6, 2, 7, 257, 3, 1, 0.5, 1.0, False),
     (16, 2, 64, 1200, 32, 8, 0.99, 1.0, True),    # G = 8, window 64: the largest supported row count (512)
     (10, 2, 50, 900, 16, 8, 0.99, 1.0, True),     # G = 5: row halves that are multiples of lcm(16, G)
+    (2, 2, 64, 700, 8, 64, 0.97, 1.0, False),     # G = 1, window 64, no mask (head-major rows, one unit)
+    (8, 2, 64, 1100, 0, 3, 0.99, 1.2, True),      # G = 4, window 64, the mask reaches deep into the matrix
 ])
 def test_head_cv_matches_oracle(ck, Hq, Hkv, L_obs, n, L_init, L_rec, kq, alpha, causal):
     w = synth.scaled(synth.WORKLOADS["cfg4"], Hq=Hq, Hkv=Hkv, L_obs=L_obs, B=1)
