@@ -244,6 +244,9 @@ def time_decode(ck, w, model, dev, steps, warmup, barrier=None, graph=True):
     return e0.elapsed_time(e1) / steps
 
 
+APPEND_US = None  # mean duration of the separate append launch, set by time_kernels
+
+
 def time_kernels(ck, w, model, dev, steps):
     """Per-kernel durations over the same steps: events around the partials kernel of every launch."""
     import torch
@@ -254,17 +257,20 @@ def time_kernels(ck, w, model, dev, steps):
     for i in range(steps):
         q, kn, vn = sets[i % len(sets)]
         for l, m in enumerate(model):
+            z, a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+            z.record()
             ck.catekv_append(m["cache"], kn[l], vn[l])
-            a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
             a.record()
             ck.catekv_decode_partials(m["cache"], q[l], m["plan"], out[l])
             b.record()
             ck.catekv_decode_combine(m["cache"], q[l], m["plan"], out[l])
             c.record()
-            ev.append((a, b, c))
+            ev.append((z, a, b, c))
     torch.cuda.synchronize()
-    part = [a.elapsed_time(b) * 1e3 for a, b, _ in ev]
-    comb = [b.elapsed_time(c) * 1e3 for _, b, c in ev]
+    part = [a.elapsed_time(b) * 1e3 for _, a, b, _ in ev]
+    comb = [b.elapsed_time(c) * 1e3 for _, _, b, c in ev]
+    global APPEND_US
+    APPEND_US = float(np.mean([z.elapsed_time(a) * 1e3 for z, a, _, _ in ev]))
     return float(np.mean(part)), float(np.median(part)), float(np.mean(comb))
 
 
@@ -623,7 +629,8 @@ def main():
                                        "(read = 1.00015 x algorithmic bytes), applied to this run's kept rows",
                      "kernel": "decode_partial_kernel", "bytes_per_launch": bytes_per_layer,
                      "us_per_launch": part_us, "us_per_launch_median": part_med_us,
-                     "frac_of_8TBs": achieved / 8000.0, "combine_us": comb_us},
+                     "frac_of_8TBs": achieved / 8000.0, "combine_us": comb_us,
+                     "append_us": APPEND_US},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e},
         "gpu_launches": args.steps * n_layers * ((1 if FUSED else 2) +
