@@ -447,6 +447,73 @@ def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8, graph=Tru
     return e0.elapsed_time(e1) * 1e3 / (steps * n_layers), attended, meta_bytes
 
 
+def time_linearity(ck, dev, B=8, Hkv=8, G=4, n=32768, budget=1024, n_layers=2, reps=6):
+    """The paper's qualitative efficiency claims on this kernel: decode time grows linearly with the share of
+    adaptive heads r (Section 4.4.1) and with their retained fraction eta (Section 4.4.2), and the consistent
+    heads' budget hardly matters (Section 4.4.3).  Synthetic pools (random rows, no selection), CUDA-graph replay
+    of the fused step.  Returns the sweeps with the R^2 of a straight-line fit."""
+    import torch
+    num_ctas = ck.catekv_decode_num_ctas()
+    n_segs = B * Hkv
+    q = torch.randn((B, Hkv * G, 128), device=dev).bfloat16()
+    kn = torch.randn((B, Hkv, 128), device=dev).bfloat16()
+    out = torch.empty((B, Hkv * G, 128), device=dev, dtype=torch.bfloat16)
+
+    def measure(r, eta, b):
+        n_ad = int(round(r * n_segs))
+        lens = np.full(n_segs, b, dtype=np.int32)
+        lens[np.linspace(0, n_segs - 1, n_ad).astype(int)] = int(eta * n)
+        model = []
+        for _ in range(n_layers):
+            c = ck.Cache(B, Hkv, lens, reps + 8, dev)
+            c.k_pool.normal_()
+            c.v_pool.normal_()
+            c.set_lengths(lens)
+            p = ck.DecodePlan(c, num_ctas)
+            ck.catekv_decode_plan(c, p)
+            model.append((c, p))
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for c, p in model:
+                    ck.catekv_append_decode_attn(c, kn, kn, q, p, out)
+        torch.cuda.current_stream().wait_stream(side)
+        g.replay()
+
+        def rep():
+            for c, _ in model:
+                ck.catekv_cache_advance(c, 1)
+            g.replay()
+        rep()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            rep()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (reps * n_layers)
+
+    def fit(x, y):
+        x, y = np.asarray(x, dtype=np.float64), np.asarray(y, dtype=np.float64)
+        a, b0 = np.polyfit(x, y, 1)
+        ss = float(((y - (a * x + b0)) ** 2).sum())
+        return 1.0 - ss / float(((y - y.mean()) ** 2).sum())
+
+    rs = [0.125, 0.25, 0.5, 0.75, 1.0]
+    t_r = [measure(r, 1.0, budget) for r in rs]
+    etas = [0.25, 0.5, 0.75, 1.0]
+    t_e = [measure(0.5, e, budget) for e in etas]
+    budgets = [512, 1024, 2048]
+    t_b = [measure(0.5, 1.0, b) for b in budgets]
+    return {"shape": f"B {B}, {Hkv} KV heads, G {G}, context {n}",
+            "adaptive_share_r": rs, "us_per_layer_step_vs_r": t_r, "r2_vs_r": fit(rs, t_r),
+            "eta": etas, "us_per_layer_step_vs_eta": t_e, "r2_vs_eta": fit(etas, t_e),
+            "consistent_budget": budgets, "us_per_layer_step_vs_budget": t_b}
+
+
 # ------------------------------------------------------------------------------------------
 # the oracle, timed as it stands, on a bounded sample
 # ------------------------------------------------------------------------------------------
@@ -689,6 +756,7 @@ def main():
                              "metadata_bytes_per_layer_step": rm, "budget_rows": 1024, "chunk": 8,
                              "note": "query-aware retrieval on the adaptive heads of the same workload: per layer "
                                      "catekv_append_retrieval, catekv_retrieve_select, catekv_decode_attn_indexed; CUDA graph replay of the step"}
+        line["linearity"] = time_linearity(ck, dev)
         rate, desc, spent = oracle_sample_rate(w, target_s=15.0)
         rows = bytes_per_layer / ROW_BYTES
         line["cpu_baseline"] = {"value": w.B / (w.layers * rows / rate), "unit": UNIT, "cores": oracle_threads(),

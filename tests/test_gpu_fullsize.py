@@ -271,3 +271,14 @@ def test_cfg3_retrieval_in_place_as_the_bench_runs_it(ck):
         soc.k_rows[s], soc.v_rows[s] = krows[got], vrows[got]
     ref, ref_lse = orc.decode_attention(soc, synth.bits(q), cells=[divmod(s, w.Hkv) for s in cells])
     H.check_attention(out, None, lse, ref, ref_lse, "cfg3 retrieval in place")
+
+
+def test_decode_time_follows_the_papers_efficiency_claims(ck):
+    # Sections 4.4.1-4.4.3: latency grows linearly with the share of adaptive heads and with their retained
+    # fraction, and the consistent heads' budget hardly matters.  Wide margins: this is a timing test.
+    lin = bench.time_linearity(ck, "cuda")
+    assert lin["r2_vs_r"] >= 0.99, lin
+    assert lin["r2_vs_eta"] >= 0.99, lin
+    t = lin["us_per_layer_step_vs_budget"]
+    assert max(t) / min(t) <= 1.15, lin
+    assert lin["us_per_layer_step_vs_r"][-1] > 3.0 * lin["us_per_layer_step_vs_r"][0], lin
