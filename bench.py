@@ -629,6 +629,8 @@ def main():
                     "for --layers layers and print its time; used for profiling that path on a small case")
     ap.add_argument("--retrieval-only", action="store_true", help="run only the query-aware retrieval decode step "
                     "(small case for profiling; use with --workload and --layers)")
+    ap.add_argument("--head-cv-only", action="store_true", help="run only catekv_head_cv on the calibration shape "
+                    "(8 prompts x 16384 tokens, 28q/4kv, window 64) and print its time; for profiling")
     ap.add_argument("--retrieval-gather", action="store_true", help="with --retrieval-only: the gather path "
                     "(catekv_retrieve_compact into a per-step cache) instead of attention in place")
     ap.add_argument("--no-extras", action="store_true", help="skip the other configs, head_cv and the oracle timing")
@@ -665,6 +667,11 @@ def main():
     graph = not args.no_graph
     global FUSED
     FUSED = not args.no_fused
+    if args.head_cv_only:
+        ms_cv = time_head_cv(ck, dev)
+        if rank == 0:
+            print(json.dumps({"head_cv_ms": ms_cv, "shape": "8 prompts x 16384 tokens, 28q/4kv, window 64"}))
+        return
     if args.retrieval_only:
         ru, ra, rm = time_retrieval(ck, w, dev, n_layers=n_layers, steps=args.steps, graph=graph,
                                     gather=args.retrieval_gather)
