@@ -60,7 +60,11 @@ def check_attention(out_f32, out_bf16, lse, ref, ref_lse, where=""):
         g = orc.bf16_to_f64(synth.bits(out_bf16))[ok]
         rb = orc.bf16_to_f64(orc.f64_to_bf16(r))
         assert rel_l2(g, rb) <= REL_L2, (where, "bf16 rel-L2", rel_l2(g, rb))
-        assert max_abs(g, rb) <= MAX_ABS, (where, "bf16 max-abs", max_abs(g, rb))
+        # Elementwise: MAX_ABS, or one bf16 ulp of the reference where that is larger (2^-6 for |x| in [2, 4)):
+        # an fp32 result within 1e-6 of a rounding tie may land on either neighbour of the rounded oracle value.
+        ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(rb), 2.0 ** -126))) - 7)
+        excess = np.abs(g - rb) - np.maximum(MAX_ABS, ulp)
+        assert np.all(excess <= 0), (where, "bf16 max-abs", max_abs(g, rb))
     if lse is not None:
         gl = lse.detach().cpu().double().numpy()[ok]
         rl = ref_lse[ok]
