@@ -57,14 +57,22 @@ def check_attention(out_f32, out_bf16, lse, ref, ref_lse, where=""):
         assert rel_l2(g, r) <= REL_L2, (where, "fp32 rel-L2", rel_l2(g, r))
         assert max_abs(g, r) <= MAX_ABS, (where, "fp32 max-abs", max_abs(g, r))
     if out_bf16 is not None:
+        # The bf16 output is the same arithmetic rounded once at the end: bit-identical to the fp32 output of the
+        # same call sequence rounded to nearest-even (which carries the parity claim against the fp64 oracle above).
+        if out_f32 is not None:
+            assert np.array_equal(synth.bits(out_bf16), synth.bits(out_f32.to(out_bf16.dtype))), (where, "bf16 != rne(fp32)")
+        # Against the oracle rounded to bf16 (like with like): rel-L2 <= 1e-3, except that an fp32 result within 1e-6
+        # of a rounding tie may land on the other neighbour.  Such flips are exactly one bf16 ulp (2^-6 for |x| in
+        # [2, 4), above the 1e-2 absolute bound) and rare; one of them on a large element of a small tensor already
+        # exceeds the rel-L2 bound, so up to 2 % of one-ulp flips are accepted in place of it.
         g = orc.bf16_to_f64(synth.bits(out_bf16))[ok]
         rb = orc.bf16_to_f64(orc.f64_to_bf16(r))
-        assert rel_l2(g, rb) <= REL_L2, (where, "bf16 rel-L2", rel_l2(g, rb))
-        # Elementwise: MAX_ABS, or one bf16 ulp of the reference where that is larger (2^-6 for |x| in [2, 4)):
-        # an fp32 result within 1e-6 of a rounding tie may land on either neighbour of the rounded oracle value.
         ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(rb), 2.0 ** -126))) - 7)
-        excess = np.abs(g - rb) - np.maximum(MAX_ABS, ulp)
-        assert np.all(excess <= 0), (where, "bf16 max-abs", max_abs(g, rb))
+        diff = np.abs(g - rb)
+        assert np.all(diff <= np.maximum(MAX_ABS, ulp)), (where, "bf16 max-abs", max_abs(g, rb))
+        flips = diff > 0
+        only_ties = np.all(diff[flips] <= ulp[flips] * 1.0000001) and flips.mean() <= 0.02
+        assert rel_l2(g, rb) <= REL_L2 or only_ties, (where, "bf16 rel-L2", rel_l2(g, rb), int(flips.sum()))
     if lse is not None:
         gl = lse.detach().cpu().double().numpy()[ok]
         rl = ref_lse[ok]
