@@ -198,3 +198,24 @@ def test_random_retrieval_in_place_equals_gather(ck, seed):
         soc.v_rows.append(oc.v_rows[s][rows])
     ref, ref_lse = orc.decode_attention(soc, synth.bits(q))
     H.check_attention(out, None, lse, ref, ref_lse, f"retrieval seed {seed} lens {lens} cs {cs} budget {budget}")
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_head_cv(ck, seed):
+    rng = np.random.default_rng(9000 + seed)
+    Hkv = int(rng.choice([1, 2, 4]))
+    G = int(rng.choice([1, 2, 3, 4, 5, 7, 8]))
+    L_obs = min(int(rng.choice([7, 16, 32, 50, 64])), 512 // G)
+    n = int(rng.integers(L_obs + 40, 2500))
+    L_init, L_rec = int(rng.integers(0, 20)), int(rng.integers(0, 40))
+    kq = float(rng.choice([0.5, 0.9, 0.99, 0.996]))
+    alpha = float(rng.choice([1.0, 0.8, 1.2]))
+    causal = bool(rng.integers(0, 2))
+    w = synth.scaled(synth.WORKLOADS["cfg4"], Hq=Hkv * G, Hkv=Hkv, L_obs=L_obs, B=1, seed=9100 + seed)
+    types = rng.integers(0, 2, size=Hkv).astype(np.uint8)
+    q, k = synth.calibration_prompt(w, 0, 0, n, types)
+    got = ck.catekv_head_cv(q.cuda(), k.cuda(), [n], L_init, L_rec, kq, alpha, causal).cpu().numpy()
+    want = orc.head_cv(synth.bits(q), synth.bits(k), [n], L_obs, L_init, L_rec, float(np.float32(kq)),
+                       float(np.float32(alpha)), causal)
+    np.testing.assert_allclose(got, want, rtol=1e-3, atol=1e-6,
+                               err_msg=str(dict(Hkv=Hkv, G=G, L_obs=L_obs, n=n, L_init=L_init, L_rec=L_rec, kq=kq)))
