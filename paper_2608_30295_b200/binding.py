@@ -163,23 +163,12 @@ class Cache:
                                   _np_ptr(self.seg_off), _np_ptr(self.seg_cap), _np_ptr(self.seg_len), None)
         self.pages = None
 
-    def attach_pages(self, n_pages: int, max_pages: int):
+    def attach_pages(self, n_pages: int, max_pages: int) -> "Pages":
         """Give the cache overflow pools of n_pages pages of 64 rows (memory only; catekv_pages_reserve hands
         the pages out).  The segments keep what they hold."""
-        n = self.B * self.Hkv
-        pg = type("Pages", (), {})()
-        pg.k_ovf = torch.empty((max(n_pages, 1) * PAGE_ROWS, self.d), dtype=torch.bfloat16, device=self.device)
-        pg.v_ovf = torch.empty_like(pg.k_ovf)
-        pg.table = np.full((n, max_pages), -1, dtype=np.int32)
-        pg.table_dev = torch.full((n, max_pages), -1, dtype=torch.int32, device=self.device)
-        pg.seg_pages = np.zeros(n, dtype=np.int32)
-        pg.seg_cap_dev = torch.from_numpy(self.seg_cap).to(self.device)
-        pg.struct = PagesStruct(max_pages, n_pages, 0, 0, pg.k_ovf.data_ptr(), pg.v_ovf.data_ptr(),
-                                pg.table_dev.data_ptr(), _np_ptr(pg.table), _np_ptr(pg.seg_pages),
-                                pg.seg_cap_dev.data_ptr())
-        self.pages = pg
-        self.struct.pages = C.pointer(pg.struct)
-        return pg
+        self.pages = Pages(self, n_pages, max_pages)
+        self.struct.pages = C.pointer(self.pages.struct)
+        return self.pages
 
     def set_lengths(self, lens):
         """Set host mirror and device lengths (used when rows are written by the caller)."""
@@ -188,6 +177,22 @@ class Cache:
 
     def kept_rows(self) -> int:
         return int(self.seg_len.sum())
+
+
+class Pages:
+    """Overflow pools, page table (device + host mirror) and per-segment page counts of one cache (memory only)."""
+
+    def __init__(self, cache: Cache, n_pages: int, max_pages: int):
+        n = cache.B * cache.Hkv
+        self.k_ovf = torch.empty((max(n_pages, 1) * PAGE_ROWS, cache.d), dtype=torch.bfloat16, device=cache.device)
+        self.v_ovf = torch.empty_like(self.k_ovf)
+        self.table = np.full((n, max_pages), -1, dtype=np.int32)
+        self.table_dev = torch.full((n, max_pages), -1, dtype=torch.int32, device=cache.device)
+        self.seg_pages = np.zeros(n, dtype=np.int32)
+        self.seg_cap_dev = torch.from_numpy(cache.seg_cap).to(cache.device)
+        self.struct = PagesStruct(max_pages, n_pages, 0, 0, self.k_ovf.data_ptr(), self.v_ovf.data_ptr(),
+                                  self.table_dev.data_ptr(), _np_ptr(self.table), _np_ptr(self.seg_pages),
+                                  self.seg_cap_dev.data_ptr())
 
 
 def catekv_append(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor):
