@@ -132,6 +132,9 @@ def expected_lengths(w, mask):
     return lens
 
 
+PLAN_HOST_US = []  # host time of every catekv_decode_plan call of build_model
+
+
 def build_model(ck, w, dev, max_new, layers=None, time_select=True):
     """Caches and plans of `layers` layers via catekv_select_compact.  Returns (layer list, select ms/layer)."""
     import torch
@@ -153,7 +156,9 @@ def build_model(ck, w, dev, max_new, layers=None, time_select=True):
         torch.cuda.synchronize()
         sel_ms.append(e0.elapsed_time(e1))
         plan = ck.DecodePlan(cache, num_ctas)
-        ck.catekv_decode_plan(cache, plan)
+        t0 = time.perf_counter()
+        ck.catekv_decode_plan(cache, plan)  # host: the schedule, plus one asynchronous copy to the device
+        PLAN_HOST_US.append((time.perf_counter() - t0) * 1e6)
         out.append({"cache": cache, "plan": plan, "mask": mask})
         del p
     torch.cuda.synchronize()
@@ -731,6 +736,7 @@ def main():
                                                  (1 if any(ck.plan_header(m["plan"])["n_slots"] for m in model) else 0)),
         "clocks": clocks,
         "select_compact": {"ms_per_layer": float(np.mean(sel_ms[1:] or sel_ms)), "layers": n_layers},
+        "plan_host_us": float(np.median(PLAN_HOST_US[:n_layers])),
     }
     del model
     torch.cuda.empty_cache()
