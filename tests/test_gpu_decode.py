@@ -248,6 +248,12 @@ def test_paged_growth_past_the_laid_out_capacity(ck, fused):
             page = int(pg.table[i, p_i])
             assert np.array_equal(synth.bits(pg.k_ovf[page * 64:page * 64 + nrows]), oc.k_rows[i][r0:r0 + nrows])
             assert np.array_equal(synth.bits(pg.v_ovf[page * 64:page * 64 + nrows]), oc.v_rows[i][r0:r0 + nrows])
+    # the variant with the library's own scratch follows the pages too: same kernel, same bits
+    out_a, out_b = torch.empty_like(out), torch.empty_like(out)
+    ck.catekv_decode_attn(cache, q, plan, out_a)
+    ck.catekv_decode_attn_noalloc(cache, q, plan, out_b)
+    torch.cuda.synchronize()
+    assert torch.equal(out_a, out_b)
     # the table row of a segment is full: one row more is refused
     with pytest.raises(ck.CatekvError) as e:
         ck.catekv_pages_reserve(cache, 64 * 3)
