@@ -447,7 +447,9 @@ static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t ch
   ta.L_obs = 0;
   ta.pool_mode = kPoolPrescored;
   ta.pool_param = cs;
-  rc = launch_topk(ta, n_segs, max_pool, st);
+  int n_masked = 0;
+  for (int s = 0; s < n_segs; ++s) n_masked += retrieval_mask[s] != 0;
+  rc = launch_topk(ta, n_segs, max_pool, n_masked, st);
   if (rc) return rc;
   if (!step_cache) return CATEKV_OK;
   GatherArgs ga;

@@ -391,40 +391,47 @@ extern "C" int catekv_debug_topk_trace(unsigned long long* host_out) {
 namespace catekv {
 #endif
 
-int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, cudaStream_t stream) {
-  static bool attr_set[64] = {};
-  int dev = 0;
-  CATEKV_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (kTopkStageMax + kTopkStageMax / 32 + 1) * 4));
-    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (kTopkStageMax + kTopkStageMax / 32 + 1) * 4));
-    if (dev >= 0 && dev < 64) attr_set[dev] = true;
-  }
-  TopkArgs a = a0;
-  const int CL = max_pool <= 16384 ? 1 : 8;  // short lists: one CTA per segment
-  const int share = ((max_pool + CL - 1) / CL + 3) / 4 * 4;
-  a.stage_entries = share <= kTopkStageMax ? share : 0;  // longer shares are read from global memory
-  const size_t smem = (size_t)(a.stage_entries + a.stage_entries / 32 + 1) * 4;
-  if (CL == 1) {
-    CATEKV_CUDA_TRY(launch_pdl(topk_kernel<1>, dim3(n_segs), dim3(kTopkThreads), smem, stream, a));
-    return CATEKV_OK;
-  }
-  // long lists: a cluster of 8 CTAs per segment
+template <int CL>
+static int launch_topk_cluster(const TopkArgs& a, int n_segs, size_t smem, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(n_segs * 8);
+  cfg.gridDim = dim3(n_segs * CL);
   cfg.blockDim = dim3(kTopkThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 8;
+  attr[0].val.clusterDim.x = CL;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  CATEKV_CUDA_TRY(cudaLaunchKernelEx(&cfg, topk_kernel<8>, a));
+  CATEKV_CUDA_TRY(cudaLaunchKernelEx(&cfg, topk_kernel<CL>, a));
+  return CATEKV_OK;
+}
+
+int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, int n_active, cudaStream_t stream) {
+  static bool attr_set[64] = {};
+  int dev = 0;
+  CATEKV_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    const int bytes = (kTopkStageMax + kTopkStageMax / 32 + 1) * 4;
+    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  TopkArgs a = a0;
+  // CTAs per segment: one for short lists, a cluster of 8 for long ones.  The cluster's barriers and exchanges cost
+  // about 10 us per call, one CTA's passes about 1.25 us per 1024 entries: the cluster pays from about 12 K entries
+  // (measured: 14.7 K entries 23 -> 17 us, 8.2 K entries 18 -> 29 us), provided the clusters of the segments that
+  // select fit one wave of resident CTAs (beyond 16 K entries a single CTA is slower in any case).
+  const int CL = (max_pool > 16384 || (max_pool >= 12288 && n_active * 8 <= 2 * 148)) ? 8 : 1;
+  const int share = ((max_pool + CL - 1) / CL + 3) / 4 * 4;
+  a.stage_entries = share <= kTopkStageMax ? share : 0;  // longer shares are read from global memory
+  const size_t smem = (size_t)(a.stage_entries + a.stage_entries / 32 + 1) * 4;
+  if (CL == 8) return launch_topk_cluster<8>(a, n_segs, smem, stream);
+  CATEKV_CUDA_TRY(launch_pdl(topk_kernel<1>, dim3(n_segs), dim3(kTopkThreads), smem, stream, a));
   return CATEKV_OK;
 }
 int launch_gather(const GatherArgs& a, int max_len, int n_segs, cudaStream_t stream) {
@@ -610,7 +617,9 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   {
     int max_pool = 0;
     for (const SelSeg& sg : segs) max_pool = sg.n_pool > max_pool ? sg.n_pool : max_pool;
-    int rc2 = launch_topk(ta, n_segs, max_pool, st);
+    int n_active = 0;
+    for (const SelSeg& sg : segs) n_active += (!sg.keep_all && sg.k_sel > 0) ? 1 : 0;
+    int rc2 = launch_topk(ta, n_segs, max_pool, n_active, st);
     if (rc2) return rc2;
   }
   GatherArgs ga;

@@ -50,7 +50,8 @@ struct GatherArgs {
 };
 
 
-int launch_topk(const TopkArgs& a, int n_segs, int max_pool, cudaStream_t stream);  // max_pool: longest pooled list
+// max_pool: longest pooled list; n_active: upper bound of the segments that select (the others leave at once)
+int launch_topk(const TopkArgs& a, int n_segs, int max_pool, int n_active, cudaStream_t stream);
 int launch_gather(const GatherArgs& a, int max_len, int n_segs, cudaStream_t stream);
 
 }  // namespace catekv
