@@ -48,6 +48,28 @@ def random_cache(B, Hkv, lens, seed, d=128):
     return oc
 
 
+def _bf16_ordinal(bits):
+    """bf16 bit patterns -> integers that are consecutive for adjacent values (+0 and -0 both map to 0)."""
+    b = np.asarray(bits).astype(np.int64)
+    mag = b & 0x7FFF
+    return np.where(b & 0x8000, -mag, mag)
+
+
+def bf16_tie_flips(got_bits, ref_bits, x_f32, ref_f64):
+    """Elements whose bf16 value differs from the rounded oracle value for the one excusable reason: the fp32 result
+    x_f32 and the oracle value sit on opposite sides of the midpoint of two adjacent bf16 numbers.
+
+    True where (i) got and ref are adjacent bf16 values and (ii) x lies within TIE_DIST of their midpoint, with
+    TIE_DIST = max |x_f32 - ref_f64| over the tensor (the measured fp32 error) + 4 fp32 ulps of x."""
+    differ = np.asarray(got_bits) != np.asarray(ref_bits)
+    adjacent = np.abs(_bf16_ordinal(got_bits) - _bf16_ordinal(ref_bits)) == 1
+    mid = 0.5 * (orc.bf16_to_f64(got_bits) + orc.bf16_to_f64(ref_bits))
+    x = np.asarray(x_f32, dtype=np.float64)
+    err = float(np.max(np.abs(x - ref_f64))) if x.size else 0.0
+    tie_dist = err + 4.0 * np.spacing(np.abs(x).astype(np.float32)).astype(np.float64)
+    return differ & adjacent & (np.abs(x - mid) <= tie_dist)
+
+
 def check_attention(out_f32, out_bf16, lse, ref, ref_lse, where=""):
     """ref: oracle fp64 [.., d]; NaN rows of ref are skipped."""
     ok = ~np.isnan(ref).any(axis=-1)
@@ -59,20 +81,24 @@ def check_attention(out_f32, out_bf16, lse, ref, ref_lse, where=""):
     if out_bf16 is not None:
         # The bf16 output is the same arithmetic rounded once at the end: bit-identical to the fp32 output of the
         # same call sequence rounded to nearest-even (which carries the parity claim against the fp64 oracle above).
-        if out_f32 is not None:
-            assert np.array_equal(synth.bits(out_bf16), synth.bits(out_f32.to(out_bf16.dtype))), (where, "bf16 != rne(fp32)")
-        # Against the oracle rounded to bf16 (like with like): rel-L2 <= 1e-3, except that an fp32 result within 1e-6
-        # of a rounding tie may land on the other neighbour.  Such flips are exactly one bf16 ulp (2^-6 for |x| in
-        # [2, 4), above the 1e-2 absolute bound) and rare; one of them on a large element of a small tensor already
-        # exceeds the rel-L2 bound, so up to 2 % of one-ulp flips are accepted in place of it.
-        g = orc.bf16_to_f64(synth.bits(out_bf16))[ok]
-        rb = orc.bf16_to_f64(orc.f64_to_bf16(r))
-        ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(rb), 2.0 ** -126))) - 7)
-        diff = np.abs(g - rb)
-        assert np.all(diff <= np.maximum(MAX_ABS, ulp)), (where, "bf16 max-abs", max_abs(g, rb))
-        flips = diff > 0
-        only_ties = np.all(diff[flips] <= ulp[flips] * 1.0000001) and flips.mean() <= 0.02
-        assert rel_l2(g, rb) <= REL_L2 or only_ties, (where, "bf16 rel-L2", rel_l2(g, rb), int(flips.sum()))
+        assert out_f32 is not None, "a bf16 output is checked together with the fp32 output of the same call"
+        assert np.array_equal(synth.bits(out_bf16), synth.bits(out_f32.to(out_bf16.dtype))), (where, "bf16 != rne(fp32)")
+        # Against the oracle rounded to bf16 (like with like).  Where the oracle's value and the fp32 result lie on
+        # opposite sides of a rounding tie they round to the two neighbours: one bf16 ulp apart (2^-6 for |x| in
+        # [2, 4), above the 1e-2 absolute bound).  Such an element is excused only when the cause shows: the two
+        # values are adjacent bf16 numbers and the fp32 result lies within TIE_DIST of their midpoint, TIE_DIST =
+        # the largest fp32-against-oracle error measured on this tensor + 4 fp32 ulps.  Every other element keeps
+        # rel-L2 <= 1e-3 and max-abs <= 1e-2.
+        gbits = synth.bits(out_bf16)[ok]
+        rbits = orc.f64_to_bf16(r)
+        g, rb = orc.bf16_to_f64(gbits), orc.bf16_to_f64(rbits)
+        x = out_f32.detach().cpu().double().numpy()[ok]
+        tie = bf16_tie_flips(gbits, rbits, x, r)
+        n_ties = int(tie.sum())
+        assert n_ties <= max(4, 0.005 * tie.size), (where, "too many rounding-tie flips to be chance", n_ties)
+        g_chk = np.where(tie, rb, g)
+        assert rel_l2(g_chk, rb) <= REL_L2, (where, "bf16 rel-L2", rel_l2(g_chk, rb), n_ties)
+        assert max_abs(g_chk, rb) <= MAX_ABS, (where, "bf16 max-abs", max_abs(g_chk, rb), n_ties)
     if lse is not None:
         gl = lse.detach().cpu().double().numpy()[ok]
         rl = ref_lse[ok]
@@ -110,4 +136,31 @@ def check_indices_band(got_idx, C, n, S, Lc, T, mode, param, where=""):
     assert set(must.tolist()) <= set(units.tolist()), (where, "missing clear winners")
     assert set(units.tolist()) <= set(may.tolist()), (where, "took a clear loser")
     assert len(units) == k_sel, where
+    return False
+
+
+def check_retrieval_band(got, scores, n, S, Lc, budget, cs, where=""):
+    """Band-aware comparison of the rows a retrieval head attends to with the oracle's (fp32 bounds on the device
+    against fp64 bounds): same length, ascending, every chunk whose bound is clearly above the k-th largest taken,
+    none clearly below it.  Returns True when the lists were identical."""
+    want = orc.retrieve_indices(scores, n, S, Lc, budget, cs)
+    got = np.asarray(got, dtype=np.int64)
+    assert got.shape == want.shape, (where, got.shape, want.shape)
+    assert np.all(np.diff(got) > 0), where
+    if np.array_equal(got, want):
+        return True
+    S2 = (S + cs - 1) // cs * cs
+    cand_end = (n - Lc) // cs * cs
+    P = scores[S2 // cs: cand_end // cs]
+    k_sel = (budget - S2 - (n - cand_end)) // cs
+    Pk = np.sort(P)[::-1][k_sel - 1]
+    tol = TIE_BAND * max(1.0, abs(Pk))
+    assert np.array_equal(got[:S2], np.arange(S2)) and np.array_equal(got[len(got) - (n - cand_end):],
+                                                                      np.arange(cand_end, n)), where
+    mid = got[S2:len(got) - (n - cand_end)]
+    assert np.all((mid - S2) % cs == np.tile(np.arange(cs), len(mid) // cs)), (where, "not whole chunks")
+    units = np.unique((mid - S2) // cs)
+    assert len(units) == k_sel, where
+    assert set(np.nonzero(P > Pk + tol)[0].tolist()) <= set(units.tolist()), (where, "missing clear winners")
+    assert set(units.tolist()) <= set(np.nonzero(P >= Pk - tol)[0].tolist()), (where, "took a clear loser")
     return False

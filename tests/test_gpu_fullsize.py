@@ -102,9 +102,9 @@ def _pick_cells(mask, want):
     return out
 
 
-def test_cfg1_32k_two_layers_steps_0_1_127(ck):
+def test_cfg1_32k_four_layers_steps_0_1_127(ck):
     w = synth.WORKLOADS["cfg1"]
-    for layer in (0, 17):
+    for layer in (0, 9, 17, 31):
         p, mask, cache, idx = _build_layer(ck, w, layer, w.decode_steps)
         cells = _pick_cells(mask, 4)
         oc = _check_selection_cells(w, p, mask, cache, idx, cells)
@@ -199,10 +199,7 @@ def test_cfg2_retrieval_on_adaptive_heads(ck):
         if rmask[s]:
             kmax, kmin = orc.retrieval_metadata(krows, cs)
             scores = orc.retrieval_scores(qb[0, s * w.G:(s + 1) * w.G], kmax, kmin)
-            want = orc.retrieve_indices(scores, L, w.sink, w.local, budget, cs)
-            assert got.shape == want.shape and np.all(np.diff(got) > 0)
-            # fp32 bounds against fp64 bounds: the sets may differ only among near-ties
-            assert len(np.setdiff1d(got, want)) <= 0.02 * len(want)
+            H.check_retrieval_band(got, scores, L, w.sink, w.local, budget, cs, f"cfg2 seg {s}")
         else:
             assert np.array_equal(got, np.arange(L))
         so = int(step.seg_off[s])
@@ -262,9 +259,7 @@ def test_cfg3_retrieval_in_place_as_the_bench_runs_it(ck):
             m = synth.bits(meta.view(torch.bfloat16).view(-1, 2, 128)[c0:c0 + kmax.shape[0]])
             assert np.array_equal(orc.bf16_to_f64(m[:, 0]), kmax) and np.array_equal(orc.bf16_to_f64(m[:, 1]), kmin)
             scores = orc.retrieval_scores(qb[b, h * w.G:(h + 1) * w.G], kmax, kmin)
-            want = orc.retrieve_indices(scores, L, w.sink, w.local, budget, cs)
-            assert got.shape == want.shape and np.all(np.diff(got) > 0)
-            assert len(np.setdiff1d(got, want)) <= 0.02 * len(want)  # fp32 against fp64 bounds: near-ties only
+            H.check_retrieval_band(got, scores, L, w.sink, w.local, budget, cs, f"cfg3 seg {s}")
         else:
             assert got_sel[s] == -1
             got = np.arange(L)

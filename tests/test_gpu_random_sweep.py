@@ -20,7 +20,9 @@ def ck():
     return pkg.binding
 
 
-@pytest.mark.parametrize("seed", range(12))
+# seeds 1262 and 3310: an fp32 result next to a bf16 rounding tie (the bf16 output lands on the other neighbour of
+# the rounded oracle value); kept as named cases of the tie rule in helpers.check_attention
+@pytest.mark.parametrize("seed", list(range(12)) + [1262, 3310])
 def test_random_decode_with_appends(ck, seed):
     rng = np.random.default_rng(1000 + seed)
     B, Hkv = int(rng.integers(1, 4)), int(rng.integers(1, 5))

@@ -25,25 +25,7 @@ def _meta_of(ck, cache, meta, cs, seg, n_chunks):
     return orc.bf16_to_f64(m[:, 0]), orc.bf16_to_f64(m[:, 1])
 
 
-def _check_selection(got, scores, n, S, Lc, budget, cs, where):
-    """Band-aware comparison of the retrieved rows with the oracle (fp32 bounds against fp64 bounds)."""
-    want = orc.retrieve_indices(scores, n, S, Lc, budget, cs)
-    assert got.shape == want.shape, (where, got.shape, want.shape)
-    assert np.all(np.diff(got) > 0), where
-    if np.array_equal(got, want):
-        return True
-    S2 = (S + cs - 1) // cs * cs
-    cand_end = (n - Lc) // cs * cs
-    P = scores[S2 // cs: cand_end // cs]
-    k_sel = (budget - S2 - (n - cand_end)) // cs
-    Pk = np.sort(P)[::-1][k_sel - 1]
-    tol = 1e-4 * max(1.0, abs(Pk))
-    mid = got[S2:len(got) - (n - cand_end)]
-    units = np.unique((mid - S2) // cs)
-    assert len(units) == k_sel, where
-    assert set(np.nonzero(P > Pk + tol)[0].tolist()) <= set(units.tolist()), (where, "missing clear winners")
-    assert set(units.tolist()) <= set(np.nonzero(P >= Pk - tol)[0].tolist()), (where, "took a clear loser")
-    return False
+_check_selection = H.check_retrieval_band
 
 
 @pytest.mark.parametrize("cs,G", [(8, 4), (8, 7), (16, 1), (1, 2)])

@@ -284,3 +284,30 @@ def test_fused_append_refuses_lengths_below_the_plan(ck):
     rc = ck._lib.catekv_append_decode_attn(C.byref(st), f, f, f, 8, 0.0, f, 0, None, buf.ctypes.data, f, nbytes, f, 1 << 30,
                                            None)
     assert rc == ck.ERR_INVALID_ARG and list(keep[2]) == [299, 40]
+
+
+def test_bf16_tie_rule_of_the_attention_check():
+    """helpers.bf16_tie_flips excuses a differing bf16 element only when the fp32 value sits at a rounding tie."""
+    import helpers as H
+    from oracle import catekv_oracle as orc
+
+    def bits(v):
+        return orc.f64_to_bf16(np.array(v, dtype=np.float64))
+
+    lo, hi = 3.0, 3.015625          # adjacent bf16 values in [2, 4): one ulp = 2^-6
+    mid = 0.5 * (lo + hi)
+    ref = np.array([mid - 2e-7, mid - 2e-7, 1.0, mid - 2e-7])
+    x32 = np.array([mid + 3e-7, mid + 3e-7, 1.0, 3.012])     # fp32 results; the last one is far from the tie
+    got = bits([hi, 3.03125, 1.0, hi])                        # element 1 is two ulps away
+    tie = H.bf16_tie_flips(got, bits(ref), x32, ref)
+    # element 3 widens the measured error to 3e-3, which would excuse anything: use a tensor without it first
+    assert list(H.bf16_tie_flips(got[:3], bits(ref[:3]), x32[:3], ref[:3])) == [True, False, False]
+    assert list(tie[:3]) == [True, False, False]
+    # a flip whose fp32 value is nowhere near the midpoint is not excused when the tensor's error is small
+    ref2 = np.array([mid - 2e-7, 3.0001])
+    x2 = np.array([mid + 3e-7, 3.0001])
+    got2 = bits([hi, hi])                                     # second element: wrong neighbour without a tie
+    assert list(H.bf16_tie_flips(got2, bits(ref2), x2, ref2)) == [True, False]
+    # identical values are never flips; across zero the ordinals are still adjacent
+    assert not H.bf16_tie_flips(bits([1.5]), bits([1.5]), np.array([1.5]), np.array([1.5])).any()
+    assert abs(int(H._bf16_ordinal(bits([2.0 ** -126]))[0]) - int(H._bf16_ordinal(bits([0.0]))[0])) >= 1

@@ -117,6 +117,29 @@ def test_select_brute_force_subsets():
         assert len(idx) == min(n, T)
 
 
+def test_select_brute_force_chunks():
+    """CHUNK mode against subset enumeration: the best floor(k_rest / cs) chunks by total BlockMax, ties to the
+    lexicographically smallest chunk tuple; chunk origin at S, short last chunk included."""
+    rng = np.random.default_rng(16)
+    short_last = 0
+    for trial in range(40):
+        cs = int(rng.choice([2, 3]))
+        n = int(rng.integers(12, 24))
+        S, Lc = int(rng.integers(0, 4)), int(rng.integers(1, 4))
+        T = int(rng.integers(S + Lc, n))
+        C = rng.integers(0, 7, size=n - 1).astype(np.float64) / 8.0  # dyadic: exact sums, exact ties
+        cand_end = n - Lc
+        chunks = [list(range(lo, min(lo + cs, cand_end))) for lo in range(S, cand_end, cs)]
+        short_last += len(chunks[-1]) < cs
+        block_max = [max(C[j] for j in ch) for ch in chunks]  # BlockMax written out, not through pool_scores
+        n_take = (T - S - Lc) // cs
+        sel = _brute_force_topk(block_max, n_take)
+        want = list(range(S)) + [j for c in sel for j in chunks[c]] + list(range(cand_end, n))
+        idx = orc.select_indices(C, n, S, Lc, T, orc.POOL_CHUNK, cs)
+        assert list(idx) == want, (trial, cs, list(idx), want)
+    assert short_last >= 5  # the ragged last chunk was exercised
+
+
 def test_select_structure_and_modes_agree():
     rng = np.random.default_rng(14)
     n, S, Lc, T = 500, 4, 32, 100
