@@ -155,6 +155,9 @@ def build_model(ck, w, dev, max_new, layers=None, time_select=True):
         e1.record()
         torch.cuda.synchronize()
         sel_ms.append(e0.elapsed_time(e1))
+        if cache.struct.reserved:  # chunk mode, short last chunk: the fused append needs the exact lengths
+            ck.catekv_cache_sync_lengths(cache)
+        ck.catekv_workspace_status(ws)  # raises if a scoring wait ran out
         plan = ck.DecodePlan(cache, num_ctas)
         t0 = time.perf_counter()
         ck.catekv_decode_plan(cache, plan)  # host: the schedule, plus one asynchronous copy to the device
@@ -393,8 +396,7 @@ def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8, graph=Tru
         m["meta"] = ck.catekv_retrieval_meta(c, cs)
         ck.catekv_retrieval_build(c, cs, m["meta"])
         m["rmask"] = (m["mask"].reshape(-1) == 0).astype(np.uint8)
-        m["ws"] = torch.empty(ck._lib.catekv_retrieve_workspace_bytes(w.B, w.Hkv, int(c.seg_cap.max())),
-                              dtype=torch.uint8, device=dev)
+        m["ws"] = ck.retrieve_workspace(c)
         m["lens"] = ck.catekv_retrieve_lengths(c, cs, m["rmask"], budget, w.sink, w.local)
         if gather:
             slens = [min(int(L), budget + 2 * cs + w.local) if m["rmask"][i] else int(L) + steps + 16

@@ -19,8 +19,11 @@
  *     launches nothing and changes no buffer.
  *   - "device" pointers are CUDA device memory owned by the caller; "host"
  *     pointers are ordinary host memory owned by the caller.  The library
- *     allocates no device memory and keeps no state between calls except the
- *     last CUDA error code (thread-local).
+ *     allocates no device memory.  Between calls it keeps the last CUDA error
+ *     code (thread-local) and, per device, a few values it looks up once (SM
+ *     count, which kernels have had their shared-memory limit raised, the
+ *     address of the fixed scratch array of catekv_decode_attn_noalloc); these
+ *     caches are atomics and safe to fill from several host threads.
  *   - Kernels are enqueued on the caller's stream (a cudaStream_t passed as
  *     void*); calls do not synchronise unless stated.
  *   - bf16 values are raw 16-bit patterns.  The head dimension d is the
@@ -48,6 +51,7 @@ extern "C" {
 #define CATEKV_ERR_CAPACITY (-3)    /* a segment would outgrow its capacity */
 #define CATEKV_ERR_WORKSPACE (-4)   /* workspace or plan buffer too small */
 #define CATEKV_ERR_CUDA (-5)        /* a CUDA call failed: see catekv_last_cuda_error() */
+#define CATEKV_ERR_DEVICE (-6)      /* a kernel reported a failure in a status block: see catekv_workspace_status() */
 
 #define CATEKV_POOL_NONE 0    /* top-k on the raw criticality C */
 #define CATEKV_POOL_CHUNK 1   /* BlockMax(C, cs) of Algorithm 1; whole chunks are selected */
@@ -89,7 +93,7 @@ typedef struct catekv_cache {
   int32_t B;              /* sequences */
   int32_t Hkv;            /* KV heads */
   int32_t d;              /* head dim, 128 */
-  int32_t reserved;
+  int32_t reserved;       /* 0; set to 1 by catekv_select_compact when seg_len (host) holds upper bounds */
   int64_t total_rows;     /* rows of each pool */
   void* k_pool;           /* device, bf16 [total_rows, d] */
   void* v_pool;           /* device, bf16 [total_rows, d] */
@@ -103,7 +107,65 @@ typedef struct catekv_cache {
                                  catekv_decode_plan, catekv_decode_attn / _partials / _combine / _noalloc,
                                  catekv_append_decode_attn and catekv_cache_regrow (as the source) follow them;
                                  every other call refuses such a cache with CATEKV_ERR_UNSUPPORTED */
+  const int32_t* seg_cap_dev; /* device [B*Hkv], copy of seg_cap, or NULL.  Kernels that write rows whose number
+                                 is decided on the device (the gather of catekv_retrieve_compact) clamp to it;
+                                 catekv_retrieve_compact requires it on its step cache */
 } catekv_cache;
+
+/*
+ * Device status block.  The first CATEKV_STATUS_BYTES of every workspace handed to catekv_select_compact,
+ * catekv_head_cv, catekv_retrieve_compact and catekv_retrieve_select belong to it.  Kernels never trap or assert:
+ * a kernel that cannot do its work records why here and returns, and the context stays usable.
+ *   CATEKV_STATUS_WAIT_EXPIRED  a bounded wait of the tensor-core scoring kernel ran out (the CTA freed its tensor
+ *                               memory and left); scores, and everything derived from them, are invalid
+ *   CATEKV_STATUS_CAPACITY      a gather was cut at the capacity of its destination segment (a replayed retrieval
+ *                               step whose step cache is too small for what the source has grown to)
+ *   CATEKV_STATUS_INDEX_RANGE   checked build only (catekv_checked_build): a device-produced row index, page or
+ *                               list position was outside its segment; the access was clamped into range
+ * kernel / segment / index describe the first failure recorded (kernel: 1 scoring, 2 top-k, 3 gather,
+ * 4 attention, 5 retrieval metadata).
+ * catekv_select_compact and catekv_head_cv clear the block when they start.  The retrieval calls never clear it
+ * (a replayed CUDA graph accumulates): zero the first CATEKV_STATUS_BYTES of a retrieval workspace once after
+ * allocating it, or read it with clear != 0.
+ */
+#define CATEKV_STATUS_BYTES 256
+#define CATEKV_STATUS_WAIT_EXPIRED 1
+#define CATEKV_STATUS_CAPACITY 2
+#define CATEKV_STATUS_INDEX_RANGE 4
+typedef struct catekv_status {
+  int32_t flags;   /* OR of CATEKV_STATUS_*; 0 = healthy */
+  int32_t kernel;
+  int32_t segment;
+  int32_t index;
+} catekv_status;
+
+/*
+ * Read the status block of workspace `ws` (device): copies it to *out (host, may be NULL) on `stream`,
+ * synchronises the stream, and with clear != 0 zeroes the block afterwards.  Returns CATEKV_OK if no flag is
+ * set, CATEKV_ERR_DEVICE if one is (the outputs of the calls that used the workspace since the block was last
+ * cleared are then not to be trusted), CATEKV_ERR_CUDA if the copy fails.
+ */
+int catekv_workspace_status(void* ws, catekv_status* out, int32_t clear, catekv_stream stream);
+
+/*
+ * Checked build (the stand-in for a memory checker on machines where none can be run): a library compiled with
+ * -DCATEKV_CHECKED (python -m paper_2608_30295_b200.build --checked) clamps every device-produced index to its
+ * segment before using it - the kept lists read by the gather, the row lists and page-table entries of the
+ * attention kernel, the positions the top-k writes, the chunk a metadata update folds into - and records the
+ * first violation in a status block of its own.  catekv_checked_build returns 1 for such a library, 0 otherwise.
+ * catekv_checked_status reads that block like catekv_workspace_status (device-wide synchronisation);
+ * CATEKV_ERR_UNSUPPORTED in an unchecked library.
+ */
+int catekv_checked_build(void);
+int catekv_checked_status(catekv_status* out, int32_t clear);
+
+/*
+ * Test hook, host side: the next n_launches launches of the scoring kernel run with their producer lane idle
+ * (no copy and no tensor-core instruction is issued) and a wait limit of 512 polls, so that every wait runs out
+ * with nothing in flight and the CATEKV_STATUS_WAIT_EXPIRED path executes.  Process-wide counter; 0 switches
+ * it off.  Nothing faults or hangs: the CTAs free their tensor memory and return.
+ */
+void catekv_test_expire_score_waits(int32_t n_launches);
 
 /* Version of this ABI (major * 1000 + minor). */
 int catekv_version(void);
@@ -188,14 +250,26 @@ typedef struct catekv_select_params {
  *   keeps every token.
  *
  *   idx_out  device int32 [B*Hkv, idx_stride] or NULL: the kept indices of each segment
- *   The host mirror cache->seg_len is exact on return.  It is computed on the host,
- *   except in CHUNK mode when (n - Lc - S) is not a multiple of cs: then the length
- *   depends on the data and the call synchronises the stream to read it back.
+ *   ws       device scratch; its first CATEKV_STATUS_BYTES are the status block (cleared by this call)
+ *   The call enqueues and returns; it never synchronises.  The host mirror cache->seg_len is
+ *   computed on the host and is exact on return, except in CHUNK mode when (n - Lc - S) is not
+ *   a multiple of cs and the head selects: whether the short last chunk is taken depends on the
+ *   scores, so the mirror then holds the upper bound (the device length is at most cs - 1 rows
+ *   shorter) and cache->reserved is set to 1.  catekv_cache_sync_lengths makes the mirror exact.
+ *   Everything that only needs an upper bound works on such a cache (capacity checks, decode
+ *   plans, catekv_decode_attn: every work item clamps to the device's length);
+ *   catekv_append_decode_attn needs exact lengths and refuses it (CATEKV_ERR_INVALID_ARG).
  *   Errors: CATEKV_ERR_CAPACITY if a kept list can exceed its segment capacity.
  */
 size_t catekv_select_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t n_max, int32_t L_obs);
 int catekv_select_compact(const catekv_select_params* p, catekv_cache* cache, int32_t* idx_out,
                           int64_t idx_stride, void* ws, size_t ws_bytes, catekv_stream stream);
+
+/*
+ * Copy the device's segment lengths into the host mirror cache->seg_len (on `stream`, which is synchronised)
+ * and clear cache->reserved.  Needed only after a catekv_select_compact that left upper bounds (see there).
+ */
+int catekv_cache_sync_lengths(catekv_cache* cache, catekv_stream stream);
 
 /* ---------------------------------------------------------------- decoding */
 
@@ -325,12 +399,18 @@ int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, 
  *   idx_out   device int32 [B*Hkv, idx_stride] or NULL: the rows taken from each segment
  *   ws        device scratch of at least catekv_retrieve_workspace_bytes(B, Hkv, largest seg_cap of `cache`)
  * Errors: CATEKV_ERR_CAPACITY if a kept list does not fit its segment of step_cache (nothing launched);
+ * CATEKV_ERR_INVALID_ARG if step_cache has no seg_cap_dev;
  * CATEKV_ERR_UNSUPPORTED for more than 2048 segments (the mask travels in the kernel arguments).
  * The call copies nothing from the host and takes every per-segment decision on the device from the device's
  * lengths; launch shapes follow the capacities.  A step (append, metadata append, this call, attention over
  * step_cache with a plan built once) can therefore be captured in a CUDA graph and replayed while the caches
  * grow; step_cache->seg_len on the host is then the value of the captured call (an upper bound: the kept
- * length moves within one chunk as the source grows).
+ * length moves within one chunk as the source grows).  The capacity check above sees the lengths of the call
+ * that was captured, not those of later replays: a step-cache segment that is copied whole (mask 0, or not
+ * longer than the budget) has to be as large as its source segment may become, one that retrieves needs
+ * budget + 2 * chunk_size rows.  On the device the gather never writes past seg_cap_dev of the step cache: a
+ * list that does not fit is cut there, step_cache's device length is set to the rows written, and
+ * CATEKV_STATUS_CAPACITY is raised in the status block at the start of `ws` (catekv_workspace_status).
  */
 size_t catekv_retrieval_meta_bytes(const catekv_cache* cache, int32_t chunk_size);
 int catekv_retrieval_build(const catekv_cache* cache, int32_t chunk_size, void* meta, catekv_stream stream);

@@ -15,9 +15,12 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libcatekv.so")
+# CATEKV_LIBRARY selects another build of the same library (the checked build, libcatekv_checked.so)
+LIB_PATH = os.environ.get("CATEKV_LIBRARY") or os.path.join(_HERE, "libcatekv.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA = 0, -1, -2, -3, -4, -5
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE = 0, -1, -2, -3, -4, -5, -6
+STATUS_BYTES = 256
+STATUS_WAIT_EXPIRED, STATUS_CAPACITY, STATUS_INDEX_RANGE = 1, 2, 4
 POOL_NONE, POOL_CHUNK, POOL_SLIDING = 0, 1, 2
 OUT_BF16, OUT_FP32 = 0, 1
 SEG_ALIGN = 128
@@ -43,7 +46,12 @@ class CacheStruct(C.Structure):
                 ("total_rows", C.c_int64), ("k_pool", C.c_void_p), ("v_pool", C.c_void_p),
                 ("seg_off_dev", C.c_void_p), ("seg_len_dev", C.c_void_p),
                 ("seg_off", C.c_void_p), ("seg_cap", C.c_void_p), ("seg_len", C.c_void_p),
-                ("pages", C.POINTER(PagesStruct))]
+                ("pages", C.POINTER(PagesStruct)), ("seg_cap_dev", C.c_void_p)]
+
+
+class StatusStruct(C.Structure):
+    _fields_ = [("flags", C.c_int32), ("kernel", C.c_int32), ("segment", C.c_int32), ("index", C.c_int32)]
+
 
 PAGE_ROWS = 64
 
@@ -102,6 +110,11 @@ def _load():
         "catekv_decode_attn_indexed": (C.c_int, [C.POINTER(CacheStruct), vp, i64, vp, vp, i32, f32, vp, i32, vp, vp, vp,
                                                  sz, vp, sz, vp]),
         "catekv_decode_attn_noalloc": (C.c_int, [C.POINTER(CacheStruct), vp, i32, f32, vp, i32, vp, vp, vp, sz, vp]),
+        "catekv_workspace_status": (C.c_int, [vp, C.POINTER(StatusStruct), i32, vp]),
+        "catekv_checked_build": (C.c_int, []),
+        "catekv_checked_status": (C.c_int, [C.POINTER(StatusStruct), i32]),
+        "catekv_test_expire_score_waits": (None, [i32]),
+        "catekv_cache_sync_lengths": (C.c_int, [C.POINTER(CacheStruct), vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -158,9 +171,11 @@ class Cache:
         self.v_pool = torch.empty((rows, d), dtype=torch.bfloat16, device=device)
         self.seg_off_dev = torch.from_numpy(self.seg_off).to(device)
         self.seg_len_dev = torch.zeros(B * Hkv, dtype=torch.int32, device=device)
+        self.seg_cap_dev = torch.from_numpy(self.seg_cap).to(device)
         self.struct = CacheStruct(B, Hkv, d, 0, self.total_rows, self.k_pool.data_ptr(), self.v_pool.data_ptr(),
                                   self.seg_off_dev.data_ptr(), self.seg_len_dev.data_ptr(),
-                                  _np_ptr(self.seg_off), _np_ptr(self.seg_cap), _np_ptr(self.seg_len), None)
+                                  _np_ptr(self.seg_off), _np_ptr(self.seg_cap), _np_ptr(self.seg_len), None,
+                                  self.seg_cap_dev.data_ptr())
         self.pages = None
 
     def attach_pages(self, n_pages: int, max_pages: int) -> "Pages":
@@ -189,7 +204,7 @@ class Pages:
         self.table = np.full((n, max_pages), -1, dtype=np.int32)
         self.table_dev = torch.full((n, max_pages), -1, dtype=torch.int32, device=cache.device)
         self.seg_pages = np.zeros(n, dtype=np.int32)
-        self.seg_cap_dev = torch.from_numpy(cache.seg_cap).to(cache.device)
+        self.seg_cap_dev = cache.seg_cap_dev
         self.struct = PagesStruct(max_pages, n_pages, 0, 0, self.k_ovf.data_ptr(), self.v_ovf.data_ptr(),
                                   self.table_dev.data_ptr(), _np_ptr(self.table), _np_ptr(self.seg_pages),
                                   self.seg_cap_dev.data_ptr())
@@ -198,6 +213,47 @@ class Pages:
 def catekv_append(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor):
     assert k_new.is_contiguous() and v_new.is_contiguous()
     _check(_lib.catekv_append(C.byref(cache.struct), k_new.data_ptr(), v_new.data_ptr(), _stream()), "catekv_append")
+
+
+def catekv_cache_sync_lengths(cache: Cache):
+    """Fetch the device's segment lengths into the host mirror (synchronises the current stream)."""
+    _check(_lib.catekv_cache_sync_lengths(C.byref(cache.struct), _stream()), "catekv_cache_sync_lengths")
+
+
+def catekv_workspace_status(ws: torch.Tensor, clear: bool = False, raise_on_error: bool = True) -> dict:
+    """Read the status block at the start of a select / head_cv / retrieval workspace (synchronises the current
+    stream).  -> {"flags", "kernel", "segment", "index"}; raises CatekvError(ERR_DEVICE) when a flag is set."""
+    st = StatusStruct()
+    rc = _lib.catekv_workspace_status(ws.data_ptr(), C.byref(st), 1 if clear else 0, _stream())
+    if rc != OK and (raise_on_error or rc != ERR_DEVICE):
+        raise CatekvError(rc, "catekv_workspace_status")
+    return {"flags": st.flags, "kernel": st.kernel, "segment": st.segment, "index": st.index}
+
+
+def catekv_checked_build() -> bool:
+    return bool(_lib.catekv_checked_build())
+
+
+def catekv_checked_status(clear: bool = False) -> dict:
+    """Checked build only: the library's own status block (device-wide synchronisation); never raises on flags."""
+    st = StatusStruct()
+    rc = _lib.catekv_checked_status(C.byref(st), 1 if clear else 0)
+    if rc not in (OK, ERR_DEVICE):
+        raise CatekvError(rc, "catekv_checked_status")
+    return {"flags": st.flags, "kernel": st.kernel, "segment": st.segment, "index": st.index}
+
+
+def catekv_test_expire_score_waits(n_launches: int):
+    """Test hook: the next n_launches scoring launches run with an idle producer lane and a 512-poll wait limit."""
+    _lib.catekv_test_expire_score_waits(int(n_launches))
+
+
+def retrieve_workspace(cache: Cache) -> torch.Tensor:
+    """A retrieval workspace for `cache` with its status block zeroed (memory only)."""
+    ws = torch.empty(_lib.catekv_retrieve_workspace_bytes(cache.B, cache.Hkv, int(cache.seg_cap.max())),
+                     dtype=torch.uint8, device=cache.device)
+    ws[:STATUS_BYTES].zero_()
+    return ws
 
 
 def catekv_cache_advance(cache: Cache, n_tokens: int = 1):
@@ -323,8 +379,7 @@ def catekv_retrieve_compact(cache: Cache, meta: torch.Tensor, chunk_size: int, q
     assert q.is_contiguous() and q.dtype == torch.bfloat16
     retrieval_mask = np.ascontiguousarray(retrieval_mask, dtype=np.uint8).reshape(-1)
     if ws is None:
-        ws = torch.empty(_lib.catekv_retrieve_workspace_bytes(cache.B, cache.Hkv, int(cache.seg_cap.max())),
-                         dtype=torch.uint8, device=cache.device)
+        ws = retrieve_workspace(cache)
     stride = 0 if idx_out is None else idx_out.stride(0)
     _check(_lib.catekv_retrieve_compact(C.byref(cache.struct), meta.data_ptr(), chunk_size, q.data_ptr(), q.shape[1],
                                         _np_ptr(retrieval_mask), budget, sink, local, C.byref(step_cache.struct),
@@ -360,7 +415,7 @@ class CacheView:
         self.seg_len = np.ascontiguousarray(lens, dtype=np.int32).reshape(-1).copy()
         b = cache.struct
         self.struct = CacheStruct(b.B, b.Hkv, b.d, 0, b.total_rows, b.k_pool, b.v_pool, b.seg_off_dev, b.seg_len_dev,
-                                  b.seg_off, b.seg_cap, _np_ptr(self.seg_len), None)
+                                  b.seg_off, b.seg_cap, _np_ptr(self.seg_len), None, b.seg_cap_dev)
 
 
 def catekv_retrieve_select(cache: Cache, meta: torch.Tensor, chunk_size: int, q: torch.Tensor, retrieval_mask,
@@ -370,8 +425,7 @@ def catekv_retrieve_select(cache: Cache, meta: torch.Tensor, chunk_size: int, q:
     assert idx.dtype == torch.int32 and sel_len.dtype == torch.int32 and idx.stride(1) == 1
     retrieval_mask = np.ascontiguousarray(retrieval_mask, dtype=np.uint8).reshape(-1)
     if ws is None:
-        ws = torch.empty(_lib.catekv_retrieve_workspace_bytes(cache.B, cache.Hkv, int(cache.seg_cap.max())),
-                         dtype=torch.uint8, device=cache.device)
+        ws = retrieve_workspace(cache)
     _check(_lib.catekv_retrieve_select(C.byref(cache.struct), meta.data_ptr(), chunk_size, q.data_ptr(), q.shape[1],
                                        _np_ptr(retrieval_mask), budget, sink, local, idx.data_ptr(), idx.stride(0),
                                        sel_len.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),

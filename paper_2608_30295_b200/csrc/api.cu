@@ -1,5 +1,6 @@
 // Host-only entry points: version, error text, pool layout, head classification.
 #include <algorithm>
+#include <atomic>
 #include <math.h>
 #include <vector>
 
@@ -8,9 +9,73 @@
 namespace catekv {
 static thread_local int g_last_cuda_error = 0;
 void set_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
+
+int sm_count() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return 148;
+  }
+  int v = cached[dev].load(std::memory_order_relaxed);
+  if (v > 0) return v;
+  if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+    cudaGetLastError();
+    return 148;
+  }
+  cached[dev].store(v, std::memory_order_relaxed);
+  return v;
+}
+
+#ifdef CATEKV_CHECKED
+static __device__ __align__(16) int32_t g_checked_status[4];
+int32_t* checked_status_ptr() {
+  static std::atomic<int32_t*> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  int32_t* p = cached[dev].load(std::memory_order_relaxed);
+  if (p) return p;
+  void* q = nullptr;
+  if (cudaGetSymbolAddress(&q, g_checked_status) != cudaSuccess) return nullptr;
+  cached[dev].store((int32_t*)q, std::memory_order_relaxed);
+  return (int32_t*)q;
+}
+#else
+int32_t* checked_status_ptr() { return nullptr; }
+#endif
+
+// copy a status block to the host, synchronise, optionally clear it
+static int read_status(int32_t* dev_block, catekv_status* out, int32_t clear, cudaStream_t st) {
+  catekv_status h = {0, 0, 0, 0};
+  CATEKV_CUDA_TRY(cudaMemcpyAsync(&h, dev_block, sizeof(h), cudaMemcpyDeviceToHost, st));
+  if (clear) CATEKV_CUDA_TRY(cudaMemsetAsync(dev_block, 0, sizeof(h), st));
+  CATEKV_CUDA_TRY(cudaStreamSynchronize(st));
+  if (out) *out = h;
+  return h.flags ? CATEKV_ERR_DEVICE : CATEKV_OK;
+}
 }  // namespace catekv
 
-extern "C" int catekv_version(void) { return 1000; }
+extern "C" int catekv_workspace_status(void* ws, catekv_status* out, int32_t clear, catekv_stream stream) {
+  if (!ws) return CATEKV_ERR_INVALID_ARG;
+  return catekv::read_status((int32_t*)ws, out, clear, (cudaStream_t)stream);
+}
+
+extern "C" int catekv_checked_build(void) {
+#ifdef CATEKV_CHECKED
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+extern "C" int catekv_checked_status(catekv_status* out, int32_t clear) {
+  int32_t* p = catekv::checked_status_ptr();
+  if (!p) return CATEKV_ERR_UNSUPPORTED;
+  CATEKV_CUDA_TRY(cudaDeviceSynchronize());
+  return catekv::read_status(p, out, clear, (cudaStream_t)0);
+}
+
+extern "C" int catekv_version(void) { return 2000; }
 
 extern "C" int catekv_last_cuda_error(void) { return catekv::g_last_cuda_error; }
 
@@ -22,6 +87,7 @@ extern "C" const char* catekv_error_string(int code) {
     case CATEKV_ERR_CAPACITY: return "segment capacity exceeded";
     case CATEKV_ERR_WORKSPACE: return "workspace or plan buffer too small";
     case CATEKV_ERR_CUDA: return "CUDA error";
+    case CATEKV_ERR_DEVICE: return "a kernel reported a failure in its status block";
     default: return "unknown error code";
   }
 }

@@ -80,8 +80,20 @@ extern "C" int catekv_cache_advance(catekv_cache* cache, int32_t n_tokens) {
   return CATEKV_OK;
 }
 
+extern "C" int catekv_cache_sync_lengths(catekv_cache* cache, catekv_stream stream) {
+  int rc = check_cache(cache);
+  if (rc) return rc;
+  const int n = cache->B * cache->Hkv;
+  CATEKV_CUDA_TRY(cudaMemcpyAsync(cache->seg_len, cache->seg_len_dev, sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToHost,
+                                  (cudaStream_t)stream));
+  CATEKV_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+  cache->reserved = 0;
+  return CATEKV_OK;
+}
+
 // Growth: every segment's valid rows move to the same segment of a cache with larger capacities.  One warp per
-// row (lanes 0-15 the K row, 16-31 the V row); block 0 of a segment records its length.
+// row (lanes 0-15 the K row, 16-31 the V row); block 0 of a segment records its length.  Like the gather, this
+// kernel writes rows a decode plan of the destination may cover: plain launch, no early signal to dependents.
 namespace catekv {
 constexpr int kRegrowRowsPerBlock = 64;
 __global__ void __launch_bounds__(256) regrow_kernel(const uint8_t* sk, const uint8_t* sv, const int32_t* s_off,
@@ -164,5 +176,6 @@ extern "C" int catekv_cache_regrow(const catekv_cache* src, catekv_cache* dst, c
                                                                page_args(src));
   CATEKV_CUDA_TRY(cudaGetLastError());
   for (int s = 0; s < n; ++s) dst->seg_len[s] = src->seg_len[s];
+  dst->reserved = src->reserved;  // upper-bound lengths stay upper bounds
   return CATEKV_OK;
 }

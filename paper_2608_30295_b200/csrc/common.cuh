@@ -28,9 +28,23 @@ void set_cuda_error(cudaError_t e);
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// SMs of the current device (looked up once per device; 148, the B200's count, when no device answers, so that
+// the workspace-size functions still work on a host without a GPU).
+int sm_count();
+
+// ---- device status block (the first CATEKV_STATUS_BYTES of a workspace, or the checked build's own block) ---
+enum KernelId { kKidScore = 1, kKidTopk = 2, kKidGather = 3, kKidAttention = 4, kKidMeta = 5 };
+// Device address of the checked build's status block; null in an unchecked library.
+int32_t* checked_status_ptr();
+
 // Launch with programmatic stream serialization: the grid may be scheduled while the previous kernel of
 // the stream is still draining; it must execute pdl_wait() before it touches anything that earlier work
 // on the stream produced.  After a kernel that never signals, this is an ordinary in-order launch.
+// Invariant the attention kernel relies on: it requests rows that were valid at plan time BEFORE its
+// pdl_wait().  A kernel that rewrites cache rows a plan already covers (gather_kernel, regrow_kernel) must
+// therefore never call pdl_launch_dependents(): as long as it does not, the dependent grid cannot start before
+// that kernel has completed and flushed, and the early requests see the rewritten rows.  Kernels that only
+// write rows behind every planned row (the appends) may signal early.
 template <class... KArgs, class... Args>
 static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                                      Args... args) {
@@ -55,6 +69,26 @@ struct ApiRange {
   ApiRange& operator=(const ApiRange&) = delete;
 };
 #define CATEKV_API_RANGE() ::catekv::ApiRange catekv_api_range_(__func__)
+
+// ---- device: record a failure in a status block {flags, kernel, segment, index}; the first reporter's details stay
+__device__ __forceinline__ void raise_status(int32_t* st, int flag, int kernel, int seg, int index) {
+  if (!st) return;
+  if (atomicOr(st, flag) == 0) {
+    st[1] = kernel;
+    st[2] = seg;
+    st[3] = index;
+  }
+}
+#ifdef CATEKV_CHECKED
+// Checked build: clamp a device-produced value into [lo, hi] and record a violation (never trap, never assert).
+__device__ __forceinline__ int checked_clamp(int v, int lo, int hi, int32_t* st, int kernel, int seg) {
+  if (v < lo || v > hi) {
+    raise_status(st, CATEKV_STATUS_INDEX_RANGE, kernel, seg, v);
+    v = v < lo ? lo : hi;
+  }
+  return v;
+}
+#endif
 
 // ---- device: programmatic dependent launch ------------------------------------------------
 // Let the next kernel of the stream be scheduled (it still waits, in pdl_wait, for this grid to finish).

@@ -11,6 +11,8 @@
 // the fp32 probabilities is lost.
 #include <math.h>
 
+#include <atomic>
+
 #include "decode.cuh"
 
 namespace catekv {
@@ -46,6 +48,8 @@ struct DecodeArgs {
   void* out;
   int32_t out_fp32;
   float* lse_out;
+  int32_t n_pages;  // pages of the overflow pools (checked build: bound of a page-table entry)
+  int32_t* chk;     // the checked build's status block, else null
 };
 
 constexpr int kStageBytes = 2 * kTile * kRowBytes;     // K tile + V tile
@@ -149,18 +153,6 @@ __device__ __forceinline__ void tile_rows(const ItemCursor& c, int i, int& start
   nvalid = c.live - start;
 }
 
-#ifdef CATEKV_TRACE
-__device__ unsigned long long g_trace[4096 * 4];
-__device__ __forceinline__ unsigned long long gtime() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-#define CATEKV_STAMP(i) do { if (threadIdx.x == 0) g_trace[blockIdx.x * 4 + (i)] = gtime(); } while (0)
-#else
-#define CATEKV_STAMP(i) do { } while (0)
-#endif
-
 template <int kMode>
 __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const DecodeArgs a) {
   constexpr bool kIndexed = kMode == kModeIndexed;
@@ -169,7 +161,6 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
   __shared__ ItemCursor s_ring[4];  // cursors of the pieces the producer has started, for the consumer
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
-  CATEKV_STAMP(0);
   pdl_launch_dependents();
   int item_begin, item_end;
   ItemCursor pc;
@@ -203,6 +194,11 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       const int32_t* row = a.page_table + (int64_t)pc.seg * a.max_pages;
       page0 = __ldg(row + min(pg0, a.max_pages - 1));
       page1 = __ldg(row + min(pg0 + 1, a.max_pages - 1));
+#ifdef CATEKV_CHECKED
+      // a page the tile's valid rows reach must have been handed out (an entry behind them may still be -1)
+      if (start + rows_left > pc.cap + pg0 * 64) page0 = checked_clamp(page0, 0, a.n_pages - 1, a.chk, kKidAttention, pc.seg);
+      if (start + rows_left > pc.cap + (pg0 + 1) * 64) page1 = checked_clamp(page1, 0, a.n_pages - 1, a.chk, kKidAttention, pc.seg);
+#endif
     }
 #pragma unroll
     for (int i = 0; i < (kTile * 16) / kDecodeThreads; ++i) {
@@ -212,6 +208,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       int64_t grow = ok ? row0 + r : 0;  // padding rows read nothing
       uint8_t* kp = a.k_pool;
       uint8_t* vp = a.v_pool;
+#ifdef CATEKV_CHECKED
+      // a list entry names a row of its own segment
+      if (kIndexed && pc.indexed && ok) ix[i] = checked_clamp(ix[i], 0, pc.cap - 1, a.chk, kKidAttention, pc.seg);
+#endif
       if (kIndexed && pc.indexed && ok) grow = (pc.row_base - pc.t0) + ix[i];
       if (kPaged && ok && start + r >= pc.cap) {  // the row lives in an overflow page
         const int o = start + r - pc.cap;
@@ -317,7 +317,6 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
       else
         cp_async_wait<kStages - 2>();
       __syncthreads();
-      if (seq == 0) CATEKV_STAMP(1);
       issue();
       if (tile == 0) {
         const uint8_t* qs = smem + kStages * kStageBytes + ((c_item - item_begin) % kStages) * kQSlotBytes;
@@ -397,7 +396,6 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     }
 
     // ---- end of the piece: finish the row sums, merge the four warps, write the result
-    if (c_item == item_end - 1) CATEKV_STAMP(2);
     if (cc.new_row >= 0 && tid == 0) a.seg_len[cc.seg] = cc.live;  // fused append: the segment has grown by one row
 #pragma unroll
     for (int sh = 4; sh <= 16; sh <<= 1) {
@@ -489,14 +487,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_partial_kernel(const
     }
   }
   cp_async_wait<0>();
-  CATEKV_STAMP(3);
 }
-
-#ifdef CATEKV_TRACE
-extern "C" int catekv_debug_trace(unsigned long long* host_out, int n_ctas) {
-  return (int)cudaMemcpyFromSymbol(host_out, g_trace, sizeof(unsigned long long) * 4 * n_ctas);
-}
-#endif
 
 // ------------------------------------------------------------------------------------------
 // Combine: merge the partials of every segment that was cut into several pieces
@@ -661,14 +652,14 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* k_ne
   float* part_lse = (float*)((uint8_t*)ws + off_lse);
   const int out_fp32 = out_dtype == CATEKV_OUT_FP32;
   if ((phases & 1) && hdr->n_items > 0) {
-    static bool attr_set[64] = {};
+    static std::atomic<bool> attr_set[64];
     int dev = 0;
     CATEKV_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
       CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<kModePlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
       CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<kModeIndexed>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
       CATEKV_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<kModePaged>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem));
-      if (dev >= 0 && dev < 64) attr_set[dev] = true;
+      if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
     }
     DecodeArgs a;
     a.k_pool = (uint8_t*)cache->k_pool;
@@ -697,6 +688,8 @@ static int decode_launch(int phases, const catekv_cache* cache, const void* k_ne
     a.v_ovf = pg.v_ovf;
     a.page_table = pg.table;
     a.max_pages = pg.max_pages;
+    a.n_pages = cache->pages ? cache->pages->n_pages : 0;
+    a.chk = checked_status_ptr();
     if (il)
       CATEKV_CUDA_TRY(launch_pdl(decode_partial_kernel<kModeIndexed>, dim3(hdr->num_ctas), dim3(kDecodeThreads), kDecodeSmem, st, a));
     else if (cache->pages)
@@ -764,6 +757,8 @@ extern "C" int catekv_append_decode_attn(catekv_cache* cache, const void* k_new,
   int rc = check_cache(cache);
   if (rc) return rc;
   if (!k_new || !v_new) return CATEKV_ERR_INVALID_ARG;
+  // the kernel places the appended row by the plan: the host lengths the plan was built from must be exact
+  if (cache->reserved) return CATEKV_ERR_INVALID_ARG;
   const int n = cache->B * cache->Hkv;
   for (int s = 0; s < n; ++s) {
     if (cache->seg_len[s] < 0) return CATEKV_ERR_INVALID_ARG;
@@ -801,19 +796,19 @@ extern "C" int catekv_decode_attn_noalloc(const catekv_cache* cache, const void*
                                           void* out, int32_t out_dtype, float* lse_out, const void* plan_host,
                                           const void* plan_dev, size_t plan_bytes, catekv_stream stream) {
   CATEKV_API_RANGE();
-  static void* scratch_of_device[64] = {};
+  static std::atomic<void*> scratch_of_device[64];
   int dev = 0;
   CATEKV_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return CATEKV_ERR_UNSUPPORTED;
-  if (!scratch_of_device[dev]) {
+  void* scratch = scratch_of_device[dev].load(std::memory_order_acquire);
+  if (!scratch) {
     // first call on this device (which is current): resolve the device address of the array
-    void* p = nullptr;
-    CATEKV_CUDA_TRY(cudaGetSymbolAddress(&p, g_decode_noalloc_scratch));
-    if (!p) return CATEKV_ERR_CUDA;
-    scratch_of_device[dev] = p;
+    CATEKV_CUDA_TRY(cudaGetSymbolAddress(&scratch, g_decode_noalloc_scratch));
+    if (!scratch) return CATEKV_ERR_CUDA;
+    scratch_of_device[dev].store(scratch, std::memory_order_release);
   }
   // decode_launch checks the plan and returns CATEKV_ERR_WORKSPACE when the partials of this plan
   // (num_ctas + B*Hkv slots) do not fit the fixed array
   return decode_launch(3, cache, nullptr, nullptr, q, Hq, sm_scale, out, out_dtype, lse_out, plan_host, plan_dev, plan_bytes,
-                       scratch_of_device[dev], (size_t)CATEKV_NOALLOC_SCRATCH_BYTES, stream);
+                       scratch, (size_t)CATEKV_NOALLOC_SCRATCH_BYTES, stream);
 }

@@ -180,21 +180,16 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
 
 struct CvWs {
   size_t off_status, off_segs, off_jobs, off_part, off_stats, off_A, bytes;
-  int keys_per_cta, n_chunks;
   int64_t row_stride;
 };
 static CvWs cv_ws_layout(int n_segs, int G, int m_max, int L_obs) {
   CvWs w;
-  int kp = 512;
-  while ((long)n_segs * ((m_max + kp - 1) / kp) > 148 * 4 && kp < (1 << 30)) kp *= 2;
-  w.keys_per_cta = kp;
-  w.n_chunks = (m_max + kp - 1) / kp;
   w.row_stride = (int64_t)align_up((size_t)m_max, 64);
   size_t o = 0;
-  w.off_status = o; o = 256;
+  w.off_status = o; o = CATEKV_STATUS_BYTES;
   w.off_segs = o; o = align_up(o + sizeof(CvSeg) * (size_t)n_segs, 256);
   w.off_jobs = o; o = align_up(o + sizeof(ScoreJob) * (size_t)n_segs, 256);
-  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs + 148 * 4) * 2 * kScoreMaxRows, 256);
+  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)score_max_ctas(n_segs) * 2 * kScoreMaxRows, 256);
   w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * kScoreMaxRows, 256);
   w.off_A = o; o = align_up(o + sizeof(float) * (size_t)n_segs * L_obs * w.row_stride, 256);
   w.bytes = o;
@@ -252,7 +247,7 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   }
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* w8 = (uint8_t*)ws;
-  CATEKV_CUDA_TRY(cudaMemsetAsync(w8 + W.off_status, 0, 256, st));
+  CATEKV_CUDA_TRY(cudaMemsetAsync(w8 + W.off_status, 0, CATEKV_STATUS_BYTES, st));
   CATEKV_CUDA_TRY(cudaMemcpyAsync(w8 + W.off_segs, segs.data(), sizeof(CvSeg) * n_segs, cudaMemcpyHostToDevice, st));
   CATEKV_CUDA_TRY(cudaMemcpyAsync(w8 + W.off_jobs, jobs.data(), sizeof(ScoreJob) * n_segs, cudaMemcpyHostToDevice, st));
   ScoreArgs sa = {};

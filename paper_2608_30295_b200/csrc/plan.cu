@@ -26,9 +26,6 @@ extern "C" int catekv_decode_plan(const catekv_cache* cache, int32_t num_ctas, v
   // since the plan was built, it stores the appended row, and it finishes one piece and starts the next (merge of
   // the warps, output, the next group's queries) while nothing new is issued.  Every non-empty segment's end is
   // therefore charged kSegEndCharge rows, so that those CTAs get fewer plan-time rows and do not finish last.
-  // Measured per-CTA stream times put the cost of a segment end at 250-330 rows' worth of streaming; between a
-  // charge of 64 and of 256 rows configs[1] went from 19.7 to 17.1 us and configs[2] from 36.3 to 34.0 us per
-  // layer-step (flat from 256 to 512).
   int64_t total = 0, charged = 0;
   for (int s = 0; s < n_segs; ++s) {
     if (cache->seg_len[s] < 0 || cache->seg_len[s] > seg_capacity(cache, s)) return CATEKV_ERR_INVALID_ARG;

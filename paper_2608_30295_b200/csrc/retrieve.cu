@@ -11,6 +11,8 @@
 //              catekv_decode_attn then runs unchanged
 #include <math.h>
 
+#include <atomic>
+
 #include "select.cuh"
 
 namespace catekv {
@@ -47,6 +49,7 @@ __global__ void __launch_bounds__(256) meta_build_kernel(const uint8_t* k_pool, 
 
 // Fold row r of a segment (its key given as this lane's 8 bytes, w) into the metadata of its chunk.
 __device__ __forceinline__ void meta_fold_row(uint8_t* meta, int64_t seg_row0, int r, int cs, int lane, uint2 w) {
+  // (checked build: the callers clamp r to the segment's capacity before they get here)
   uint8_t* dst = meta + (seg_row0 / cs + r / cs) * (2 * kRowBytes) + lane * 8;
   if (r % cs == 0) {
     *reinterpret_cast<uint2*>(dst) = w;
@@ -63,14 +66,18 @@ __device__ __forceinline__ void meta_fold_row(uint8_t* meta, int64_t seg_row0, i
 
 // After an append: fold the newest row (index len - 1) into its chunk.  One warp per segment.
 __global__ void __launch_bounds__(128) meta_append_kernel(const int32_t* seg_off, const int32_t* seg_len, const uint8_t* k_new,
-                                                          uint8_t* meta, int cs, int n_segs) {
+                                                          uint8_t* meta, int cs, int n_segs, const int32_t* seg_cap,
+                                                          int32_t* chk) {
   const int seg = blockIdx.x * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   pdl_launch_dependents();
   pdl_wait();  // the length and k_new come from earlier kernels of the stream
   if (seg >= n_segs) return;
-  const int r = seg_len[seg] - 1;
+  int r = seg_len[seg] - 1;
   if (r < 0) return;
+#ifdef CATEKV_CHECKED
+  if (seg_cap) r = checked_clamp(r, 0, seg_cap[seg] - 1, chk, kKidMeta, seg);
+#endif
   const uint2 w = *reinterpret_cast<const uint2*>(k_new + (size_t)seg * kRowBytes + lane * 8);
   meta_fold_row(meta, seg_off[seg], r, cs, lane, w);
 }
@@ -79,13 +86,17 @@ __global__ void __launch_bounds__(128) meta_append_kernel(const int32_t* seg_off
 // 16-31 the V row (16 bytes each), all 32 fold the key into its chunk, lane 0 bumps the length.
 __global__ void __launch_bounds__(128) append_meta_kernel(uint8_t* k_pool, uint8_t* v_pool, const int32_t* seg_off,
                                                           int32_t* seg_len, const uint8_t* k_new, const uint8_t* v_new,
-                                                          uint8_t* meta, int cs, int n_segs) {
+                                                          uint8_t* meta, int cs, int n_segs, const int32_t* seg_cap,
+                                                          int32_t* chk) {
   const int seg = blockIdx.x * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   pdl_launch_dependents();
   pdl_wait();
   if (seg >= n_segs) return;
-  const int len = seg_len[seg];
+  int len = seg_len[seg];
+#ifdef CATEKV_CHECKED
+  if (seg_cap) len = checked_clamp(len, 0, seg_cap[seg] - 1, chk, kKidMeta, seg);  // the row must fit the segment
+#endif
   const int64_t row0 = seg_off[seg];
   const int c = lane & 15;
   const uint8_t* src = (lane < 16 ? k_new : v_new) + (size_t)seg * kRowBytes + c * 16;
@@ -262,7 +273,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) retrieval_score_kernel(const Re
 }
 
 struct RetWs {
-  size_t off_segs, off_P, off_idx, bytes;
+  size_t off_status, off_segs, off_P, off_idx, bytes;
   int64_t p_stride, idx_stride;
 };
 static RetWs ret_ws_layout(int n_segs, int max_len) {
@@ -270,6 +281,7 @@ static RetWs ret_ws_layout(int n_segs, int max_len) {
   w.p_stride = (int64_t)align_up((size_t)(max_len > 0 ? max_len : 1), 64);
   w.idx_stride = w.p_stride;
   size_t o = 0;
+  w.off_status = o; o = CATEKV_STATUS_BYTES;
   w.off_segs = o; o = align_up(o + sizeof(SelSeg) * (size_t)n_segs, 256);
   w.off_P = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.p_stride, 256);
   w.off_idx = o; o = align_up(o + sizeof(int32_t) * (size_t)n_segs * w.idx_stride, 256);
@@ -322,7 +334,8 @@ extern "C" int catekv_retrieval_append(const catekv_cache* cache, int32_t chunk_
   if (!chunk_size_ok(chunk_size)) return CATEKV_ERR_UNSUPPORTED;
   const int n_segs = cache->B * cache->Hkv;
   CATEKV_CUDA_TRY(launch_pdl(meta_append_kernel, dim3((n_segs + 3) / 4), dim3(128), 0, (cudaStream_t)stream,
-                             cache->seg_off_dev, cache->seg_len_dev, (const uint8_t*)k_new, (uint8_t*)meta, chunk_size, n_segs));
+                             cache->seg_off_dev, cache->seg_len_dev, (const uint8_t*)k_new, (uint8_t*)meta, chunk_size, n_segs,
+                             cache->seg_cap_dev, checked_status_ptr()));
   return CATEKV_OK;
 }
 
@@ -340,7 +353,8 @@ extern "C" int catekv_append_retrieval(catekv_cache* cache, const void* k_new, c
   }
   CATEKV_CUDA_TRY(launch_pdl(append_meta_kernel, dim3((n_segs + 3) / 4), dim3(128), 0, (cudaStream_t)stream,
                              (uint8_t*)cache->k_pool, (uint8_t*)cache->v_pool, cache->seg_off_dev, cache->seg_len_dev,
-                             (const uint8_t*)k_new, (const uint8_t*)v_new, (uint8_t*)meta, chunk_size, n_segs));
+                             (const uint8_t*)k_new, (const uint8_t*)v_new, (uint8_t*)meta, chunk_size, n_segs,
+                             cache->seg_cap_dev, checked_status_ptr()));
   for (int s = 0; s < n_segs; ++s) cache->seg_len[s] += 1;
   return CATEKV_OK;
 }
@@ -362,6 +376,7 @@ static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t ch
     rc = check_cache_r(step_cache);
     if (rc) return rc;
     if (step_cache->B != cache->B || step_cache->Hkv != cache->Hkv) return CATEKV_ERR_INVALID_ARG;
+    if (!step_cache->seg_cap_dev) return CATEKV_ERR_INVALID_ARG;  // the gather clamps to it on the device
   } else if (!idx_out || !sel_len) {
     return CATEKV_ERR_INVALID_ARG;
   }
@@ -412,16 +427,16 @@ static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t ch
     int n_ret = 0;
     for (int s = 0; s < n_segs; ++s) n_ret += retrieval_mask[s] != 0;
     const int tiles = (max_pool + kRsTile - 1) / kRsTile;
-    int gx = n_ret > 0 ? (2 * 148) / n_ret : 1;
+    int gx = n_ret > 0 ? (2 * sm_count()) / n_ret : 1;
     if (gx > tiles) gx = tiles;
     if (gx > 64) gx = 64;
     if (gx < 1) gx = 1;
-    static bool attr_set[64] = {};
+    static std::atomic<bool> attr_set[64];
     int dev = 0;
     CATEKV_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
       CATEKV_CUDA_TRY(cudaFuncSetAttribute(retrieval_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRsSmem));
-      if (dev >= 0 && dev < 64) attr_set[dev] = true;
+      if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
     }
     sa.seg_len = cache->seg_len_dev;
     sa.seg_off = cache->seg_off_dev;
@@ -469,6 +484,8 @@ static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t ch
   ga.idx_out = idx_out;
   ga.idx_out_stride = idx_stride;
   ga.Hkv = cache->Hkv;
+  ga.seg_cap = step_cache->seg_cap_dev;
+  ga.status = (int32_t*)(w8 + W.off_status);
   rc = launch_gather(ga, max_step_cap, n_segs, st);
   if (rc) return rc;
   for (int s = 0; s < n_segs; ++s) step_cache->seg_len[s] = retrieval_decide(cache->seg_len[s], retrieval_mask[s] != 0, rp).len_ub;

@@ -26,6 +26,8 @@
 #include <cuda.h>
 #include <math.h>
 
+#include <atomic>
+
 #include "score.cuh"
 
 namespace catekv {
@@ -98,8 +100,8 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 // Bounded wait for a phase of an mbarrier.  Returns false if it never completed or if another thread of
 // the CTA has given up (abort flag), in which case the flag is (also) raised by this thread.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     uint32_t done;
     asm volatile(
         "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
@@ -234,13 +236,13 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
 
   if (warp == 8) {
     // ================= TMA + MMA issue: one elected lane =================
-    if (lane == 0) {
+    if (lane == 0 && !a.idle_producer) {
       for (int tl = 0; tl < 2 && tl < n_tiles; ++tl) load_tile(tl);
       const uint32_t idesc = kStats ? umma_idesc_bf16(128, 128) : umma_idesc_bf16(128, sh.NW);
       for (int v = 0; v < U; ++v) {
         const int tile = v / UPT, sub = v - tile * UPT;
-        if (sub == 0 && !mbar_wait(bar_full + 8 * (tile & 1), (uint32_t)((tile >> 1) & 1), s_abort)) break;
-        if (v >= NSLOT && !mbar_wait(bar_free + 8 * (v % NSLOT), (uint32_t)(((v / NSLOT) - 1) & 1), s_abort)) break;
+        if (sub == 0 && !mbar_wait(bar_full + 8 * (tile & 1), (uint32_t)((tile >> 1) & 1), s_abort, a.spin_limit)) break;
+        if (v >= NSLOT && !mbar_wait(bar_free + 8 * (v % NSLOT), (uint32_t)(((v / NSLOT) - 1) & 1), s_abort, a.spin_limit)) break;
         tc_fence_after();
         const uint32_t sk = s_k + (tile & 1) * kKStageBytes;
         const uint32_t d = tmem + (uint32_t)((v % NSLOT) * slot_w);
@@ -270,7 +272,7 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
 
     for (int u = 0; u < U; ++u) {
       const int tile = u / UPT, sub = u - tile * UPT;
-      if (!mbar_wait(bar_done + 8 * (u % NSLOT), (uint32_t)((u / NSLOT) & 1), s_abort)) break;
+      if (!mbar_wait(bar_done + 8 * (u % NSLOT), (uint32_t)((u / NSLOT) & 1), s_abort, a.spin_limit)) break;
       tc_fence_after();
       // the MMAs of this tile have read its stage: re-arm the stage with the tile after next
       if (tid == 0 && sub == UPT - 1 && tile + 2 < n_tiles) load_tile(tile + 2);
@@ -433,7 +435,7 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
   __syncthreads();
   if (warp == 8) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(n_cols) : "memory");
   if (*s_abort) {
-    if (tid == 0) atomicExch(a.status, 1);
+    if (tid == 0) raise_status(a.status, CATEKV_STATUS_WAIT_EXPIRED, kKidScore, (int)blockIdx.y, (int)blockIdx.x);
     return;
   }
   if (kStats) {
@@ -507,8 +509,21 @@ static int make_k_map(const ScoreArgs& a, CUtensorMap* map) {
   return r == CUDA_SUCCESS ? CATEKV_OK : CATEKV_ERR_UNSUPPORTED;
 }
 
+// Test hook (catekv_test_expire_score_waits): launches left that run with an idle producer lane.
+static std::atomic<int> g_expire_launches{0};
+
 template <int MODE>
-static int launch_one(const ScoreArgs& a, const ScoreShape& sh, const CUtensorMap& map, cudaStream_t stream) {
+static int launch_one(const ScoreArgs& a0, const ScoreShape& sh, const CUtensorMap& map, cudaStream_t stream) {
+  ScoreArgs a = a0;
+  a.spin_limit = kSpinLimit;
+  a.idle_producer = 0;
+  int left = g_expire_launches.load(std::memory_order_relaxed);
+  while (left > 0 && !g_expire_launches.compare_exchange_weak(left, left - 1)) {
+  }
+  if (left > 0) {
+    a.spin_limit = 512;
+    a.idle_producer = 1;
+  }
   const size_t smem = score_smem_bytes(sh);
   CATEKV_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   score_tc_kernel<MODE><<<dim3(a.n_chunks, a.n_jobs), kScThreads, smem, stream>>>(map, a, sh);
@@ -518,7 +533,8 @@ static int launch_one(const ScoreArgs& a, const ScoreShape& sh, const CUtensorMa
 
 int score_keys_per_cta(int n_jobs, int max_keys) {
   if (n_jobs < 1) n_jobs = 1;
-  int chunks = (296 + n_jobs / 2) / n_jobs;  // about 296 CTAs in all
+  const int ctas = 2 * sm_count();                 // the kernel runs two CTAs per SM
+  int chunks = (ctas + n_jobs / 2) / n_jobs;  // about one full wave in all
   if (chunks < 1) chunks = 1;
   int kp = ((max_keys + chunks - 1) / chunks + kKeyTile - 1) / kKeyTile * kKeyTile;
   if (kp < 4 * kKeyTile) kp = 4 * kKeyTile;  // at least a few tiles per CTA: the queries are staged once per CTA
@@ -546,3 +562,7 @@ int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream) {
 }
 
 }  // namespace catekv
+
+extern "C" void catekv_test_expire_score_waits(int32_t n_launches) {
+  catekv::g_expire_launches.store(n_launches > 0 ? n_launches : 0);
+}

@@ -25,7 +25,9 @@ struct ScoreArgs {
   int32_t n_chunks;       // grid.x: ceil(max key range / keys_per_cta)
   float2* stats_part;     // [n_jobs][n_chunks][kScoreMaxRows]  per-CTA (row max in the log2 domain, row sum)
   float2* stats;          // [n_jobs][kScoreMaxRows]            merged (row max, row sum)
-  int32_t* status;        // device word, set to 1 if a tensor-core wait ever expired (never in a healthy run)
+  int32_t* status;        // device status block: CATEKV_STATUS_WAIT_EXPIRED is raised if a tensor-core wait ever runs out
+  uint32_t spin_limit;    // polls a wait may take (set by score_launch)
+  int32_t idle_producer;  // test hook: the TMA / MMA lane issues nothing, so every wait runs out (set by score_launch)
   float* out;             // column sums C[job][j - j_begin], or the dense matrix A[job][i * m + (j - j_begin)], m = j_end - j_begin
   int64_t out_job_stride;
 };
@@ -34,8 +36,11 @@ enum ScoreMode { kScoreStats = 0, kScoreColsum = 1, kScoreMatrix = 2 };
 
 constexpr int kScoreMaxRows = 512;  // G * L_obs may not exceed this (8 heads x 64 window rows)
 // Keys per CTA for n_jobs jobs of at most max_keys keys: a multiple of 128 chosen so that the grid is close to two
-// CTAs per SM in whole waves (never more than 592 CTAs unless there are more jobs than that).
+// CTAs per SM in whole waves (never more than score_max_ctas(n_jobs)).
 int score_keys_per_cta(int n_jobs, int max_keys);
+// Upper bound of n_jobs * n_chunks for keys_per_cta = score_keys_per_cta(n_jobs, .): the per-CTA row partials of
+// pass 1 are sized by it.  (chunks = round(2 SMs / jobs), so jobs * chunks <= 2 SMs + jobs / 2.)
+static inline int score_max_ctas(int n_jobs) { return n_jobs + 4 * sm_count(); }
 // Enqueue: pass 1 (row max / sum partials), their merge, and pass 2 (column sums or matrix).
 int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream);
 

@@ -3,6 +3,7 @@
 // head's segment of the pool.
 #include <math.h>
 
+#include <atomic>
 #include <vector>
 
 #include <cooperative_groups.h>
@@ -17,19 +18,6 @@ namespace catekv {
 
 constexpr int kTopkThreads = 1024;
 
-#ifdef CATEKV_TOPK_TRACE
-__device__ unsigned long long g_topk_trace[64 * 16];
-#define TOPK_STAMP(i)                                                                       \
-  do {                                                                                      \
-    if (threadIdx.x == 0 && blockIdx.x < 64) {                                              \
-      unsigned long long t_;                                                                \
-      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                                 \
-      g_topk_trace[blockIdx.x * 16 + (i)] = t_;                                             \
-    }                                                                                       \
-  } while (0)
-#else
-#define TOPK_STAMP(i)
-#endif
 
 // Block-wide exclusive scan of a packed pair (lo 32 bits, hi 32 bits) over 1024 threads.
 __device__ __forceinline__ unsigned long long block_excl_scan(unsigned long long v, unsigned long long* s_warp,
@@ -76,7 +64,6 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     if (a.mark_keep_all && rank == 0 && threadIdx.x == 0) a.seg_len_dev[seg] = -1;
     return;
   }
-  TOPK_STAMP(0);
   __shared__ unsigned int hist[256];
   __shared__ unsigned int hsum[256];
   __shared__ unsigned long long s_warp[33];
@@ -194,7 +181,6 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
       gmax = max(gmax, CL > 1 ? *cluster.map_shared_rank(&s_mm[1], r) : s_mm[1]);
     }
     auto ldp = [&](int i) { return staged ? stage[sp(i)] : Pg[lo + i]; };  // entry i of this CTA's share
-    TOPK_STAMP(1);
     // ---- radix select of the k_sel-th largest pooled score (scores are >= 0, so their bit patterns order as
     // integers).  The bits above the highest bit in which the extremes differ are common to all entries and become
     // the prefix; the nb bits below are resolved from the top, up to 8 per pass, with the CTAs' histograms summed
@@ -245,7 +231,6 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
       prefix = s_pair[0];
       need = s_pair[1];
       nb = shift;
-      TOPK_STAMP(2 + pass_no);
       ++pass_no;
     }
     const unsigned int thr = prefix, need_eq = need;  // threshold bits; ties taken (lowest index first)
@@ -255,6 +240,14 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     // entries go, and it writes them in order.
     const int cs = (a.pool_mode == CATEKV_POOL_CHUNK || a.pool_mode == kPoolPrescored) ? a.pool_param : 1;
     auto emit = [&](int c, unsigned int rnk) {  // pooled entry c of the segment is the rnk-th selected one
+#ifdef CATEKV_CHECKED
+      // the rank must be one of the k_sel slots and the list position inside the segment's row of idx
+      rnk = (unsigned int)checked_clamp((int)rnk, 0, s.k_sel - 1, a.chk, kKidTopk, seg);
+      if ((int64_t)S + ((int64_t)rnk + 1) * cs > a.idx_stride) {
+        raise_status(a.chk, CATEKV_STATUS_INDEX_RANGE, kKidTopk, seg, (int)rnk);
+        return;
+      }
+#endif
       if (cs == 1) {
         idx[S + rnk] = S + c;
       } else {
@@ -281,7 +274,6 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
         if (r < rank) ex += t;
         all += t;
       }
-      TOPK_STAMP(6);
       for (int i = r0; i < r1; ++i) {
         const unsigned int v = stage[sp(i)];
         const bool gt = v > thr, eq = v == thr;
@@ -308,7 +300,6 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
         if (r < rank) run += t;
         all += t;
       }
-      TOPK_STAMP(6);
       for (int base = lo; base < hi; base += 4 * kTopkThreads) {
         const int c4 = base + tid * 4;
         unsigned int v[4];
@@ -332,7 +323,6 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
         run += tot;
       }
     }
-    TOPK_STAMP(7);
     // selected tokens: whole chunks, except that the last chunk of the range may be short
     n_sel_tokens = s.k_sel * cs;
     if (cs > 1) {
@@ -352,17 +342,28 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     for (int i = tid; i < n_tail; i += kTopkThreads) idx[S + n_sel_tokens + i] = s.cand_end + i;
     if (tid == 0) a.seg_len_dev[seg] = S + n_sel_tokens + n_tail;
   }
-  TOPK_STAMP(8);
 }
 
 constexpr int kGatherRowsPerBlock = 64;
 
 // One warp per kept row: lanes 0-15 move the K row, lanes 16-31 the V row (16 bytes each).
+// This kernel rewrites rows that a decode plan may already cover: it is launched without the programmatic-launch
+// attribute and never signals its dependents early (see launch_pdl), so the attention kernel that follows cannot
+// request those rows before they are written.
 __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
   const int seg = blockIdx.y;
   const SelSeg s = a.segs[seg];
-  const int len = s.keep_all ? s.n : a.seg_len_dev[seg];  // a straight copy keeps all n rows
-  if (s.keep_all && blockIdx.x == 0 && threadIdx.x == 0) a.seg_len_dev[seg] = s.n;
+  int len = s.keep_all ? s.n : a.seg_len_dev[seg];  // a straight copy keeps all n rows
+  // Never write past the destination segment: a list that does not fit (a replayed retrieval step whose step
+  // cache is too small for what the source has grown to) is cut at the capacity, the length says so, and the
+  // status block records it.  Every block of the segment takes the same decision.
+  const int cap = a.seg_cap ? a.seg_cap[seg] : 0x7fffffff;
+  const bool cut = len > cap;
+  if (cut) len = cap;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (s.keep_all || cut) a.seg_len_dev[seg] = len;
+    if (cut) raise_status(a.status, CATEKV_STATUS_CAPACITY, kKidGather, seg, s.keep_all ? s.n : cap + 1);
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = seg / a.Hkv, h = seg % a.Hkv;
   const int64_t off = a.seg_off[seg];
@@ -374,7 +375,10 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
   for (int i = warp; i < kGatherRowsPerBlock; i += 8) {
     const int r = r0 + i;
     if (r >= len) break;
-    const int tok = s.keep_all ? r : a.idx[(size_t)seg * a.idx_stride + r];
+    int tok = s.keep_all ? r : a.idx[(size_t)seg * a.idx_stride + r];
+#ifdef CATEKV_CHECKED
+    tok = checked_clamp(tok, 0, s.n - 1, a.chk, kKidGather, seg);  // a kept index names a row of the source list
+#endif
     const uint4 val = __ldg(reinterpret_cast<const uint4*>(src_base + (int64_t)tok * a.st));
     *reinterpret_cast<uint4*>(dst_base + (int64_t)r * kRowBytes) = val;
     if (a.idx_out && lane == 0) a.idx_out[(size_t)seg * a.idx_out_stride + r] = tok;
@@ -382,14 +386,6 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
 }
 
 constexpr int kTopkStageMax = 32768;  // pooled entries a CTA may stage in shared memory (132 KB with the padding)
-
-#ifdef CATEKV_TOPK_TRACE
-}  // namespace catekv
-extern "C" int catekv_debug_topk_trace(unsigned long long* host_out) {
-  return (int)cudaMemcpyFromSymbol(host_out, catekv::g_topk_trace, sizeof(unsigned long long) * 64 * 16);
-}
-namespace catekv {
-#endif
 
 template <int CL>
 static int launch_topk_cluster(const TopkArgs& a, int n_segs, size_t smem, cudaStream_t stream) {
@@ -412,21 +408,22 @@ static int launch_topk_cluster(const TopkArgs& a, int n_segs, size_t smem, cudaS
 }
 
 int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, int n_active, cudaStream_t stream) {
-  static bool attr_set[64] = {};
+  static std::atomic<bool> attr_set[64];
   int dev = 0;
   CATEKV_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+  if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
     const int bytes = (kTopkStageMax + kTopkStageMax / 32 + 1) * 4;
     CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
   }
   TopkArgs a = a0;
-  // CTAs per segment: one for short lists, a cluster of 8 for long ones.  The cluster's barriers and exchanges cost
-  // about 10 us per call, one CTA's passes about 1.25 us per 1024 entries: the cluster pays from about 12 K entries
-  // (measured: 14.7 K entries 23 -> 17 us, 8.2 K entries 18 -> 29 us), provided the clusters of the segments that
-  // select fit one wave of resident CTAs (beyond 16 K entries a single CTA is slower in any case).
-  const int CL = (max_pool > 16384 || (max_pool >= 12288 && n_active * 8 <= 2 * 148)) ? 8 : 1;
+  a.chk = checked_status_ptr();
+  // CTAs per segment: one for short lists, a cluster of 8 for long ones.  The cluster's barriers and exchanges
+  // have a fixed cost, one CTA's passes grow with the list: the cluster pays from about 12 K entries, provided the
+  // clusters of the segments that select fit one wave of resident CTAs (two per SM); beyond 16 K entries a single
+  // CTA is slower in any case.
+  const int CL = (max_pool > 16384 || (max_pool >= 12288 && n_active * 8 <= 2 * sm_count())) ? 8 : 1;
   const int share = ((max_pool + CL - 1) / CL + 3) / 4 * 4;
   a.stage_entries = share <= kTopkStageMax ? share : 0;  // longer shares are read from global memory
   const size_t smem = (size_t)(a.stage_entries + a.stage_entries / 32 + 1) * 4;
@@ -434,7 +431,9 @@ int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, int n_active, cuda
   CATEKV_CUDA_TRY(launch_pdl(topk_kernel<1>, dim3(n_segs), dim3(kTopkThreads), smem, stream, a));
   return CATEKV_OK;
 }
-int launch_gather(const GatherArgs& a, int max_len, int n_segs, cudaStream_t stream) {
+int launch_gather(const GatherArgs& a0, int max_len, int n_segs, cudaStream_t stream) {
+  GatherArgs a = a0;
+  a.chk = checked_status_ptr();
   // at least one block per segment: block 0 also records the length of a straight copy
   const int gx = max_len > 0 ? (max_len + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock : 1;
   gather_kernel<<<dim3(gx, n_segs), 256, 0, stream>>>(a);
@@ -442,30 +441,20 @@ int launch_gather(const GatherArgs& a, int max_len, int n_segs, cudaStream_t str
   return CATEKV_OK;
 }
 
-static int keys_per_cta_for(int n_segs, int n_sc_max) {
-  // the smallest power-of-two multiple of 512 keys that keeps the grid within 4 CTAs per SM
-  int kp = 512;
-  while ((long)n_segs * ((n_sc_max + kp - 1) / kp) > 148 * 4 && kp < (1 << 30)) kp *= 2;
-  return kp;
-}
-
 struct SelWs {
   size_t off_status, off_segs, off_jobs, off_part, off_stats, off_C, off_P, off_idx, bytes;
-  int keys_per_cta, n_chunks;
   int64_t c_stride, idx_stride;
 };
 static SelWs sel_ws_layout(int n_segs, int G, int n_max, int L_obs) {
   SelWs w;
   const int n_sc = n_max > L_obs ? n_max - L_obs : 1;
-  w.keys_per_cta = keys_per_cta_for(n_segs, n_sc);
-  w.n_chunks = (n_sc + w.keys_per_cta - 1) / w.keys_per_cta;
   w.c_stride = (int64_t)align_up((size_t)n_sc, 64);
   w.idx_stride = (int64_t)align_up((size_t)n_max, 64);
   size_t o = 0;
-  w.off_status = o; o = 256;
+  w.off_status = o; o = CATEKV_STATUS_BYTES;
   w.off_segs = o; o = align_up(o + sizeof(SelSeg) * (size_t)n_segs, 256);
   w.off_jobs = o; o = align_up(o + sizeof(ScoreJob) * (size_t)n_segs, 256);
-  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)(n_segs + 148 * 4) * 2 * kScoreMaxRows, 256);
+  w.off_part = o; o = align_up(o + sizeof(float2) * (size_t)score_max_ctas(n_segs) * 2 * kScoreMaxRows, 256);
   w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)n_segs * kScoreMaxRows, 256);
   w.off_C = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.c_stride, 256);
   w.off_P = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.c_stride, 256);
@@ -520,7 +509,7 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   std::vector<SelSeg> segs(n_segs);
   std::vector<ScoreJob> jobs;
   std::vector<int32_t> new_len(n_segs);
-  bool need_readback = false;
+  bool need_readback = false;  // CHUNK mode with a short last chunk: the kept length depends on the scores
   int max_len_ub = 0, n_sc_jobs_max = 0;
   const int S = p->sink, Lc = p->local;
   for (int b = 0; b < p->B; ++b) {
@@ -572,7 +561,7 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   uint8_t* w8 = (uint8_t*)ws;
   SelSeg* d_segs = (SelSeg*)(w8 + W.off_segs);
   ScoreJob* d_jobs = (ScoreJob*)(w8 + W.off_jobs);
-  CATEKV_CUDA_TRY(cudaMemsetAsync(w8 + W.off_status, 0, 256, st));
+  CATEKV_CUDA_TRY(cudaMemsetAsync(w8 + W.off_status, 0, CATEKV_STATUS_BYTES, st));
   CATEKV_CUDA_TRY(cudaMemcpyAsync(d_segs, segs.data(), sizeof(SelSeg) * n_segs, cudaMemcpyHostToDevice, st));
   if (!jobs.empty()) {
     CATEKV_CUDA_TRY(cudaMemcpyAsync(d_jobs, jobs.data(), sizeof(ScoreJob) * jobs.size(), cudaMemcpyHostToDevice, st));
@@ -593,7 +582,7 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
     sa.causal = 0;  // every scored key precedes every window query
     sa.scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
     sa.keys_per_cta = score_keys_per_cta((int)jobs.size(), n_sc_jobs_max);
-    sa.n_chunks = (n_sc_jobs_max + sa.keys_per_cta - 1) / sa.keys_per_cta;  // jobs * chunks <= 592 + jobs: fits the partials
+    sa.n_chunks = (n_sc_jobs_max + sa.keys_per_cta - 1) / sa.keys_per_cta;  // jobs * chunks <= score_max_ctas(jobs): fits the partials
     sa.stats_part = (float2*)(w8 + W.off_part);
     sa.stats = (float2*)(w8 + W.off_stats);
     sa.status = (int32_t*)(w8 + W.off_status);
@@ -639,17 +628,17 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   ga.idx_out_stride = idx_stride;
   ga.Hkv = p->Hkv;
   ga.src_seg_off = nullptr;
+  ga.seg_cap = cache->seg_cap_dev;  // the host check above is exact here; the clamp can only fire on a caller's error
+  ga.status = (int32_t*)(w8 + W.off_status);
   {
     int rc2 = launch_gather(ga, max_len_ub, n_segs, st);
     if (rc2) return rc2;
   }
 
-  if (need_readback) {
-    // a short last chunk makes the kept length depend on the scores: fetch the device's lengths
-    CATEKV_CUDA_TRY(cudaMemcpyAsync(cache->seg_len, cache->seg_len_dev, sizeof(int32_t) * n_segs, cudaMemcpyDeviceToHost, st));
-    CATEKV_CUDA_TRY(cudaStreamSynchronize(st));
-  } else {
-    for (int i = 0; i < n_segs; ++i) cache->seg_len[i] = new_len[i];
-  }
+  // A short last chunk makes the kept length depend on the scores: the mirror then holds the upper bound (the
+  // device's length is at most cs - 1 rows shorter) and the cache is marked; catekv_cache_sync_lengths fetches
+  // the exact lengths when the caller wants them.
+  for (int i = 0; i < n_segs; ++i) cache->seg_len[i] = new_len[i];
+  cache->reserved = need_readback ? 1 : 0;
   return CATEKV_OK;
 }

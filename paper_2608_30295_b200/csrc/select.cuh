@@ -30,6 +30,7 @@ struct TopkArgs {
   int32_t sink, L_obs, pool_mode, pool_param;  // the always-kept tail of a segment is [cand_end, n)
   int32_t mark_keep_all;  // 1: a keep_all segment gets seg_len_dev = -1 ("the whole list") instead of being skipped
   int32_t stage_entries;  // set by launch_topk: pooled entries per CTA that the dynamic shared memory holds
+  int32_t* chk;           // set by launch_topk: the checked build's status block, else null
 };
 
 struct GatherArgs {
@@ -47,6 +48,9 @@ struct GatherArgs {
   int32_t* idx_out;
   int64_t idx_out_stride;
   int32_t Hkv;
+  const int32_t* seg_cap;  // capacity of every destination segment (device), or null: the copy is cut there
+  int32_t* status;         // status block of the caller's workspace: CATEKV_STATUS_CAPACITY when a copy was cut
+  int32_t* chk;            // set by launch_gather: the checked build's status block, else null
 };
 
 

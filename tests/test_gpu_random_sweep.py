@@ -84,6 +84,8 @@ def test_random_select(ck, seed):
     idx = torch.full((B * Hkv, n), -1, dtype=torch.int32, device="cuda")
     ck.catekv_select_compact(p["q_win"].cuda(), p["k"].cuda(), p["v"].cuda(), seq_len, mask, cache, budget, eta, sink,
                              local, mode, param, idx_out=idx)
+    if cache.struct.reserved:
+        ck.catekv_cache_sync_lengths(cache)
     torch.cuda.synchronize()
     idx = idx.cpu().numpy()
     qw, k, v = synth.bits(p["q_win"]), synth.bits(p["k"]), synth.bits(p["v"])

@@ -167,8 +167,7 @@ def test_retrieval_step_replayed_as_cuda_graph(ck, indexed):
     vn = torch.empty_like(kn)
     out = torch.empty((B, Hkv * G, 128), dtype=torch.float32, device="cuda")
     idx = torch.full((B * Hkv, max(lens) + steps + 2), -1, dtype=torch.int32, device="cuda")
-    ws = torch.empty(ck._lib.catekv_retrieve_workspace_bytes(B, Hkv, int(cache.seg_cap.max())), dtype=torch.uint8,
-                     device="cuda")
+    ws = ck.retrieve_workspace(cache)
     sel = torch.full((B * Hkv,), -99, dtype=torch.int32, device="cuda")
     if indexed:
         view = ck.CacheView(cache, ck.catekv_retrieve_lengths(cache, cs, mask, budget, sink, local))

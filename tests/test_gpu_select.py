@@ -32,6 +32,11 @@ def _select(ck, w, p, mask, budget, eta, mode, param, max_new=0, seq_len=None):
     idx = torch.full((w.B * w.Hkv, w.n), -1, dtype=torch.int32, device="cuda")
     ck.catekv_select_compact(p["q_win"].cuda(), p["k"].cuda(), p["v"].cuda(), seq_len, mask, cache, budget, eta,
                              w.sink, w.local, mode, param, idx_out=idx)
+    if cache.struct.reserved:  # chunk mode with a short last chunk: the host lengths are upper bounds until synced
+        bound = cache.seg_len.copy()
+        ck.catekv_cache_sync_lengths(cache)
+        assert np.all(cache.seg_len <= bound) and np.all(bound - cache.seg_len < max(param, 1))
+        assert cache.struct.reserved == 0
     torch.cuda.synchronize()
     return cache, idx.cpu().numpy()
 
