@@ -254,52 +254,61 @@ def time_decode(ck, w, model, dev, steps, warmup, barrier=None, graph=True):
 
 APPEND_US = None  # mean duration of the separate append launch, set by time_kernels
 
+# DRAM bytes per algorithmic byte of decode_partial_kernel: dram__bytes_read.sum over 512 B x kept rows, from the
+# ncu capture of the two-layer configs[2] case (profiles/decode_partial_kernel_cfg2_2layers.md); traffic grows in
+# proportion to the kept rows (every row crosses DRAM once), so the ratio is applied to each run's own bytes.
+TRAFFIC_READ_RATIO = 1.0002
+TRAFFIC_WRITE_BYTES = 4.6e6  # per launch in that capture (partials, outputs); does not grow with the rows
 
-def time_kernels(ck, w, model, dev, steps):
-    """Per-kernel durations over the same steps: events around the partials kernel of every launch."""
+
+def _graph_of(fn):
+    """Capture fn() (library calls on the current stream) into a CUDA graph."""
     import torch
-    L = len(model)
-    sets = make_step_inputs(w, L, dev)
-    out = torch.empty((L, w.B, w.Hq, w.d), dtype=torch.bfloat16, device=dev)
-    ev = []
-    for i in range(steps):
-        q, kn, vn = sets[i % len(sets)]
-        for l, m in enumerate(model):
-            ck.catekv_append(m["cache"], kn[l], vn[l])
-            a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
-            a.record()
-            ck.catekv_decode_partials(m["cache"], q[l], m["plan"], out[l])
-            b.record()
-            ck.catekv_decode_combine(m["cache"], q[l], m["plan"], out[l])
-            c.record()
-            ev.append((a, b, c))
-    torch.cuda.synchronize()
-    part = [a.elapsed_time(b) * 1e3 for a, b, _ in ev]
-    comb = [b.elapsed_time(c) * 1e3 for _, b, c in ev]
-    # the separate append launch: a CUDA graph of one catekv_append per layer (between host launches the events
-    # above mostly see launch gaps), replayed a few times
-    global APPEND_US
-    q, kn, vn = sets[0]
     g = torch.cuda.CUDAGraph()
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
         with torch.cuda.graph(g, stream=side):
-            for l, m in enumerate(model):
-                ck.catekv_append(m["cache"], kn[l], vn[l])
+            fn()
     torch.cuda.current_stream().wait_stream(side)
-    g.replay()  # the capture advanced the host mirrors by one row: make the device follow
+    return g
+
+
+def _time_graph(g, reps, before=None):
+    import torch
+    g.replay()
+    torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    reps = 3
-    for m in model:
-        ck.catekv_cache_advance(m["cache"], reps)
     e0.record()
     for _ in range(reps):
+        if before:
+            before()
         g.replay()
     e1.record()
     torch.cuda.synchronize()
-    APPEND_US = e0.elapsed_time(e1) * 1e3 / (reps * L)
-    return float(np.mean(part)), float(np.median(part)), float(np.mean(comb))
+    return e0.elapsed_time(e1) * 1e3 / reps  # us per replay
+
+
+def time_kernels(ck, w, model, dev, steps):
+    """Average duration of the attention-partials launch in the launch regime of the timed step: a CUDA graph of
+    catekv_decode_partials over all layers (the same programmatic-launch chain, without the combine launches),
+    replayed `steps` times, CUDA events around the replays, divided by the number of launches.  Also: the same
+    for the combine launches and for the separate append launch.  Returns (partials us, combine us)."""
+    import torch
+    L = len(model)
+    q, kn, vn = make_step_inputs(w, L, dev, n_sets=1)[0]
+    out = torch.empty((L, w.B, w.Hq, w.d), dtype=torch.bfloat16, device=dev)
+    g_part = _graph_of(lambda: [ck.catekv_decode_partials(m["cache"], q[l], m["plan"], out[l]) for l, m in enumerate(model)])
+    part = _time_graph(g_part, steps) / L
+    g_comb = _graph_of(lambda: [ck.catekv_decode_combine(m["cache"], q[l], m["plan"], out[l]) for l, m in enumerate(model)])
+    comb = _time_graph(g_comb, steps) / L
+    global APPEND_US
+    g_app = _graph_of(lambda: [ck.catekv_append(m["cache"], kn[l], vn[l]) for l, m in enumerate(model)])
+    reps = 3
+    for m in model:  # the capture advanced the host mirrors by one row; the replays below add reps + 1 rows
+        ck.catekv_cache_advance(m["cache"], reps)
+    APPEND_US = _time_graph(g_app, reps) / L
+    return part, comb
 
 
 def time_e2e(ck, w, model, dev, steps, warmup, barrier=None, graph=True):
@@ -620,6 +629,61 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def measure_workload(ck, w, dev, n_layers, steps, warmup, barrier, graph, peaks, peak_src, world, sampler):
+    """Build the workload's caches, time the decode step (device-resident and end to end) and the attention kernel
+    in the same launch regime; returns the pieces of a bench line.  Frees the model before returning."""
+    import torch
+    total_steps = 3 * (warmup + steps) + 24
+    model, sel_ms = build_model(ck, w, dev, max_new=total_steps, layers=n_layers)
+    plan_us = float(np.median(PLAN_HOST_US[-n_layers:]))
+    if sampler:
+        sampler.start()
+    ms = max_over_ranks(time_decode(ck, w, model, dev, steps, warmup, barrier, graph), dev)
+    clocks = sampler.stop() if sampler else None
+    bytes_per_layer = float(np.mean(kept_bytes(model)))
+    part_us, comb_us = time_kernels(ck, w, model, dev, max(3, min(steps, 10)))
+    ms_e2e, h2d, d2h = time_e2e(ck, w, model, dev, steps, warmup, barrier, graph)
+    ms_e2e = max_over_ranks(ms_e2e, dev)
+    has_combine = any(ck.plan_header(m["plan"])["n_slots"] for m in model)
+    del model
+    torch.cuda.empty_cache()
+    scale_layers = w.layers / n_layers  # only != 1 when --layers is used for profiling
+    achieved = bytes_per_layer / (part_us * 1e-6) / 1e9
+    return {
+        "value": world * w.B / (ms * scale_layers * 1e-3),
+        "ms_per_step": ms,
+        "us_per_layer_step": ms * 1e3 / n_layers,
+        "step_hbm_gbs": bytes_per_layer / (ms * 1e-3 / n_layers) / 1e9,
+        "config": {"workload": w.name, "layers": n_layers, "batch": w.B, "context": w.n, "q_heads": w.Hq,
+                   "kv_heads": w.Hkv, "head_dim": w.d, "budget_consistent": w.budget, "eta_adaptive": w.eta,
+                   "window": w.L_obs, "replicas": world,
+                   "l2": "no flush: per-layer working set %.0f MB x %d layers, far above the 126 MB L2"
+                         % (bytes_per_layer / 1e6, n_layers),
+                   "step": "one decode token of the whole model: per layer " +
+                           ("catekv_append_decode_attn (append fused into the attention launch)" if FUSED
+                            else "catekv_append + catekv_decode_attn"),
+                   "launch": "CUDA graph replay of the step" if graph else "host launches"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src,
+                     "traffic": bytes_per_layer * TRAFFIC_READ_RATIO + TRAFFIC_WRITE_BYTES,
+                     "traffic_source": "ncu dram__bytes_read.sum / algorithmic bytes = 1.0002 and about 4.6 MB of "
+                                       "dram__bytes_write.sum per launch on the two-layer configs[2] case, scaled "
+                                       "by this run's kept rows (every kept row crosses DRAM once)",
+                     "kernel": "decode_partial_kernel", "bytes_per_launch": bytes_per_layer,
+                     "us_per_launch": part_us,
+                     "us_per_launch_how": "CUDA graph of catekv_decode_partials over all layers (the step's launch "
+                                          "chain without the combine launches), CUDA events around its replays, "
+                                          "divided by the launches",
+                     "frac_of_8TBs": achieved / 8000.0, "combine_us": comb_us, "append_us": APPEND_US},
+        "e2e": {"value": world * w.B / (ms_e2e * scale_layers * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
+        "gpu_launches": steps * n_layers * ((1 if FUSED else 2) + (1 if has_combine else 0)),
+        "clocks": clocks,
+        "select_compact": {"ms_per_layer": float(np.mean(sel_ms[1:] or sel_ms)), "layers": n_layers},
+        "plan_host_us": plan_us,
+    }
+
+
 # ------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -670,7 +734,6 @@ def main():
     peaks, peak_src = measured_peaks()
     w = synth.WORKLOADS[args.workload]
     n_layers = args.layers or w.layers
-    total_steps = 3 * (args.warmup + args.steps) + 24
     graph = not args.no_graph
     global FUSED
     FUSED = not args.no_fused
@@ -686,84 +749,46 @@ def main():
             print(json.dumps({"workload": w.name, "layers": n_layers, "retrieval_us_per_layer_step": ru,
                               "attended_bytes_per_layer_step": ra, "metadata_bytes_per_layer_step": rm}))
         return
-    model, sel_ms = build_model(ck, w, dev, max_new=total_steps, layers=n_layers)
     if args.select_only:
+        model, sel_ms = build_model(ck, w, dev, max_new=8, layers=n_layers)
         if rank == 0:
             print(json.dumps({"workload": w.name, "layers": n_layers, "select_compact_ms_per_layer": sel_ms}))
         return
 
     vis = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
     sampler = ClockSampler(vis[local_rank] if local_rank < len(vis) else local_rank)
-    sampler.start()
-    ms = max_over_ranks(time_decode(ck, w, model, dev, args.steps, args.warmup, barrier, graph), dev)
-    clocks = sampler.stop()
-    bytes_per_layer = float(np.mean(kept_bytes(model)))
-    part_us, part_med_us, comb_us = time_kernels(ck, w, model, dev, max(2, min(args.steps, 5)))
-    ms_e2e, h2d, d2h = time_e2e(ck, w, model, dev, args.steps, args.warmup, barrier, graph)
-    ms_e2e = max_over_ranks(ms_e2e, dev)
-
-    scale_layers = w.layers / n_layers  # only != 1 when --layers is used for profiling
-    value = world * w.B / (ms * scale_layers * 1e-3)
-    e2e_value = world * w.B / (ms_e2e * scale_layers * 1e-3)
-    achieved = bytes_per_layer / (part_us * 1e-6) / 1e9
+    r = measure_workload(ck, w, dev, n_layers, args.steps, args.warmup, barrier, graph, peaks, peak_src, world, sampler)
+    bytes_per_layer = r["roofline"]["bytes_per_launch"]
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-        "data": "synthetic",
-        "config": {"workload": w.name, "layers": n_layers, "batch": w.B, "context": w.n, "q_heads": w.Hq,
-                   "kv_heads": w.Hkv, "head_dim": w.d, "budget_consistent": w.budget, "eta_adaptive": w.eta,
-                   "window": w.L_obs, "replicas": world,
-                   "l2": "no flush: per-layer working set %.0f MB x %d layers, far above the 126 MB L2"
-                         % (bytes_per_layer / 1e6, n_layers),
-                   "step": "one decode token of the whole model: per layer " +
-                           ("catekv_append_decode_attn (append fused into the attention launch)" if FUSED
-                            else "catekv_append + catekv_decode_attn"),
-                   "launch": "CUDA graph replay of the step" if graph else "host launches"},
-        "us_per_layer_step": ms * 1e3 / n_layers,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src,
-                     # DRAM read+write bytes per launch: one-pass ncu capture of this workload's own launches
-                     # (profiles/decode_partial_kernel_cfg3_traffic.md): reads = 1.00015 x algorithmic bytes,
-                     # about 1.25 MB of writes; the configs[2] small case gave the same ratio
-                     "traffic": bytes_per_layer * 1.00015 + 1.25e6,
-                     "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the configs[3] launches "
-                                       "(read = 1.00015 x algorithmic bytes), applied to this run's kept rows",
-                     "kernel": "decode_partial_kernel", "bytes_per_launch": bytes_per_layer,
-                     "us_per_launch": part_us, "us_per_launch_median": part_med_us,
-                     "frac_of_8TBs": achieved / 8000.0, "combine_us": comb_us,
-                     "append_us": APPEND_US},
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": ms_e2e},
-        "gpu_launches": args.steps * n_layers * ((1 if FUSED else 2) +
-                                                 (1 if any(ck.plan_header(m["plan"])["n_slots"] for m in model) else 0)),
-        "clocks": clocks,
-        "select_compact": {"ms_per_layer": float(np.mean(sel_ms[1:] or sel_ms)), "layers": n_layers},
-        "plan_host_us": float(np.median(PLAN_HOST_US[:n_layers])),
+        "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": r["config"],
+        "us_per_layer_step": r["us_per_layer_step"],
+        "roofline": r["roofline"],
+        "e2e": r["e2e"],
+        "gpu_launches": r["gpu_launches"],
+        "clocks": r["clocks"],
+        "select_compact": r["select_compact"],
+        "plan_host_us": r["plan_host_us"],
     }
-    del model
-    torch.cuda.empty_cache()
-
     if rank == 0 and not args.no_extras:
-        # the other configurations, decode only, a few layers each (parity-test cases, reported for context)
+        # the other configurations over all their layers, each with its own roofline and end-to-end blocks
+        # (configs[2] and configs[4] carry the 70 %-of-HBM target; configs[1] is reported, not gated)
         table = {}
         for name in ("cfg1", "cfg2", "cfg4"):
             if name == w.name:
                 continue
             wo = synth.WORKLOADS[name]
-            nl = min(wo.layers, 8)
-            mo, so = build_model(ck, wo, dev, max_new=96, layers=nl)
-            t = time_decode(ck, wo, mo, dev, 10, 3)
-            pu, pm, cu = time_kernels(ck, wo, mo, dev, 3)
-            by = float(np.mean(kept_bytes(mo)))
-            table[name] = {"layers_timed": nl, "us_per_layer_step": t * 1e3 / nl, "partials_us": pu,
-                           "bytes_per_layer_step": by, "hbm_gbs": by / (pu * 1e-6) / 1e9,
-                           "frac_of_measured": by / (pu * 1e-6) / 1e9 / peaks["hbm_gbs"],
+            ro = measure_workload(ck, wo, dev, wo.layers, 10, 3, None, graph, peaks, peak_src, 1, None)
+            table[name] = {"layers_timed": wo.layers, "tokens_per_s": ro["value"], "ms_per_step": ro["ms_per_step"],
+                           "us_per_layer_step": ro["us_per_layer_step"], "roofline": ro["roofline"], "e2e": ro["e2e"],
+                           "bytes_per_layer_step": ro["roofline"]["bytes_per_launch"],
                            # the whole replayed layer-step (attention + combine, append fused) against the same bytes
-                           "step_hbm_gbs": by / (t * 1e-3 / nl) / 1e9,
-                           "step_frac_of_measured": by / (t * 1e-3 / nl) / 1e9 / peaks["hbm_gbs"],
-                           "select_ms_per_layer": float(np.mean(so[1:] or so))}
-            del mo
-            torch.cuda.empty_cache()
+                           "step_hbm_gbs": ro["step_hbm_gbs"],
+                           "step_frac_of_measured": ro["step_hbm_gbs"] / peaks["hbm_gbs"],
+                           "step_frac_of_8TBs": ro["step_hbm_gbs"] / 8000.0,
+                           "select_ms_per_layer": ro["select_compact"]["ms_per_layer"]}
         line["other_configs"] = table
         line["head_cv"] = {"ms": time_head_cv(ck, dev), "shape": "8 prompts x 16384 tokens, 28q/4kv, window 64"}
         ru, ra, rm = time_retrieval(ck, w, dev)
