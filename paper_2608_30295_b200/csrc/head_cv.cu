@@ -267,8 +267,7 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   sa.causal = causal ? 1 : 0;
   sa.g_major = L_obs == 64 ? 1 : 0;  // the paper's window: head-major rows make the group mean a register sum
   sa.scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
-  sa.keys_per_cta = score_keys_per_cta(n_segs, m_max);
-  sa.n_chunks = (m_max + sa.keys_per_cta - 1) / sa.keys_per_cta;
+  sa.max_keys = m_max;
   sa.stats_part = (float2*)(w8 + W.off_part);
   sa.stats = (float2*)(w8 + W.off_stats);
   sa.status = (int32_t*)(w8 + W.off_status);

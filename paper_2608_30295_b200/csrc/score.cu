@@ -15,12 +15,13 @@
 //       one key, so C_j = sum_r exp2(x_rj - m_r) / l_r and A_ij = mean_g (...) are thread-local
 //       sums over TMEM columns and the global writes are coalesced over keys.
 //
-// Warp roles: warp 8 (one elected lane) waits for a K tile, issues the eight k-steps of
-// tcgen05.mma per unit and commits them to an mbarrier; warps 0-7 are the epilogue (two per
-// TMEM lane quarter, each half of a unit's columns): they wait for the unit, read the
-// accumulators with tcgen05.ld, do the exp2 arithmetic and hand the TMEM slot back.  The thread
-// that observes the last unit of a tile complete re-arms that tile's stage with the next TMA
-// load.  There is no CTA-wide barrier in the main loop.  Every mbarrier wait is bounded: on
+// Warp roles: warp 9 (one elected lane) is the TMA producer: it refills a K stage as soon as the
+// MMAs that read it have completed (a tcgen05.commit on the stage's "empty" barrier), however far
+// the epilogue lags.  Warp 8 (one elected lane) waits for a K tile, issues the eight k-steps of
+// tcgen05.mma per unit and commits them to the unit's "done" barrier; warps 0-7 are the epilogue
+// (two per TMEM lane quarter, each half of a unit's columns): they wait for the unit, read the
+// accumulators with tcgen05.ld into registers, hand the TMEM slot back at once and then do the
+// exp2 arithmetic.  There is no CTA-wide barrier in the main loop.  Every mbarrier wait is bounded: on
 // expiry the thread raises a CTA-wide abort flag (which ends all other waits early) and a status
 // word in the workspace; the CTA then frees its TMEM and returns.
 #include <cuda.h>
@@ -33,7 +34,7 @@
 namespace catekv {
 
 constexpr int kEpiThreads = 256;                   // 8 epilogue warps: two per TMEM lane quarter, each takes half the columns
-constexpr int kScThreads = kEpiThreads + 32;       // + the TMA / MMA warp
+constexpr int kScThreads = kEpiThreads + 64;       // + the MMA warp (8) and the TMA warp (9)
 constexpr int kKeyTile = 128;                       // keys per tile
 constexpr int kKBlockBytes = kKeyTile * 128;        // one 64-element k-block of a K tile
 constexpr int kKStageBytes = 2 * kKBlockBytes;      // K tile: 128 keys x 128 dims bf16
@@ -127,20 +128,38 @@ __device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* ma
       "l"(map), "r"(d0), "r"(j0), "r"(h), "r"(b), "r"(bar)
       : "memory");
 }
-// 32 consecutive TMEM columns of this thread's lane
+// 32 consecutive TMEM columns of this thread's lane, straight into float registers.  The load is asynchronous:
+// tmem_wait_ld32 must run before the values are used (it takes the registers as operands, so that no use can
+// be scheduled ahead of it).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]), "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15]), "=f"(v[16]), "=f"(v[17]), "=f"(v[18]), "=f"(v[19]), "=f"(v[20]), "=f"(v[21]), "=f"(v[22]), "=f"(v[23]), "=f"(v[24]), "=f"(v[25]), "=f"(v[26]), "=f"(v[27]), "=f"(v[28]), "=f"(v[29]), "=f"(v[30]), "=f"(v[31])
+               : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_wait_ld32(float (&v)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n"
+               : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7]), "+f"(v[8]), "+f"(v[9]), "+f"(v[10]), "+f"(v[11]), "+f"(v[12]), "+f"(v[13]), "+f"(v[14]), "+f"(v[15]), "+f"(v[16]), "+f"(v[17]), "+f"(v[18]), "+f"(v[19]), "+f"(v[20]), "+f"(v[21]), "+f"(v[22]), "+f"(v[23]), "+f"(v[24]), "+f"(v[25]), "+f"(v[26]), "+f"(v[27]), "+f"(v[28]), "+f"(v[29]), "+f"(v[30]), "+f"(v[31])
+               :
+               : "memory");
+}
+// 64 consecutive TMEM columns of this thread's lane, straight into float registers.  The load is asynchronous:
+// tmem_wait_ld64 must run before the values are used (it takes the registers as operands, so that no use can
+// be scheduled ahead of it).
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%64];\n"
+               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]), "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15]), "=f"(v[16]), "=f"(v[17]), "=f"(v[18]), "=f"(v[19]), "=f"(v[20]), "=f"(v[21]), "=f"(v[22]), "=f"(v[23]), "=f"(v[24]), "=f"(v[25]), "=f"(v[26]), "=f"(v[27]), "=f"(v[28]), "=f"(v[29]), "=f"(v[30]), "=f"(v[31]), "=f"(v[32]), "=f"(v[33]), "=f"(v[34]), "=f"(v[35]), "=f"(v[36]), "=f"(v[37]), "=f"(v[38]), "=f"(v[39]), "=f"(v[40]), "=f"(v[41]), "=f"(v[42]), "=f"(v[43]), "=f"(v[44]), "=f"(v[45]), "=f"(v[46]), "=f"(v[47]), "=f"(v[48]), "=f"(v[49]), "=f"(v[50]), "=f"(v[51]), "=f"(v[52]), "=f"(v[53]), "=f"(v[54]), "=f"(v[55]), "=f"(v[56]), "=f"(v[57]), "=f"(v[58]), "=f"(v[59]), "=f"(v[60]), "=f"(v[61]), "=f"(v[62]), "=f"(v[63])
+               : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_wait_ld64(float (&v)[64]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n"
+               : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7]), "+f"(v[8]), "+f"(v[9]), "+f"(v[10]), "+f"(v[11]), "+f"(v[12]), "+f"(v[13]), "+f"(v[14]), "+f"(v[15]), "+f"(v[16]), "+f"(v[17]), "+f"(v[18]), "+f"(v[19]), "+f"(v[20]), "+f"(v[21]), "+f"(v[22]), "+f"(v[23]), "+f"(v[24]), "+f"(v[25]), "+f"(v[26]), "+f"(v[27]), "+f"(v[28]), "+f"(v[29]), "+f"(v[30]), "+f"(v[31]), "+f"(v[32]), "+f"(v[33]), "+f"(v[34]), "+f"(v[35]), "+f"(v[36]), "+f"(v[37]), "+f"(v[38]), "+f"(v[39]), "+f"(v[40]), "+f"(v[41]), "+f"(v[42]), "+f"(v[43]), "+f"(v[44]), "+f"(v[45]), "+f"(v[46]), "+f"(v[47]), "+f"(v[48]), "+f"(v[49]), "+f"(v[50]), "+f"(v[51]), "+f"(v[52]), "+f"(v[53]), "+f"(v[54]), "+f"(v[55]), "+f"(v[56]), "+f"(v[57]), "+f"(v[58]), "+f"(v[59]), "+f"(v[60]), "+f"(v[61]), "+f"(v[62]), "+f"(v[63])
+               :
+               : "memory");
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
 // offset of the 16-byte chunk c (0..15) of row r inside a two-k-block SW128 region of `rows` rows
@@ -166,10 +185,11 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
   const uint32_t s_q = s_base;
   const uint32_t s_k = s_q + 2 * q_block;
   float* s_f = reinterpret_cast<float*>(smem + 2 * q_block + 2 * kKStageBytes);  // pass 1: (m, l)[2][512]; pass 2: m'[R]
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_f + 4 * kScoreMaxRows);         // full[2], done[4], free[4]
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 10);
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_f + 4 * kScoreMaxRows);         // full[2], done[4], free[4], empty[2]
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 12);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   const uint32_t bar_full = smem_u32(s_bar), bar_done = smem_u32(s_bar + 2), bar_free = smem_u32(s_bar + 6);
+  const uint32_t bar_empty = smem_u32(s_bar + 10);  // a K stage has been read by all the MMAs of its tile
 
   constexpr bool kStats = MODE == kScoreStats;
   const int UPT = kStats ? sh.MT : sh.NH;          // MMA units per key tile
@@ -212,6 +232,7 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
     for (int i = 0; i < 2; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar_full + 8 * i));
     for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar_done + 8 * i));
     for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 8;\n" ::"r"(bar_free + 8 * i));  // one arrival per epilogue warp
+    for (int i = 0; i < 2; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar_empty + 8 * i));
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (warp == 8) {
@@ -237,7 +258,6 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
   if (warp == 8) {
     // ================= TMA + MMA issue: one elected lane =================
     if (lane == 0 && !a.idle_producer) {
-      for (int tl = 0; tl < 2 && tl < n_tiles; ++tl) load_tile(tl);
       const uint32_t idesc = kStats ? umma_idesc_bf16(128, 128) : umma_idesc_bf16(128, sh.NW);
       for (int v = 0; v < U; ++v) {
         const int tile = v / UPT, sub = v - tile * UPT;
@@ -257,6 +277,16 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
             umma_bf16(d, umma_desc_sw128(ak), umma_desc_sw128(aq + sub * sh.NW * 128), idesc, kk ? 1u : 0u);
         }
         umma_commit(bar_done + 8 * (v % NSLOT));
+        if (sub == UPT - 1) umma_commit(bar_empty + 8 * (tile & 1));  // the tile's stage may be refilled once these MMAs are done
+      }
+    }
+    __syncwarp();
+  } else if (warp == 9) {
+    // ================= TMA producer: one elected lane keeps both K stages in flight =================
+    if (lane == 0 && !a.idle_producer) {
+      for (int tile = 0; tile < n_tiles; ++tile) {
+        if (tile >= 2 && !mbar_wait(bar_empty + 8 * (tile & 1), (uint32_t)(((tile >> 1) - 1) & 1), s_abort, a.spin_limit)) break;
+        load_tile(tile);
       }
     }
     __syncwarp();
@@ -270,34 +300,54 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
     float col_acc = 0.f;  // pass 2, column sums: this key's sum over this thread's rows of the tile
     float macc[32];       // pass 2, head-major matrix: this key's entries of this thread's 32 window rows
 
+    // hand the TMEM slot of unit u back to the MMA warp: once per epilogue warp, after its last load of the unit
+    auto release_slot = [&](int u) {
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_free + 8 * (u % NSLOT));
+    };
+
     for (int u = 0; u < U; ++u) {
       const int tile = u / UPT, sub = u - tile * UPT;
       if (!mbar_wait(bar_done + 8 * (u % NSLOT), (uint32_t)((u / NSLOT) & 1), s_abort, a.spin_limit)) break;
       tc_fence_after();
-      // the MMAs of this tile have read its stage: re-arm the stage with the tile after next
-      if (tid == 0 && sub == UPT - 1 && tile + 2 < n_tiles) load_tile(tile + 2);
       const uint32_t tbase = tmem + lane_base + (uint32_t)((u % NSLOT) * slot_w);
       const int j0 = j_lo + tile * kKeyTile;
 
       if (kStats) {
-        // this thread's query row, keys [64 * half, 64 * half + 64) of the tile
+        // this thread's query row, keys [64 * half, 64 * half + 64) of the tile: one 64-column load, after which
+        // the TMEM slot goes straight back to the MMA warp (the arithmetic below runs on registers)
         const int r = sub * 128 + lane_row;
         const int i = a.g_major ? r % a.L_obs : r / a.G;
         const int lim = a.causal ? job.n - a.L_obs + i : 0x7fffffff;  // last key this window row sees
         const int jmax = min(j_hi - 1, lim);                          // keys j <= jmax are live
-        float m = s_f[2 * (half * kScoreMaxRows + r)], l = s_f[2 * (half * kScoreMaxRows + r) + 1];
-#pragma unroll 1
-        for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 32) {
-          if (j0 + c0 >= j_hi) break;  // uniform: the rest of the tile is padding
-          float x[32];
-          tmem_ld32(tbase + c0, x);
-          if (j0 + c0 + 31 > jmax) {  // tail of the key range or the causal edge: mask entry by entry
+        const int c0 = half * 64;
+        const bool any = j0 + c0 < j_hi;  // uniform: otherwise this half of the tile is padding
+        float x[64];
+        if (any) {
+          tmem_ld64(tbase + c0, x);
+          tmem_wait_ld64(x);
+        }
+        release_slot(u);
+        if (any) {
+          float m = s_f[2 * (half * kScoreMaxRows + r)], l = s_f[2 * (half * kScoreMaxRows + r) + 1];
+          if (j0 + c0 + 63 > jmax) {  // tail of the key range or the causal edge: mask entry by entry
 #pragma unroll
-            for (int c = 0; c < 32; ++c) x[c] = (j0 + c0 + c <= jmax) ? x[c] : -INFINITY;
+            for (int c = 0; c < 64; ++c) x[c] = (j0 + c0 + c <= jmax) ? x[c] : -INFINITY;
           }
-          float mx = x[0];
+          // four independent chains of three-input maxima
+          float mx0 = fmax3(x[0], x[1], x[2]), mx1 = fmax3(x[3], x[4], x[5]);
+          float mx2 = fmax3(x[6], x[7], x[8]), mx3 = fmax3(x[9], x[10], x[11]);
 #pragma unroll
-          for (int c = 1; c < 32; ++c) mx = fmaxf(mx, x[c]);
+          for (int c = 12; c < 60; c += 8) {
+            mx0 = fmax3(mx0, x[c], x[c + 1]);
+            mx1 = fmax3(mx1, x[c + 2], x[c + 3]);
+            mx2 = fmax3(mx2, x[c + 4], x[c + 5]);
+            mx3 = fmax3(mx3, x[c + 6], x[c + 7]);
+          }
+          mx0 = fmax3(mx0, x[60], x[61]);
+          mx1 = fmax3(mx1, x[62], x[63]);
+          float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
           mx *= a.scale_log2;  // the scale is positive: the max commutes with it
           if (mx > m) {
             l *= fast_exp2(m - mx);
@@ -306,7 +356,7 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
           if (m > -INFINITY) {
             float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-            for (int c = 0; c < 32; c += 4) {
+            for (int c = 0; c < 64; c += 4) {
               s0 += fast_exp2(fmaf(x[c], a.scale_log2, -m));
               s1 += fast_exp2(fmaf(x[c + 1], a.scale_log2, -m));
               s2 += fast_exp2(fmaf(x[c + 2], a.scale_log2, -m));
@@ -314,9 +364,9 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
             }
             l += (s0 + s1) + (s2 + s3);
           }
+          s_f[2 * (half * kScoreMaxRows + r)] = m;
+          s_f[2 * (half * kScoreMaxRows + r) + 1] = l;
         }
-        s_f[2 * (half * kScoreMaxRows + r)] = m;
-        s_f[2 * (half * kScoreMaxRows + r) + 1] = l;
       } else {
         // this thread's key; the unit's rows [r_begin, r_end) are cut between the two halves: at a multiple of 32
         // columns for the column sums, at a multiple of G for the matrix (whole window rows per thread)
@@ -328,25 +378,53 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
         if (MODE == kScoreColsum) {
           if (sub == 0) col_acc = 0.f;
           float c0s = 0.f, c1s = 0.f, c2s = 0.f, c3s = 0.f;
+          // 64 rows per load where that many are left, else 32; the slot is handed back after the last load
 #pragma unroll 1
-          for (int rr = r0; rr < r1; rr += 32) {
-            float x[32];
-            tmem_ld32(tbase + (rr - r_begin), x);
-            if (rr + 32 <= r1) {
+          for (int rr = r0; rr < r1;) {
+            const int left = r1 - rr;
+            if (left > 32) {
+              float x[64];
+              tmem_ld64(tbase + (rr - r_begin), x);
+              tmem_wait_ld64(x);
+              if (rr + 64 >= r1) release_slot(u);
+              if (left >= 64) {
 #pragma unroll
-              for (int c = 0; c < 32; c += 4) {
-                const float4 mm = *reinterpret_cast<const float4*>(s_f + rr + c);  // rr is a multiple of 16
-                c0s += fast_exp2(fmaf(x[c], a.scale_log2, -mm.x));
-                c1s += fast_exp2(fmaf(x[c + 1], a.scale_log2, -mm.y));
-                c2s += fast_exp2(fmaf(x[c + 2], a.scale_log2, -mm.z));
-                c3s += fast_exp2(fmaf(x[c + 3], a.scale_log2, -mm.w));
+                for (int c = 0; c < 64; c += 4) {
+                  const float4 mm = *reinterpret_cast<const float4*>(s_f + rr + c);  // rr is a multiple of 16
+                  c0s += fast_exp2(fmaf(x[c], a.scale_log2, -mm.x));
+                  c1s += fast_exp2(fmaf(x[c + 1], a.scale_log2, -mm.y));
+                  c2s += fast_exp2(fmaf(x[c + 2], a.scale_log2, -mm.z));
+                  c3s += fast_exp2(fmaf(x[c + 3], a.scale_log2, -mm.w));
+                }
+              } else {
+#pragma unroll
+                for (int c = 0; c < 64; ++c)
+                  if (c < left) c0s += fast_exp2(fmaf(x[c], a.scale_log2, -s_f[rr + c]));
               }
+              rr += 64;
             } else {
+              float x[32];
+              tmem_ld32(tbase + (rr - r_begin), x);
+              tmem_wait_ld32(x);
+              release_slot(u);  // at most 32 rows were left: this was the last load
+              if (left == 32) {
 #pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (rr + c < r1) c0s += fast_exp2(fmaf(x[c], a.scale_log2, -s_f[rr + c]));
+                for (int c = 0; c < 32; c += 4) {
+                  const float4 mm = *reinterpret_cast<const float4*>(s_f + rr + c);
+                  c0s += fast_exp2(fmaf(x[c], a.scale_log2, -mm.x));
+                  c1s += fast_exp2(fmaf(x[c + 1], a.scale_log2, -mm.y));
+                  c2s += fast_exp2(fmaf(x[c + 2], a.scale_log2, -mm.z));
+                  c3s += fast_exp2(fmaf(x[c + 3], a.scale_log2, -mm.w));
+                }
+              } else {
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                  if (c < left) c0s += fast_exp2(fmaf(x[c], a.scale_log2, -s_f[rr + c]));
+              }
+              rr += 32;
             }
           }
+          if (r0 >= r1) release_slot(u);  // nothing to read for this thread's half
           col_acc += (c0s + c1s) + (c2s + c3s);
           // the two threads of a key add their shares to the zero-initialised output: 0 + x + y is the same
           // in either order, so the result does not depend on timing
@@ -370,6 +448,7 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
             if (col < r_begin || col >= r_end) continue;  // another unit's columns
             float x[32];
             tmem_ld32(tbase + (col - r_begin), x);
+            tmem_wait_ld32(x);
 #pragma unroll
             for (int c = 0; c < 32; c += 4) {
               const float4 mm = *reinterpret_cast<const float4*>(s_f + col + c);
@@ -405,6 +484,7 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
           for (int rr = r0; rr < r1; rr += 32) {
             float x[32];
             tmem_ld32(tbase + (rr - r_begin), x);
+            tmem_wait_ld32(x);
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
               if (rr + c < r1) {
@@ -421,10 +501,7 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
           }
         }
       }
-      // hand the TMEM slot back to the MMA warp
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_free + 8 * (u % NSLOT));
+      if (MODE == kScoreMatrix) release_slot(u);  // the other modes handed it back right after their last load
     }
   }
 
@@ -473,7 +550,7 @@ __global__ void __launch_bounds__(256) score_stats_merge_kernel(const ScoreArgs 
 }
 
 static size_t score_smem_bytes(const ScoreShape& sh) {
-  return 1024 + 2 * (size_t)sh.q_rows * 128 + 2 * kKStageBytes + 4 * kScoreMaxRows * sizeof(float) + 10 * sizeof(uint64_t) + 16;
+  return 1024 + 2 * (size_t)sh.q_rows * 128 + 2 * kKStageBytes + 4 * kScoreMaxRows * sizeof(float) + 12 * sizeof(uint64_t) + 16;
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point lookup (libcuda is not linked)
@@ -541,24 +618,26 @@ int score_keys_per_cta(int n_jobs, int max_keys) {
   return kp;
 }
 
-int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream) {
-  if (a.n_jobs <= 0 || a.n_chunks <= 0) return CATEKV_OK;
-  if (a.G * a.L_obs > kScoreMaxRows || a.keys_per_cta % kKeyTile || !a.status) return CATEKV_ERR_UNSUPPORTED;
-  if (a.g_major && (a.L_obs != 64 || out_mode != kScoreMatrix)) return CATEKV_ERR_UNSUPPORTED;
-  const ScoreShape sh = score_shape(a.G, a.L_obs);
+int score_launch(const ScoreArgs& a0, ScoreMode out_mode, cudaStream_t stream) {
+  if (a0.n_jobs <= 0 || a0.max_keys <= 0) return CATEKV_OK;
+  if (a0.G * a0.L_obs > kScoreMaxRows || !a0.status) return CATEKV_ERR_UNSUPPORTED;
+  if (a0.g_major && (a0.L_obs != 64 || out_mode != kScoreMatrix)) return CATEKV_ERR_UNSUPPORTED;
+  const ScoreShape sh = score_shape(a0.G, a0.L_obs);
   CUtensorMap map;
-  int rc = make_k_map(a, &map);
+  int rc = make_k_map(a0, &map);
   if (rc) return rc;
+  if (out_mode == kScoreColsum)  // the two epilogue threads of a key add their shares into a zeroed vector
+    CATEKV_CUDA_TRY(cudaMemsetAsync(a0.out, 0, sizeof(float) * (size_t)a0.n_jobs * a0.out_job_stride, stream));
+  // (Scoring the jobs in groups whose keys fit the L2 together, both passes of a group back to back, was measured
+  // and lost: the smaller grids and extra launches cost more than the second pass gains from L2 hits.)
+  ScoreArgs a = a0;
+  a.keys_per_cta = score_keys_per_cta(a.n_jobs, a.max_keys);
+  a.n_chunks = (a.max_keys + a.keys_per_cta - 1) / a.keys_per_cta;  // jobs * chunks <= score_max_ctas(jobs): fits the partials
   rc = launch_one<kScoreStats>(a, sh, map, stream);
   if (rc) return rc;
   score_stats_merge_kernel<<<dim3((sh.R + 7) / 8, a.n_jobs), 256, 0, stream>>>(a, sh.R);
   CATEKV_CUDA_TRY(cudaGetLastError());
-  if (out_mode == kScoreColsum) {
-    // the two epilogue threads of a key add their shares into a zeroed vector
-    CATEKV_CUDA_TRY(cudaMemsetAsync(a.out, 0, sizeof(float) * (size_t)a.n_jobs * a.out_job_stride, stream));
-    return launch_one<kScoreColsum>(a, sh, map, stream);
-  }
-  return launch_one<kScoreMatrix>(a, sh, map, stream);
+  return out_mode == kScoreColsum ? launch_one<kScoreColsum>(a, sh, map, stream) : launch_one<kScoreMatrix>(a, sh, map, stream);
 }
 
 }  // namespace catekv

@@ -21,8 +21,9 @@ struct ScoreArgs {
   int32_t g_major;        // row order of the window queries: 0: r = i * G + g; 1: r = g * L_obs + i (matrix mode, L_obs = 64)
   int32_t B, Hkv, n_max;  // extents of k (sequences, KV heads, tokens) for the TMA descriptor
   float scale_log2;       // log2(e) / sqrt(d)
-  int32_t keys_per_cta;   // multiple of 128
-  int32_t n_chunks;       // grid.x: ceil(max key range / keys_per_cta)
+  int32_t max_keys;       // longest key range of any job
+  int32_t keys_per_cta;   // multiple of 128 (set by score_launch, per group of jobs)
+  int32_t n_chunks;       // grid.x: ceil(max key range / keys_per_cta) (set by score_launch)
   float2* stats_part;     // [n_jobs][n_chunks][kScoreMaxRows]  per-CTA (row max in the log2 domain, row sum)
   float2* stats;          // [n_jobs][kScoreMaxRows]            merged (row max, row sum)
   int32_t* status;        // device status block: CATEKV_STATUS_WAIT_EXPIRED is raised if a tensor-core wait ever runs out

@@ -581,8 +581,7 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
     sa.L_obs = p->L_obs;
     sa.causal = 0;  // every scored key precedes every window query
     sa.scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
-    sa.keys_per_cta = score_keys_per_cta((int)jobs.size(), n_sc_jobs_max);
-    sa.n_chunks = (n_sc_jobs_max + sa.keys_per_cta - 1) / sa.keys_per_cta;  // jobs * chunks <= score_max_ctas(jobs): fits the partials
+    sa.max_keys = n_sc_jobs_max;
     sa.stats_part = (float2*)(w8 + W.off_part);
     sa.stats = (float2*)(w8 + W.off_stats);
     sa.status = (int32_t*)(w8 + W.off_status);
