@@ -19,9 +19,12 @@
 // MMAs that read it have completed (a tcgen05.commit on the stage's "empty" barrier), however far
 // the epilogue lags.  Warp 8 (one elected lane) waits for a K tile, issues the eight k-steps of
 // tcgen05.mma per unit and commits them to the unit's "done" barrier; warps 0-7 are the epilogue
-// (two per TMEM lane quarter, each half of a unit's columns): they wait for the unit, read the
-// accumulators with tcgen05.ld into registers, hand the TMEM slot back at once and then do the
-// exp2 arithmetic.  There is no CTA-wide barrier in the main loop.  Every mbarrier wait is bounded: on
+// (two groups of four, one warp per TMEM lane quarter): the groups take alternate units, so that
+// one group's exponentials overlap the other group's wait, load and maximum; a group waits for its
+// unit, reads the accumulators with tcgen05.ld into registers 64 columns at a time, hands the TMEM
+// slot back right after its last load and then finishes the exp2 arithmetic.  (The head-major
+// matrix mode keeps both groups on every unit, half the columns each.)  There is no CTA-wide
+// barrier in the main loop.  Every mbarrier wait is bounded: on
 // expiry the thread raises a CTA-wide abort flag (which ends all other waits early) and a status
 // word in the workspace; the CTA then frees its TMEM and returns.
 #include <cuda.h>
@@ -192,6 +195,7 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
   const uint32_t bar_empty = smem_u32(s_bar + 10);  // a K stage has been read by all the MMAs of its tile
 
   constexpr bool kStats = MODE == kScoreStats;
+  constexpr bool kPingPong = MODE != kScoreMatrix;  // the two groups of four epilogue warps take alternate units
   const int UPT = kStats ? sh.MT : sh.NH;          // MMA units per key tile
   const int NSLOT = kStats ? sh.nslot1 : 2;
   const int slot_w = kStats ? 128 : sh.slotw2;
@@ -231,7 +235,9 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
     *s_abort = 0;
     for (int i = 0; i < 2; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar_full + 8 * i));
     for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar_done + 8 * i));
-    for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 8;\n" ::"r"(bar_free + 8 * i));  // one arrival per epilogue warp
+    // a slot is handed back by the epilogue warps that read it: the 4 warps of the group that owns the unit, or
+    // (matrix mode) all 8, two per lane quarter with half the columns each
+    for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar_free + 8 * i), "r"(kPingPong ? 4 : 8));
     for (int i = 0; i < 2; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar_empty + 8 * i));
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
@@ -307,7 +313,10 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
       if (lane == 0) mbar_arrive(bar_free + 8 * (u % NSLOT));
     };
 
-    for (int u = 0; u < U; ++u) {
+    // Row statistics and column sums: the two groups of four warps take alternate units (a group reads all the
+    // columns of its units), so that one group's exponentials overlap the other group's wait, load and maximum.
+    // Matrix mode: both groups work on every unit, half the columns each.
+    for (int u = kPingPong ? half : 0; u < U; u += kPingPong ? 2 : 1) {
       const int tile = u / UPT, sub = u - tile * UPT;
       if (!mbar_wait(bar_done + 8 * (u % NSLOT), (uint32_t)((u / NSLOT) & 1), s_abort, a.spin_limit)) break;
       tc_fence_after();
@@ -315,68 +324,71 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
       const int j0 = j_lo + tile * kKeyTile;
 
       if (kStats) {
-        // this thread's query row, keys [64 * half, 64 * half + 64) of the tile: one 64-column load, after which
-        // the TMEM slot goes straight back to the MMA warp (the arithmetic below runs on registers)
+        // this thread's query row against the tile's 128 keys, 64 columns at a time; after the second load the TMEM
+        // slot goes straight back to the MMA warp (the arithmetic runs on registers)
         const int r = sub * 128 + lane_row;
         const int i = a.g_major ? r % a.L_obs : r / a.G;
         const int lim = a.causal ? job.n - a.L_obs + i : 0x7fffffff;  // last key this window row sees
         const int jmax = min(j_hi - 1, lim);                          // keys j <= jmax are live
-        const int c0 = half * 64;
-        const bool any = j0 + c0 < j_hi;  // uniform: otherwise this half of the tile is padding
-        float x[64];
-        if (any) {
-          tmem_ld64(tbase + c0, x);
-          tmem_wait_ld64(x);
-        }
-        release_slot(u);
-        if (any) {
-          float m = s_f[2 * (half * kScoreMaxRows + r)], l = s_f[2 * (half * kScoreMaxRows + r) + 1];
-          if (j0 + c0 + 63 > jmax) {  // tail of the key range or the causal edge: mask entry by entry
+        float m = s_f[2 * (half * kScoreMaxRows + r)], l = s_f[2 * (half * kScoreMaxRows + r) + 1];
 #pragma unroll
-            for (int c = 0; c < 64; ++c) x[c] = (j0 + c0 + c <= jmax) ? x[c] : -INFINITY;
+        for (int hh = 0; hh < 2; ++hh) {
+          const int c0 = hh * 64;
+          const bool any = j0 + c0 < j_hi;  // uniform: otherwise this half of the tile is padding
+          float x[64];
+          if (any) {
+            tmem_ld64(tbase + c0, x);
+            tmem_wait_ld64(x);
           }
-          // four independent chains of three-input maxima
-          float mx0 = fmax3(x[0], x[1], x[2]), mx1 = fmax3(x[3], x[4], x[5]);
-          float mx2 = fmax3(x[6], x[7], x[8]), mx3 = fmax3(x[9], x[10], x[11]);
+          if (hh == 1) release_slot(u);
+          if (any) {
+            if (j0 + c0 + 63 > jmax) {  // tail of the key range or the causal edge: mask entry by entry
 #pragma unroll
-          for (int c = 12; c < 60; c += 8) {
-            mx0 = fmax3(mx0, x[c], x[c + 1]);
-            mx1 = fmax3(mx1, x[c + 2], x[c + 3]);
-            mx2 = fmax3(mx2, x[c + 4], x[c + 5]);
-            mx3 = fmax3(mx3, x[c + 6], x[c + 7]);
-          }
-          mx0 = fmax3(mx0, x[60], x[61]);
-          mx1 = fmax3(mx1, x[62], x[63]);
-          float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-          mx *= a.scale_log2;  // the scale is positive: the max commutes with it
-          if (mx > m) {
-            l *= fast_exp2(m - mx);
-            m = mx;
-          }
-          if (m > -INFINITY) {
-            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-            for (int c = 0; c < 64; c += 4) {
-              s0 += fast_exp2(fmaf(x[c], a.scale_log2, -m));
-              s1 += fast_exp2(fmaf(x[c + 1], a.scale_log2, -m));
-              s2 += fast_exp2(fmaf(x[c + 2], a.scale_log2, -m));
-              s3 += fast_exp2(fmaf(x[c + 3], a.scale_log2, -m));
+              for (int c = 0; c < 64; ++c) x[c] = (j0 + c0 + c <= jmax) ? x[c] : -INFINITY;
             }
-            l += (s0 + s1) + (s2 + s3);
+            // four independent chains of three-input maxima
+            float mx0 = fmax3(x[0], x[1], x[2]), mx1 = fmax3(x[3], x[4], x[5]);
+            float mx2 = fmax3(x[6], x[7], x[8]), mx3 = fmax3(x[9], x[10], x[11]);
+#pragma unroll
+            for (int c = 12; c < 60; c += 8) {
+              mx0 = fmax3(mx0, x[c], x[c + 1]);
+              mx1 = fmax3(mx1, x[c + 2], x[c + 3]);
+              mx2 = fmax3(mx2, x[c + 4], x[c + 5]);
+              mx3 = fmax3(mx3, x[c + 6], x[c + 7]);
+            }
+            mx0 = fmax3(mx0, x[60], x[61]);
+            mx1 = fmax3(mx1, x[62], x[63]);
+            float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+            mx *= a.scale_log2;  // the scale is positive: the max commutes with it
+            if (mx > m) {
+              l *= fast_exp2(m - mx);
+              m = mx;
+            }
+            if (m > -INFINITY) {
+              float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+              for (int c = 0; c < 64; c += 4) {
+                s0 += fast_exp2(fmaf(x[c], a.scale_log2, -m));
+                s1 += fast_exp2(fmaf(x[c + 1], a.scale_log2, -m));
+                s2 += fast_exp2(fmaf(x[c + 2], a.scale_log2, -m));
+                s3 += fast_exp2(fmaf(x[c + 3], a.scale_log2, -m));
+              }
+              l += (s0 + s1) + (s2 + s3);
+            }
           }
-          s_f[2 * (half * kScoreMaxRows + r)] = m;
-          s_f[2 * (half * kScoreMaxRows + r) + 1] = l;
         }
+        s_f[2 * (half * kScoreMaxRows + r)] = m;
+        s_f[2 * (half * kScoreMaxRows + r) + 1] = l;
       } else {
-        // this thread's key; the unit's rows [r_begin, r_end) are cut between the two halves: at a multiple of 32
-        // columns for the column sums, at a multiple of G for the matrix (whole window rows per thread)
+        // this thread's key against the unit's rows [r_begin, r_end)
         const int j = j0 + lane_row;
         const int r_begin = sub * sh.NW, r_end = min(sh.R, r_begin + sh.NW);
-        const int cut = MODE == kScoreColsum ? min(r_end, r_begin + ((r_end - r_begin) / 2 + 31) / 32 * 32)
-                                             : r_begin + ((r_end - r_begin) / 2 / a.G) * a.G;
-        const int r0 = half ? cut : r_begin, r1 = half ? r_end : cut;
+        // column sums: all of the unit's rows; matrix: the rows are cut between the halves at a multiple of G
+        const int cut = r_begin + ((r_end - r_begin) / 2 / a.G) * a.G;
+        const int r0 = MODE == kScoreColsum ? r_begin : (half ? cut : r_begin);
+        const int r1 = MODE == kScoreColsum ? r_end : (half ? r_end : cut);
         if (MODE == kScoreColsum) {
-          if (sub == 0) col_acc = 0.f;
+          col_acc = 0.f;
           float c0s = 0.f, c1s = 0.f, c2s = 0.f, c3s = 0.f;
           // 64 rows per load where that many are left, else 32; the slot is handed back after the last load
 #pragma unroll 1
@@ -426,10 +438,14 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
           }
           if (r0 >= r1) release_slot(u);  // nothing to read for this thread's half
           col_acc += (c0s + c1s) + (c2s + c3s);
-          // the two threads of a key add their shares to the zero-initialised output: 0 + x + y is the same
-          // in either order, so the result does not depend on timing
-          if (sub == UPT - 1 && j < j_hi)
-            atomicAdd(a.out + (size_t)blockIdx.y * a.out_job_stride + (j - job.j_begin), col_acc * inv_g);
+          // One unit per tile: this thread holds the key's whole sum.  Two units per tile (more than 256 rows):
+          // they belong to different groups, whose threads add their shares to the zero-initialised output
+          // (0 + x + y is the same in either order, so the result does not depend on timing).
+          if (j < j_hi) {
+            float* dst = a.out + (size_t)blockIdx.y * a.out_job_stride + (j - job.j_begin);
+            if (UPT == 1) *dst = col_acc * inv_g;
+            else atomicAdd(dst, col_acc * inv_g);
+          }
         } else if (a.g_major) {
           // group-mean matrix with head-major rows and L_obs = 64: this thread owns the window rows 32 * half + c
           // (c = 0..31) of its key; head g's logits for them are the 32 TMEM columns from g * 64 + 32 * half on, so
@@ -626,7 +642,7 @@ int score_launch(const ScoreArgs& a0, ScoreMode out_mode, cudaStream_t stream) {
   CUtensorMap map;
   int rc = make_k_map(a0, &map);
   if (rc) return rc;
-  if (out_mode == kScoreColsum)  // the two epilogue threads of a key add their shares into a zeroed vector
+  if (out_mode == kScoreColsum && sh.NH > 1)  // two units per tile add their shares into a zeroed vector
     CATEKV_CUDA_TRY(cudaMemsetAsync(a0.out, 0, sizeof(float) * (size_t)a0.n_jobs * a0.out_job_stride, stream));
   // (Scoring the jobs in groups whose keys fit the L2 together, both passes of a group back to back, was measured
   // and lost: the smaller grids and extra launches cost more than the second pass gains from L2 hits.)
