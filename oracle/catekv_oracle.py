@@ -22,6 +22,12 @@ What each function follows
                                       grows by the decoded token.
 * attention, decode_attention       : Algorithm 1, "Attention(q, k, v)"; the
                                       plain softmax-attention definition.
+* window_attention, scored_range_lse, window_scores_from_lse
+                                    : Algorithm 1, pre-filling stage: the
+                                      attention rows of the last L_obs prefill
+                                      queries (what a prefill pass computes for
+                                      those positions), their log-sum-exp, and
+                                      the token criticality re-derived from it.
 * attention_recall                  : Section 3.4 (attention weight recall of a
                                       kept set, Fig. 4).
 * token_budget (streaming type)     : Section 4.2.4 (sink + recent heads).
@@ -190,6 +196,62 @@ def window_scores(qwin_bits: np.ndarray, k_bits: np.ndarray, L_obs: int) -> np.n
         Q = bf16_to_f64(qwin_bits[g])
         A = _row_softmax((Q @ K.T) / math.sqrt(d))
         C += A.sum(axis=0)
+    return C / G
+
+
+def window_attention(qwin_bits: np.ndarray, k_bits: np.ndarray, v_bits: np.ndarray, L_obs: int,
+                     scale: Optional[float] = None):
+    """The prefill attention of the observation window (Algorithm 1, pre-filling stage: the queries
+    Q[-L_obs:] whose scores select the tokens are ordinary prefill queries).
+
+    qwin_bits [G, L_obs, d], k_bits / v_bits [n, d].  Window row i sits at position n - L_obs + i and, being a
+    prefill query, attends causally to keys 0 .. n - L_obs + i.  Returns (out [G, L_obs, d], lse [G, L_obs]):
+    softmax(scale * q K^T) V over that prefix and the natural-log sum of exp(logits).
+    """
+    G, Lw, d = qwin_bits.shape
+    assert Lw == L_obs
+    n = k_bits.shape[0]
+    if scale is None or scale == 0:
+        scale = 1.0 / math.sqrt(d)
+    K, V = bf16_to_f64(k_bits), bf16_to_f64(v_bits)
+    out = np.zeros((G, L_obs, d))
+    lse = np.zeros((G, L_obs))
+    for g in range(G):
+        Q = bf16_to_f64(qwin_bits[g])
+        for i in range(L_obs):
+            pos = n - L_obs + i
+            out[g, i], lse[g, i] = attention(Q[i], K[:pos + 1], V[:pos + 1], scale)
+    return out, lse
+
+
+def scored_range_lse(qwin_bits: np.ndarray, k_bits: np.ndarray, L_obs: int) -> np.ndarray:
+    """Natural-log sum of exp(q_i . k_j / sqrt(d)) of every window row over the scored keys j < n - L_obs alone:
+    the normaliser of the softmax in Algorithm 1's "token criticality" line.  [G, L_obs].
+    (It relates to the causal log-sum-exp of window_attention by
+    exp(lse_full) = exp(lse_scored) + sum over the window's own keys j <= n - L_obs + i of exp(logit).)"""
+    G, Lw, d = qwin_bits.shape
+    n = k_bits.shape[0]
+    K = bf16_to_f64(k_bits[: n - L_obs])
+    out = np.zeros((G, L_obs))
+    for g in range(G):
+        S = (bf16_to_f64(qwin_bits[g]) @ K.T) / math.sqrt(d)
+        m = S.max(axis=1)
+        out[g] = m + np.log(np.exp(S - m[:, None]).sum(axis=1))
+    return out
+
+
+def window_scores_from_lse(qwin_bits: np.ndarray, k_bits: np.ndarray, L_obs: int, lse_sel: np.ndarray) -> np.ndarray:
+    """Token criticality C of Algorithm 1 with the softmax normaliser given instead of computed:
+    C_j = mean_g sum_i exp(q_gi . k_j / sqrt(d) - lse_sel[g, i]) for the scored keys j < n - L_obs."""
+    G, Lw, d = qwin_bits.shape
+    n = k_bits.shape[0]
+    ns = n - L_obs
+    K = bf16_to_f64(k_bits[:ns])
+    C = np.zeros(ns)
+    for g in range(G):
+        Q = bf16_to_f64(qwin_bits[g])
+        S = (Q @ K.T) / math.sqrt(d)
+        C += np.exp(S - lse_sel[g][:, None]).sum(axis=0)
     return C / G
 
 

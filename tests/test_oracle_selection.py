@@ -258,3 +258,72 @@ def test_attention_recall_pins(golden_dir):
     s = [0.25 * sum(float(a) * float(b) for a, b in zip(K3[j], q3)) for j in range(200)]
     Z = math.fsum(math.exp(x) for x in s)
     assert r == pytest.approx(math.fsum(math.exp(s[j]) for j in kept) / Z, rel=1e-12)
+
+
+def test_window_attention_against_library_sdpa_and_brute_force():
+    rng = np.random.default_rng(60)
+    G, L_obs, n, d = 3, 5, 23, 16
+    qw = orc.f64_to_bf16(rng.standard_normal((G, L_obs, d)))
+    k = orc.f64_to_bf16(rng.standard_normal((n, d)))
+    v = orc.f64_to_bf16(rng.standard_normal((n, d)))
+    out, lse = orc.window_attention(qw, k, v, L_obs)
+    Q = torch.from_numpy(orc.bf16_to_f64(qw))
+    K = torch.from_numpy(orc.bf16_to_f64(k))
+    V = torch.from_numpy(orc.bf16_to_f64(v))
+    pos = torch.arange(n - L_obs, n)[:, None]
+    allowed = torch.arange(n)[None, :] <= pos                      # [L_obs, n]: causal prefix of every window row
+    ref = torch.nn.functional.scaled_dot_product_attention(Q[None], K[None, None].expand(1, G, n, d),
+                                                           V[None, None].expand(1, G, n, d), attn_mask=allowed)[0]
+    np.testing.assert_allclose(out, ref.numpy(), rtol=1e-12, atol=1e-14)
+    logits = torch.einsum("gid,jd->gij", Q, K) / math.sqrt(d)
+    ref_lse = torch.logsumexp(logits.masked_fill(~allowed, -math.inf), dim=-1)
+    np.testing.assert_allclose(lse, ref_lse.numpy(), rtol=1e-13)
+    # pure Python, one row: the last window row sees every key, the first one n - L_obs + 1 keys
+    for g, i in ((0, L_obs - 1), (2, 0)):
+        q = [float(x) for x in orc.bf16_to_f64(qw[g, i])]
+        m = n - L_obs + i + 1
+        s = [sum(a * float(b) for a, b in zip(q, orc.bf16_to_f64(k[j]))) / math.sqrt(d) for j in range(m)]
+        Z = math.fsum(math.exp(x) for x in s)
+        want = [math.fsum(math.exp(s[j]) * float(orc.bf16_to_f64(v[j])[e]) for j in range(m)) / Z for e in range(d)]
+        np.testing.assert_allclose(out[g, i], want, rtol=1e-12)
+        assert lse[g, i] == pytest.approx(math.log(Z), rel=1e-13)
+
+
+def test_window_attention_closed_form_identical_keys():
+    # identical keys: uniform weights over the causal prefix -> the mean of its values, lse = logit + log(prefix)
+    rng = np.random.default_rng(61)
+    G, L_obs, n, d = 2, 4, 12, 8
+    qw = orc.f64_to_bf16(rng.standard_normal((G, L_obs, d)))
+    k = np.tile(orc.f64_to_bf16(rng.standard_normal((1, d))), (n, 1))
+    v = orc.f64_to_bf16(rng.standard_normal((n, d)))
+    out, lse = orc.window_attention(qw, k, v, L_obs)
+    V = orc.bf16_to_f64(v)
+    for g in range(G):
+        for i in range(L_obs):
+            m = n - L_obs + i + 1
+            np.testing.assert_allclose(out[g, i], V[:m].mean(axis=0), rtol=1e-13, atol=1e-15)
+            logit = float(orc.bf16_to_f64(qw[g, i]) @ orc.bf16_to_f64(k[0])) / math.sqrt(d)
+            assert lse[g, i] == pytest.approx(logit + math.log(m), rel=1e-13)
+
+
+def test_criticality_from_the_prefill_log_sum_exp():
+    # the scored range's normaliser against a library logsumexp, its relation to the causal one, and C rebuilt from it
+    rng = np.random.default_rng(62)
+    G, L_obs, n, d = 4, 6, 50, 16
+    qw = orc.f64_to_bf16(rng.standard_normal((G, L_obs, d)))
+    k = orc.f64_to_bf16(rng.standard_normal((n, d)))
+    v = orc.f64_to_bf16(rng.standard_normal((n, d)))
+    _, lse_full = orc.window_attention(qw, k, v, L_obs)
+    lse_sel = orc.scored_range_lse(qw, k, L_obs)
+    Q = torch.from_numpy(orc.bf16_to_f64(qw))
+    K = torch.from_numpy(orc.bf16_to_f64(k))
+    logits = torch.einsum("gid,jd->gij", Q, K) / math.sqrt(d)
+    np.testing.assert_allclose(lse_sel, torch.logsumexp(logits[:, :, : n - L_obs], dim=-1).numpy(), rtol=1e-13)
+    # exp(lse_full) = exp(lse_scored) + the window's own causal keys
+    for g in range(G):
+        for i in range(L_obs):
+            own = math.fsum(math.exp(float(logits[g, i, j])) for j in range(n - L_obs, n - L_obs + i + 1))
+            assert math.exp(lse_full[g, i]) == pytest.approx(math.exp(lse_sel[g, i]) + own, rel=1e-12)
+    C = orc.window_scores_from_lse(qw, k, L_obs, lse_sel)
+    np.testing.assert_allclose(C, orc.window_scores(qw, k, L_obs), rtol=1e-11)
+    assert abs(C.sum() - L_obs) < 1e-10
