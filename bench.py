@@ -386,6 +386,46 @@ def time_head_cv(ck, dev):
     return e0.elapsed_time(e1) / 3
 
 
+def time_window_attn(ck, w, dev, layer=0, reps=5):
+    """catekv_window_attn on the workload's prefill shape (one layer), and catekv_select_compact with and without the
+    normaliser it delivers.  Returns a dict of milliseconds and the bytes / flops the attention call has to move."""
+    import torch
+    from workloads import synth
+    p = synth.prefill_layer(w, layer, dev)
+    mask = p["head_mask"]
+    ws = torch.empty(ck._lib.catekv_window_attn_workspace_bytes(w.B, w.Hq, w.Hkv, w.n, w.L_obs), dtype=torch.uint8, device=dev)
+    sws = torch.empty(ck.catekv_select_workspace_bytes(w.B, w.Hq, w.Hkv, w.n, w.L_obs), dtype=torch.uint8, device=dev)
+    cache = ck.Cache(w.B, w.Hkv, expected_lengths(w, mask), 8, dev)
+
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    res = {}
+    lse_sc = [None]
+
+    def wa():
+        lse_sc[0] = ck.catekv_window_attn(p["q_win"], p["k"], p["v"], p["seq_len"], out_dtype=torch.bfloat16, ws=ws)[2]
+    res["window_attn_ms"] = timed(wa)
+    sel = lambda lse: ck.catekv_select_compact(p["q_win"], p["k"], p["v"], p["seq_len"], mask, cache, w.budget, w.eta, w.sink,
+                                               w.local, w.pool_mode, w.pool_param, ws=sws, row_lse_scored=lse)
+    res["select_ms"] = timed(lambda: sel(None))
+    res["select_with_normaliser_ms"] = timed(lambda: sel(lse_sc[0]))
+    kv_bytes = w.B * w.Hkv * w.n * 256
+    res["k_bytes"] = kv_bytes
+    res["hbm_bytes_window_attn"] = 3 * kv_bytes  # K twice (normalisers, P V), V once
+    res["flops_window_attn"] = 2.0 * w.B * w.Hq * w.L_obs * w.n * w.d * 4  # Q K^T twice, P_hi V, P_lo V
+    return res
+
+
 def time_retrieval(ck, w, dev, n_layers=4, budget=1024, cs=8, steps=8, graph=True, gather=False):
     """Decode step with query-aware retrieval on the adaptive heads (budget rows per adaptive head, chunk size 8):
     per layer catekv_append_retrieval + catekv_retrieve_select + catekv_decode_attn_indexed
@@ -704,6 +744,8 @@ def main():
                     "(8 prompts x 16384 tokens, 28q/4kv, window 64) and print its time; for profiling")
     ap.add_argument("--retrieval-gather", action="store_true", help="with --retrieval-only: the gather path "
                     "(catekv_retrieve_compact into a per-step cache) instead of attention in place")
+    ap.add_argument("--window-attn-only", action="store_true", help="run only catekv_window_attn and the selection "
+                    "with and without its normaliser on the workload's prefill shape; for profiling")
     ap.add_argument("--no-extras", action="store_true", help="skip the other configs, head_cv and the oracle timing")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -741,6 +783,11 @@ def main():
         ms_cv = time_head_cv(ck, dev)
         if rank == 0:
             print(json.dumps({"head_cv_ms": ms_cv, "shape": "8 prompts x 16384 tokens, 28q/4kv, window 64"}))
+        return
+    if args.window_attn_only:
+        res = time_window_attn(ck, w, dev)
+        if rank == 0:
+            print(json.dumps({"workload": w.name, **res}))
         return
     if args.retrieval_only:
         ru, ra, rm = time_retrieval(ck, w, dev, n_layers=n_layers, steps=args.steps, graph=graph,
@@ -796,6 +843,12 @@ def main():
                              "metadata_bytes_per_layer_step": rm, "budget_rows": 1024, "chunk": 8,
                              "note": "query-aware retrieval on the adaptive heads of the same workload: per layer "
                                      "catekv_append_retrieval, catekv_retrieve_select, catekv_decode_attn_indexed; CUDA graph replay of the step"}
+        wa = time_window_attn(ck, synth.WORKLOADS["cfg2"], dev)
+        wa["tflops"] = wa["flops_window_attn"] / (wa["window_attn_ms"] * 1e-3) / 1e12
+        wa["hbm_gbs"] = wa["hbm_bytes_window_attn"] / (wa["window_attn_ms"] * 1e-3) / 1e9
+        wa["note"] = ("configs[2] prefill shape, one layer: catekv_window_attn (prefill rows of the observation window "
+                      "+ their normalisers) and catekv_select_compact with / without that normaliser")
+        line["window_attn"] = wa
         line["linearity"] = time_linearity(ck, dev)
         rate, desc, spent = oracle_sample_rate(w, target_s=15.0)
         rows = bytes_per_layer / ROW_BYTES

@@ -237,6 +237,10 @@ typedef struct catekv_select_params {
   int64_t kv_stride_b, kv_stride_h, kv_stride_t; /* element strides of k and v; d contiguous */
   const int32_t* seq_len;    /* host [B]: n of each sequence */
   const uint8_t* head_mask;  /* host [B*Hkv]: 0 = adaptive, 1 = consistent, 2 = streaming (T = sink + local; Section 4.2.4) */
+  const float* row_lse_scored; /* device float [B, Hq, L_obs] or NULL: natural-log sum of exp(q.k / sqrt(d)) of every
+                                  window query over the scored keys [0, n - L_obs), as catekv_window_attn (or any
+                                  prefill attention pass that tracks it) delivers it.  With it the call skips its
+                                  own first pass over K (the row maxima and sums) */
 } catekv_select_params;
 
 /*
@@ -264,6 +268,28 @@ typedef struct catekv_select_params {
 size_t catekv_select_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t n_max, int32_t L_obs);
 int catekv_select_compact(const catekv_select_params* p, catekv_cache* cache, int32_t* idx_out,
                           int64_t idx_stride, void* ws, size_t ws_bytes, catekv_stream stream);
+
+/*
+ * Algorithm 1, pre-filling stage, seen from the prefill side: the window queries Q[-L_obs:] are ordinary prefill
+ * queries, so their attention rows and softmax normalisers exist before any scoring starts.  This call is the
+ * library's stand-in for that part of a prefill attention pass: for the last L_obs queries of every query head,
+ *   out        = softmax(q K[:pos+1]^T / sqrt(d)) V[:pos+1], the causal attention row at position pos = n - L_obs + i
+ *   lse        = natural-log sum of exp(logits) over that causal prefix (what attention kernels return as LSE)
+ *   lse_scored = the same sum over the scored keys [0, n - L_obs) alone: the normaliser of the softmax in the
+ *                "token criticality" line; hand it to catekv_select_compact as row_lse_scored
+ * bf16 inputs, fp32 accumulation; the probabilities enter the P V product as a bf16 hi + lo pair.
+ *   q_win  device bf16 [B, Hq, L_obs, d] contiguous;  k, v  device bf16 with element strides, d contiguous
+ *   seq_len host [B], n >= L_obs;  out device [B, Hq, L_obs, d] bf16 or float per out_dtype
+ *   lse_out, lse_scored_out device float [B, Hq, L_obs] or NULL (-inf where a row has no key)
+ *   ws device scratch of at least catekv_window_attn_workspace_bytes(...); its first CATEKV_STATUS_BYTES are the
+ *   status block (cleared by this call).
+ * K is read twice (row normalisers, then P V), V once.
+ */
+size_t catekv_window_attn_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t n_max, int32_t L_obs);
+int catekv_window_attn(const void* q_win, const void* k, const void* v, int64_t kv_stride_b, int64_t kv_stride_h,
+                       int64_t kv_stride_t, const int32_t* seq_len, int32_t B, int32_t Hq, int32_t Hkv, int32_t d,
+                       int32_t L_obs, void* out, int32_t out_dtype, float* lse_out, float* lse_scored_out, void* ws,
+                       size_t ws_bytes, catekv_stream stream);
 
 /*
  * Copy the device's segment lengths into the host mirror cache->seg_len (on `stream`, which is synchronised)

@@ -63,7 +63,7 @@ class SelectParams(C.Structure):
                 ("reserved", C.c_int32),
                 ("q_win", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p),
                 ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64), ("kv_stride_t", C.c_int64),
-                ("seq_len", C.c_void_p), ("head_mask", C.c_void_p)]
+                ("seq_len", C.c_void_p), ("head_mask", C.c_void_p), ("row_lse_scored", C.c_void_p)]
 
 
 def _load():
@@ -115,6 +115,8 @@ def _load():
         "catekv_checked_status": (C.c_int, [C.POINTER(StatusStruct), i32]),
         "catekv_test_expire_score_waits": (None, [i32]),
         "catekv_cache_sync_lengths": (C.c_int, [C.POINTER(CacheStruct), vp]),
+        "catekv_window_attn_workspace_bytes": (sz, [i32, i32, i32, i32, i32]),
+        "catekv_window_attn": (C.c_int, [vp, vp, vp, i64, i64, i64, vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, sz, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -478,8 +480,9 @@ def catekv_select_workspace_bytes(B, Hq, Hkv, n_max, L_obs) -> int:
 def catekv_select_compact(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_len, head_mask, cache: Cache,
                           budget_consistent: int, eta_adaptive: float, sink: int, local: int, pool_mode: int,
                           pool_param: int, ws: Optional[torch.Tensor] = None,
-                          idx_out: Optional[torch.Tensor] = None):
-    """q_win [B,Hq,L_obs,d] bf16 contiguous; k, v [B,Hkv,n_max,d] bf16 (any strides, d contiguous)."""
+                          idx_out: Optional[torch.Tensor] = None, row_lse_scored: Optional[torch.Tensor] = None):
+    """q_win [B,Hq,L_obs,d] bf16 contiguous; k, v [B,Hkv,n_max,d] bf16 (any strides, d contiguous).
+    row_lse_scored: float32 [B,Hq,L_obs] from catekv_window_attn (the call then skips its first pass over K)."""
     B, Hq, L_obs, d = q_win.shape
     Hkv, n_max = k.shape[1], k.shape[2]
     assert q_win.is_contiguous() and k.stride(3) == 1 and v.stride() == k.stride()
@@ -489,11 +492,36 @@ def catekv_select_compact(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
         ws = torch.empty(catekv_select_workspace_bytes(B, Hq, Hkv, n_max, L_obs), dtype=torch.uint8, device=k.device)
     p = SelectParams(B, Hq, Hkv, d, L_obs, sink, local, budget_consistent, eta_adaptive, pool_mode, pool_param, 0,
                      q_win.data_ptr(), k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1), k.stride(2),
-                     _np_ptr(seq_len), _np_ptr(head_mask))
+                     _np_ptr(seq_len), _np_ptr(head_mask), _dev_ptr(row_lse_scored))
+    if row_lse_scored is not None:
+        assert row_lse_scored.dtype == torch.float32 and row_lse_scored.is_contiguous()
+        assert tuple(row_lse_scored.shape) == (B, Hq, L_obs)
     stride = 0 if idx_out is None else idx_out.stride(0)
     _check(_lib.catekv_select_compact(C.byref(p), C.byref(cache.struct), _dev_ptr(idx_out), stride, ws.data_ptr(),
                                       ws.numel(), _stream()), "catekv_select_compact")
     return ws
+
+
+def catekv_window_attn(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_len, out_dtype=torch.float32,
+                       ws: Optional[torch.Tensor] = None):
+    """-> (out [B,Hq,L_obs,d], lse [B,Hq,L_obs], lse_scored [B,Hq,L_obs]) on the device: the causal attention rows of
+    the last L_obs queries, their log-sum-exp, and the log-sum-exp over the scored keys [0, n - L_obs) alone."""
+    B, Hq, L_obs, d = q_win.shape
+    Hkv, n_max = k.shape[1], k.shape[2]
+    assert q_win.is_contiguous() and k.stride(3) == 1 and v.stride() == k.stride()
+    seq_len = np.ascontiguousarray(seq_len, dtype=np.int32).reshape(-1)
+    if ws is None:
+        ws = torch.empty(_lib.catekv_window_attn_workspace_bytes(B, Hq, Hkv, n_max, L_obs), dtype=torch.uint8,
+                         device=k.device)
+    out = torch.empty((B, Hq, L_obs, d), dtype=out_dtype, device=k.device)
+    lse = torch.empty((B, Hq, L_obs), dtype=torch.float32, device=k.device)
+    lse_scored = torch.empty_like(lse)
+    od = OUT_BF16 if out_dtype == torch.bfloat16 else OUT_FP32
+    assert out_dtype in (torch.bfloat16, torch.float32)
+    _check(_lib.catekv_window_attn(q_win.data_ptr(), k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1), k.stride(2),
+                                   _np_ptr(seq_len), B, Hq, Hkv, d, L_obs, out.data_ptr(), od, lse.data_ptr(),
+                                   lse_scored.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "catekv_window_attn")
+    return out, lse, lse_scored
 
 
 def catekv_head_cv_workspace_bytes(B, Hq, Hkv, n_max, L_obs, L_init, L_rec) -> int:

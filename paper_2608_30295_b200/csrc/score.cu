@@ -33,15 +33,12 @@
 #include <atomic>
 
 #include "score.cuh"
+#include "tc.cuh"
 
 namespace catekv {
 
 constexpr int kEpiThreads = 256;                   // 8 epilogue warps: two per TMEM lane quarter, each takes half the columns
 constexpr int kScThreads = kEpiThreads + 64;       // + the MMA warp (8) and the TMA warp (9)
-constexpr int kKeyTile = 128;                       // keys per tile
-constexpr int kKBlockBytes = kKeyTile * 128;        // one 64-element k-block of a K tile
-constexpr int kKStageBytes = 2 * kKBlockBytes;      // K tile: 128 keys x 128 dims bf16
-constexpr uint32_t kSpinLimit = 1u << 22;
 
 struct ScoreShape {
   int R;         // query rows
@@ -72,102 +69,6 @@ static ScoreShape score_shape(int G, int L_obs) {
   while (c < 2 * s.slotw2) c *= 2;
   s.cols2 = c;
   return s;
-}
-
-// ---- tcgen05 / mbarrier wrappers ----------------------------------------------------------
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
-  // K-major, SWIZZLE_128B: rows of 128 bytes, 8-row groups 1024 bytes apart
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
-  d |= (uint64_t)1 << 16;               // leading byte offset: unused for this layout
-  d |= (uint64_t)(1024 >> 4) << 32;     // stride byte offset
-  d |= (uint64_t)1 << 46;               // descriptor version
-  d |= (uint64_t)2 << 61;               // SWIZZLE_128B
-  return d;
-}
-__device__ __forceinline__ uint32_t umma_idesc_bf16(int M, int N) {
-  // D = f32, A = B = bf16, both K-major
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(tmem_d),
-      "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
-// Bounded wait for a phase of an mbarrier.  Returns false if it never completed or if another thread of
-// the CTA has given up (abort flag), in which case the flag is (also) raised by this thread.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
-  for (uint32_t it = 0; it < limit; ++it) {
-    uint32_t done;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    if (done) return true;
-    if ((it & 255u) == 255u && *abort_flag) break;
-  }
-  *abort_flag = 1;
-  return false;
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
-}
-// one 64-column x 128-row box of K (rank-4 map: d, token, head, sequence) into shared memory
-__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* map, int d0, int j0, int h, int b, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n" ::"r"(dst),
-      "l"(map), "r"(d0), "r"(j0), "r"(h), "r"(b), "r"(bar)
-      : "memory");
-}
-// 32 consecutive TMEM columns of this thread's lane, straight into float registers.  The load is asynchronous:
-// tmem_wait_ld32 must run before the values are used (it takes the registers as operands, so that no use can
-// be scheduled ahead of it).
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
-               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]), "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15]), "=f"(v[16]), "=f"(v[17]), "=f"(v[18]), "=f"(v[19]), "=f"(v[20]), "=f"(v[21]), "=f"(v[22]), "=f"(v[23]), "=f"(v[24]), "=f"(v[25]), "=f"(v[26]), "=f"(v[27]), "=f"(v[28]), "=f"(v[29]), "=f"(v[30]), "=f"(v[31])
-               : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_wait_ld32(float (&v)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;\n"
-               : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7]), "+f"(v[8]), "+f"(v[9]), "+f"(v[10]), "+f"(v[11]), "+f"(v[12]), "+f"(v[13]), "+f"(v[14]), "+f"(v[15]), "+f"(v[16]), "+f"(v[17]), "+f"(v[18]), "+f"(v[19]), "+f"(v[20]), "+f"(v[21]), "+f"(v[22]), "+f"(v[23]), "+f"(v[24]), "+f"(v[25]), "+f"(v[26]), "+f"(v[27]), "+f"(v[28]), "+f"(v[29]), "+f"(v[30]), "+f"(v[31])
-               :
-               : "memory");
-}
-// 64 consecutive TMEM columns of this thread's lane, straight into float registers.  The load is asynchronous:
-// tmem_wait_ld64 must run before the values are used (it takes the registers as operands, so that no use can
-// be scheduled ahead of it).
-__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%64];\n"
-               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]), "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15]), "=f"(v[16]), "=f"(v[17]), "=f"(v[18]), "=f"(v[19]), "=f"(v[20]), "=f"(v[21]), "=f"(v[22]), "=f"(v[23]), "=f"(v[24]), "=f"(v[25]), "=f"(v[26]), "=f"(v[27]), "=f"(v[28]), "=f"(v[29]), "=f"(v[30]), "=f"(v[31]), "=f"(v[32]), "=f"(v[33]), "=f"(v[34]), "=f"(v[35]), "=f"(v[36]), "=f"(v[37]), "=f"(v[38]), "=f"(v[39]), "=f"(v[40]), "=f"(v[41]), "=f"(v[42]), "=f"(v[43]), "=f"(v[44]), "=f"(v[45]), "=f"(v[46]), "=f"(v[47]), "=f"(v[48]), "=f"(v[49]), "=f"(v[50]), "=f"(v[51]), "=f"(v[52]), "=f"(v[53]), "=f"(v[54]), "=f"(v[55]), "=f"(v[56]), "=f"(v[57]), "=f"(v[58]), "=f"(v[59]), "=f"(v[60]), "=f"(v[61]), "=f"(v[62]), "=f"(v[63])
-               : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_wait_ld64(float (&v)[64]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;\n"
-               : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7]), "+f"(v[8]), "+f"(v[9]), "+f"(v[10]), "+f"(v[11]), "+f"(v[12]), "+f"(v[13]), "+f"(v[14]), "+f"(v[15]), "+f"(v[16]), "+f"(v[17]), "+f"(v[18]), "+f"(v[19]), "+f"(v[20]), "+f"(v[21]), "+f"(v[22]), "+f"(v[23]), "+f"(v[24]), "+f"(v[25]), "+f"(v[26]), "+f"(v[27]), "+f"(v[28]), "+f"(v[29]), "+f"(v[30]), "+f"(v[31]), "+f"(v[32]), "+f"(v[33]), "+f"(v[34]), "+f"(v[35]), "+f"(v[36]), "+f"(v[37]), "+f"(v[38]), "+f"(v[39]), "+f"(v[40]), "+f"(v[41]), "+f"(v[42]), "+f"(v[43]), "+f"(v[44]), "+f"(v[45]), "+f"(v[46]), "+f"(v[47]), "+f"(v[48]), "+f"(v[49]), "+f"(v[50]), "+f"(v[51]), "+f"(v[52]), "+f"(v[53]), "+f"(v[54]), "+f"(v[55]), "+f"(v[56]), "+f"(v[57]), "+f"(v[58]), "+f"(v[59]), "+f"(v[60]), "+f"(v[61]), "+f"(v[62]), "+f"(v[63])
-               :
-               : "memory");
-}
-__device__ __forceinline__ float fmax3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-
-// offset of the 16-byte chunk c (0..15) of row r inside a two-k-block SW128 region of `rows` rows
-__device__ __forceinline__ uint32_t sw128_off(int r, int c, int rows) {
-  return (uint32_t)((c >> 3) * rows * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
 template <int MODE>
@@ -569,39 +470,6 @@ static size_t score_smem_bytes(const ScoreShape& sh) {
   return 1024 + 2 * (size_t)sh.q_rows * 128 + 2 * kKStageBytes + 4 * kScoreMaxRows * sizeof(float) + 12 * sizeof(uint64_t) + 16;
 }
 
-// cuTensorMapEncodeTiled through the runtime's driver entry point lookup (libcuda is not linked)
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-  }
-  return fn;
-}
-
-// K as a rank-4 tensor (d, token, head, sequence) with the caller's strides; box = 64 columns x 128 tokens,
-// 128-byte swizzle, out-of-range tokens read as zero
-static int make_k_map(const ScoreArgs& a, CUtensorMap* map) {
-  EncodeTiledFn enc = encode_tiled_fn();
-  if (!enc) return CATEKV_ERR_CUDA;
-  if (((uintptr_t)a.k & 15) || (a.st * 2) % 16 || (a.sh * 2) % 16 || (a.sb * 2) % 16 || a.st <= 0) return CATEKV_ERR_UNSUPPORTED;
-  const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)a.n_max, (cuuint64_t)a.Hkv, (cuuint64_t)a.B};
-  const cuuint64_t strides[3] = {(cuuint64_t)a.st * 2, (cuuint64_t)(a.Hkv > 1 ? a.sh : a.st * a.n_max) * 2,
-                                 (cuuint64_t)(a.B > 1 ? a.sb : (a.Hkv > 1 ? a.sh * a.Hkv : a.st * a.n_max)) * 2};
-  const cuuint32_t box[4] = {64, (cuuint32_t)kKeyTile, 1, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<uint16_t*>(a.k), dims, strides, box, estr,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? CATEKV_OK : CATEKV_ERR_UNSUPPORTED;
-}
-
 // Test hook (catekv_test_expire_score_waits): launches left that run with an idle producer lane.
 static std::atomic<int> g_expire_launches{0};
 
@@ -640,19 +508,23 @@ int score_launch(const ScoreArgs& a0, ScoreMode out_mode, cudaStream_t stream) {
   if (a0.g_major && (a0.L_obs != 64 || out_mode != kScoreMatrix)) return CATEKV_ERR_UNSUPPORTED;
   const ScoreShape sh = score_shape(a0.G, a0.L_obs);
   CUtensorMap map;
-  int rc = make_k_map(a0, &map);
+  const KvTensor kt = {a0.k, a0.sb, a0.sh, a0.st, a0.B, a0.Hkv, a0.n_max};
+  int rc = make_kv_map(kt, &map);
   if (rc) return rc;
   if (out_mode == kScoreColsum && sh.NH > 1)  // two units per tile add their shares into a zeroed vector
     CATEKV_CUDA_TRY(cudaMemsetAsync(a0.out, 0, sizeof(float) * (size_t)a0.n_jobs * a0.out_job_stride, stream));
   // (Scoring the jobs in groups whose keys fit the L2 together, both passes of a group back to back, was measured
   // and lost: the smaller grids and extra launches cost more than the second pass gains from L2 hits.)
   ScoreArgs a = a0;
-  a.keys_per_cta = score_keys_per_cta(a.n_jobs, a.max_keys);
+  a.keys_per_cta = score_keys_per_cta(a.n_jobs_split > 0 ? a.n_jobs_split : a.n_jobs, a.max_keys);
   a.n_chunks = (a.max_keys + a.keys_per_cta - 1) / a.keys_per_cta;  // jobs * chunks <= score_max_ctas(jobs): fits the partials
-  rc = launch_one<kScoreStats>(a, sh, map, stream);
-  if (rc) return rc;
-  score_stats_merge_kernel<<<dim3((sh.R + 7) / 8, a.n_jobs), 256, 0, stream>>>(a, sh.R);
-  CATEKV_CUDA_TRY(cudaGetLastError());
+  if (!a.stats_given) {
+    rc = launch_one<kScoreStats>(a, sh, map, stream);
+    if (rc) return rc;
+    score_stats_merge_kernel<<<dim3((sh.R + 7) / 8, a.n_jobs), 256, 0, stream>>>(a, sh.R);
+    CATEKV_CUDA_TRY(cudaGetLastError());
+  }
+  if (out_mode == kScoreStats) return CATEKV_OK;  // the caller wants the row statistics only
   return out_mode == kScoreColsum ? launch_one<kScoreColsum>(a, sh, map, stream) : launch_one<kScoreMatrix>(a, sh, map, stream);
 }
 

@@ -22,6 +22,8 @@ struct ScoreArgs {
   int32_t B, Hkv, n_max;  // extents of k (sequences, KV heads, tokens) for the TMA descriptor
   float scale_log2;       // log2(e) / sqrt(d)
   int32_t max_keys;       // longest key range of any job
+  int32_t n_jobs_split;   // jobs the key ranges are cut for (0: n_jobs); smaller when some jobs are known to be tiny
+  int32_t stats_given;    // 1: `stats` already holds every row's (max, sum): the first pass and its merge are skipped
   int32_t keys_per_cta;   // multiple of 128 (set by score_launch, per group of jobs)
   int32_t n_chunks;       // grid.x: ceil(max key range / keys_per_cta) (set by score_launch)
   float2* stats_part;     // [n_jobs][n_chunks][kScoreMaxRows]  per-CTA (row max in the log2 domain, row sum)

@@ -344,6 +344,17 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
   }
 }
 
+// Row statistics from a given normaliser: stats[job][r] = (log-sum-exp of row r over the scored keys in the log2 domain,
+// 1), so that the second scoring pass computes exp2(logit - lse) directly.  Row r = i * G + g.
+__global__ void stats_from_lse_kernel(const ScoreJob* jobs, const float* lse, float2* stats, int R, int G, int L_obs, int Hq) {
+  const ScoreJob job = jobs[blockIdx.x];
+  for (int r = threadIdx.x; r < R; r += blockDim.x) {
+    const int i = r / G, g = r - i * G;
+    const float v = lse[((size_t)job.b * Hq + job.h * G + g) * L_obs + i];
+    stats[(size_t)blockIdx.x * kScoreMaxRows + r] = v > -INFINITY ? make_float2(v * 1.4426950408889634f, 1.f) : make_float2(-INFINITY, 0.f);
+  }
+}
+
 constexpr int kGatherRowsPerBlock = 64;
 
 // One warp per kept row: lanes 0-15 move the K row, lanes 16-31 the V row (16 bytes each).
@@ -582,6 +593,13 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
     sa.causal = 0;  // every scored key precedes every window query
     sa.scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
     sa.max_keys = n_sc_jobs_max;
+    if (p->row_lse_scored) {
+      // the prefill pass already knows every window row's normaliser over the scored keys: no first pass over K
+      stats_from_lse_kernel<<<(unsigned)jobs.size(), 128, 0, st>>>(d_jobs, p->row_lse_scored, (float2*)(w8 + W.off_stats),
+                                                                  G * p->L_obs, G, p->L_obs, p->Hq);
+      CATEKV_CUDA_TRY(cudaGetLastError());
+      sa.stats_given = 1;
+    }
     sa.stats_part = (float2*)(w8 + W.off_part);
     sa.stats = (float2*)(w8 + W.off_stats);
     sa.status = (int32_t*)(w8 + W.off_status);

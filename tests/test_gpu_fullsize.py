@@ -268,3 +268,29 @@ def test_cfg3_retrieval_in_place_as_the_bench_runs_it(ck):
         soc.k_rows[s], soc.v_rows[s] = krows[got], vrows[got]
     ref, ref_lse = orc.decode_attention(soc, synth.bits(q), cells=[divmod(s, w.Hkv) for s in cells])
     H.check_attention(out, None, lse, ref, ref_lse, "cfg3 retrieval in place")
+
+
+def test_cfg2_window_attention_and_selection_from_its_normaliser(ck):
+    # configs[2] shape (128K keys, 4 x 32 window rows per KV head): the prefill rows of the window, their normalisers,
+    # and catekv_select_compact fed with them instead of running its own first pass over K
+    w = synth.WORKLOADS["cfg2"]
+    p = synth.prefill_layer(w, 1, "cuda")
+    mask = p["head_mask"]
+    out, lse, lse_sc = ck.catekv_window_attn(p["q_win"], p["k"], p["v"], p["seq_len"])
+    out16, _, _ = ck.catekv_window_attn(p["q_win"], p["k"], p["v"], p["seq_len"], out_dtype=torch.bfloat16)
+    cells = _pick_cells(mask, 2)
+    qb = synth.bits(p["q_win"])
+    for (b, h) in cells:
+        kb, vb = synth.bits(p["k"][b, h]), synth.bits(p["v"][b, h])
+        sl = slice(h * w.G, (h + 1) * w.G)
+        ref, ref_lse = orc.window_attention(qb[b, sl], kb, vb, w.L_obs)
+        H.check_attention(out[b, sl].reshape(-1, w.d), out16[b, sl].reshape(-1, w.d), lse[b, sl].reshape(-1),
+                          ref.reshape(-1, w.d), ref_lse.reshape(-1), f"cfg2 window b{b} h{h}")
+        ref_sc = orc.scored_range_lse(qb[b, sl], kb, w.L_obs)
+        assert np.all(np.abs(lse_sc[b, sl].cpu().double().numpy() - ref_sc) <= 1e-3)
+    cache = ck.Cache(w.B, w.Hkv, bench.expected_lengths(w, mask), 8, "cuda")
+    idx = torch.full((w.B * w.Hkv, w.n), -1, dtype=torch.int32, device="cuda")
+    ck.catekv_select_compact(p["q_win"], p["k"], p["v"], p["seq_len"], mask, cache, w.budget, w.eta, w.sink, w.local,
+                             w.pool_mode, w.pool_param, idx_out=idx, row_lse_scored=lse_sc)
+    torch.cuda.synchronize()
+    _check_selection_cells(w, p, mask, cache, idx, cells)
