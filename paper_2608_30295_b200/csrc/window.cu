@@ -236,14 +236,14 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   if (*s_abort && tid == 0) raise_status(a.status, CATEKV_STATUS_WAIT_EXPIRED, kKidScore, (int)blockIdx.y, (int)blockIdx.x);
 }
 
-// Merge the statistics of the scored keys (job 2s) and of the window's own keys (job 2s + 1) of every row.
+// Merge the statistics of the scored keys (job s) and of the window's own keys (job n_segs + s) of every row.
 __global__ void window_stats_kernel(const float2* stats, const ScoreJob* jobs, int R, int G, int L_obs, int Hq, float* mfull,
                                     float* lse_out, float* lse_scored_out) {
   const int seg = blockIdx.x;
   const ScoreJob job = jobs[seg];
   const float ln2 = 0.6931471805599453f;
   for (int r = threadIdx.x; r < R; r += blockDim.x) {
-    const float2 sa = stats[(size_t)(2 * seg) * kScoreMaxRows + r], sb = stats[(size_t)(2 * seg + 1) * kScoreMaxRows + r];
+    const float2 sa = stats[(size_t)seg * kScoreMaxRows + r], sb = stats[(size_t)(gridDim.x + seg) * kScoreMaxRows + r];
     const float m = fmaxf(sa.x, sb.x);
     float l = 0.f;
     if (sa.y > 0.f) l += sa.y * exp2f(sa.x - m);
@@ -298,8 +298,9 @@ static WaWs wa_ws_layout(int n_segs, int G, int n_max, int L_obs) {
   WaWs w;
   const int R = G * L_obs;
   w.MT = (R + 127) / 128;
-  // key ranges: about one CTA per SM over all (segment, M tile) pairs, in whole tiles, at least four tiles each
-  int chunks = (sm_count() + n_segs * w.MT / 2) / (n_segs * w.MT);
+  // key ranges: at most one CTA per SM over all (segment, M tile) pairs (the kernel runs one CTA per SM: a grid
+  // just above the SM count would take two waves), in whole tiles, at least four tiles each
+  int chunks = sm_count() / (n_segs * w.MT);
   if (chunks < 1) chunks = 1;
   int kp = ((n_max + chunks - 1) / chunks + kKeyTile - 1) / kKeyTile * kKeyTile;
   if (kp < 4 * kKeyTile) kp = 4 * kKeyTile;
@@ -350,8 +351,9 @@ extern "C" int catekv_window_attn(const void* q_win, const void* k, const void* 
   for (int b = 0; b < B; ++b)
     for (int h = 0; h < Hkv; ++h) {
       const int s = b * Hkv + h, n = seq_len[b];
-      jobs2[2 * s] = ScoreJob{b, h, n, 0, n - L_obs, 0};      // the scored keys
-      jobs2[2 * s + 1] = ScoreJob{b, h, n, n - L_obs, n, 0};  // the window's own keys (causal)
+      // the scored jobs first: their CTAs fill the machine in one wave, the one-tile window jobs follow
+      jobs2[s] = ScoreJob{b, h, n, 0, n - L_obs, 0};           // the scored keys
+      jobs2[n_segs + s] = ScoreJob{b, h, n, n - L_obs, n, 0};  // the window's own keys (causal)
       jobs[s] = ScoreJob{b, h, n, 0, n, 0};
     }
   cudaStream_t st = (cudaStream_t)stream;

@@ -61,13 +61,22 @@ def bf16_tie_flips(got_bits, ref_bits, x_f32, ref_f64):
 
     True where (i) got and ref are adjacent bf16 values and (ii) x lies within TIE_DIST of their midpoint, with
     TIE_DIST = max |x_f32 - ref_f64| over the tensor (the measured fp32 error) + 4 fp32 ulps of x."""
+    return bf16_tie_analysis(got_bits, ref_bits, x_f32, ref_f64)[0]
+
+
+def bf16_tie_analysis(got_bits, ref_bits, x_f32, ref_f64):
+    """-> (mask of excused elements, number of such elements to expect).  An fp32 value falls within TIE_DIST of a
+    rounding midpoint with probability 2 TIE_DIST / ulp (ulp: the bf16 spacing at that magnitude) when it is spread
+    evenly between two bf16 neighbours; the sum of these probabilities is the expected count."""
     differ = np.asarray(got_bits) != np.asarray(ref_bits)
     adjacent = np.abs(_bf16_ordinal(got_bits) - _bf16_ordinal(ref_bits)) == 1
     mid = 0.5 * (orc.bf16_to_f64(got_bits) + orc.bf16_to_f64(ref_bits))
     x = np.asarray(x_f32, dtype=np.float64)
     err = float(np.max(np.abs(x - ref_f64))) if x.size else 0.0
     tie_dist = err + 4.0 * np.spacing(np.abs(x).astype(np.float32)).astype(np.float64)
-    return differ & adjacent & (np.abs(x - mid) <= tie_dist)
+    ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(np.asarray(ref_f64, dtype=np.float64)), 2.0 ** -126))) - 7)
+    expected = float(np.minimum(1.0, 2.0 * tie_dist / ulp).sum())
+    return differ & adjacent & (np.abs(x - mid) <= tie_dist), expected
 
 
 def check_attention(out_f32, out_bf16, lse, ref, ref_lse, where=""):
@@ -87,15 +96,16 @@ def check_attention(out_f32, out_bf16, lse, ref, ref_lse, where=""):
         # opposite sides of a rounding tie they round to the two neighbours: one bf16 ulp apart (2^-6 for |x| in
         # [2, 4), above the 1e-2 absolute bound).  Such an element is excused only when the cause shows: the two
         # values are adjacent bf16 numbers and the fp32 result lies within TIE_DIST of their midpoint, TIE_DIST =
-        # the largest fp32-against-oracle error measured on this tensor + 4 fp32 ulps.  Every other element keeps
-        # rel-L2 <= 1e-3 and max-abs <= 1e-2.
+        # the largest fp32-against-oracle error measured on this tensor + 4 fp32 ulps, and there may be no more of
+        # them than that distance explains.  Every other element keeps rel-L2 <= 1e-3 and max-abs <= 1e-2.
         gbits = synth.bits(out_bf16)[ok]
         rbits = orc.f64_to_bf16(r)
         g, rb = orc.bf16_to_f64(gbits), orc.bf16_to_f64(rbits)
         x = out_f32.detach().cpu().double().numpy()[ok]
-        tie = bf16_tie_flips(gbits, rbits, x, r)
+        tie, expected = bf16_tie_analysis(gbits, rbits, x, r)
         n_ties = int(tie.sum())
-        assert n_ties <= max(4, 0.005 * tie.size), (where, "too many rounding-tie flips to be chance", n_ties)
+        # no more such elements than chance explains: three times the expected count (+ 4 for small tensors)
+        assert n_ties <= 4 + 3.0 * expected, (where, "too many rounding-tie flips to be chance", n_ties, expected)
         g_chk = np.where(tie, rb, g)
         assert rel_l2(g_chk, rb) <= REL_L2, (where, "bf16 rel-L2", rel_l2(g_chk, rb), n_ties)
         assert max_abs(g_chk, rb) <= MAX_ABS, (where, "bf16 max-abs", max_abs(g_chk, rb), n_ties)
