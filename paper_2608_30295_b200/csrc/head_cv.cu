@@ -42,6 +42,7 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
   const int rank = (int)cluster.block_rank();
   const CvSeg s = a.segs[seg];
   __shared__ unsigned int hist[256];
+  __shared__ unsigned int hcopies[256 * kHistCopies];
   __shared__ unsigned int hsum[256];
   __shared__ unsigned int s_pair[2];
   __shared__ unsigned int s_mm[2];
@@ -95,7 +96,7 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
     const int shift = nb - wbits;
     const unsigned int dmask = (1u << wbits) - 1u;
     const unsigned int pmask = shift + wbits >= 32 ? 0u : (0xffffffffu << (shift + wbits));
-    if (tid < 256) hist[tid] = 0;
+    radix_hist_zero(hcopies);
     __syncthreads();
     for (int c0 = lo; c0 < hi; c0 += 4 * kCvThreads) {  // whole warps stay in the loop: the vote needs them
       unsigned int v[4];
@@ -114,12 +115,14 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
         int same;
         __match_all_sync(0xffffffffu, dgt, &same);
         if (same) {
-          if (hit && lane == 0) atomicAdd(&hist[dgt], 32u);
+          if (hit && lane == 0) radix_hist_add(hcopies, dgt, 32u);
         } else if (hit) {
-          atomicAdd(&hist[dgt], 1u);
+          radix_hist_add(hcopies, dgt, 1u);
         }
       }
     }
+    __syncthreads();
+    radix_hist_fold(hcopies, hist);
     cluster.sync();  // all histograms complete
     if (tid < 256) {
       unsigned int t = 0;

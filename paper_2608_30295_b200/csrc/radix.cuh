@@ -6,6 +6,26 @@
 
 namespace catekv {
 
+// The digit histograms are kept in kHistCopies interleaved copies (bin d of copy c at word d * kHistCopies + c), a lane
+// adds to copy lane % kHistCopies: in the first passes most entries share their top digits, and atomics on one
+// address serialise.  A CTA folds its copies into a plain 256-bin histogram before anybody reads it.
+constexpr int kHistCopies = 8;
+__device__ __forceinline__ void radix_hist_zero(unsigned int* hcopies) {
+  for (int i = threadIdx.x; i < 256 * kHistCopies; i += blockDim.x) hcopies[i] = 0;
+}
+__device__ __forceinline__ void radix_hist_add(unsigned int* hcopies, unsigned int digit, unsigned int count) {
+  atomicAdd(&hcopies[digit * kHistCopies + (threadIdx.x & (kHistCopies - 1))], count);
+}
+// threads 0..255: bin tid of the folded histogram
+__device__ __forceinline__ void radix_hist_fold(const unsigned int* hcopies, unsigned int* hist) {
+  if (threadIdx.x < 256) {
+    unsigned int t = 0;
+#pragma unroll
+    for (int c = 0; c < kHistCopies; ++c) t += hcopies[threadIdx.x * kHistCopies + c];
+    hist[threadIdx.x] = t;
+  }
+}
+
 // One warp picks the radix digit that holds the `need`-th largest entry from a 256-bin histogram `h` (bins of
 // larger digits first): lane L owns the 8 bins 255 - 8L .. 248 - 8L, a shuffle scan gives the count in the bins
 // above a lane's, and the lane whose bins reach `need` writes the extended prefix and what is still needed
