@@ -1,6 +1,7 @@
 // Head identification statistic (Section 3.2, Eq. 1-4): observation matrix, matrix-global
 // percentile threshold, per-column counts, coefficient of variation.
 #include <math.h>
+#include <string.h>
 
 #include <vector>
 
@@ -250,9 +251,13 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   }
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* w8 = (uint8_t*)ws;
-  CATEKV_CUDA_TRY(cudaMemsetAsync(w8 + W.off_status, 0, CATEKV_STATUS_BYTES, st));
-  CATEKV_CUDA_TRY(cudaMemcpyAsync(w8 + W.off_segs, segs.data(), sizeof(CvSeg) * n_segs, cudaMemcpyHostToDevice, st));
-  CATEKV_CUDA_TRY(cudaMemcpyAsync(w8 + W.off_jobs, jobs.data(), sizeof(ScoreJob) * n_segs, cudaMemcpyHostToDevice, st));
+  {
+    // one copy brings the cleared status block, the segment table and the job list (they are adjacent in the workspace)
+    std::vector<uint8_t> head(W.off_jobs + sizeof(ScoreJob) * (size_t)n_segs, 0);
+    memcpy(head.data() + W.off_segs, segs.data(), sizeof(CvSeg) * n_segs);
+    memcpy(head.data() + W.off_jobs, jobs.data(), sizeof(ScoreJob) * n_segs);
+    CATEKV_CUDA_TRY(cudaMemcpyAsync(w8, head.data(), head.size(), cudaMemcpyHostToDevice, st));
+  }
   ScoreArgs sa = {};
   sa.q_win = (const uint16_t*)q_win;
   sa.k = (const uint16_t*)k;

@@ -75,6 +75,12 @@ template <int MODE>
 __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_constant__ CUtensorMap k_map, const ScoreArgs a,
                                                               const ScoreShape sh) {
   extern __shared__ uint8_t smem_raw[];
+  // Programmatic dependent launch: the next kernel of the chain (merge, second pass, top-k) may be scheduled while
+  // this grid drains.  The first pass has nothing to wait for but its inputs, which a stream-ordered copy or a
+  // kernel that never signals early produced; the second pass sets up (queries, barriers, tensor memory) and then
+  // waits for the merged statistics.
+  pdl_launch_dependents();
+  if (MODE == kScoreStats) pdl_wait();
   const ScoreJob job = a.jobs[blockIdx.y];
   const int j_lo = job.j_begin + blockIdx.x * a.keys_per_cta;
   if (j_lo >= job.j_end) return;
@@ -126,6 +132,7 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
     }
   } else {
     // m'_r = m_r + log2(l_r): exp2(x - m'_r) is the normalised probability; rows without mass get +inf (-> 0)
+    pdl_wait();  // the statistics are the preceding kernel's output
     const float2* st = a.stats + (size_t)blockIdx.y * kScoreMaxRows;
     for (int r = tid; r < sh.R; r += kScThreads) {
       const float2 v = st[r];
@@ -442,6 +449,8 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
 
 // Merge the per-CTA row partials: stats[job][row] = (max, sum).  One warp per row.
 __global__ void __launch_bounds__(256) score_stats_merge_kernel(const ScoreArgs a, int R) {
+  pdl_launch_dependents();
+  pdl_wait();  // the partials are the preceding kernel's output
   const int jobi = blockIdx.y;
   const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -487,8 +496,7 @@ static int launch_one(const ScoreArgs& a0, const ScoreShape& sh, const CUtensorM
   }
   const size_t smem = score_smem_bytes(sh);
   CATEKV_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  score_tc_kernel<MODE><<<dim3(a.n_chunks, a.n_jobs), kScThreads, smem, stream>>>(map, a, sh);
-  CATEKV_CUDA_TRY(cudaGetLastError());
+  CATEKV_CUDA_TRY(launch_pdl(score_tc_kernel<MODE>, dim3(a.n_chunks, a.n_jobs), dim3(kScThreads), smem, stream, map, a, sh));
   return CATEKV_OK;
 }
 
@@ -521,8 +529,7 @@ int score_launch(const ScoreArgs& a0, ScoreMode out_mode, cudaStream_t stream) {
   if (!a.stats_given) {
     rc = launch_one<kScoreStats>(a, sh, map, stream);
     if (rc) return rc;
-    score_stats_merge_kernel<<<dim3((sh.R + 7) / 8, a.n_jobs), 256, 0, stream>>>(a, sh.R);
-    CATEKV_CUDA_TRY(cudaGetLastError());
+    CATEKV_CUDA_TRY(launch_pdl(score_stats_merge_kernel, dim3((sh.R + 7) / 8, a.n_jobs), dim3(256), 0, stream, a, sh.R));
   }
   if (out_mode == kScoreStats) return CATEKV_OK;  // the caller wants the row statistics only
   return out_mode == kScoreColsum ? launch_one<kScoreColsum>(a, sh, map, stream) : launch_one<kScoreMatrix>(a, sh, map, stream);

@@ -2,6 +2,7 @@
 // top-k with lowest-index tie-break -> ascending kept list -> gather of K/V rows into the
 // head's segment of the pool.
 #include <math.h>
+#include <string.h>
 
 #include <atomic>
 #include <vector>
@@ -572,10 +573,14 @@ extern "C" int catekv_select_compact(const catekv_select_params* p, catekv_cache
   uint8_t* w8 = (uint8_t*)ws;
   SelSeg* d_segs = (SelSeg*)(w8 + W.off_segs);
   ScoreJob* d_jobs = (ScoreJob*)(w8 + W.off_jobs);
-  CATEKV_CUDA_TRY(cudaMemsetAsync(w8 + W.off_status, 0, CATEKV_STATUS_BYTES, st));
-  CATEKV_CUDA_TRY(cudaMemcpyAsync(d_segs, segs.data(), sizeof(SelSeg) * n_segs, cudaMemcpyHostToDevice, st));
+  {
+    // one copy brings the cleared status block, the segment table and the job list (they are adjacent in the workspace)
+    std::vector<uint8_t> head(W.off_jobs + sizeof(ScoreJob) * jobs.size(), 0);
+    memcpy(head.data() + W.off_segs, segs.data(), sizeof(SelSeg) * n_segs);
+    if (!jobs.empty()) memcpy(head.data() + W.off_jobs, jobs.data(), sizeof(ScoreJob) * jobs.size());
+    CATEKV_CUDA_TRY(cudaMemcpyAsync(w8, head.data(), head.size(), cudaMemcpyHostToDevice, st));
+  }
   if (!jobs.empty()) {
-    CATEKV_CUDA_TRY(cudaMemcpyAsync(d_jobs, jobs.data(), sizeof(ScoreJob) * jobs.size(), cudaMemcpyHostToDevice, st));
     ScoreArgs sa = {};
     sa.q_win = (const uint16_t*)p->q_win;
     sa.k = (const uint16_t*)p->k;

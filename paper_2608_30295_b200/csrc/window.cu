@@ -19,6 +19,7 @@
 // 64 keys each).  Every mbarrier wait is bounded: on expiry the CTA raises the abort flag, frees its tensor memory,
 // records CATEKV_STATUS_WAIT_EXPIRED and returns.
 #include <math.h>
+#include <string.h>
 
 #include <atomic>
 #include <vector>
@@ -358,9 +359,13 @@ extern "C" int catekv_window_attn(const void* q_win, const void* k, const void* 
     }
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* w8 = (uint8_t*)ws;
-  CATEKV_CUDA_TRY(cudaMemsetAsync(w8 + W.off_status, 0, CATEKV_STATUS_BYTES, st));
-  CATEKV_CUDA_TRY(cudaMemcpyAsync(w8 + W.off_jobs2, jobs2.data(), sizeof(ScoreJob) * jobs2.size(), cudaMemcpyHostToDevice, st));
-  CATEKV_CUDA_TRY(cudaMemcpyAsync(w8 + W.off_jobs, jobs.data(), sizeof(ScoreJob) * jobs.size(), cudaMemcpyHostToDevice, st));
+  {
+    // one copy brings the cleared status block and both job lists (they are adjacent in the workspace)
+    std::vector<uint8_t> head(W.off_jobs + sizeof(ScoreJob) * jobs.size(), 0);
+    memcpy(head.data() + W.off_jobs2, jobs2.data(), sizeof(ScoreJob) * jobs2.size());
+    memcpy(head.data() + W.off_jobs, jobs.data(), sizeof(ScoreJob) * jobs.size());
+    CATEKV_CUDA_TRY(cudaMemcpyAsync(w8, head.data(), head.size(), cudaMemcpyHostToDevice, st));
+  }
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
   ScoreArgs sa = {};
   sa.q_win = (const uint16_t*)q_win;
