@@ -421,8 +421,8 @@ def time_window_attn(ck, w, dev, layer=0, reps=5):
     res["select_with_normaliser_ms"] = timed(lambda: sel(lse_sc[0]))
     kv_bytes = w.B * w.Hkv * w.n * 256
     res["k_bytes"] = kv_bytes
-    res["hbm_bytes_window_attn"] = 3 * kv_bytes  # K twice (normalisers, P V), V once
-    res["flops_window_attn"] = 2.0 * w.B * w.Hq * w.L_obs * w.n * w.d * 4  # Q K^T twice, P_hi V, P_lo V
+    res["hbm_bytes_window_attn"] = 2 * kv_bytes * ((w.G * w.L_obs + 127) // 128)  # K and V once per 128-row tile of the window
+    res["flops_window_attn"] = 2.0 * w.B * w.Hq * w.L_obs * w.n * w.d * 3  # Q K^T, P_hi V, P_lo V
     return res
 
 

@@ -283,7 +283,7 @@ int catekv_select_compact(const catekv_select_params* p, catekv_cache* cache, in
  *   lse_out, lse_scored_out device float [B, Hq, L_obs] or NULL (-inf where a row has no key)
  *   ws device scratch of at least catekv_window_attn_workspace_bytes(...); its first CATEKV_STATUS_BYTES are the
  *   status block (cleared by this call).
- * K is read twice (row normalisers, then P V), V once.
+ * One sweep: K and V are each read once.
  */
 size_t catekv_window_attn_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t n_max, int32_t L_obs);
 int catekv_window_attn(const void* q_win, const void* k, const void* v, int64_t kv_stride_b, int64_t kv_stride_h,

@@ -3,21 +3,22 @@
 // their log-sum-exp and the log-sum-exp over the scored keys [0, n - L_obs) alone, which is the softmax normaliser
 // of the token-criticality line.  catekv_select_compact takes the latter in place of its own first pass over K.
 //
-//   1. row statistics (score_tc_kernel, statistics mode): two jobs per (sequence, KV head), the scored keys
-//      [0, n - L_obs) and the window's own keys [n - L_obs, n) under the causal mask;
-//   2. window_stats_kernel merges the two into the causal normaliser of every row and writes both log-sum-exps;
-//   3. window_pv_kernel: O[rows x d] = sum over key tiles of P V with P = exp2(logit - normaliser) already final,
-//      so the accumulator in tensor memory is never rescaled.  Per key tile: S = Q K^T (tcgen05.mma, accumulator
-//      slot in TMEM), the epilogue warps turn S into P and write it to shared memory as a bf16 hi + lo pair in the
-//      K-major SWIZZLE_128B operand layout, and two more chains of tcgen05.mma add P_hi V and P_lo V (V as the
-//      MN-major B operand, straight from the TMA tile) to O in TMEM.  A CTA owns a range of keys of one
-//      (sequence, KV head) and 128 query rows; the ranges' partial outputs are summed in a fixed order by
-//   4. window_reduce_kernel, which also converts to the output type.
+// One sweep over K and V.  window_pv_kernel: a CTA owns a range of keys of one (sequence, KV head) and 128 query
+// rows.  Per 128-key tile: S = Q K^T (tcgen05.mma into one of two TMEM slots); an epilogue thread owns a query row,
+// finds the tile's maximum, turns S into P = exp2(logit - ref) against the row's reference value, adds the row sums
+// (all visible keys; scored keys only) and writes P to shared memory as a bf16 hi + lo pair in the K-major
+// SWIZZLE_128B operand layout; two more chains of tcgen05.mma add P_hi V and P_lo V (V as the MN-major B operand,
+// straight from the TMA tile) to O in TMEM.  The reference only moves when a tile's maximum exceeds it by more than
+// 2^8 (P stays below 256, far inside what bf16 hi + lo and the fp32 accumulator carry); then the row's O is read from
+// TMEM, scaled and stored back before the tile's P V is issued.  The ranges' partial results (O, reference, sums)
+// are merged in range order by window_reduce_kernel, which also writes the two log-sum-exps.
 //
-// Warp roles of window_pv_kernel: warp 9 (one lane) feeds the K and V stages by TMA; warp 8 (one lane) issues
-// every MMA, the S of tile t + 1 before the P V of tile t; warps 0-7 are the epilogue (two per TMEM lane quarter,
-// 64 keys each).  Every mbarrier wait is bounded: on expiry the CTA raises the abort flag, frees its tensor memory,
-// records CATEKV_STATUS_WAIT_EXPIRED and returns.
+// Warp roles: warp 9 (one lane) feeds the K and V stages by TMA; warp 8 (one lane) issues every MMA, the S of tile
+// t + 1 before the P V of tile t; warps 0-7 are the epilogue (two per TMEM lane quarter, 64 keys and 64 columns of
+// O each); the two threads of a row exchange their half-tile maxima through shared memory (a named barrier per
+// pair of warps) and so keep the same reference.  Every mbarrier
+// wait is bounded: on expiry the CTA raises the abort flag, frees its tensor memory, records
+// CATEKV_STATUS_WAIT_EXPIRED and returns.
 #include <math.h>
 #include <string.h>
 
@@ -33,15 +34,18 @@ constexpr int kWaThreads = 320;
 constexpr int kWaTmemCols = 512;       // S slots at columns 0 and 128, O at 256
 constexpr int kWaOCol = 256;
 constexpr int kWaTileBytes = 128 * 256;  // a [128 x 128] bf16 tile: Q rows, a K or V stage, P hi, P lo
+constexpr int kWaStateWords = 5;         // per row and key range: reference, sum (visible keys) x 2 halves, sum (scored keys) x 2 halves
+constexpr float kWaTau = 8.f;            // a row's reference follows a tile maximum that exceeds it by more than 2^kWaTau
 
 struct WinArgs {
   const uint16_t* q_win;  // [B, Hq, L_obs, d]
   const ScoreJob* jobs;   // [n_segs]: b, h, n (j_begin / j_end unused)
-  const float* mfull;     // [n_segs][kScoreMaxRows]: log2-domain causal normaliser of every row; +inf: the row has no mass
   int32_t G, L_obs, R, Hq;
   float scale_log2;
   int32_t keys_per_cta, n_chunks;
-  float* part;            // [n_segs][MT][n_chunks][128 rows][128 d]
+  float* part;            // [n_segs][MT][n_chunks][128 rows][128 d]: O relative to the range's reference
+  float* part_s;          // [n_segs][MT][n_chunks][kWaStateWords][128 rows]: reference (log2 domain), the two half-threads'
+                          //                                       sums over the visible keys, over the scored keys
   int32_t* status;
   uint32_t spin_limit;
 };
@@ -65,8 +69,8 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   const uint32_t s_v = s_k + 2 * kWaTileBytes;
   const uint32_t s_ph = s_v + 2 * kWaTileBytes;
   const uint32_t s_pl = s_ph + kWaTileBytes;
-  float* s_m = reinterpret_cast<float*>(smem + 7 * kWaTileBytes);
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_m + 128);
+  float* s_xch = reinterpret_cast<float*>(smem + 7 * kWaTileBytes);  // [2 halves][128 rows]: half-tile maxima
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_xch + 256);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 16);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   const uint32_t bar0 = smem_u32(s_bar);
@@ -84,10 +88,6 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
     cp_async16(s_q + sw128_off(row, c, 128), src, ok);
   }
   cp_async_commit();
-  for (int row = tid; row < 128; row += kWaThreads) {
-    const int r = mt * 128 + row;
-    s_m[row] = r < a.R ? a.mfull[(size_t)blockIdx.y * kScoreMaxRows + r] : INFINITY;
-  }
   if (tid == 0) {
     *s_abort = 0;
     for (int i = 0; i < 15; ++i) {
@@ -173,11 +173,15 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   } else {
     // ================= epilogue warps =================
     const int lane_row = (warp & 3) * 32 + lane;  // this thread's TMEM lane = its query row of the M tile
-    const int half = warp >> 2;                   // keys [64 * half, 64 * half + 64) of every tile
+    const int half = warp >> 2;                   // keys [64 * half, 64 * half + 64) of every tile, d [64 * half, ...) of O
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const int r = mt * 128 + lane_row;
-    const int pos = n - a.L_obs + (r < a.R ? r / a.G : 0);  // the row's own position: it sees keys j <= pos
-    const float mr = s_m[lane_row];
+    const bool row_ok = r < a.R;
+    const int pos = n - a.L_obs + (row_ok ? r / a.G : 0);  // the row's own position: it sees keys j <= pos
+    const int n_sc = n - a.L_obs;                           // keys below are scored keys
+    // The two threads of a row (warps w and w + 4) keep the same reference: each tile they exchange the maxima of
+    // their halves through shared memory and take the same decision.  The sums stay per thread.
+    float ref = -INFINITY, l = 0.f, lsc = 0.f;
     bool alive = true;
     for (int t = 0; t < n_tiles; ++t) {
       const int st = t & 1;
@@ -190,41 +194,103 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_free_s + 8 * st);  // the S slot goes back to the MMA warp
       const int jb = j_lo + t * kKeyTile + half * 64;   // key of x[0]
-      const bool edge = jb + 63 > n - a.L_obs;          // uniform: some key of the block may be masked for some row
+      const bool edge = jb + 63 >= n_sc;                // uniform: the block reaches the window's own keys (or the end)
+      if (edge) {
 #pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        float p = fast_exp2(fmaf(x[c], a.scale_log2, -mr));
-        if (edge) p = (jb + c <= pos) ? p : 0.f;
-        x[c] = p;
+        for (int c = 0; c < 64; ++c) x[c] = (jb + c <= pos) ? x[c] : -INFINITY;
       }
-      // P of the previous tile must have been consumed before this one overwrites it
-      if (t >= 1 && !mbar_wait(bar_p_free, (uint32_t)((t - 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
+      // ---- the tile's maximum over the keys this row sees: this half, then the partner's through shared memory
+      float m0 = fmax3(x[0], x[1], x[2]), m1 = fmax3(x[3], x[4], x[5]);
+      float m2 = fmax3(x[6], x[7], x[8]), m3 = fmax3(x[9], x[10], x[11]);
 #pragma unroll
-      for (int c = 0; c < 64; c += 8) {
-        uint32_t hi[4], lo[4];
+      for (int c = 12; c < 60; c += 8) {
+        m0 = fmax3(m0, x[c], x[c + 1]);
+        m1 = fmax3(m1, x[c + 2], x[c + 3]);
+        m2 = fmax3(m2, x[c + 4], x[c + 5]);
+        m3 = fmax3(m3, x[c + 6], x[c + 7]);
+      }
+      m0 = fmax3(m0, x[60], x[61]);
+      m1 = fmax3(m1, x[62], x[63]);
+      float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+      s_xch[half * 128 + lane_row] = mx;
+      asm volatile("bar.sync %0, 64;\n" ::"r"(1 + (warp & 3)) : "memory");  // the two warps of this lane quarter
+      mx = fmaxf(mx, s_xch[(half ^ 1) * 128 + lane_row]);
+      asm volatile("bar.sync %0, 64;\n" ::"r"(1 + (warp & 3)) : "memory");  // both have read: the slots may be rewritten
+      mx = row_ok ? mx * a.scale_log2 : -INFINITY;  // the scale is positive: the max commutes with it
+      const bool grow = mx > ref + kWaTau;  // also the first tile with a visible key (ref = -inf)
+      const float nref = grow ? mx : ref;
+      const bool rescale = grow && ref > -INFINITY;
+      const float factor = rescale ? fast_exp2(ref - nref) : 1.f;
+      ref = nref;
+      // ---- P = exp2(logit - reference) (masked entries are -inf -> 0), its row sums, the hi + lo operand tiles
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, ssc = 0.f;
+#pragma unroll
+      for (int c = 0; c < 64; c += 4) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const float h0 = bf16_round(x[c + 2 * e]), h1 = bf16_round(x[c + 2 * e + 1]);
-          hi[e] = pack_bf16(h0, h1);
-          lo[e] = pack_bf16(x[c + 2 * e] - h0, x[c + 2 * e + 1] - h1);
+          const float p = ref > -INFINITY ? fast_exp2(fmaf(x[c + e], a.scale_log2, -ref)) : 0.f;
+          if (edge) ssc += (jb + c + e < n_sc) ? p : 0.f;
+          x[c + e] = p;
         }
+        s0 += x[c];
+        s1 += x[c + 1];
+        s2 += x[c + 2];
+        s3 += x[c + 3];
+      }
+      const float sum = (s0 + s1) + (s2 + s3);
+      l = l * factor + sum;
+      lsc = lsc * factor + (edge ? ssc : sum);
+      uint32_t ph[32], pl[32];  // the probabilities as bf16 hi + lo pairs
+#pragma unroll
+      for (int c = 0; c < 64; c += 2) {
+        // hi = the upper 16 bits (a byte permute, no conversion; p - hi is exact in fp32), lo = p - hi rounded to bf16:
+        // hi + lo carries 16 significant bits of p.  Conversions share the special-function pipe with the
+        // exponentials, so only the lo half uses one.
+        const uint32_t b0 = __float_as_uint(x[c]), b1 = __float_as_uint(x[c + 1]);
+        ph[c / 2] = __byte_perm(b0, b1, 0x7632);
+        pl[c / 2] = pack_bf16(x[c] - __uint_as_float(b0 & 0xffff0000u), x[c + 1] - __uint_as_float(b1 & 0xffff0000u));
+      }
+      // All of the above ran under the previous tile's P V; that must have completed before O is touched and the
+      // P buffer rewritten
+      if (t >= 1 && !mbar_wait(bar_p_free, (uint32_t)((t - 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
+      if (__any_sync(0xffffffffu, rescale)) {  // this thread's 64 columns of its row of O
+        tc_fence_after();
+#pragma unroll 1
+        for (int c0 = 0; c0 < 64; c0 += 32) {
+          float o[32];
+          tmem_ld32(tmem + lane_base + (uint32_t)(kWaOCol + half * 64 + c0), o);
+          tmem_wait_ld32(o);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] *= factor;
+          tmem_st32(tmem + lane_base + (uint32_t)(kWaOCol + half * 64 + c0), o);
+        }
+        tmem_wait_st();
+      }
+#pragma unroll
+      for (int c = 0; c < 64; c += 8) {
         const uint32_t off = sw128_off(lane_row, half * 8 + (c >> 3), 128);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(s_ph + off), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(s_pl + off), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(s_ph + off), "r"(ph[c / 2]), "r"(ph[c / 2 + 1]), "r"(ph[c / 2 + 2]), "r"(ph[c / 2 + 3]) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(s_pl + off), "r"(pl[c / 2]), "r"(pl[c / 2 + 1]), "r"(pl[c / 2 + 2]), "r"(pl[c / 2 + 3]) : "memory");
       }
       fence_async_smem();  // generic-proxy writes of P before the async-proxy reads of the MMAs
+      tc_fence_before();   // the rescaled O before the MMAs that accumulate into it
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_p_ready);
+      if (lane == 0) mbar_arrive(bar_p_ready);  // the MMA warp may issue this tile's P V
     }
-    // ---- the CTA's partial output: this thread's row, 64 of the 128 d
+    // ---- the CTA's partial result: this thread's row, 64 of the 128 d, and its share of the row's state
     if (alive && mbar_wait(bar_done_o, 0u, s_abort, a.spin_limit)) {
       tc_fence_after();
       float o[64];
       tmem_ld64(tmem + lane_base + (uint32_t)(kWaOCol + half * 64), o);
       tmem_wait_ld64(o);
-      float* dst = a.part + ((((size_t)blockIdx.y * gridDim.z + mt) * a.n_chunks + blockIdx.x) * 128 + lane_row) * 128 + half * 64;
+      const size_t cta = ((size_t)blockIdx.y * gridDim.z + mt) * a.n_chunks + blockIdx.x;
+      float* dst = a.part + (cta * 128 + lane_row) * 128 + half * 64;
 #pragma unroll
       for (int c = 0; c < 64; c += 4) *reinterpret_cast<float4*>(dst + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+      float* ds = a.part_s + cta * (kWaStateWords * 128);
+      if (half == 0) ds[lane_row] = ref;
+      ds[(1 + half) * 128 + lane_row] = l;
+      ds[(3 + half) * 128 + lane_row] = lsc;
     }
   }
 
@@ -237,30 +303,12 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   if (*s_abort && tid == 0) raise_status(a.status, CATEKV_STATUS_WAIT_EXPIRED, kKidScore, (int)blockIdx.y, (int)blockIdx.x);
 }
 
-// Merge the statistics of the scored keys (job s) and of the window's own keys (job n_segs + s) of every row.
-__global__ void window_stats_kernel(const float2* stats, const ScoreJob* jobs, int R, int G, int L_obs, int Hq, float* mfull,
-                                    float* lse_out, float* lse_scored_out) {
-  const int seg = blockIdx.x;
-  const ScoreJob job = jobs[seg];
-  const float ln2 = 0.6931471805599453f;
-  for (int r = threadIdx.x; r < R; r += blockDim.x) {
-    const float2 sa = stats[(size_t)seg * kScoreMaxRows + r], sb = stats[(size_t)(gridDim.x + seg) * kScoreMaxRows + r];
-    const float m = fmaxf(sa.x, sb.x);
-    float l = 0.f;
-    if (sa.y > 0.f) l += sa.y * exp2f(sa.x - m);
-    if (sb.y > 0.f) l += sb.y * exp2f(sb.x - m);
-    const float full = l > 0.f ? m + log2f(l) : INFINITY;
-    mfull[(size_t)seg * kScoreMaxRows + r] = full;
-    const int i = r / G, g = r - i * G;
-    const size_t o = ((size_t)job.b * Hq + job.h * G + g) * L_obs + i;
-    if (lse_out) lse_out[o] = l > 0.f ? full * ln2 : -INFINITY;
-    if (lse_scored_out) lse_scored_out[o] = sa.y > 0.f ? (sa.x + log2f(sa.y)) * ln2 : -INFINITY;
-  }
-}
-
-// Sum the partial outputs of a (sequence, KV head)'s key ranges in range order; one warp per query row.
-__global__ void __launch_bounds__(128) window_reduce_kernel(const float* part, const ScoreJob* jobs, int keys_per_cta, int n_chunks,
-                                                            int MT, int R, int G, int L_obs, int Hq, void* out, int out_fp32) {
+// Merge the partial results of a (sequence, KV head)'s key ranges in range order: out = sum_c 2^(ref_c - M) O_c /
+// sum_c 2^(ref_c - M) l_c with M the largest reference; the same weights give the two log-sum-exps.  One warp per
+// query row; a lane owns four d.
+__global__ void __launch_bounds__(128) window_reduce_kernel(const float* part, const float* part_s, const ScoreJob* jobs,
+                                                            int keys_per_cta, int n_chunks, int MT, int R, int G, int L_obs, int Hq,
+                                                            void* out, int out_fp32, float* lse_out, float* lse_scored_out) {
   const int seg = blockIdx.y;
   const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -268,17 +316,34 @@ __global__ void __launch_bounds__(128) window_reduce_kernel(const float* part, c
   const ScoreJob job = jobs[seg];
   const int used = (job.n + keys_per_cta - 1) / keys_per_cta;
   const int mt = r >> 7, row = r & 127;
-  const float* p = part + ((((size_t)seg * MT + mt) * n_chunks) * 128 + row) * 128 + lane * 4;
+  const size_t cta0 = ((size_t)seg * MT + mt) * n_chunks;
+  const float* ps = part_s + cta0 * (kWaStateWords * 128) + row;
+  constexpr size_t kStep = (size_t)kWaStateWords * 128;  // words from one range's state to the next
+  float M = -INFINITY;
+  for (int c = 0; c < used; ++c) M = fmaxf(M, ps[c * kStep]);
+  const float* p = part + (cta0 * 128 + row) * 128 + lane * 4;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float L = 0.f, Lsc = 0.f;
   for (int c = 0; c < used; ++c) {
+    const float ref = ps[c * kStep];
+    if (ref == -INFINITY) continue;  // the row saw none of this range's keys
+    const float w = exp2f(ref - M);
     const float4 v = *reinterpret_cast<const float4*>(p + (size_t)c * 128 * 128);
-    acc.x += v.x;
-    acc.y += v.y;
-    acc.z += v.z;
-    acc.w += v.w;
+    acc.x += w * v.x;
+    acc.y += w * v.y;
+    acc.z += w * v.z;
+    acc.w += w * v.w;
+    L += w * (ps[c * kStep + 128] + ps[c * kStep + 256]);
+    Lsc += w * (ps[c * kStep + 384] + ps[c * kStep + 512]);
   }
+  const float inv = L > 0.f ? 1.f / L : 0.f;
+  acc.x *= inv;
+  acc.y *= inv;
+  acc.z *= inv;
+  acc.w *= inv;
   const int i = r / G, g = r - i * G;
-  const size_t o = (((size_t)job.b * Hq + job.h * G + g) * L_obs + i) * kD + lane * 4;
+  const size_t orow = ((size_t)job.b * Hq + job.h * G + g) * L_obs + i;
+  const size_t o = orow * kD + lane * 4;
   if (out_fp32) {
     *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + o) = acc;
   } else {
@@ -287,12 +352,18 @@ __global__ void __launch_bounds__(128) window_reduce_kernel(const float* part, c
     pk.y = pack_bf16(acc.z, acc.w);
     *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(out) + o) = pk;
   }
+  if (lane == 0) {
+    const float ln2 = 0.6931471805599453f;
+    if (lse_out) lse_out[orow] = L > 0.f ? (M + log2f(L)) * ln2 : -INFINITY;
+    if (lse_scored_out) lse_scored_out[orow] = Lsc > 0.f ? (M + log2f(Lsc)) * ln2 : -INFINITY;
+  }
 }
 
-constexpr size_t kWaSmemBytes = 1024 + 7 * (size_t)kWaTileBytes + 128 * sizeof(float) + 16 * sizeof(uint64_t) + 16;
+constexpr size_t kWaSmemBytes = 1024 + 7 * (size_t)kWaTileBytes + 256 * sizeof(float) + 16 * sizeof(uint64_t) + 16;
+static_assert(kWaSmemBytes <= 227 * 1024, "window_pv_kernel: one CTA's shared memory");
 
 struct WaWs {
-  size_t off_status, off_jobs2, off_jobs, off_part_stats, off_stats, off_mfull, off_part, bytes;
+  size_t off_status, off_jobs, off_part, off_part_s, bytes;
   int keys_per_cta, n_chunks, MT;
 };
 static WaWs wa_ws_layout(int n_segs, int G, int n_max, int L_obs) {
@@ -307,14 +378,12 @@ static WaWs wa_ws_layout(int n_segs, int G, int n_max, int L_obs) {
   if (kp < 4 * kKeyTile) kp = 4 * kKeyTile;
   w.keys_per_cta = kp;
   w.n_chunks = (n_max + kp - 1) / kp;
+  const size_t ctas = (size_t)n_segs * w.MT * w.n_chunks;
   size_t o = 0;
   w.off_status = o; o = CATEKV_STATUS_BYTES;
-  w.off_jobs2 = o; o = align_up(o + sizeof(ScoreJob) * (size_t)(2 * n_segs), 256);
   w.off_jobs = o; o = align_up(o + sizeof(ScoreJob) * (size_t)n_segs, 256);
-  w.off_part_stats = o; o = align_up(o + sizeof(float2) * (size_t)score_max_ctas(2 * n_segs) * 2 * kScoreMaxRows, 256);
-  w.off_stats = o; o = align_up(o + sizeof(float2) * (size_t)(2 * n_segs) * kScoreMaxRows, 256);
-  w.off_mfull = o; o = align_up(o + sizeof(float) * (size_t)n_segs * kScoreMaxRows, 256);
-  w.off_part = o; o = align_up(o + sizeof(float) * (size_t)n_segs * w.MT * w.n_chunks * 128 * 128, 256);
+  w.off_part = o; o = align_up(o + sizeof(float) * ctas * 128 * 128, 256);
+  w.off_part_s = o; o = align_up(o + sizeof(float) * ctas * kWaStateWords * 128, 256);
   w.bytes = o;
   return w;
 }
@@ -348,54 +417,20 @@ extern "C" int catekv_window_attn(const void* q_win, const void* k, const void* 
   const WaWs W = wa_ws_layout(n_segs, G, n_max, L_obs);
   if (ws_bytes < W.bytes) return CATEKV_ERR_WORKSPACE;
 
-  std::vector<ScoreJob> jobs2(2 * n_segs), jobs(n_segs);
+  std::vector<ScoreJob> jobs(n_segs);
   for (int b = 0; b < B; ++b)
-    for (int h = 0; h < Hkv; ++h) {
-      const int s = b * Hkv + h, n = seq_len[b];
-      // the scored jobs first: their CTAs fill the machine in one wave, the one-tile window jobs follow
-      jobs2[s] = ScoreJob{b, h, n, 0, n - L_obs, 0};           // the scored keys
-      jobs2[n_segs + s] = ScoreJob{b, h, n, n - L_obs, n, 0};  // the window's own keys (causal)
-      jobs[s] = ScoreJob{b, h, n, 0, n, 0};
-    }
+    for (int h = 0; h < Hkv; ++h) jobs[b * Hkv + h] = ScoreJob{b, h, seq_len[b], 0, seq_len[b], 0};
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* w8 = (uint8_t*)ws;
   {
-    // one copy brings the cleared status block and both job lists (they are adjacent in the workspace)
+    // one copy brings the cleared status block and the job list (they are adjacent in the workspace)
     std::vector<uint8_t> head(W.off_jobs + sizeof(ScoreJob) * jobs.size(), 0);
-    memcpy(head.data() + W.off_jobs2, jobs2.data(), sizeof(ScoreJob) * jobs2.size());
     memcpy(head.data() + W.off_jobs, jobs.data(), sizeof(ScoreJob) * jobs.size());
     CATEKV_CUDA_TRY(cudaMemcpyAsync(w8, head.data(), head.size(), cudaMemcpyHostToDevice, st));
   }
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
-  ScoreArgs sa = {};
-  sa.q_win = (const uint16_t*)q_win;
-  sa.k = (const uint16_t*)k;
-  sa.sb = kv_stride_b;
-  sa.sh = kv_stride_h;
-  sa.st = kv_stride_t;
-  sa.jobs = (const ScoreJob*)(w8 + W.off_jobs2);
-  sa.n_jobs = 2 * n_segs;
-  sa.n_jobs_split = n_segs;  // the window jobs are one CTA each: the key ranges are cut for the scored jobs alone
-  sa.Hq = Hq;
-  sa.B = B;
-  sa.Hkv = Hkv;
-  sa.n_max = n_max;
-  sa.G = G;
-  sa.L_obs = L_obs;
-  sa.causal = 1;
-  sa.scale_log2 = scale_log2;
-  sa.max_keys = n_max > L_obs ? n_max - L_obs : L_obs;
-  if (sa.max_keys < L_obs) sa.max_keys = L_obs;
-  sa.stats_part = (float2*)(w8 + W.off_part_stats);
-  sa.stats = (float2*)(w8 + W.off_stats);
-  sa.status = (int32_t*)(w8 + W.off_status);
-  int rc = score_launch(sa, kScoreStats, st);
-  if (rc) return rc;
   const int R = G * L_obs;
-  float* mfull = (float*)(w8 + W.off_mfull);
-  window_stats_kernel<<<n_segs, 128, 0, st>>>(sa.stats, (const ScoreJob*)(w8 + W.off_jobs), R, G, L_obs, Hq, mfull, lse_out,
-                                              lse_scored_out);
-  CATEKV_CUDA_TRY(cudaGetLastError());
+  int rc;
 
   CUtensorMap k_map, v_map;
   const KvTensor kt = {(const uint16_t*)k, kv_stride_b, kv_stride_h, kv_stride_t, B, Hkv, n_max};
@@ -414,7 +449,6 @@ extern "C" int catekv_window_attn(const void* q_win, const void* k, const void* 
   WinArgs wa = {};
   wa.q_win = (const uint16_t*)q_win;
   wa.jobs = (const ScoreJob*)(w8 + W.off_jobs);
-  wa.mfull = mfull;
   wa.G = G;
   wa.L_obs = L_obs;
   wa.R = R;
@@ -423,12 +457,14 @@ extern "C" int catekv_window_attn(const void* q_win, const void* k, const void* 
   wa.keys_per_cta = W.keys_per_cta;
   wa.n_chunks = W.n_chunks;
   wa.part = (float*)(w8 + W.off_part);
+  wa.part_s = (float*)(w8 + W.off_part_s);
   wa.status = (int32_t*)(w8 + W.off_status);
   wa.spin_limit = kSpinLimit;
   window_pv_kernel<<<dim3(W.n_chunks, n_segs, W.MT), kWaThreads, kWaSmemBytes, st>>>(k_map, v_map, wa);
   CATEKV_CUDA_TRY(cudaGetLastError());
-  window_reduce_kernel<<<dim3((R + 3) / 4, n_segs), 128, 0, st>>>(wa.part, wa.jobs, W.keys_per_cta, W.n_chunks, W.MT, R, G, L_obs,
-                                                                  Hq, out, out_dtype == CATEKV_OUT_FP32);
+  window_reduce_kernel<<<dim3((R + 3) / 4, n_segs), 128, 0, st>>>(wa.part, wa.part_s, wa.jobs, W.keys_per_cta, W.n_chunks, W.MT, R,
+                                                                  G, L_obs, Hq, out, out_dtype == CATEKV_OUT_FP32, lse_out,
+                                                                  lse_scored_out);
   CATEKV_CUDA_TRY(cudaGetLastError());
   return CATEKV_OK;
 }
