@@ -30,6 +30,10 @@ struct CvArgs {
 
 constexpr int kCvThreads = 1024;
 constexpr int kCvCluster = 8;
+#ifndef CATEKV_CV_UNROLL
+#define CATEKV_CV_UNROLL 16
+#endif
+constexpr int kCvUnroll = CATEKV_CV_UNROLL;  // loads a thread keeps in flight in the sweeps over its share of the matrix
 
 // One thread-block cluster of 8 CTAs per (sequence, KV head): Phi = alpha * percentile element (Eq. 2),
 // C_j = #{i: A_ij >= Phi} (Eq. 3), cv = std_pop(C) / mean(C) (Eq. 4) from exact integer sums.
@@ -59,12 +63,12 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
 
   // ---- extremes of the bit patterns
   unsigned int vmin = 0xffffffffu, vmax = 0u;
-  for (int c0 = lo + tid; c0 < hi; c0 += 4 * kCvThreads) {  // four loads in flight
-    unsigned int v[4];
+  for (int c0 = lo + tid; c0 < hi; c0 += kCvUnroll * kCvThreads) {  // several loads in flight
+    unsigned int v[kCvUnroll];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) v[e] = (c0 + e * kCvThreads < hi) ? Ab[c0 + e * kCvThreads] : 0u;
+    for (int e = 0; e < kCvUnroll; ++e) v[e] = (c0 + e * kCvThreads < hi) ? Ab[c0 + e * kCvThreads] : 0u;
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
+    for (int e = 0; e < kCvUnroll; ++e)
       if (c0 + e * kCvThreads < hi) {
         vmin = min(vmin, v[e]);
         vmax = max(vmax, v[e]);
@@ -99,17 +103,17 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
     const unsigned int pmask = shift + wbits >= 32 ? 0u : (0xffffffffu << (shift + wbits));
     radix_hist_zero(hcopies);
     __syncthreads();
-    for (int c0 = lo; c0 < hi; c0 += 4 * kCvThreads) {  // whole warps stay in the loop: the vote needs them
-      unsigned int v[4];
-      bool in[4];
+    for (int c0 = lo; c0 < hi; c0 += kCvUnroll * kCvThreads) {  // whole warps stay in the loop: the vote needs them
+      unsigned int v[kCvUnroll];
+      bool in[kCvUnroll];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
+      for (int e = 0; e < kCvUnroll; ++e) {
         const int c = c0 + e * kCvThreads + tid;
         in[e] = c < hi;
         v[e] = in[e] ? Ab[c] : 0u;
       }
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
+      for (int e = 0; e < kCvUnroll; ++e) {
         const bool hit = in[e] && (v[e] & pmask) == prefix;
         // a warp whose lanes all fall in one bin adds once; otherwise every hit adds for itself
         const unsigned int dgt = hit ? ((v[e] >> shift) & dmask) : 0x100u;
