@@ -426,6 +426,7 @@ int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, int n_active, cuda
   if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
     const int bytes = (kTopkStageMax + kTopkStageMax / 32 + 1) * 4;
     CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
   }
@@ -435,11 +436,15 @@ int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, int n_active, cuda
   // have a fixed cost, one CTA's passes grow with the list: the cluster pays from about 12 K entries, provided the
   // clusters of the segments that select fit one wave of resident CTAs (two per SM); beyond 16 K entries a single
   // CTA is slower in any case.
-  const int CL = (max_pool > 16384 || (max_pool >= 12288 && n_active * 8 <= 2 * sm_count())) ? 8 : 1;
+  int CL = (max_pool > 16384 || (max_pool >= 12288 && n_active * 8 <= 2 * sm_count())) ? 8 : 1;
+  // many long lists: clusters of 4 when those fit one wave and clusters of 8 would need two (a share of up to
+  // kTopkStageMax entries is still staged in shared memory)
+  if (CL == 8 && n_active * 8 > 2 * sm_count() && n_active * 4 <= 2 * sm_count() && (max_pool + 3) / 4 <= kTopkStageMax) CL = 4;
   const int share = ((max_pool + CL - 1) / CL + 3) / 4 * 4;
   a.stage_entries = share <= kTopkStageMax ? share : 0;  // longer shares are read from global memory
   const size_t smem = (size_t)(a.stage_entries + a.stage_entries / 32 + 1) * 4;
   if (CL == 8) return launch_topk_cluster<8>(a, n_segs, smem, stream);
+  if (CL == 4) return launch_topk_cluster<4>(a, n_segs, smem, stream);
   CATEKV_CUDA_TRY(launch_pdl(topk_kernel<1>, dim3(n_segs), dim3(kTopkThreads), smem, stream, a));
   return CATEKV_OK;
 }
