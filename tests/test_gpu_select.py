@@ -217,3 +217,37 @@ def test_streaming_heads_and_attention_recall(ck):
     assert np.allclose(rec[8:12], 1.0, atol=1e-4) and np.allclose(rec[20:24], 1.0, atol=1e-4)  # adaptive: everything kept
     # consistent heads lean on their planted keys: they recall more mass than the streaming heads of this input
     assert rec[4:8].mean() > rec[0:4].mean()
+
+
+def test_token_major_kv_layout_gives_identical_results(ck):
+    """K and V as [B, n, Hkv, d] views (token-major storage, the head stride smaller than the token stride): the
+    strides go into the tensor map and the gather; selection, window attention and the CV score must not change a bit."""
+    w = synth.scaled(synth.WORKLOADS["cfg0"], B=2, n=1500, budget=200, seed=77)
+    p = synth.prefill_layer(w, 0)
+    mask = p["head_mask"]
+    qw, k, v = p["q_win"].cuda(), p["k"].cuda(), p["v"].cuda()
+    kt = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)   # same values, strides (n*Hkv*d, d, Hkv*d, 1)
+    vt = v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert kt.stride() != k.stride() and torch.equal(kt, k)
+    seq_len = [w.n, 1203]
+    lens = []
+    for b in range(w.B):
+        lens += [w.budget if mask[b, h] else seq_len[b] for h in range(w.Hkv)]
+    res = []
+    for kk, vv in ((k, v), (kt, vt)):
+        cache = ck.Cache(w.B, w.Hkv, lens, 0, "cuda")
+        idx = torch.full((w.B * w.Hkv, w.n), -1, dtype=torch.int32, device="cuda")
+        ck.catekv_select_compact(qw, kk, vv, seq_len, mask, cache, w.budget, 1.0, w.sink, w.local, orc.POOL_SLIDING, 7,
+                                 idx_out=idx)
+        wa = ck.catekv_window_attn(qw, kk, vv, seq_len)
+        cv = ck.catekv_head_cv(qw, kk, seq_len, 16, 40, 0.99, 1.0, True)
+        torch.cuda.synchronize()
+        res.append((cache.seg_len.copy(), idx.clone(), cache.k_pool.clone(), cache.v_pool.clone(), wa, cv))
+    a, b = res
+    assert np.array_equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    for s in range(w.B * w.Hkv):
+        o, L = int(ck.catekv_cache_layout(w.B, w.Hkv, lens, 0)[0][s]), int(a[0][s])
+        assert torch.equal(a[2][o:o + L], b[2][o:o + L]) and torch.equal(a[3][o:o + L], b[3][o:o + L])
+    for x, y in zip(a[4], b[4]):
+        assert torch.equal(x, y)
+    assert torch.equal(a[5], b[5])
