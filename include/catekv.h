@@ -160,7 +160,8 @@ int catekv_checked_build(void);
 int catekv_checked_status(catekv_status* out, int32_t clear);
 
 /*
- * Test hook, host side: the next n_launches launches of the scoring kernel run with their producer lane idle
+ * Test hook, host side: the next n_launches launches of the tensor-core kernels (window scoring, window
+ * attention) run with their producer lanes idle
  * (no copy and no tensor-core instruction is issued) and a wait limit of 512 polls, so that every wait runs out
  * with nothing in flight and the CATEKV_STATUS_WAIT_EXPIRED path executes.  Process-wide counter; 0 switches
  * it off.  Nothing faults or hangs: the CTAs free their tensor memory and return.

@@ -482,15 +482,20 @@ static size_t score_smem_bytes(const ScoreShape& sh) {
 // Test hook (catekv_test_expire_score_waits): launches left that run with an idle producer lane.
 static std::atomic<int> g_expire_launches{0};
 
+// true if this launch is one of those the test hook asked to run with an idle producer lane
+bool score_take_expire_launch() {
+  int left = g_expire_launches.load(std::memory_order_relaxed);
+  while (left > 0 && !g_expire_launches.compare_exchange_weak(left, left - 1)) {
+  }
+  return left > 0;
+}
+
 template <int MODE>
 static int launch_one(const ScoreArgs& a0, const ScoreShape& sh, const CUtensorMap& map, cudaStream_t stream) {
   ScoreArgs a = a0;
   a.spin_limit = kSpinLimit;
   a.idle_producer = 0;
-  int left = g_expire_launches.load(std::memory_order_relaxed);
-  while (left > 0 && !g_expire_launches.compare_exchange_weak(left, left - 1)) {
-  }
-  if (left > 0) {
+  if (score_take_expire_launch()) {
     a.spin_limit = 512;
     a.idle_producer = 1;
   }

@@ -44,6 +44,9 @@ int score_keys_per_cta(int n_jobs, int max_keys);
 // Upper bound of n_jobs * n_chunks for keys_per_cta = score_keys_per_cta(n_jobs, .): the per-CTA row partials of
 // pass 1 are sized by it.  (chunks = round(2 SMs / jobs), so jobs * chunks <= 2 SMs + jobs / 2.)
 static inline int score_max_ctas(int n_jobs) { return n_jobs + 4 * sm_count(); }
+// Test hook (catekv_test_expire_score_waits): true if the launch about to be made is to run with an idle producer
+// lane and a short wait limit; consumes one of the requested launches.
+bool score_take_expire_launch();
 // Enqueue: pass 1 (row max / sum partials), their merge, and pass 2 (column sums or matrix).
 int score_launch(const ScoreArgs& a, ScoreMode out_mode, cudaStream_t stream);
 

@@ -15,7 +15,7 @@
 //
 // Warp roles: warp 9 (one lane) feeds the K and V stages by TMA; warp 8 (one lane) issues every MMA, the S of tile
 // t + 1 before the P V of tile t; warps 0-7 are the epilogue (two per TMEM lane quarter, 64 keys and 64 columns of
-// O each); the two threads of a row exchange their half-tile maxima through shared memory (a named barrier per
+// O each); the two threads of a row exchange their half-tile maxima through shared memory (a pair of mbarriers per
 // pair of warps) and so keep the same reference.  Every mbarrier
 // wait is bounded: on expiry the CTA raises the abort flag, frees its tensor memory, records
 // CATEKV_STATUS_WAIT_EXPIRED and returns.
@@ -48,6 +48,7 @@ struct WinArgs {
                           //                                       sums over the visible keys, over the scored keys
   int32_t* status;
   uint32_t spin_limit;
+  int32_t idle_producer;  // test hook: the TMA and MMA lanes issue nothing, so every wait runs out
 };
 
 __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_constant__ CUtensorMap k_map,
@@ -71,12 +72,14 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   const uint32_t s_pl = s_ph + kWaTileBytes;
   float* s_xch = reinterpret_cast<float*>(smem + 7 * kWaTileBytes);  // [2 halves][128 rows]: half-tile maxima
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_xch + 256);
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 16);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 24);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   const uint32_t bar0 = smem_u32(s_bar);
   const uint32_t bar_full_k = bar0, bar_empty_k = bar0 + 16, bar_full_v = bar0 + 32, bar_empty_v = bar0 + 48;
   const uint32_t bar_done_s = bar0 + 64, bar_free_s = bar0 + 80, bar_p_ready = bar0 + 96, bar_p_free = bar0 + 104;
   const uint32_t bar_done_o = bar0 + 112;
+  // per TMEM lane quarter, for the pair of epilogue warps that share it: maxima written / maxima read
+  const uint32_t bar_xw = bar0 + 120, bar_xr = bar0 + 152;
 
   // ---- set-up: this M tile's query rows (row r = i * G + g), their normalisers, barriers, tensor memory
   for (int id = tid; id < 128 * 16; id += kWaThreads) {
@@ -90,9 +93,10 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   cp_async_commit();
   if (tid == 0) {
     *s_abort = 0;
-    for (int i = 0; i < 15; ++i) {
+    for (int i = 0; i < 23; ++i) {
       const uint32_t bar = bar0 + 8 * i;
-      const int count = (bar == bar_free_s || bar == bar_free_s + 8 || bar == bar_p_ready) ? 8 : 1;  // one arrival per epilogue warp
+      // one arrival per epilogue warp (8), per warp of a pair (2), or one
+      const int count = (bar == bar_free_s || bar == bar_free_s + 8 || bar == bar_p_ready) ? 8 : (bar >= bar_xw ? 2 : 1);
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
     }
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -110,7 +114,7 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
 
   if (warp == 9) {
     // ================= TMA producer =================
-    if (lane == 0) {
+    if (lane == 0 && !a.idle_producer) {
       for (int tile = 0; tile < n_tiles; ++tile) {
         const int st = tile & 1;
         const uint32_t par = (uint32_t)(((tile >> 1) - 1) & 1);
@@ -128,7 +132,7 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
     __syncwarp();
   } else if (warp == 8) {
     // ================= MMA issue =================
-    if (lane == 0) {
+    if (lane == 0 && !a.idle_producer) {
       const uint32_t idesc_s = umma_idesc_bf16(128, 128);      // S[rows x keys]: A = Q, B = K, both K-major
       const uint32_t idesc_o = umma_idesc_bf16_bmn(128, 128);  // O[rows x d]: A = P (K-major), B = V (MN-major)
       auto issue_s = [&](int t) -> bool {
@@ -212,10 +216,16 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
       m0 = fmax3(m0, x[60], x[61]);
       m1 = fmax3(m1, x[62], x[63]);
       float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+      // (bounded mbarrier waits, not a named barrier: a partner that has given up must not leave this warp waiting)
+      const int quarter = warp & 3;
+      if (t >= 1 && !mbar_wait(bar_xr + 8 * quarter, (uint32_t)((t - 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
       s_xch[half * 128 + lane_row] = mx;
-      asm volatile("bar.sync %0, 64;\n" ::"r"(1 + (warp & 3)) : "memory");  // the two warps of this lane quarter
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_xw + 8 * quarter);
+      if (!mbar_wait(bar_xw + 8 * quarter, (uint32_t)(t & 1), s_abort, a.spin_limit)) { alive = false; break; }
       mx = fmaxf(mx, s_xch[(half ^ 1) * 128 + lane_row]);
-      asm volatile("bar.sync %0, 64;\n" ::"r"(1 + (warp & 3)) : "memory");  // both have read: the slots may be rewritten
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_xr + 8 * quarter);  // this warp has read: after both, the slots may be rewritten
       mx = row_ok ? mx * a.scale_log2 : -INFINITY;  // the scale is positive: the max commutes with it
       const bool grow = mx > ref + kWaTau;  // also the first tile with a visible key (ref = -inf)
       const float nref = grow ? mx : ref;
@@ -359,7 +369,7 @@ __global__ void __launch_bounds__(128) window_reduce_kernel(const float* part, c
   }
 }
 
-constexpr size_t kWaSmemBytes = 1024 + 7 * (size_t)kWaTileBytes + 256 * sizeof(float) + 16 * sizeof(uint64_t) + 16;
+constexpr size_t kWaSmemBytes = 1024 + 7 * (size_t)kWaTileBytes + 256 * sizeof(float) + 24 * sizeof(uint64_t) + 16;
 static_assert(kWaSmemBytes <= 227 * 1024, "window_pv_kernel: one CTA's shared memory");
 
 struct WaWs {
@@ -460,6 +470,10 @@ extern "C" int catekv_window_attn(const void* q_win, const void* k, const void* 
   wa.part_s = (float*)(w8 + W.off_part_s);
   wa.status = (int32_t*)(w8 + W.off_status);
   wa.spin_limit = kSpinLimit;
+  if (score_take_expire_launch()) {
+    wa.spin_limit = 512;
+    wa.idle_producer = 1;
+  }
   window_pv_kernel<<<dim3(W.n_chunks, n_segs, W.MT), kWaThreads, kWaSmemBytes, st>>>(k_map, v_map, wa);
   CATEKV_CUDA_TRY(cudaGetLastError());
   window_reduce_kernel<<<dim3((R + 3) / 4, n_segs), 128, 0, st>>>(wa.part, wa.part_s, wa.jobs, W.keys_per_cta, W.n_chunks, W.MT, R,

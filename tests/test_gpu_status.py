@@ -79,6 +79,24 @@ def test_expired_waits_in_head_cv_are_reported(ck):
     np.testing.assert_allclose(cv, ref, rtol=1e-3)
 
 
+def test_expired_waits_in_window_attention_are_reported(ck):
+    w = synth.scaled(synth.WORKLOADS["cfg0"], n=1500)
+    p = synth.prefill_layer(w, 0)
+    qw, k, v = p["q_win"].cuda(), p["k"].cuda(), p["v"].cuda()
+    ws = torch.empty(ck._lib.catekv_window_attn_workspace_bytes(w.B, w.Hq, w.Hkv, w.n, w.L_obs), dtype=torch.uint8,
+                     device="cuda")
+    ck.catekv_test_expire_score_waits(1)
+    ck.catekv_window_attn(qw, k, v, [w.n], ws=ws)
+    st = ck.catekv_workspace_status(ws, raise_on_error=False)
+    assert st["flags"] & ck.STATUS_WAIT_EXPIRED
+    out, lse, _ = ck.catekv_window_attn(qw, k, v, [w.n], ws=ws)   # same workspace, healthy call
+    assert ck.catekv_workspace_status(ws)["flags"] == 0
+    ref, ref_lse = orc.window_attention(synth.bits(p["q_win"])[0, :w.G], synth.bits(p["k"])[0, 0], synth.bits(p["v"])[0, 0],
+                                        w.L_obs)
+    H.check_attention(out[0, :w.G].reshape(-1, w.d), None, lse[0, :w.G].reshape(-1), ref.reshape(-1, w.d),
+                      ref_lse.reshape(-1), "after an expired call")
+
+
 def test_replayed_gather_is_cut_at_the_step_cache_capacity(ck):
     """A retrieval step captured once and replayed while the source grows past what the step cache can hold: the
     copy stops at the capacity, nothing behind the segment is written, and the status block reports it."""
