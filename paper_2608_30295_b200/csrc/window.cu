@@ -233,19 +233,22 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
       const float factor = rescale ? fast_exp2(ref - nref) : 1.f;
       ref = nref;
       // ---- P = exp2(logit - reference) (masked entries are -inf -> 0), its row sums, the hi + lo operand tiles
+      const float nref_neg = ref > -INFINITY ? -ref : -INFINITY;  // no reference yet: every P is exp2(-inf) = 0
       float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, ssc = 0.f;
 #pragma unroll
       for (int c = 0; c < 64; c += 4) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float p = ref > -INFINITY ? fast_exp2(fmaf(x[c + e], a.scale_log2, -ref)) : 0.f;
-          if (edge) ssc += (jb + c + e < n_sc) ? p : 0.f;
-          x[c + e] = p;
-        }
+        x[c] = fast_exp2(fmaf(x[c], a.scale_log2, nref_neg));
+        x[c + 1] = fast_exp2(fmaf(x[c + 1], a.scale_log2, nref_neg));
+        x[c + 2] = fast_exp2(fmaf(x[c + 2], a.scale_log2, nref_neg));
+        x[c + 3] = fast_exp2(fmaf(x[c + 3], a.scale_log2, nref_neg));
         s0 += x[c];
         s1 += x[c + 1];
         s2 += x[c + 2];
         s3 += x[c + 3];
+      }
+      if (edge) {  // a branch of its own (the condition is uniform), so that ordinary tiles do not carry this code
+#pragma unroll
+        for (int c = 0; c < 64; ++c) ssc += (jb + c < n_sc) ? x[c] : 0.f;
       }
       const float sum = (s0 + s1) + (s2 + s3);
       l = l * factor + sum;
