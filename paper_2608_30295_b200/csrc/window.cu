@@ -14,9 +14,9 @@
 // are merged in range order by window_reduce_kernel, which also writes the two log-sum-exps.
 //
 // Warp roles: warp 9 (one lane) feeds the K and V stages by TMA; warp 8 (one lane) issues every MMA, the S of tile
-// t + 1 before the P V of tile t; warps 0-7 are the epilogue (two per TMEM lane quarter, 64 keys and 64 columns of
-// O each); the two threads of a row exchange their half-tile maxima through shared memory (a pair of mbarriers per
-// pair of warps) and so keep the same reference.  Every mbarrier
+// t + 1 before the P V of tile t; warps 0-15 are the epilogue (four per TMEM lane quarter, 32 keys and 32 columns of
+// O each); the four threads of a row exchange their part-tile maxima through shared memory (a pair of mbarriers per
+// lane quarter) and so keep the same reference.  Every mbarrier
 // wait is bounded: on expiry the CTA raises the abort flag, frees its tensor memory, records
 // CATEKV_STATUS_WAIT_EXPIRED and returns.
 #include <math.h>
@@ -30,12 +30,20 @@
 
 namespace catekv {
 
-constexpr int kWaThreads = 320;
+constexpr int kWaEpiWarps = 16;                    // four per TMEM lane quarter, 32 keys (and 32 columns of O) each
+constexpr int kWaSub = kWaEpiWarps / 4;            // epilogue threads per query row
+constexpr int kWaCols = 128 / kWaSub;              // columns of S (keys) and of O a thread owns
+constexpr int kWaThreads = (kWaEpiWarps + 2) * 32;  // + the MMA warp and the TMA warp
 constexpr int kWaTmemCols = 512;       // S slots at columns 0 and 128, O at 256
 constexpr int kWaOCol = 256;
 constexpr int kWaTileBytes = 128 * 256;  // a [128 x 128] bf16 tile: Q rows, a K or V stage, P hi, P lo
-constexpr int kWaStateWords = 5;         // per row and key range: reference, sum (visible keys) x 2 halves, sum (scored keys) x 2 halves
+constexpr int kWaStateWords = 1 + 2 * kWaSub;  // per row and key range: reference, the threads' sums (visible keys), (scored keys)
 constexpr float kWaTau = 8.f;            // a row's reference follows a tile maximum that exceeds it by more than 2^kWaTau
+
+// All a CTA may have.  The carve-up needs 231 632 bytes from a 1024-byte-aligned base, which leaves 816 bytes for the
+// alignment of the base (in practice the dynamic shared memory of a kernel without static shared memory starts
+// aligned); the kernel checks that it fits and otherwise reports through the status block instead of running.
+constexpr size_t kWaSmemBytes = 227 * 1024;
 
 struct WinArgs {
   const uint16_t* q_win;  // [B, Hq, L_obs, d]
@@ -44,7 +52,7 @@ struct WinArgs {
   float scale_log2;
   int32_t keys_per_cta, n_chunks;
   float* part;            // [n_segs][MT][n_chunks][128 rows][128 d]: O relative to the range's reference
-  float* part_s;          // [n_segs][MT][n_chunks][kWaStateWords][128 rows]: reference (log2 domain), the two half-threads'
+  float* part_s;          // [n_segs][MT][n_chunks][kWaStateWords][128 rows]: reference (log2 domain), the row's threads'
                           //                                       sums over the visible keys, over the scored keys
   int32_t* status;
   uint32_t spin_limit;
@@ -70,15 +78,15 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   const uint32_t s_v = s_k + 2 * kWaTileBytes;
   const uint32_t s_ph = s_v + 2 * kWaTileBytes;
   const uint32_t s_pl = s_ph + kWaTileBytes;
-  float* s_xch = reinterpret_cast<float*>(smem + 7 * kWaTileBytes);  // [2 halves][128 rows]: half-tile maxima
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_xch + 256);
+  float* s_xch = reinterpret_cast<float*>(smem + 7 * kWaTileBytes);  // [kWaSub][128 rows]: the threads' part-tile maxima
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_xch + kWaSub * 128);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 24);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   const uint32_t bar0 = smem_u32(s_bar);
   const uint32_t bar_full_k = bar0, bar_empty_k = bar0 + 16, bar_full_v = bar0 + 32, bar_empty_v = bar0 + 48;
   const uint32_t bar_done_s = bar0 + 64, bar_free_s = bar0 + 80, bar_p_ready = bar0 + 96, bar_p_free = bar0 + 104;
   const uint32_t bar_done_o = bar0 + 112;
-  // per TMEM lane quarter, for the pair of epilogue warps that share it: maxima written / maxima read
+  // per TMEM lane quarter, for the epilogue warps that share it: maxima written / maxima read
   const uint32_t bar_xw = bar0 + 120, bar_xr = bar0 + 152;
 
   // ---- set-up: this M tile's query rows (row r = i * G + g), their normalisers, barriers, tensor memory
@@ -95,13 +103,19 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
     *s_abort = 0;
     for (int i = 0; i < 23; ++i) {
       const uint32_t bar = bar0 + 8 * i;
-      // one arrival per epilogue warp (8), per warp of a pair (2), or one
-      const int count = (bar == bar_free_s || bar == bar_free_s + 8 || bar == bar_p_ready) ? 8 : (bar >= bar_xw ? 2 : 1);
+      // one arrival per epilogue warp, per warp of a lane quarter, or one
+      const int count = (bar == bar_free_s || bar == bar_free_s + 8 || bar == bar_p_ready) ? kWaEpiWarps
+                                                                                            : (bar >= bar_xw ? kWaSub : 1);
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
     }
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
-  if (warp == 8) {
+  // the carve-up above must fit what was requested whatever the alignment of the dynamic shared memory's base
+  if (s_base + 7 * kWaTileBytes + kWaSub * 128 * 4 + 24 * 8 + 16 > smem_u32(smem_raw) + (uint32_t)kWaSmemBytes) {
+    if (tid == 0) raise_status(a.status, CATEKV_STATUS_WAIT_EXPIRED, kKidScore, (int)blockIdx.y, -1);
+    return;
+  }
+  if (warp == kWaEpiWarps) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(s_tmem)), "r"(kWaTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
@@ -112,7 +126,7 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
 
-  if (warp == 9) {
+  if (warp == kWaEpiWarps + 1) {
     // ================= TMA producer =================
     if (lane == 0 && !a.idle_producer) {
       for (int tile = 0; tile < n_tiles; ++tile) {
@@ -130,7 +144,7 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
       }
     }
     __syncwarp();
-  } else if (warp == 8) {
+  } else if (warp == kWaEpiWarps) {
     // ================= MMA issue =================
     if (lane == 0 && !a.idle_producer) {
       const uint32_t idesc_s = umma_idesc_bf16(128, 128);      // S[rows x keys]: A = Q, B = K, both K-major
@@ -177,88 +191,103 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   } else {
     // ================= epilogue warps =================
     const int lane_row = (warp & 3) * 32 + lane;  // this thread's TMEM lane = its query row of the M tile
-    const int half = warp >> 2;                   // keys [64 * half, 64 * half + 64) of every tile, d [64 * half, ...) of O
-    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const int sub = warp >> 2;                    // keys [kWaCols * sub, ...) of every tile, the same columns of O
+    const int quarter = warp & 3;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     const int r = mt * 128 + lane_row;
     const bool row_ok = r < a.R;
     const int pos = n - a.L_obs + (row_ok ? r / a.G : 0);  // the row's own position: it sees keys j <= pos
     const int n_sc = n - a.L_obs;                           // keys below are scored keys
-    // The two threads of a row (warps w and w + 4) keep the same reference: each tile they exchange the maxima of
-    // their halves through shared memory and take the same decision.  The sums stay per thread.
+    // The kWaSub threads of a row keep the same reference: each tile they exchange the maxima of their parts through
+    // shared memory and take the same decision.  The exchange is off the critical path: P is formed against the
+    // reference as it stands while the maxima travel, and only when the tile's maximum turns out to exceed it by more
+    // than 2^kWaTau (rare after the first tiles) is the tile reread from TMEM and P formed again.  Sums stay per thread.
     float ref = -INFINITY, l = 0.f, lsc = 0.f;
     bool alive = true;
     for (int t = 0; t < n_tiles; ++t) {
       const int st = t & 1;
       if (!mbar_wait(bar_done_s + 8 * st, (uint32_t)((t >> 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
       tc_fence_after();
-      float x[64];
-      tmem_ld64(tmem + lane_base + (uint32_t)(st * 128 + half * 64), x);
-      tmem_wait_ld64(x);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_free_s + 8 * st);  // the S slot goes back to the MMA warp
-      const int jb = j_lo + t * kKeyTile + half * 64;   // key of x[0]
-      const bool edge = jb + 63 >= n_sc;                // uniform: the block reaches the window's own keys (or the end)
-      if (edge) {
+      const uint32_t s_addr = tmem + lane_base + (uint32_t)(st * 128 + sub * kWaCols);
+      const int jb = j_lo + t * kKeyTile + sub * kWaCols;  // key of x[0]
+      const bool edge = jb + kWaCols - 1 >= n_sc;           // uniform: the block reaches the window's own keys (or the end)
+      float x[kWaCols];
+      auto load_logits = [&]() {
+        tmem_ld32(s_addr, x);
+        tmem_wait_ld32(x);
+        if (edge) {
 #pragma unroll
-        for (int c = 0; c < 64; ++c) x[c] = (jb + c <= pos) ? x[c] : -INFINITY;
-      }
-      // ---- the tile's maximum over the keys this row sees: this half, then the partner's through shared memory
+          for (int c = 0; c < kWaCols; ++c) x[c] = (jb + c <= pos) ? x[c] : -INFINITY;
+        }
+      };
+      float sum = 0.f;
+      auto form_p = [&]() {  // x: logits -> P against `ref`; sum: their total
+        const float nref_neg = ref > -INFINITY ? -ref : -INFINITY;  // no reference yet: every P is exp2(-inf) = 0
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int c = 0; c < kWaCols; c += 4) {
+          x[c] = fast_exp2(fmaf(x[c], a.scale_log2, nref_neg));
+          x[c + 1] = fast_exp2(fmaf(x[c + 1], a.scale_log2, nref_neg));
+          x[c + 2] = fast_exp2(fmaf(x[c + 2], a.scale_log2, nref_neg));
+          x[c + 3] = fast_exp2(fmaf(x[c + 3], a.scale_log2, nref_neg));
+          s0 += x[c];
+          s1 += x[c + 1];
+          s2 += x[c + 2];
+          s3 += x[c + 3];
+        }
+        sum = (s0 + s1) + (s2 + s3);
+      };
+      load_logits();
+      // ---- this thread's maximum over the keys its row sees goes to the row's other threads
       float m0 = fmax3(x[0], x[1], x[2]), m1 = fmax3(x[3], x[4], x[5]);
       float m2 = fmax3(x[6], x[7], x[8]), m3 = fmax3(x[9], x[10], x[11]);
 #pragma unroll
-      for (int c = 12; c < 60; c += 8) {
+      for (int c = 12; c < 28; c += 8) {
         m0 = fmax3(m0, x[c], x[c + 1]);
         m1 = fmax3(m1, x[c + 2], x[c + 3]);
         m2 = fmax3(m2, x[c + 4], x[c + 5]);
         m3 = fmax3(m3, x[c + 6], x[c + 7]);
       }
-      m0 = fmax3(m0, x[60], x[61]);
-      m1 = fmax3(m1, x[62], x[63]);
+      m0 = fmax3(m0, x[28], x[29]);
+      m1 = fmax3(m1, x[30], x[31]);
       float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
       // (bounded mbarrier waits, not a named barrier: a partner that has given up must not leave this warp waiting)
-      const int quarter = warp & 3;
       if (t >= 1 && !mbar_wait(bar_xr + 8 * quarter, (uint32_t)((t - 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
-      s_xch[half * 128 + lane_row] = mx;
+      s_xch[sub * 128 + lane_row] = mx;
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_xw + 8 * quarter);
+      // ---- P against the reference as it stands, while the maxima travel
+      form_p();
       if (!mbar_wait(bar_xw + 8 * quarter, (uint32_t)(t & 1), s_abort, a.spin_limit)) { alive = false; break; }
-      mx = fmaxf(mx, s_xch[(half ^ 1) * 128 + lane_row]);
+#pragma unroll
+      for (int k = 0; k < kWaSub; ++k) mx = fmaxf(mx, s_xch[k * 128 + lane_row]);
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_xr + 8 * quarter);  // this warp has read: after both, the slots may be rewritten
+      if (lane == 0) mbar_arrive(bar_xr + 8 * quarter);  // this warp has read: after all, the slots may be rewritten
       mx = row_ok ? mx * a.scale_log2 : -INFINITY;  // the scale is positive: the max commutes with it
       const bool grow = mx > ref + kWaTau;  // also the first tile with a visible key (ref = -inf)
-      const float nref = grow ? mx : ref;
       const bool rescale = grow && ref > -INFINITY;
-      const float factor = rescale ? fast_exp2(ref - nref) : 1.f;
-      ref = nref;
-      // ---- P = exp2(logit - reference) (masked entries are -inf -> 0), its row sums, the hi + lo operand tiles
-      const float nref_neg = ref > -INFINITY ? -ref : -INFINITY;  // no reference yet: every P is exp2(-inf) = 0
-      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, ssc = 0.f;
-#pragma unroll
-      for (int c = 0; c < 64; c += 4) {
-        x[c] = fast_exp2(fmaf(x[c], a.scale_log2, nref_neg));
-        x[c + 1] = fast_exp2(fmaf(x[c + 1], a.scale_log2, nref_neg));
-        x[c + 2] = fast_exp2(fmaf(x[c + 2], a.scale_log2, nref_neg));
-        x[c + 3] = fast_exp2(fmaf(x[c + 3], a.scale_log2, nref_neg));
-        s0 += x[c];
-        s1 += x[c + 1];
-        s2 += x[c + 2];
-        s3 += x[c + 3];
+      const float factor = rescale ? fast_exp2(ref - mx) : 1.f;
+      if (__any_sync(0xffffffffu, grow)) {  // the same lanes in all the warps of the quarter: the tile once more
+        ref = grow ? mx : ref;
+        load_logits();
+        form_p();
       }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_free_s + 8 * st);  // the S slot goes back to the MMA warp
+      float ssc = sum;
       if (edge) {  // a branch of its own (the condition is uniform), so that ordinary tiles do not carry this code
+        ssc = 0.f;
 #pragma unroll
-        for (int c = 0; c < 64; ++c) ssc += (jb + c < n_sc) ? x[c] : 0.f;
+        for (int c = 0; c < kWaCols; ++c) ssc += (jb + c < n_sc) ? x[c] : 0.f;
       }
-      const float sum = (s0 + s1) + (s2 + s3);
       l = l * factor + sum;
-      lsc = lsc * factor + (edge ? ssc : sum);
-      uint32_t ph[32], pl[32];  // the probabilities as bf16 hi + lo pairs
+      lsc = lsc * factor + ssc;
+      uint32_t ph[kWaCols / 2], pl[kWaCols / 2];  // the probabilities as bf16 hi + lo pairs
 #pragma unroll
-      for (int c = 0; c < 64; c += 2) {
+      for (int c = 0; c < kWaCols; c += 2) {
         // hi = the upper 16 bits (a byte permute, no conversion; p - hi is exact in fp32), lo = p - hi rounded to bf16:
-        // hi + lo carries 16 significant bits of p.  Conversions share the special-function pipe with the
-        // exponentials, so only the lo half uses one.
+        // hi + lo carries 16 significant bits of p.
         const uint32_t b0 = __float_as_uint(x[c]), b1 = __float_as_uint(x[c + 1]);
         ph[c / 2] = __byte_perm(b0, b1, 0x7632);
         pl[c / 2] = pack_bf16(x[c] - __uint_as_float(b0 & 0xffff0000u), x[c + 1] - __uint_as_float(b1 & 0xffff0000u));
@@ -266,22 +295,19 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
       // All of the above ran under the previous tile's P V; that must have completed before O is touched and the
       // P buffer rewritten
       if (t >= 1 && !mbar_wait(bar_p_free, (uint32_t)((t - 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
-      if (__any_sync(0xffffffffu, rescale)) {  // this thread's 64 columns of its row of O
+      if (__any_sync(0xffffffffu, rescale)) {  // this thread's columns of its row of O
         tc_fence_after();
-#pragma unroll 1
-        for (int c0 = 0; c0 < 64; c0 += 32) {
-          float o[32];
-          tmem_ld32(tmem + lane_base + (uint32_t)(kWaOCol + half * 64 + c0), o);
-          tmem_wait_ld32(o);
+        float o[32];
+        tmem_ld32(tmem + lane_base + (uint32_t)(kWaOCol + sub * kWaCols), o);
+        tmem_wait_ld32(o);
 #pragma unroll
-          for (int c = 0; c < 32; ++c) o[c] *= factor;
-          tmem_st32(tmem + lane_base + (uint32_t)(kWaOCol + half * 64 + c0), o);
-        }
+        for (int c = 0; c < 32; ++c) o[c] *= factor;
+        tmem_st32(tmem + lane_base + (uint32_t)(kWaOCol + sub * kWaCols), o);
         tmem_wait_st();
       }
 #pragma unroll
-      for (int c = 0; c < 64; c += 8) {
-        const uint32_t off = sw128_off(lane_row, half * 8 + (c >> 3), 128);
+      for (int c = 0; c < kWaCols; c += 8) {
+        const uint32_t off = sw128_off(lane_row, sub * (kWaCols / 8) + (c >> 3), 128);
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(s_ph + off), "r"(ph[c / 2]), "r"(ph[c / 2 + 1]), "r"(ph[c / 2 + 2]), "r"(ph[c / 2 + 3]) : "memory");
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(s_pl + off), "r"(pl[c / 2]), "r"(pl[c / 2 + 1]), "r"(pl[c / 2 + 2]), "r"(pl[c / 2 + 3]) : "memory");
       }
@@ -290,20 +316,20 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_p_ready);  // the MMA warp may issue this tile's P V
     }
-    // ---- the CTA's partial result: this thread's row, 64 of the 128 d, and its share of the row's state
+    // ---- the CTA's partial result: this thread's row, its columns of O, and its share of the row's state
     if (alive && mbar_wait(bar_done_o, 0u, s_abort, a.spin_limit)) {
       tc_fence_after();
-      float o[64];
-      tmem_ld64(tmem + lane_base + (uint32_t)(kWaOCol + half * 64), o);
-      tmem_wait_ld64(o);
+      float o[32];
+      tmem_ld32(tmem + lane_base + (uint32_t)(kWaOCol + sub * kWaCols), o);
+      tmem_wait_ld32(o);
       const size_t cta = ((size_t)blockIdx.y * gridDim.z + mt) * a.n_chunks + blockIdx.x;
-      float* dst = a.part + (cta * 128 + lane_row) * 128 + half * 64;
+      float* dst = a.part + (cta * 128 + lane_row) * 128 + sub * kWaCols;
 #pragma unroll
-      for (int c = 0; c < 64; c += 4) *reinterpret_cast<float4*>(dst + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+      for (int c = 0; c < 32; c += 4) *reinterpret_cast<float4*>(dst + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
       float* ds = a.part_s + cta * (kWaStateWords * 128);
-      if (half == 0) ds[lane_row] = ref;
-      ds[(1 + half) * 128 + lane_row] = l;
-      ds[(3 + half) * 128 + lane_row] = lsc;
+      if (sub == 0) ds[lane_row] = ref;
+      ds[(1 + sub) * 128 + lane_row] = l;
+      ds[(1 + kWaSub + sub) * 128 + lane_row] = lsc;
     }
   }
 
@@ -312,7 +338,7 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
     for (int i = 0; i < 200; ++i) __nanosleep(1000);
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kWaTmemCols) : "memory");
+  if (warp == kWaEpiWarps) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kWaTmemCols) : "memory");
   if (*s_abort && tid == 0) raise_status(a.status, CATEKV_STATUS_WAIT_EXPIRED, kKidScore, (int)blockIdx.y, (int)blockIdx.x);
 }
 
@@ -346,8 +372,14 @@ __global__ void __launch_bounds__(128) window_reduce_kernel(const float* part, c
     acc.y += w * v.y;
     acc.z += w * v.z;
     acc.w += w * v.w;
-    L += w * (ps[c * kStep + 128] + ps[c * kStep + 256]);
-    Lsc += w * (ps[c * kStep + 384] + ps[c * kStep + 512]);
+    float lc = 0.f, lscc = 0.f;
+#pragma unroll
+    for (int k = 0; k < kWaSub; ++k) {
+      lc += ps[c * kStep + (1 + k) * 128];
+      lscc += ps[c * kStep + (1 + kWaSub + k) * 128];
+    }
+    L += w * lc;
+    Lsc += w * lscc;
   }
   const float inv = L > 0.f ? 1.f / L : 0.f;
   acc.x *= inv;
@@ -372,8 +404,7 @@ __global__ void __launch_bounds__(128) window_reduce_kernel(const float* part, c
   }
 }
 
-constexpr size_t kWaSmemBytes = 1024 + 7 * (size_t)kWaTileBytes + 256 * sizeof(float) + 24 * sizeof(uint64_t) + 16;
-static_assert(kWaSmemBytes <= 227 * 1024, "window_pv_kernel: one CTA's shared memory");
+static_assert(kWaCols == 32, "the epilogue is written for 32 columns per thread");
 
 struct WaWs {
   size_t off_status, off_jobs, off_part, off_part_s, bytes;
