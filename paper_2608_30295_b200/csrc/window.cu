@@ -4,21 +4,24 @@
 // of the token-criticality line.  catekv_select_compact takes the latter in place of its own first pass over K.
 //
 // One sweep over K and V.  window_pv_kernel: a CTA owns a range of keys of one (sequence, KV head) and 128 query
-// rows.  Per 128-key tile: S = Q K^T (tcgen05.mma into one of two TMEM slots); an epilogue thread owns a query row,
-// finds the tile's maximum, turns S into P = exp2(logit - ref) against the row's reference value, adds the row sums
-// (all visible keys; scored keys only) and writes P to shared memory as a bf16 hi + lo pair in the K-major
-// SWIZZLE_128B operand layout; two more chains of tcgen05.mma add P_hi V and P_lo V (V as the MN-major B operand,
-// straight from the TMA tile) to O in TMEM.  The reference only moves when a tile's maximum exceeds it by more than
-// 2^8 (P stays below 256, far inside what bf16 hi + lo and the fp32 accumulator carry); then the row's O is read from
-// TMEM, scaled and stored back before the tile's P V is issued.  The ranges' partial results (O, reference, sums)
-// are merged in range order by window_reduce_kernel, which also writes the two log-sum-exps.
+// rows.  Per 128-key tile: S = Q K^T (tcgen05.mma into one of two TMEM slots); an epilogue thread owns a query row
+// and 64 of the tile's keys: it finds their maximum, the row's threads agree on the row's reference value, and it
+// turns its part of S into P = exp2(logit - ref), adds the row sums (all visible keys; scored keys only) and writes P
+// back over the same TMEM columns as a bf16 hi + lo pair (hi in the first 16 of every 32 columns, lo in the last 16,
+// two values per column).  P never touches shared memory: 16 more tcgen05.mma take it from TMEM as their A operand
+// and add P_hi V and P_lo V (V as the MN-major B operand, straight from the TMA tile) to O in TMEM.  The reference
+// only moves when a tile's maximum exceeds it by more than 2^8 (P stays below 256, far inside what bf16 hi + lo and
+// the fp32 accumulator carry); then the row's O is read from TMEM, scaled and stored back before the tile's P V is
+// issued.  The ranges' partial results (O, reference, sums) are merged in range order by window_reduce_kernel,
+// which also writes the two log-sum-exps.
 //
-// Warp roles: warp 9 (one lane) feeds the K and V stages by TMA; warp 8 (one lane) issues every MMA, the S of tile
-// t + 1 before the P V of tile t; warps 0-15 are the epilogue (four per TMEM lane quarter, 32 keys and 32 columns of
-// O each); the four threads of a row exchange their part-tile maxima through shared memory (a pair of mbarriers per
-// lane quarter) and so keep the same reference.  Every mbarrier
-// wait is bounded: on expiry the CTA raises the abort flag, frees its tensor memory, records
-// CATEKV_STATUS_WAIT_EXPIRED and returns.
+// Warp roles: warps 17 and 18 (one lane each) feed the three K stages and the two V stages by TMA; warp 16 (one
+// lane) issues every MMA: S(0), S(1), then per tile P V(t) followed by S(t + 2) into the slot P V(t) has just read
+// (the tensor pipe keeps issue order); warps 0-15 are the epilogue, two groups of eight (two warps per TMEM lane
+// quarter: 64 keys each) that take alternate tiles in alternate slots, so that one group's exponentials overlap the
+// other group's loads, maxima and hand-shakes.  Only the decision "does the reference move" is serial from tile to
+// tile (a barrier between the groups; the reference sits in shared memory).  Every mbarrier wait is bounded: on
+// expiry the CTA raises the abort flag, frees its tensor memory, records CATEKV_STATUS_WAIT_EXPIRED and returns.
 #include <math.h>
 #include <string.h>
 
@@ -30,20 +33,19 @@
 
 namespace catekv {
 
-constexpr int kWaEpiWarps = 16;                    // four per TMEM lane quarter, 32 keys (and 32 columns of O) each
-constexpr int kWaSub = kWaEpiWarps / 4;            // epilogue threads per query row
-constexpr int kWaCols = 128 / kWaSub;              // columns of S (keys) and of O a thread owns
-constexpr int kWaThreads = (kWaEpiWarps + 2) * 32;  // + the MMA warp and the TMA warp
-constexpr int kWaTmemCols = 512;       // S slots at columns 0 and 128, O at 256
+constexpr int kWaEpiWarps = 16;                     // two groups of eight: two warps per TMEM lane quarter and group
+constexpr int kWaSub = 4;                           // epilogue threads per query row (2 groups x 2 halves)
+constexpr int kWaThreads = (kWaEpiWarps + 3) * 32;  // + the MMA warp and the two TMA warps (K, V)
+constexpr int kWaKStages = 3, kWaVStages = 2;
+constexpr int kWaTmemCols = 512;         // S / P slots at columns 0 and 128, O at 256
 constexpr int kWaOCol = 256;
-constexpr int kWaTileBytes = 128 * 256;  // a [128 x 128] bf16 tile: Q rows, a K or V stage, P hi, P lo
+constexpr int kWaTileBytes = 128 * 256;  // a [128 x 128] bf16 tile: the Q rows, a K or V stage
 constexpr int kWaStateWords = 1 + 2 * kWaSub;  // per row and key range: reference, the threads' sums (visible keys), (scored keys)
 constexpr float kWaTau = 8.f;            // a row's reference follows a tile maximum that exceeds it by more than 2^kWaTau
-
-// All a CTA may have.  The carve-up needs 231 632 bytes from a 1024-byte-aligned base, which leaves 816 bytes for the
-// alignment of the base (in practice the dynamic shared memory of a kernel without static shared memory starts
-// aligned); the kernel checks that it fits and otherwise reports through the status block instead of running.
-constexpr size_t kWaSmemBytes = 227 * 1024;
+constexpr int kWaBarriers = 36;
+constexpr size_t kWaSmemBytes = 1024 + (size_t)(1 + kWaKStages + kWaVStages) * kWaTileBytes + (4 * 128 + 256) * sizeof(float) +
+                                kWaBarriers * sizeof(uint64_t) + 16;
+static_assert(kWaSmemBytes <= 227 * 1024, "window_pv_kernel: one CTA's shared memory");
 
 struct WinArgs {
   const uint16_t* q_win;  // [B, Hq, L_obs, d]
@@ -58,6 +60,21 @@ struct WinArgs {
   uint32_t spin_limit;
   int32_t idle_producer;  // test hook: the TMA and MMA lanes issue nothing, so every wait runs out
 };
+
+__device__ __forceinline__ float max32(const float (&x)[32]) {
+  float m0 = fmax3(x[0], x[1], x[2]), m1 = fmax3(x[3], x[4], x[5]);
+  float m2 = fmax3(x[6], x[7], x[8]), m3 = fmax3(x[9], x[10], x[11]);
+#pragma unroll
+  for (int c = 12; c < 28; c += 8) {
+    m0 = fmax3(m0, x[c], x[c + 1]);
+    m1 = fmax3(m1, x[c + 2], x[c + 3]);
+    m2 = fmax3(m2, x[c + 4], x[c + 5]);
+    m3 = fmax3(m3, x[c + 6], x[c + 7]);
+  }
+  m0 = fmax3(m0, x[28], x[29]);
+  m1 = fmax3(m1, x[30], x[31]);
+  return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
 
 __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_constant__ CUtensorMap k_map,
                                                                 const __grid_constant__ CUtensorMap v_map, const WinArgs a) {
@@ -75,21 +92,20 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   uint8_t* smem = smem_raw + (s_base - smem_u32(smem_raw));
   const uint32_t s_q = s_base;
   const uint32_t s_k = s_q + kWaTileBytes;
-  const uint32_t s_v = s_k + 2 * kWaTileBytes;
-  const uint32_t s_ph = s_v + 2 * kWaTileBytes;
-  const uint32_t s_pl = s_ph + kWaTileBytes;
-  float* s_xch = reinterpret_cast<float*>(smem + 7 * kWaTileBytes);  // [kWaSub][128 rows]: the threads' part-tile maxima
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_xch + kWaSub * 128);
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 24);
+  const uint32_t s_v = s_k + kWaKStages * kWaTileBytes;
+  float* s_xch = reinterpret_cast<float*>(smem + (1 + kWaKStages + kWaVStages) * kWaTileBytes);  // [group][half][row]: part-tile maxima
+  float* s_ref = s_xch + 4 * 128;  // [tile parity][row]: the row's reference after the decision for a tile of that parity
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_ref + 256);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + kWaBarriers);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   const uint32_t bar0 = smem_u32(s_bar);
-  const uint32_t bar_full_k = bar0, bar_empty_k = bar0 + 16, bar_full_v = bar0 + 32, bar_empty_v = bar0 + 48;
-  const uint32_t bar_done_s = bar0 + 64, bar_free_s = bar0 + 80, bar_p_ready = bar0 + 96, bar_p_free = bar0 + 104;
-  const uint32_t bar_done_o = bar0 + 112;
-  // per TMEM lane quarter, for the epilogue warps that share it: maxima written / maxima read
-  const uint32_t bar_xw = bar0 + 120, bar_xr = bar0 + 152;
+  auto B = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  // barrier indices
+  constexpr int kFullK = 0, kEmptyK = 3, kFullV = 6, kEmptyV = 8, kDoneS = 10, kPReady = 12, kPvDone = 14, kDoneO = 15, kDec = 16,
+                kXw = 17, kXr = 25;  // kXw / kXr: [group][quarter]
+  static_assert(kXr + 8 <= kWaBarriers, "barrier table");
 
-  // ---- set-up: this M tile's query rows (row r = i * G + g), their normalisers, barriers, tensor memory
+  // ---- set-up: this M tile's query rows (row r = i * G + g), the row references, barriers, tensor memory
   for (int id = tid; id < 128 * 16; id += kWaThreads) {
     const int row = id >> 4, c = id & 15;
     const int r = mt * 128 + row;
@@ -99,21 +115,15 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
     cp_async16(s_q + sw128_off(row, c, 128), src, ok);
   }
   cp_async_commit();
+  for (int row = tid; row < 256; row += kWaThreads) s_ref[row] = -INFINITY;
   if (tid == 0) {
     *s_abort = 0;
-    for (int i = 0; i < 23; ++i) {
-      const uint32_t bar = bar0 + 8 * i;
-      // one arrival per epilogue warp, per warp of a lane quarter, or one
-      const int count = (bar == bar_free_s || bar == bar_free_s + 8 || bar == bar_p_ready) ? kWaEpiWarps
-                                                                                            : (bar >= bar_xw ? kWaSub : 1);
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+    for (int i = 0; i < kWaBarriers; ++i) {
+      // arrivals: the 8 warps of an epilogue group (P ready, decision), the 2 warps of a group's lane quarter (maxima), else one
+      const int count = (i == kPReady || i == kPReady + 1 || i == kDec) ? 8 : (i >= kXw ? 2 : 1);
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(B(i)), "r"(count));
     }
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-  }
-  // the carve-up above must fit what was requested whatever the alignment of the dynamic shared memory's base
-  if (s_base + 7 * kWaTileBytes + kWaSub * 128 * 4 + 24 * 8 + 16 > smem_u32(smem_raw) + (uint32_t)kWaSmemBytes) {
-    if (tid == 0) raise_status(a.status, CATEKV_STATUS_WAIT_EXPIRED, kKidScore, (int)blockIdx.y, -1);
-    return;
   }
   if (warp == kWaEpiWarps) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(s_tmem)), "r"(kWaTmemCols) : "memory");
@@ -127,105 +137,169 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   const uint32_t tmem = *s_tmem;
 
   if (warp == kWaEpiWarps + 1) {
-    // ================= TMA producer =================
+    // ================= TMA producer, K: three stages, refilled as soon as the S that read one has completed
     if (lane == 0 && !a.idle_producer) {
-      for (int tile = 0; tile < n_tiles; ++tile) {
-        const int st = tile & 1;
-        const uint32_t par = (uint32_t)(((tile >> 1) - 1) & 1);
-        const int j0 = j_lo + tile * kKeyTile;
-        if (tile >= 2 && !mbar_wait(bar_empty_k + 8 * st, par, s_abort, a.spin_limit)) break;
-        mbar_expect_tx(bar_full_k + 8 * st, kWaTileBytes);
-        tma_load_box(s_k + st * kWaTileBytes, &k_map, 0, j0, job.h, job.b, bar_full_k + 8 * st);
-        tma_load_box(s_k + st * kWaTileBytes + kKBlockBytes, &k_map, 64, j0, job.h, job.b, bar_full_k + 8 * st);
-        if (tile >= 2 && !mbar_wait(bar_empty_v + 8 * st, par, s_abort, a.spin_limit)) break;
-        mbar_expect_tx(bar_full_v + 8 * st, kWaTileBytes);
-        tma_load_box(s_v + st * kWaTileBytes, &v_map, 0, j0, job.h, job.b, bar_full_v + 8 * st);
-        tma_load_box(s_v + st * kWaTileBytes + kKBlockBytes, &v_map, 64, j0, job.h, job.b, bar_full_v + 8 * st);
+      for (int t = 0; t < n_tiles; ++t) {
+        const int st = t % kWaKStages, use = t / kWaKStages;
+        if (use >= 1 && !mbar_wait(B(kEmptyK + st), (uint32_t)((use - 1) & 1), s_abort, a.spin_limit)) break;
+        const int j0 = j_lo + t * kKeyTile;
+        mbar_expect_tx(B(kFullK + st), kWaTileBytes);
+        tma_load_box(s_k + st * kWaTileBytes, &k_map, 0, j0, job.h, job.b, B(kFullK + st));
+        tma_load_box(s_k + st * kWaTileBytes + kKBlockBytes, &k_map, 64, j0, job.h, job.b, B(kFullK + st));
+      }
+    }
+    __syncwarp();
+  } else if (warp == kWaEpiWarps + 2) {
+    // ================= TMA producer, V: two stages, refilled when the P V that read one has completed
+    if (lane == 0 && !a.idle_producer) {
+      for (int t = 0; t < n_tiles; ++t) {
+        const int st = t % kWaVStages, use = t / kWaVStages;
+        if (use >= 1 && !mbar_wait(B(kEmptyV + st), (uint32_t)((use - 1) & 1), s_abort, a.spin_limit)) break;
+        const int j0 = j_lo + t * kKeyTile;
+        mbar_expect_tx(B(kFullV + st), kWaTileBytes);
+        tma_load_box(s_v + st * kWaTileBytes, &v_map, 0, j0, job.h, job.b, B(kFullV + st));
+        tma_load_box(s_v + st * kWaTileBytes + kKBlockBytes, &v_map, 64, j0, job.h, job.b, B(kFullV + st));
       }
     }
     __syncwarp();
   } else if (warp == kWaEpiWarps) {
-    // ================= MMA issue =================
+    // ================= MMA issue: S(0), S(1), then per tile P V(t) and S(t + 2) into the slot P V(t) has just read
     if (lane == 0 && !a.idle_producer) {
       const uint32_t idesc_s = umma_idesc_bf16(128, 128);      // S[rows x keys]: A = Q, B = K, both K-major
-      const uint32_t idesc_o = umma_idesc_bf16_bmn(128, 128);  // O[rows x d]: A = P (K-major), B = V (MN-major)
+      const uint32_t idesc_o = umma_idesc_bf16_bmn(128, 128);  // O[rows x d]: A = P (in TMEM), B = V (MN-major)
       auto issue_s = [&](int t) -> bool {
-        const int st = t & 1;
-        if (!mbar_wait(bar_full_k + 8 * st, (uint32_t)((t >> 1) & 1), s_abort, a.spin_limit)) return false;
-        if (t >= 2 && !mbar_wait(bar_free_s + 8 * st, (uint32_t)(((t >> 1) - 1) & 1), s_abort, a.spin_limit)) return false;
+        const int st = t % kWaKStages;
+        if (!mbar_wait(B(kFullK + st), (uint32_t)((t / kWaKStages) & 1), s_abort, a.spin_limit)) return false;
         tc_fence_after();
         const uint32_t sk = s_k + st * kWaTileBytes;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t off = (kk >> 2) * kKBlockBytes + (kk & 3) * 32;
-          umma_bf16(tmem + (uint32_t)(st * 128), umma_desc_sw128(s_q + off), umma_desc_sw128(sk + off), idesc_s, kk ? 1u : 0u);
+          umma_bf16(tmem + (uint32_t)((t & 1) * 128), umma_desc_sw128(s_q + off), umma_desc_sw128(sk + off), idesc_s, kk ? 1u : 0u);
         }
-        umma_commit(bar_done_s + 8 * st);
-        umma_commit(bar_empty_k + 8 * st);
+        umma_commit(B(kDoneS + (t & 1)));
+        umma_commit(B(kEmptyK + st));
         return true;
       };
-      bool ok = issue_s(0);
+      bool ok = issue_s(0) && (n_tiles < 2 || issue_s(1));
       for (int t = 0; ok && t < n_tiles; ++t) {
-        if (t + 1 < n_tiles && !issue_s(t + 1)) break;
-        const int st = t & 1;
-        if (!mbar_wait(bar_p_ready, (uint32_t)(t & 1), s_abort, a.spin_limit)) break;
-        if (!mbar_wait(bar_full_v + 8 * st, (uint32_t)((t >> 1) & 1), s_abort, a.spin_limit)) break;
+        const int g = t & 1, sv_st = t % kWaVStages;
+        if (!mbar_wait(B(kPReady + g), (uint32_t)((t >> 1) & 1), s_abort, a.spin_limit)) break;
+        if (!mbar_wait(B(kFullV + sv_st), (uint32_t)((t / kWaVStages) & 1), s_abort, a.spin_limit)) break;
         tc_fence_after();
-        const uint32_t sv = s_v + st * kWaTileBytes;
+        const uint32_t sv = s_v + sv_st * kWaTileBytes;
+        const uint32_t slot = tmem + (uint32_t)(g * 128);
+        // P of the 32-key block b of the tile sits in the block's own 32 columns of the slot: hi in the first 16
+        // (two bf16 per column), lo in the last 16; a k-step is 16 keys = 8 columns
 #pragma unroll
         for (int part = 0; part < 2; ++part) {
-          const uint32_t sp = part ? s_pl : s_ph;
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {  // 16 keys per step
-            const uint32_t aoff = (kk >> 2) * kKBlockBytes + (kk & 3) * 32;
-            umma_bf16(tmem + kWaOCol, umma_desc_sw128(sp + aoff), umma_desc_sw128_mn(sv + kk * 2048, kKBlockBytes), idesc_o,
-                      (t | part | kk) ? 1u : 0u);
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t acol = (uint32_t)((kk >> 1) * 32 + part * 16 + (kk & 1) * 8);
+            umma_bf16_ta(tmem + kWaOCol, slot + acol, umma_desc_sw128_mn(sv + kk * 2048, kKBlockBytes), idesc_o,
+                         (t | part | kk) ? 1u : 0u);
           }
         }
-        umma_commit(bar_p_free);
-        umma_commit(bar_empty_v + 8 * st);
-        if (t == n_tiles - 1) umma_commit(bar_done_o);
+        umma_commit(B(kPvDone));
+        umma_commit(B(kEmptyV + sv_st));
+        if (t == n_tiles - 1) umma_commit(B(kDoneO));
+        if (t + 2 < n_tiles && !issue_s(t + 2)) break;  // executes after P V(t): the tensor pipe keeps issue order
       }
     }
     __syncwarp();
   } else {
-    // ================= epilogue warps =================
-    const int lane_row = (warp & 3) * 32 + lane;  // this thread's TMEM lane = its query row of the M tile
-    const int sub = warp >> 2;                    // keys [kWaCols * sub, ...) of every tile, the same columns of O
-    const int quarter = warp & 3;
+    // ================= epilogue: group g = warp / 8 takes the tiles t = g, g + 2, ... in slot g
+    const int g = warp >> 3;
+    const int quarter = warp & 3, half = (warp >> 2) & 1;  // TMEM lane quarter; keys [64 half, 64 half + 64) of the tile
+    const int lane_row = quarter * 32 + lane;              // this thread's TMEM lane = its query row of the M tile
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     const int r = mt * 128 + lane_row;
     const bool row_ok = r < a.R;
     const int pos = n - a.L_obs + (row_ok ? r / a.G : 0);  // the row's own position: it sees keys j <= pos
     const int n_sc = n - a.L_obs;                           // keys below are scored keys
-    // The kWaSub threads of a row keep the same reference: each tile they exchange the maxima of their parts through
-    // shared memory and take the same decision.  The exchange is off the critical path: P is formed against the
-    // reference as it stands while the maxima travel, and only when the tile's maximum turns out to exceed it by more
-    // than 2^kWaTau (rare after the first tiles) is the tile reread from TMEM and P formed again.  Sums stay per thread.
-    float ref = -INFINITY, l = 0.f, lsc = 0.f;
+    const uint32_t s_slot = tmem + lane_base + (uint32_t)(g * 128 + half * 64);
+    float* xch_mine = s_xch + (g * 2 + half) * 128 + lane_row;
+    const float* xch_other = s_xch + (g * 2 + (half ^ 1)) * 128 + lane_row;
+    // The four threads of a row (two groups x two halves) share one reference, kept in shared memory: the decision
+    // for tile t (does the reference move?) follows the decision for tile t - 1 of the other group, but only the
+    // short decision is serial: the exponentials of a tile run while the other group is at work on the next one.
+    float my_ref = -INFINITY, l = 0.f, lsc = 0.f;  // this thread's sums and the reference they are relative to
     bool alive = true;
-    for (int t = 0; t < n_tiles; ++t) {
-      const int st = t & 1;
-      if (!mbar_wait(bar_done_s + 8 * st, (uint32_t)((t >> 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
+    for (int t = g; t < n_tiles; t += 2) {
+      const int use = t >> 1;
+      if (!mbar_wait(B(kDoneS + g), (uint32_t)(use & 1), s_abort, a.spin_limit)) { alive = false; break; }
       tc_fence_after();
-      const uint32_t s_addr = tmem + lane_base + (uint32_t)(st * 128 + sub * kWaCols);
-      const int jb = j_lo + t * kKeyTile + sub * kWaCols;  // key of x[0]
-      const bool edge = jb + kWaCols - 1 >= n_sc;           // uniform: the block reaches the window's own keys (or the end)
-      float x[kWaCols];
-      auto load_logits = [&]() {
-        tmem_ld32(s_addr, x);
+      const int jb = j_lo + t * kKeyTile + half * 64;  // key of this thread's first column
+      const bool edge = jb + 63 >= n_sc;               // uniform: the block reaches the window's own keys (or the end)
+      // ---- pass 1: this thread's maximum over the keys its row sees, exchanged with the other half
+      float mx = -INFINITY;
+#pragma unroll
+      for (int blk = 0; blk < 2; ++blk) {
+        float x[32];
+        tmem_ld32(s_slot + blk * 32, x);
         tmem_wait_ld32(x);
         if (edge) {
 #pragma unroll
-          for (int c = 0; c < kWaCols; ++c) x[c] = (jb + c <= pos) ? x[c] : -INFINITY;
+          for (int c = 0; c < 32; ++c) x[c] = (jb + blk * 32 + c <= pos) ? x[c] : -INFINITY;
         }
-      };
-      float sum = 0.f;
-      auto form_p = [&]() {  // x: logits -> P against `ref`; sum: their total
-        const float nref_neg = ref > -INFINITY ? -ref : -INFINITY;  // no reference yet: every P is exp2(-inf) = 0
+        mx = fmaxf(mx, max32(x));
+      }
+      if (use >= 1 && !mbar_wait(B(kXr + g * 4 + quarter), (uint32_t)((use - 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
+      *xch_mine = mx;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(B(kXw + g * 4 + quarter));
+      if (!mbar_wait(B(kXw + g * 4 + quarter), (uint32_t)(use & 1), s_abort, a.spin_limit)) { alive = false; break; }
+      mx = fmaxf(mx, *xch_other);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(B(kXr + g * 4 + quarter));  // read: after both halves, the slots may be rewritten
+      mx = row_ok ? mx * a.scale_log2 : -INFINITY;  // the scale is positive: the max commutes with it
+      // ---- the decision, after the other group's for the tile before
+      if (t >= 1 && !mbar_wait(B(kDec), (uint32_t)((t - 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
+      // (two copies by tile parity: this tile reads the one the tile before wrote and writes the other, so the two
+      // halves of a row never race on it)
+      const float ref_old = s_ref[((t & 1) ^ 1) * 128 + lane_row];
+      const bool grow = mx > ref_old + kWaTau;  // also the first tile with a visible key (reference -inf)
+      const float ref = grow ? mx : ref_old;
+      const bool rescale = grow && ref_old > -INFINITY;
+      if (half == 0) s_ref[(t & 1) * 128 + lane_row] = ref;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(B(kDec));
+      if (__any_sync(0xffffffffu, rescale)) {
+        // O moves to the new reference before this tile's P V is issued; the P V of the tile before must be done
+        if (!mbar_wait(B(kPvDone), (uint32_t)((t - 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
+        tc_fence_after();
+        const float factor = rescale ? fast_exp2(ref_old - ref) : 1.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < 64; c0 += 32) {
+          float o[32];
+          tmem_ld32(tmem + lane_base + (uint32_t)(kWaOCol + half * 64 + c0), o);
+          tmem_wait_ld32(o);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] *= factor;
+          tmem_st32(tmem + lane_base + (uint32_t)(kWaOCol + half * 64 + c0), o);
+        }
+        tmem_wait_st();
+      }
+      if (ref > my_ref) {  // this thread's sums move to the reference in force
+        const float f = my_ref > -INFINITY ? fast_exp2(my_ref - ref) : 0.f;
+        l *= f;
+        lsc *= f;
+        my_ref = ref;
+      }
+      // ---- pass 2: P = exp2(logit - reference) per 32-key block, written over the block's own columns of S
+      const float nref_neg = ref > -INFINITY ? -ref : -INFINITY;  // no reference yet: every P is exp2(-inf) = 0
+#pragma unroll
+      for (int blk = 0; blk < 2; ++blk) {
+        float x[32];
+        tmem_ld32(s_slot + blk * 32, x);
+        tmem_wait_ld32(x);
+        if (edge) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) x[c] = (jb + blk * 32 + c <= pos) ? x[c] : -INFINITY;
+        }
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-        for (int c = 0; c < kWaCols; c += 4) {
+        for (int c = 0; c < 32; c += 4) {
           x[c] = fast_exp2(fmaf(x[c], a.scale_log2, nref_neg));
           x[c + 1] = fast_exp2(fmaf(x[c + 1], a.scale_log2, nref_neg));
           x[c + 2] = fast_exp2(fmaf(x[c + 2], a.scale_log2, nref_neg));
@@ -235,101 +309,50 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
           s2 += x[c + 2];
           s3 += x[c + 3];
         }
-        sum = (s0 + s1) + (s2 + s3);
-      };
-      load_logits();
-      // ---- this thread's maximum over the keys its row sees goes to the row's other threads
-      float m0 = fmax3(x[0], x[1], x[2]), m1 = fmax3(x[3], x[4], x[5]);
-      float m2 = fmax3(x[6], x[7], x[8]), m3 = fmax3(x[9], x[10], x[11]);
+        const float sum = (s0 + s1) + (s2 + s3);
+        float ssc = sum;
+        if (edge) {  // a branch of its own (the condition is uniform), so that ordinary tiles do not carry this code
+          ssc = 0.f;
 #pragma unroll
-      for (int c = 12; c < 28; c += 8) {
-        m0 = fmax3(m0, x[c], x[c + 1]);
-        m1 = fmax3(m1, x[c + 2], x[c + 3]);
-        m2 = fmax3(m2, x[c + 4], x[c + 5]);
-        m3 = fmax3(m3, x[c + 6], x[c + 7]);
+          for (int c = 0; c < 32; ++c) ssc += (jb + blk * 32 + c < n_sc) ? x[c] : 0.f;
+        }
+        l += sum;
+        lsc += ssc;
+        uint32_t ph[16], pl[16];  // the block's probabilities as bf16 hi + lo pairs
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          // hi = the upper 16 bits (a byte permute, no conversion; p - hi is exact in fp32), lo = p - hi rounded to bf16:
+          // hi + lo carries 16 significant bits of p
+          const uint32_t b0 = __float_as_uint(x[c]), b1 = __float_as_uint(x[c + 1]);
+          ph[c / 2] = __byte_perm(b0, b1, 0x7632);
+          pl[c / 2] = pack_bf16(x[c] - __uint_as_float(b0 & 0xffff0000u), x[c + 1] - __uint_as_float(b1 & 0xffff0000u));
+        }
+        tmem_st16u(s_slot + blk * 32, ph);
+        tmem_st16u(s_slot + blk * 32 + 16, pl);
       }
-      m0 = fmax3(m0, x[28], x[29]);
-      m1 = fmax3(m1, x[30], x[31]);
-      float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-      // (bounded mbarrier waits, not a named barrier: a partner that has given up must not leave this warp waiting)
-      if (t >= 1 && !mbar_wait(bar_xr + 8 * quarter, (uint32_t)((t - 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
-      s_xch[sub * 128 + lane_row] = mx;
+      tmem_wait_st();
+      tc_fence_before();  // P (and a rescaled O) before the MMAs that read them
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_xw + 8 * quarter);
-      // ---- P against the reference as it stands, while the maxima travel
-      form_p();
-      if (!mbar_wait(bar_xw + 8 * quarter, (uint32_t)(t & 1), s_abort, a.spin_limit)) { alive = false; break; }
-#pragma unroll
-      for (int k = 0; k < kWaSub; ++k) mx = fmaxf(mx, s_xch[k * 128 + lane_row]);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_xr + 8 * quarter);  // this warp has read: after all, the slots may be rewritten
-      mx = row_ok ? mx * a.scale_log2 : -INFINITY;  // the scale is positive: the max commutes with it
-      const bool grow = mx > ref + kWaTau;  // also the first tile with a visible key (ref = -inf)
-      const bool rescale = grow && ref > -INFINITY;
-      const float factor = rescale ? fast_exp2(ref - mx) : 1.f;
-      if (__any_sync(0xffffffffu, grow)) {  // the same lanes in all the warps of the quarter: the tile once more
-        ref = grow ? mx : ref;
-        load_logits();
-        form_p();
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_free_s + 8 * st);  // the S slot goes back to the MMA warp
-      float ssc = sum;
-      if (edge) {  // a branch of its own (the condition is uniform), so that ordinary tiles do not carry this code
-        ssc = 0.f;
-#pragma unroll
-        for (int c = 0; c < kWaCols; ++c) ssc += (jb + c < n_sc) ? x[c] : 0.f;
-      }
-      l = l * factor + sum;
-      lsc = lsc * factor + ssc;
-      uint32_t ph[kWaCols / 2], pl[kWaCols / 2];  // the probabilities as bf16 hi + lo pairs
-#pragma unroll
-      for (int c = 0; c < kWaCols; c += 2) {
-        // hi = the upper 16 bits (a byte permute, no conversion; p - hi is exact in fp32), lo = p - hi rounded to bf16:
-        // hi + lo carries 16 significant bits of p.
-        const uint32_t b0 = __float_as_uint(x[c]), b1 = __float_as_uint(x[c + 1]);
-        ph[c / 2] = __byte_perm(b0, b1, 0x7632);
-        pl[c / 2] = pack_bf16(x[c] - __uint_as_float(b0 & 0xffff0000u), x[c + 1] - __uint_as_float(b1 & 0xffff0000u));
-      }
-      // All of the above ran under the previous tile's P V; that must have completed before O is touched and the
-      // P buffer rewritten
-      if (t >= 1 && !mbar_wait(bar_p_free, (uint32_t)((t - 1) & 1), s_abort, a.spin_limit)) { alive = false; break; }
-      if (__any_sync(0xffffffffu, rescale)) {  // this thread's columns of its row of O
-        tc_fence_after();
-        float o[32];
-        tmem_ld32(tmem + lane_base + (uint32_t)(kWaOCol + sub * kWaCols), o);
-        tmem_wait_ld32(o);
-#pragma unroll
-        for (int c = 0; c < 32; ++c) o[c] *= factor;
-        tmem_st32(tmem + lane_base + (uint32_t)(kWaOCol + sub * kWaCols), o);
-        tmem_wait_st();
-      }
-#pragma unroll
-      for (int c = 0; c < kWaCols; c += 8) {
-        const uint32_t off = sw128_off(lane_row, sub * (kWaCols / 8) + (c >> 3), 128);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(s_ph + off), "r"(ph[c / 2]), "r"(ph[c / 2 + 1]), "r"(ph[c / 2 + 2]), "r"(ph[c / 2 + 3]) : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(s_pl + off), "r"(pl[c / 2]), "r"(pl[c / 2 + 1]), "r"(pl[c / 2 + 2]), "r"(pl[c / 2 + 3]) : "memory");
-      }
-      fence_async_smem();  // generic-proxy writes of P before the async-proxy reads of the MMAs
-      tc_fence_before();   // the rescaled O before the MMAs that accumulate into it
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_p_ready);  // the MMA warp may issue this tile's P V
+      if (lane == 0) mbar_arrive(B(kPReady + g));  // the MMA warp may issue this tile's P V
     }
-    // ---- the CTA's partial result: this thread's row, its columns of O, and its share of the row's state
-    if (alive && mbar_wait(bar_done_o, 0u, s_abort, a.spin_limit)) {
+    // ---- the CTA's partial result: this thread's row, 32 of the 128 d, and its sums relative to the final reference
+    if (alive && mbar_wait(B(kDec), (uint32_t)((n_tiles - 1) & 1), s_abort, a.spin_limit) &&
+        mbar_wait(B(kDoneO), 0u, s_abort, a.spin_limit)) {
       tc_fence_after();
+      const int sub = g * 2 + half;
+      const float ref_end = s_ref[((n_tiles - 1) & 1) * 128 + lane_row];
+      const float f = (my_ref > -INFINITY && ref_end > my_ref) ? fast_exp2(my_ref - ref_end) : 1.f;
       float o[32];
-      tmem_ld32(tmem + lane_base + (uint32_t)(kWaOCol + sub * kWaCols), o);
+      tmem_ld32(tmem + lane_base + (uint32_t)(kWaOCol + sub * 32), o);
       tmem_wait_ld32(o);
       const size_t cta = ((size_t)blockIdx.y * gridDim.z + mt) * a.n_chunks + blockIdx.x;
-      float* dst = a.part + (cta * 128 + lane_row) * 128 + sub * kWaCols;
+      float* dst = a.part + (cta * 128 + lane_row) * 128 + sub * 32;
 #pragma unroll
       for (int c = 0; c < 32; c += 4) *reinterpret_cast<float4*>(dst + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
       float* ds = a.part_s + cta * (kWaStateWords * 128);
-      if (sub == 0) ds[lane_row] = ref;
-      ds[(1 + sub) * 128 + lane_row] = l;
-      ds[(1 + kWaSub + sub) * 128 + lane_row] = lsc;
+      if (sub == 0) ds[lane_row] = ref_end;
+      ds[(1 + sub) * 128 + lane_row] = l * f;
+      ds[(1 + kWaSub + sub) * 128 + lane_row] = lsc * f;
     }
   }
 
@@ -404,7 +427,6 @@ __global__ void __launch_bounds__(128) window_reduce_kernel(const float* part, c
   }
 }
 
-static_assert(kWaCols == 32, "the epilogue is written for 32 columns per thread");
 
 struct WaWs {
   size_t off_status, off_jobs, off_part, off_part_s, bytes;
