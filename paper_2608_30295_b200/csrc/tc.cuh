@@ -113,6 +113,17 @@ __device__ __forceinline__ void umma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, u
       "r"(tmem_a), "l"(db), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same with the B descriptor handed over as its two 32-bit halves: the high half of a descriptor is a constant of
+// the layout and the low half is the start address >> 4 plus constants, so a loop over k-steps and stages advances
+// it with one 32-bit add (the issuing thread is alone in its warp: every instruction it saves shortens the chain).
+__device__ __forceinline__ void umma_bf16_ta_lohi(uint32_t tmem_d, uint32_t tmem_a, uint32_t db_lo, uint32_t db_hi, uint32_t idesc,
+                                                  uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n .reg .b64 db;\n mov.b64 db, {%2, %3};\n setp.ne.b32 p, %5, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}\n" ::"r"(tmem_d),
+      "r"(tmem_a), "r"(db_lo), "r"(db_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // store 16 consecutive TMEM columns of this thread's lane as raw words (asynchronous: tmem_wait_st before anything depends on it)
 __device__ __forceinline__ void tmem_st16u(uint32_t taddr, const uint32_t (&v)[16]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"

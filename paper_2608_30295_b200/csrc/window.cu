@@ -4,7 +4,8 @@
 // of the token-criticality line.  catekv_select_compact takes the latter in place of its own first pass over K.
 //
 // One sweep over K and V.  window_pv_kernel: a CTA owns a range of keys of one (sequence, KV head) and 128 query
-// rows.  Per 128-key tile: S = Q K^T (tcgen05.mma into one of two TMEM slots); an epilogue thread owns a query row
+// rows, which it keeps in tensor memory.  Per 128-key tile: S = Q K^T (tcgen05.mma with Q as the A operand from
+// TMEM, so that only the K tile is fetched from shared memory, into one of two TMEM slots); an epilogue thread owns a query row
 // and 64 of the tile's keys: it finds their maximum, the row's threads agree on the row's reference value, and it
 // turns its part of S into P = exp2(logit - ref), adds the row sums (all visible keys; scored keys only) and writes P
 // back over the same TMEM columns as a bf16 hi + lo pair (hi in the first 16 of every 32 columns, lo in the last 16,
@@ -15,7 +16,7 @@
 // issued.  The ranges' partial results (O, reference, sums) are merged in range order by window_reduce_kernel,
 // which also writes the two log-sum-exps.
 //
-// Warp roles: warps 17 and 18 (one lane each) feed the three K stages and the two V stages by TMA; warp 16 (one
+// Warp roles: warps 17 and 18 (one lane each) feed the three K stages and the three V stages by TMA; warp 16 (one
 // lane) issues every MMA: S(0), S(1), then per tile P V(t) followed by S(t + 2) into the slot P V(t) has just read
 // (the tensor pipe keeps issue order); warps 0-15 are the epilogue, two groups of eight (two warps per TMEM lane
 // quarter: 64 keys each) that take alternate tiles in alternate slots, so that one group's exponentials overlap the
@@ -36,14 +37,14 @@ namespace catekv {
 constexpr int kWaEpiWarps = 16;                     // two groups of eight: two warps per TMEM lane quarter and group
 constexpr int kWaSub = 4;                           // epilogue threads per query row (2 groups x 2 halves)
 constexpr int kWaThreads = (kWaEpiWarps + 3) * 32;  // + the MMA warp and the two TMA warps (K, V)
-constexpr int kWaKStages = 3, kWaVStages = 2;
-constexpr int kWaTmemCols = 512;         // S / P slots at columns 0 and 128, O at 256
-constexpr int kWaOCol = 256;
-constexpr int kWaTileBytes = 128 * 256;  // a [128 x 128] bf16 tile: the Q rows, a K or V stage
+constexpr int kWaKStages = 3, kWaVStages = 3;
+constexpr int kWaTmemCols = 512;         // S / P slots at columns 0 and 128, O at 256, Q (bf16, two per column) at 384
+constexpr int kWaOCol = 256, kWaQCol = 384;
+constexpr int kWaTileBytes = 128 * 256;  // a [128 x 128] bf16 tile: a K or V stage
 constexpr int kWaStateWords = 1 + 2 * kWaSub;  // per row and key range: reference, the threads' sums (visible keys), (scored keys)
 constexpr float kWaTau = 8.f;            // a row's reference follows a tile maximum that exceeds it by more than 2^kWaTau
 constexpr int kWaBarriers = 36;
-constexpr size_t kWaSmemBytes = 1024 + (size_t)(1 + kWaKStages + kWaVStages) * kWaTileBytes + (4 * 128 + 256) * sizeof(float) +
+constexpr size_t kWaSmemBytes = 1024 + (size_t)(kWaKStages + kWaVStages) * kWaTileBytes + (4 * 128 + 256) * sizeof(float) +
                                 kWaBarriers * sizeof(uint64_t) + 16;
 static_assert(kWaSmemBytes <= 227 * 1024, "window_pv_kernel: one CTA's shared memory");
 
@@ -90,10 +91,9 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
 
   const uint32_t s_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (s_base - smem_u32(smem_raw));
-  const uint32_t s_q = s_base;
-  const uint32_t s_k = s_q + kWaTileBytes;
+  const uint32_t s_k = s_base;
   const uint32_t s_v = s_k + kWaKStages * kWaTileBytes;
-  float* s_xch = reinterpret_cast<float*>(smem + (1 + kWaKStages + kWaVStages) * kWaTileBytes);  // [group][half][row]: part-tile maxima
+  float* s_xch = reinterpret_cast<float*>(smem + (kWaKStages + kWaVStages) * kWaTileBytes);  // [group][half][row]: part-tile maxima
   float* s_ref = s_xch + 4 * 128;  // [tile parity][row]: the row's reference after the decision for a tile of that parity
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_ref + 256);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + kWaBarriers);
@@ -101,20 +101,12 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   const uint32_t bar0 = smem_u32(s_bar);
   auto B = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   // barrier indices
-  constexpr int kFullK = 0, kEmptyK = 3, kFullV = 6, kEmptyV = 8, kDoneS = 10, kPReady = 12, kPvDone = 14, kDoneO = 15, kDec = 16,
-                kXw = 17, kXr = 25;  // kXw / kXr: [group][quarter]
+  constexpr int kFullK = 0, kEmptyK = 3, kFullV = 6, kEmptyV = 9, kDoneS = 12, kPReady = 14, kPvDone = 16, kDoneO = 17, kDec = 18,
+                kXw = 19, kXr = 27;  // kXw / kXr: [group][quarter]
   static_assert(kXr + 8 <= kWaBarriers, "barrier table");
 
-  // ---- set-up: this M tile's query rows (row r = i * G + g), the row references, barriers, tensor memory
-  for (int id = tid; id < 128 * 16; id += kWaThreads) {
-    const int row = id >> 4, c = id & 15;
-    const int r = mt * 128 + row;
-    const int ok = r < a.R ? 16 : 0;
-    const int i = ok ? r / a.G : 0, g = ok ? r - i * a.G : 0;
-    const uint16_t* src = a.q_win + (((int64_t)job.b * a.Hq + job.h * a.G + g) * a.L_obs + i) * kD + c * 8;
-    cp_async16(s_q + sw128_off(row, c, 128), src, ok);
-  }
-  cp_async_commit();
+  // ---- set-up: the row references, barriers, tensor memory; then this M tile's query rows (row r = i * G + g) go
+  // into tensor memory, where the S MMAs take them as their A operand (lane = row, two bf16 per column)
   for (int row = tid; row < 256; row += kWaThreads) s_ref[row] = -INFINITY;
   if (tid == 0) {
     *s_abort = 0;
@@ -129,12 +121,33 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(s_tmem)), "r"(kWaTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
-  cp_async_wait<0>();
-  fence_async_smem();  // Q was written through the generic proxy; the MMAs read it through the async proxy
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
+  if (warp < kWaEpiWarps) {
+    // four threads per row, 32 of its 128 values (16 columns) each
+    const int row = (warp & 3) * 32 + lane, part = warp >> 2;
+    const int r = mt * 128 + row;
+    uint32_t w[16];
+    if (r < a.R) {
+      const int i = r / a.G, g = r - i * a.G;
+      const uint4* src = reinterpret_cast<const uint4*>(a.q_win + (((int64_t)job.b * a.Hq + job.h * a.G + g) * a.L_obs + i) * kD + part * 32);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const uint4 v = __ldg(src + c);
+        w[4 * c] = v.x, w[4 * c + 1] = v.y, w[4 * c + 2] = v.z, w[4 * c + 3] = v.w;
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < 16; ++c) w[c] = 0u;
+    }
+    tmem_st16u(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(kWaQCol + part * 16), w);
+    tmem_wait_st();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
 
   if (warp == kWaEpiWarps + 1) {
     // ================= TMA producer, K: three stages, refilled as soon as the S that read one has completed
@@ -150,7 +163,7 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
     }
     __syncwarp();
   } else if (warp == kWaEpiWarps + 2) {
-    // ================= TMA producer, V: two stages, refilled when the P V that read one has completed
+    // ================= TMA producer, V: three stages, refilled when the P V that read one has completed
     if (lane == 0 && !a.idle_producer) {
       for (int t = 0; t < n_tiles; ++t) {
         const int st = t % kWaVStages, use = t / kWaVStages;
@@ -165,18 +178,22 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
   } else if (warp == kWaEpiWarps) {
     // ================= MMA issue: S(0), S(1), then per tile P V(t) and S(t + 2) into the slot P V(t) has just read
     if (lane == 0 && !a.idle_producer) {
-      const uint32_t idesc_s = umma_idesc_bf16(128, 128);      // S[rows x keys]: A = Q, B = K, both K-major
+      const uint32_t idesc_s = umma_idesc_bf16(128, 128);      // S[rows x keys]: A = Q (in TMEM), B = K (K-major)
       const uint32_t idesc_o = umma_idesc_bf16_bmn(128, 128);  // O[rows x d]: A = P (in TMEM), B = V (MN-major)
+      // B descriptors as (low, high) halves: high is constant, low = (address >> 4) + constants
+      const uint64_t dk0 = umma_desc_sw128(s_k), dv0 = umma_desc_sw128_mn(s_v, kKBlockBytes);
+      const uint32_t dk_hi = (uint32_t)(dk0 >> 32), dv_hi = (uint32_t)(dv0 >> 32);
+      const uint32_t dk_lo0 = (uint32_t)dk0, dv_lo0 = (uint32_t)dv0;
       auto issue_s = [&](int t) -> bool {
         const int st = t % kWaKStages;
         if (!mbar_wait(B(kFullK + st), (uint32_t)((t / kWaKStages) & 1), s_abort, a.spin_limit)) return false;
         tc_fence_after();
-        const uint32_t sk = s_k + st * kWaTileBytes;
+        const uint32_t lo = dk_lo0 + (uint32_t)(st * (kWaTileBytes >> 4));
+        const uint32_t d = tmem + (uint32_t)((t & 1) * 128);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t off = (kk >> 2) * kKBlockBytes + (kk & 3) * 32;
-          umma_bf16(tmem + (uint32_t)((t & 1) * 128), umma_desc_sw128(s_q + off), umma_desc_sw128(sk + off), idesc_s, kk ? 1u : 0u);
-        }
+        for (int kk = 0; kk < 8; ++kk)  // 16 of the 128 head dimensions per step: 8 columns of Q in TMEM, 32 bytes of every K row
+          umma_bf16_ta_lohi(d, tmem + (uint32_t)(kWaQCol + kk * 8), lo + (uint32_t)((kk >> 2) * (kKBlockBytes >> 4) + (kk & 3) * 2),
+                            dk_hi, idesc_s, kk ? 1u : 0u);
         umma_commit(B(kDoneS + (t & 1)));
         umma_commit(B(kEmptyK + st));
         return true;
@@ -187,18 +204,17 @@ __global__ void __launch_bounds__(kWaThreads, 1) window_pv_kernel(const __grid_c
         if (!mbar_wait(B(kPReady + g), (uint32_t)((t >> 1) & 1), s_abort, a.spin_limit)) break;
         if (!mbar_wait(B(kFullV + sv_st), (uint32_t)((t / kWaVStages) & 1), s_abort, a.spin_limit)) break;
         tc_fence_after();
-        const uint32_t sv = s_v + sv_st * kWaTileBytes;
+        const uint32_t lo = dv_lo0 + (uint32_t)(sv_st * (kWaTileBytes >> 4));
         const uint32_t slot = tmem + (uint32_t)(g * 128);
+        const uint32_t first = t ? 1u : 0u;
         // P of the 32-key block b of the tile sits in the block's own 32 columns of the slot: hi in the first 16
-        // (two bf16 per column), lo in the last 16; a k-step is 16 keys = 8 columns
+        // (two bf16 per column), lo in the last 16; a k-step is 16 keys = 8 columns of P and 2 KB of the V tile
 #pragma unroll
         for (int part = 0; part < 2; ++part) {
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t acol = (uint32_t)((kk >> 1) * 32 + part * 16 + (kk & 1) * 8);
-            umma_bf16_ta(tmem + kWaOCol, slot + acol, umma_desc_sw128_mn(sv + kk * 2048, kKBlockBytes), idesc_o,
-                         (t | part | kk) ? 1u : 0u);
-          }
+          for (int kk = 0; kk < 8; ++kk)
+            umma_bf16_ta_lohi(tmem + kWaOCol, slot + (uint32_t)((kk >> 1) * 32 + part * 16 + (kk & 1) * 8), lo + (uint32_t)(kk * 128), dv_hi,
+                              idesc_o, (part | kk) ? 1u : first);
         }
         umma_commit(B(kPvDone));
         umma_commit(B(kEmptyV + sv_st));
