@@ -142,16 +142,6 @@ __host__ __device__ inline SelSeg retrieval_decide(int n, bool enabled, const Re
   return d;
 }
 
-// Monotone map of arbitrary finite floats to non-negative floats whose bit patterns order the same way as the
-// values (what the radix select of the top-k kernel needs): flip so that larger values get larger unsigned
-// patterns, then clear the sign by halving the range.  Values one ulp apart may merge into a tie: within the
-// parity tolerance band.
-__device__ __forceinline__ float monotone_key(float x) {
-  const uint32_t u = __float_as_uint(x);
-  const uint32_t k = (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // unsigned order == float order
-  return __uint_as_float(k >> 1);                                 // non-negative pattern
-}
-
 // bound(c, g) = [kmax_c | kmin_c] . [max(q_g, 0) | min(q_g, 0)]: a [chunks x 256] x [256 x 8 heads] product, so the
 // tensor cores take it (mma.m16n8k16, chunks are M, the group's heads N = 8).  A CTA streams 64-chunk tiles of the
 // metadata (32 KB, contiguous) through a 3-stage cp.async pipeline into XOR-swizzled shared memory; each of its 4
@@ -462,6 +452,7 @@ static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t ch
   ta.L_obs = 0;
   ta.pool_mode = kPoolPrescored;
   ta.pool_param = cs;
+  ta.row_is_seg = 1;  // retrieval_score_kernel writes the scores of segment s to row s
   int n_masked = 0;
   for (int s = 0; s < n_segs; ++s) n_masked += retrieval_mask[s] != 0;
   rc = launch_topk(ta, n_segs, max_pool, n_masked, st);

@@ -49,6 +49,32 @@ __device__ __forceinline__ unsigned long long block_excl_scan(unsigned long long
   return res;
 }
 
+// Pooled entry c of segment seg is the rnk-th selected one: its tokens go to slot rnk of the kept list (cs tokens
+// per slot; the last chunk of the range may be short).
+__device__ __forceinline__ void topk_emit(const TopkArgs& a, const SelSeg& s, int seg, int32_t* idx, int cs, int c,
+                                          unsigned int rnk) {
+  const int S = a.sink;
+#ifdef CATEKV_CHECKED
+  // the rank must be one of the k_sel slots and the list position inside the segment's row of idx
+  rnk = (unsigned int)checked_clamp((int)rnk, 0, s.k_sel - 1, a.chk, kKidTopk, seg);
+  if ((int64_t)S + ((int64_t)rnk + 1) * cs > a.idx_stride) {
+    raise_status(a.chk, CATEKV_STATUS_INDEX_RANGE, kKidTopk, seg, (int)rnk);
+    return;
+  }
+#endif
+  if (cs == 1) {
+    idx[S + rnk] = S + c;
+  } else {
+    const int l2 = S + c * cs, h2 = min(l2 + cs, s.cand_end);
+    int32_t* dst = idx + S + (size_t)rnk * cs;
+    if ((cs & 3) == 0 && h2 - l2 == cs && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+      for (int u = 0; u < cs; u += 4) *reinterpret_cast<int4*>(dst + u) = make_int4(l2 + u, l2 + u + 1, l2 + u + 2, l2 + u + 3);
+    } else {
+      for (int u = l2; u < h2; ++u) dst[u - l2] = u;
+    }
+  }
+}
+
 // One thread-block cluster of CL CTAs (1 or 8) per segment that selects: pooling, radix select of the k-th largest
 // pooled score, ordered compaction into the ascending kept list.  Every CTA owns a contiguous share of the pooled
 // entries.  The CTAs meet only through distributed shared memory: the per-pass digit histograms and the per-CTA
@@ -240,22 +266,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
     // an exclusive scan over the block (plus the totals of the CTAs before this one) says where its selected
     // entries go, and it writes them in order.
     const int cs = (a.pool_mode == CATEKV_POOL_CHUNK || a.pool_mode == kPoolPrescored) ? a.pool_param : 1;
-    auto emit = [&](int c, unsigned int rnk) {  // pooled entry c of the segment is the rnk-th selected one
-#ifdef CATEKV_CHECKED
-      // the rank must be one of the k_sel slots and the list position inside the segment's row of idx
-      rnk = (unsigned int)checked_clamp((int)rnk, 0, s.k_sel - 1, a.chk, kKidTopk, seg);
-      if ((int64_t)S + ((int64_t)rnk + 1) * cs > a.idx_stride) {
-        raise_status(a.chk, CATEKV_STATUS_INDEX_RANGE, kKidTopk, seg, (int)rnk);
-        return;
-      }
-#endif
-      if (cs == 1) {
-        idx[S + rnk] = S + c;
-      } else {
-        const int l2 = S + c * cs, h2 = min(l2 + cs, s.cand_end);
-        for (int u = l2; u < h2; ++u) idx[S + rnk * cs + (u - l2)] = u;
-      }
-    };
+    auto emit = [&](int c, unsigned int rnk) { topk_emit(a, s, seg, idx, cs, c, rnk); };
     unsigned long long all = 0;  // packed: low = entries above the threshold, high = entries equal to it
     if (staged) {
       const int E = (n_loc + kTopkThreads - 1) / kTopkThreads;
@@ -345,6 +356,257 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
   }
 }
 
+// ---- short prescored lists (the per-step retrieval: a few thousand chunk scores per segment) -------------------------
+// One CTA per segment, the whole list in shared memory, thread t owning entries t, t + 1024, ...  The kernel runs
+// once per segment on a cold instruction cache, so every loop over a thread's entries stays rolled: the steps are
+//   1. a 1024-bin histogram over the scores mapped linearly between the extremes of the first 1024 entries (monotone
+//      in the score, and spread over the bins where the scores are: their bit patterns crowd into a few exponents),
+//      a suffix scan (thread t owns bin 1023 - t) finds the bin that holds the k-th largest entry;
+//   2. that bin's entries (a few, as a rule) are ranked against one another by (score descending, index ascending):
+//      the k-th entry's pattern is the threshold and the rank gives the number of ties to take;
+//   3. more than kTsRank entries in the bin (many equal or nearly equal scores): histogram passes over their bit
+//      patterns, 10 bits at a time between the extremes of what is left, until the bin is resolved or small;
+//   4. ordered compaction: the warps' votes give one bitmap of the entries above the threshold and one of those at
+//      it; thread t takes word t of both (32 consecutive entries), one scan over the counts, the writes.
+// Per entry two flags live in registers: above the threshold for sure (gtm), still a candidate (cand).
+constexpr int kTsPer = 16;     // entries a thread may own
+constexpr int kTsBins = 1024;  // == kTopkThreads: one bin per thread in the scan
+constexpr int kTsRank = 256;   // candidates resolved by ranking
+constexpr int kTopkSmallMax = kTsPer * kTopkThreads;
+
+__global__ void __launch_bounds__(kTopkThreads) topk_small_kernel(const TopkArgs a) {
+  __shared__ unsigned int hist[kTsBins];
+  __shared__ unsigned int s_gt[kTopkSmallMax / 32], s_eq[kTopkSmallMax / 32];
+  __shared__ unsigned int s_tot[32];
+  __shared__ unsigned int s_mm[2];
+  __shared__ unsigned int s_sel[3];
+  __shared__ unsigned int s_ncand;
+  __shared__ unsigned int s_cv[kTsRank];
+  __shared__ int s_ci[kTsRank];
+  __shared__ unsigned int s_thr[2];
+  __shared__ int s_last;
+  extern __shared__ __align__(16) unsigned int sv[];  // the list (small_pool entries, rounded up to 4), then its digits
+  unsigned short* sd = reinterpret_cast<unsigned short*>(sv + (a.small_pool + 3) / 4 * 4);
+  const int seg = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
+  hist[tid] = 0;
+  (tid < 512 ? s_gt : s_eq)[tid & 511] = 0u;
+  if (tid == 0) {
+    s_mm[0] = 0xffffffffu;
+    s_mm[1] = 0u;
+    s_ncand = 0u;
+    s_last = 0;
+    s_sel[0] = 0u, s_sel[1] = 1u, s_sel[2] = 1u;
+  }
+  pdl_wait();  // the decisions and the scores come from earlier kernels of the stream
+  // The scores are requested before the decision has arrived: entries past the list's end are masked out below
+  // (they lie inside the row, whose stride covers small_pool entries rounded up to 4).
+  const unsigned int* Pg = reinterpret_cast<const unsigned int*>(a.P + (size_t)seg * a.c_stride);
+  {
+    const uint32_t sv_addr = smem_u32(sv);
+#pragma unroll 1
+    for (int i = tid * 4; i < a.small_pool; i += 4 * kTopkThreads) cp_async16(sv_addr + i * 4, Pg + i, 16);
+    cp_async_commit();
+  }
+  const SelSeg s = a.segs[seg];
+  if (s.keep_all) {
+    cp_async_wait<0>();
+    if (a.mark_keep_all && tid == 0) a.seg_len_dev[seg] = -1;
+    return;
+  }
+  int32_t* idx = a.idx + (size_t)seg * a.idx_stride;
+  const int S = a.sink, cs = a.pool_param;
+  const int E = (s.n_pool + kTopkThreads - 1) / kTopkThreads;  // entries of the busiest thread (<= kTsPer)
+  int n_sel_tokens = 0;
+  cp_async_wait<0>();
+  __syncthreads();  // the list is in shared memory; the histogram and the extremes are initialised
+  if (s.k_sel > 0) {
+    unsigned int cand = 0u, gtm = 0u, need = (unsigned int)s.k_sel;
+    // The range of the first histogram comes from a sample, the first 1024 entries: scores outside it fall into
+    // the first or the last bin, which keeps the digits monotone (a crowded bin is resolved like any other).
+    unsigned int vmin = 0xffffffffu, vmax = 0u;
+    if (tid < s.n_pool) vmin = vmax = sv[tid];
+#pragma unroll 1
+    for (int e = 0; e < E; ++e)
+      if (e * kTopkThreads + tid < s.n_pool) cand |= 1u << e;
+    vmin = __reduce_min_sync(0xffffffffu, vmin);
+    vmax = __reduce_max_sync(0xffffffffu, vmax);
+    if (lane == 0) {
+      atomicMin(&s_mm[0], vmin);
+      atomicMax(&s_mm[1], vmax);
+    }
+    __syncthreads();
+    unsigned int base = s_mm[0];
+    unsigned int range = s_mm[1] - base;
+    {
+      bool linear = true;
+      const float xmin = key_to_score(base);
+      const float scale = (float)(kTsBins - 1) / (key_to_score(s_mm[1]) - xmin);
+      int shift = 0;
+      auto digit = [&](unsigned int val) -> int {
+        if (linear) {
+          // monotone in val, also when the sample's range is empty (scale infinite): a product that is not a number
+          // converts to 0, an infinite or negative one is clamped
+          const int d = (int)((key_to_score(val) - xmin) * scale);
+          return min(max(d, 0), kTsBins - 1);
+        }
+        return (int)((val - base) >> shift);
+      };
+      while (true) {
+#pragma unroll 1
+        for (int e = 0; e < E; ++e)
+          if ((cand >> e) & 1u) {
+            const int d = digit(sv[e * kTopkThreads + tid]);
+            sd[e * kTopkThreads + tid] = (unsigned short)d;
+            atomicAdd(&hist[d], 1u);
+          }
+        __syncthreads();
+        // suffix scan over the bins, larger digits first; every thread clears the bin it read for the next pass
+        const unsigned int cnt = hist[kTsBins - 1 - tid];
+        hist[kTsBins - 1 - tid] = 0u;
+        unsigned int inc = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned int y = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += y;
+        }
+        if (lane == 31) s_tot[warp] = inc;
+        if (tid == 0) {
+          s_mm[0] = 0xffffffffu;
+          s_mm[1] = 0u;
+        }
+        __syncthreads();
+        inc += __reduce_add_sync(0xffffffffu, lane < warp ? s_tot[lane] : 0u);
+        if (inc - cnt < need && need <= inc) {  // this thread's bin holds the need-th largest candidate
+          s_sel[0] = (unsigned int)(kTsBins - 1 - tid);
+          s_sel[1] = need - (inc - cnt);
+          s_sel[2] = cnt;
+        }
+        __syncthreads();
+        const int b = (int)s_sel[0];
+        need = s_sel[1];
+        const unsigned int m = s_sel[2];
+        const bool rank_it = m != need && !(!linear && shift == 0) && m <= (unsigned int)kTsRank;
+#pragma unroll 1
+        for (int e = 0; e < E; ++e)
+          if ((cand >> e) & 1u) {
+            const int d = sd[e * kTopkThreads + tid];
+            if (d > b) gtm |= 1u << e;
+            if (d != b) {
+              cand &= ~(1u << e);
+            } else if (rank_it) {  // the bin's entries are ranked against one another below
+              const unsigned int pos = atomicAdd(&s_ncand, 1u);
+              if (pos < (unsigned int)kTsRank) {
+                s_cv[pos] = sv[e * kTopkThreads + tid];
+                s_ci[pos] = e * kTopkThreads + tid;
+              }
+            }
+          }
+        if (m == need) break;              // the whole bin is taken
+        if (!linear && shift == 0) break;  // the bin is one bit pattern: need of its entries, lowest indices first
+        if (rank_it) {
+          __syncthreads();
+          if (tid < (int)m) {
+            const unsigned int mv = s_cv[tid];
+            const int mi = s_ci[tid];
+            unsigned int rank = 0, ties_before = 0;
+#pragma unroll 4
+            for (int j = 0; j < (int)m; ++j) {
+              const unsigned int vj = s_cv[j];
+              const bool tie_before = vj == mv && s_ci[j] < mi;
+              rank += (vj > mv) || tie_before;
+              ties_before += tie_before;
+            }
+            if (rank == need - 1u) {
+              s_thr[0] = mv;
+              s_thr[1] = ties_before + 1u;
+            }
+          }
+          __syncthreads();
+          const unsigned int thr = s_thr[0];
+          need = s_thr[1];
+#pragma unroll 1
+          for (int e = 0; e < E; ++e)
+            if ((cand >> e) & 1u) {
+              const unsigned int val = sv[e * kTopkThreads + tid];
+              if (val > thr) gtm |= 1u << e;
+              if (val != thr) cand &= ~(1u << e);
+            }
+          break;
+        }
+        // a crowded bin: go on with the bit patterns of what is left, between their extremes
+        unsigned int cmin = 0xffffffffu, cmax = 0u;
+#pragma unroll 1
+        for (int e = 0; e < E; ++e)
+          if ((cand >> e) & 1u) {
+            const unsigned int val = sv[e * kTopkThreads + tid];
+            cmin = min(cmin, val);
+            cmax = max(cmax, val);
+          }
+        cmin = __reduce_min_sync(0xffffffffu, cmin);
+        cmax = __reduce_max_sync(0xffffffffu, cmax);
+        if (lane == 0 && cmin <= cmax) {
+          atomicMin(&s_mm[0], cmin);
+          atomicMax(&s_mm[1], cmax);
+        }
+        __syncthreads();
+        base = s_mm[0];
+        range = s_mm[1] - base;
+        if (range == 0u) break;  // all that is left ties
+        linear = false;
+        shift = max(0, 32 - __clz(range) - 10);
+      }
+    }
+    // ---- ordered compaction: entries above the threshold (gtm) and the first `need` of those at it (cand).
+    // Warp w's entries of step e are the 32 consecutive entries of bitmap word e * 32 + w (the words were cleared
+    // at the start; few entries have a flag set).
+    for (unsigned int mk = gtm; mk; mk &= mk - 1u) atomicOr(&s_gt[(__ffs(mk) - 1) * 32 + warp], 1u << lane);
+    for (unsigned int mk = cand; mk; mk &= mk - 1u) atomicOr(&s_eq[(__ffs(mk) - 1) * 32 + warp], 1u << lane);
+    __syncthreads();
+    const int n_words = (s.n_pool + 31) / 32;  // <= 512: thread t < n_words takes word t
+    const unsigned int g = tid < n_words ? s_gt[tid] : 0u, q = tid < n_words ? s_eq[tid] : 0u;
+    const unsigned int mine = (unsigned int)__popc(g) | ((unsigned int)__popc(q) << 16);
+    unsigned int inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned int y = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += y;
+    }
+    if (lane == 31) s_tot[warp] = inc;
+    __syncthreads();
+    const unsigned int ex = inc - mine + __reduce_add_sync(0xffffffffu, lane < warp ? s_tot[lane] : 0u);
+    const int last = s.n_pool - 1;
+    const int last_sz = s.cand_end - (S + last * cs);
+    {
+      unsigned int eq_before = ex >> 16;
+      unsigned int rnk = (ex & 0xffffu) + min(eq_before, need);  // slot of this thread's next selected entry
+      unsigned int bits = g | q;
+      while (bits) {
+        const int e = __ffs(bits) - 1;
+        bits &= bits - 1u;
+        const bool gt = (g >> e) & 1u;
+        if (gt || eq_before < need) {
+          const int c = tid * 32 + e;
+          if (rnk < (unsigned int)s.k_sel) topk_emit(a, s, seg, idx, cs, c, rnk);
+          if (c == last) s_last = 1;
+          ++rnk;
+        }
+        eq_before += gt ? 0u : 1u;
+      }
+    }
+    // selected tokens: whole chunks, except that the last chunk of the range may be short
+    n_sel_tokens = s.k_sel * cs;
+    if (last_sz < cs) {
+      __syncthreads();
+      if (s_last) n_sel_tokens -= cs - last_sz;
+    }
+  }
+  for (int i = tid; i < S; i += kTopkThreads) idx[i] = i;
+  const int n_tail = s.n - s.cand_end;  // the always-kept most recent tokens
+  for (int i = tid; i < n_tail; i += kTopkThreads) idx[S + n_sel_tokens + i] = s.cand_end + i;
+  if (tid == 0) a.seg_len_dev[seg] = S + n_sel_tokens + n_tail;
+}
+
 // Row statistics from a given normaliser: stats[job][r] = (log-sum-exp of row r over the scored keys in the log2 domain,
 // 1), so that the second scoring pass computes exp2(logit - lse) directly.  Row r = i * G + g.
 __global__ void stats_from_lse_kernel(const ScoreJob* jobs, const float* lse, float2* stats, int R, int G, int L_obs, int Hq) {
@@ -428,10 +690,17 @@ int launch_topk(const TopkArgs& a0, int n_segs, int max_pool, int n_active, cuda
     CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    CATEKV_CUDA_TRY(cudaFuncSetAttribute(topk_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkSmallMax * 6));
     if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
   }
   TopkArgs a = a0;
   a.chk = checked_status_ptr();
+  if (a.pool_mode == kPoolPrescored && a.row_is_seg && max_pool <= kTopkSmallMax && (max_pool + 3) / 4 * 4 <= a.c_stride) {
+    // short prescored lists: one CTA per segment with the list in registers
+    a.small_pool = max_pool;
+    CATEKV_CUDA_TRY(launch_pdl(topk_small_kernel, dim3(n_segs), dim3(kTopkThreads), (size_t)((max_pool + 3) / 4 * 4) * 6, stream, a));
+    return CATEKV_OK;
+  }
   // CTAs per segment: one for short lists, a cluster of 8 for long ones.  The cluster's barriers and exchanges
   // have a fixed cost, one CTA's passes grow with the list: the cluster pays from about 12 K entries, provided the
   // clusters of the segments that select fit one wave of resident CTAs (two per SM); beyond 16 K entries a single

@@ -31,7 +31,23 @@ struct TopkArgs {
   int32_t mark_keep_all;  // 1: a keep_all segment gets seg_len_dev = -1 ("the whole list") instead of being skipped
   int32_t stage_entries;  // set by launch_topk: pooled entries per CTA that the dynamic shared memory holds
   int32_t* chk;           // set by launch_topk: the checked build's status block, else null
+  int32_t row_is_seg;     // 1 (prescored lists only): the score row of segment s is row s, whatever its job says
+  int32_t small_pool;     // set by launch_topk for topk_small_kernel: bound of the pooled entries of a segment
 };
+
+// Monotone map of arbitrary finite floats to non-negative floats whose bit patterns order the same way as the
+// values (what the radix select of the top-k kernels needs): flip so that larger values get larger unsigned
+// patterns, then clear the sign by halving the range.  Values one ulp apart may merge into a tie: within the
+// parity tolerance band.  key_to_score inverts it up to that last bit (still monotone).
+__device__ __forceinline__ float monotone_key(float x) {
+  const uint32_t u = __float_as_uint(x);
+  const uint32_t k = (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // unsigned order == float order
+  return __uint_as_float(k >> 1);                                 // non-negative pattern
+}
+__device__ __forceinline__ float key_to_score(uint32_t key) {
+  const uint32_t k = key << 1;
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 
 struct GatherArgs {
   const SelSeg* segs;

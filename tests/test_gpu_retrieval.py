@@ -299,3 +299,55 @@ def test_retrieve_select_and_indexed_attention(ck, cs, G, num_ctas):
     with pytest.raises(ck.CatekvError) as e:
         ck.catekv_retrieve_select(cache, meta, cs, q, mask, budget, sink, local, idx[:, :100].contiguous(), sel)
     assert e.value.code == ck.ERR_INVALID_ARG
+
+
+def _one_dim_case(ck, levels, budget, cs=8, sink=4, local=32):
+    """One segment whose keys live on dimension 0 only and a query that is 1 there: the bound of a chunk is the
+    largest of its keys' values, exact on both sides, so the selection must equal the oracle's list (ties to the
+    lowest chunk) and not just agree within the band."""
+    n = len(levels)
+    K = np.zeros((n, 128))
+    K[:, 0] = levels
+    oc = orc.HybridCache(1, 1, 128)
+    oc.k_rows.append(orc.f64_to_bf16(K))
+    oc.v_rows.append(orc.f64_to_bf16(np.zeros((n, 128))))
+    assert np.array_equal(orc.bf16_to_f64(oc.k_rows[0])[:, 0], levels)  # the levels are bf16 values
+    cache = H.device_cache_from_oracle(ck, oc, 0)
+    meta = ck.catekv_retrieval_meta(cache, cs)
+    ck.catekv_retrieval_build(cache, cs, meta)
+    qv = np.zeros((1, 2, 128))
+    qv[:, :, 0] = 1.0
+    q = synth.from_bits(orc.f64_to_bf16(qv), "cuda")
+    kmax, kmin = orc.retrieval_metadata(oc.k_rows[0], cs)
+    scores = orc.retrieval_scores(qv[0], kmax, kmin)
+    want = orc.retrieve_indices(scores, n, sink, local, budget, cs)
+    idx = torch.full((1, len(want) + 8), -7, dtype=torch.int32, device="cuda")
+    sel = torch.full((1,), -99, dtype=torch.int32, device="cuda")
+    ck.catekv_retrieve_select(cache, meta, cs, q, [1], budget, sink, local, idx, sel)
+    torch.cuda.synchronize()
+    assert int(sel[0]) == len(want)
+    assert np.array_equal(idx[0, :len(want)].cpu().numpy().astype(np.int64), want)
+    assert torch.all(idx[0, len(want):] == -7)
+
+
+@pytest.mark.parametrize("case", ["three_levels", "all_equal", "outlier", "two_neighbours", "negative", "random"])
+@pytest.mark.parametrize("n,budget", [(8192 + 40, 1024), (3000, 520), (20000, 2048)])
+def test_retrieval_selection_with_ties_and_crowded_scores(ck, case, n, budget):
+    """The short-list selection kernel on score distributions that stress each of its steps: hundreds of exact
+    ties at the threshold, one score for all, an outlier that squeezes every other score into one histogram bin,
+    two adjacent bf16 values, negative scores, and plain random ones."""
+    rng = np.random.default_rng(len(case) * 1000 + n)
+    chunk_level = {
+        "three_levels": lambda c: rng.integers(1, 4, c).astype(np.float64),
+        "all_equal": lambda c: np.full(c, 1.5),
+        "outlier": lambda c: np.concatenate([[4096.0], rng.integers(0, 256, c - 1) / 256.0]),
+        "two_neighbours": lambda c: np.where(rng.random(c) < 0.5, 2.0, 2.015625),
+        "negative": lambda c: -rng.integers(1, 200, c) / 16.0,
+        "random": lambda c: orc.bf16_to_f64(orc.f64_to_bf16(rng.standard_normal(c))),
+    }[case]
+    n_chunks = (n + 7) // 8
+    lv = chunk_level(n_chunks)
+    if case == "outlier":
+        lv = np.roll(lv, n_chunks // 2)
+    levels = np.repeat(lv, 8)[:n]
+    _one_dim_case(ck, levels, budget)
