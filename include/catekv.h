@@ -109,7 +109,8 @@ typedef struct catekv_cache {
                                  every other call refuses such a cache with CATEKV_ERR_UNSUPPORTED */
   const int32_t* seg_cap_dev; /* device [B*Hkv], copy of seg_cap, or NULL.  Kernels that write rows whose number
                                  is decided on the device (the gather of catekv_retrieve_compact) clamp to it;
-                                 catekv_retrieve_compact requires it on its step cache */
+                                 catekv_retrieve_compact requires it on its step cache, and both retrieval calls
+                                 on `cache` (the scoring kernel shares out its work by the capacities) */
 } catekv_cache;
 
 /*
@@ -426,7 +427,7 @@ int catekv_decode_combine(const catekv_cache* cache, const void* q, int32_t Hq, 
  *   idx_out   device int32 [B*Hkv, idx_stride] or NULL: the rows taken from each segment
  *   ws        device scratch of at least catekv_retrieve_workspace_bytes(B, Hkv, largest seg_cap of `cache`)
  * Errors: CATEKV_ERR_CAPACITY if a kept list does not fit its segment of step_cache (nothing launched);
- * CATEKV_ERR_INVALID_ARG if step_cache has no seg_cap_dev;
+ * CATEKV_ERR_INVALID_ARG if cache or step_cache has no seg_cap_dev;
  * CATEKV_ERR_UNSUPPORTED for more than 2048 segments (the mask travels in the kernel arguments).
  * The call copies nothing from the host and takes every per-segment decision on the device from the device's
  * lengths; launch shapes follow the capacities.  A step (append, metadata append, this call, attention over

@@ -143,121 +143,223 @@ __host__ __device__ inline SelSeg retrieval_decide(int n, bool enabled, const Re
 }
 
 // bound(c, g) = [kmax_c | kmin_c] . [max(q_g, 0) | min(q_g, 0)]: a [chunks x 256] x [256 x 8 heads] product, so the
-// tensor cores take it (mma.m16n8k16, chunks are M, the group's heads N = 8).  A CTA streams 64-chunk tiles of the
-// metadata (32 KB, contiguous) through a 3-stage cp.async pipeline into XOR-swizzled shared memory; each of its 4
-// warps owns 16 chunks of a tile, takes the maximum over the heads and writes one score per chunk.
+// tensor cores take it (mma.m16n8k16, chunks are M, the group's heads N = 8).  The 64-chunk tiles (32 KB, contiguous)
+// of all segments that retrieve, laid end to end, are cut into equal shares, one per CTA of a persistent grid: a CTA
+// streams its tiles through a 3-stage cp.async pipeline into XOR-swizzled shared memory, across segment boundaries
+// (it reloads the group's queries there); each of its 4 warps owns 16 chunks of a tile, takes the maximum over the
+// heads and writes one score per chunk.  The cut is made over the tiles the segments' capacities allow, so that it
+// does not move while the caches grow (a captured step stays valid); tiles past a segment's live end are skipped.
 constexpr int kRsTile = 64, kRsThreads = 128, kRsStages = 3;
 constexpr int kRsRowBytes = 2 * kRowBytes;                 // one chunk: 256 bf16
 constexpr int kRsStageBytes = kRsTile * kRsRowBytes;
-constexpr int kRsSmem = kRsStages * kRsStageBytes + kMaxG * kRsRowBytes;
+constexpr int kRsSmemFixed = kRsStages * kRsStageBytes;
+static size_t rs_smem_bytes(int n_segs) { return (size_t)kRsSmemFixed + (size_t)n_segs * 4 + align_up((size_t)n_segs * 2, 16); }
 __device__ __forceinline__ uint32_t rs_off(int row, int piece) {  // 16-byte piece (0..31) of a 512-byte row
   return (uint32_t)(row * kRsRowBytes + ((piece ^ (row & 7)) << 4));
+}
+// 64-chunk tiles that the candidate chunks of a segment of capacity cap can fill at most
+__host__ __device__ inline int rs_tiles_cap(int cap, const RetParams& p) {
+  const int pool = (cap - p.sink2) / p.cs;
+  return pool > 0 ? (pool + kRsTile - 1) / kRsTile : 0;
 }
 
 struct RetScoreArgs {
   RetParams p;
   RetMask mask;
-  const int32_t* seg_len;  // the source cache's lengths and offsets
+  const int32_t* seg_len;  // the source cache's lengths, offsets and capacities
   const int32_t* seg_off;
+  const int32_t* seg_cap;
   const uint8_t* meta;
   const uint16_t* q;
-  int32_t Hq, G;
+  int32_t Hq, G, n_segs;
   float* P;
   int64_t p_stride;
   SelSeg* segs;  // out: the decision per segment, for the top-k and gather kernels that follow
 };
-struct RetJobView {
-  int32_t b, h, chunk0 /* global index of the first candidate chunk */, n_pool /* candidate chunks */;
-};
 
 __global__ void __launch_bounds__(kRsThreads, 2) retrieval_score_kernel(const RetScoreArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  const int seg = blockIdx.y;
-  pdl_launch_dependents();
-  pdl_wait();  // lengths, metadata and queries come from earlier kernels of the stream
-  SelSeg d = retrieval_decide(a.seg_len[seg], (a.mask.w[seg >> 5] >> (seg & 31)) & 1u, a.p);
-  const bool scores = !d.keep_all && d.k_sel > 0;
-  if (scores) d.job = seg;  // score row = segment index
-  if (blockIdx.x == 0 && threadIdx.x == 0) a.segs[seg] = d;
-  if (!scores) return;  // this segment selects nothing
-  const RetJobView job = {seg / a.p.Hkv, seg % a.p.Hkv, a.seg_off[seg] / a.p.cs + a.p.sink2 / a.p.cs, d.n_pool};
-  const uint8_t* meta = a.meta;
-  const uint16_t* q = a.q;
-  const int Hq = a.Hq, G = a.G;
-  float* P = a.P;
-  const int64_t p_stride = a.p_stride;
-  // this CTA's chunks: an equal share, in whole tiles
-  const int tiles_total = (job.n_pool + kRsTile - 1) / kRsTile;
-  const int tiles_per = (tiles_total + gridDim.x - 1) / gridDim.x;
-  const int tile_lo = blockIdx.x * tiles_per, tile_hi = min(tiles_total, tile_lo + tiles_per);
-  if (tile_lo >= tile_hi) return;
+  __shared__ int s_wsum[kRsThreads / 32];
+  __shared__ int s_start[2];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = lane >> 2, t = lane & 3;
-  const uint32_t s_stage = smem_u32(smem);
-  uint16_t* s_q = reinterpret_cast<uint16_t*>(smem + kRsStages * kRsStageBytes);  // [8][256]: max(q,0) | min(q,0)
-  const uint8_t* src0 = meta + (int64_t)job.chunk0 * kRsRowBytes;
-  auto issue = [&](int tile) {
-    if (tile < tile_hi) {
-      const uint32_t sb = s_stage + ((tile - tile_lo) % kRsStages) * kRsStageBytes;
-      const int c0 = tile * kRsTile;
-#pragma unroll
-      for (int i = 0; i < (kRsTile * 32) / kRsThreads; ++i) {
-        const int id = tid + i * kRsThreads;
-        const int r = id >> 5, pc = id & 31;
-        const int ok = (c0 + r) < job.n_pool ? 16 : 0;
-        cp_async16(sb + rs_off(r, pc), src0 + (int64_t)(ok ? c0 + r : 0) * kRsRowBytes + pc * 16, ok);
-      }
+  const int n_segs = a.n_segs;
+  int32_t* s_npool = reinterpret_cast<int32_t*>(smem + kRsSmemFixed);             // live candidate chunks per segment
+  uint16_t* s_tcap = reinterpret_cast<uint16_t*>(s_npool + n_segs);               // tiles by capacity per segment
+  pdl_launch_dependents();
+  // ---- this CTA's share of the tiles (from the capacities: nothing an earlier kernel of the stream writes)
+  const int per = (n_segs + kRsThreads - 1) / kRsThreads;  // consecutive segments per thread
+  int my_sum = 0;
+  for (int k = 0; k < per; ++k) {
+    const int sg = tid * per + k;
+    if (sg < n_segs) {
+      const int tc = ((a.mask.w[sg >> 5] >> (sg & 31)) & 1u) ? rs_tiles_cap(a.seg_cap[sg], a.p) : 0;
+      s_tcap[sg] = (uint16_t)tc;
+      my_sum += tc;
     }
-    cp_async_commit();
-  };
-  issue(tile_lo);
-  issue(tile_lo + 1);
-  // the group's queries, split by sign (exact in bf16); heads >= G are zero
-  for (int i = tid; i < kMaxG * kD; i += kRsThreads) {
-    const int hd = i / kD, e = i % kD;
-    uint16_t v = 0;
-    if (hd < G) v = q[((int64_t)job.b * Hq + job.h * G + hd) * kD + e];
-    const bool neg = v & 0x8000u;
-    s_q[hd * 256 + e] = neg ? 0 : v;
-    s_q[hd * 256 + 128 + e] = neg ? v : 0;
+  }
+  int inc = my_sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  if (lane == 31) s_wsum[warp] = inc;
+  if (tid == 0) s_start[0] = -1;
+  __syncthreads();
+  int total = 0;
+#pragma unroll
+  for (int w = 0; w < kRsThreads / 32; ++w) {
+    if (w < warp) inc += s_wsum[w];
+    total += s_wsum[w];
+  }
+  const int64_t g_lo = (int64_t)blockIdx.x * total / gridDim.x, g_hi = (int64_t)(blockIdx.x + 1) * total / gridDim.x;
+  {
+    int64_t off = inc - my_sum;  // tiles before this thread's segments
+    if (off <= g_lo && g_lo < off + my_sum)
+      for (int k = 0; k < per; ++k) {
+        const int sg = tid * per + k;
+        const int tc = s_tcap[sg];
+        if (g_lo < off + tc) {
+          s_start[0] = sg;
+          s_start[1] = (int)(g_lo - off);
+          break;
+        }
+        off += tc;
+      }
+  }
+  pdl_wait();  // lengths, metadata and queries come from earlier kernels of the stream
+  // ---- the decision of every segment (the CTAs share the writes), and its live candidate chunks
+  for (int k = 0; k < per; ++k) {
+    const int sg = tid * per + k;
+    if (sg < n_segs) {
+      SelSeg d = retrieval_decide(a.seg_len[sg], (a.mask.w[sg >> 5] >> (sg & 31)) & 1u, a.p);
+      const bool scores = !d.keep_all && d.k_sel > 0;
+      if (scores) d.job = sg;  // score row = segment index
+      s_npool[sg] = scores ? d.n_pool : 0;
+      if (sg % gridDim.x == blockIdx.x) a.segs[sg] = d;
+    }
   }
   __syncthreads();
-  uint32_t qf[16][2];
+  if (g_lo >= g_hi || s_start[0] < 0) return;
+  const int Hq = a.Hq, G = a.G, Hkv = a.p.Hkv, cs = a.p.cs;
+  const int g = lane >> 2, t = lane & 3;
+  const uint32_t s_stage = smem_u32(smem);
+  const int n_tiles = (int)(g_hi - g_lo);
+  struct Cursor {
+    int seg, lt;         // segment and tile within it
+    int n_pool;          // live candidate chunks of the segment
+    const uint8_t* src;  // metadata of its first candidate chunk
+  };
+  auto enter = [&](Cursor& c) {
+    c.n_pool = c.seg < n_segs ? s_npool[c.seg] : 0;
+    c.src = a.meta + (int64_t)(c.seg < n_segs ? a.seg_off[c.seg] / cs + a.p.sink2 / cs : 0) * kRsRowBytes;
+  };
+  auto advance = [&](Cursor& c) {
+    if (++c.lt >= (int)s_tcap[c.seg]) {
+      do {
+        ++c.seg;
+      } while (c.seg < n_segs && s_tcap[c.seg] == 0);
+      c.lt = 0;
+      enter(c);
+    }
+  };
+  Cursor ci = {s_start[0], s_start[1], 0, nullptr};  // the tile requested next
+  enter(ci);
+  Cursor cc = ci;  // the tile computed next
+  int issued = 0;
+  auto issue = [&]() {
+    if (issued < n_tiles && ci.seg < n_segs) {
+      const int n_pool = ci.n_pool;
+      const int c0 = ci.lt * kRsTile;
+      if (c0 < n_pool) {
+        const uint8_t* src0 = ci.src;
+        const uint32_t sb = s_stage + (issued % kRsStages) * kRsStageBytes;
 #pragma unroll
-  for (int ks = 0; ks < 16; ++ks) {
-    qf[ks][0] = *reinterpret_cast<const uint32_t*>(s_q + g * 256 + ks * 16 + 2 * t);
-    qf[ks][1] = *reinterpret_cast<const uint32_t*>(s_q + g * 256 + ks * 16 + 8 + 2 * t);
-  }
-  for (int tile = tile_lo; tile < tile_hi; ++tile) {
+        for (int i = 0; i < (kRsTile * 32) / kRsThreads; ++i) {
+          const int id = tid + i * kRsThreads;
+          const int r = id >> 5, pc = id & 31;
+          const int ok = (c0 + r) < n_pool ? 16 : 0;
+          cp_async16(sb + rs_off(r, pc), src0 + (int64_t)(ok ? c0 + r : 0) * kRsRowBytes + pc * 16, ok);
+        }
+      }
+      advance(ci);
+    }
+    ++issued;
+    cp_async_commit();
+  };
+  issue();
+  issue();
+  // B fragments of head g = lane / 4 of the group (zero from head G on): [max(q, 0) | min(q, 0)], the split by sign
+  // being exact in bf16.  The words of the segment after the current one are requested ahead, so that a CTA whose
+  // share crosses a segment boundary does not wait for them there.
+  uint32_t qf[16][2], q_next[16];
+  auto next_seg_of = [&](int sg) {
+    do {
+      ++sg;
+    } while (sg < n_segs && s_tcap[sg] == 0);
+    return sg;
+  };
+  auto load_q = [&](int sg, uint32_t (&raw)[16]) {
+    const uint16_t* qp = a.q + ((int64_t)(sg / Hkv) * Hq + (sg % Hkv) * G + g) * kD;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      raw[2 * ks] = (g < G && sg < n_segs) ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 2 * t) : 0u;
+      raw[2 * ks + 1] = (g < G && sg < n_segs) ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + 2 * t) : 0u;
+    }
+  };
+  int q_seg = -1, q_next_seg = cc.seg;
+  load_q(q_next_seg, q_next);
+  for (int it = 0; it < n_tiles; ++it) {
     cp_async_wait<kRsStages - 2>();
     __syncthreads();
-    issue(tile + kRsStages - 1);
-    const uint32_t sb = s_stage + ((tile - tile_lo) % kRsStages) * kRsStageBytes;
-    const int row0 = warp * 16;
-    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb2[4] = {0.f, 0.f, 0.f, 0.f};
-    const int r = row0 + (lane & 7) + ((lane >> 3) & 1) * 8;
-    const int padd = lane >> 4;
+    issue();
+    const int n_pool = cc.n_pool;
+    const int c0 = cc.lt * kRsTile;
+    if (c0 < n_pool) {
+      if (cc.seg != q_seg) {
+        q_seg = cc.seg;
+        if (q_next_seg != q_seg) load_q(q_seg, q_next);  // a segment without live tiles lay in between
 #pragma unroll
-    for (int ks = 0; ks < 16; ks += 2) {
-      uint32_t af[4];
-      ldmatrix_x4(af, sb + rs_off(r, ks * 2 + padd));
-      mma_bf16_16816(sa, af, qf[ks][0], qf[ks][1]);
-      ldmatrix_x4(af, sb + rs_off(r, ks * 2 + 2 + padd));
-      mma_bf16_16816(sb2, af, qf[ks + 1][0], qf[ks + 1][1]);
-    }
-    // c0, c1: chunk row0 + g, heads 2t, 2t+1;  c2, c3: chunk row0 + g + 8
-    float lo = fmaxf(2 * t < G ? sa[0] + sb2[0] : -INFINITY, 2 * t + 1 < G ? sa[1] + sb2[1] : -INFINITY);
-    float hi = fmaxf(2 * t < G ? sa[2] + sb2[2] : -INFINITY, 2 * t + 1 < G ? sa[3] + sb2[3] : -INFINITY);
+        for (int ks = 0; ks < 8; ++ks)
 #pragma unroll
-    for (int o = 1; o <= 2; o <<= 1) {
-      lo = fmaxf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
-      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+          for (int j = 0; j < 2; ++j) {
+            const uint32_t w = q_next[2 * ks + j];
+            const uint32_t pos = ((w & 0x8000u) ? 0u : (w & 0xffffu)) | ((w & 0x80000000u) ? 0u : (w & 0xffff0000u));
+            qf[ks][j] = pos;
+            qf[ks + 8][j] = w ^ pos;
+          }
+        q_next_seg = next_seg_of(q_seg);
+        load_q(q_next_seg, q_next);
+      }
+      const uint32_t sb = s_stage + (it % kRsStages) * kRsStageBytes;
+      const int row0 = warp * 16;
+      float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb2[4] = {0.f, 0.f, 0.f, 0.f};
+      const int r = row0 + (lane & 7) + ((lane >> 3) & 1) * 8;
+      const int padd = lane >> 4;
+#pragma unroll
+      for (int ks = 0; ks < 16; ks += 2) {
+        uint32_t af[4];
+        ldmatrix_x4(af, sb + rs_off(r, ks * 2 + padd));
+        mma_bf16_16816(sa, af, qf[ks][0], qf[ks][1]);
+        ldmatrix_x4(af, sb + rs_off(r, ks * 2 + 2 + padd));
+        mma_bf16_16816(sb2, af, qf[ks + 1][0], qf[ks + 1][1]);
+      }
+      // c0, c1: chunk row0 + g, heads 2t, 2t+1;  c2, c3: chunk row0 + g + 8
+      float lo = fmaxf(2 * t < G ? sa[0] + sb2[0] : -INFINITY, 2 * t + 1 < G ? sa[1] + sb2[1] : -INFINITY);
+      float hi = fmaxf(2 * t < G ? sa[2] + sb2[2] : -INFINITY, 2 * t + 1 < G ? sa[3] + sb2[3] : -INFINITY);
+#pragma unroll
+      for (int o = 1; o <= 2; o <<= 1) {
+        lo = fmaxf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+      }
+      if (t == 0) {
+        const int c = c0 + row0 + g;
+        float* Prow = a.P + (size_t)cc.seg * a.p_stride;
+        if (c < n_pool) Prow[c] = monotone_key(lo);
+        if (c + 8 < n_pool) Prow[c + 8] = monotone_key(hi);
+      }
     }
-    if (t == 0) {
-      const int c = tile * kRsTile + row0 + g;
-      if (c < job.n_pool) P[(size_t)blockIdx.y * p_stride + c] = monotone_key(lo);
-      if (c + 8 < job.n_pool) P[(size_t)blockIdx.y * p_stride + c + 8] = monotone_key(hi);
-    }
+    if (cc.seg < n_segs) advance(cc);
   }
   cp_async_wait<0>();
 }
@@ -371,6 +473,7 @@ static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t ch
     return CATEKV_ERR_INVALID_ARG;
   }
   if (!meta || !q || !retrieval_mask || !ws) return CATEKV_ERR_INVALID_ARG;
+  if (!cache->seg_cap_dev) return CATEKV_ERR_INVALID_ARG;  // the scoring kernel shares out its tiles by the capacities
   if (!chunk_size_ok(chunk_size)) return CATEKV_ERR_UNSUPPORTED;
   if (Hq <= 0 || Hq % cache->Hkv || budget < 0 || sink < 0 || local < 0) return CATEKV_ERR_INVALID_ARG;
   const int G = Hq / cache->Hkv;
@@ -412,32 +515,37 @@ static int retrieve_impl(const catekv_cache* cache, const void* meta, int32_t ch
   SelSeg* d_segs = (SelSeg*)(w8 + W.off_segs);
   float* P = (float*)(w8 + W.off_P);
   {
-    // CTAs per segment: one wave of resident CTAs (2 per SM) over the segments that retrieve, so that a CTA
-    // streams many 64-chunk tiles through its pipeline and no partial wave trails; never more CTAs than tiles
-    int n_ret = 0;
-    for (int s = 0; s < n_segs; ++s) n_ret += retrieval_mask[s] != 0;
-    const int tiles = (max_pool + kRsTile - 1) / kRsTile;
-    int gx = n_ret > 0 ? (2 * sm_count()) / n_ret : 1;
+    // one wave of resident CTAs (2 per SM), never more CTAs than tiles
+    int64_t tiles = 0;
+    for (int s = 0; s < n_segs; ++s) {
+      const int tc = retrieval_mask[s] ? rs_tiles_cap(cache->seg_cap[s], rp) : 0;
+      if (tc > 65535) return CATEKV_ERR_UNSUPPORTED;  // the kernel keeps the tile counts as 16-bit numbers
+      tiles += tc;
+    }
+    int64_t gx = 2 * sm_count();
     if (gx > tiles) gx = tiles;
-    if (gx > 64) gx = 64;
     if (gx < 1) gx = 1;
+    const size_t smem = rs_smem_bytes(n_segs);
     static std::atomic<bool> attr_set[64];
     int dev = 0;
     CATEKV_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
-      CATEKV_CUDA_TRY(cudaFuncSetAttribute(retrieval_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRsSmem));
+      CATEKV_CUDA_TRY(cudaFuncSetAttribute(retrieval_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)rs_smem_bytes(kRetMaxSegs)));
       if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
     }
     sa.seg_len = cache->seg_len_dev;
     sa.seg_off = cache->seg_off_dev;
+    sa.seg_cap = cache->seg_cap_dev;
     sa.meta = (const uint8_t*)meta;
     sa.q = (const uint16_t*)q;
     sa.Hq = Hq;
     sa.G = G;
+    sa.n_segs = n_segs;
     sa.P = P;
     sa.p_stride = W.p_stride;
     sa.segs = d_segs;
-    CATEKV_CUDA_TRY(launch_pdl(retrieval_score_kernel, dim3(gx, (unsigned)n_segs), dim3(kRsThreads), kRsSmem, st, sa));
+    CATEKV_CUDA_TRY(launch_pdl(retrieval_score_kernel, dim3((unsigned)gx), dim3(kRsThreads), smem, st, sa));
   }
   TopkArgs ta = {};
   ta.segs = d_segs;

@@ -351,3 +351,41 @@ def test_retrieval_selection_with_ties_and_crowded_scores(ck, case, n, budget):
         lv = np.roll(lv, n_chunks // 2)
     levels = np.repeat(lv, 8)[:n]
     _one_dim_case(ck, levels, budget)
+
+
+def test_retrieval_many_short_segments(ck):
+    """A thousand segments of one to three metadata tiles each: a CTA of the scoring kernel walks across several
+    segments (masked out, too short to select, and empty ones among them); every selection is checked."""
+    rng = np.random.default_rng(97)
+    B, Hkv, G, cs = 125, 8, 2, 8
+    budget, sink, local = 200, 4, 16
+    lens = rng.integers(300, 1400, B * Hkv)
+    lens[rng.random(B * Hkv) < 0.1] = 0
+    lens[rng.random(B * Hkv) < 0.1] = 150          # not longer than the budget: kept whole
+    mask = (rng.random(B * Hkv) < 0.8).astype(np.uint8)
+    oc = H.random_cache(B, Hkv, lens.tolist(), seed=97)
+    cache = H.device_cache_from_oracle(ck, oc, max_new=8)
+    meta = ck.catekv_retrieval_meta(cache, cs)
+    ck.catekv_retrieval_build(cache, cs, meta)
+    q = synth.randn_bf16((B, Hkv * G, 128), "cuda", 97, "q")
+    qb = orc.bf16_to_f64(synth.bits(q))
+    want = ck.catekv_retrieve_lengths(cache, cs, mask, budget, sink, local)
+    idx = torch.full((B * Hkv, int(want.max()) + 3), -7, dtype=torch.int32, device="cuda")
+    sel = torch.full((B * Hkv,), -99, dtype=torch.int32, device="cuda")
+    ck.catekv_retrieve_select(cache, meta, cs, q, mask, budget, sink, local, idx, sel)
+    torch.cuda.synchronize()
+    got_sel = sel.cpu().tolist()
+    idx = idx.cpu().numpy()
+    n_selecting = 0
+    for s, L in enumerate(lens.tolist()):
+        if mask[s] and L > budget:
+            n_selecting += 1
+            assert got_sel[s] == want[s], s
+            kmax, kmin = orc.retrieval_metadata(oc.k_rows[s], cs)
+            b, h = divmod(s, Hkv)
+            scores = orc.retrieval_scores(qb[b, h * G:(h + 1) * G], kmax, kmin)
+            _check_selection(idx[s, :want[s]].astype(np.int64), scores, L, sink, local, budget, cs, f"seg {s}")
+            assert np.all(idx[s, want[s]:] == -7)
+        else:
+            assert got_sel[s] == -1 and np.all(idx[s] == -7), s
+    assert n_selecting > 500
