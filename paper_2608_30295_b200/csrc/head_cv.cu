@@ -3,6 +3,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <atomic>
 #include <vector>
 
 #include <cooperative_groups.h>
@@ -34,13 +35,20 @@ constexpr int kCvCluster = 8;
 #define CATEKV_CV_UNROLL 16
 #endif
 constexpr int kCvUnroll = CATEKV_CV_UNROLL;  // loads a thread keeps in flight in the sweeps over its share of the matrix
+constexpr int kCvListCap = 16384;            // entries of the threshold bin a CTA can keep in shared memory
+constexpr int kCvBins = 2048;                // == 256 * kHistCopies: the fast path reuses the copies' array
+static_assert(kCvBins == 256 * kHistCopies && kCvBins == 2 * kCvThreads, "two bins per thread in the scan");
 
 // One thread-block cluster of 8 CTAs per (sequence, KV head): Phi = alpha * percentile element (Eq. 2),
 // C_j = #{i: A_ij >= Phi} (Eq. 3), cv = std_pop(C) / mean(C) (Eq. 4) from exact integer sums.
-// The percentile element is found by a radix select on the bit patterns (entries are >= 0): every CTA owns a
-// contiguous share of the flat matrix; the bits above the highest bit in which the smallest and largest entry
-// differ are common, the rest is resolved 8 bits per pass with the CTAs' histograms summed through distributed
-// shared memory.  For the counts every CTA owns a range of columns; the sums meet in CTA 0.
+// The percentile element is found by a radix select on the bit patterns (entries are >= 0); every CTA owns a
+// contiguous share of the flat matrix and the CTAs' histograms are summed through distributed shared memory.
+// Fast path, two sweeps over the matrix: a 2048-bin histogram of the patterns' top bits (entries are below 2, so
+// bits 30..19 fit: exponent and four mantissa bits) finds the bin of the percentile element; a second sweep copies
+// that bin's entries into shared memory, where two more levels (bits 18..8, bits 7..0) resolve it.  If an entry
+// is 2 or more, or a CTA's part of the bin does not fit its list, the general path takes over: extremes, then the
+// bits below the highest one in which they differ, 8 per sweep.  For the counts every CTA owns a range of
+// columns; the sums meet in CTA 0.
 __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
   cg::cluster_group cluster = cg::this_cluster();
   const int seg = blockIdx.x / kCvCluster;
@@ -53,6 +61,8 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
   __shared__ unsigned int s_mm[2];
   __shared__ unsigned long long red[2][32];
   __shared__ unsigned long long s_sums[2];
+  __shared__ unsigned int s_pick[2], s_big, s_nlist, s_wtot[32];
+  extern __shared__ unsigned int s_list[];  // kCvListCap entries
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* A = a.A + (size_t)seg * a.seg_stride;
   const unsigned int* Ab = reinterpret_cast<const unsigned int*>(A);
@@ -61,6 +71,133 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
   const int per = ((N + kCvCluster - 1) / kCvCluster + 3) / 4 * 4;
   const int lo = min(N, rank * per), hi = min(N, lo + per);
 
+  // ---- fast path
+  bool have_thr = false;
+  unsigned int thr_bits = 0u;
+  {
+    unsigned int* h2k = hcopies;
+    // Sum of the CTAs' histograms, suffix scan (thread t owns bins 2047 - 2t and 2046 - 2t), and the bin that
+    // holds the need-th largest entry with what is still needed inside it.  The caller ends with a cluster
+    // barrier before anybody's histogram is written again.
+    auto pick = [&](unsigned int need_in, unsigned int& bin, unsigned int& need_out) {
+      cluster.sync();  // all histograms complete
+      unsigned int c_hi = 0, c_lo = 0;
+#pragma unroll
+      for (int r = 0; r < kCvCluster; ++r) {
+        const unsigned int* hp = cluster.map_shared_rank(h2k, r);
+        c_hi += hp[kCvBins - 1 - 2 * tid];
+        c_lo += hp[kCvBins - 2 - 2 * tid];
+      }
+      const unsigned int cnt = c_hi + c_lo;
+      unsigned int inc = cnt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int y = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += y;
+      }
+      if (lane == 31) s_wtot[warp] = inc;
+      __syncthreads();
+      inc += __reduce_add_sync(0xffffffffu, lane < warp ? s_wtot[lane] : 0u);
+      const unsigned int before = inc - cnt;
+      if (before < need_in && need_in <= before + c_hi) {
+        s_pick[0] = (unsigned int)(kCvBins - 1 - 2 * tid);
+        s_pick[1] = need_in - before;
+      } else if (before + c_hi < need_in && need_in <= inc) {
+        s_pick[0] = (unsigned int)(kCvBins - 2 - 2 * tid);
+        s_pick[1] = need_in - before - c_hi;
+      }
+      __syncthreads();
+      bin = s_pick[0];
+      need_out = s_pick[1];
+    };
+    for (int i = tid; i < kCvBins; i += kCvThreads) h2k[i] = 0u;
+    if (tid == 0) {
+      s_big = 0u;
+      s_nlist = 0u;
+      s_pick[0] = 0u;
+      s_pick[1] = 1u;
+    }
+    __syncthreads();
+    bool big = false;
+    for (int c0 = lo; c0 < hi; c0 += kCvUnroll * kCvThreads) {  // whole warps stay in the loop: the vote needs them
+      unsigned int v[kCvUnroll];
+      bool in[kCvUnroll];
+#pragma unroll
+      for (int e = 0; e < kCvUnroll; ++e) {
+        const int c = c0 + e * kCvThreads + tid;
+        in[e] = c < hi;
+        v[e] = in[e] ? Ab[c] : 0u;
+      }
+#pragma unroll
+      for (int e = 0; e < kCvUnroll; ++e) {
+        unsigned int dgt = v[e] >> 19;
+        if (dgt >= (unsigned int)kCvBins) {
+          big = true;
+          dgt = kCvBins - 1;
+        }
+        if (!in[e]) dgt = 0xffffu;
+        // a warp whose lanes all fall in one bin adds once; otherwise every entry adds for itself
+        int same;
+        __match_all_sync(0xffffffffu, dgt, &same);
+        if (same) {
+          if (in[e] && lane == 0) atomicAdd(&h2k[dgt], 32u);
+        } else if (in[e]) {
+          atomicAdd(&h2k[dgt], 1u);
+        }
+      }
+    }
+    if (big) s_big = 1u;
+    unsigned int b1, need1;
+    pick((unsigned int)s.need, b1, need1);
+    unsigned int own_max = 0u, big_any = 0u;
+#pragma unroll
+    for (int r = 0; r < kCvCluster; ++r) {
+      own_max = max(own_max, cluster.map_shared_rank(h2k, r)[b1]);
+      big_any |= *cluster.map_shared_rank(&s_big, r);
+    }
+    cluster.sync();  // the peers have read this CTA's histogram and flag
+    if (!big_any && own_max <= (unsigned int)kCvListCap) {  // the same decision in every CTA of the cluster
+      // second sweep: this CTA's entries of bin b1 go to its list
+      for (int c0 = lo; c0 < hi; c0 += kCvUnroll * kCvThreads) {
+        unsigned int v[kCvUnroll];
+#pragma unroll
+        for (int e = 0; e < kCvUnroll; ++e) {
+          const int c = c0 + e * kCvThreads + tid;
+          v[e] = c < hi ? Ab[c] : 0xffffffffu;  // a pattern that is in no bin
+        }
+#pragma unroll
+        for (int e = 0; e < kCvUnroll; ++e) {
+          const bool hit = (v[e] >> 19) == b1;
+          const unsigned int votes = __ballot_sync(0xffffffffu, hit);
+          if (votes) {
+            unsigned int base = 0;
+            if (lane == 0) base = atomicAdd(&s_nlist, (unsigned int)__popc(votes));
+            base = __shfl_sync(0xffffffffu, base, 0);
+            if (hit) s_list[base + __popc(votes & ((1u << lane) - 1u))] = v[e];
+          }
+        }
+      }
+      for (int i = tid; i < kCvBins; i += kCvThreads) h2k[i] = 0u;
+      __syncthreads();
+      const int n_list = (int)s_nlist;
+      for (int i = tid; i < n_list; i += kCvThreads) atomicAdd(&h2k[(s_list[i] >> 8) & 0x7ffu], 1u);
+      unsigned int b2, need2;
+      pick(need1, b2, need2);
+      cluster.sync();
+      for (int i = tid; i < kCvBins; i += kCvThreads) h2k[i] = 0u;
+      __syncthreads();
+      for (int i = tid; i < n_list; i += kCvThreads) {
+        const unsigned int v = s_list[i];
+        if (((v >> 8) & 0x7ffu) == b2) atomicAdd(&h2k[v & 0xffu], 1u);
+      }
+      unsigned int b3, need3;
+      pick(need2, b3, need3);
+      cluster.sync();
+      thr_bits = (b1 << 19) | (b2 << 8) | b3;
+      have_thr = true;
+    }
+  }
+  if (!have_thr) {
   // ---- extremes of the bit patterns
   unsigned int vmin = 0xffffffffu, vmax = 0u;
   for (int c0 = lo + tid; c0 < hi; c0 += kCvUnroll * kCvThreads) {  // several loads in flight
@@ -142,7 +279,9 @@ __global__ void __launch_bounds__(kCvThreads) cv_kernel(const CvArgs a) {
     need = s_pair[1];
     nb = shift;
   }
-  const float phi = __uint_as_float(prefix) * a.alpha;
+  thr_bits = prefix;
+  }
+  const float phi = __uint_as_float(thr_bits) * a.alpha;
 
   // ---- column counts over this CTA's columns
   const int cper = (m + kCvCluster - 1) / kCvCluster;
@@ -295,8 +434,18 @@ extern "C" int catekv_head_cv(const void* q_win, const void* k, int64_t k_stride
   ca.alpha = alpha;
   ca.cv_out = cv_out;
   cudaLaunchConfig_t cfg = {};
+  {
+    static std::atomic<bool> attr_set[64];
+    int dev = 0;
+    CATEKV_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
+      CATEKV_CUDA_TRY(cudaFuncSetAttribute(cv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCvListCap * 4));
+      if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
+    }
+  }
   cfg.gridDim = dim3(n_segs * kCvCluster);
   cfg.blockDim = dim3(kCvThreads);
+  cfg.dynamicSmemBytes = kCvListCap * 4;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;

@@ -76,3 +76,19 @@ def test_head_mask_reproduces_oracle(ck):
     mask = ck.catekv_classify_heads(got, 0.5)
     assert np.array_equal(mask, orc.static_head_mask(want, 0.5))
     assert np.array_equal(mask, types.reshape(-1))
+
+
+@pytest.mark.parametrize("L_rec,kq,alpha", [(64, 0.99, 1.0), (4, 0.9, 1.0), (4, 0.5, 0.8)])
+def test_head_cv_when_the_entries_crowd_into_one_bin(ck, L_rec, kq, alpha):
+    """Zero queries: every window row attends uniformly, so all entries of the matrix are 1 / (visible keys of the
+    row) and share one bin of the percentile kernel's first histogram; a CTA's part of it exceeds its list and the
+    general radix path runs.  With L_rec < L_obs the causal mask gives the rows different key counts (a few dozen
+    distinct values and zeros), else all entries are equal and the score is 0."""
+    Hq, Hkv, L_obs, n, L_init = 8, 2, 64, 2400, 16
+    w = synth.scaled(synth.WORKLOADS["cfg4"], Hq=Hq, Hkv=Hkv, L_obs=L_obs, B=1)
+    q, k = synth.calibration_prompt(w, 0, 0, n, np.array([1, 0], dtype=np.uint8))
+    q = torch.zeros_like(q)
+    got, want = _cv_both(ck, q, k, [n], L_obs, L_init, L_rec, kq, alpha, True)
+    np.testing.assert_allclose(got, want, rtol=CV_RTOL, atol=1e-6)
+    if L_rec >= L_obs:
+        assert np.all(got == 0.0)
