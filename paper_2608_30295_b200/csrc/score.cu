@@ -366,32 +366,61 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
           }
           const int i_min = j - (job.n - a.L_obs);  // causal: window row i sees key j iff i >= i_min
           const bool edge = a.causal && __any_sync(0xffffffffu, i_min > half * 32);
-#pragma unroll 1
-          for (int gg = 0; gg < a.G; ++gg) {
-            const int col = gg * 64 + half * 32;
-            if (col < r_begin || col >= r_end) continue;  // another unit's columns
-            float x[32];
-            tmem_ld32(tbase + (col - r_begin), x);
-            tmem_wait_ld32(x);
+          // the heads whose 32 columns lie in this unit are consecutive; they are read 16 columns at a time, the
+          // next load in flight while the current one's exponentials run, and the slot goes back to the MMA warp
+          // after the last load.  Piece p: head p / 2, columns 16 * (p % 2) of this thread's 32.
+          auto add_piece = [&](const float (&x)[16], int p) {
+            const int col = (p >> 1) * 64 + half * 32 + (p & 1) * 16;
+            const int cb = (p & 1) * 16;
 #pragma unroll
-            for (int c = 0; c < 32; c += 4) {
+            for (int c = 0; c < 16; c += 4) {
               const float4 mm = *reinterpret_cast<const float4*>(s_f + col + c);
               float e0 = fast_exp2(fmaf(x[c], a.scale_log2, -mm.x));
               float e1 = fast_exp2(fmaf(x[c + 1], a.scale_log2, -mm.y));
               float e2 = fast_exp2(fmaf(x[c + 2], a.scale_log2, -mm.z));
               float e3 = fast_exp2(fmaf(x[c + 3], a.scale_log2, -mm.w));
               if (edge) {
-                const int i0 = half * 32 + c;
+                const int i0 = half * 32 + cb + c;
                 e0 = i0 >= i_min ? e0 : 0.f;
                 e1 = i0 + 1 >= i_min ? e1 : 0.f;
                 e2 = i0 + 2 >= i_min ? e2 : 0.f;
                 e3 = i0 + 3 >= i_min ? e3 : 0.f;
               }
-              macc[c] += e0;
-              macc[c + 1] += e1;
-              macc[c + 2] += e2;
-              macc[c + 3] += e3;
+              if (p & 1) {
+                macc[16 + c] += e0, macc[17 + c] += e1, macc[18 + c] += e2, macc[19 + c] += e3;
+              } else {
+                macc[c] += e0, macc[c + 1] += e1, macc[c + 2] += e2, macc[c + 3] += e3;
+              }
             }
+          };
+          auto in_unit = [&](int gg) {
+            const int col = gg * 64 + half * 32;
+            return gg < a.G && col >= r_begin && col < r_end;
+          };
+          auto taddr_of = [&](int p) { return tbase + (uint32_t)((p >> 1) * 64 + half * 32 + (p & 1) * 16 - r_begin); };
+          int g_first = 0;
+          while (g_first < a.G && !in_unit(g_first)) ++g_first;
+          int g_last = g_first;
+          while (in_unit(g_last)) ++g_last;  // one past the unit's last head
+          if (g_first < g_last) {
+            float xa[16], xb[16];
+            int p = 2 * g_first;
+            const int p_end = 2 * g_last;  // an even number of pieces
+            tmem_ld16(taddr_of(p), xa);
+            tmem_wait_ld16(xa);
+#pragma unroll 1
+            for (; p < p_end; p += 2) {
+              tmem_ld16(taddr_of(p + 1), xb);
+              add_piece(xa, p);
+              tmem_wait_ld16(xb);
+              const bool more = p + 2 < p_end;
+              if (more) tmem_ld16(taddr_of(p + 2), xa);
+              else release_slot(u);
+              add_piece(xb, p + 1);
+              if (more) tmem_wait_ld16(xa);
+            }
+          } else {
+            release_slot(u);
           }
           if (sub == UPT - 1 && j < j_hi) {
 #pragma unroll
@@ -425,7 +454,7 @@ __global__ void __launch_bounds__(kScThreads, 2) score_tc_kernel(const __grid_co
           }
         }
       }
-      if (MODE == kScoreMatrix) release_slot(u);  // the other modes handed it back right after their last load
+      if (MODE == kScoreMatrix && !a.g_major) release_slot(u);  // the others handed it back right after their last load
     }
   }
 
