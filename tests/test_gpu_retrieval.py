@@ -325,6 +325,9 @@ def _one_dim_case(ck, levels, budget, cs=8, sink=4, local=32):
     sel = torch.full((1,), -99, dtype=torch.int32, device="cuda")
     ck.catekv_retrieve_select(cache, meta, cs, q, [1], budget, sink, local, idx, sel)
     torch.cuda.synchronize()
+    if int(sel[0]) == -1:  # the whole list
+        assert np.array_equal(want, np.arange(n)) and torch.all(idx[0] == -7)
+        return
     assert int(sel[0]) == len(want)
     assert np.array_equal(idx[0, :len(want)].cpu().numpy().astype(np.int64), want)
     assert torch.all(idx[0, len(want):] == -7)
@@ -389,3 +392,32 @@ def test_retrieval_many_short_segments(ck):
         else:
             assert got_sel[s] == -1 and np.all(idx[s] == -7), s
     assert n_selecting > 500
+
+
+def test_retrieval_selection_random_exact_cases(ck):
+    """Seeded sweep over chunk sizes, lengths, budgets, sink / local sizes and score distributions (few levels, one
+    value, an outlier, two adjacent bf16 values, negative, normal, heavy-tailed with both signs), every case with
+    scores that are exact on both sides: the device's list must equal the oracle's."""
+    rng = np.random.default_rng(2024)
+    for it in range(60):
+        cs = int(rng.choice([1, 2, 4, 8, 16]))
+        n = int(rng.integers(50, 40000)) if cs >= 4 else int(rng.integers(50, 12000))
+        sink, local = int(rng.integers(0, 20)), int(rng.integers(0, 100))
+        budget = int(rng.integers(8, max(9, n)))
+        nch = (n + cs - 1) // cs
+        kind = it % 7
+        if kind == 0:
+            lv = rng.integers(1, 4, nch).astype(np.float64)
+        elif kind == 1:
+            lv = np.full(nch, 0.75)
+        elif kind == 2:
+            lv = np.roll(np.concatenate([[4096.0], rng.integers(0, 256, nch - 1) / 256.0]), int(rng.integers(0, nch)))
+        elif kind == 3:
+            lv = np.where(rng.random(nch) < 0.5, 2.0, 2.015625)
+        elif kind == 4:
+            lv = -rng.integers(1, 200, nch) / 16.0
+        elif kind == 5:
+            lv = orc.bf16_to_f64(orc.f64_to_bf16(rng.standard_normal(nch)))
+        else:
+            lv = orc.bf16_to_f64(orc.f64_to_bf16(np.exp(3 * rng.standard_normal(nch)) * rng.choice([-1, 1], nch)))
+        _one_dim_case(ck, np.repeat(lv, cs)[:n], budget, cs=cs, sink=sink, local=local)
