@@ -841,11 +841,16 @@ def main():
         ru, ra, rm = time_retrieval(ck, w, dev)
         line["retrieval"] = {"us_per_layer_step": ru, "attended_bytes_per_layer_step": ra,
                              "metadata_bytes_per_layer_step": rm, "budget_rows": 1024, "chunk": 8,
+                             # the step's bytes (chunk metadata + attended rows) at the measured copy bandwidth
+                             "hbm_bound_us": (ra + rm) / (peaks["hbm_gbs"] * 1e3),
+                             "frac_of_hbm_bound": (ra + rm) / (peaks["hbm_gbs"] * 1e3) / ru,
                              "note": "query-aware retrieval on the adaptive heads of the same workload: per layer "
                                      "catekv_append_retrieval, catekv_retrieve_select, catekv_decode_attn_indexed; CUDA graph replay of the step"}
         wa = time_window_attn(ck, synth.WORKLOADS["cfg2"], dev)
         wa["tflops"] = wa["flops_window_attn"] / (wa["window_attn_ms"] * 1e-3) / 1e12
         wa["hbm_gbs"] = wa["hbm_bytes_window_attn"] / (wa["window_attn_ms"] * 1e-3) / 1e9
+        wa["frac_of_bf16_peak"] = wa["tflops"] / peaks["bf16_tflops"]  # the whole call against the burst GEMM figure
+        wa["frac_of_hbm_peak"] = wa["hbm_gbs"] / peaks["hbm_gbs"]
         wa["note"] = ("configs[2] prefill shape, one layer: catekv_window_attn (prefill rows of the observation window "
                       "+ their normalisers) and catekv_select_compact with / without that normaliser")
         line["window_attn"] = wa
