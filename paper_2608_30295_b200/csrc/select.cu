@@ -408,7 +408,12 @@ __global__ void __launch_bounds__(kTopkThreads) topk_small_kernel(const TopkArgs
     for (int i = tid * 4; i < a.small_pool; i += 4 * kTopkThreads) cp_async16(sv_addr + i * 4, Pg + i, 16);
     cp_async_commit();
   }
-  const SelSeg s = a.segs[seg];
+  SelSeg s = a.segs[seg];
+  if (s.n_pool > a.small_pool) {  // cannot happen with decisions taken from lengths within the capacities
+    raise_status(a.chk, CATEKV_STATUS_INDEX_RANGE, kKidTopk, seg, s.n_pool);  // (a.chk is null outside the checked build)
+    s.n_pool = a.small_pool;
+    s.k_sel = min(s.k_sel, s.n_pool);
+  }
   if (s.keep_all) {
     cp_async_wait<0>();
     if (a.mark_keep_all && tid == 0) a.seg_len_dev[seg] = -1;
