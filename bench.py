@@ -386,6 +386,22 @@ def time_head_cv(ck, dev):
     return e0.elapsed_time(e1) / 3
 
 
+def select_block(w, ms, n_layers, kept_bytes, peaks):
+    """catekv_select_compact per layer against what bounds it: the bytes it has to move (K twice, for the two scoring
+    passes, and the kept K/V rows in and out of the gather) at the measured copy bandwidth, and its exponentials (two
+    per logit) at the special-function pipe's 16 per clock per SM and the maximum SM clock."""
+    import torch
+    k_bytes = w.B * w.Hkv * w.n * w.d * 2
+    hbm_us = (2 * k_bytes + 2 * kept_bytes) / (peaks["hbm_gbs"] * 1e3)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    exps = 2.0 * w.B * w.Hq * w.L_obs * w.n
+    sfu_us = exps / (sms * 16 * 1965.0)  # 1965 MHz: clocks.max.sm
+    gather_us = 2 * kept_bytes / (peaks["hbm_gbs"] * 1e3)
+    bound_us = max(hbm_us, sfu_us + gather_us)
+    return {"ms_per_layer": ms, "layers": n_layers, "hbm_bound_us": hbm_us, "sfu_plus_gather_bound_us": sfu_us + gather_us,
+            "frac_of_bound": bound_us / (ms * 1e3)}
+
+
 def time_window_attn(ck, w, dev, layer=0, reps=5):
     """catekv_window_attn on the workload's prefill shape (one layer), and catekv_select_compact with and without the
     normaliser it delivers.  Returns a dict of milliseconds and the bytes / flops the attention call has to move."""
@@ -719,7 +735,7 @@ def measure_workload(ck, w, dev, n_layers, steps, warmup, barrier, graph, peaks,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
         "gpu_launches": steps * n_layers * ((1 if FUSED else 2) + (1 if has_combine else 0)),
         "clocks": clocks,
-        "select_compact": {"ms_per_layer": float(np.mean(sel_ms[1:] or sel_ms)), "layers": n_layers},
+        "select_compact": select_block(w, float(np.mean(sel_ms[1:] or sel_ms)), n_layers, bytes_per_layer, peaks),
         "plan_host_us": plan_us,
     }
 
@@ -835,7 +851,8 @@ def main():
                            "step_hbm_gbs": ro["step_hbm_gbs"],
                            "step_frac_of_measured": ro["step_hbm_gbs"] / peaks["hbm_gbs"],
                            "step_frac_of_8TBs": ro["step_hbm_gbs"] / 8000.0,
-                           "select_ms_per_layer": ro["select_compact"]["ms_per_layer"]}
+                           "select_ms_per_layer": ro["select_compact"]["ms_per_layer"],
+                           "select_compact": ro["select_compact"]}
         line["other_configs"] = table
         line["head_cv"] = {"ms": time_head_cv(ck, dev), "shape": "8 prompts x 16384 tokens, 28q/4kv, window 64"}
         ru, ra, rm = time_retrieval(ck, w, dev)
