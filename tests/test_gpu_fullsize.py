@@ -294,3 +294,22 @@ def test_cfg2_window_attention_and_selection_from_its_normaliser(ck):
                              w.pool_mode, w.pool_param, idx_out=idx, row_lse_scored=lse_sc)
     torch.cuda.synchronize()
     _check_selection_cells(w, p, mask, cache, idx, cells)
+
+
+def test_cfg4_window_attention_sampled_heads(ck):
+    # configs[4] shape: 256K keys, 7 x 64 = 448 window rows per KV head (four 128-row tiles, the last one half
+    # full, nine key ranges per tile).  The oracle checks the rows of three sampled query heads one by one.
+    w = synth.WORKLOADS["cfg4"]
+    p = synth.prefill_layer(w, 0, "cuda")
+    out, lse, lse_sc = ck.catekv_window_attn(p["q_win"], p["k"], p["v"], p["seq_len"])
+    out16, _, _ = ck.catekv_window_attn(p["q_win"], p["k"], p["v"], p["seq_len"], out_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    qb = synth.bits(p["q_win"])
+    for (b, hq) in [(0, 0), (1, 13), (3, 27)]:  # first, a middle and the last head (the last rows of a last tile)
+        h = hq // w.G
+        kb, vb = synth.bits(p["k"][b, h]), synth.bits(p["v"][b, h])
+        ref, ref_lse = orc.window_attention(qb[b, hq:hq + 1], kb, vb, w.L_obs)
+        H.check_attention(out[b, hq], out16[b, hq], lse[b, hq], ref.reshape(-1, w.d), ref_lse.reshape(-1),
+                          f"cfg4 window b{b} head {hq}")
+        ref_sc = orc.scored_range_lse(qb[b, hq:hq + 1], kb, w.L_obs)
+        assert np.all(np.abs(lse_sc[b, hq].cpu().double().numpy() - ref_sc.reshape(-1)) <= 1e-3)
