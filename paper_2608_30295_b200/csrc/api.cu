@@ -75,7 +75,7 @@ extern "C" int catekv_checked_status(catekv_status* out, int32_t clear) {
   return catekv::read_status(p, out, clear, (cudaStream_t)0);
 }
 
-extern "C" int catekv_version(void) { return 2000; }
+extern "C" int catekv_version(void) { return 2001; }
 
 extern "C" int catekv_last_cuda_error(void) { return catekv::g_last_cuda_error; }
 

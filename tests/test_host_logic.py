@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol(ck):
     for name in declared:
         assert hasattr(lib, name), name
     assert declared == set(ck.EXPORTS)
-    assert ck.catekv_version() == 2000
+    assert ck.catekv_version() == 2001
     assert ck._lib.catekv_error_string(-3) == b"segment capacity exceeded"
 
 
