@@ -369,10 +369,11 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkArgs a) {
 //   4. ordered compaction: the warps' votes give one bitmap of the entries above the threshold and one of those at
 //      it; thread t takes word t of both (32 consecutive entries), one scan over the counts, the writes.
 // Per entry two flags live in registers: above the threshold for sure (gtm), still a candidate (cand).
-constexpr int kTsPer = 16;     // entries a thread may own
+constexpr int kTsPer = 32;     // entries a thread may own (one flag bit each in two 32-bit registers)
 constexpr int kTsBins = 1024;  // == kTopkThreads: one bin per thread in the scan
 constexpr int kTsRank = 256;   // candidates resolved by ranking
 constexpr int kTopkSmallMax = kTsPer * kTopkThreads;
+static_assert(kTopkSmallMax / 32 == kTopkThreads, "one bitmap word per thread");
 
 __global__ void __launch_bounds__(kTopkThreads) topk_small_kernel(const TopkArgs a) {
   __shared__ unsigned int hist[kTsBins];
@@ -390,7 +391,8 @@ __global__ void __launch_bounds__(kTopkThreads) topk_small_kernel(const TopkArgs
   const int seg = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_launch_dependents();
   hist[tid] = 0;
-  (tid < 512 ? s_gt : s_eq)[tid & 511] = 0u;
+  s_gt[tid] = 0u;  // kTopkSmallMax / 32 == kTopkThreads words each
+  s_eq[tid] = 0u;
   if (tid == 0) {
     s_mm[0] = 0xffffffffu;
     s_mm[1] = 0u;
@@ -568,7 +570,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_small_kernel(const TopkArgs
     for (unsigned int mk = gtm; mk; mk &= mk - 1u) atomicOr(&s_gt[(__ffs(mk) - 1) * 32 + warp], 1u << lane);
     for (unsigned int mk = cand; mk; mk &= mk - 1u) atomicOr(&s_eq[(__ffs(mk) - 1) * 32 + warp], 1u << lane);
     __syncthreads();
-    const int n_words = (s.n_pool + 31) / 32;  // <= 512: thread t < n_words takes word t
+    const int n_words = (s.n_pool + 31) / 32;  // <= 1024: thread t < n_words takes word t
     const unsigned int g = tid < n_words ? s_gt[tid] : 0u, q = tid < n_words ? s_eq[tid] : 0u;
     const unsigned int mine = (unsigned int)__popc(g) | ((unsigned int)__popc(q) << 16);
     unsigned int inc = mine;

@@ -334,7 +334,7 @@ def _one_dim_case(ck, levels, budget, cs=8, sink=4, local=32):
 
 
 @pytest.mark.parametrize("case", ["three_levels", "all_equal", "outlier", "two_neighbours", "negative", "random"])
-@pytest.mark.parametrize("n,budget", [(8192 + 40, 1024), (3000, 520), (20000, 2048)])
+@pytest.mark.parametrize("n,budget", [(8192 + 40, 1024), (3000, 520), (20000, 2048), (230000, 4096)])
 def test_retrieval_selection_with_ties_and_crowded_scores(ck, case, n, budget):
     """The short-list selection kernel on score distributions that stress each of its steps: hundreds of exact
     ties at the threshold, one score for all, an outlier that squeezes every other score into one histogram bin,
